@@ -1,0 +1,147 @@
+/*
+ * osscar.h -- C ABI of the B200 implementation of the OSSCAR per-layer solve
+ * (one-shot structured pruning as a combinatorial problem, arXiv 2403.12983).
+ *
+ * Problem (Section 2, Eq. MIQP; Section 3.1, Eq. deff/struc).  A layer has a dense weight
+ * W_hat (d1 x m) and calibration inputs X (n x d1).  The rows of W_hat are split into
+ * d1/g contiguous groups of g rows (one per input neuron, per conv input channel or per
+ * attention head); group q holds rows q*g .. q*g+g-1 (0-based).  Exactly k groups may stay
+ * non-zero.  With H = X^T X and G = H W_hat, the reconstruction error of a kept set S is
+ *     obj(S) = min_W ||X W_hat - X W||_F^2 = const - Tr(G_I^T (H_II)^-1 G_I),
+ * I = rows of the kept groups, const = Tr(W_hat^T H W_hat)  (Eq. optf; obj = 2 f + const,
+ * with the paper's S being the complementary, pruned set).  The library builds H and G,
+ * picks a starting support and runs the swap form of Algorithm 1 (t_hat = 2, p_hat = 0) on
+ * the device, moving (H_II)^-1, the optimal weights and the residual with the low-rank
+ * identities of Proposition 1 instead of re-solving.
+ *
+ * Conventions.  All matrices are dense, row-major, leading dimension = number of columns.
+ * "device" / "host" says where a pointer must live.  The caller owns every buffer; the
+ * library allocates only a small control block per context.  Every call returns a status
+ * (OSSCAR_OK or a negative error); nothing throws, aborts or traps.  Work is enqueued on the
+ * context's stream; a call synchronises that stream once, at its end, iff it has host
+ * outputs.  A failed call leaves its outputs unspecified and the context usable.
+ * There is no CPU path: without a CUDA device every call fails with OSSCAR_E_CUDA.
+ */
+#ifndef OSSCAR_H_
+#define OSSCAR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct osscar_ctx osscar_ctx;
+
+enum {
+    OSSCAR_OK = 0,
+    OSSCAR_E_ARG = -1,        /* null pointer, bad enum, bad flag                           */
+    OSSCAR_E_SHAPE = -2,      /* sizes inconsistent (d1 % g, k out of range, g too large)   */
+    OSSCAR_E_NOTPD = -3,      /* H restricted to the kept rows is not positive definite     */
+    OSSCAR_E_WORKSPACE = -4,  /* workspace missing or too small                             */
+    OSSCAR_E_CUDA = -5,       /* a CUDA runtime/driver call failed                          */
+    OSSCAR_E_TIMEOUT = -6,    /* a bounded device-side wait ran out                         */
+    OSSCAR_E_STATE = -7       /* call order violated (e.g. search before init)              */
+};
+enum { OSSCAR_BF16 = 0, OSSCAR_FP32 = 1 };
+enum { OSSCAR_GRAM_BEGIN = 1, OSSCAR_GRAM_END = 2 };
+enum { OSSCAR_INIT_ENERGY = 0, OSSCAR_INIT_MAGNITUDE = 1, OSSCAR_INIT_USER = 2 };
+enum { OSSCAR_SCORE_INDEPENDENT = 0, OSSCAR_SCORE_PAIR_EXACT = 1 };
+enum { OSSCAR_ACCEPT_IMPROVING = 0, OSSCAR_ACCEPT_ALWAYS = 1 };
+enum { OSSCAR_STOP_MAX_SWAPS = 0, OSSCAR_STOP_NO_IMPROVEMENT = 1, OSSCAR_STOP_GUARD = 2 };
+
+#define OSSCAR_MAX_GROUP 96   /* largest supported group size g */
+
+/* Context bound to one device and one stream (a cudaStream_t passed as void*, NULL = the
+ * legacy default stream).  create allocates a few KB of device and pinned host memory. */
+int osscar_create(osscar_ctx** out, int device, void* cuda_stream);
+int osscar_destroy(osscar_ctx* ctx);
+
+/* Scratch needed by init_support / local_search / objective for a layer of this shape.
+ * The caller allocates it on the device (256-byte aligned) and lends it with set_workspace;
+ * it must stay alive, and untouched by others, from init_support to the end of local_search. */
+int osscar_workspace_bytes(int64_t d1, int64_t m, int32_t g, int32_t k, size_t* bytes /*host*/);
+int osscar_set_workspace(osscar_ctx* ctx, void* dev_ptr, size_t bytes);
+
+/*
+ * Gram and cross term of a dense layer (Section 2, dense-layer paragraph: H = X^T X,
+ * G = X^T X W_hat; conv layers pass the unfolded patch matrix, attention/FC2 layers the
+ * token activations).  X is given in row blocks ("chunks" of tokens):
+ *   flags & BEGIN : H := Xc^T Xc, otherwise H += Xc^T Xc   (split over calibration rows);
+ *   flags & END   : H += damp * mean(diag H) * I (damp = 0: none; not in the paper),
+ *                   G := H W_hat, *const_term := Tr(W_hat^T G), then one stream sync.
+ * X: device, n_rows x d1, bf16 (tensor cores, fp32 accumulation) or fp32.  For bf16 the
+ * pointer must be 16-byte aligned and d1 a multiple of 8.  W: device d1 x m fp32 (read on END).
+ * H: device d1 x d1 fp32, G: device d1 x m fp32, const_term: host (written on END).
+ * n_rows may be 0 (nothing is added).
+ */
+int osscar_gram(osscar_ctx* ctx, const void* X, int x_dtype, int64_t n_rows, int64_t d1,
+                const float* W, int64_t m, int flags, float damp,
+                float* H, float* G, double* const_term);
+
+/*
+ * Starting support and search state (Algorithm 1, line 1, for a k-group support instead of
+ * the dense start).  mode ENERGY keeps the k groups with the largest Tr(W_q^T H_qq W_q),
+ * MAGNITUDE the k largest ||W_q||_F^2 (the paper's MP rule, Appendix B.1), ties to the
+ * smaller id; USER reads k distinct ids from `support`.  Builds (H_II)^-1, V = (H_II)^-1 G_I
+ * (Eq. tmp5), the residual R = G - H[:,I] V and the Schur complements of every pruned group
+ * (the C^-1 of Case 2 in the proof of Proposition 1) in the workspace.
+ * H, G, W: device, as produced by osscar_gram (H symmetric).  support: device int32[k],
+ * sorted ids on return.  obj0: host, obj of the starting support.  Synchronises once.
+ * Errors: E_NOTPD if a pivot block of H_II fails its Cholesky factorisation.
+ */
+int osscar_init_support(osscar_ctx* ctx, const float* H, const float* G, const float* W,
+                        int64_t d1, int64_t m, int32_t g, int32_t k, int mode,
+                        int32_t* support, double* obj0);
+
+typedef struct {
+    int32_t max_swaps;        /* >= 0                                                        */
+    int32_t score_mode;       /* OSSCAR_SCORE_*                                              */
+    int32_t accept_mode;      /* OSSCAR_ACCEPT_*                                             */
+    int32_t refresh_every;    /* rebuild the state from H every this many swaps; 0 = never   */
+    double  accept_rel_tol;   /* IMPROVING: accept iff delta <= -tol * obj (1e-5 if < 0)     */
+    uint64_t wait_limit_cycles; /* bound of device-side waits; 0 = default                   */
+} osscar_search_params;
+
+typedef struct {
+    int32_t n_swaps, stop_reason, n_refresh, status;
+    double  obj_init, obj_final;     /* obj_final is recomputed from the final state         */
+    float   ms_search;               /* device time of the swap loop                         */
+} osscar_search_result;
+
+/*
+ * Swap search (Section 3.2: Eq. local with t_hat = 2, p_hat = 0; scores of Eq. impact;
+ * state moved by Cases 1-3 of Proposition 1).  Each step scores every kept group (rise of
+ * obj if dropped) and every pruned group (fall of obj if added), takes the cheapest drop and
+ * the most valuable add (PAIR_EXACT: the best exact pair), computes the exact change of obj
+ * for that pair, applies the accept rule and updates the state; the loop runs on the device
+ * with no host round trip per swap.
+ * support_out: device int32[k] (sorted).  W_out: device d1 x m fp32, rows of pruned groups
+ * zero.  obj_trace: device double[max_swaps+1], entry 0 = starting obj.  swap_trace: device
+ * int32[2*max_swaps], (group out, group in) per accepted swap.  result: host.
+ * Synchronises once at the end.
+ */
+int osscar_local_search(osscar_ctx* ctx, const osscar_search_params* params,
+                        int32_t* support_out, float* W_out,
+                        double* obj_trace, int32_t* swap_trace,
+                        osscar_search_result* result);
+
+/* Tr((W - Wt)^T H (W - Wt)) for any candidate Wt (Eq. obj-ver2 re-centred at W_hat); does not
+ * touch the search state but uses the workspace (2*d1*m floats at its start are overwritten,
+ * so call it before init_support or after local_search).  H, W, Wt: device; obj: host. */
+int osscar_objective(osscar_ctx* ctx, const float* H, const float* W, const float* Wt,
+                     int64_t d1, int64_t m, double* obj);
+
+/* Test hook (not part of the contract): copy one piece of the search state to `dst` (device).
+ * which: 0 Hinv (n_I x n_I), 1 V (n_I x m), 2 R of pruned slots (n_J x m), 3 c (double,
+ * (d1/g-k) x g x g), 4 slot->group permutation (int32[d1/g]), 5 drop scores (double[k]),
+ * 6 add scores (double[d1/g-k]).  Scores are those of the last scoring pass. */
+int osscar_debug_get_state(osscar_ctx* ctx, int which, void* dst);
+
+const char* osscar_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* OSSCAR_H_ */

@@ -1,0 +1,254 @@
+"""ctypes binding of include/osscar.h.  Argument marshalling only."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import Iterable, Optional
+
+import torch
+
+from . import build as _build
+
+OK = 0
+E_ARG, E_SHAPE, E_NOTPD, E_WORKSPACE, E_CUDA, E_TIMEOUT, E_STATE = -1, -2, -3, -4, -5, -6, -7
+BF16, FP32 = 0, 1
+GRAM_BEGIN, GRAM_END = 1, 2
+INIT_ENERGY, INIT_MAGNITUDE, INIT_USER = 0, 1, 2
+SCORE_INDEPENDENT, SCORE_PAIR_EXACT = 0, 1
+ACCEPT_IMPROVING, ACCEPT_ALWAYS = 0, 1
+STOP_MAX_SWAPS, STOP_NO_IMPROVEMENT, STOP_GUARD = 0, 1, 2
+STOP_NAMES = {0: "max_swaps", 1: "no_improvement", 2: "guard"}
+
+EXPORTS = ["osscar_create", "osscar_destroy", "osscar_workspace_bytes", "osscar_set_workspace",
+           "osscar_gram", "osscar_init_support", "osscar_local_search", "osscar_objective",
+           "osscar_debug_get_state", "osscar_status_string"]
+
+
+class SearchParams(C.Structure):
+    _fields_ = [("max_swaps", C.c_int32), ("score_mode", C.c_int32), ("accept_mode", C.c_int32),
+                ("refresh_every", C.c_int32), ("accept_rel_tol", C.c_double), ("wait_limit_cycles", C.c_uint64)]
+
+
+class SearchResult(C.Structure):
+    _fields_ = [("n_swaps", C.c_int32), ("stop_reason", C.c_int32), ("n_refresh", C.c_int32), ("status", C.c_int32),
+                ("obj_init", C.c_double), ("obj_final", C.c_double), ("ms_search", C.c_float)]
+
+
+class OsscarError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = lib().osscar_status_string(status).decode() if _LIB is not None else "?"
+        super().__init__(f"{where}: {msg} ({status})")
+
+
+_LIB = None
+
+
+def lib_path() -> str:
+    return _build.LIB_PATH
+
+
+def lib() -> C.CDLL:
+    """Loads libosscar.so (building it with nvcc first if the sources are newer).  Raises if absent."""
+    global _LIB
+    if _LIB is not None:
+        return _LIB
+    path = _build.LIB_PATH
+    if not os.path.exists(path) or (os.environ.get("OSSCAR_NO_REBUILD") is None and _build.needs_build()):
+        _build.build()
+    L = C.CDLL(path)
+    vp, i32, i64 = C.c_void_p, C.c_int32, C.c_int64
+    L.osscar_status_string.restype = C.c_char_p
+    L.osscar_status_string.argtypes = [C.c_int]
+    L.osscar_create.argtypes = [C.POINTER(vp), C.c_int, vp]
+    L.osscar_destroy.argtypes = [vp]
+    L.osscar_workspace_bytes.argtypes = [i64, i64, i32, i32, C.POINTER(C.c_size_t)]
+    L.osscar_set_workspace.argtypes = [vp, vp, C.c_size_t]
+    L.osscar_gram.argtypes = [vp, vp, C.c_int, i64, i64, vp, i64, C.c_int, C.c_float, vp, vp, C.POINTER(C.c_double)]
+    L.osscar_init_support.argtypes = [vp, vp, vp, vp, i64, i64, i32, i32, C.c_int, vp, C.POINTER(C.c_double)]
+    L.osscar_local_search.argtypes = [vp, C.POINTER(SearchParams), vp, vp, vp, vp, C.POINTER(SearchResult)]
+    L.osscar_objective.argtypes = [vp, vp, vp, vp, i64, i64, C.POINTER(C.c_double)]
+    L.osscar_debug_get_state.argtypes = [vp, C.c_int, vp]
+    for name in EXPORTS:
+        if name != "osscar_status_string":
+            getattr(L, name).restype = C.c_int
+    _LIB = L
+    return L
+
+
+def _check(status: int, where: str):
+    if status != OK:
+        raise OsscarError(status, where)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _dev_f32(t: torch.Tensor, name: str) -> torch.Tensor:
+    if not (t.is_cuda and t.dtype == torch.float32 and t.is_contiguous()):
+        raise ValueError(f"{name} must be a contiguous fp32 CUDA tensor")
+    return t
+
+
+def osscar_workspace_bytes(d1: int, m: int, g: int, k: int) -> int:
+    out = C.c_size_t(0)
+    _check(lib().osscar_workspace_bytes(d1, m, g, k, C.byref(out)), "osscar_workspace_bytes")
+    return out.value
+
+
+@dataclass
+class SearchOutput:
+    support: torch.Tensor        # int32[k], sorted kept group ids (device)
+    W: torch.Tensor              # d1 x m fp32, pruned rows zero (device)
+    obj_trace: torch.Tensor      # float64[n_swaps + 1] (device)
+    swap_trace: torch.Tensor     # int32[n_swaps, 2] (group out, group in) (device)
+    n_swaps: int
+    stop_reason: str
+    n_refresh: int
+    obj_init: float
+    obj_final: float
+    ms_search: float
+
+
+class Solver:
+    """One context (device + stream) and its caller-owned workspace."""
+
+    def __init__(self, device: Optional[int] = None, stream: Optional[torch.cuda.Stream] = None):
+        if not torch.cuda.is_available():
+            raise OsscarError(E_CUDA, "Solver: no CUDA device; this library has no CPU path")
+        self.device = torch.cuda.current_device() if device is None else int(device)
+        self.stream = stream
+        handle = C.c_void_p()
+        sptr = C.c_void_p(stream.cuda_stream) if stream is not None else C.c_void_p(torch.cuda.current_stream(self.device).cuda_stream)
+        _check(lib().osscar_create(C.byref(handle), self.device, sptr), "osscar_create")
+        self._h = handle
+        self._ws = None
+        self._shape = None
+        self._keep = []
+
+    def close(self):
+        if getattr(self, "_h", None):
+            lib().osscar_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -------------------------------------------------------------- workspace
+    def ensure_workspace(self, d1: int, m: int, g: int, k: int):
+        need = osscar_workspace_bytes(d1, m, g, k)
+        if self._ws is None or self._ws.numel() < need:
+            self._ws = None
+            self._ws = torch.empty(need, dtype=torch.uint8, device=f"cuda:{self.device}")
+        _check(lib().osscar_set_workspace(self._h, _ptr(self._ws), self._ws.numel()), "osscar_set_workspace")
+        return need
+
+    # -------------------------------------------------------------- calls of include/osscar.h
+    def gram_chunk(self, X: torch.Tensor, H: torch.Tensor, flags: int, W=None, G=None, damp: float = 0.0) -> Optional[float]:
+        if X.dtype == torch.bfloat16:
+            xd = BF16
+        elif X.dtype == torch.float32:
+            xd = FP32
+        else:
+            raise ValueError("X must be bf16 or fp32")
+        if not (X.is_cuda and X.is_contiguous() and X.dim() == 2):
+            raise ValueError("X must be a contiguous 2-D CUDA tensor")
+        n, d1 = X.shape
+        _dev_f32(H, "H")
+        const = C.c_double(0.0)
+        m = 0
+        if flags & GRAM_END:
+            _dev_f32(W, "W"); _dev_f32(G, "G")
+            m = W.shape[1]
+        _check(lib().osscar_gram(self._h, _ptr(X), xd, n, d1, _ptr(W), m, flags, damp, _ptr(H), _ptr(G), C.byref(const)), "osscar_gram")
+        return const.value if flags & GRAM_END else None
+
+    def gram(self, chunks: Iterable[torch.Tensor], W: torch.Tensor, damp: float = 0.0):
+        """H, G, const from an iterable of row blocks of X (each a CUDA tensor)."""
+        _dev_f32(W, "W")
+        d1, m = W.shape
+        H = torch.empty(d1, d1, dtype=torch.float32, device=W.device)
+        G = torch.empty(d1, m, dtype=torch.float32, device=W.device)
+        chunks = list(chunks) if not isinstance(chunks, (list, tuple)) else chunks
+        const = None
+        for i, Xc in enumerate(chunks):
+            flags = (GRAM_BEGIN if i == 0 else 0) | (GRAM_END if i == len(chunks) - 1 else 0)
+            const = self.gram_chunk(Xc, H, flags, W, G, damp)
+        return H, G, const
+
+    def init_support(self, H, G, W, g: int, k: int, mode: int = INIT_ENERGY, support: Optional[torch.Tensor] = None):
+        _dev_f32(H, "H"); _dev_f32(G, "G"); _dev_f32(W, "W")
+        d1, m = W.shape
+        self.ensure_workspace(d1, m, g, k)
+        if support is None:
+            support = torch.empty(k, dtype=torch.int32, device=W.device)
+        else:
+            support = support.to(device=W.device, dtype=torch.int32).contiguous().clone()
+        obj0 = C.c_double(0.0)
+        self._keep = [H, G, W]
+        self._shape = (d1, m, g, k)
+        _check(lib().osscar_init_support(self._h, _ptr(H), _ptr(G), _ptr(W), d1, m, g, k, mode, _ptr(support), C.byref(obj0)),
+               "osscar_init_support")
+        return support, obj0.value
+
+    def local_search(self, max_swaps: int, score_mode: int = SCORE_INDEPENDENT, accept_mode: int = ACCEPT_IMPROVING,
+                     refresh_every: int = 0, accept_rel_tol: float = -1.0) -> SearchOutput:
+        d1, m, g, k = self._shape
+        dev = self._keep[0].device
+        support = torch.empty(k, dtype=torch.int32, device=dev)
+        W_out = torch.empty(d1, m, dtype=torch.float32, device=dev)
+        obj_trace = torch.zeros(max_swaps + 1, dtype=torch.float64, device=dev)
+        swap_trace = torch.zeros(max(1, 2 * max_swaps), dtype=torch.int32, device=dev)
+        prm = SearchParams(max_swaps, score_mode, accept_mode, refresh_every, accept_rel_tol, 0)
+        res = SearchResult()
+        _check(lib().osscar_local_search(self._h, C.byref(prm), _ptr(support), _ptr(W_out), _ptr(obj_trace), _ptr(swap_trace),
+                                         C.byref(res)), "osscar_local_search")
+        n = res.n_swaps
+        return SearchOutput(support, W_out, obj_trace[:n + 1], swap_trace[:2 * n].view(n, 2), n,
+                            STOP_NAMES.get(res.stop_reason, str(res.stop_reason)), res.n_refresh,
+                            res.obj_init, res.obj_final, res.ms_search)
+
+    def objective(self, H, W, Wt) -> float:
+        _dev_f32(H, "H"); _dev_f32(W, "W"); _dev_f32(Wt, "Wt")
+        d1, m = W.shape
+        need = 2 * d1 * m * 4
+        if self._ws is None or self._ws.numel() < need:
+            self._ws = torch.empty(need, dtype=torch.uint8, device=W.device)
+            _check(lib().osscar_set_workspace(self._h, _ptr(self._ws), self._ws.numel()), "osscar_set_workspace")
+        out = C.c_double(0.0)
+        _check(lib().osscar_objective(self._h, _ptr(H), _ptr(W), _ptr(Wt), d1, m, C.byref(out)), "osscar_objective")
+        return out.value
+
+    def debug_state(self, which: int) -> torch.Tensor:
+        d1, m, g, k = self._shape
+        nI, ng = k * g, d1 // g
+        dev = self._keep[0].device
+        shapes = {0: ((nI, nI), torch.float32), 1: ((nI, m), torch.float32), 2: ((d1 - nI, m), torch.float32),
+                  3: ((ng - k, g, g), torch.float64), 4: ((ng,), torch.int32), 5: ((k,), torch.float64),
+                  6: ((ng - k,), torch.float64)}
+        shape, dt = shapes[which]
+        out = torch.empty(shape, dtype=dt, device=dev)
+        _check(lib().osscar_debug_get_state(self._h, which, _ptr(out)), "osscar_debug_get_state")
+        return out
+
+
+# ---------------------------------------------------------------------- functional forms (same names as the C ABI)
+def osscar_gram(solver: Solver, chunks, W, damp: float = 0.0):
+    return solver.gram(chunks, W, damp)
+
+
+def osscar_init_support(solver: Solver, H, G, W, g, k, mode=INIT_ENERGY, support=None):
+    return solver.init_support(H, G, W, g, k, mode, support)
+
+
+def osscar_local_search(solver: Solver, max_swaps, **kw) -> SearchOutput:
+    return solver.local_search(max_swaps, **kw)
+
+
+def osscar_objective(solver: Solver, H, W, Wt) -> float:
+    return solver.objective(H, W, Wt)

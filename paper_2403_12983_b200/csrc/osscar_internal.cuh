@@ -1,0 +1,96 @@
+// Internal declarations shared by the translation units of libosscar.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stddef.h>
+#include "osscar.h"
+
+namespace osscar {
+
+constexpr int kPadF = 32;   // leading dimensions of internal fp32 matrices are padded to this many floats
+
+static inline int64_t round_up(int64_t x, int64_t a) { return (x + a - 1) / a * a; }
+
+// Device-side control block of the swap loop.  Lives in the context's small device allocation.
+struct SearchCtl {
+    int32_t done;            // set once the loop has stopped; later kernels return at once
+    int32_t stop_reason;
+    int32_t status;          // OSSCAR_OK or an error raised on the device
+    int32_t n_swaps;
+    int32_t n_refresh;
+    int32_t sel_slot;        // kept slot leaving
+    int32_t sel_t;           // pruned slot (0-based among pruned slots) entering
+    int32_t pad0;
+    double  obj;             // running objective
+    double  sel_D;           // drop score of the chosen slot
+    double  delta;           // exact change of obj of the chosen swap
+    double  const_term;
+    double  acc[4];          // scratch accumulators (traces, objective reductions)
+};
+
+// Geometry of one layer's search state inside the caller's workspace.
+struct Layout {
+    int64_t d1, m, ng;       // rows of W, columns of W, number of groups
+    int32_t g, k;
+    int64_t nI, nJ;          // kept rows, pruned rows
+    int64_t ldp;             // leading dimension of Hp (slot-permuted H)
+    int64_t ldh;             // leading dimension of Hinv, and padded length of the n_I-vectors
+    int64_t ldm;             // leading dimension of V, R, K, Vq
+    // offsets in bytes from the workspace base
+    size_t off_Hp, off_Hinv, off_V, off_R, off_big;
+    size_t off_y, off_b, off_u2, off_bC, off_u2c, off_u, off_d, off_K, off_Vq;
+    size_t off_vec_begin, off_vec_end;   // the staged vectors (zeroed once when the state is built)
+    size_t off_vnorm, off_rnorm, off_D, off_A, off_c, off_small, off_gramV, off_gramR;
+    size_t off_perm, off_slotof, off_energy, off_panel;
+    size_t bytes;
+};
+int make_layout(int64_t d1, int64_t m, int32_t g, int32_t k, Layout* L);
+
+}  // namespace osscar
+
+struct osscar_ctx {
+    int device;
+    cudaStream_t stream;
+    osscar::SearchCtl* ctl;          // device
+    osscar::SearchCtl* ctl_host;     // pinned mirror
+    volatile int32_t* done_flag_host; // pinned, device-mapped: copy of ctl->done pushed by the device
+    int32_t* done_flag_dev;          // device alias of done_flag_host
+    void* ws;
+    size_t ws_bytes;
+    osscar::Layout L;
+    bool have_state;
+    const float* H;                  // caller's matrices bound by init_support
+    const float* G;
+    const float* W;
+    cudaEvent_t ev0, ev1;
+    double gram_rows;                // rows accumulated since GRAM_BEGIN (bookkeeping only)
+};
+
+namespace osscar {
+
+// ---- sgemm.cu: C = alpha * op(A) * B + beta * C on the fp32 pipes ----------------------------
+// A is M x K (lda) or, with transA, stored K x M; B is K x N (ldb) or, with transB, stored N x K.
+// `done` (may be null): device flag; when non-zero the kernel returns without touching C.
+cudaError_t sgemm(cudaStream_t st, bool transA, bool transB, int64_t M, int64_t N, int64_t K,
+                  float alpha, const float* A, int64_t lda, const float* B, int64_t ldb,
+                  float beta, float* C, int64_t ldc, const int32_t* done = nullptr);
+
+// ---- gram_tc.cu: H (+)= Xc^T Xc on the tensor cores (bf16 in, fp32 out) ----------------------
+cudaError_t gram_bf16_tcgen05(cudaStream_t st, const void* X, int64_t n_rows, int64_t d1,
+                              float* H, bool accumulate, int32_t* status_dev);
+cudaError_t gram_mirror(cudaStream_t st, float* H, int64_t d1);   // copy upper triangle to lower
+
+// ---- state.cu: support selection and state construction --------------------------------------
+int select_support(osscar_ctx* ctx, int mode, int32_t* support);
+int build_state(osscar_ctx* ctx, bool guarded);
+cudaError_t gather_rows(cudaStream_t st, const float* src, int64_t m, int g, const int32_t* perm,
+                        int64_t slot_row0, int64_t nrows, float* dst, int64_t ld);
+cudaError_t trace_product(cudaStream_t st, const float* A, int64_t lda, const float* B, int64_t ldb,
+                          int64_t rows, int64_t cols, double* out_dev);   // *out = sum A.*B
+
+// ---- search.cu -------------------------------------------------------------------------------
+int run_search(osscar_ctx* ctx, const osscar_search_params* p, int32_t* support_out, float* W_out,
+               double* obj_trace, int32_t* swap_trace, osscar_search_result* res);
+cudaError_t score_pass(osscar_ctx* ctx);   // full scoring pass from the current state (fills D, A)
+
+}  // namespace osscar

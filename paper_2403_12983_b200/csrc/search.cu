@@ -1,0 +1,806 @@
+// Device-resident swap search: scoring (Eq. impact), selection, exact swap change and the
+// rank-2g update of (H_II)^-1, V, R and the Schur complements (Proposition 1, Cases 1-3),
+// on a slot-permuted layout in which kept rows occupy slots [0, n_I) and pruned rows the rest.
+//
+// Notation inside one step.  r = rows of the leaving slot, q = rows of the entering pruned slot,
+//   C = Hinv[r,r], b = Hinv[:,r], h = Hp[q, 0:n_I]^T, y = Hinv h, P = y[r,:]^T (= H_qI Hinv_Ir),
+//   K = C^-1 V_r, R1 = R_q + P K, c1 = c_q + P C^-1 P^T, Vq = c1^-1 R1 (new rows of V),
+//   u2 = y - b C^-1 y_r on kept rows (0 on r), u = Hp[:,I] b, d = Hp[:,q] - Hp[:,I] u2.
+//   Hinv' = Hinv - b C^-1 b^T + u2 c1^-1 u2^T (rows/cols r: -u2 c1^-1, block rr: c1^-1)
+//   V'    = V - b K - u2 Vq (rows r: Vq)        R' = R + u K - d Vq        obj' = obj + delta
+//   c_l'  = c_l + u_l C^-1 u_l^T - d_l c1^-1 d_l^T,   delta = Tr(C^-1 V_r V_r^T) - Tr(c1^-1 R1 R1^T).
+#include "osscar_internal.cuh"
+#include <math.h>
+#include <float.h>
+#include <limits.h>
+
+namespace osscar {
+namespace {
+
+constexpr double kAddPivotTol = 1e-6;   // pruned group ineligible if min pivot of c <= tol * max diag(H_qq)
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ float block_sum_f(float v, float* red) {      // result in every thread
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    v = warp_sum(v);
+    __syncthreads();
+    if (lane == 0) red[w] = v;
+    __syncthreads();
+    float s = 0.f;
+    for (int i = 0; i < (int)(blockDim.x >> 5); ++i) s += red[i];
+    return s;
+}
+
+struct Ptrs {
+    float *Hp, *Hinv, *V, *R, *y, *b, *u2, *bC, *u2c, *u, *d, *K, *Vq, *vnorm, *rnorm;
+    double *D, *A, *c, *small, *gramV, *gramR;
+    int32_t *perm, *slotof;
+    SearchCtl* ctl;
+    int32_t* done_host;
+    int64_t nI, nJ, ldp, ldh, ldm, m, ng;
+    int g, k;
+};
+// layout of the `small` region (doubles, each g*g): indices of the matrices
+enum { S_CINV = 0, S_C1INV, S_Q1, S_Q1C, S_M2, S_GV, S_GX, S_GR, S_C, S_P, S_T1, S_T2, S_T3, S_C1, S_L, S_LI };
+
+// ------------------------------------------------------------------ row norms / group Grams
+// norm[i] = ||M[i, 0:ld)||^2 (pads are zero); one block per row.
+__global__ void k_row_norms(const float* __restrict__ M, int64_t ld, float* __restrict__ norm, const SearchCtl* ctl)
+{
+    if (ctl->done) return;
+    __shared__ float red[32];
+    const float4* row = reinterpret_cast<const float4*>(M + (int64_t)blockIdx.x * ld);
+    float acc = 0.f;
+    for (int64_t c = threadIdx.x; c < ld / 4; c += blockDim.x) {
+        const float4 v = row[c];
+        acc += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+    }
+    acc = block_sum_f(acc, red);
+    if (threadIdx.x == 0) norm[blockIdx.x] = acc;
+}
+
+// gram[grp][a][b] = M[grp*g+a,:] . M[grp*g+b,:]; grid (groups, g), warps loop over b.
+__global__ void k_group_gram(const float* __restrict__ M, int64_t ld, int g, double* __restrict__ gram, const SearchCtl* ctl)
+{
+    if (ctl->done) return;
+    const int64_t grp = blockIdx.x;
+    const int a = blockIdx.y;
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    const float4* ra = reinterpret_cast<const float4*>(M + (grp * g + a) * ld);
+    for (int b = w; b < g; b += nw) {
+        const float4* rb = reinterpret_cast<const float4*>(M + (grp * g + b) * ld);
+        float s = 0.f;
+        for (int64_t c = lane; c < ld / 4; c += 32) {
+            const float4 x = ra[c], z = rb[c];
+            s += x.x * z.x + x.y * z.y + x.z * z.z + x.w * z.w;
+        }
+        s = warp_sum(s);
+        if (lane == 0) gram[(grp * g + a) * g + b] = (double)s;
+    }
+}
+
+// Block-cooperative Cholesky inverse of the g x g SPD matrix M (ld g, overwritten by its factor).
+// Lw, Out: g x g work / result.  Returns the smallest pivot (<= 0 when not positive definite).
+__device__ double chol_inverse(double* M, double* Lw, double* Out, int g)
+{
+    __shared__ double minpiv;
+    const int t = threadIdx.x, nt = blockDim.x;
+    if (t == 0) minpiv = DBL_MAX;
+    __syncthreads();
+    for (int j = 0; j < g; ++j) {
+        if (t == 0) {
+            double dd = M[j * g + j];
+            if (dd < minpiv) minpiv = dd;
+            if (!(dd > 0.0)) { minpiv = -1.0; dd = 1.0; }
+            M[j * g + j] = sqrt(dd);
+        }
+        __syncthreads();
+        const double djj = M[j * g + j];
+        for (int i = j + 1 + t; i < g; i += nt) M[i * g + j] /= djj;
+        __syncthreads();
+        const int rem = g - j - 1;
+        for (int idx = t; idx < rem * rem; idx += nt) {
+            const int i = j + 1 + idx / rem, c = j + 1 + idx % rem;
+            if (c <= i) M[i * g + c] -= M[i * g + j] * M[c * g + j];
+        }
+        __syncthreads();
+    }
+    for (int c = t; c < g; c += nt) {
+        for (int i = 0; i < g; ++i) {
+            double s = (i == c) ? 1.0 : 0.0;
+            for (int kx = c; kx < i; ++kx) s -= M[i * g + kx] * Lw[kx * g + c];
+            Lw[i * g + c] = (i < c) ? 0.0 : s / M[i * g + i];
+        }
+    }
+    __syncthreads();
+    for (int idx = t; idx < g * g; idx += nt) {
+        const int i = idx / g, j = idx % g;
+        double s = 0.0;
+        for (int kx = (i > j ? i : j); kx < g; ++kx) s += Lw[kx * g + i] * Lw[kx * g + j];
+        Out[idx] = s;
+    }
+    __syncthreads();
+    return minpiv;
+}
+// C = op(A) * op(B), all g x g, block-cooperative.
+__device__ void mat_mul(const double* A, bool tA, const double* B, bool tB, double* C, int g)
+{
+    for (int idx = threadIdx.x; idx < g * g; idx += blockDim.x) {
+        const int i = idx / g, j = idx % g;
+        double s = 0.0;
+        for (int kx = 0; kx < g; ++kx)
+            s += (tA ? A[kx * g + i] : A[i * g + kx]) * (tB ? B[j * g + kx] : B[kx * g + j]);
+        C[idx] = s;
+    }
+    __syncthreads();
+}
+__device__ double mat_trace_prod(const double* A, const double* B, int g, double* red)   // sum A .* B^T = Tr(A B)
+{
+    double s = 0.0;
+    for (int idx = threadIdx.x; idx < g * g; idx += blockDim.x) s += A[idx] * B[(idx % g) * g + idx / g];
+    s = warp_sum(s);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = s;
+    __syncthreads();
+    double tot = 0.0;
+    for (int i = 0; i < (int)(blockDim.x >> 5); ++i) tot += red[i];
+    __syncthreads();
+    return tot;
+}
+
+// Scores of groups of more than one row: score = Tr(M^-1 Gram); one block per group.
+// kind 0: kept slots (M = Hinv_rr, Gram of V rows) -> D; kind 1: pruned slots (M = c, Gram of R rows) -> A.
+__global__ void k_scores_general(Ptrs p, int kind)
+{
+    if (p.ctl->done) return;
+    extern __shared__ double smd[];
+    const int g = p.g;
+    double* M = smd; double* Lw = smd + g * g; double* Out = Lw + g * g;
+    __shared__ double red[32];
+    const int64_t grp = blockIdx.x;
+    double scale = 0.0;
+    for (int idx = threadIdx.x; idx < g * g; idx += blockDim.x) {
+        const int i = idx / g, j = idx % g;
+        if (kind == 0) {
+            M[idx] = 0.5 * ((double)p.Hinv[(grp * g + i) * p.ldh + grp * g + j] + (double)p.Hinv[(grp * g + j) * p.ldh + grp * g + i]);
+        } else {
+            M[idx] = 0.5 * (p.c[grp * g * g + idx] + p.c[grp * g * g + j * g + i]);
+        }
+    }
+    if (kind == 1) {
+        for (int i = 0; i < g; ++i) {
+            const double hd = p.Hp[(p.nI + grp * g + i) * p.ldp + p.nI + grp * g + i];
+            if (hd > scale) scale = hd;
+        }
+    }
+    __syncthreads();
+    const double piv = chol_inverse(M, Lw, Out, g);
+    const double* gram = (kind == 0 ? p.gramV : p.gramR) + grp * g * g;
+    const double tr = mat_trace_prod(Out, gram, g, red);
+    if (threadIdx.x == 0) {
+        if (kind == 0) p.D[grp] = (piv > 0.0) ? tr : INFINITY;
+        else p.A[grp] = (piv > kAddPivotTol * scale) ? tr : -INFINITY;
+    }
+}
+
+// ------------------------------------------------------------------ selection
+// Cheapest drop (min D, ties -> smaller group id) and most valuable add (max A, ties -> smaller id).
+__global__ void __launch_bounds__(1024) k_select(Ptrs p)
+{
+    SearchCtl* ctl = p.ctl;
+    if (ctl->done) return;
+    __shared__ double sv[32]; __shared__ int sid[32]; __shared__ int sidx[32];
+    const int t = threadIdx.x, lane = t & 31, w = t >> 5;
+    const int npr = (int)(p.ng - p.k);
+    for (int pass = 0; pass < 2; ++pass) {
+        const int n = pass == 0 ? p.k : npr;
+        double best = INFINITY; int bid = INT_MAX; int bidx = -1;
+        for (int i = t; i < n; i += blockDim.x) {
+            double v;
+            if (pass == 0) {
+                if (p.g == 1) {
+                    const double hd = p.Hinv[(int64_t)i * p.ldh + i];
+                    v = hd > 0.0 ? (double)p.vnorm[i] / hd : INFINITY;
+                    p.D[i] = v;
+                } else v = p.D[i];
+            } else {
+                if (p.g == 1) {
+                    const double cc = p.c[i];
+                    const double hd = p.Hp[(p.nI + i) * p.ldp + p.nI + i];
+                    v = cc > kAddPivotTol * hd ? (double)p.rnorm[i] / cc : -INFINITY;
+                    p.A[i] = v;
+                } else v = p.A[i];
+                v = -v;
+            }
+            const int id = p.perm[pass == 0 ? i : p.k + i];
+            if (v < best || (v == best && id < bid)) { best = v; bid = id; bidx = i; }
+        }
+        for (int o = 16; o > 0; o >>= 1) {
+            const double ov = __shfl_xor_sync(0xffffffffu, best, o);
+            const int oid = __shfl_xor_sync(0xffffffffu, bid, o);
+            const int oidx = __shfl_xor_sync(0xffffffffu, bidx, o);
+            if (ov < best || (ov == best && oid < bid)) { best = ov; bid = oid; bidx = oidx; }
+        }
+        __syncthreads();
+        if (lane == 0) { sv[w] = best; sid[w] = bid; sidx[w] = bidx; }
+        __syncthreads();
+        if (t == 0) {
+            for (int i = 1; i < (int)(blockDim.x >> 5); ++i)
+                if (sv[i] < best || (sv[i] == best && sid[i] < bid)) { best = sv[i]; bid = sid[i]; bidx = sidx[i]; }
+            const bool ok = bidx >= 0 && isfinite(best);
+            if (pass == 0) { ctl->sel_slot = bidx; ctl->sel_D = best; }
+            else ctl->sel_t = bidx;
+            if (!ok) { ctl->done = 1; ctl->stop_reason = OSSCAR_STOP_GUARD; *p.done_host = 1; }
+        }
+        __syncthreads();
+    }
+}
+
+// ------------------------------------------------------------------ y = Hinv h  (one warp per row, grid.y = e)
+__global__ void __launch_bounds__(256) k_ypass(Ptrs p)
+{
+    if (p.ctl->done) return;
+    const int e = blockIdx.y;
+    const int lane = threadIdx.x & 31;
+    const int64_t s = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (s >= p.nI) return;
+    const float4* hrow = reinterpret_cast<const float4*>(p.Hp + (p.nI + (int64_t)p.ctl->sel_t * p.g + e) * p.ldp);
+    const float4* arow = reinterpret_cast<const float4*>(p.Hinv + s * p.ldh);
+    float a0 = 0.f, a1 = 0.f;
+    const int64_t n4 = p.ldh / 4;
+    int64_t c = lane;
+    for (; c + 32 < n4; c += 64) {
+        const float4 x0 = arow[c], x1 = arow[c + 32];
+        const float4 h0 = __ldg(hrow + c), h1 = __ldg(hrow + c + 32);
+        a0 += x0.x * h0.x + x0.y * h0.y + x0.z * h0.z + x0.w * h0.w;
+        a1 += x1.x * h1.x + x1.y * h1.y + x1.z * h1.z + x1.w * h1.w;
+    }
+    for (; c < n4; c += 32) {
+        const float4 x0 = arow[c]; const float4 h0 = __ldg(hrow + c);
+        a0 += x0.x * h0.x + x0.y * h0.y + x0.z * h0.z + x0.w * h0.w;
+    }
+    a0 = warp_sum(a0 + a1);
+    if (lane == 0) p.y[(int64_t)e * p.ldh + s] = a0;
+}
+
+// Grams of the chosen rows: GV = V_r V_r^T, GX = V_r R_q^T, GR = R_q R_q^T; one warp per entry.
+__global__ void __launch_bounds__(256) k_pairgram(Ptrs p)
+{
+    if (p.ctl->done) return;
+    const int g = p.g;
+    const int64_t wid = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (wid >= 3LL * g * g) return;
+    const int which = (int)(wid / (g * g)), a = (int)((wid / g) % g), b = (int)(wid % g);
+    const int lane = threadIdx.x & 31;
+    const float* Vr = p.V + (int64_t)p.ctl->sel_slot * g * p.ldm;
+    const float* Rq = p.R + (int64_t)p.ctl->sel_t * g * p.ldm;
+    const float4* x = reinterpret_cast<const float4*>((which == 2 ? Rq : Vr) + (int64_t)a * p.ldm);
+    const float4* z = reinterpret_cast<const float4*>((which == 0 ? Vr : Rq) + (int64_t)b * p.ldm);
+    float s = 0.f;
+    for (int64_t c = lane; c < p.ldm / 4; c += 32) {
+        const float4 xa = x[c], zb = z[c];
+        s += xa.x * zb.x + xa.y * zb.y + xa.z * zb.z + xa.w * zb.w;
+    }
+    s = warp_sum(s);
+    if (lane == 0) p.small[(S_GV + which) * g * g + a * g + b] = (double)s;
+}
+
+// One block: the g x g algebra of the step, the exact change of obj and the accept decision.
+__global__ void __launch_bounds__(256)
+k_small(Ptrs p, int accept_mode, double accept_tol, int max_swaps, double* __restrict__ obj_trace, int32_t* __restrict__ swap_trace)
+{
+    SearchCtl* ctl = p.ctl;
+    if (ctl->done) return;
+    __shared__ double red[32];
+    const int g = p.g, gg = g * g;
+    double* S = p.small;
+    double *Cinv = S + S_CINV * gg, *c1inv = S + S_C1INV * gg, *Q1 = S + S_Q1 * gg, *Q1c = S + S_Q1C * gg, *M2 = S + S_M2 * gg;
+    double *GV = S + S_GV * gg, *GX = S + S_GX * gg, *GR = S + S_GR * gg, *C = S + S_C * gg, *P = S + S_P * gg;
+    double *T1 = S + S_T1 * gg, *T2 = S + S_T2 * gg, *T3 = S + S_T3 * gg, *c1 = S + S_C1 * gg, *Lw = S + S_L * gg;
+    const int64_t r0 = (int64_t)ctl->sel_slot * g;
+    const int64_t tq = ctl->sel_t;
+    for (int idx = threadIdx.x; idx < gg; idx += blockDim.x) {
+        const int i = idx / g, j = idx % g;
+        C[idx] = 0.5 * ((double)p.Hinv[(r0 + i) * p.ldh + r0 + j] + (double)p.Hinv[(r0 + j) * p.ldh + r0 + i]);
+        P[idx] = (double)p.y[(int64_t)i * p.ldh + r0 + j];           // P[a][b] = y_a[r_b]
+    }
+    __syncthreads();
+    const double pivC = chol_inverse(C, Lw, Cinv, g);
+    const double Ds = mat_trace_prod(Cinv, GV, g, red);               // Tr(C^-1 V_r V_r^T)
+    // R1 R1^T = GR + P (Cinv GX) + (P Cinv GX)^T + P Cinv GV Cinv P^T
+    mat_mul(Cinv, false, GX, false, T1, g);                           // K R_q^T
+    mat_mul(P, false, T1, false, T2, g);                              // P K R_q^T
+    mat_mul(P, false, Cinv, false, T1, g);                            // P Cinv
+    mat_mul(T1, false, GV, false, T3, g);                             // P Cinv GV
+    mat_mul(T3, false, T1, true, Lw, g);                              // P Cinv GV Cinv P^T  (Lw reused as scratch)
+    for (int idx = threadIdx.x; idx < gg; idx += blockDim.x) {
+        const int i = idx / g, j = idx % g;
+        T3[idx] = GR[idx] + T2[idx] + T2[j * g + i] + Lw[idx];
+    }
+    __syncthreads();
+    mat_mul(T1, false, P, true, T2, g);                               // P Cinv P^T
+    for (int idx = threadIdx.x; idx < gg; idx += blockDim.x) {
+        const int i = idx / g, j = idx % g;
+        const double cq = 0.5 * (p.c[tq * gg + idx] + p.c[tq * gg + j * g + i]);
+        c1[idx] = cq + 0.5 * (T2[idx] + T2[j * g + i]);
+    }
+    __syncthreads();
+    const double pivc1 = chol_inverse(c1, Lw, c1inv, g);
+    const double gain = mat_trace_prod(c1inv, T3, g, red);
+    const double delta = Ds - gain;
+    mat_mul(Cinv, false, P, true, Q1, g);                             // Q1 = Cinv y_r = Cinv P^T
+    mat_mul(Q1, false, c1inv, false, Q1c, g);                         // Q1 c1inv
+    mat_mul(c1inv, false, T1, false, M2, g);                          // c1inv P Cinv
+    if (threadIdx.x == 0) {
+        const double obj = ctl->obj;
+        bool stop = false; int reason = 0;
+        if (!(pivC > 0.0) || !(pivc1 > 0.0) || !isfinite(delta)) { stop = true; reason = OSSCAR_STOP_GUARD; }
+        else if (accept_mode == OSSCAR_ACCEPT_IMPROVING && !(delta <= -accept_tol * obj)) { stop = true; reason = OSSCAR_STOP_NO_IMPROVEMENT; }
+        ctl->delta = delta;
+        if (stop) { ctl->done = 1; ctl->stop_reason = reason; *p.done_host = 1; }
+        else {
+            const int n = ctl->n_swaps;
+            swap_trace[2 * n] = p.perm[ctl->sel_slot];
+            swap_trace[2 * n + 1] = p.perm[p.k + tq];
+            obj_trace[n + 1] = obj + delta;
+            ctl->obj = obj + delta;
+            ctl->n_swaps = n + 1;
+        }
+    }
+}
+
+// Staged vectors of the step.  Part A (threads over kept rows s): b, bC = b C^-1, u2, u2c = u2 c1^-1.
+// Part B (threads over columns): K = C^-1 V_r, Vq = c1^-1 R_q + (c1^-1 P C^-1) V_r.
+__global__ void __launch_bounds__(256) k_prep(Ptrs p)
+{
+    if (p.ctl->done) return;
+    const int g = p.g, gg = g * g;
+    const double* S = p.small;
+    const double *Cinv = S + S_CINV * gg, *c1inv = S + S_C1INV * gg, *Q1 = S + S_Q1 * gg, *Q1c = S + S_Q1C * gg, *M2 = S + S_M2 * gg;
+    const int64_t r0 = (int64_t)p.ctl->sel_slot * g;
+    const int64_t q0 = (int64_t)p.ctl->sel_t * g;
+    const int64_t nA = p.nI * g, nB = p.ldm * g;
+    for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < nA + nB; idx += (int64_t)gridDim.x * blockDim.x) {
+        if (idx < nA) {
+            const int e = (int)(idx / p.nI); const int64_t s = idx % p.nI;
+            double bc = 0.0, bq = 0.0, bqc = 0.0, yc = 0.0;
+            for (int f = 0; f < g; ++f) {
+                const double bf = (double)p.Hinv[(r0 + f) * p.ldh + s];
+                bc += bf * Cinv[f * g + e];
+                bq += bf * Q1[f * g + e];
+                bqc += bf * Q1c[f * g + e];
+                yc += (double)p.y[(int64_t)f * p.ldh + s] * c1inv[f * g + e];
+            }
+            const bool in_r = s >= r0 && s < r0 + g;
+            p.b[(int64_t)e * p.ldh + s] = p.Hinv[(r0 + e) * p.ldh + s];
+            p.bC[(int64_t)e * p.ldh + s] = (float)bc;
+            p.u2[(int64_t)e * p.ldh + s] = in_r ? 0.f : (float)((double)p.y[(int64_t)e * p.ldh + s] - bq);
+            p.u2c[(int64_t)e * p.ldh + s] = in_r ? 0.f : (float)(yc - bqc);
+        } else {
+            const int64_t j = idx - nA;
+            const int e = (int)(j / p.ldm); const int64_t c = j % p.ldm;
+            double kk = 0.0, vq = 0.0;
+            for (int f = 0; f < g; ++f) {
+                const double vr = (double)p.V[(r0 + f) * p.ldm + c];
+                const double rq = (double)p.R[(q0 + f) * p.ldm + c];
+                kk += Cinv[e * g + f] * vr;
+                vq += c1inv[e * g + f] * rq + M2[e * g + f] * vr;
+            }
+            p.K[(int64_t)e * p.ldm + c] = (float)kk;
+            p.Vq[(int64_t)e * p.ldm + c] = (float)vq;
+        }
+    }
+}
+
+// u_l = Hp[l, 0:n_I] b,  d_l = Hp[l, q] - Hp[l, 0:n_I] u2   for the pruned rows and the g leaving rows.
+// One warp handles RPW consecutive rows for one e (grid.y = e).
+template <int RPW>
+__global__ void __launch_bounds__(256) k_hpass(Ptrs p)
+{
+    if (p.ctl->done) return;
+    const int e = blockIdx.y, g = p.g;
+    const int lane = threadIdx.x & 31;
+    const int64_t nrows = p.nJ + g;
+    const int64_t l0 = ((int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * RPW;
+    if (l0 >= nrows) return;
+    const int64_t r0 = (int64_t)p.ctl->sel_slot * g;
+    const int64_t qcol = p.nI + (int64_t)p.ctl->sel_t * g + e;
+    const float4* rows[RPW];
+#pragma unroll
+    for (int i = 0; i < RPW; ++i) {
+        int64_t l = l0 + i; if (l >= nrows) l = nrows - 1;
+        const int64_t hrow = l < p.nJ ? p.nI + l : r0 + (l - p.nJ);
+        rows[i] = reinterpret_cast<const float4*>(p.Hp + hrow * p.ldp);
+    }
+    const float4* bv = reinterpret_cast<const float4*>(p.b + (int64_t)e * p.ldh);
+    const float4* uv = reinterpret_cast<const float4*>(p.u2 + (int64_t)e * p.ldh);
+    float au[RPW], ad[RPW];
+#pragma unroll
+    for (int i = 0; i < RPW; ++i) { au[i] = 0.f; ad[i] = 0.f; }
+    for (int64_t c = lane; c < p.ldh / 4; c += 32) {
+        const float4 bb = __ldg(bv + c), uu = __ldg(uv + c);
+#pragma unroll
+        for (int i = 0; i < RPW; ++i) {
+            const float4 x = rows[i][c];
+            au[i] += x.x * bb.x + x.y * bb.y + x.z * bb.z + x.w * bb.w;
+            ad[i] += x.x * uu.x + x.y * uu.y + x.z * uu.z + x.w * uu.w;
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < RPW; ++i) {
+        const float su = warp_sum(au[i]), sd = warp_sum(ad[i]);
+        const int64_t l = l0 + i;
+        if (lane == 0 && l < nrows) {
+            p.u[l * g + e] = su;
+            p.d[l * g + e] = reinterpret_cast<const float*>(rows[i])[qcol] - sd;
+        }
+    }
+}
+
+// Hinv' = Hinv - bC b^T + u2c u2^T; rows/columns of r take -u2c, the rr block c1^-1.
+// Block: 256 threads x float4 = 1024 columns, RT rows.
+constexpr int HI_RT = 8;
+__global__ void __launch_bounds__(256) k_update_hinv(Ptrs p)
+{
+    if (p.ctl->done) return;
+    const int g = p.g;
+    const int64_t c4 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;     // float4 column index
+    if (c4 * 4 >= p.ldh) return;
+    const int64_t col = c4 * 4;
+    const int64_t r0 = (int64_t)p.ctl->sel_slot * g;
+    const int64_t row0 = (int64_t)blockIdx.y * HI_RT;
+    const double* c1inv = p.small + S_C1INV * g * g;
+    if (g == 1) {
+        const float4 bb = reinterpret_cast<const float4*>(p.b)[c4];
+        const float4 uu = reinterpret_cast<const float4*>(p.u2)[c4];
+        const float4 uc = reinterpret_cast<const float4*>(p.u2c)[c4];
+#pragma unroll
+        for (int i = 0; i < HI_RT; ++i) {
+            const int64_t s = row0 + i;
+            if (s >= p.nI) break;
+            float4* ptr = reinterpret_cast<float4*>(p.Hinv + s * p.ldh) + c4;
+            float4 h = *ptr;
+            if (s == r0) {
+                h.x = -uc.x; h.y = -uc.y; h.z = -uc.z; h.w = -uc.w;
+            } else {
+                const float nb = -p.bC[s], us = p.u2c[s];
+                h.x = fmaf(us, uu.x, fmaf(nb, bb.x, h.x));
+                h.y = fmaf(us, uu.y, fmaf(nb, bb.y, h.y));
+                h.z = fmaf(us, uu.z, fmaf(nb, bb.z, h.z));
+                h.w = fmaf(us, uu.w, fmaf(nb, bb.w, h.w));
+            }
+            float* hf = reinterpret_cast<float*>(&h);
+            if (r0 >= col && r0 < col + 4) hf[r0 - col] = (s == r0) ? (float)c1inv[0] : -p.u2c[s];
+            *ptr = h;
+        }
+        return;
+    }
+    for (int i = 0; i < HI_RT; ++i) {
+        const int64_t s = row0 + i;
+        if (s >= p.nI) break;
+        float4* ptr = reinterpret_cast<float4*>(p.Hinv + s * p.ldh) + c4;
+        float4 h = *ptr;
+        float* hf = reinterpret_cast<float*>(&h);
+        const bool srow = s >= r0 && s < r0 + g;
+        for (int j = 0; j < 4; ++j) {
+            const int64_t sc = col + j;
+            const bool scol = sc >= r0 && sc < r0 + g;
+            float v;
+            if (srow && scol) v = (float)c1inv[(s - r0) * g + (sc - r0)];
+            else if (srow) v = -p.u2c[(s - r0) * p.ldh + sc];
+            else if (scol) v = -p.u2c[(sc - r0) * p.ldh + s];
+            else {
+                v = hf[j];
+                for (int e = 0; e < g; ++e) {
+                    v = fmaf(-p.bC[(int64_t)e * p.ldh + s], p.b[(int64_t)e * p.ldh + sc], v);
+                    v = fmaf(p.u2c[(int64_t)e * p.ldh + s], p.u2[(int64_t)e * p.ldh + sc], v);
+                }
+            }
+            hf[j] = v;
+        }
+        *ptr = h;
+    }
+}
+
+// Row updates of V (kind 0) and R (kind 1) with the squared row norm of the result (g = 1 scoring).
+//   V'[s] = V[s] - sum_e b[e][s] K[e] - sum_e u2[e][s] Vq[e]         (rows of r: Vq)
+//   R'[l] = R[l] + sum_e u[l][e] K[e] - sum_e d[l][e] Vq[e]          (rows of q: K[e] - sum_f d[nJ+e][f] Vq[f])
+// For g = 1 the R pass also moves c and the kept pass nothing else.  One block per ROWS rows.
+constexpr int UP_ROWS = 4;
+__global__ void __launch_bounds__(256) k_update_rows(Ptrs p, int kind)
+{
+    if (p.ctl->done) return;
+    __shared__ float red[32];
+    const int g = p.g;
+    float* M = kind == 0 ? p.V : p.R;
+    const int64_t nrows = kind == 0 ? p.nI : p.nJ;
+    const int64_t special0 = (kind == 0 ? (int64_t)p.ctl->sel_slot : (int64_t)p.ctl->sel_t) * g;
+    const int64_t n4 = p.ldm / 4;
+    const int64_t row0 = (int64_t)blockIdx.x * UP_ROWS;
+    for (int i = 0; i < UP_ROWS; ++i) {
+        const int64_t s = row0 + i;
+        if (s >= nrows) break;
+        const bool special = s >= special0 && s < special0 + g;
+        float4* row = reinterpret_cast<float4*>(M + s * p.ldm);
+        float nrm = 0.f;
+        for (int64_t c = threadIdx.x; c < n4; c += blockDim.x) {
+            float4 v;
+            if (special) {
+                const int e = (int)(s - special0);
+                if (kind == 0) v = reinterpret_cast<const float4*>(p.Vq + (int64_t)e * p.ldm)[c];
+                else {
+                    v = reinterpret_cast<const float4*>(p.K + (int64_t)e * p.ldm)[c];
+                    for (int f = 0; f < g; ++f) {
+                        const float df = -p.d[(p.nJ + e) * g + f];
+                        const float4 q = reinterpret_cast<const float4*>(p.Vq + (int64_t)f * p.ldm)[c];
+                        v.x = fmaf(df, q.x, v.x); v.y = fmaf(df, q.y, v.y); v.z = fmaf(df, q.z, v.z); v.w = fmaf(df, q.w, v.w);
+                    }
+                }
+            } else {
+                v = row[c];
+                for (int e = 0; e < g; ++e) {
+                    const float ck = kind == 0 ? -p.b[(int64_t)e * p.ldh + s] : p.u[s * g + e];
+                    const float cq = kind == 0 ? -p.u2[(int64_t)e * p.ldh + s] : -p.d[s * g + e];
+                    const float4 kk = reinterpret_cast<const float4*>(p.K + (int64_t)e * p.ldm)[c];
+                    const float4 q = reinterpret_cast<const float4*>(p.Vq + (int64_t)e * p.ldm)[c];
+                    v.x = fmaf(cq, q.x, fmaf(ck, kk.x, v.x));
+                    v.y = fmaf(cq, q.y, fmaf(ck, kk.y, v.y));
+                    v.z = fmaf(cq, q.z, fmaf(ck, kk.z, v.z));
+                    v.w = fmaf(cq, q.w, fmaf(ck, kk.w, v.w));
+                }
+            }
+            row[c] = v;
+            nrm += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+        }
+        if (g == 1) {
+            nrm = block_sum_f(nrm, red);
+            if (threadIdx.x == 0) {
+                if (kind == 0) p.vnorm[s] = nrm;
+                else {
+                    p.rnorm[s] = nrm;
+                    const double Cinv = p.small[S_CINV], c1inv = p.small[S_C1INV];
+                    if (special) { const double dd = p.d[p.nJ]; p.c[s] = Cinv - dd * dd * c1inv; }
+                    else { const double uu = p.u[s], dd = p.d[s]; p.c[s] += uu * uu * Cinv - dd * dd * c1inv; }
+                }
+            }
+        }
+    }
+}
+
+// c_l' = c_l + u_l C^-1 u_l^T - d_l c1^-1 d_l^T for every pruned slot (g > 1); the entering slot receives
+// the leaving group: c' = C^-1 - d_r c1^-1 d_r^T.  One block per pruned slot.
+__global__ void __launch_bounds__(128) k_update_c(Ptrs p)
+{
+    if (p.ctl->done) return;
+    const int g = p.g, gg = g * g;
+    const int64_t t = blockIdx.x;
+    const bool special = t == p.ctl->sel_t;
+    const double* Cinv = p.small + S_CINV * gg;
+    const double* c1inv = p.small + S_C1INV * gg;
+    const float* ul = p.u + (special ? p.nJ : t * g) * g;     // g x g, row a = row of the group
+    const float* dl = p.d + (special ? p.nJ : t * g) * g;
+    for (int idx = threadIdx.x; idx < gg; idx += blockDim.x) {
+        const int a = idx / g, b2 = idx % g;
+        double s = special ? Cinv[idx] : p.c[t * gg + idx];
+        for (int e = 0; e < g; ++e) {
+            double tu = 0.0, td = 0.0;
+            for (int f = 0; f < g; ++f) {
+                if (!special) tu += Cinv[e * g + f] * (double)ul[b2 * g + f];
+                td += c1inv[e * g + f] * (double)dl[b2 * g + f];
+            }
+            if (!special) s += (double)ul[a * g + e] * tu;
+            s -= (double)dl[a * g + e] * td;
+        }
+        p.c[t * gg + idx] = s;      // each thread reads only its own old entry
+    }
+}
+
+// Exchange the rows (phase 0) or columns (phase 1) of Hp that belong to the leaving and entering groups;
+// phase 1 also exchanges the two groups in the slot permutation.
+__global__ void __launch_bounds__(256) k_hswap(Ptrs p, int phase)
+{
+    if (p.ctl->done) return;
+    const int g = p.g;
+    const int64_t a0 = (int64_t)p.ctl->sel_slot * g, b0 = p.nI + (int64_t)p.ctl->sel_t * g;
+    const int64_t n = p.ldp * g;
+    for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < n; idx += (int64_t)gridDim.x * blockDim.x) {
+        const int e = (int)(idx / p.ldp); const int64_t x = idx % p.ldp;
+        float *pa, *pb;
+        if (phase == 0) { pa = p.Hp + (a0 + e) * p.ldp + x; pb = p.Hp + (b0 + e) * p.ldp + x; }
+        else {
+            if (x >= p.nI + p.nJ) continue;
+            pa = p.Hp + x * p.ldp + a0 + e; pb = p.Hp + x * p.ldp + b0 + e;
+        }
+        const float va = *pa, vb = *pb;
+        *pa = vb; *pb = va;
+    }
+    if (phase == 1 && blockIdx.x == 0 && threadIdx.x == 0) {
+        const int s = p.ctl->sel_slot, t = p.k + p.ctl->sel_t;
+        const int gi = p.perm[s], gj = p.perm[t];
+        p.perm[s] = gj; p.perm[t] = gi;
+        p.slotof[gj] = s; p.slotof[gi] = t;
+    }
+}
+
+// ------------------------------------------------------------------ finalize
+__global__ void k_scatter_rows(Ptrs p, float* __restrict__ W_out)
+{
+    const int64_t s = blockIdx.x;
+    const int64_t row = (int64_t)p.perm[s / p.g] * p.g + s % p.g;
+    for (int64_t c = threadIdx.x; c < p.m; c += blockDim.x) W_out[row * p.m + c] = p.V[s * p.ldm + c];
+}
+__global__ void k_sorted_support(Ptrs p, int32_t* __restrict__ out)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= p.k) return;
+    const int id = p.perm[i];
+    int rank = 0;
+    for (int j = 0; j < p.k; ++j) rank += p.perm[j] < id;
+    out[rank] = id;
+}
+__global__ void k_begin(SearchCtl* ctl, double* obj_trace, int32_t* done_host)
+{
+    ctl->done = 0; ctl->stop_reason = OSSCAR_STOP_MAX_SWAPS; ctl->n_swaps = 0; ctl->n_refresh = 0;
+    obj_trace[0] = ctl->obj;
+    ctl->acc[2] = ctl->obj;
+    *done_host = 0;
+}
+__global__ void k_count_refresh(SearchCtl* ctl) { if (!ctl->done) ctl->n_refresh += 1; }
+__global__ void k_final_obj(SearchCtl* ctl) { ctl->acc[3] = ctl->const_term - ctl->acc[1]; }
+
+Ptrs make_ptrs(osscar_ctx* ctx)
+{
+    const Layout& L = ctx->L;
+    char* ws = (char*)ctx->ws;
+    Ptrs p;
+    p.Hp = (float*)(ws + L.off_Hp); p.Hinv = (float*)(ws + L.off_Hinv); p.V = (float*)(ws + L.off_V);
+    p.R = (float*)(ws + L.off_R);
+    p.y = (float*)(ws + L.off_y); p.b = (float*)(ws + L.off_b); p.u2 = (float*)(ws + L.off_u2);
+    p.bC = (float*)(ws + L.off_bC); p.u2c = (float*)(ws + L.off_u2c);
+    p.u = (float*)(ws + L.off_u); p.d = (float*)(ws + L.off_d);
+    p.K = (float*)(ws + L.off_K); p.Vq = (float*)(ws + L.off_Vq);
+    p.vnorm = (float*)(ws + L.off_vnorm); p.rnorm = (float*)(ws + L.off_rnorm);
+    p.D = (double*)(ws + L.off_D); p.A = (double*)(ws + L.off_A); p.c = (double*)(ws + L.off_c);
+    p.small = (double*)(ws + L.off_small); p.gramV = (double*)(ws + L.off_gramV); p.gramR = (double*)(ws + L.off_gramR);
+    p.perm = (int32_t*)(ws + L.off_perm); p.slotof = (int32_t*)(ws + L.off_slotof);
+    p.ctl = ctx->ctl; p.done_host = ctx->done_flag_dev;
+    p.nI = L.nI; p.nJ = L.nJ; p.ldp = L.ldp; p.ldh = L.ldh; p.ldm = L.ldm; p.m = L.m; p.ng = L.ng;
+    p.g = L.g; p.k = L.k;
+    return p;
+}
+
+#define CK(x) do { cudaError_t e_ = (x); if (e_ != cudaSuccess) return OSSCAR_E_CUDA; } while (0)
+
+// Everything the selection needs from a freshly built or freshly updated state.
+cudaError_t enqueue_scores(osscar_ctx* ctx, const Ptrs& p, bool norms)
+{
+    cudaStream_t st = ctx->stream;
+    if (p.g == 1) {
+        if (norms) {
+            k_row_norms<<<(unsigned)p.nI, 256, 0, st>>>(p.V, p.ldm, p.vnorm, p.ctl);
+            if (p.nJ > 0) k_row_norms<<<(unsigned)p.nJ, 256, 0, st>>>(p.R, p.ldm, p.rnorm, p.ctl);
+        }
+    } else {
+        const size_t smem = 3 * (size_t)p.g * p.g * sizeof(double);
+        cudaError_t e = cudaFuncSetAttribute(k_scores_general, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        k_group_gram<<<dim3((unsigned)p.k, (unsigned)p.g), 256, 0, st>>>(p.V, p.ldm, p.g, p.gramV, p.ctl);
+        k_scores_general<<<(unsigned)p.k, 256, smem, st>>>(p, 0);
+        if (p.nJ > 0) {
+            k_group_gram<<<dim3((unsigned)(p.ng - p.k), (unsigned)p.g), 256, 0, st>>>(p.R, p.ldm, p.g, p.gramR, p.ctl);
+            k_scores_general<<<(unsigned)(p.ng - p.k), 256, smem, st>>>(p, 1);
+        }
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t score_pass(osscar_ctx* ctx)
+{
+    Ptrs p = make_ptrs(ctx);
+    cudaError_t e = enqueue_scores(ctx, p, true);
+    if (e != cudaSuccess) return e;
+    k_select<<<1, 1024, 0, ctx->stream>>>(p);      // also leaves the score vectors D and A readable
+    return cudaGetLastError();
+}
+
+int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* support_out, float* W_out,
+               double* obj_trace, int32_t* swap_trace, osscar_search_result* res)
+{
+    const Layout& L = ctx->L;
+    cudaStream_t st = ctx->stream;
+    Ptrs p = make_ptrs(ctx);
+    const int g = L.g;
+    const double tol = prm->accept_rel_tol < 0 ? 1e-5 : prm->accept_rel_tol;
+    const int max_swaps = (L.nJ > 0) ? prm->max_swaps : 0;
+
+    k_begin<<<1, 1, 0, st>>>(ctx->ctl, obj_trace, ctx->done_flag_dev);
+    CK(cudaGetLastError());
+    CK(cudaEventRecord(ctx->ev0, st));
+    if (max_swaps > 0) CK(enqueue_scores(ctx, p, true));
+
+    const int batch = 32;
+    cudaEvent_t evb[2];
+    CK(cudaEventCreateWithFlags(&evb[0], cudaEventDisableTiming));
+    CK(cudaEventCreateWithFlags(&evb[1], cudaEventDisableTiming));
+    int rc = OSSCAR_OK;
+    const unsigned yblocks = (unsigned)((L.nI + 7) / 8);
+    constexpr int RPW = 4;
+    const unsigned hblocks = (unsigned)((L.nJ + g + 8 * RPW - 1) / (8 * RPW));
+    const unsigned prep_blocks = (unsigned)(((L.nI + L.ldm) * g + 255) / 256);
+    for (int it = 0; it < max_swaps && rc == OSSCAR_OK; ++it) {
+        if (it % batch == 0) {
+            const int bi = it / batch;
+            if (bi >= 2) {      // stay at most two batches ahead of the device, and stop feeding a finished loop
+                if (cudaEventSynchronize(evb[bi & 1]) != cudaSuccess) { rc = OSSCAR_E_CUDA; break; }
+                if (*ctx->done_flag_host) break;
+            }
+        }
+        if (prm->refresh_every > 0 && it > 0 && it % prm->refresh_every == 0) {
+            rc = build_state(ctx, true);
+            if (rc != OSSCAR_OK) break;
+            k_count_refresh<<<1, 1, 0, st>>>(ctx->ctl);
+            if (enqueue_scores(ctx, p, true) != cudaSuccess) { rc = OSSCAR_E_CUDA; break; }
+        }
+        k_select<<<1, 1024, 0, st>>>(p);
+        k_pairgram<<<(unsigned)((3 * g * g + 7) / 8), 256, 0, st>>>(p);
+        k_ypass<<<dim3(yblocks, g), 256, 0, st>>>(p);
+        k_small<<<1, 256, 0, st>>>(p, prm->accept_mode, tol, max_swaps, obj_trace, swap_trace);
+        k_prep<<<prep_blocks, 256, 0, st>>>(p);
+        k_hpass<RPW><<<dim3(hblocks, g), 256, 0, st>>>(p);
+        k_update_hinv<<<dim3((unsigned)((L.ldh / 4 + 255) / 256), (unsigned)((L.nI + HI_RT - 1) / HI_RT)), 256, 0, st>>>(p);
+        k_update_rows<<<(unsigned)((L.nI + UP_ROWS - 1) / UP_ROWS), 256, 0, st>>>(p, 0);
+        k_update_rows<<<(unsigned)((L.nJ + UP_ROWS - 1) / UP_ROWS), 256, 0, st>>>(p, 1);
+        if (g > 1) {
+            k_update_c<<<(unsigned)(L.ng - L.k), 128, 0, st>>>(p);
+            if (enqueue_scores(ctx, p, false) != cudaSuccess) { rc = OSSCAR_E_CUDA; break; }
+        }
+        k_hswap<<<(unsigned)((L.ldp * g + 255) / 256), 256, 0, st>>>(p, 0);
+        k_hswap<<<(unsigned)((L.ldp * g + 255) / 256), 256, 0, st>>>(p, 1);
+        if (cudaGetLastError() != cudaSuccess) { rc = OSSCAR_E_CUDA; break; }
+        if ((it + 1) % batch == 0) {
+            if (cudaEventRecord(evb[(it / batch) & 1], st) != cudaSuccess) { rc = OSSCAR_E_CUDA; break; }
+        }
+    }
+    cudaEventDestroy(evb[0]);
+    cudaEventDestroy(evb[1]);
+    if (rc != OSSCAR_OK) { cudaStreamSynchronize(st); return rc; }
+    CK(cudaEventRecord(ctx->ev1, st));
+
+    // results: weights, support, objective recomputed from the final state
+    CK(cudaMemsetAsync(W_out, 0, sizeof(float) * L.d1 * L.m, st));
+    k_scatter_rows<<<(unsigned)L.nI, 256, 0, st>>>(p, W_out);
+    k_sorted_support<<<(L.k + 255) / 256, 256, 0, st>>>(p, support_out);
+    {
+        float* big = (float*)((char*)ctx->ws + L.off_big);
+        // G_I in slot order, then Tr(G_I^T V)
+        CK(gather_rows(st, ctx->G, L.m, L.g, p.perm, 0, L.nI, big, L.ldm));
+        CK(trace_product(st, big, L.ldm, p.V, L.ldm, L.nI, L.m, &ctx->ctl->acc[1]));
+        k_final_obj<<<1, 1, 0, st>>>(ctx->ctl);
+    }
+    CK(cudaGetLastError());
+    CK(cudaMemcpyAsync(ctx->ctl_host, ctx->ctl, sizeof(SearchCtl), cudaMemcpyDeviceToHost, st));
+    CK(cudaStreamSynchronize(st));
+    float ms = 0.f;
+    CK(cudaEventElapsedTime(&ms, ctx->ev0, ctx->ev1));
+    res->n_swaps = ctx->ctl_host->n_swaps;
+    res->stop_reason = ctx->ctl_host->stop_reason;
+    res->n_refresh = ctx->ctl_host->n_refresh;
+    res->status = ctx->ctl_host->status;
+    res->obj_init = ctx->ctl_host->acc[2];
+    res->obj_final = ctx->ctl_host->acc[3];
+    res->ms_search = ms;
+    return ctx->ctl_host->status;
+}
+
+}  // namespace osscar

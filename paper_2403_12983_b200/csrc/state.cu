@@ -1,0 +1,412 @@
+// Starting support and construction of the search state for a given support:
+// slot-permuted copy of H, (H_II)^-1 by an in-place blocked exchange (Gauss-Jordan) inversion,
+// V = (H_II)^-1 G_I (Eq. tmp5), residual R, Schur complements c (Case 2 of Proposition 1).
+#include "osscar_internal.cuh"
+#include <math.h>
+
+namespace osscar {
+namespace {
+
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+// Block-wide sum (blockDim.x multiple of 32, <= 1024); result valid in thread 0.
+__device__ double block_sum(double v) {
+    __shared__ double red[32];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    v = warp_sum(v);
+    __syncthreads();
+    if (lane == 0) red[w] = v;
+    __syncthreads();
+    if (w == 0) {
+        v = (lane < (int)((blockDim.x + 31) >> 5)) ? red[lane] : 0.0;
+        v = warp_sum(v);
+    }
+    return v;
+}
+
+// e_q = Tr(W_q^T H_qq W_q) (mode 0) or ||W_q||_F^2 (mode 1); one block per group.
+__global__ void k_energy(const float* __restrict__ H, const float* __restrict__ W, int64_t d1, int64_t m,
+                         int g, int mode, double* __restrict__ e)
+{
+    const int64_t q = blockIdx.x;
+    const float* Wq = W + q * g * m;
+    double acc = 0.0;
+    for (int64_t c = threadIdx.x; c < m; c += blockDim.x) {
+        if (mode == OSSCAR_INIT_MAGNITUDE) {
+            for (int a = 0; a < g; ++a) { double w = Wq[a * m + c]; acc += w * w; }
+        } else {
+            for (int a = 0; a < g; ++a) {
+                double t = 0.0;
+                const float* Hrow = H + (q * g + a) * d1 + q * g;
+                for (int b = 0; b < g; ++b) t += (double)Hrow[b] * (double)Wq[b * m + c];
+                acc += (double)Wq[a * m + c] * t;
+            }
+        }
+    }
+    acc = block_sum(acc);
+    if (threadIdx.x == 0) e[q] = acc;
+}
+
+// kept[q] = 1 iff fewer than k groups beat q (larger energy, or equal energy and smaller id).
+__global__ void k_rank_select(const double* __restrict__ e, int64_t ng, int k, int32_t* __restrict__ kept)
+{
+    const int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (q >= ng) return;
+    const double eq = e[q];
+    int rank = 0;
+    for (int64_t p = 0; p < ng; ++p) {
+        const double ep = e[p];
+        rank += (ep > eq) || (ep == eq && p < q);
+    }
+    kept[q] = rank < k;
+}
+
+__global__ void k_user_support(const int32_t* __restrict__ support, int k, int64_t ng,
+                               int32_t* __restrict__ kept, SearchCtl* ctl)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= k) return;
+    const int q = support[i];
+    if (q < 0 || q >= ng) { ctl->status = OSSCAR_E_ARG; return; }
+    if (atomicExch(&kept[q], 1) != 0) ctl->status = OSSCAR_E_ARG;   // duplicate id
+}
+
+// Slots: kept groups in ascending id order take slots 0..k-1, pruned groups k..ng-1.
+__global__ void k_build_perm(const int32_t* __restrict__ kept, int64_t ng, int k,
+                             int32_t* __restrict__ perm, int32_t* __restrict__ slotof,
+                             int32_t* __restrict__ support)
+{
+    const int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (q >= ng) return;
+    int before_kept = 0;
+    for (int64_t p = 0; p < q; ++p) before_kept += kept[p];
+    const int slot = kept[q] ? before_kept : k + (int)(q - before_kept);
+    perm[slot] = (int32_t)q;
+    slotof[q] = slot;
+    if (kept[q]) support[slot] = (int32_t)q;
+}
+
+// Hp[i][j] = H[row(i)][row(j)], row(i) = perm[i / g] * g + i % g.
+__global__ void k_gather_sym(const float* __restrict__ H, int64_t d1, int g, const int32_t* __restrict__ perm,
+                             float* __restrict__ Hp, int64_t ldp)
+{
+    const int64_t i = blockIdx.x;
+    const int64_t ri = (int64_t)perm[i / g] * g + i % g;
+    for (int64_t j = (int64_t)blockIdx.y * blockDim.x + threadIdx.x; j < ldp; j += (int64_t)gridDim.y * blockDim.x) {
+        float v = 0.f;
+        if (j < d1) {
+            const int64_t rj = (int64_t)perm[j / g] * g + j % g;
+            v = H[ri * d1 + rj];
+        }
+        Hp[i * ldp + j] = v;
+    }
+}
+
+// dst[i][0..ld) = src[row(slot0*g + i)][0..m) zero-padded, for i in [0, nrows).
+__global__ void k_gather_rows(const float* __restrict__ src, int64_t m, int g, const int32_t* __restrict__ perm,
+                              int64_t slot_row0, float* __restrict__ dst, int64_t ld)
+{
+    const int64_t i = blockIdx.x;
+    const int64_t s = slot_row0 + i;
+    const float* row = src + ((int64_t)perm[s / g] * g + s % g) * m;
+    for (int64_t c = threadIdx.x; c < ld; c += blockDim.x) dst[i * ld + c] = c < m ? row[c] : 0.f;
+}
+
+// dst (rows x ldd, zero padded) = src[0:rows, 0:cols] (lds)
+__global__ void k_copy_pad(const float* __restrict__ src, int64_t lds, int64_t rows, int64_t cols,
+                           float* __restrict__ dst, int64_t ldd)
+{
+    const int64_t i = blockIdx.x;
+    for (int64_t c = threadIdx.x; c < ldd; c += blockDim.x) dst[i * ldd + c] = c < cols ? src[i * lds + c] : 0.f;
+}
+
+// ---------------------------------------------------------------- blocked exchange inversion
+constexpr int NB = 64;
+
+// Inverse of the nb x nb pivot block A[p0:p0+nb, p0:p0+nb] by Cholesky in fp64 (one block).
+// Raises OSSCAR_E_NOTPD in ctl->status when a pivot is not positive.
+__global__ void __launch_bounds__(256)
+k_pivot_inverse(const float* __restrict__ A, int64_t lda, int64_t p0, int nb, float* __restrict__ Dinv, SearchCtl* ctl)
+{
+    extern __shared__ double sm[];
+    double* L = sm;                 // nb x nb, lower Cholesky factor, then its inverse
+    double* R = sm + NB * NB;       // result
+    const int t = threadIdx.x;
+    for (int idx = t; idx < nb * nb; idx += blockDim.x) {
+        int i = idx / nb, j = idx % nb;
+        // symmetrise: the two triangles can differ in the last bits
+        L[i * NB + j] = 0.5 * ((double)A[(p0 + i) * lda + p0 + j] + (double)A[(p0 + j) * lda + p0 + i]);
+    }
+    __syncthreads();
+    __shared__ int bad;
+    if (t == 0) bad = 0;
+    __syncthreads();
+    for (int j = 0; j < nb; ++j) {
+        if (t == 0) {
+            double d = L[j * NB + j];
+            if (!(d > 0.0)) { bad = 1; d = 1.0; }
+            L[j * NB + j] = sqrt(d);
+        }
+        __syncthreads();
+        const double djj = L[j * NB + j];
+        for (int i = j + 1 + t; i < nb; i += blockDim.x) L[i * NB + j] /= djj;
+        __syncthreads();
+        // trailing update of the lower triangle
+        const int rem = nb - j - 1;
+        for (int idx = t; idx < rem * rem; idx += blockDim.x) {
+            int i = j + 1 + idx / rem, c = j + 1 + idx % rem;
+            if (c <= i) L[i * NB + c] -= L[i * NB + j] * L[c * NB + j];
+        }
+        __syncthreads();
+    }
+    // R = L^-1 (lower): column by column forward substitution, one thread per column
+    for (int c = t; c < nb; c += blockDim.x) {
+        for (int i = 0; i < nb; ++i) {
+            double s = (i == c) ? 1.0 : 0.0;
+            for (int kx = c; kx < i; ++kx) s -= L[i * NB + kx] * R[kx * NB + c];
+            R[i * NB + c] = (i < c) ? 0.0 : s / L[i * NB + i];
+        }
+    }
+    __syncthreads();
+    // Dinv = R^T R
+    for (int idx = t; idx < nb * nb; idx += blockDim.x) {
+        int i = idx / nb, j = idx % nb;
+        double s = 0.0;
+        for (int kx = (i > j ? i : j); kx < nb; ++kx) s += R[kx * NB + i] * R[kx * NB + j];
+        Dinv[i * NB + j] = (float)s;
+    }
+    if (t == 0 && bad) ctl->status = OSSCAR_E_NOTPD;
+}
+
+// U = A[p0:p0+nb, 0:n) (copy of the pivot rows), and zero T's pivot rows afterwards is done in k_zero_rows.
+__global__ void k_copy_rows(const float* __restrict__ A, int64_t lda, int64_t p0, int nb, int64_t n,
+                            float* __restrict__ U, int64_t ldu)
+{
+    const int i = blockIdx.y;
+    if (i >= nb) return;
+    for (int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; c < n; c += (int64_t)gridDim.x * blockDim.x)
+        U[i * ldu + c] = A[(p0 + i) * lda + c];
+}
+__global__ void k_zero_rows(float* __restrict__ T, int64_t ldt, int64_t p0, int nb, int ncols)
+{
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx < nb * ncols) T[(p0 + idx / ncols) * ldt + idx % ncols] = 0.f;
+}
+// A[:, P] = T (rows outside P), A[P, :] = Un (columns outside P), A[P, P] = Dinv.
+__global__ void k_gj_writeback(float* __restrict__ A, int64_t lda, int64_t n, int64_t p0, int nb,
+                               const float* __restrict__ T, int64_t ldt, const float* __restrict__ Un, int64_t ldu,
+                               const float* __restrict__ Dinv)
+{
+    const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= n * nb) return;
+    {   // column panel: element (row, p0 + j)
+        const int64_t row = idx / nb; const int j = (int)(idx % nb);
+        if (row < p0 || row >= p0 + nb) A[row * lda + p0 + j] = T[row * ldt + j];
+    }
+    {   // row panel: element (p0 + i, col)
+        const int i = (int)(idx / n); const int64_t col = idx % n;
+        float v;
+        if (col >= p0 && col < p0 + nb) v = Dinv[i * NB + (col - p0)];
+        else v = Un[i * ldu + col];
+        A[(p0 + i) * lda + col] = v;
+    }
+}
+
+// c_t[a][b] = Hp[J_ta][J_tb] - sum_s Pm[ta][s] * Hp[J_tb][s]  for pruned slot t; one block per t.
+__global__ void k_schur(const float* __restrict__ Hp, int64_t ldp, const float* __restrict__ Pm, int64_t ldpm,
+                        int64_t nI, int g, double* __restrict__ c)
+{
+    const int64_t t = blockIdx.x;
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    for (int pair = w; pair < g * g; pair += nw) {
+        const int a = pair / g, b = pair % g;
+        const float* pr = Pm + (t * g + a) * ldpm;
+        const float* hr = Hp + (nI + t * g + b) * ldp;
+        double s = 0.0;
+        for (int64_t x = lane; x < nI; x += 32) s += (double)pr[x] * (double)hr[x];
+        s = warp_sum(s);
+        if (lane == 0) c[(t * g + a) * g + b] = (double)Hp[(nI + t * g + a) * ldp + nI + t * g + b] - s;
+    }
+}
+
+__global__ void k_trace_product(const float* __restrict__ A, int64_t lda, const float* __restrict__ B, int64_t ldb,
+                                int64_t rows, int64_t cols, double* __restrict__ out)
+{
+    double acc = 0.0;
+    for (int64_t r = blockIdx.x; r < rows; r += gridDim.x)
+        for (int64_t c = threadIdx.x; c < cols; c += blockDim.x)
+            acc += (double)A[r * lda + c] * (double)B[r * ldb + c];
+    acc = block_sum(acc);
+    if (threadIdx.x == 0) atomicAdd(out, acc);
+}
+
+__global__ void k_set_obj(SearchCtl* ctl)   // obj = const - Tr(G_I^T V), with acc[0] = const, acc[1] = trace
+{
+    ctl->const_term = ctl->acc[0];
+    ctl->obj = ctl->acc[0] - ctl->acc[1];
+}
+
+#define CK(x) do { cudaError_t e_ = (x); if (e_ != cudaSuccess) return OSSCAR_E_CUDA; } while (0)
+
+}  // namespace
+
+cudaError_t gather_rows(cudaStream_t st, const float* src, int64_t m, int g, const int32_t* perm,
+                        int64_t slot_row0, int64_t nrows, float* dst, int64_t ld)
+{
+    if (nrows > 0) k_gather_rows<<<(unsigned)nrows, 256, 0, st>>>(src, m, g, perm, slot_row0, dst, ld);
+    return cudaGetLastError();
+}
+
+cudaError_t trace_product(cudaStream_t st, const float* A, int64_t lda, const float* B, int64_t ldb,
+                          int64_t rows, int64_t cols, double* out_dev)
+{
+    cudaError_t e = cudaMemsetAsync(out_dev, 0, sizeof(double), st);
+    if (e != cudaSuccess) return e;
+    if (rows > 0 && cols > 0) {
+        int grid = (int)(rows < 1184 ? rows : 1184);
+        k_trace_product<<<grid, 256, 0, st>>>(A, lda, B, ldb, rows, cols, out_dev);
+    }
+    return cudaGetLastError();
+}
+
+int make_layout(int64_t d1, int64_t m, int32_t g, int32_t k, Layout* L)
+{
+    if (d1 <= 0 || m <= 0 || g <= 0 || g > OSSCAR_MAX_GROUP || d1 % g != 0) return OSSCAR_E_SHAPE;
+    const int64_t ng = d1 / g;
+    if (k < 1 || k > ng) return OSSCAR_E_SHAPE;
+    L->d1 = d1; L->m = m; L->ng = ng; L->g = g; L->k = k;
+    L->nI = (int64_t)k * g; L->nJ = d1 - L->nI;
+    L->ldp = round_up(d1, kPadF); L->ldh = round_up(L->nI, kPadF); L->ldm = round_up(m, kPadF);
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off += (bytes + 255) / 256 * 256; return o; };
+    const int64_t nI = L->nI, nJ = L->nJ, ldh = L->ldh, ldm = L->ldm;
+    // `big` first: osscar_objective uses the start of the workspace as 2 * d1 * ldm floats
+    int64_t big = nI * ldm;
+    if (nJ * ldh > big) big = nJ * ldh;
+    if (2 * d1 * ldm > big) big = 2 * d1 * ldm;
+    L->off_big = take(sizeof(float) * big);
+    L->off_Hp = take(sizeof(float) * d1 * L->ldp);
+    L->off_Hinv = take(sizeof(float) * nI * ldh);
+    L->off_V = take(sizeof(float) * nI * ldm);
+    L->off_R = take(sizeof(float) * (nJ > 0 ? nJ : 1) * ldm);
+    L->off_y = take(sizeof(float) * ldh * g);
+    L->off_vec_begin = L->off_y;
+    L->off_b = take(sizeof(float) * ldh * g);
+    L->off_u2 = take(sizeof(float) * ldh * g);
+    L->off_bC = take(sizeof(float) * ldh * g);
+    L->off_u2c = take(sizeof(float) * ldh * g);
+    L->off_u = take(sizeof(float) * (nJ + g) * g);
+    L->off_d = take(sizeof(float) * (nJ + g) * g);
+    L->off_K = take(sizeof(float) * g * ldm);
+    L->off_Vq = take(sizeof(float) * g * ldm);
+    L->off_vec_end = off;
+    L->off_vnorm = take(sizeof(float) * nI);
+    L->off_rnorm = take(sizeof(float) * (nJ > 0 ? nJ : 1));
+    L->off_D = take(sizeof(double) * k);
+    L->off_A = take(sizeof(double) * (ng - k > 0 ? ng - k : 1));
+    L->off_c = take(sizeof(double) * (ng - k > 0 ? ng - k : 1) * g * g);
+    L->off_small = take(sizeof(double) * 16 * g * g + 256);
+    L->off_gramV = take(sizeof(double) * k * g * g);
+    L->off_gramR = take(sizeof(double) * (ng - k > 0 ? ng - k : 1) * g * g);
+    L->off_perm = take(sizeof(int32_t) * ng);
+    L->off_slotof = take(sizeof(int32_t) * ng);
+    L->off_energy = take(sizeof(double) * ng + sizeof(int32_t) * ng);
+    L->off_panel = take(sizeof(float) * (nI * NB + 2 * NB * ldh + NB * NB));
+    L->bytes = off;
+    return OSSCAR_OK;
+}
+
+int select_support(osscar_ctx* ctx, int mode, int32_t* support)
+{
+    const Layout& L = ctx->L;
+    cudaStream_t st = ctx->stream;
+    char* ws = (char*)ctx->ws;
+    double* e = (double*)(ws + L.off_energy);
+    int32_t* kept = (int32_t*)(e + L.ng);
+    int32_t* perm = (int32_t*)(ws + L.off_perm);
+    int32_t* slotof = (int32_t*)(ws + L.off_slotof);
+    const int nb = (int)((L.ng + 255) / 256);
+    if (mode == OSSCAR_INIT_USER) {
+        CK(cudaMemsetAsync(kept, 0, sizeof(int32_t) * L.ng, st));
+        k_user_support<<<(L.k + 255) / 256, 256, 0, st>>>(support, L.k, L.ng, kept, ctx->ctl);
+    } else {
+        k_energy<<<(unsigned)L.ng, 128, 0, st>>>(ctx->H, ctx->W, L.d1, L.m, L.g, mode, e);
+        k_rank_select<<<nb, 256, 0, st>>>(e, L.ng, L.k, kept);
+    }
+    k_build_perm<<<nb, 256, 0, st>>>(kept, L.ng, L.k, perm, slotof, support);
+    CK(cudaGetLastError());
+    return OSSCAR_OK;
+}
+
+// Rebuilds every piece of the search state from H, G and the current slot permutation.
+// With `guarded`, the kernels that can be skipped return at once when the loop has stopped.
+int build_state(osscar_ctx* ctx, bool guarded)
+{
+    const Layout& L = ctx->L;
+    cudaStream_t st = ctx->stream;
+    char* ws = (char*)ctx->ws;
+    float* Hp = (float*)(ws + L.off_Hp);
+    float* Hinv = (float*)(ws + L.off_Hinv);
+    float* V = (float*)(ws + L.off_V);
+    float* R = (float*)(ws + L.off_R);
+    float* big = (float*)(ws + L.off_big);
+    double* c = (double*)(ws + L.off_c);
+    const int32_t* perm = (const int32_t*)(ws + L.off_perm);
+    float* T = (float*)(ws + L.off_panel);
+    float* U = T + L.nI * NB;
+    float* Un = U + NB * L.ldh;
+    float* Dinv = Un + NB * L.ldh;
+    const int32_t* done = guarded ? &ctx->ctl->done : nullptr;
+    const int64_t nI = L.nI, nJ = L.nJ;
+
+    {   // slot-permuted copy of H
+        dim3 grid((unsigned)L.d1, (unsigned)((L.ldp + 255) / 256 < 64 ? (L.ldp + 255) / 256 : 64));
+        k_gather_sym<<<grid, 256, 0, st>>>(ctx->H, L.d1, L.g, perm, Hp, L.ldp);
+    }
+    CK(cudaMemsetAsync(ws + L.off_vec_begin, 0, L.off_vec_end - L.off_vec_begin, st));
+    k_copy_pad<<<(unsigned)nI, 256, 0, st>>>(Hp, L.ldp, nI, nI, Hinv, L.ldh);
+    CK(cudaGetLastError());
+    CK(cudaFuncSetAttribute(k_pivot_inverse, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * NB * NB * (int)sizeof(double)));
+    for (int64_t p0 = 0; p0 < nI; p0 += NB) {
+        const int nb = (int)(nI - p0 < NB ? nI - p0 : NB);
+        k_pivot_inverse<<<1, 256, 2 * NB * NB * sizeof(double), st>>>(Hinv, L.ldh, p0, nb, Dinv, ctx->ctl);
+        // T = A[:, P] * Dinv
+        CK(sgemm(st, false, false, nI, nb, nb, 1.f, Hinv + p0, L.ldh, Dinv, NB, 0.f, T, NB, done));
+        k_zero_rows<<<(nb * nb + 255) / 256, 256, 0, st>>>(T, NB, p0, nb, nb);
+        {
+            dim3 grid((unsigned)((nI + 255) / 256 < 32 ? (nI + 255) / 256 : 32), (unsigned)nb);
+            k_copy_rows<<<grid, 256, 0, st>>>(Hinv, L.ldh, p0, nb, nI, U, L.ldh);
+        }
+        CK(sgemm(st, false, false, nb, nI, nb, -1.f, Dinv, NB, U, L.ldh, 0.f, Un, L.ldh, done));
+        CK(sgemm(st, false, false, nI, nI, nb, -1.f, T, NB, U, L.ldh, 1.f, Hinv, L.ldh, done));
+        k_gj_writeback<<<(unsigned)((nI * nb + 255) / 256), 256, 0, st>>>(Hinv, L.ldh, nI, p0, nb, T, NB, Un, L.ldh, Dinv);
+    }
+    CK(cudaGetLastError());
+    // V = Hinv * G_I
+    k_gather_rows<<<(unsigned)nI, 256, 0, st>>>(ctx->G, L.m, L.g, perm, 0, big, L.ldm);
+    CK(sgemm(st, false, false, nI, L.m, nI, 1.f, Hinv, L.ldh, big, L.ldm, 0.f, V, L.ldm, done));
+    // obj = Tr(W^T G) - Tr(G_I^T V)
+    CK(trace_product(st, ctx->W, L.m, ctx->G, L.m, L.d1, L.m, &ctx->ctl->acc[0]));
+    CK(trace_product(st, big, L.ldm, V, L.ldm, nI, L.m, &ctx->ctl->acc[1]));
+    k_set_obj<<<1, 1, 0, st>>>(ctx->ctl);
+    if (nJ > 0) {
+        // R_J = G_J - Hp[J, I] V
+        k_gather_rows<<<(unsigned)nJ, 256, 0, st>>>(ctx->G, L.m, L.g, perm, nI, R, L.ldm);
+        CK(sgemm(st, false, false, nJ, L.m, nI, -1.f, Hp + nI * L.ldp, L.ldp, V, L.ldm, 1.f, R, L.ldm, done));
+        // Pm = Hp[J, I] Hinv, then the Schur complements
+        CK(sgemm(st, false, false, nJ, nI, nI, 1.f, Hp + nI * L.ldp, L.ldp, Hinv, L.ldh, 0.f, big, L.ldh, done));
+        k_schur<<<(unsigned)(L.ng - L.k), 256, 0, st>>>(Hp, L.ldp, big, L.ldh, nI, L.g, c);
+    }
+    CK(cudaGetLastError());
+    return OSSCAR_OK;
+}
+
+}  // namespace osscar

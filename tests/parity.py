@@ -1,0 +1,72 @@
+"""Shared helpers of the GPU parity tests: oracle problems and the step-by-step comparison of a
+GPU swap trace with the fp64 oracle (re-basing the oracle at non-decisive steps)."""
+import numpy as np
+import torch
+
+import workloads
+from oracle import osscar_oracle as orc
+
+GAP = 1e-5      # relative best-vs-second-best gap above which the oracle's choice is binding
+
+
+def oracle_problem(wl):
+    chunks = [c.float().numpy().astype(np.float64) for c in wl.x_chunks()]
+    W = wl.weight().numpy().astype(np.float64)
+    H, G, const = orc.gram_chunked(chunks, W, wl.damp)
+    return chunks, W, H, G, const
+
+
+def follow_trace(H, G, const, g, S0, swaps, gpu_obj, score_mode="independent", accept="improving",
+                 mode="lowrank", max_swaps=None, gpu_stop=None, obj_rtol=1e-4):
+    """Walks the GPU's swap sequence with the oracle.  Returns (search, n_rebased).
+
+    At each step the oracle proposes its swap from its own fp64 state.  If the GPU made the same
+    swap, fine.  Otherwise the step must be non-decisive for the oracle (runner-up within GAP) and
+    the GPU's choice must itself be within GAP of the oracle's best scores; the oracle is then moved
+    to the GPU's support and the walk continues.  The running objective must agree throughout.
+    """
+    srch = orc.Search(H, G, const, g, S0, mode=mode, score_mode=score_mode, accept=accept)
+    rebased = 0
+    assert gpu_obj[0] == __import__("pytest").approx(srch.st.obj, rel=obj_rtol)
+    for step, (i_out, j_in) in enumerate(swaps):
+        info = srch.propose(keep_scores=True)
+        assert info is not None, f"step {step}: oracle has no candidate"
+        slot = int(np.nonzero(srch.st.S == i_out)[0][0]) if i_out in srch.st.S else None
+        assert slot is not None and j_in in srch.st.c, f"step {step}: GPU swap ({i_out},{j_in}) not possible"
+        if (info.i_out, info.j_in) != (i_out, j_in):
+            if score_mode == "independent":
+                Dbest, Abest = info.D[info.slot], info.A[info.j_in]
+                ok_out = info.D[slot] <= Dbest * (1 + GAP) + 1e-300
+                ok_in = info.A[j_in] >= Abest * (1 - GAP) - 1e-300
+                assert ok_out and ok_in, (
+                    f"step {step}: GPU ({i_out},{j_in}) vs oracle ({info.i_out},{info.j_in}); "
+                    f"D {info.D[slot]:.9g} vs {Dbest:.9g}, A {info.A[j_in]:.9g} vs {Abest:.9g}")
+            else:
+                pruned = np.array(sorted(srch.st.c.keys()))
+                dgpu = info.pair_delta[slot, int(np.nonzero(pruned == j_in)[0][0])]
+                assert abs(dgpu - info.delta) <= GAP * abs(info.delta), f"step {step}: pair not admissible"
+            rebased += 1
+            delta = orc.swap_delta_closed_form(srch.H, srch.st, g, slot, j_in)
+        else:
+            delta = info.delta
+        if accept == "improving":
+            # the GPU accepted this swap: the oracle must agree unless the margin is tiny
+            thr = -srch.eps_acc * srch.st.obj
+            assert delta <= thr or abs(delta - thr) <= GAP * srch.st.obj, f"step {step}: accepted a non-improving swap"
+        srch.apply(slot, j_in)
+        assert gpu_obj[step + 1] == __import__("pytest").approx(srch.st.obj, rel=obj_rtol), f"step {step}: objective drifted"
+    # after the GPU's last swap: it either hit max_swaps or stopped because the next swap did not improve
+    if gpu_stop == "no_improvement":
+        info = srch.propose(keep_scores=True)
+        if info is not None and info.accepted:
+            near_tie = info.gap_out <= GAP or info.gap_in <= GAP
+            assert info.accept_margin <= GAP or near_tie, \
+                f"GPU stopped but the oracle would go on (delta {info.delta}, obj {srch.st.obj})"
+    elif gpu_stop == "max_swaps":
+        assert len(swaps) == max_swaps
+    return srch, rebased
+
+
+def rel_fro(a, b):
+    a = np.asarray(a, np.float64); b = np.asarray(b, np.float64)
+    return float(np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-300))

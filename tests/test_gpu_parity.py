@@ -1,0 +1,292 @@
+"""Parity of the CUDA path (through the C ABI) with the fp64 CPU oracle.  Needs a B200."""
+import numpy as np
+import pytest
+import torch
+
+import workloads
+from oracle import osscar_oracle as orc
+from tests.parity import GAP, follow_trace, oracle_problem, rel_fro
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def osscar():
+    import paper_2403_12983_b200 as pkg
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    pkg.lib()          # fails loudly if libosscar.so cannot be built / loaded
+    return pkg
+
+
+@pytest.fixture()
+def solver(osscar):
+    s = osscar.Solver()
+    yield s
+    s.close()
+
+
+def dev(x, dtype=torch.float32):
+    return torch.as_tensor(np.ascontiguousarray(x), dtype=dtype).cuda()
+
+
+# ------------------------------------------------------------------------------------ Gram
+GRAM_CASES = [
+    # name, overrides: several 128x256 tiles, ragged column tail, token count not a multiple of 64
+    ("c2", dict(n=1000, d1=840, m=72, k=400, chunk_rows=384)),
+    ("c5", dict(n=700, d1=264, m=40, k=80, chunk_rows=700)),
+    ("c3", dict(n=2100, d1=8 * 80, m=96, g=80, k=4, chunk_rows=1024)),
+    ("c2", dict(n=130, d1=8, m=3, k=4, chunk_rows=64)),
+]
+
+
+@pytest.mark.parametrize("name,over", GRAM_CASES)
+def test_gram_bf16_tensor_core(solver, name, over):
+    wl = workloads.config(name, **over)
+    chunks, W, H64, G64, const64 = oracle_problem(wl)
+    H, G, const = solver.gram([c.cuda() for c in wl.x_chunks()], wl.weight().cuda(), wl.damp)
+    Hg, Gg = H.cpu().numpy().astype(np.float64), G.cpu().numpy().astype(np.float64)
+    scale = np.sqrt(np.outer(np.diag(H64), np.diag(H64)))
+    # bf16 products are exact in fp32; only the fp32 accumulation order differs from the fp64 sum
+    assert np.max(np.abs(Hg - H64) / scale) < 2e-6
+    assert np.array_equal(Hg, Hg.T)
+    gs = np.linalg.norm(G64, axis=1, keepdims=True) + 1e-300
+    assert np.max(np.abs(Gg - G64) / gs) < 1e-5
+    assert const == pytest.approx(const64, rel=1e-5)
+
+
+@pytest.mark.parametrize("name,over", [("c1", {}), ("c4", dict(n=49 * 12, d1=9 * 37, m=50, k=12, chunk_rows=49 * 5))])
+def test_gram_fp32(solver, name, over):
+    wl = workloads.config(name, **over)
+    chunks, W, H64, G64, const64 = oracle_problem(wl)
+    H, G, const = solver.gram([c.cuda() for c in wl.x_chunks()], wl.weight().cuda(), wl.damp)
+    Hg = H.cpu().numpy().astype(np.float64)
+    scale = np.sqrt(np.outer(np.diag(H64), np.diag(H64)))
+    assert np.max(np.abs(Hg - H64) / scale) < 5e-6
+    assert np.array_equal(Hg, Hg.T)
+    assert rel_fro(G.cpu().numpy(), G64) < 1e-5
+    assert const == pytest.approx(const64, rel=1e-5)
+
+
+def test_gram_empty_and_single_chunk_flags(solver, osscar):
+    wl = workloads.config("c2", n=256, d1=64, m=8, k=32, chunk_rows=256)
+    X = wl.x_chunk(0).cuda(); W = wl.weight().cuda()
+    H = torch.full((64, 64), 7.0, device="cuda"); G = torch.empty(64, 8, device="cuda")
+    b = osscar.binding
+    # an empty first block clears H, the data then accumulates, END mirrors and builds G
+    solver.gram_chunk(X[:0], H, b.GRAM_BEGIN)
+    solver.gram_chunk(X, H, 0)
+    const = solver.gram_chunk(X[:0], H, b.GRAM_END, W, G, 0.0)
+    H2, G2, const2 = solver.gram([X], W, 0.0)
+    assert torch.equal(H, H2) and torch.equal(G, G2) and const == const2
+
+
+# ------------------------------------------------------------------------------------ state after init
+STATE_CASES = [
+    ("c1", {}, 0),
+    ("c2", dict(n=3000, d1=520, m=150, k=207, chunk_rows=2048), 0),
+    ("c5", dict(n=3000, d1=520, m=150, k=156, chunk_rows=2048), 1),
+    ("c4", dict(n=49 * 30, d1=9 * 70, m=100, k=33, chunk_rows=49 * 30), 0),
+    ("c3", dict(n=4096, d1=10 * 24, m=90, g=24, k=5, chunk_rows=4096), 2),
+]
+
+
+@pytest.mark.parametrize("name,over,seed", STATE_CASES)
+def test_init_support_and_state(solver, name, over, seed):
+    wl = workloads.config(name, seed=seed, **over)
+    chunks, W, H64, G64, const64 = oracle_problem(wl)
+    # feed the oracle's own H and G (rounded to fp32) so that only the state construction is compared
+    H, G, Wd = dev(H64), dev(G64), dev(W)
+    Hr, Gr = H.cpu().numpy().astype(np.float64), G.cpu().numpy().astype(np.float64)
+    const_r = float(np.sum(W * Gr))
+    S0, e = orc.init_support(Hr, W, wl.g, wl.k)
+    support, obj0 = solver.init_support(H, G, Wd, wl.g, wl.k)
+    assert np.array_equal(support.cpu().numpy(), S0)
+    st = orc.fresh_state(Hr, Gr, const_r, S0, wl.g)
+    perm = solver.debug_state(4).cpu().numpy()
+    assert np.array_equal(perm[:wl.k], S0) and np.array_equal(np.sort(perm), np.arange(wl.ngroups))
+    assert obj0 == pytest.approx(st.obj, rel=1e-5)
+    assert rel_fro(solver.debug_state(0).cpu().numpy(), st.Hinv) < 2e-5
+    assert rel_fro(solver.debug_state(1).cpu().numpy(), st.V) < 2e-5
+    rows_J = orc.rows_of(perm[wl.k:], wl.g)
+    assert rel_fro(solver.debug_state(2).cpu().numpy(), st.R[rows_J]) < 2e-5
+    c = solver.debug_state(3).cpu().numpy()
+    for t, q in enumerate(perm[wl.k:]):
+        assert np.allclose(c[t], st.c[int(q)], rtol=1e-4, atol=1e-5 * np.abs(st.c[int(q)]).max())
+    D, A = orc.drop_scores(st, wl.g), orc.add_scores(st, wl.g, wl.ngroups, Hr)
+    assert np.allclose(solver.debug_state(5).cpu().numpy(), D, rtol=1e-4)
+    assert np.allclose(solver.debug_state(6).cpu().numpy(), A[perm[wl.k:]], rtol=1e-4)
+
+
+def test_init_user_and_magnitude_modes(solver, osscar):
+    wl = workloads.config("c2", n=2048, d1=96, m=24, k=40, chunk_rows=2048)
+    chunks, W, H64, G64, const64 = oracle_problem(wl)
+    H, G, Wd = dev(H64), dev(G64), dev(W)
+    b = osscar.binding
+    Sm, _ = orc.init_support(H64, W, 1, 40, "magnitude")
+    s, _ = solver.init_support(H, G, Wd, 1, 40, mode=b.INIT_MAGNITUDE)
+    assert np.array_equal(s.cpu().numpy(), Sm)
+    user = np.array(sorted(np.random.default_rng(0).choice(96, 40, replace=False)))[::-1].copy()
+    s, obj = solver.init_support(H, G, Wd, 1, 40, mode=b.INIT_USER, support=torch.as_tensor(user))
+    assert np.array_equal(s.cpu().numpy(), np.sort(user))
+    assert obj == pytest.approx(orc.solve_support(H64, G64, const64, user, 1)[1], rel=1e-4)
+
+
+# ------------------------------------------------------------------------------------ search
+SEARCH_CASES = [
+    ("c1", {}, 0, 50),
+    ("c1", {}, 1, 50),
+    ("c1", {}, 2, 50),
+    ("c2", dict(n=8192, d1=1000, m=300, k=437, chunk_rows=4096), 0, 200),
+    ("c2", dict(n=4096, d1=520, m=150, k=207, chunk_rows=4096), 1, 200),
+    ("c5", dict(n=8192, d1=1000, m=300, k=300, chunk_rows=4096), 0, 200),
+    ("c5", dict(n=4096, d1=520, m=150, k=156, chunk_rows=4096), 2, 200),
+    ("c4", dict(n=49 * 40, d1=9 * 100, m=130, k=50, chunk_rows=49 * 40), 0, 100),
+    ("c4", dict(n=49 * 40, d1=9 * 100, m=130, k=50, chunk_rows=49 * 40), 1, 100),
+    ("c3", dict(n=8192, d1=12 * 40, m=200, g=40, k=6, chunk_rows=8192, score_mode="independent"), 0, 30),
+]
+
+
+def run_gpu_search(solver, wl, H, G, Wd, max_swaps, accept_always=False, S0=None):
+    import paper_2403_12983_b200.binding as b
+    if S0 is None:
+        support, obj0 = solver.init_support(H, G, Wd, wl.g, wl.k)
+    else:
+        support, obj0 = solver.init_support(H, G, Wd, wl.g, wl.k, mode=b.INIT_USER, support=torch.as_tensor(S0))
+    out = solver.local_search(max_swaps, accept_mode=b.ACCEPT_ALWAYS if accept_always else b.ACCEPT_IMPROVING)
+    return support.cpu().numpy(), obj0, out
+
+
+@pytest.mark.parametrize("name,over,seed,max_swaps", SEARCH_CASES)
+def test_search_matches_oracle_given_H(solver, name, over, seed, max_swaps):
+    """Search parity with H, G handed over from the oracle (fp32-rounded): isolates the swap loop."""
+    wl = workloads.config(name, seed=seed, **over)
+    chunks, W, H64, G64, const64 = oracle_problem(wl)
+    H, G, Wd = dev(H64), dev(G64), dev(W)
+    Hr, Gr = H.cpu().numpy().astype(np.float64), G.cpu().numpy().astype(np.float64)
+    const_r = float(np.sum(W * Gr))
+    S0, obj0, out = run_gpu_search(solver, wl, H, G, Wd, max_swaps)
+    S0o, _ = orc.init_support(Hr, W, wl.g, wl.k)
+    assert np.array_equal(S0, S0o)
+    swaps = [tuple(int(v) for v in r) for r in out.swap_trace.cpu().numpy()]
+    gobj = out.obj_trace.cpu().numpy()
+    srch, rebased = follow_trace(Hr, Gr, const_r, wl.g, S0, swaps, gobj, gpu_stop=out.stop_reason, max_swaps=max_swaps)
+    S_or, W_or, _, _ = srch.result()
+    assert np.array_equal(out.support.cpu().numpy(), S_or)                       # identical final support
+    assert np.all(np.diff(gobj) < 0)                                             # accepted swaps lower obj
+    assert out.obj_final == pytest.approx(srch.st.obj, rel=1e-4)
+    assert gobj[-1] == pytest.approx(out.obj_final, rel=1e-4)                    # running == recomputed
+    assert rel_fro(out.W.cpu().numpy(), W_or) < 1e-3
+    Wg = out.W.cpu().numpy()
+    pruned_rows = np.setdiff1d(np.arange(wl.d1), orc.rows_of(S_or, wl.g))
+    assert np.all(Wg[pruned_rows] == 0)
+    # state-independent cross-check of the objective through its own entry point
+    assert solver.objective(H, Wd, out.W) == pytest.approx(srch.st.obj, rel=2e-4)
+    assert len(swaps) >= 1
+
+
+@pytest.mark.parametrize("name,over,seed,max_swaps", [SEARCH_CASES[0], SEARCH_CASES[4], SEARCH_CASES[6], SEARCH_CASES[7]])
+def test_end_to_end_from_X(solver, name, over, seed, max_swaps):
+    """Whole path from X: Gram on the GPU, then init and search; compared with the oracle run from X."""
+    wl = workloads.config(name, seed=seed, **over)
+    chunks, W, H64, G64, const64 = oracle_problem(wl)
+    Wd = wl.weight().cuda()
+    H, G, const = solver.gram([c.cuda() for c in wl.x_chunks()], Wd, wl.damp)
+    S0, obj0, out = run_gpu_search(solver, wl, H, G, Wd, max_swaps)
+    S0o, e = orc.init_support(H64, W, wl.g, wl.k)
+    if not np.array_equal(S0, S0o):
+        # only groups whose energies tie within GAP at the selection boundary may differ
+        diff = np.setxor1d(S0, S0o)
+        thr = np.sort(e)[-wl.k]
+        assert np.all(np.abs(e[diff] - thr) <= GAP * thr)
+    swaps = [tuple(int(v) for v in r) for r in out.swap_trace.cpu().numpy()]
+    gobj = out.obj_trace.cpu().numpy()
+    srch, rebased = follow_trace(H64, G64, const64, wl.g, S0, swaps, gobj, gpu_stop=out.stop_reason, max_swaps=max_swaps)
+    S_or, W_or, _, _ = srch.result()
+    assert np.array_equal(out.support.cpu().numpy(), S_or)
+    assert out.obj_final == pytest.approx(srch.st.obj, rel=1e-4)
+    assert rel_fro(out.W.cpu().numpy(), W_or) < 1e-3
+
+
+def test_accept_always_runs_fixed_iterations_and_refresh(solver, osscar):
+    wl = workloads.config("c2", n=4096, d1=520, m=150, k=207, chunk_rows=4096)
+    chunks, W, H64, G64, const64 = oracle_problem(wl)
+    H, G, Wd = dev(H64), dev(G64), dev(W)
+    Hr, Gr = H.cpu().numpy().astype(np.float64), G.cpu().numpy().astype(np.float64)
+    const_r = float(np.sum(W * Gr))
+    b = osscar.binding
+    S0, obj0 = solver.init_support(H, G, Wd, 1, wl.k)
+    out = solver.local_search(40, accept_mode=b.ACCEPT_ALWAYS, refresh_every=16)
+    assert out.n_swaps == 40 and out.stop_reason == "max_swaps" and out.n_refresh == 2
+    swaps = [tuple(int(v) for v in r) for r in out.swap_trace.cpu().numpy()]
+    srch, _ = follow_trace(Hr, Gr, const_r, 1, S0.cpu().numpy(), swaps, out.obj_trace.cpu().numpy(),
+                           accept="always", gpu_stop="max_swaps", max_swaps=40)
+    assert np.array_equal(out.support.cpu().numpy(), srch.result()[0])
+    assert out.obj_final == pytest.approx(srch.st.obj, rel=1e-4)
+
+
+def test_state_after_search_is_consistent(solver):
+    """After many swaps the updated (H_II)^-1 is still the inverse and V, R match a fresh solve."""
+    wl = workloads.config("c5", n=4096, d1=520, m=150, k=156, chunk_rows=4096, seed=3)
+    chunks, W, H64, G64, const64 = oracle_problem(wl)
+    H, G, Wd = dev(H64), dev(G64), dev(W)
+    Hr, Gr = H.cpu().numpy().astype(np.float64), G.cpu().numpy().astype(np.float64)
+    import paper_2403_12983_b200.binding as b
+    solver.init_support(H, G, Wd, 1, wl.k)
+    out = solver.local_search(60, accept_mode=b.ACCEPT_ALWAYS)
+    perm = solver.debug_state(4).cpu().numpy()
+    I = perm[:wl.k]
+    Hinv = solver.debug_state(0).cpu().numpy().astype(np.float64)
+    assert np.abs(Hinv @ Hr[np.ix_(I, I)] - np.eye(wl.k)).max() < 1e-3
+    st = orc.fresh_state(Hr, Gr, float(np.sum(W * Gr)), I, 1)
+    assert rel_fro(solver.debug_state(1).cpu().numpy(), st.V) < 1e-4
+    assert rel_fro(solver.debug_state(2).cpu().numpy(), st.R[perm[wl.k:]]) < 1e-4
+    c = solver.debug_state(3).cpu().numpy().reshape(-1)
+    assert np.allclose(c, [st.c[int(q)][0, 0] for q in perm[wl.k:]], rtol=1e-3)
+
+
+# ------------------------------------------------------------------------------------ edge cases and errors
+def test_edge_cases(solver, osscar):
+    b = osscar.binding
+    wl = workloads.config("c2", n=1024, d1=64, m=16, k=64, chunk_rows=1024)
+    chunks, W, H64, G64, const64 = oracle_problem(wl)
+    H, G, Wd = dev(H64), dev(G64), dev(W)
+    # every group kept: nothing to swap, the dense weights come back and obj is ~0
+    S, obj0 = solver.init_support(H, G, Wd, 1, 64)
+    out = solver.local_search(10)
+    assert out.n_swaps == 0 and np.array_equal(out.support.cpu().numpy(), np.arange(64))
+    assert rel_fro(out.W.cpu().numpy(), W) < 1e-4 and abs(out.obj_final) < 1e-4 * const64
+    # a single kept group and max_swaps = 0
+    S, obj0 = solver.init_support(H, G, Wd, 1, 1)
+    out = solver.local_search(0)
+    assert out.n_swaps == 0 and out.stop_reason == "max_swaps"
+    assert obj0 == pytest.approx(orc.solve_support(H64, G64, const64, S.cpu().numpy(), 1)[1], rel=1e-5)
+
+
+def test_errors_are_reported_not_raised_on_device(solver, osscar):
+    b = osscar.binding
+    wl = workloads.config("c2", n=512, d1=64, m=16, k=32, chunk_rows=512)
+    chunks, W, H64, G64, const64 = oracle_problem(wl)
+    H, G, Wd = dev(H64), dev(G64), dev(W)
+    with pytest.raises(osscar.OsscarError) as ei:
+        solver.init_support(H, G, Wd, 5, 3)                 # 64 % 5 != 0
+    assert ei.value.status == b.E_SHAPE
+    with pytest.raises(osscar.OsscarError) as ei:
+        solver.init_support(H, G, Wd, 1, 65)                # k > groups
+    assert ei.value.status == b.E_SHAPE
+    fresh = osscar.Solver()
+    with pytest.raises(osscar.OsscarError) as ei:
+        fresh._shape = (64, 16, 1, 32); fresh._keep = [H, G, Wd]
+        fresh.local_search(5)                                # no state yet
+    assert ei.value.status == b.E_STATE
+    fresh.close()
+    # duplicated column -> H_II singular -> E_NOTPD, and the context stays usable afterwards
+    Hs = H64.copy(); Hs[:, 1] = Hs[:, 0]; Hs[1, :] = Hs[0, :]
+    user = torch.arange(32, dtype=torch.int32)
+    with pytest.raises(osscar.OsscarError) as ei:
+        solver.init_support(dev(Hs), G, Wd, 1, 32, mode=b.INIT_USER, support=user)
+    assert ei.value.status == b.E_NOTPD
+    S, obj0 = solver.init_support(H, G, Wd, 1, 32)
+    assert obj0 > 0
+    with pytest.raises(osscar.OsscarError) as ei:
+        solver.init_support(H, G, Wd, 1, 32, mode=b.INIT_USER, support=torch.zeros(32, dtype=torch.int32))
+    assert ei.value.status == b.E_ARG
