@@ -75,6 +75,7 @@ int osscar_create(osscar_ctx** out, int device, void* cuda_stream)
     ctx->stream = (cudaStream_t)cuda_stream;
     bool ok = cudaMalloc((void**)&ctx->ctl, sizeof(SearchCtl)) == cudaSuccess
            && cudaMemset(ctx->ctl, 0, sizeof(SearchCtl)) == cudaSuccess
+           && cudaMalloc((void**)&ctx->partials, sizeof(double) * kTracePartials) == cudaSuccess
            && cudaHostAlloc((void**)&ctx->ctl_host, sizeof(SearchCtl), cudaHostAllocDefault) == cudaSuccess
            && cudaHostAlloc((void**)&ctx->done_flag_host, 64, cudaHostAllocMapped) == cudaSuccess
            && cudaHostGetDevicePointer((void**)&ctx->done_flag_dev, (void*)ctx->done_flag_host, 0) == cudaSuccess
@@ -90,6 +91,7 @@ int osscar_destroy(osscar_ctx* ctx)
     if (!ctx) return OSSCAR_E_ARG;
     DeviceGuard guard(ctx->device);
     if (ctx->ctl) cudaFree(ctx->ctl);
+    if (ctx->partials) cudaFree(ctx->partials);
     if (ctx->ctl_host) cudaFreeHost(ctx->ctl_host);
     if (ctx->done_flag_host) cudaFreeHost((void*)ctx->done_flag_host);
     if (ctx->ev0) cudaEventDestroy(ctx->ev0);
@@ -153,7 +155,7 @@ int osscar_gram(osscar_ctx* ctx, const void* X, int x_dtype, int64_t n_rows, int
         k_add_damp<<<64, 256, 0, st>>>(H, d1, damp, &ctx->ctl->acc[0]);
     }
     CKC(sgemm(st, false, false, d1, m, d1, 1.f, H, d1, W, m, 0.f, G, m));
-    CKC(trace_product(st, W, m, G, m, d1, m, &ctx->ctl->acc[1]));
+    CKC(trace_product(st, W, m, G, m, d1, m, ctx->partials, &ctx->ctl->acc[1]));
     CKC(cudaMemcpyAsync(ctx->ctl_host, ctx->ctl, sizeof(SearchCtl), cudaMemcpyDeviceToHost, st));
     CKC(cudaStreamSynchronize(st));
     if (ctx->ctl_host->status != OSSCAR_OK) return ctx->ctl_host->status;
@@ -220,7 +222,7 @@ int osscar_objective(osscar_ctx* ctx, const float* H, const float* W, const floa
     float* HE = E + d1 * m;
     k_sub<<<1184, 256, 0, st>>>(W, Wt, E, d1 * m);
     CKC(sgemm(st, false, false, d1, m, d1, 1.f, H, d1, E, m, 0.f, HE, m));
-    CKC(trace_product(st, E, m, HE, m, d1, m, &ctx->ctl->acc[0]));
+    CKC(trace_product(st, E, m, HE, m, d1, m, ctx->partials, &ctx->ctl->acc[0]));
     CKC(cudaMemcpyAsync(ctx->ctl_host, ctx->ctl, sizeof(SearchCtl), cudaMemcpyDeviceToHost, st));
     CKC(cudaStreamSynchronize(st));
     *obj = ctx->ctl_host->acc[0];

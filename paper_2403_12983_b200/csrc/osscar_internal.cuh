@@ -7,6 +7,7 @@
 
 namespace osscar {
 
+constexpr int kTracePartials = 1184;   // blocks of a trace reduction; the context owns that many doubles
 constexpr int kPadF = 32;   // leading dimensions of internal fp32 matrices are padded to this many floats
 
 static inline int64_t round_up(int64_t x, int64_t a) { return (x + a - 1) / a * a; }
@@ -53,6 +54,7 @@ struct osscar_ctx {
     cudaStream_t stream;
     osscar::SearchCtl* ctl;          // device
     osscar::SearchCtl* ctl_host;     // pinned mirror
+    double* partials;                // device, kTracePartials doubles: stage 1 of deterministic reductions
     volatile int32_t* done_flag_host; // pinned, device-mapped: copy of ctl->done pushed by the device
     int32_t* done_flag_dev;          // device alias of done_flag_host
     void* ws;
@@ -86,7 +88,7 @@ int build_state(osscar_ctx* ctx, bool guarded);
 cudaError_t gather_rows(cudaStream_t st, const float* src, int64_t m, int g, const int32_t* perm,
                         int64_t slot_row0, int64_t nrows, float* dst, int64_t ld);
 cudaError_t trace_product(cudaStream_t st, const float* A, int64_t lda, const float* B, int64_t ldb,
-                          int64_t rows, int64_t cols, double* out_dev);   // *out = sum A.*B
+                          int64_t rows, int64_t cols, double* partials, double* out_dev);   // *out = sum A.*B
 
 // ---- search.cu -------------------------------------------------------------------------------
 int run_search(osscar_ctx* ctx, const osscar_search_params* p, int32_t* support_out, float* W_out,

@@ -785,7 +785,7 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
         float* big = (float*)((char*)ctx->ws + L.off_big);
         // G_I in slot order, then Tr(G_I^T V)
         CK(gather_rows(st, ctx->G, L.m, L.g, p.perm, 0, L.nI, big, L.ldm));
-        CK(trace_product(st, big, L.ldm, p.V, L.ldm, L.nI, L.m, &ctx->ctl->acc[1]));
+        CK(trace_product(st, big, L.ldm, p.V, L.ldm, L.nI, L.m, ctx->partials, &ctx->ctl->acc[1]));
         k_final_obj<<<1, 1, 0, st>>>(ctx->ctl);
     }
     CK(cudaGetLastError());

@@ -12,11 +12,6 @@ __device__ __forceinline__ double warp_sum(double v) {
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
     return v;
 }
-__device__ __forceinline__ float warp_sum(float v) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-    return v;
-}
 // Block-wide sum (blockDim.x multiple of 32, <= 1024); result valid in thread 0.
 __device__ double block_sum(double v) {
     __shared__ double red[32];
@@ -130,11 +125,13 @@ __global__ void k_copy_pad(const float* __restrict__ src, int64_t lds, int64_t r
 
 // ---------------------------------------------------------------- blocked exchange inversion
 constexpr int NB = 64;
+constexpr double kPivotRelTol = 1e-7;
 
 // Inverse of the nb x nb pivot block A[p0:p0+nb, p0:p0+nb] by Cholesky in fp64 (one block).
 // Raises OSSCAR_E_NOTPD in ctl->status when a pivot is not positive.
 __global__ void __launch_bounds__(256)
-k_pivot_inverse(const float* __restrict__ A, int64_t lda, int64_t p0, int nb, float* __restrict__ Dinv, SearchCtl* ctl)
+k_pivot_inverse(const float* __restrict__ A, int64_t lda, int64_t p0, int nb, float* __restrict__ Dinv,
+                const float* __restrict__ Hp, int64_t ldp, SearchCtl* ctl)
 {
     extern __shared__ double sm[];
     double* L = sm;                 // nb x nb, lower Cholesky factor, then its inverse
@@ -152,7 +149,8 @@ k_pivot_inverse(const float* __restrict__ A, int64_t lda, int64_t p0, int nb, fl
     for (int j = 0; j < nb; ++j) {
         if (t == 0) {
             double d = L[j * NB + j];
-            if (!(d > 0.0)) { bad = 1; d = 1.0; }
+            // a pivot that fp32 data cannot tell from zero counts as not positive
+            if (!(d > kPivotRelTol * (double)Hp[(p0 + j) * ldp + p0 + j])) { bad = 1; d = 1.0; }
             L[j * NB + j] = sqrt(d);
         }
         __syncthreads();
@@ -237,15 +235,23 @@ __global__ void k_schur(const float* __restrict__ Hp, int64_t ldp, const float* 
     }
 }
 
+// Two deterministic stages: per-block partial sums, then one block adds them in a fixed order.
 __global__ void k_trace_product(const float* __restrict__ A, int64_t lda, const float* __restrict__ B, int64_t ldb,
-                                int64_t rows, int64_t cols, double* __restrict__ out)
+                                int64_t rows, int64_t cols, double* __restrict__ partial)
 {
     double acc = 0.0;
     for (int64_t r = blockIdx.x; r < rows; r += gridDim.x)
         for (int64_t c = threadIdx.x; c < cols; c += blockDim.x)
             acc += (double)A[r * lda + c] * (double)B[r * ldb + c];
     acc = block_sum(acc);
-    if (threadIdx.x == 0) atomicAdd(out, acc);
+    if (threadIdx.x == 0) partial[blockIdx.x] = acc;
+}
+__global__ void k_sum_partials(const double* __restrict__ partial, int n, double* __restrict__ out)
+{
+    double acc = 0.0;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) acc += partial[i];
+    acc = block_sum(acc);
+    if (threadIdx.x == 0) *out = acc;
 }
 
 __global__ void k_set_obj(SearchCtl* ctl)   // obj = const - Tr(G_I^T V), with acc[0] = const, acc[1] = trace
@@ -266,14 +272,12 @@ cudaError_t gather_rows(cudaStream_t st, const float* src, int64_t m, int g, con
 }
 
 cudaError_t trace_product(cudaStream_t st, const float* A, int64_t lda, const float* B, int64_t ldb,
-                          int64_t rows, int64_t cols, double* out_dev)
+                          int64_t rows, int64_t cols, double* partials, double* out_dev)
 {
-    cudaError_t e = cudaMemsetAsync(out_dev, 0, sizeof(double), st);
-    if (e != cudaSuccess) return e;
-    if (rows > 0 && cols > 0) {
-        int grid = (int)(rows < 1184 ? rows : 1184);
-        k_trace_product<<<grid, 256, 0, st>>>(A, lda, B, ldb, rows, cols, out_dev);
-    }
+    if (rows <= 0 || cols <= 0) return cudaMemsetAsync(out_dev, 0, sizeof(double), st);
+    const int grid = (int)(rows < kTracePartials ? rows : kTracePartials);
+    k_trace_product<<<grid, 256, 0, st>>>(A, lda, B, ldb, rows, cols, partials);
+    k_sum_partials<<<1, 256, 0, st>>>(partials, grid, out_dev);
     return cudaGetLastError();
 }
 
@@ -377,7 +381,7 @@ int build_state(osscar_ctx* ctx, bool guarded)
     CK(cudaFuncSetAttribute(k_pivot_inverse, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * NB * NB * (int)sizeof(double)));
     for (int64_t p0 = 0; p0 < nI; p0 += NB) {
         const int nb = (int)(nI - p0 < NB ? nI - p0 : NB);
-        k_pivot_inverse<<<1, 256, 2 * NB * NB * sizeof(double), st>>>(Hinv, L.ldh, p0, nb, Dinv, ctx->ctl);
+        k_pivot_inverse<<<1, 256, 2 * NB * NB * sizeof(double), st>>>(Hinv, L.ldh, p0, nb, Dinv, Hp, L.ldp, ctx->ctl);
         // T = A[:, P] * Dinv
         CK(sgemm(st, false, false, nI, nb, nb, 1.f, Hinv + p0, L.ldh, Dinv, NB, 0.f, T, NB, done));
         k_zero_rows<<<(nb * nb + 255) / 256, 256, 0, st>>>(T, NB, p0, nb, nb);
@@ -392,10 +396,11 @@ int build_state(osscar_ctx* ctx, bool guarded)
     CK(cudaGetLastError());
     // V = Hinv * G_I
     k_gather_rows<<<(unsigned)nI, 256, 0, st>>>(ctx->G, L.m, L.g, perm, 0, big, L.ldm);
+    if (L.ldm != L.m) CK(cudaMemsetAsync(V, 0, sizeof(float) * nI * L.ldm, st));     // padding columns stay zero
     CK(sgemm(st, false, false, nI, L.m, nI, 1.f, Hinv, L.ldh, big, L.ldm, 0.f, V, L.ldm, done));
     // obj = Tr(W^T G) - Tr(G_I^T V)
-    CK(trace_product(st, ctx->W, L.m, ctx->G, L.m, L.d1, L.m, &ctx->ctl->acc[0]));
-    CK(trace_product(st, big, L.ldm, V, L.ldm, nI, L.m, &ctx->ctl->acc[1]));
+    CK(trace_product(st, ctx->W, L.m, ctx->G, L.m, L.d1, L.m, ctx->partials, &ctx->ctl->acc[0]));
+    CK(trace_product(st, big, L.ldm, V, L.ldm, nI, L.m, ctx->partials, &ctx->ctl->acc[1]));
     k_set_obj<<<1, 1, 0, st>>>(ctx->ctl);
     if (nJ > 0) {
         // R_J = G_J - Hp[J, I] V
