@@ -1,0 +1,360 @@
+"""Benchmark of the OSSCAR per-layer solve on B200.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c5] [--impl ours|reference]
+
+One "step" is one whole layer solve (Gram over all token chunks, cross term, starting support and state,
+device-resident swap search, result) on one synthetic layer.  With N > 1 (torchrun) every rank solves an
+independent replica of the layer (seed = rank): the solve does not shard, so scaling is weak and there is
+no collective on the data path.  Prints one JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+import workloads  # noqa: E402
+
+METRIC = "swaps/s of the device-resident swap search (layer-solve seconds in ms_per_step)"
+UNIT = "swaps/s"
+CPU_SAMPLE = dict(n=4096, d1=2048, m=512, k=614, chunk_rows=4096)    # same value structure as c5, 1/14 of its width
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# ------------------------------------------------------------------------------------------ helpers
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.QUERY}",
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); smax.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        busy = [c for c in sm if c > 0]
+        return {"sm_mhz": statistics.median(busy) if busy else None, "sm_max_mhz": max(smax) if smax else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def dist_env():
+    rank = int(os.environ.get("RANK", "0")); world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+def reduce_over_ranks(values: dict, world: int, backend_device):
+    """max over ranks for keys starting with 'max_', sum for 'sum_' (all-reduce; identity when world == 1)."""
+    if world == 1:
+        return dict(values)
+    import torch.distributed as dist
+    out = {}
+    for key, val in values.items():
+        t = torch.tensor([float(val)], dtype=torch.float64, device=backend_device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX if key.startswith("max_") else dist.ReduceOp.SUM)
+        out[key] = float(t.item())
+    return out
+
+
+def swap_bytes(nI, nJ, m):
+    """Algorithmic HBM bytes of one swap of the fused single-pass scheme (fp32)."""
+    return 4 * (3 * nI * nI + 2 * nI * m + 2 * nJ * m + nJ * nI)
+
+
+KERNEL_BYTES = {   # algorithmic bytes per launch of the streaming kernels of a step
+    "y_pass": lambda nI, nJ, m: 4 * nI * nI,
+    "h_pass": lambda nI, nJ, m: 4 * nJ * nI,
+    "update_hinv": lambda nI, nJ, m: 8 * nI * nI,
+    "update_v": lambda nI, nJ, m: 8 * nI * m,
+    "update_r": lambda nI, nJ, m: 8 * nJ * m,
+}
+
+
+# ------------------------------------------------------------------------------------------ reference arm (CPU oracle)
+def oracle_step(wl, max_swaps):
+    import numpy as np
+    from oracle import osscar_oracle as orc
+    t0 = time.perf_counter()
+    chunks = [c.float().numpy() for c in wl.x_chunks()]
+    W = wl.weight().numpy().astype(np.float64)
+    t1 = time.perf_counter()
+    H, G, const = orc.gram_chunked(chunks, W, wl.damp)
+    S0, _ = orc.init_support(H, W, wl.g, wl.k)
+    srch = orc.Search(H, G, const, wl.g, S0, mode="lowrank", eps_acc=wl.eps_acc)
+    t2 = time.perf_counter()
+    srch.run(max_swaps)
+    t3 = time.perf_counter()
+    return {"solve_s": t3 - t1, "search_s": t3 - t2, "swaps": len(srch.swap_trace), "gen_s": t1 - t0}
+
+
+def cpu_baseline(max_swaps=40):
+    wl = workloads.config("c5", **CPU_SAMPLE)
+    r = oracle_step(wl, max_swaps)
+    cores = torch.get_num_threads()
+    return {"value": r["swaps"] / max(r["search_s"], 1e-9), "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": (f"fp64 NumPy oracle (low-rank-update mode) on a c5-structured layer cut to d1={wl.d1}, m={wl.m}, "
+                       f"k={wl.k}, n={wl.n}: {r['swaps']} swaps in {r['search_s']:.2f} s, whole solve {r['solve_s']:.2f} s"),
+            "layer_solve_s": r["solve_s"]}
+
+
+def run_reference(args):
+    rank, world, _ = dist_env()
+    if rank != 0:
+        return
+    wl = workloads.config("c5", **CPU_SAMPLE)
+    for _ in range(args.warmup):
+        oracle_step(wl, 5)
+    tot, swaps, search = 0.0, 0, 0.0
+    for _ in range(args.steps):
+        r = oracle_step(wl, 40)
+        tot += r["solve_s"]; swaps += r["swaps"]; search += r["search_s"]
+    value = swaps / max(search, 1e-9)
+    cores = torch.get_num_threads()
+    sample = (f"fp64 NumPy oracle on a c5-structured layer cut to d1={wl.d1}, m={wl.m}, k={wl.k}, n={wl.n}, "
+              f"at most 40 swaps per step")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * tot / max(args.steps, 1), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "c5 (OPT-30B-shaped FC2) bounded sample: " + sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+# ------------------------------------------------------------------------------------------ our arm
+def run_ours(args):
+    rank, world, local = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the solve has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    import paper_2403_12983_b200 as pkg
+    from paper_2403_12983_b200 import binding as b
+
+    over = {}
+    if args.tokens:
+        over["n"] = args.tokens
+    wl = workloads.config(args.workload, seed=rank, **over)
+    max_swaps = args.max_swaps if args.max_swaps is not None else wl.max_swaps
+    accept = b.ACCEPT_ALWAYS if args.accept_always else b.ACCEPT_IMPROVING
+    solver = pkg.Solver(local)
+    W = wl.weight(dev)
+    x_dev = [wl.x_chunk(c, dev) for c in range(wl.n_chunks)]          # inputs resident in HBM
+    torch.cuda.synchronize()
+    H = torch.empty(wl.d1, wl.d1, dtype=torch.float32, device=dev)
+    G = torch.empty(wl.d1, wl.m, dtype=torch.float32, device=dev)
+    nI, nJ, m = wl.k * wl.g, wl.d1 - wl.k * wl.g, wl.m
+
+    def step(x_chunks, W_in, prof=0):
+        return pkg.solve_layer(solver, x_chunks, W_in, wl.g, wl.k, max_swaps, damp=wl.damp, accept_mode=accept, accept_rel_tol=wl.eps_acc,
+                               profile_samples=prof, H=H, G=G)
+
+    def barrier():
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        res = step(x_dev, W)
+    # ---------------- device-resident timing
+    sampler = ClockSampler(local)
+    barrier()
+    sampler.start()
+    launches0 = b.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    phase = {"gram": 0.0, "gram_end": 0.0, "init": 0.0, "search": 0.0, "search_loop": 0.0}
+    kern = {}
+    swaps = 0
+    e0.record()
+    for _ in range(args.steps):
+        res = step(x_dev, W, prof=8)
+        for key in phase:
+            phase[key] += res.ms[key]
+        for key, val in res.ms_kernel.items():
+            kern[key] = kern.get(key, 0.0) + val
+        swaps += res.n_swaps
+    e1.record()
+    barrier()
+    launches = b.launch_count() - launches0
+    clocks = sampler.stop()
+    total_ms = e0.elapsed_time(e1)
+    K = max(args.steps, 1)
+
+    # ---------------- end to end: host buffers, copies inside the timed region
+    e2e = None
+    if not args.no_e2e:
+        try:
+            x_host = [c.to("cpu").pin_memory() for c in x_dev]
+            W_host = W.to("cpu").pin_memory()
+            pinned = {"W": torch.empty(wl.d1, wl.m, dtype=torch.float32).pin_memory()}
+            del x_dev
+            torch.cuda.empty_cache()
+            r = step(x_host, W_host)                         # warm-up of the copy path
+            pkg.result_to_host(r, pinned)
+            barrier()
+            f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e_swaps, e_search, h2d, d2h = 0, 0.0, 0, 0
+            nrep = max(1, min(K, 2))
+            f0.record()
+            for _ in range(nrep):
+                r = step(x_host, W_host)
+                back = pkg.result_to_host(r, pinned)
+                e_swaps += r.n_swaps; h2d += r.io["h2d"]; d2h += back["bytes"]
+            f1.record()
+            barrier()
+            e_ms = f0.elapsed_time(f1)
+            e2e = {"ms_per_step": e_ms / nrep, "swaps": e_swaps, "h2d": h2d // nrep, "d2h": d2h // nrep}
+        except RuntimeError as exc:                           # e.g. pinned allocation refused
+            e2e = {"error": str(exc)[:200]}
+
+    red = reduce_over_ranks({"max_total_ms": total_ms, "sum_swaps": swaps, "max_search_ms": phase["search_loop"],
+                             "max_e2e_ms": (e2e or {}).get("ms_per_step", 0.0), "sum_e2e_swaps": (e2e or {}).get("swaps", 0)},
+                            world, dev)
+    if rank != 0:
+        if world > 1:
+            torch.distributed.destroy_process_group()
+        return
+
+    pk = peaks()
+    ms_step = red["max_total_ms"] / K
+    search_s = red["max_search_ms"] / 1e3
+    value = red["sum_swaps"] / max(search_s, 1e-9)
+    # dominant kernel among the streaming kernels of a swap, and the Gram kernel, by share of the step
+    kern_avg = {k2: v / K for k2, v in kern.items()}
+    per_step_swaps = swaps / K
+    shares = {k2: v * per_step_swaps for k2, v in kern_avg.items()}
+    shares["gram_tcgen05"] = phase["gram"] / K
+    dom = max(shares, key=shares.get) if shares else "gram_tcgen05"
+    if dom in KERNEL_BYTES and kern_avg.get(dom, 0) > 0:
+        bytes_per_launch = KERNEL_BYTES[dom](nI, nJ, m)
+        ach = bytes_per_launch / (kern_avg[dom] * 1e-3) / 1e9
+        roof = {"kernel": dom, "bound": "hbm", "achieved": ach, "peak": pk["hbm_gbs"], "unit": "GB/s",
+                "frac": ach / pk["hbm_gbs"], "traffic": None, "bytes_per_launch": bytes_per_launch,
+                "ms_per_launch": kern_avg[dom], "peak_source": pk["source"]}
+    else:
+        tm_, tn_ = -(-wl.d1 // 128), -(-wl.d1 // 256)
+        tiles = sum(tn_ - t // 2 for t in range(tm_))
+        flops = 2.0 * 128 * 256 * tiles * wl.n
+        ach = flops / (phase["gram"] / K * 1e-3) / 1e12
+        roof = {"kernel": "k_gram_tcgen05", "bound": "tensor", "achieved": ach, "peak": pk["bf16_tflops_sustained"],
+                "unit": "TFLOP/s", "frac": ach / pk["bf16_tflops_sustained"], "traffic": None,
+                "flops_per_step": flops, "peak_source": pk["source"] + " (sustained)"}
+    tm_, tn_ = -(-wl.d1 // 128), -(-wl.d1 // 256)
+    tiles = sum(tn_ - t // 2 for t in range(tm_))
+    gram_exec_tflops = 2.0 * 128 * 256 * tiles * wl.n / max(phase["gram"] / K * 1e-3, 1e-12) / 1e12
+    loop_gbs = swap_bytes(nI, nJ, m) * per_step_swaps / max(phase["search_loop"] / K * 1e-3, 1e-12) / 1e9
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32 (bf16 tensor-core Gram, fp32 accumulate)", "data": "synthetic",
+        "config": {"workload": f"{wl.name}: d1={wl.d1} m={wl.m} g={wl.g} k={wl.k} n={wl.n} in {wl.n_chunks} chunks, "
+                               f"max_swaps={max_swaps}, accept={'always' if args.accept_always else 'improving'} (eps {wl.eps_acc:g}), damp={wl.damp}",
+                   "l2": "inputs larger than L2 (X, H and the search state are each > 126 MB)" if wl.d1 >= 8192 else
+                         "state smaller than L2; numbers are cache-resident",
+                   "replicas": world},
+        "clocks": clocks,
+        "layer_solve_s": ms_step / 1e3,
+        "swaps_per_step": per_step_swaps, "stop_reason": res.stop_reason,
+        "obj_init": res.obj_init, "obj_final": res.obj_final,
+        "phases_ms": {k2: v / K for k2, v in phase.items()},
+        "kernel_ms": kern_avg,
+        "gram": {"executed_tflops": gram_exec_tflops, "dense_equiv_tflops": 2.0 * wl.n * wl.d1 ** 2 / max(phase["gram"] / K * 1e-3, 1e-12) / 1e12,
+                 "frac_of_bf16_peak": gram_exec_tflops / pk["bf16_tflops_sustained"], "peak": pk["bf16_tflops_sustained"],
+                 "peak_source": pk["source"] + " (sustained)"},
+        "swap_loop": {"gbs": loop_gbs, "bytes_per_swap": swap_bytes(nI, nJ, m), "frac_of_hbm": loop_gbs / pk["hbm_gbs"],
+                      "peak": pk["hbm_gbs"], "peak_source": pk["source"]},
+        "roofline": roof,
+        "gpu_launches": int(launches),
+    }
+    if e2e and "ms_per_step" in e2e:
+        e_val = red["sum_e2e_swaps"] / max(min(K, 2), 1) / max(red["max_e2e_ms"] * 1e-3, 1e-9)
+        out["e2e"] = {"value": e_val, "unit": "swaps per second of whole-solve time, host buffers", "ms_per_step": red["max_e2e_ms"],
+                      "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"]}
+    else:
+        out["e2e"] = {"value": None, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0,
+                      "note": (e2e or {}).get("error", "skipped")}
+    if world == 1 and not args.no_cpu:
+        out["cpu_baseline"] = cpu_baseline()
+    print(json.dumps(out))
+    if world > 1:
+        torch.distributed.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c5")
+    ap.add_argument("--tokens", type=int, default=None, help="override the number of calibration rows")
+    ap.add_argument("--max-swaps", type=int, default=None)
+    ap.add_argument("--accept-always", action="store_true", help="paper-literal fixed number of iterations")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

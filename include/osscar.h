@@ -101,13 +101,19 @@ typedef struct {
     int32_t accept_mode;      /* OSSCAR_ACCEPT_*                                             */
     int32_t refresh_every;    /* rebuild the state from H every this many swaps; 0 = never   */
     double  accept_rel_tol;   /* IMPROVING: accept iff delta <= -tol * obj (1e-5 if < 0)     */
-    uint64_t wait_limit_cycles; /* bound of device-side waits; 0 = default                   */
+    int32_t profile_samples;  /* time each kernel of this many evenly spaced steps (0..8)    */
+    int32_t reserved;         /* must be 0                                                   */
 } osscar_search_params;
+
+#define OSSCAR_NUM_STEP_KERNELS 12   /* select, pair Grams, y pass, small algebra, staging, H pass,
+                                        Hinv update, V update, R update, group scores, H row swap, H column swap */
 
 typedef struct {
     int32_t n_swaps, stop_reason, n_refresh, status;
     double  obj_init, obj_final;     /* obj_final is recomputed from the final state         */
     float   ms_search;               /* device time of the swap loop                         */
+    int32_t n_profiled;              /* steps that were timed kernel by kernel and did a swap */
+    float   ms_kernel[OSSCAR_NUM_STEP_KERNELS]; /* mean device time of each kernel over those steps */
 } osscar_search_result;
 
 /*
@@ -140,6 +146,9 @@ int osscar_objective(osscar_ctx* ctx, const float* H, const float* W, const floa
 int osscar_debug_get_state(osscar_ctx* ctx, int which, void* dst);
 
 const char* osscar_status_string(int status);
+
+/* Number of kernels this library has launched in this process so far (all contexts). */
+uint64_t osscar_launch_count(void);
 
 #ifdef __cplusplus
 }

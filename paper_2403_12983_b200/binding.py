@@ -22,17 +22,22 @@ STOP_NAMES = {0: "max_swaps", 1: "no_improvement", 2: "guard"}
 
 EXPORTS = ["osscar_create", "osscar_destroy", "osscar_workspace_bytes", "osscar_set_workspace",
            "osscar_gram", "osscar_init_support", "osscar_local_search", "osscar_objective",
-           "osscar_debug_get_state", "osscar_status_string"]
+           "osscar_debug_get_state", "osscar_status_string", "osscar_launch_count"]
 
 
 class SearchParams(C.Structure):
     _fields_ = [("max_swaps", C.c_int32), ("score_mode", C.c_int32), ("accept_mode", C.c_int32),
-                ("refresh_every", C.c_int32), ("accept_rel_tol", C.c_double), ("wait_limit_cycles", C.c_uint64)]
+                ("refresh_every", C.c_int32), ("accept_rel_tol", C.c_double), ("profile_samples", C.c_int32), ("reserved", C.c_int32)]
 
 
 class SearchResult(C.Structure):
     _fields_ = [("n_swaps", C.c_int32), ("stop_reason", C.c_int32), ("n_refresh", C.c_int32), ("status", C.c_int32),
-                ("obj_init", C.c_double), ("obj_final", C.c_double), ("ms_search", C.c_float)]
+                ("obj_init", C.c_double), ("obj_final", C.c_double), ("ms_search", C.c_float),
+                ("n_profiled", C.c_int32), ("ms_kernel", C.c_float * 12)]
+
+
+STEP_KERNELS = ["select", "pair_grams", "y_pass", "small_algebra", "staging", "h_pass", "update_hinv", "update_v",
+                "update_r", "group_scores", "h_swap_rows", "h_swap_cols"]
 
 
 class OsscarError(RuntimeError):
@@ -70,8 +75,10 @@ def lib() -> C.CDLL:
     L.osscar_local_search.argtypes = [vp, C.POINTER(SearchParams), vp, vp, vp, vp, C.POINTER(SearchResult)]
     L.osscar_objective.argtypes = [vp, vp, vp, vp, i64, i64, C.POINTER(C.c_double)]
     L.osscar_debug_get_state.argtypes = [vp, C.c_int, vp]
+    L.osscar_launch_count.restype = C.c_uint64
+    L.osscar_launch_count.argtypes = []
     for name in EXPORTS:
-        if name != "osscar_status_string":
+        if name not in ("osscar_status_string", "osscar_launch_count"):
             getattr(L, name).restype = C.c_int
     _LIB = L
     return L
@@ -92,6 +99,10 @@ def _dev_f32(t: torch.Tensor, name: str) -> torch.Tensor:
     return t
 
 
+def launch_count() -> int:
+    return int(lib().osscar_launch_count())
+
+
 def osscar_workspace_bytes(d1: int, m: int, g: int, k: int) -> int:
     out = C.c_size_t(0)
     _check(lib().osscar_workspace_bytes(d1, m, g, k, C.byref(out)), "osscar_workspace_bytes")
@@ -110,6 +121,7 @@ class SearchOutput:
     obj_init: float
     obj_final: float
     ms_search: float
+    ms_kernel: dict              # mean device ms per kernel of a step over the profiled steps ({} if none)
 
 
 class Solver:
@@ -197,21 +209,22 @@ class Solver:
         return support, obj0.value
 
     def local_search(self, max_swaps: int, score_mode: int = SCORE_INDEPENDENT, accept_mode: int = ACCEPT_IMPROVING,
-                     refresh_every: int = 0, accept_rel_tol: float = -1.0) -> SearchOutput:
+                     refresh_every: int = 0, accept_rel_tol: float = -1.0, profile_samples: int = 0) -> SearchOutput:
         d1, m, g, k = self._shape
         dev = self._keep[0].device
         support = torch.empty(k, dtype=torch.int32, device=dev)
         W_out = torch.empty(d1, m, dtype=torch.float32, device=dev)
         obj_trace = torch.zeros(max_swaps + 1, dtype=torch.float64, device=dev)
         swap_trace = torch.zeros(max(1, 2 * max_swaps), dtype=torch.int32, device=dev)
-        prm = SearchParams(max_swaps, score_mode, accept_mode, refresh_every, accept_rel_tol, 0)
+        prm = SearchParams(max_swaps, score_mode, accept_mode, refresh_every, accept_rel_tol, profile_samples, 0)
         res = SearchResult()
         _check(lib().osscar_local_search(self._h, C.byref(prm), _ptr(support), _ptr(W_out), _ptr(obj_trace), _ptr(swap_trace),
                                          C.byref(res)), "osscar_local_search")
         n = res.n_swaps
         return SearchOutput(support, W_out, obj_trace[:n + 1], swap_trace[:2 * n].view(n, 2), n,
                             STOP_NAMES.get(res.stop_reason, str(res.stop_reason)), res.n_refresh,
-                            res.obj_init, res.obj_final, res.ms_search)
+                            res.obj_init, res.obj_final, res.ms_search,
+                            {n: res.ms_kernel[i] for i, n in enumerate(STEP_KERNELS)} if res.n_profiled > 0 else {})
 
     def objective(self, H, W, Wt) -> float:
         _dev_f32(H, "H"); _dev_f32(W, "W"); _dev_f32(Wt, "Wt")

@@ -313,6 +313,7 @@ cudaError_t gram_mirror(cudaStream_t st, float* H, int64_t d1)
 {
     const unsigned nb = (unsigned)((d1 + 31) / 32);
     k_mirror<<<dim3(nb, nb), dim3(32, 8), 0, st>>>(H, d1);
+    count_launches(1);
     return cudaGetLastError();
 }
 
@@ -346,6 +347,7 @@ cudaError_t gram_bf16_tcgen05(cudaStream_t st, const void* X, int64_t n_rows, in
         attr_set = true;
     }
     const int grid = num_tiles < sms ? num_tiles : sms;
+    count_launches(1);
     k_gram_tcgen05<<<grid, NUM_THREADS, SMEM_BYTES, st>>>(tmap, n_rows, d1, H, accumulate ? 1 : 0, num_tiles, TM, TN, status_dev);
     return cudaGetLastError();
 }

@@ -5,6 +5,8 @@
 
 using namespace osscar;
 
+namespace osscar { unsigned long long g_launches = 0; }
+
 namespace {
 
 #define CKC(x) do { cudaError_t e_ = (x); if (e_ != cudaSuccess) return OSSCAR_E_CUDA; } while (0)
@@ -44,6 +46,8 @@ __global__ void k_sub(const float* __restrict__ A, const float* __restrict__ B, 
 }  // namespace
 
 extern "C" {
+
+uint64_t osscar_launch_count(void) { return g_launches; }
 
 const char* osscar_status_string(int s)
 {
@@ -135,6 +139,7 @@ int osscar_gram(osscar_ctx* ctx, const void* X, int x_dtype, int64_t n_rows, int
     if (!guard.ok) return OSSCAR_E_CUDA;
     cudaStream_t st = ctx->stream;
     k_clear_status<<<1, 1, 0, st>>>(ctx->ctl);
+    count_launches(1);
     if (begin) ctx->gram_rows = 0;
     if (begin && n_rows == 0) CKC(cudaMemsetAsync(H, 0, sizeof(float) * d1 * d1, st));
     if (n_rows > 0) {
@@ -153,6 +158,7 @@ int osscar_gram(osscar_ctx* ctx, const void* X, int x_dtype, int64_t n_rows, int
         CKC(cudaMemsetAsync(&ctx->ctl->acc[0], 0, sizeof(double), st));
         k_diag_sum<<<64, 256, 0, st>>>(H, d1, &ctx->ctl->acc[0]);
         k_add_damp<<<64, 256, 0, st>>>(H, d1, damp, &ctx->ctl->acc[0]);
+        count_launches(2);
     }
     CKC(sgemm(st, false, false, d1, m, d1, 1.f, H, d1, W, m, 0.f, G, m));
     CKC(trace_product(st, W, m, G, m, d1, m, ctx->partials, &ctx->ctl->acc[1]));
@@ -198,7 +204,7 @@ int osscar_local_search(osscar_ctx* ctx, const osscar_search_params* params,
     if (params->max_swaps < 0 || (params->max_swaps > 0 && !swap_trace)) return OSSCAR_E_ARG;
     if (params->score_mode != OSSCAR_SCORE_INDEPENDENT && params->score_mode != OSSCAR_SCORE_PAIR_EXACT) return OSSCAR_E_ARG;
     if (params->accept_mode != OSSCAR_ACCEPT_IMPROVING && params->accept_mode != OSSCAR_ACCEPT_ALWAYS) return OSSCAR_E_ARG;
-    if (params->refresh_every < 0) return OSSCAR_E_ARG;
+    if (params->refresh_every < 0 || params->profile_samples < 0 || params->profile_samples > 8 || params->reserved != 0) return OSSCAR_E_ARG;
     if (!ctx->have_state) return OSSCAR_E_STATE;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return OSSCAR_E_CUDA;
@@ -221,6 +227,7 @@ int osscar_objective(osscar_ctx* ctx, const float* H, const float* W, const floa
     float* E = (float*)ctx->ws;
     float* HE = E + d1 * m;
     k_sub<<<1184, 256, 0, st>>>(W, Wt, E, d1 * m);
+    count_launches(1);
     CKC(sgemm(st, false, false, d1, m, d1, 1.f, H, d1, E, m, 0.f, HE, m));
     CKC(trace_product(st, E, m, HE, m, d1, m, ctx->partials, &ctx->ctl->acc[0]));
     CKC(cudaMemcpyAsync(ctx->ctl_host, ctx->ctl, sizeof(SearchCtl), cudaMemcpyDeviceToHost, st));

@@ -10,6 +10,9 @@ namespace osscar {
 constexpr int kTracePartials = 1184;   // blocks of a trace reduction; the context owns that many doubles
 constexpr int kPadF = 32;   // leading dimensions of internal fp32 matrices are padded to this many floats
 
+extern unsigned long long g_launches;      // kernels launched by the library (host-side count)
+static inline void count_launches(unsigned long long n) { g_launches += n; }
+
 static inline int64_t round_up(int64_t x, int64_t a) { return (x + a - 1) / a * a; }
 
 // Device-side control block of the swap loop.  Lives in the context's small device allocation.

@@ -687,6 +687,7 @@ cudaError_t enqueue_scores(osscar_ctx* ctx, const Ptrs& p, bool norms)
     if (p.g == 1) {
         if (norms) {
             k_row_norms<<<(unsigned)p.nI, 256, 0, st>>>(p.V, p.ldm, p.vnorm, p.ctl);
+            count_launches(p.nJ > 0 ? 2 : 1);
             if (p.nJ > 0) k_row_norms<<<(unsigned)p.nJ, 256, 0, st>>>(p.R, p.ldm, p.rnorm, p.ctl);
         }
     } else {
@@ -695,6 +696,7 @@ cudaError_t enqueue_scores(osscar_ctx* ctx, const Ptrs& p, bool norms)
         if (e != cudaSuccess) return e;
         k_group_gram<<<dim3((unsigned)p.k, (unsigned)p.g), 256, 0, st>>>(p.V, p.ldm, p.g, p.gramV, p.ctl);
         k_scores_general<<<(unsigned)p.k, 256, smem, st>>>(p, 0);
+        count_launches(p.nJ > 0 ? 4 : 2);
         if (p.nJ > 0) {
             k_group_gram<<<dim3((unsigned)(p.ng - p.k), (unsigned)p.g), 256, 0, st>>>(p.R, p.ldm, p.g, p.gramR, p.ctl);
             k_scores_general<<<(unsigned)(p.ng - p.k), 256, smem, st>>>(p, 1);
@@ -711,6 +713,7 @@ cudaError_t score_pass(osscar_ctx* ctx)
     cudaError_t e = enqueue_scores(ctx, p, true);
     if (e != cudaSuccess) return e;
     k_select<<<1, 1024, 0, ctx->stream>>>(p);      // also leaves the score vectors D and A readable
+    count_launches(1);
     return cudaGetLastError();
 }
 
@@ -725,6 +728,7 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
     const int max_swaps = (L.nJ > 0) ? prm->max_swaps : 0;
 
     k_begin<<<1, 1, 0, st>>>(ctx->ctl, obj_trace, ctx->done_flag_dev);
+    count_launches(1);
     CK(cudaGetLastError());
     CK(cudaEventRecord(ctx->ev0, st));
     if (max_swaps > 0) CK(enqueue_scores(ctx, p, true));
@@ -733,11 +737,21 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
     cudaEvent_t evb[2];
     CK(cudaEventCreateWithFlags(&evb[0], cudaEventDisableTiming));
     CK(cudaEventCreateWithFlags(&evb[1], cudaEventDisableTiming));
+    // optional kernel-by-kernel timing of a few evenly spaced steps
+    constexpr int NK = OSSCAR_NUM_STEP_KERNELS;
+    const int nprof = max_swaps > 0 ? (prm->profile_samples < max_swaps ? prm->profile_samples : max_swaps) : 0;
+    cudaEvent_t evp[8][NK + 1];
+    int prof_it[8];
+    for (int i = 0; i < nprof; ++i) {
+        prof_it[i] = (2 << i) - 1 < max_swaps ? (2 << i) - 1 : max_swaps - nprof + i;   // steps 1, 3, 7, 15, ...
+        for (int j = 0; j <= NK; ++j) CK(cudaEventCreate(&evp[i][j]));
+    }
     int rc = OSSCAR_OK;
     const unsigned yblocks = (unsigned)((L.nI + 7) / 8);
     constexpr int RPW = 4;
     const unsigned hblocks = (unsigned)((L.nJ + g + 8 * RPW - 1) / (8 * RPW));
     const unsigned prep_blocks = (unsigned)(((L.nI + L.ldm) * g + 255) / 256);
+    int next_prof = 0;
     for (int it = 0; it < max_swaps && rc == OSSCAR_OK; ++it) {
         if (it % batch == 0) {
             const int bi = it / batch;
@@ -750,23 +764,34 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
             rc = build_state(ctx, true);
             if (rc != OSSCAR_OK) break;
             k_count_refresh<<<1, 1, 0, st>>>(ctx->ctl);
+            count_launches(1);
             if (enqueue_scores(ctx, p, true) != cudaSuccess) { rc = OSSCAR_E_CUDA; break; }
         }
-        k_select<<<1, 1024, 0, st>>>(p);
-        k_pairgram<<<(unsigned)((3 * g * g + 7) / 8), 256, 0, st>>>(p);
-        k_ypass<<<dim3(yblocks, g), 256, 0, st>>>(p);
-        k_small<<<1, 256, 0, st>>>(p, prm->accept_mode, tol, max_swaps, obj_trace, swap_trace);
-        k_prep<<<prep_blocks, 256, 0, st>>>(p);
-        k_hpass<RPW><<<dim3(hblocks, g), 256, 0, st>>>(p);
+        cudaEvent_t* pe = nullptr;
+        if (next_prof < nprof && prof_it[next_prof] == it) pe = evp[next_prof++];
+        int slot = 0;
+        auto mark = [&]() { if (pe) cudaEventRecord(pe[slot], st); ++slot; };
+        mark();
+        k_select<<<1, 1024, 0, st>>>(p);                                                         mark();
+        k_pairgram<<<(unsigned)((3 * g * g + 7) / 8), 256, 0, st>>>(p);                          mark();
+        k_ypass<<<dim3(yblocks, g), 256, 0, st>>>(p);                                            mark();
+        k_small<<<1, 256, 0, st>>>(p, prm->accept_mode, tol, max_swaps, obj_trace, swap_trace);  mark();
+        k_prep<<<prep_blocks, 256, 0, st>>>(p);                                                  mark();
+        k_hpass<RPW><<<dim3(hblocks, g), 256, 0, st>>>(p);                                       mark();
         k_update_hinv<<<dim3((unsigned)((L.ldh / 4 + 255) / 256), (unsigned)((L.nI + HI_RT - 1) / HI_RT)), 256, 0, st>>>(p);
-        k_update_rows<<<(unsigned)((L.nI + UP_ROWS - 1) / UP_ROWS), 256, 0, st>>>(p, 0);
-        k_update_rows<<<(unsigned)((L.nJ + UP_ROWS - 1) / UP_ROWS), 256, 0, st>>>(p, 1);
+        mark();
+        k_update_rows<<<(unsigned)((L.nI + UP_ROWS - 1) / UP_ROWS), 256, 0, st>>>(p, 0);          mark();
+        k_update_rows<<<(unsigned)((L.nJ + UP_ROWS - 1) / UP_ROWS), 256, 0, st>>>(p, 1);          mark();
+        count_launches(9);
         if (g > 1) {
             k_update_c<<<(unsigned)(L.ng - L.k), 128, 0, st>>>(p);
+            count_launches(1);
             if (enqueue_scores(ctx, p, false) != cudaSuccess) { rc = OSSCAR_E_CUDA; break; }
         }
-        k_hswap<<<(unsigned)((L.ldp * g + 255) / 256), 256, 0, st>>>(p, 0);
-        k_hswap<<<(unsigned)((L.ldp * g + 255) / 256), 256, 0, st>>>(p, 1);
+        mark();
+        k_hswap<<<(unsigned)((L.ldp * g + 255) / 256), 256, 0, st>>>(p, 0);                       mark();
+        k_hswap<<<(unsigned)((L.ldp * g + 255) / 256), 256, 0, st>>>(p, 1);                       mark();
+        count_launches(2);
         if (cudaGetLastError() != cudaSuccess) { rc = OSSCAR_E_CUDA; break; }
         if ((it + 1) % batch == 0) {
             if (cudaEventRecord(evb[(it / batch) & 1], st) != cudaSuccess) { rc = OSSCAR_E_CUDA; break; }
@@ -774,7 +799,11 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
     }
     cudaEventDestroy(evb[0]);
     cudaEventDestroy(evb[1]);
-    if (rc != OSSCAR_OK) { cudaStreamSynchronize(st); return rc; }
+    if (rc != OSSCAR_OK) {
+        cudaStreamSynchronize(st);
+        for (int i = 0; i < nprof; ++i) for (int j = 0; j <= NK; ++j) cudaEventDestroy(evp[i][j]);
+        return rc;
+    }
     CK(cudaEventRecord(ctx->ev1, st));
 
     // results: weights, support, objective recomputed from the final state
@@ -787,6 +816,7 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
         CK(gather_rows(st, ctx->G, L.m, L.g, p.perm, 0, L.nI, big, L.ldm));
         CK(trace_product(st, big, L.ldm, p.V, L.ldm, L.nI, L.m, ctx->partials, &ctx->ctl->acc[1]));
         k_final_obj<<<1, 1, 0, st>>>(ctx->ctl);
+        count_launches(3);
     }
     CK(cudaGetLastError());
     CK(cudaMemcpyAsync(ctx->ctl_host, ctx->ctl, sizeof(SearchCtl), cudaMemcpyDeviceToHost, st));
@@ -800,6 +830,20 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
     res->obj_init = ctx->ctl_host->acc[2];
     res->obj_final = ctx->ctl_host->acc[3];
     res->ms_search = ms;
+    // kernel times of the sampled steps that really swapped (a stopped loop runs empty kernels)
+    int used = 0;
+    for (int i = 0; i < nprof; ++i) {
+        if (i < next_prof && prof_it[i] < res->n_swaps) {
+            for (int j = 0; j < NK; ++j) {
+                float t = 0.f;
+                if (cudaEventElapsedTime(&t, evp[i][j], evp[i][j + 1]) == cudaSuccess) res->ms_kernel[j] += t;
+            }
+            ++used;
+        }
+        for (int j = 0; j <= NK; ++j) cudaEventDestroy(evp[i][j]);
+    }
+    for (int j = 0; j < NK && used > 0; ++j) res->ms_kernel[j] /= (float)used;
+    res->n_profiled = used;
     return ctx->ctl_host->status;
 }
 

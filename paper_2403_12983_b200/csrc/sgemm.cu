@@ -108,6 +108,7 @@ cudaError_t sgemm(cudaStream_t st, bool transA, bool transB, int64_t M, int64_t 
     if (transB) return cudaErrorInvalidValue;
     if (M <= 0 || N <= 0) return cudaSuccess;
     dim3 grid((unsigned)((N + BN - 1) / BN), (unsigned)((M + BM - 1) / BM));
+    count_launches(1);
     if (transA) sgemm_kernel<true><<<grid, NT, 0, st>>>(M, N, K, alpha, A, lda, B, ldb, beta, C, ldc, done);
     else        sgemm_kernel<false><<<grid, NT, 0, st>>>(M, N, K, alpha, A, lda, B, ldb, beta, C, ldc, done);
     return cudaGetLastError();

@@ -267,7 +267,7 @@ __global__ void k_set_obj(SearchCtl* ctl)   // obj = const - Tr(G_I^T V), with a
 cudaError_t gather_rows(cudaStream_t st, const float* src, int64_t m, int g, const int32_t* perm,
                         int64_t slot_row0, int64_t nrows, float* dst, int64_t ld)
 {
-    if (nrows > 0) k_gather_rows<<<(unsigned)nrows, 256, 0, st>>>(src, m, g, perm, slot_row0, dst, ld);
+    if (nrows > 0) { k_gather_rows<<<(unsigned)nrows, 256, 0, st>>>(src, m, g, perm, slot_row0, dst, ld); count_launches(1); }
     return cudaGetLastError();
 }
 
@@ -278,6 +278,7 @@ cudaError_t trace_product(cudaStream_t st, const float* A, int64_t lda, const fl
     const int grid = (int)(rows < kTracePartials ? rows : kTracePartials);
     k_trace_product<<<grid, 256, 0, st>>>(A, lda, B, ldb, rows, cols, partials);
     k_sum_partials<<<1, 256, 0, st>>>(partials, grid, out_dev);
+    count_launches(2);
     return cudaGetLastError();
 }
 
@@ -346,6 +347,7 @@ int select_support(osscar_ctx* ctx, int mode, int32_t* support)
         k_rank_select<<<nb, 256, 0, st>>>(e, L.ng, L.k, kept);
     }
     k_build_perm<<<nb, 256, 0, st>>>(kept, L.ng, L.k, perm, slotof, support);
+    count_launches(mode == OSSCAR_INIT_USER ? 2 : 3);
     CK(cudaGetLastError());
     return OSSCAR_OK;
 }
@@ -377,6 +379,7 @@ int build_state(osscar_ctx* ctx, bool guarded)
     }
     CK(cudaMemsetAsync(ws + L.off_vec_begin, 0, L.off_vec_end - L.off_vec_begin, st));
     k_copy_pad<<<(unsigned)nI, 256, 0, st>>>(Hp, L.ldp, nI, nI, Hinv, L.ldh);
+    count_launches(2);
     CK(cudaGetLastError());
     CK(cudaFuncSetAttribute(k_pivot_inverse, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * NB * NB * (int)sizeof(double)));
     for (int64_t p0 = 0; p0 < nI; p0 += NB) {
@@ -392,6 +395,7 @@ int build_state(osscar_ctx* ctx, bool guarded)
         CK(sgemm(st, false, false, nb, nI, nb, -1.f, Dinv, NB, U, L.ldh, 0.f, Un, L.ldh, done));
         CK(sgemm(st, false, false, nI, nI, nb, -1.f, T, NB, U, L.ldh, 1.f, Hinv, L.ldh, done));
         k_gj_writeback<<<(unsigned)((nI * nb + 255) / 256), 256, 0, st>>>(Hinv, L.ldh, nI, p0, nb, T, NB, Un, L.ldh, Dinv);
+        count_launches(4);     // pivot inverse, zero rows, copy rows, write-back (the GEMMs count themselves)
     }
     CK(cudaGetLastError());
     // V = Hinv * G_I
@@ -402,6 +406,7 @@ int build_state(osscar_ctx* ctx, bool guarded)
     CK(trace_product(st, ctx->W, L.m, ctx->G, L.m, L.d1, L.m, ctx->partials, &ctx->ctl->acc[0]));
     CK(trace_product(st, big, L.ldm, V, L.ldm, nI, L.m, ctx->partials, &ctx->ctl->acc[1]));
     k_set_obj<<<1, 1, 0, st>>>(ctx->ctl);
+    count_launches(2);
     if (nJ > 0) {
         // R_J = G_J - Hp[J, I] V
         k_gather_rows<<<(unsigned)nJ, 256, 0, st>>>(ctx->G, L.m, L.g, perm, nI, R, L.ldm);
@@ -409,6 +414,7 @@ int build_state(osscar_ctx* ctx, bool guarded)
         // Pm = Hp[J, I] Hinv, then the Schur complements
         CK(sgemm(st, false, false, nJ, nI, nI, 1.f, Hp + nI * L.ldp, L.ldp, Hinv, L.ldh, 0.f, big, L.ldh, done));
         k_schur<<<(unsigned)(L.ng - L.k), 256, 0, st>>>(Hp, L.ldp, big, L.ldh, nI, L.g, c);
+        count_launches(2);
     }
     CK(cudaGetLastError());
     return OSSCAR_OK;

@@ -17,7 +17,7 @@ def oracle_problem(wl):
 
 
 def follow_trace(H, G, const, g, S0, swaps, gpu_obj, score_mode="independent", accept="improving",
-                 mode="lowrank", max_swaps=None, gpu_stop=None, obj_rtol=1e-4):
+                 mode="lowrank", max_swaps=None, gpu_stop=None, obj_rtol=1e-4, eps_acc=orc.EPS_ACC):
     """Walks the GPU's swap sequence with the oracle.  Returns (search, n_rebased).
 
     At each step the oracle proposes its swap from its own fp64 state.  If the GPU made the same
@@ -25,7 +25,7 @@ def follow_trace(H, G, const, g, S0, swaps, gpu_obj, score_mode="independent", a
     the GPU's choice must itself be within GAP of the oracle's best scores; the oracle is then moved
     to the GPU's support and the walk continues.  The running objective must agree throughout.
     """
-    srch = orc.Search(H, G, const, g, S0, mode=mode, score_mode=score_mode, accept=accept)
+    srch = orc.Search(H, G, const, g, S0, mode=mode, score_mode=score_mode, accept=accept, eps_acc=eps_acc)
     rebased = 0
     assert gpu_obj[0] == __import__("pytest").approx(srch.st.obj, rel=obj_rtol)
     for step, (i_out, j_in) in enumerate(swaps):
@@ -51,8 +51,10 @@ def follow_trace(H, G, const, g, S0, swaps, gpu_obj, score_mode="independent", a
             delta = info.delta
         if accept == "improving":
             # the GPU accepted this swap: the oracle must agree unless the margin is tiny
+            # (delta is a difference of two scores, each known to about GAP relative: that sets the tie band)
             thr = -srch.eps_acc * srch.st.obj
-            assert delta <= thr or abs(delta - thr) <= GAP * srch.st.obj, f"step {step}: accepted a non-improving swap"
+            band = GAP * (abs(info.D[slot]) + abs(info.D[slot] - delta)) if info.D is not None else GAP * srch.st.obj
+            assert delta <= thr or abs(delta - thr) <= band, f"step {step}: accepted a non-improving swap"
         srch.apply(slot, j_in)
         assert gpu_obj[step + 1] == __import__("pytest").approx(srch.st.obj, rel=obj_rtol), f"step {step}: objective drifted"
     # after the GPU's last swap: it either hit max_swaps or stopped because the next swap did not improve
@@ -60,7 +62,9 @@ def follow_trace(H, G, const, g, S0, swaps, gpu_obj, score_mode="independent", a
         info = srch.propose(keep_scores=True)
         if info is not None and info.accepted:
             near_tie = info.gap_out <= GAP or info.gap_in <= GAP
-            assert info.accept_margin <= GAP or near_tie, \
+            Dsel = info.D[info.slot] if info.D is not None else srch.st.obj
+            band = GAP * (abs(Dsel) + abs(Dsel - info.delta))
+            assert abs(info.delta + srch.eps_acc * srch.st.obj) <= band or near_tie, \
                 f"GPU stopped but the oracle would go on (delta {info.delta}, obj {srch.st.obj})"
     elif gpu_stop == "max_swaps":
         assert len(swaps) == max_swaps

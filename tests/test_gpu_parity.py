@@ -153,7 +153,8 @@ def run_gpu_search(solver, wl, H, G, Wd, max_swaps, accept_always=False, S0=None
         support, obj0 = solver.init_support(H, G, Wd, wl.g, wl.k)
     else:
         support, obj0 = solver.init_support(H, G, Wd, wl.g, wl.k, mode=b.INIT_USER, support=torch.as_tensor(S0))
-    out = solver.local_search(max_swaps, accept_mode=b.ACCEPT_ALWAYS if accept_always else b.ACCEPT_IMPROVING)
+    out = solver.local_search(max_swaps, accept_mode=b.ACCEPT_ALWAYS if accept_always else b.ACCEPT_IMPROVING,
+                              accept_rel_tol=wl.eps_acc)
     return support.cpu().numpy(), obj0, out
 
 
@@ -170,7 +171,8 @@ def test_search_matches_oracle_given_H(solver, name, over, seed, max_swaps):
     assert np.array_equal(S0, S0o)
     swaps = [tuple(int(v) for v in r) for r in out.swap_trace.cpu().numpy()]
     gobj = out.obj_trace.cpu().numpy()
-    srch, rebased = follow_trace(Hr, Gr, const_r, wl.g, S0, swaps, gobj, gpu_stop=out.stop_reason, max_swaps=max_swaps)
+    srch, rebased = follow_trace(Hr, Gr, const_r, wl.g, S0, swaps, gobj, gpu_stop=out.stop_reason, max_swaps=max_swaps,
+                                 eps_acc=wl.eps_acc)
     S_or, W_or, _, _ = srch.result()
     assert np.array_equal(out.support.cpu().numpy(), S_or)                       # identical final support
     assert np.all(np.diff(gobj) < 0)                                             # accepted swaps lower obj
@@ -231,7 +233,8 @@ def test_end_to_end_from_X(solver, name, over, seed, max_swaps):
         assert np.all(np.abs(e[diff] - thr) <= GAP * thr)
     swaps = [tuple(int(v) for v in r) for r in out.swap_trace.cpu().numpy()]
     gobj = out.obj_trace.cpu().numpy()
-    srch, rebased = follow_trace(H64, G64, const64, wl.g, S0, swaps, gobj, gpu_stop=out.stop_reason, max_swaps=max_swaps)
+    srch, rebased = follow_trace(H64, G64, const64, wl.g, S0, swaps, gobj, gpu_stop=out.stop_reason, max_swaps=max_swaps,
+                                 eps_acc=wl.eps_acc)
     S_or, W_or, _, _ = srch.result()
     assert np.array_equal(out.support.cpu().numpy(), S_or)
     assert out.obj_final == pytest.approx(srch.st.obj, rel=1e-4)

@@ -43,6 +43,7 @@ class Workload:
     x_dtype: torch.dtype
     seed: int = 0
     damp: float = 0.0
+    eps_acc: float = 1e-5               # a swap is accepted iff it lowers obj by more than eps_acc * obj
     score_mode: str = "independent"     # or "pair_exact"
     w_std: float = 0.02
     chunk_rows: int = CHUNK_ROWS
@@ -154,10 +155,10 @@ def config(name: str, seed: int = 0, **over) -> Workload:
                       x_dtype=torch.float32, w_std=1.0 / 8.0, params={"mix": 0.3})
     elif name == "c2":    # OPT-1.3B-shaped FC2 neurons
         wl = Workload("c2", "fc2_relu", n=262144, d1=8192, m=2048, g=1, k=4096, max_swaps=2000,
-                      x_dtype=torch.bfloat16, damp=1e-2, params={"rank": 64, "rho": 1.0})
+                      x_dtype=torch.bfloat16, damp=1e-2, eps_acc=1e-7, params={"rank": 64, "rho": 1.0})
     elif name == "c3":    # OPT-2.7B-shaped attention heads
         wl = Workload("c3", "attn_heads", n=262144, d1=2560, m=2560, g=80, k=16, max_swaps=200,
-                      x_dtype=torch.bfloat16, damp=1e-2, score_mode="pair_exact",
+                      x_dtype=torch.bfloat16, damp=1e-2, eps_acc=1e-7, score_mode="pair_exact",
                       params={"corr": 0.5, "outlier_frac": 0.01, "outlier_scale": 20.0})
     elif name == "c4":    # ResNet50-shaped 3x3 conv input channels
         wl = Workload("c4", "conv_unfold", n=6272, d1=4608, m=512, g=9, k=256, max_swaps=500,
@@ -165,7 +166,7 @@ def config(name: str, seed: int = 0, **over) -> Workload:
                       chunk_rows=6272, params={"kh": 3, "kw": 3, "fh": 7, "fw": 7, "pad": 1})
     elif name == "c5":    # OPT-30B-shaped FC2 neurons with outlier channels
         wl = Workload("c5", "fc2_relu", n=262144, d1=28672, m=7168, g=1, k=8602, max_swaps=5000,
-                      x_dtype=torch.bfloat16, damp=1e-2,
+                      x_dtype=torch.bfloat16, damp=1e-2, eps_acc=1e-7,
                       params={"rank": 64, "rho": 1.0, "outlier_frac": 0.005, "outlier_scale": 30.0})
     else:
         raise ValueError(name)
