@@ -145,6 +145,29 @@ int osscar_objective(osscar_ctx* ctx, const float* H, const float* W, const floa
  * 6 add scores (double[d1/g-k]).  Scores are those of the last scoring pass. */
 int osscar_debug_get_state(osscar_ctx* ctx, int which, void* dst);
 
+/*
+ * Allocation-free trace reduction (the paper has no counterpart; this is a service entry point).
+ * *out = sum_ij A[i][j] * B[i][j] over rows x cols, in fp64 and in a fixed summation order -- for instance
+ * const = Tr(W^T G) or the identity obj = Tr(W_J^T R_J).  It is the two-stage reduction the library uses
+ * internally, except that its scratch (one double per row) is a fixed array inside the library image instead
+ * of memory from cudaMalloc.  It is meant for callers that must not allocate while they run: code that has
+ * already handed all free device memory to its own pool, real-time loops that cannot afford the device-wide
+ * synchronisation an allocation may cause, or plug-ins that are forbidden to change the memory footprint.
+ * It needs no context and calls neither cudaMalloc nor cudaFree nor any allocating library routine.
+ *   A, B: device fp32, row-major with leading dimensions lda, ldb >= cols.  out: host.
+ *   rows <= OSSCAR_NOALLOC_MAX_ROWS, else OSSCAR_E_SHAPE (the built-in scratch is 65536 + 32 doubles,
+ *   about 512 KB, resident on every GPU that loads the library until the process exits).
+ *   device: ordinal that owns A and B; cuda_stream: a cudaStream_t (NULL = legacy default stream).
+ * The first call on a device looks up the device address of the built-in array; make that call before any
+ * stream capture begins.  All calls share the array and it keeps the previous call's contents (each call
+ * overwrites every slot it later reads, so old contents never reach the result); calls whose kernels can
+ * overlap on the GPU -- different streams, different threads -- race on it and must be serialised by the caller.
+ * Synchronises the stream once, at its end.
+ */
+#define OSSCAR_NOALLOC_MAX_ROWS 65536
+int osscar_trace_noalloc(const float* A, int64_t lda, const float* B, int64_t ldb,
+                         int64_t rows, int64_t cols, int device, void* cuda_stream, double* out);
+
 const char* osscar_status_string(int status);
 
 /* Number of kernels this library has launched in this process so far (all contexts). */

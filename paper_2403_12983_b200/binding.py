@@ -22,7 +22,7 @@ STOP_NAMES = {0: "max_swaps", 1: "no_improvement", 2: "guard"}
 
 EXPORTS = ["osscar_create", "osscar_destroy", "osscar_workspace_bytes", "osscar_set_workspace",
            "osscar_gram", "osscar_init_support", "osscar_local_search", "osscar_objective",
-           "osscar_debug_get_state", "osscar_status_string", "osscar_launch_count"]
+           "osscar_debug_get_state", "osscar_status_string", "osscar_launch_count", "osscar_trace_noalloc"]
 
 
 class SearchParams(C.Structure):
@@ -75,6 +75,7 @@ def lib() -> C.CDLL:
     L.osscar_local_search.argtypes = [vp, C.POINTER(SearchParams), vp, vp, vp, vp, C.POINTER(SearchResult)]
     L.osscar_objective.argtypes = [vp, vp, vp, vp, i64, i64, C.POINTER(C.c_double)]
     L.osscar_debug_get_state.argtypes = [vp, C.c_int, vp]
+    L.osscar_trace_noalloc.argtypes = [vp, i64, vp, i64, i64, i64, C.c_int, vp, C.POINTER(C.c_double)]
     L.osscar_launch_count.restype = C.c_uint64
     L.osscar_launch_count.argtypes = []
     for name in EXPORTS:
@@ -97,6 +98,20 @@ def _dev_f32(t: torch.Tensor, name: str) -> torch.Tensor:
     if not (t.is_cuda and t.dtype == torch.float32 and t.is_contiguous()):
         raise ValueError(f"{name} must be a contiguous fp32 CUDA tensor")
     return t
+
+
+def osscar_trace_noalloc(A: torch.Tensor, B: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> float:
+    """sum(A * B) in fp64 through the allocation-free entry point (scratch built into the library; rows <= 65536).
+    For callers that may not allocate device memory; calls on one GPU must not overlap."""
+    if not (A.is_cuda and B.is_cuda and A.dtype == torch.float32 and B.dtype == torch.float32 and A.dim() == 2
+            and A.shape == B.shape and A.stride(1) == 1 and B.stride(1) == 1):
+        raise ValueError("A and B must be fp32 CUDA matrices of one shape with unit column stride")
+    dev = A.device.index
+    sptr = C.c_void_p((stream or torch.cuda.current_stream(dev)).cuda_stream)
+    out = C.c_double(0.0)
+    _check(lib().osscar_trace_noalloc(_ptr(A), A.stride(0), _ptr(B), B.stride(0), A.shape[0], A.shape[1], dev, sptr,
+                                      C.byref(out)), "osscar_trace_noalloc")
+    return out.value
 
 
 def launch_count() -> int:
