@@ -109,9 +109,10 @@ def reduce_over_ranks(values: dict, world: int, backend_device):
     return out
 
 
-def swap_bytes(nI, nJ, m):
-    """Algorithmic HBM bytes of one swap of the fused single-pass scheme (fp32)."""
-    return 4 * (3 * nI * nI + 2 * nI * m + 2 * nJ * m + nJ * nI)
+def swap_bytes(nI, nJ, m, fused_y=False):
+    """Algorithmic HBM bytes of one swap (fp32): Hinv read+write, V and R_J read+write, H[J,I] read once, and
+    the y = Hinv h pass (n_I^2 more) unless it is fused into the Hinv update."""
+    return 4 * ((2 if fused_y else 3) * nI * nI + 2 * nI * m + 2 * nJ * m + nJ * nI)
 
 
 KERNEL_BYTES = {   # algorithmic bytes per launch of the streaming kernels of a step
@@ -120,6 +121,9 @@ KERNEL_BYTES = {   # algorithmic bytes per launch of the streaming kernels of a 
     "update_hinv": lambda nI, nJ, m: 8 * nI * nI,
     "update_v": lambda nI, nJ, m: 8 * nI * m,
     "update_r": lambda nI, nJ, m: 8 * nJ * m,
+    "l1_hpass_update_v": lambda nI, nJ, m: 4 * nJ * nI + 8 * nI * m,
+    "l2_update_r_swap": lambda nI, nJ, m: 8 * nJ * m,
+    "l4_update_hinv_y": lambda nI, nJ, m: 8 * nI * nI,
 }
 
 
@@ -191,6 +195,9 @@ def run_ours(args):
     over = {}
     if args.tokens:
         over["n"] = args.tokens
+    for key in ("d1", "m", "k"):
+        if getattr(args, key) is not None:
+            over[key] = getattr(args, key)
     wl = workloads.config(args.workload, seed=rank, **over)
     max_swaps = args.max_swaps if args.max_swaps is not None else wl.max_swaps
     accept = b.ACCEPT_ALWAYS if args.accept_always else b.ACCEPT_IMPROVING
@@ -299,7 +306,8 @@ def run_ours(args):
     tm_, tn_ = -(-wl.d1 // 128), -(-wl.d1 // 256)
     tiles = sum(tn_ - t // 2 for t in range(tm_))
     gram_exec_tflops = 2.0 * 128 * 256 * tiles * wl.n / max(phase["gram"] / K * 1e-3, 1e-12) / 1e12
-    loop_gbs = swap_bytes(nI, nJ, m) * per_step_swaps / max(phase["search_loop"] / K * 1e-3, 1e-12) / 1e9
+    fused = wl.g == 1
+    loop_gbs = swap_bytes(nI, nJ, m, fused) * per_step_swaps / max(phase["search_loop"] / K * 1e-3, 1e-12) / 1e9
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -318,7 +326,7 @@ def run_ours(args):
         "gram": {"executed_tflops": gram_exec_tflops, "dense_equiv_tflops": 2.0 * wl.n * wl.d1 ** 2 / max(phase["gram"] / K * 1e-3, 1e-12) / 1e12,
                  "frac_of_bf16_peak": gram_exec_tflops / pk["bf16_tflops_sustained"], "peak": pk["bf16_tflops_sustained"],
                  "peak_source": pk["source"] + " (sustained)"},
-        "swap_loop": {"gbs": loop_gbs, "bytes_per_swap": swap_bytes(nI, nJ, m), "frac_of_hbm": loop_gbs / pk["hbm_gbs"],
+        "swap_loop": {"gbs": loop_gbs, "bytes_per_swap": swap_bytes(nI, nJ, m, fused), "frac_of_hbm": loop_gbs / pk["hbm_gbs"],
                       "peak": pk["hbm_gbs"], "peak_source": pk["source"]},
         "roofline": roof,
         "gpu_launches": int(launches),
@@ -345,6 +353,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c5")
     ap.add_argument("--tokens", type=int, default=None, help="override the number of calibration rows")
+    ap.add_argument("--d1", type=int, default=None, help="override the layer width (profiling cases)")
+    ap.add_argument("--m", type=int, default=None)
+    ap.add_argument("--k", type=int, default=None)
     ap.add_argument("--max-swaps", type=int, default=None)
     ap.add_argument("--accept-always", action="store_true", help="paper-literal fixed number of iterations")
     ap.add_argument("--no-e2e", action="store_true")

@@ -38,6 +38,8 @@ class SearchResult(C.Structure):
 
 STEP_KERNELS = ["select", "pair_grams", "y_pass", "small_algebra", "staging", "h_pass", "update_hinv", "update_v",
                 "update_r", "group_scores", "h_swap_rows", "h_swap_cols"]
+# single-row groups run a fused five-launch step
+STEP_KERNELS_G1 = ["decide", "l1_hpass_update_v", "l2_update_r_swap", "select_in", "l4_update_hinv_y"]
 
 
 class OsscarError(RuntimeError):
@@ -239,7 +241,8 @@ class Solver:
         return SearchOutput(support, W_out, obj_trace[:n + 1], swap_trace[:2 * n].view(n, 2), n,
                             STOP_NAMES.get(res.stop_reason, str(res.stop_reason)), res.n_refresh,
                             res.obj_init, res.obj_final, res.ms_search,
-                            {n: res.ms_kernel[i] for i, n in enumerate(STEP_KERNELS)} if res.n_profiled > 0 else {})
+                            {n: res.ms_kernel[i] for i, n in enumerate(STEP_KERNELS_G1 if g == 1 else STEP_KERNELS)}
+                            if res.n_profiled > 0 else {})
 
     def objective(self, H, W, Wt) -> float:
         _dev_f32(H, "H"); _dev_f32(W, "W"); _dev_f32(Wt, "Wt")

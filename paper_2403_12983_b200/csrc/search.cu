@@ -657,6 +657,8 @@ __global__ void k_begin(SearchCtl* ctl, double* obj_trace, int32_t* done_host)
 __global__ void k_count_refresh(SearchCtl* ctl) { if (!ctl->done) ctl->n_refresh += 1; }
 __global__ void k_final_obj(SearchCtl* ctl) { ctl->acc[3] = ctl->const_term - ctl->acc[1]; }
 
+#include "search_g1.cuh"
+
 Ptrs make_ptrs(osscar_ctx* ctx)
 {
     const Layout& L = ctx->L;
@@ -732,6 +734,14 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
     CK(cudaGetLastError());
     CK(cudaEventRecord(ctx->ev0, st));
     if (max_swaps > 0) CK(enqueue_scores(ctx, p, true));
+    auto bootstrap_g1 = [&]() -> cudaError_t {       // score vectors, first entering group and its y from the current state
+        k_scores_g1<<<(unsigned)((L.d1 + 255) / 256), 256, 0, st>>>(p);
+        k_select_in_g1<<<1, 1024, 0, st>>>(p);
+        k_ypass<<<dim3((unsigned)((L.nI + 7) / 8), 1), 256, 0, st>>>(p);
+        count_launches(3);
+        return cudaGetLastError();
+    };
+    if (max_swaps > 0 && g == 1) CK(bootstrap_g1());
 
     const int batch = 32;
     cudaEvent_t evb[2];
@@ -766,32 +776,45 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
             k_count_refresh<<<1, 1, 0, st>>>(ctx->ctl);
             count_launches(1);
             if (enqueue_scores(ctx, p, true) != cudaSuccess) { rc = OSSCAR_E_CUDA; break; }
+            if (g == 1 && bootstrap_g1() != cudaSuccess) { rc = OSSCAR_E_CUDA; break; }
         }
         cudaEvent_t* pe = nullptr;
         if (next_prof < nprof && prof_it[next_prof] == it) pe = evp[next_prof++];
         int slot = 0;
         auto mark = [&]() { if (pe) cudaEventRecord(pe[slot], st); ++slot; };
         mark();
-        k_select<<<1, 1024, 0, st>>>(p);                                                         mark();
-        k_pairgram<<<(unsigned)((3 * g * g + 7) / 8), 256, 0, st>>>(p);                          mark();
-        k_ypass<<<dim3(yblocks, g), 256, 0, st>>>(p);                                            mark();
-        k_small<<<1, 256, 0, st>>>(p, prm->accept_mode, tol, max_swaps, obj_trace, swap_trace);  mark();
-        k_prep<<<prep_blocks, 256, 0, st>>>(p);                                                  mark();
-        k_hpass<RPW><<<dim3(hblocks, g), 256, 0, st>>>(p);                                       mark();
-        k_update_hinv<<<dim3((unsigned)((L.ldh / 4 + 255) / 256), (unsigned)((L.nI + HI_RT - 1) / HI_RT)), 256, 0, st>>>(p);
-        mark();
-        k_update_rows<<<(unsigned)((L.nI + UP_ROWS - 1) / UP_ROWS), 256, 0, st>>>(p, 0);          mark();
-        k_update_rows<<<(unsigned)((L.nJ + UP_ROWS - 1) / UP_ROWS), 256, 0, st>>>(p, 1);          mark();
-        count_launches(9);
-        if (g > 1) {
-            k_update_c<<<(unsigned)(L.ng - L.k), 128, 0, st>>>(p);
-            count_launches(1);
-            if (enqueue_scores(ctx, p, false) != cudaSuccess) { rc = OSSCAR_E_CUDA; break; }
+        if (g == 1) {
+            // single-row groups: decide, {H pass || V}, {R || slot exchange}, next entering group, {Hinv + next y}
+            const unsigned nbV = (unsigned)((L.nI + 7) / 8), nbH = (unsigned)((L.nJ + 1 + 7) / 8);
+            const unsigned nbR = (unsigned)((L.nJ + 7) / 8);
+            k_decide_g1<<<1, 1024, 0, st>>>(p, prm->accept_mode, tol, obj_trace, swap_trace);   mark();
+            k_l1_g1<<<nbV + nbH, 256, 0, st>>>(p, nbV);                                          mark();
+            k_l2_g1<<<nbR + 32, 256, 0, st>>>(p, nbR);                                           mark();
+            k_select_in_g1<<<1, 1024, 0, st>>>(p);                                               mark();
+            k_l4_g1<<<nbV, 256, 0, st>>>(p);                                                     mark();
+            count_launches(5);
+        } else {
+            k_select<<<1, 1024, 0, st>>>(p);                                                         mark();
+            k_pairgram<<<(unsigned)((3 * g * g + 7) / 8), 256, 0, st>>>(p);                          mark();
+            k_ypass<<<dim3(yblocks, g), 256, 0, st>>>(p);                                            mark();
+            k_small<<<1, 256, 0, st>>>(p, prm->accept_mode, tol, max_swaps, obj_trace, swap_trace);  mark();
+            k_prep<<<prep_blocks, 256, 0, st>>>(p);                                                  mark();
+            k_hpass<RPW><<<dim3(hblocks, g), 256, 0, st>>>(p);                                       mark();
+            k_update_hinv<<<dim3((unsigned)((L.ldh / 4 + 255) / 256), (unsigned)((L.nI + HI_RT - 1) / HI_RT)), 256, 0, st>>>(p);
+            mark();
+            k_update_rows<<<(unsigned)((L.nI + UP_ROWS - 1) / UP_ROWS), 256, 0, st>>>(p, 0);          mark();
+            k_update_rows<<<(unsigned)((L.nJ + UP_ROWS - 1) / UP_ROWS), 256, 0, st>>>(p, 1);          mark();
+            count_launches(9);
+            if (g > 1) {
+                k_update_c<<<(unsigned)(L.ng - L.k), 128, 0, st>>>(p);
+                count_launches(1);
+                if (enqueue_scores(ctx, p, false) != cudaSuccess) { rc = OSSCAR_E_CUDA; break; }
+            }
+            mark();
+            k_hswap<<<(unsigned)((L.ldp * g + 255) / 256), 256, 0, st>>>(p, 0);                       mark();
+            k_hswap<<<(unsigned)((L.ldp * g + 255) / 256), 256, 0, st>>>(p, 1);                       mark();
+            count_launches(2);
         }
-        mark();
-        k_hswap<<<(unsigned)((L.ldp * g + 255) / 256), 256, 0, st>>>(p, 0);                       mark();
-        k_hswap<<<(unsigned)((L.ldp * g + 255) / 256), 256, 0, st>>>(p, 1);                       mark();
-        count_launches(2);
         if (cudaGetLastError() != cudaSuccess) { rc = OSSCAR_E_CUDA; break; }
         if ((it + 1) % batch == 0) {
             if (cudaEventRecord(evb[(it / batch) & 1], st) != cudaSuccess) { rc = OSSCAR_E_CUDA; break; }

@@ -1,0 +1,376 @@
+// Swap step for single-row groups (g = 1): five launches per swap, each matrix streamed once.
+// Included by search.cu (same translation unit: uses its Ptrs, reductions and small-matrix slots).
+//
+//   decide      one block: i* = argmin D, exact change of obj, accept test, staged vectors b, u2, K, Vq
+//   L1          H pass (u_l, d_l for every pruned row and the leaving row)  ||  V update + drop scores D
+//   L2          R update + Schur complements + add scores A                 ||  slot exchange in Hp
+//   select_in   q* = argmax A for the NEXT step
+//   L4          Hinv update fused with y_next = Hinv' * Hp[q_next, 0:n_I]^T (the next step's y pass)
+//
+// Scalars of a step live in p.small (doubles): [S_CINV] = 1/C, [S_C1INV] = 1/c1, [G1_Q1] = P/C,
+// [G1_M2] = P/(C c1), [G1_HDIAG] = H diagonal entry of the leaving row.
+#pragma once
+
+constexpr int G1_Q1 = 2, G1_M2 = 3, G1_HDIAG = 4;
+
+__device__ __forceinline__ void fma4(float4& v, float a, const float4& x) {
+    v.x = fmaf(a, x.x, v.x); v.y = fmaf(a, x.y, v.y); v.z = fmaf(a, x.z, v.z); v.w = fmaf(a, x.w, v.w);
+}
+__device__ __forceinline__ float dot4(const float4& a, const float4& b) {
+    return a.x * b.x + a.y * b.y + a.z * b.z + a.w * b.w;
+}
+
+// D[s] = ||V_s||^2 / Hinv_ss and A[t] = ||R_t||^2 / c_t from the row norms (start of a search / after a refresh).
+__global__ void k_scores_g1(Ptrs p)
+{
+    if (p.ctl->done) return;
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < p.nI) {
+        const double hd = p.Hinv[i * p.ldh + i];
+        p.D[i] = hd > 0.0 ? (double)p.vnorm[i] / hd : INFINITY;
+    } else if (i < p.nI + p.nJ) {
+        const int64_t t = i - p.nI;
+        const double cc = p.c[t];
+        const double hd = p.Hp[(p.nI + t) * p.ldp + p.nI + t];
+        p.A[t] = cc > kAddPivotTol * hd ? (double)p.rnorm[t] / cc : -INFINITY;
+    }
+}
+
+// Block-wide arg-min of val[i] (ties -> smaller group id); result broadcast through shared memory.
+__device__ void block_argmin(const double* __restrict__ val, const int32_t* __restrict__ ids, int n, bool negate,
+                             double* best_out, int* idx_out)
+{
+    __shared__ double sv[32]; __shared__ int sid[32]; __shared__ int sidx[32];
+    const int t = threadIdx.x, lane = t & 31, w = t >> 5;
+    double best = INFINITY; int bid = INT_MAX, bidx = -1;
+    for (int i0 = t; i0 < n; i0 += 4 * blockDim.x) {          // four independent loads in flight per thread
+        double vv[4]; int ii[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int i = i0 + j * blockDim.x;
+            vv[j] = i < n ? val[i] : (negate ? -INFINITY : INFINITY);
+            ii[j] = i < n ? ids[i] : INT_MAX;
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int i = i0 + j * blockDim.x;
+            const double v = negate ? -vv[j] : vv[j];
+            if (i < n && (v < best || (v == best && ii[j] < bid))) { best = v; bid = ii[j]; bidx = i; }
+        }
+    }
+    for (int o = 16; o > 0; o >>= 1) {
+        const double ov = __shfl_xor_sync(0xffffffffu, best, o);
+        const int oid = __shfl_xor_sync(0xffffffffu, bid, o);
+        const int oidx = __shfl_xor_sync(0xffffffffu, bidx, o);
+        if (ov < best || (ov == best && oid < bid)) { best = ov; bid = oid; bidx = oidx; }
+    }
+    __syncthreads();
+    if (lane == 0) { sv[w] = best; sid[w] = bid; sidx[w] = bidx; }
+    __syncthreads();
+    if (t == 0) {
+        for (int i = 1; i < (int)(blockDim.x >> 5); ++i)
+            if (sv[i] < best || (sv[i] == best && sid[i] < bid)) { best = sv[i]; bid = sid[i]; bidx = sidx[i]; }
+        sv[0] = best; sidx[0] = bidx;
+    }
+    __syncthreads();
+    *best_out = negate ? -sv[0] : sv[0];
+    *idx_out = sidx[0];
+    __syncthreads();
+}
+
+// q* = argmax A (the group that enters at the next step).
+__global__ void __launch_bounds__(1024) k_select_in_g1(Ptrs p)
+{
+    SearchCtl* ctl = p.ctl;
+    if (ctl->done) return;
+    double best; int idx;
+    block_argmin(p.A, p.perm + p.k, (int)p.nJ, true, &best, &idx);
+    if (threadIdx.x == 0) {
+        ctl->sel_t = idx;
+        if (idx < 0 || !isfinite(best)) { ctl->done = 1; ctl->stop_reason = OSSCAR_STOP_GUARD; *p.done_host = 1; }
+    }
+}
+
+// One block: leaving row, exact change of obj, accept test, traces, staged vectors.
+__global__ void __launch_bounds__(1024)
+k_decide_g1(Ptrs p, int accept_mode, double accept_tol, double* __restrict__ obj_trace, int32_t* __restrict__ swap_trace)
+{
+    SearchCtl* ctl = p.ctl;
+    if (ctl->done) return;
+    __shared__ float redf[32];
+    __shared__ int s_stop;
+    double Dbest; int slot;
+    block_argmin(p.D, p.perm, p.k, false, &Dbest, &slot);
+    const int64_t t = ctl->sel_t;
+    if (slot < 0 || !isfinite(Dbest)) {
+        if (threadIdx.x == 0) { ctl->done = 1; ctl->stop_reason = OSSCAR_STOP_GUARD; *p.done_host = 1; }
+        return;
+    }
+    const int64_t r0 = slot;
+    // cross term V_r . R_q
+    const float4* vr = reinterpret_cast<const float4*>(p.V + r0 * p.ldm);
+    const float4* rq = reinterpret_cast<const float4*>(p.R + t * p.ldm);
+    float acc = 0.f;
+    for (int64_t c = threadIdx.x; c < p.ldm / 4; c += blockDim.x) acc += dot4(vr[c], rq[c]);
+    const double GX = (double)block_sum_f(acc, redf);
+    if (threadIdx.x == 0) {
+        const double C = p.Hinv[r0 * p.ldh + r0], P = p.y[r0], cq = p.c[t];
+        const double GV = p.vnorm[r0], GR = p.rnorm[t];
+        const double Cinv = 1.0 / C;
+        const double Ds = GV * Cinv;
+        const double RR1 = GR + 2.0 * P * Cinv * GX + P * P * Cinv * Cinv * GV;
+        const double c1 = cq + P * P * Cinv;
+        const double c1inv = 1.0 / c1;
+        const double delta = Ds - c1inv * RR1;
+        const double obj = ctl->obj;
+        bool stop = false; int reason = 0;
+        if (!(C > 0.0) || !(c1 > 0.0) || !isfinite(delta)) { stop = true; reason = OSSCAR_STOP_GUARD; }
+        else if (accept_mode == OSSCAR_ACCEPT_IMPROVING && !(delta <= -accept_tol * obj)) { stop = true; reason = OSSCAR_STOP_NO_IMPROVEMENT; }
+        ctl->delta = delta; ctl->sel_D = Ds; ctl->sel_slot = slot;
+        if (stop) { ctl->done = 1; ctl->stop_reason = reason; *p.done_host = 1; }
+        else {
+            const int n = ctl->n_swaps;
+            swap_trace[2 * n] = p.perm[slot];
+            swap_trace[2 * n + 1] = p.perm[p.k + t];
+            obj_trace[n + 1] = obj + delta;
+            ctl->obj = obj + delta;
+            ctl->n_swaps = n + 1;
+            p.small[S_CINV] = Cinv; p.small[S_C1INV] = c1inv;
+            p.small[G1_Q1] = Cinv * P; p.small[G1_M2] = c1inv * P * Cinv;
+            p.small[G1_HDIAG] = p.Hp[r0 * p.ldp + r0];
+        }
+        s_stop = stop;
+    }
+    __syncthreads();
+    if (s_stop) return;
+    const float Q1 = (float)p.small[G1_Q1];
+    const double Cinv = p.small[S_CINV], c1inv = p.small[S_C1INV], M2 = p.small[G1_M2];
+    const float* hrow = p.Hinv + r0 * p.ldh;
+    // float4 wide (pads of Hinv rows, y, V, R are zero, so the padded tails stay zero)
+    const float4* hrow4 = reinterpret_cast<const float4*>(hrow);
+    const float4* y4 = reinterpret_cast<const float4*>(p.y);
+    float4* b4 = reinterpret_cast<float4*>(p.b);
+    float4* u4 = reinterpret_cast<float4*>(p.u2);
+    for (int64_t c = threadIdx.x; c < p.ldh / 4; c += blockDim.x) {
+        const float4 bs = hrow4[c], yy = y4[c];
+        float4 uu = make_float4(fmaf(-bs.x, Q1, yy.x), fmaf(-bs.y, Q1, yy.y), fmaf(-bs.z, Q1, yy.z), fmaf(-bs.w, Q1, yy.w));
+        const int64_t rc = r0 - c * 4;
+        uu.x = rc == 0 ? 0.f : uu.x; uu.y = rc == 1 ? 0.f : uu.y; uu.z = rc == 2 ? 0.f : uu.z; uu.w = rc == 3 ? 0.f : uu.w;
+        b4[c] = bs;
+        u4[c] = uu;
+    }
+    const float4* v4 = reinterpret_cast<const float4*>(p.V + r0 * p.ldm);
+    const float4* r4 = reinterpret_cast<const float4*>(p.R + t * p.ldm);
+    float4* k4 = reinterpret_cast<float4*>(p.K);
+    float4* q4 = reinterpret_cast<float4*>(p.Vq);
+    const float fC = (float)Cinv, fc1 = (float)c1inv, fM2 = (float)M2;
+    for (int64_t c = threadIdx.x; c < p.ldm / 4; c += blockDim.x) {
+        const float4 v = v4[c], r = r4[c];
+        k4[c] = make_float4(fC * v.x, fC * v.y, fC * v.z, fC * v.w);
+        q4[c] = make_float4(fmaf(fc1, r.x, fM2 * v.x), fmaf(fc1, r.y, fM2 * v.y), fmaf(fc1, r.z, fM2 * v.z), fmaf(fc1, r.w, fM2 * v.w));
+    }
+}
+
+// Row update M'[s] = M[s] + ck_s K + cq_s Vq with the squared norm of the new row: one warp per row, eight
+// 16-byte loads in flight per lane, K and Vq re-read through L1.  kind 0: V (ck = -b_s, cq = -u2_s, row r0 := Vq,
+// D' written), kind 1: R (ck = u_l, cq = -d_l, row of the entering slot := K - d_r Vq, c' and A' written).
+constexpr int G1_U = 8;
+__device__ __forceinline__ void update_row_g1(const Ptrs& p, int kind, int64_t s)
+{
+    const int lane = threadIdx.x & 31;
+    float* M = kind == 0 ? p.V : p.R;
+    const int64_t special = kind == 0 ? (int64_t)p.ctl->sel_slot : (int64_t)p.ctl->sel_t;
+    const int64_t n4 = p.ldm / 4;
+    const float4* K4 = reinterpret_cast<const float4*>(p.K);
+    const float4* Q4 = reinterpret_cast<const float4*>(p.Vq);
+    float4* row = reinterpret_cast<float4*>(M + s * p.ldm);
+    const bool sp = s == special;
+    float ck, cq;
+    if (kind == 0) { ck = -p.b[s]; cq = -p.u2[s]; }
+    else { ck = p.u[s]; cq = -p.d[s]; }
+    const float dr = kind == 1 ? p.d[p.nJ] : 0.f;
+    if (sp) { ck = kind == 0 ? 0.f : 1.f; cq = kind == 0 ? 1.f : -dr; }      // new row = ck K + cq Vq
+    float nrm = 0.f;
+    for (int64_t c0 = lane; c0 < n4; c0 += 32 * G1_U) {
+        float4 v[G1_U];
+#pragma unroll
+        for (int j = 0; j < G1_U; ++j) {
+            const int64_t c = c0 + 32 * j;
+            if (!sp && c < n4) v[j] = row[c];
+            else v[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int j = 0; j < G1_U; ++j) {
+            const int64_t c = c0 + 32 * j;
+            if (c < n4) {
+                fma4(v[j], ck, __ldg(K4 + c));
+                fma4(v[j], cq, __ldg(Q4 + c));
+                row[c] = v[j];
+                nrm += dot4(v[j], v[j]);
+            }
+        }
+    }
+    nrm = warp_sum(nrm);
+    if (lane == 0) {
+        const double Cinv = p.small[S_CINV], c1inv = p.small[S_C1INV];
+        if (kind == 0) {
+            p.vnorm[s] = nrm;
+            double hd;
+            if (sp) hd = c1inv;
+            else {
+                const double bs = p.b[s], us = p.u2[s];
+                hd = (double)p.Hinv[s * p.ldh + s] - bs * bs * Cinv + us * us * c1inv;
+            }
+            p.D[s] = hd > 0.0 ? (double)nrm / hd : INFINITY;
+        } else {
+            p.rnorm[s] = nrm;
+            double cc, hd;
+            if (sp) { cc = Cinv - (double)dr * (double)dr * c1inv; hd = p.small[G1_HDIAG]; }
+            else {
+                const double uu = p.u[s], dd = p.d[s];
+                cc = p.c[s] + uu * uu * Cinv - dd * dd * c1inv;
+                hd = p.Hp[(p.nI + s) * p.ldp + p.nI + s];
+            }
+            p.c[s] = cc;
+            p.A[s] = cc > kAddPivotTol * hd ? (double)nrm / cc : -INFINITY;
+        }
+    }
+}
+
+// u_l = Hp[l, 0:n_I] . b and d_l = Hp[l, q] - Hp[l, 0:n_I] . u2 for pruned row l (l = n_J: the leaving row);
+// one warp per row.
+__device__ __forceinline__ void hpass_row_g1(const Ptrs& p, int64_t l)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t hrow = l < p.nJ ? p.nI + l : (int64_t)p.ctl->sel_slot;
+    const int64_t qcol = p.nI + (int64_t)p.ctl->sel_t;
+    const float4* row = reinterpret_cast<const float4*>(p.Hp + hrow * p.ldp);
+    const float4* bv = reinterpret_cast<const float4*>(p.b);
+    const float4* uv = reinterpret_cast<const float4*>(p.u2);
+    const int64_t n4 = p.ldh / 4;
+    float au = 0.f, ad = 0.f;
+    for (int64_t c0 = lane; c0 < n4; c0 += 32 * G1_U) {
+        float4 x[G1_U];
+#pragma unroll
+        for (int j = 0; j < G1_U; ++j) {
+            const int64_t c = c0 + 32 * j;
+            x[j] = c < n4 ? row[c] : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int j = 0; j < G1_U; ++j) {
+            const int64_t c = c0 + 32 * j;
+            if (c < n4) { au += dot4(x[j], __ldg(bv + c)); ad += dot4(x[j], __ldg(uv + c)); }
+        }
+    }
+    au = warp_sum(au); ad = warp_sum(ad);
+    if (lane == 0) {
+        p.u[l] = au;
+        p.d[l] = reinterpret_cast<const float*>(row)[qcol] - ad;
+    }
+}
+
+// L1: blocks [0, nbV) update V (one row per warp), the rest run the H pass (one row per warp).
+__global__ void __launch_bounds__(256) k_l1_g1(Ptrs p, unsigned nbV)
+{
+    if (p.ctl->done) return;
+    const int w = threadIdx.x >> 5;
+    if (blockIdx.x < nbV) {
+        const int64_t s = (int64_t)blockIdx.x * 8 + w;
+        if (s < p.nI) update_row_g1(p, 0, s);
+    } else {
+        const int64_t l = (int64_t)(blockIdx.x - nbV) * 8 + w;
+        if (l < p.nJ + 1) hpass_row_g1(p, l);
+    }
+}
+
+// Exchange of the leaving kept slot a and the entering pruned slot b in Hp (rows and columns) and in the
+// slot permutation.  Work item ranges: [0, ldp) the two rows, [ldp, 2 ldp) the two columns.
+__device__ __forceinline__ void hswap_g1(const Ptrs& p, int64_t idx, int64_t stride)
+{
+    const int64_t a = p.ctl->sel_slot, b = p.nI + (int64_t)p.ctl->sel_t;
+    const int64_t d1 = p.nI + p.nJ;
+    for (; idx < 2 * p.ldp; idx += stride) {
+        if (idx < p.ldp) {
+            const int64_t x = idx;
+            if (x == a) {           // the 2 x 2 intersection, one thread: new[a][a]=old[b][b], new[a][b]=old[b][a], ...
+                const float aa = p.Hp[a * p.ldp + a], ab = p.Hp[a * p.ldp + b], ba = p.Hp[b * p.ldp + a], bb = p.Hp[b * p.ldp + b];
+                p.Hp[a * p.ldp + a] = bb; p.Hp[a * p.ldp + b] = ba; p.Hp[b * p.ldp + a] = ab; p.Hp[b * p.ldp + b] = aa;
+            } else if (x != b) {
+                const float va = p.Hp[a * p.ldp + x], vb = p.Hp[b * p.ldp + x];
+                p.Hp[a * p.ldp + x] = vb; p.Hp[b * p.ldp + x] = va;
+            }
+        } else {
+            const int64_t x = idx - p.ldp;
+            if (x < d1 && x != a && x != b) {
+                const float va = p.Hp[x * p.ldp + a], vb = p.Hp[x * p.ldp + b];
+                p.Hp[x * p.ldp + a] = vb; p.Hp[x * p.ldp + b] = va;
+            }
+        }
+    }
+}
+
+// L2: blocks [0, nbR) update R (+ c, A), one row per warp; the remaining blocks exchange the two slots in Hp.
+__global__ void __launch_bounds__(256) k_l2_g1(Ptrs p, unsigned nbR)
+{
+    if (p.ctl->done) return;
+    if (blockIdx.x < nbR) {
+        const int64_t s = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+        if (s < p.nJ) update_row_g1(p, 1, s);
+        return;
+    }
+    const int64_t nsw = gridDim.x - nbR;
+    hswap_g1(p, (int64_t)(blockIdx.x - nbR) * blockDim.x + threadIdx.x, nsw * blockDim.x);
+    if (blockIdx.x == nbR && threadIdx.x == 0) {
+        const int s = p.ctl->sel_slot, t = p.k + p.ctl->sel_t;
+        const int gi = p.perm[s], gj = p.perm[t];
+        p.perm[s] = gj; p.perm[t] = gi;
+        p.slotof[gj] = s; p.slotof[gi] = t;
+    }
+}
+
+// L4: Hinv' = Hinv - (b/C) b^T + (u2/c1) u2^T (row and column r0: -u2/c1, corner 1/c1) and, in the same pass,
+// y_next = Hinv' h with h = Hp[row of the next entering group, 0:n_I].  One warp per row.
+__global__ void __launch_bounds__(256, 4) k_l4_g1(Ptrs p)
+{
+    if (p.ctl->done) return;
+    const int lane = threadIdx.x & 31;
+    const int64_t s = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (s >= p.nI) return;
+    const int64_t r0 = p.ctl->sel_slot;
+    const float Cinv = (float)p.small[S_CINV], c1inv = (float)p.small[S_C1INV];
+    const float4* b4 = reinterpret_cast<const float4*>(p.b);
+    const float4* u4 = reinterpret_cast<const float4*>(p.u2);
+    const float4* h4 = reinterpret_cast<const float4*>(p.Hp + (p.nI + (int64_t)p.ctl->sel_t) * p.ldp);
+    float4* row = reinterpret_cast<float4*>(p.Hinv + s * p.ldh);
+    const bool srow = s == r0;
+    // row r0 becomes -u2/c1: treat it as 0 * old - 0 * b + (-1/c1) * u2
+    const float nb = srow ? 0.f : -p.b[s] * Cinv;
+    const float us = srow ? -c1inv : p.u2[s] * c1inv;
+    const float corner = srow ? c1inv : -us;           // value of column r0 in this row
+    const int64_t n4 = p.ldh / 4;
+    float yacc = 0.f;
+    for (int64_t c0 = lane; c0 < n4; c0 += 32 * G1_U) {
+        float4 h[G1_U];
+#pragma unroll
+        for (int j = 0; j < G1_U; ++j) {
+            const int64_t c = c0 + 32 * j;
+            if (!srow && c < n4) h[j] = row[c];
+            else h[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int j = 0; j < G1_U; ++j) {
+            const int64_t c = c0 + 32 * j;
+            if (c < n4) {
+                fma4(h[j], nb, __ldg(b4 + c));
+                fma4(h[j], us, __ldg(u4 + c));
+                const int64_t rc = r0 - c * 4;           // position of column r0 inside this float4, if any
+                h[j].x = rc == 0 ? corner : h[j].x; h[j].y = rc == 1 ? corner : h[j].y;
+                h[j].z = rc == 2 ? corner : h[j].z; h[j].w = rc == 3 ? corner : h[j].w;
+                row[c] = h[j];
+                yacc += dot4(h[j], __ldg(h4 + c));
+            }
+        }
+    }
+    yacc = warp_sum(yacc);
+    if (lane == 0) p.y[s] = yacc;
+}
