@@ -120,7 +120,8 @@ typedef struct {
  * Swap search (Section 3.2: Eq. local with t_hat = 2, p_hat = 0; scores of Eq. impact;
  * state moved by Cases 1-3 of Proposition 1).  Each step scores every kept group (rise of
  * obj if dropped) and every pruned group (fall of obj if added), takes the cheapest drop and
- * the most valuable add (PAIR_EXACT: the best exact pair), computes the exact change of obj
+ * the most valuable add (PAIR_EXACT: the pair with the best exact change among all k * (d1/g - k) pairs,
+ * which must not exceed 2^20, else OSSCAR_E_SHAPE), computes the exact change of obj
  * for that pair, applies the accept rule and updates the state; the loop runs on the device
  * with no host round trip per swap.
  * support_out: device int32[k] (sorted).  W_out: device d1 x m fp32, rows of pruned groups

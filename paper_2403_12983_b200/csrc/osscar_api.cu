@@ -206,6 +206,7 @@ int osscar_local_search(osscar_ctx* ctx, const osscar_search_params* params,
     if (params->accept_mode != OSSCAR_ACCEPT_IMPROVING && params->accept_mode != OSSCAR_ACCEPT_ALWAYS) return OSSCAR_E_ARG;
     if (params->refresh_every < 0 || params->profile_samples < 0 || params->profile_samples > 8 || params->reserved != 0) return OSSCAR_E_ARG;
     if (!ctx->have_state) return OSSCAR_E_STATE;
+    if (params->score_mode == OSSCAR_SCORE_PAIR_EXACT && ctx->L.nJ > 0 && ctx->L.pair_capacity == 0) return OSSCAR_E_SHAPE;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return OSSCAR_E_CUDA;
     memset(result, 0, sizeof(*result));

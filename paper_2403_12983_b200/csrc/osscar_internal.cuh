@@ -8,6 +8,7 @@
 namespace osscar {
 
 constexpr int kTracePartials = 1184;   // blocks of a trace reduction; the context owns that many doubles
+constexpr int64_t kMaxPairs = 1 << 20;     // PAIR_EXACT scores at most this many (kept, pruned) pairs per step
 constexpr int kPadF = 32;   // leading dimensions of internal fp32 matrices are padded to this many floats
 
 extern unsigned long long g_launches;      // kernels launched by the library (host-side count)
@@ -46,6 +47,8 @@ struct Layout {
     size_t off_vec_begin, off_vec_end;   // the staged vectors (zeroed once when the state is built)
     size_t off_vnorm, off_rnorm, off_D, off_A, off_c, off_small, off_gramV, off_gramR;
     size_t off_perm, off_slotof, off_energy, off_panel;
+    size_t off_pairCinv, off_pairKK, off_pairScratch, off_pairDelta;   // PAIR_EXACT scoring
+    int64_t pair_capacity;                                             // pairs the workspace can score
     size_t bytes;
 };
 int make_layout(int64_t d1, int64_t m, int32_t g, int32_t k, Layout* L);

@@ -43,6 +43,7 @@ __device__ float block_sum_f(float v, float* red) {      // result in every thre
 struct Ptrs {
     float *Hp, *Hinv, *V, *R, *y, *b, *u2, *bC, *u2c, *u, *d, *K, *Vq, *vnorm, *rnorm;
     double *D, *A, *c, *small, *gramV, *gramR;
+    double *pairCinv, *pairKK, *pairScratch, *pairDelta;     // PAIR_EXACT scoring
     int32_t *perm, *slotof;
     SearchCtl* ctl;
     int32_t* done_host;
@@ -657,6 +658,116 @@ __global__ void k_begin(SearchCtl* ctl, double* obj_trace, int32_t* done_host)
 __global__ void k_count_refresh(SearchCtl* ctl) { if (!ctl->done) ctl->n_refresh += 1; }
 __global__ void k_final_obj(SearchCtl* ctl) { ctl->acc[3] = ctl->const_term - ctl->acc[1]; }
 
+// ------------------------------------------------------------------ exhaustive pair scoring (PAIR_EXACT)
+// For every kept slot s and pruned slot t the exact change of obj of swapping them (Case 3 = Case 1 then Case 2):
+//   delta(s,t) = D_s - Tr(c1^-1 R1 R1^T),  P = Pm[t-rows, s-cols] with Pm = Hp[J,I] Hinv,  T1 = P C_s^-1,
+//   c1 = c_t + T1 P^T,  R1 R1^T = GR_t + T1 GX + (T1 GX)^T + P (C_s^-1 GV_s C_s^-1) P^T,  GX = V_s R_t^T.
+constexpr int kPairBlocks = 296;
+constexpr int kPairTemps = 8;
+
+// Per kept slot: C_s^-1, KK_s = C_s^-1 GV_s C_s^-1 and D_s (block per slot; dynamic smem 3 g^2 doubles).
+__global__ void k_pair_slots(Ptrs p)
+{
+    if (p.ctl->done) return;
+    extern __shared__ double smd[];
+    __shared__ double red[32];
+    const int g = p.g, gg = g * g;
+    double* M = smd; double* Lw = smd + gg; double* T = Lw + gg;
+    const int64_t s = blockIdx.x;
+    double* Cinv = p.pairCinv + s * gg;
+    double* KK = p.pairKK + s * gg;
+    for (int idx = threadIdx.x; idx < gg; idx += blockDim.x) {
+        const int i = idx / g, j = idx % g;
+        M[idx] = 0.5 * ((double)p.Hinv[(s * g + i) * p.ldh + s * g + j] + (double)p.Hinv[(s * g + j) * p.ldh + s * g + i]);
+    }
+    __syncthreads();
+    const double piv = chol_inverse(M, Lw, Cinv, g);
+    const double* GV = p.gramV + s * gg;
+    mat_mul(Cinv, false, GV, false, T, g);
+    mat_mul(T, false, Cinv, false, KK, g);
+    const double tr = mat_trace_prod(Cinv, GV, g, red);
+    if (threadIdx.x == 0) p.D[s] = piv > 0.0 ? tr : INFINITY;
+}
+
+__global__ void __launch_bounds__(256)
+k_pair_delta(Ptrs p, const float* __restrict__ Pm, int64_t ldpm, const float* __restrict__ XG, int64_t ldxg, int64_t npairs)
+{
+    if (p.ctl->done) return;
+    __shared__ double red[32];
+    const int g = p.g, gg = g * g;
+    const int64_t npr = p.ng - p.k;
+    double* S = p.pairScratch + (int64_t)blockIdx.x * kPairTemps * gg;
+    double *P = S, *GX = S + gg, *T1 = S + 2 * gg, *c1 = S + 3 * gg, *RR = S + 4 * gg, *TMP = S + 5 * gg, *Lw = S + 6 * gg, *OUT = S + 7 * gg;
+    for (int64_t pair = blockIdx.x; pair < npairs; pair += gridDim.x) {
+        const int64_t s = pair / npr, t = pair % npr;
+        const double Ds = p.D[s], At = p.A[t];
+        if (!isfinite(Ds) || !isfinite(At)) {            // a side that cannot move
+            if (threadIdx.x == 0) p.pairDelta[pair] = INFINITY;
+            continue;
+        }
+        const double* Cinv = p.pairCinv + s * gg;
+        const double* KK = p.pairKK + s * gg;
+        for (int idx = threadIdx.x; idx < gg; idx += blockDim.x) {
+            const int a = idx / g, b = idx % g;
+            P[idx] = (double)Pm[(t * g + a) * ldpm + s * g + b];
+            GX[idx] = (double)XG[(s * g + a) * ldxg + t * g + b];
+        }
+        __syncthreads();
+        mat_mul(P, false, Cinv, false, T1, g);                   // P C^-1
+        mat_mul(T1, false, P, true, TMP, g);                     // P C^-1 P^T
+        for (int idx = threadIdx.x; idx < gg; idx += blockDim.x) {
+            const int i = idx / g, j = idx % g;
+            c1[idx] = 0.5 * (p.c[t * gg + idx] + p.c[t * gg + j * g + i]) + 0.5 * (TMP[idx] + TMP[j * g + i]);
+        }
+        __syncthreads();
+        mat_mul(T1, false, GX, false, TMP, g);                   // P C^-1 V_s R_t^T
+        mat_mul(P, false, KK, false, OUT, g);                    // P KK
+        mat_mul(OUT, false, P, true, RR, g);                     // P KK P^T
+        for (int idx = threadIdx.x; idx < gg; idx += blockDim.x) {
+            const int i = idx / g, j = idx % g;
+            RR[idx] += p.gramR[t * gg + idx] + TMP[idx] + TMP[j * g + i];
+        }
+        __syncthreads();
+        const double piv = chol_inverse(c1, Lw, OUT, g);
+        const double gain = mat_trace_prod(OUT, RR, g, red);
+        if (threadIdx.x == 0) p.pairDelta[pair] = piv > 0.0 ? Ds - gain : INFINITY;
+        __syncthreads();
+    }
+}
+
+// Best pair: smallest delta, ties to the smaller leaving id, then the smaller entering id.
+__global__ void __launch_bounds__(1024) k_pair_select(Ptrs p, int64_t npairs)
+{
+    SearchCtl* ctl = p.ctl;
+    if (ctl->done) return;
+    __shared__ double sv[32]; __shared__ int so[32], si[32]; __shared__ long long sx[32];
+    const int64_t npr = p.ng - p.k;
+    const int t = threadIdx.x, lane = t & 31, w = t >> 5;
+    double best = INFINITY; int bo = INT_MAX, bi = INT_MAX; long long bx = -1;
+    auto better = [](double v, int o, int i, double bv, int bo2, int bi2) {
+        return v < bv || (v == bv && (o < bo2 || (o == bo2 && i < bi2)));
+    };
+    for (int64_t pair = t; pair < npairs; pair += blockDim.x) {
+        const double v = p.pairDelta[pair];
+        const int o = p.perm[pair / npr], i = p.perm[p.k + pair % npr];
+        if (better(v, o, i, best, bo, bi)) { best = v; bo = o; bi = i; bx = pair; }
+    }
+    for (int off = 16; off > 0; off >>= 1) {
+        const double ov = __shfl_xor_sync(0xffffffffu, best, off);
+        const int oo = __shfl_xor_sync(0xffffffffu, bo, off), oi = __shfl_xor_sync(0xffffffffu, bi, off);
+        const long long ox = __shfl_xor_sync(0xffffffffu, bx, off);
+        if (better(ov, oo, oi, best, bo, bi)) { best = ov; bo = oo; bi = oi; bx = ox; }
+    }
+    if (lane == 0) { sv[w] = best; so[w] = bo; si[w] = bi; sx[w] = bx; }
+    __syncthreads();
+    if (t == 0) {
+        for (int j = 1; j < (int)(blockDim.x >> 5); ++j)
+            if (better(sv[j], so[j], si[j], best, bo, bi)) { best = sv[j]; bo = so[j]; bi = si[j]; bx = sx[j]; }
+        if (bx < 0 || !isfinite(best)) { ctl->done = 1; ctl->stop_reason = OSSCAR_STOP_GUARD; *p.done_host = 1; }
+        else { ctl->sel_slot = (int)(bx / npr); ctl->sel_t = (int)(bx % npr); ctl->sel_D = p.D[bx / npr]; }
+    }
+}
+
 #include "search_g1.cuh"
 
 Ptrs make_ptrs(osscar_ctx* ctx)
@@ -674,6 +785,8 @@ Ptrs make_ptrs(osscar_ctx* ctx)
     p.D = (double*)(ws + L.off_D); p.A = (double*)(ws + L.off_A); p.c = (double*)(ws + L.off_c);
     p.small = (double*)(ws + L.off_small); p.gramV = (double*)(ws + L.off_gramV); p.gramR = (double*)(ws + L.off_gramR);
     p.perm = (int32_t*)(ws + L.off_perm); p.slotof = (int32_t*)(ws + L.off_slotof);
+    p.pairCinv = (double*)(ws + L.off_pairCinv); p.pairKK = (double*)(ws + L.off_pairKK);
+    p.pairScratch = (double*)(ws + L.off_pairScratch); p.pairDelta = (double*)(ws + L.off_pairDelta);
     p.ctl = ctx->ctl; p.done_host = ctx->done_flag_dev;
     p.nI = L.nI; p.nJ = L.nJ; p.ldp = L.ldp; p.ldh = L.ldh; p.ldm = L.ldm; p.m = L.m; p.ng = L.ng;
     p.g = L.g; p.k = L.k;
@@ -683,10 +796,10 @@ Ptrs make_ptrs(osscar_ctx* ctx)
 #define CK(x) do { cudaError_t e_ = (x); if (e_ != cudaSuccess) return OSSCAR_E_CUDA; } while (0)
 
 // Everything the selection needs from a freshly built or freshly updated state.
-cudaError_t enqueue_scores(osscar_ctx* ctx, const Ptrs& p, bool norms)
+cudaError_t enqueue_scores(osscar_ctx* ctx, const Ptrs& p, bool norms, bool general = false)
 {
     cudaStream_t st = ctx->stream;
-    if (p.g == 1) {
+    if (p.g == 1 && !general) {
         if (norms) {
             k_row_norms<<<(unsigned)p.nI, 256, 0, st>>>(p.V, p.ldm, p.vnorm, p.ctl);
             count_launches(p.nJ > 0 ? 2 : 1);
@@ -733,7 +846,28 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
     count_launches(1);
     CK(cudaGetLastError());
     CK(cudaEventRecord(ctx->ev0, st));
-    if (max_swaps > 0) CK(enqueue_scores(ctx, p, true));
+    const bool pair = prm->score_mode == OSSCAR_SCORE_PAIR_EXACT;
+    const bool fast = g == 1 && !pair;            // fused five-launch step for single-row groups
+    const int64_t npairs = (int64_t)L.k * (L.ng - L.k);
+    if (max_swaps > 0) CK(enqueue_scores(ctx, p, true, pair));
+    auto pair_scores = [&]() -> cudaError_t {      // PAIR_EXACT: exact change of obj of every (kept, pruned) pair
+        float* Pm = (float*)((char*)ctx->ws + L.off_big);
+        const int64_t ldj = round_up(L.nJ, kPadF);
+        float* XG = Pm + L.nJ * L.ldh;
+        cudaError_t e = sgemm(st, false, false, L.nJ, L.nI, L.nI, 1.f, p.Hp + L.nI * L.ldp, L.ldp, p.Hinv, L.ldh, 0.f, Pm, L.ldh,
+                              &ctx->ctl->done);
+        if (e != cudaSuccess) return e;
+        e = sgemm(st, false, true, L.nI, L.nJ, L.m, 1.f, p.V, L.ldm, p.R, L.ldm, 0.f, XG, ldj, &ctx->ctl->done);
+        if (e != cudaSuccess) return e;
+        const size_t smem = 3 * (size_t)g * g * sizeof(double);
+        e = cudaFuncSetAttribute(k_pair_slots, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        k_pair_slots<<<(unsigned)L.k, 256, smem, st>>>(p);
+        k_pair_delta<<<(unsigned)(npairs < kPairBlocks ? npairs : kPairBlocks), 256, 0, st>>>(p, Pm, L.ldh, XG, ldj, npairs);
+        k_pair_select<<<1, 1024, 0, st>>>(p, npairs);
+        count_launches(3);
+        return cudaGetLastError();
+    };
     auto bootstrap_g1 = [&]() -> cudaError_t {       // score vectors, first entering group and its y from the current state
         k_scores_g1<<<(unsigned)((L.d1 + 255) / 256), 256, 0, st>>>(p);
         k_select_in_g1<<<1, 1024, 0, st>>>(p);
@@ -741,7 +875,7 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
         count_launches(3);
         return cudaGetLastError();
     };
-    if (max_swaps > 0 && g == 1) CK(bootstrap_g1());
+    if (max_swaps > 0 && fast) CK(bootstrap_g1());
 
     const int batch = 32;
     cudaEvent_t evb[2];
@@ -775,15 +909,15 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
             if (rc != OSSCAR_OK) break;
             k_count_refresh<<<1, 1, 0, st>>>(ctx->ctl);
             count_launches(1);
-            if (enqueue_scores(ctx, p, true) != cudaSuccess) { rc = OSSCAR_E_CUDA; break; }
-            if (g == 1 && bootstrap_g1() != cudaSuccess) { rc = OSSCAR_E_CUDA; break; }
+            if (enqueue_scores(ctx, p, true, pair) != cudaSuccess) { rc = OSSCAR_E_CUDA; break; }
+            if (fast && bootstrap_g1() != cudaSuccess) { rc = OSSCAR_E_CUDA; break; }
         }
         cudaEvent_t* pe = nullptr;
         if (next_prof < nprof && prof_it[next_prof] == it) pe = evp[next_prof++];
         int slot = 0;
         auto mark = [&]() { if (pe) cudaEventRecord(pe[slot], st); ++slot; };
         mark();
-        if (g == 1) {
+        if (fast) {
             // single-row groups: decide, {H pass || V}, {R || slot exchange}, next entering group, {Hinv + next y}
             const unsigned nbV = (unsigned)((L.nI + 7) / 8), nbH = (unsigned)((L.nJ + 1 + 7) / 8);
             const unsigned nbR = (unsigned)((L.nJ + 7) / 8);
@@ -794,7 +928,9 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
             k_l4_g1<<<nbV, 256, 0, st>>>(p);                                                     mark();
             count_launches(5);
         } else {
-            k_select<<<1, 1024, 0, st>>>(p);                                                         mark();
+            if (pair) { if (pair_scores() != cudaSuccess) { rc = OSSCAR_E_CUDA; break; } }
+            else k_select<<<1, 1024, 0, st>>>(p);
+            mark();
             k_pairgram<<<(unsigned)((3 * g * g + 7) / 8), 256, 0, st>>>(p);                          mark();
             k_ypass<<<dim3(yblocks, g), 256, 0, st>>>(p);                                            mark();
             k_small<<<1, 256, 0, st>>>(p, prm->accept_mode, tol, max_swaps, obj_trace, swap_trace);  mark();
@@ -808,7 +944,9 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
             if (g > 1) {
                 k_update_c<<<(unsigned)(L.ng - L.k), 128, 0, st>>>(p);
                 count_launches(1);
-                if (enqueue_scores(ctx, p, false) != cudaSuccess) { rc = OSSCAR_E_CUDA; break; }
+            }
+            if (g > 1 || pair) {
+                if (enqueue_scores(ctx, p, false, pair) != cudaSuccess) { rc = OSSCAR_E_CUDA; break; }
             }
             mark();
             k_hswap<<<(unsigned)((L.ldp * g + 255) / 256), 256, 0, st>>>(p, 0);                       mark();

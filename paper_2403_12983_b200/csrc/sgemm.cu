@@ -9,7 +9,7 @@ namespace {
 constexpr int BM = 128, BN = 128, BK = 16, NT = 256;
 constexpr int PADA = 4;
 
-template <bool TA>
+template <bool TA, bool TB>
 __global__ void __launch_bounds__(NT)
 sgemm_kernel(int64_t M, int64_t N, int64_t K, float alpha, const float* __restrict__ A, int64_t lda,
              const float* __restrict__ B, int64_t ldb, float beta, float* __restrict__ C, int64_t ldc,
@@ -17,7 +17,7 @@ sgemm_kernel(int64_t M, int64_t N, int64_t K, float alpha, const float* __restri
 {
     if (done && *done) return;
     __shared__ float As[2][BK][BM + PADA];
-    __shared__ float Bs[2][BK][BN];
+    __shared__ float Bs[2][BK][BN + PADA];
     const int t = threadIdx.x;
     const int tx = t & 15, ty = t >> 4;
     const int64_t m0 = (int64_t)blockIdx.y * BM, n0 = (int64_t)blockIdx.x * BN;
@@ -42,9 +42,15 @@ sgemm_kernel(int64_t M, int64_t N, int64_t K, float alpha, const float* __restri
                 int64_t gk = k0 + kk, gm = m0 + mm;
                 ra[i] = (gk < K && gm < M) ? A[gm * lda + gk] : 0.f;
             }
-            int kk = idx >> 7, nn = idx & 127;
-            int64_t gk = k0 + kk, gn = n0 + nn;
-            rb[i] = (gk < K && gn < N) ? B[gk * ldb + gn] : 0.f;
+            if (TB) {           // B stored N x K: element (nn, kk) contiguous in kk
+                int nn = idx >> 4, kk = idx & 15;
+                int64_t gk = k0 + kk, gn = n0 + nn;
+                rb[i] = (gk < K && gn < N) ? B[gn * ldb + gk] : 0.f;
+            } else {            // B stored K x N
+                int kk = idx >> 7, nn = idx & 127;
+                int64_t gk = k0 + kk, gn = n0 + nn;
+                rb[i] = (gk < K && gn < N) ? B[gk * ldb + gn] : 0.f;
+            }
         }
     };
     auto store_tiles = [&](int buf) {
@@ -53,7 +59,8 @@ sgemm_kernel(int64_t M, int64_t N, int64_t K, float alpha, const float* __restri
             int idx = t + i * NT;
             if (TA) As[buf][idx >> 7][idx & 127] = ra[i];
             else    As[buf][idx & 15][idx >> 4] = ra[i];
-            Bs[buf][idx >> 7][idx & 127] = rb[i];
+            if (TB) Bs[buf][idx & 15][idx >> 4] = rb[i];
+            else    Bs[buf][idx >> 7][idx & 127] = rb[i];
         }
     };
 
@@ -105,12 +112,13 @@ cudaError_t sgemm(cudaStream_t st, bool transA, bool transB, int64_t M, int64_t 
                   float alpha, const float* A, int64_t lda, const float* B, int64_t ldb,
                   float beta, float* C, int64_t ldc, const int32_t* done)
 {
-    if (transB) return cudaErrorInvalidValue;
     if (M <= 0 || N <= 0) return cudaSuccess;
     dim3 grid((unsigned)((N + BN - 1) / BN), (unsigned)((M + BM - 1) / BM));
     count_launches(1);
-    if (transA) sgemm_kernel<true><<<grid, NT, 0, st>>>(M, N, K, alpha, A, lda, B, ldb, beta, C, ldc, done);
-    else        sgemm_kernel<false><<<grid, NT, 0, st>>>(M, N, K, alpha, A, lda, B, ldb, beta, C, ldc, done);
+    if (transA && transB) return cudaErrorInvalidValue;
+    if (transA)      sgemm_kernel<true, false><<<grid, NT, 0, st>>>(M, N, K, alpha, A, lda, B, ldb, beta, C, ldc, done);
+    else if (transB) sgemm_kernel<false, true><<<grid, NT, 0, st>>>(M, N, K, alpha, A, lda, B, ldb, beta, C, ldc, done);
+    else             sgemm_kernel<false, false><<<grid, NT, 0, st>>>(M, N, K, alpha, A, lda, B, ldb, beta, C, ldc, done);
     return cudaGetLastError();
 }
 

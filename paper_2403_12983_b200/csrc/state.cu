@@ -297,6 +297,9 @@ int make_layout(int64_t d1, int64_t m, int32_t g, int32_t k, Layout* L)
     int64_t big = nI * ldm;
     if (nJ * ldh > big) big = nJ * ldh;
     if (2 * d1 * ldm > big) big = 2 * d1 * ldm;
+    const int64_t npairs = (int64_t)k * (ng - k);
+    L->pair_capacity = npairs <= kMaxPairs ? npairs : 0;
+    if (L->pair_capacity > 0 && nJ * ldh + nI * round_up(nJ, kPadF) > big) big = nJ * ldh + nI * round_up(nJ, kPadF);
     L->off_big = take(sizeof(float) * big);
     L->off_Hp = take(sizeof(float) * d1 * L->ldp);
     L->off_Hinv = take(sizeof(float) * nI * ldh);
@@ -325,6 +328,12 @@ int make_layout(int64_t d1, int64_t m, int32_t g, int32_t k, Layout* L)
     L->off_slotof = take(sizeof(int32_t) * ng);
     L->off_energy = take(sizeof(double) * ng + sizeof(int32_t) * ng);
     L->off_panel = take(sizeof(float) * (nI * NB + 2 * NB * ldh + NB * NB));
+    const size_t gg8 = sizeof(double) * g * g;
+    const bool pairs_ok = L->pair_capacity > 0;
+    L->off_pairCinv = take(pairs_ok ? gg8 * k : 8);
+    L->off_pairKK = take(pairs_ok ? gg8 * k : 8);
+    L->off_pairScratch = take(pairs_ok ? gg8 * 8 * 296 : 8);
+    L->off_pairDelta = take(pairs_ok ? sizeof(double) * L->pair_capacity : 8);
     L->bytes = off;
     return OSSCAR_OK;
 }

@@ -217,6 +217,41 @@ def test_group_updates_follow_oracle_with_forced_swaps(solver, osscar, name, ove
         assert np.allclose(c[t], st.c[int(q)], rtol=1e-3, atol=1e-4 * np.abs(st.c[int(q)]).max())
 
 
+PAIR_CASES = [
+    ("c3", dict(n=8192, d1=12 * 40, m=200, g=40, k=6, chunk_rows=8192), 0, 12, False),
+    ("c3", dict(n=8192, d1=12 * 40, m=200, g=40, k=6, chunk_rows=8192), 1, 8, True),
+    ("c3", dict(n=16384, d1=32 * 80, m=384, g=80, k=16, chunk_rows=16384), 0, 6, True),     # c3's own head layout
+    ("c4", dict(n=49 * 40, d1=9 * 40, m=130, k=20, chunk_rows=49 * 40, score_mode="pair_exact"), 0, 10, False),
+    ("c1", dict(score_mode="pair_exact"), 0, 20, False),                                    # single-row groups
+]
+
+
+@pytest.mark.parametrize("name,over,seed,max_swaps,always", PAIR_CASES)
+def test_pair_exact_search_matches_oracle(solver, osscar, name, over, seed, max_swaps, always):
+    """Exhaustive pair scoring (Eq. local solved exactly for one swap): every step must take the oracle's best pair."""
+    b = osscar.binding
+    wl = workloads.config(name, seed=seed, **over)
+    assert wl.score_mode == "pair_exact"
+    chunks, W, H64, G64, const64 = oracle_problem(wl)
+    H, G, Wd = dev(H64), dev(G64), dev(W)
+    Hr, Gr = H.cpu().numpy().astype(np.float64), G.cpu().numpy().astype(np.float64)
+    const_r = float(np.sum(W * Gr))
+    S0, obj0 = solver.init_support(H, G, Wd, wl.g, wl.k)
+    out = solver.local_search(max_swaps, score_mode=b.SCORE_PAIR_EXACT,
+                              accept_mode=b.ACCEPT_ALWAYS if always else b.ACCEPT_IMPROVING, accept_rel_tol=wl.eps_acc)
+    swaps = [tuple(int(v) for v in r) for r in out.swap_trace.cpu().numpy()]
+    srch, rebased = follow_trace(Hr, Gr, const_r, wl.g, S0.cpu().numpy(), swaps, out.obj_trace.cpu().numpy(),
+                                 score_mode="pair_exact", accept="always" if always else "improving",
+                                 gpu_stop=out.stop_reason, max_swaps=max_swaps, eps_acc=wl.eps_acc)
+    assert np.array_equal(out.support.cpu().numpy(), srch.result()[0])
+    assert out.obj_final == pytest.approx(srch.st.obj, rel=1e-4)
+    assert rel_fro(out.W.cpu().numpy(), srch.result()[1]) < 1e-3
+    if always:
+        assert out.n_swaps == max_swaps
+    else:
+        assert np.all(np.diff(out.obj_trace.cpu().numpy()) < 0)
+
+
 @pytest.mark.parametrize("name,over,seed,max_swaps", [SEARCH_CASES[0], SEARCH_CASES[4], SEARCH_CASES[6], SEARCH_CASES[7]])
 def test_end_to_end_from_X(solver, name, over, seed, max_swaps):
     """Whole path from X: Gram on the GPU, then init and search; compared with the oracle run from X."""
