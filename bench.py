@@ -211,6 +211,7 @@ def run_ours(args):
 
     def step(x_chunks, W_in, prof=0):
         return pkg.solve_layer(solver, x_chunks, W_in, wl.g, wl.k, max_swaps, damp=wl.damp, accept_mode=accept, accept_rel_tol=wl.eps_acc,
+                               score_mode=b.SCORE_PAIR_EXACT if wl.score_mode == "pair_exact" else b.SCORE_INDEPENDENT,
                                profile_samples=prof, H=H, G=G)
 
     def barrier():
@@ -306,7 +307,7 @@ def run_ours(args):
     tm_, tn_ = -(-wl.d1 // 128), -(-wl.d1 // 256)
     tiles = sum(tn_ - t // 2 for t in range(tm_))
     gram_exec_tflops = 2.0 * 128 * 256 * tiles * wl.n / max(phase["gram"] / K * 1e-3, 1e-12) / 1e12
-    fused = wl.g == 1
+    fused = wl.g == 1 and wl.score_mode != "pair_exact"
     loop_gbs = swap_bytes(nI, nJ, m, fused) * per_step_swaps / max(phase["search_loop"] / K * 1e-3, 1e-12) / 1e9
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,

@@ -578,11 +578,14 @@ __global__ void __launch_bounds__(256) k_update_rows(Ptrs p, int kind)
 }
 
 // c_l' = c_l + u_l C^-1 u_l^T - d_l c1^-1 d_l^T for every pruned slot (g > 1); the entering slot receives
-// the leaving group: c' = C^-1 - d_r c1^-1 d_r^T.  One block per pruned slot.
-__global__ void __launch_bounds__(128) k_update_c(Ptrs p)
+// the leaving group: c' = C^-1 - d_r c1^-1 d_r^T.  One block per pruned slot; T = u_l C^-1 and d_l c1^-1 are
+// staged in shared memory (2 g^2 doubles) so the work is O(g^3) per slot.
+__global__ void __launch_bounds__(256) k_update_c(Ptrs p)
 {
     if (p.ctl->done) return;
+    extern __shared__ double smc[];
     const int g = p.g, gg = g * g;
+    double* TU = smc; double* TD = smc + gg;
     const int64_t t = blockIdx.x;
     const bool special = t == p.ctl->sel_t;
     const double* Cinv = p.small + S_CINV * gg;
@@ -590,16 +593,21 @@ __global__ void __launch_bounds__(128) k_update_c(Ptrs p)
     const float* ul = p.u + (special ? p.nJ : t * g) * g;     // g x g, row a = row of the group
     const float* dl = p.d + (special ? p.nJ : t * g) * g;
     for (int idx = threadIdx.x; idx < gg; idx += blockDim.x) {
+        const int a = idx / g, f = idx % g;
+        double tu = 0.0, td = 0.0;
+        for (int e = 0; e < g; ++e) {
+            if (!special) tu += (double)ul[a * g + e] * Cinv[e * g + f];
+            td += (double)dl[a * g + e] * c1inv[e * g + f];
+        }
+        TU[idx] = tu; TD[idx] = td;
+    }
+    __syncthreads();
+    for (int idx = threadIdx.x; idx < gg; idx += blockDim.x) {
         const int a = idx / g, b2 = idx % g;
         double s = special ? Cinv[idx] : p.c[t * gg + idx];
-        for (int e = 0; e < g; ++e) {
-            double tu = 0.0, td = 0.0;
-            for (int f = 0; f < g; ++f) {
-                if (!special) tu += Cinv[e * g + f] * (double)ul[b2 * g + f];
-                td += c1inv[e * g + f] * (double)dl[b2 * g + f];
-            }
-            if (!special) s += (double)ul[a * g + e] * tu;
-            s -= (double)dl[a * g + e] * td;
+        for (int f = 0; f < g; ++f) {
+            if (!special) s += TU[a * g + f] * (double)ul[b2 * g + f];
+            s -= TD[a * g + f] * (double)dl[b2 * g + f];
         }
         p.c[t * gg + idx] = s;      // each thread reads only its own old entry
     }
@@ -877,6 +885,7 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
     };
     if (max_swaps > 0 && fast) CK(bootstrap_g1());
 
+    if (g > 1) CK(cudaFuncSetAttribute(k_update_c, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(2 * (size_t)g * g * sizeof(double))));
     const int batch = 32;
     cudaEvent_t evb[2];
     CK(cudaEventCreateWithFlags(&evb[0], cudaEventDisableTiming));
@@ -896,6 +905,7 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
     const unsigned hblocks = (unsigned)((L.nJ + g + 8 * RPW - 1) / (8 * RPW));
     const unsigned prep_blocks = (unsigned)(((L.nI + L.ldm) * g + 255) / 256);
     int next_prof = 0;
+    int nmarks = 0;                 // events recorded per profiled step (depends on the step variant)
     for (int it = 0; it < max_swaps && rc == OSSCAR_OK; ++it) {
         if (it % batch == 0) {
             const int bi = it / batch;
@@ -942,7 +952,7 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
             k_update_rows<<<(unsigned)((L.nJ + UP_ROWS - 1) / UP_ROWS), 256, 0, st>>>(p, 1);          mark();
             count_launches(9);
             if (g > 1) {
-                k_update_c<<<(unsigned)(L.ng - L.k), 128, 0, st>>>(p);
+                k_update_c<<<(unsigned)(L.ng - L.k), 256, 2 * (size_t)g * g * sizeof(double), st>>>(p);
                 count_launches(1);
             }
             if (g > 1 || pair) {
@@ -953,6 +963,7 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
             k_hswap<<<(unsigned)((L.ldp * g + 255) / 256), 256, 0, st>>>(p, 1);                       mark();
             count_launches(2);
         }
+        if (pe) nmarks = slot;
         if (cudaGetLastError() != cudaSuccess) { rc = OSSCAR_E_CUDA; break; }
         if ((it + 1) % batch == 0) {
             if (cudaEventRecord(evb[(it / batch) & 1], st) != cudaSuccess) { rc = OSSCAR_E_CUDA; break; }
@@ -995,7 +1006,7 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
     int used = 0;
     for (int i = 0; i < nprof; ++i) {
         if (i < next_prof && prof_it[i] < res->n_swaps) {
-            for (int j = 0; j < NK; ++j) {
+            for (int j = 0; j + 1 < nmarks && j < NK; ++j) {
                 float t = 0.f;
                 if (cudaEventElapsedTime(&t, evp[i][j], evp[i][j + 1]) == cudaSuccess) res->ms_kernel[j] += t;
             }
