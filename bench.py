@@ -144,7 +144,7 @@ def oracle_step(wl, max_swaps):
     return {"solve_s": t3 - t1, "search_s": t3 - t2, "swaps": len(srch.swap_trace), "gen_s": t1 - t0}
 
 
-def cpu_baseline(max_swaps=40):
+def cpu_baseline(max_swaps=250):
     wl = workloads.config("c5", **CPU_SAMPLE)
     r = oracle_step(wl, max_swaps)
     cores = torch.get_num_threads()
@@ -290,11 +290,16 @@ def run_ours(args):
     shares = {k2: v * per_step_swaps for k2, v in kern_avg.items()}
     shares["gram_tcgen05"] = phase["gram"] / K
     dom = max(shares, key=shares.get) if shares else "gram_tcgen05"
+    # dram bytes / algorithmic bytes measured with ncu on a mid-size case (profiles/swap_step_g1_kernels_mid_size.md);
+    # traffic grows in proportion to the rows streamed, so the ratio carries over to a full-size launch
+    traffic_ratio = {"l1_hpass_update_v": 1.010, "l2_update_r_swap": 0.915, "l4_update_hinv_y": 0.807}
     if dom in KERNEL_BYTES and kern_avg.get(dom, 0) > 0:
         bytes_per_launch = KERNEL_BYTES[dom](nI, nJ, m)
         ach = bytes_per_launch / (kern_avg[dom] * 1e-3) / 1e9
         roof = {"kernel": dom, "bound": "hbm", "achieved": ach, "peak": pk["hbm_gbs"], "unit": "GB/s",
-                "frac": ach / pk["hbm_gbs"], "traffic": None, "bytes_per_launch": bytes_per_launch,
+                "frac": ach / pk["hbm_gbs"],
+                "traffic": int(traffic_ratio[dom] * bytes_per_launch) if dom in traffic_ratio else None,
+                "bytes_per_launch": bytes_per_launch,
                 "ms_per_launch": kern_avg[dom], "peak_source": pk["source"]}
     else:
         tm_, tn_ = -(-wl.d1 // 128), -(-wl.d1 // 256)
