@@ -71,6 +71,8 @@ int osscar_set_workspace(osscar_ctx* ctx, void* dev_ptr, size_t bytes);
  *   flags & BEGIN : H := Xc^T Xc, otherwise H += Xc^T Xc   (split over calibration rows);
  *   flags & END   : H += damp * mean(diag H) * I (damp = 0: none; not in the paper),
  *                   G := H W_hat, *const_term := Tr(W_hat^T G), then one stream sync.
+ *                   With a workspace set, G is formed on the tensor cores (three-term bf16 split, fp32-accurate)
+ *                   and the workspace contents are overwritten; without one it runs on the fp32 pipes.
  * X: device, n_rows x d1, bf16 (tensor cores, fp32 accumulation) or fp32.  For bf16 the
  * pointer must be 16-byte aligned and d1 a multiple of 8.  W: device d1 x m fp32 (read on END).
  * H: device d1 x d1 fp32, G: device d1 x m fp32, const_term: host (written on END).

@@ -1,0 +1,322 @@
+// fp32-accurate GEMM on the tensor cores: C = alpha * A * B + beta * C with A (M x K) and B (K x N) row-major fp32.
+// Used for the dense contractions around the search: G = H W (Section 2), V = (H_II)^-1 G_I (Eq. tmp5),
+// the residual R, the Schur-complement products and the rank-64 updates of the block inversion.
+//
+// Each fp32 operand is split into three bf16 terms (x = x1 + x2 + x3, 8 mantissa bits each); the product keeps the
+// six terms down to 2^-24 relative: x1y1, x1y2, x2y1, x1y3, x2y2, x3y1.  The kernel is the persistent TMA /
+// tcgen05 / TMEM pipeline of the Gram kernel with three changes: A is K-major (rows of 128 bytes, SWIZZLE_128B),
+// every 64-wide k-block is visited six times (one term pair each), and the TMEM accumulator is drained into fp32
+// registers every kFlush k-blocks: tcgen05.mma adds into its accumulator with truncation, so long accumulation
+// chains would cost accuracy; the register sums are round-to-nearest.
+//   warp 0: TMA producer     warp 1: MMA issuer     warps 2-9: accumulate (TMEM -> registers) and write C
+// K is processed in panels sized to the caller's scratch (the bf16 terms of one panel of A and B live there).
+#include "osscar_internal.cuh"
+#include <cuda_bf16.h>
+#include "tc_common.cuh"
+
+namespace osscar {
+namespace {
+
+using namespace tc;
+
+constexpr int TILE_M = 128, TILE_N = 256, BLOCK_K = 64, UMMA_K = 16, STAGES = 4;
+constexpr int A_BYTES = TILE_M * BLOCK_K * 2;                 // 16384: one box of 128 rows x 128 bytes
+constexpr int BOX_BYTES = 64 * BLOCK_K * 2;                   // 8192: 64 columns of B x 64 k-rows
+constexpr int B_BYTES = (TILE_N / 64) * BOX_BYTES;            // 32768
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256;
+constexpr int NUM_THREADS = 320;                              // 10 warps
+constexpr int TMEM_COLS = 512;
+constexpr int kFlush = 2;                                     // k-blocks (x 6 term pairs) per TMEM accumulation chain
+constexpr int kTerms = 6;
+constexpr int BAND = 8;                                       // tile rows per raster band
+
+// kind::f16, D fp32, A/B bf16, A K-major, B MN-major, M = 128, N = 256.
+constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16)
+                          | ((uint32_t)(TILE_N >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
+
+// A tile: K-major, SWIZZLE_128B: rows of 128 bytes, 8-row swizzle atoms 1024 bytes apart (stride byte offset);
+// the leading byte offset is not used by swizzled K-major layouts.
+__device__ __forceinline__ uint64_t desc_a(uint32_t saddr) {
+    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+// B tile: MN-major, SWIZZLE_128B: 64-column boxes 8192 bytes apart (leading), 8-k-row atoms 1024 bytes apart (stride).
+__device__ __forceinline__ uint64_t desc_b(uint32_t saddr) {
+    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(BOX_BYTES >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+
+struct Maps { CUtensorMap a[3]; CUtensorMap b[3]; };
+
+__device__ __forceinline__ void tile_of(int id, int TM, int TN, int* tm, int* tn) {
+    // bands of BAND tile rows, column-major inside a band: concurrent CTAs share A rows and B columns in L2
+    const int per_band = BAND * TN;
+    const int b = id / per_band, r = id % per_band;
+    const int rows = min(BAND, TM - b * BAND);
+    *tn = r / rows; *tm = b * BAND + r % rows;
+}
+
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+k_gemm3(const __grid_constant__ Maps maps, int64_t M, int64_t N, int64_t K, float alpha, float beta,
+        float* __restrict__ C, int64_t ldc, int vec_ok, int32_t* __restrict__ status, const int32_t* __restrict__ done)
+{
+    if (done && *done) return;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t tiles_base = (raw + 1023u) & ~1023u;
+    uint8_t* bar_ptr = smem_raw + (tiles_base - raw) + STAGES * STAGE_BYTES;
+    const uint32_t bars = tiles_base + STAGES * STAGE_BYTES;
+    auto full_bar = [&](int s) { return bars + 8u * s; };
+    auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
+    auto tfull_bar = [&](int b) { return bars + 8u * (2 * STAGES + b); };
+    auto tempty_bar = [&](int b) { return bars + 8u * (2 * STAGES + 2 + b); };
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_ptr + 8 * (2 * STAGES + 4));
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_ptr + 8 * (2 * STAGES + 4) + 8);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int TM = (int)((M + TILE_M - 1) / TILE_M), TN = (int)((N + TILE_N - 1) / TILE_N);
+    // the band raster enumerates BAND * TN ids per band; the last band may be short
+    const int full_bands = TM / BAND, rem_rows = TM % BAND;
+    const int num_ids = full_bands * BAND * TN + rem_rows * TN;
+    const int nkb = (int)((K + BLOCK_K - 1) / BLOCK_K);
+    const int nflush = (nkb + kFlush - 1) / kFlush;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 8); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "n"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int id = blockIdx.x; id < num_ids && ok; id += gridDim.x) {
+                int tm, tn;
+                tile_of(id, TM, TN, &tm, &tn);
+                for (int kb = 0; kb < nkb && ok; ++kb) {
+                    for (int term = 0; term < kTerms; ++term, ++it) {
+                        // term pairs, small products first: (3,1) (2,2) (1,3) (2,1) (1,2) (1,1)
+                        const int pa = (0x001012 >> (4 * term)) & 0xF;      // index of the A term: 2,1,0,1,0,0
+                        const int pb = (0x010210 >> (4 * term)) & 0xF;      // index of the B term: 0,1,2,0,1,0
+                        const int s = it % STAGES;
+                        const uint32_t ph = (it / STAGES) & 1;
+                        if (!mbar_wait(empty_bar(s), ph ^ 1, abort_flag)) { ok = false; break; }
+                        mbar_expect_tx(full_bar(s), STAGE_BYTES);
+                        const uint32_t a_dst = tiles_base + s * STAGE_BYTES;
+                        const uint32_t b_dst = a_dst + A_BYTES;
+                        tma_load_2d(a_dst, &maps.a[pa], full_bar(s), kb * BLOCK_K, tm * TILE_M);
+#pragma unroll
+                        for (int i = 0; i < TILE_N / 64; ++i)
+                            tma_load_2d(b_dst + i * BOX_BYTES, &maps.b[pb], full_bar(s), tn * TILE_N + i * 64, kb * BLOCK_K);
+                    }
+                }
+            }
+            if (*abort_flag) {
+                const uint32_t first = it > STAGES ? it - STAGES : 0;
+                for (uint32_t j = first; j < it; ++j) {
+                    const long long t0 = clock64();
+                    while (!mbar_try_wait(full_bar(j % STAGES), (j / STAGES) & 1))
+                        if (clock64() - t0 > kWaitLimitCycles) break;
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            uint32_t it = 0, fl = 0;            // stage counter, flush counter (selects the TMEM buffer)
+            bool ok = true;
+            for (int id = blockIdx.x; id < num_ids && ok; id += gridDim.x) {
+                for (int f = 0; f < nflush && ok; ++f, ++fl) {
+                    const int buf = fl & 1;
+                    if (!mbar_wait(tempty_bar(buf), ((fl >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint32_t d_tmem = tmem_base + (uint32_t)(buf * TILE_N);
+                    const int kb1 = min(nkb, (f + 1) * kFlush);
+                    bool first = true;
+                    for (int kb = f * kFlush; kb < kb1 && ok; ++kb) {
+                        for (int term = 0; term < kTerms; ++term, ++it) {
+                            const int s = it % STAGES;
+                            const uint32_t ph = (it / STAGES) & 1;
+                            if (!mbar_wait(full_bar(s), ph, abort_flag)) { ok = false; break; }
+                            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                            const uint32_t a_src = tiles_base + s * STAGE_BYTES;
+                            const uint32_t b_src = a_src + A_BYTES;
+#pragma unroll
+                            for (int j = 0; j < BLOCK_K / UMMA_K; ++j) {
+                                // A: +32 bytes per 16 k inside the 128-byte row; B: +16 k-rows of 128 bytes
+                                umma_f16(d_tmem, desc_a(a_src + j * 32), desc_b(b_src + j * (UMMA_K * 128)), kIdesc, first ? 0u : 1u);
+                                first = false;
+                            }
+                            umma_commit(empty_bar(s));
+                        }
+                    }
+                    if (ok) umma_commit(tfull_bar(buf));
+                }
+            }
+        }
+    } else {
+        // warps 2..9: lane group = warp % 4, column half = (warp - 2) / 4
+        const int lg = warp & 3, half = (warp - 2) >> 2;
+        uint32_t fl = 0;
+        bool ok = true;
+        for (int id = blockIdx.x; id < num_ids && ok; id += gridDim.x) {
+            int tm, tn;
+            tile_of(id, TM, TN, &tm, &tn);
+            float acc[128];
+#pragma unroll
+            for (int j = 0; j < 128; ++j) acc[j] = 0.f;
+            for (int f = 0; f < nflush && ok; ++f, ++fl) {
+                const int buf = fl & 1;
+                if (!mbar_wait(tfull_bar(buf), (fl >> 1) & 1, abort_flag)) { ok = false; break; }
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t r[32];
+                    tmem_ld32(tmem_base + ((uint32_t)(lg * 32) << 16) + (uint32_t)(buf * TILE_N + half * 128 + c * 32), r);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) acc[c * 32 + j] += __uint_as_float(r[j]);
+                }
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) mbar_arrive(tempty_bar(buf));
+            }
+            if (!ok) break;
+            const int64_t grow = (int64_t)tm * TILE_M + lg * 32 + lane;
+            const int64_t gcol0 = (int64_t)tn * TILE_N + half * 128;
+            if (grow < M) {
+                float* crow = C + grow * ldc;
+                if (vec_ok) {
+#pragma unroll
+                    for (int j = 0; j < 128; j += 4) {
+                        if (gcol0 + j < N) {        // N is a multiple of 4 on this path
+                            float4* dst = reinterpret_cast<float4*>(crow + gcol0 + j);
+                            float4 v = make_float4(alpha * acc[j], alpha * acc[j + 1], alpha * acc[j + 2], alpha * acc[j + 3]);
+                            if (beta != 0.f) {
+                                const float4 o = *dst;
+                                v.x = fmaf(beta, o.x, v.x); v.y = fmaf(beta, o.y, v.y); v.z = fmaf(beta, o.z, v.z); v.w = fmaf(beta, o.w, v.w);
+                            }
+                            *dst = v;
+                        }
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 128; ++j) {
+                        if (gcol0 + j < N) {
+                            float v = alpha * acc[j];
+                            if (beta != 0.f) v = fmaf(beta, crow[gcol0 + j], v);
+                            crow[gcol0 + j] = v;
+                        }
+                    }
+                }
+            }
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "n"(TMEM_COLS) : "memory");
+    }
+    if (threadIdx.x == 0 && *abort_flag) *status = OSSCAR_E_TIMEOUT;
+}
+
+// x = x1 + x2 + x3 with bf16 terms (round to nearest each time); dst rows are ldd wide, the tail is zero.
+__global__ void k_split3(const float* __restrict__ src, int64_t lds, int64_t rows, int64_t cols,
+                         __nv_bfloat16* __restrict__ d1, __nv_bfloat16* __restrict__ d2, __nv_bfloat16* __restrict__ d3,
+                         int64_t ldd, const int32_t* __restrict__ done)
+{
+    if (done && *done) return;
+    const int64_t total = rows * ldd;
+    for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t r = idx / ldd, c = idx % ldd;
+        float x = c < cols ? src[r * lds + c] : 0.f;
+        const __nv_bfloat16 a = __float2bfloat16_rn(x);
+        x -= __bfloat162float(a);
+        const __nv_bfloat16 b = __float2bfloat16_rn(x);
+        x -= __bfloat162float(b);
+        d1[idx] = a; d2[idx] = b; d3[idx] = __float2bfloat16_rn(x);
+    }
+}
+
+bool encode_2d(PFN_encodeTiled enc, CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer, uint64_t ld_elems,
+               uint32_t box_inner, uint32_t box_outer)
+{
+    const cuuint64_t dims[2] = {inner, outer};
+    const cuuint64_t strides[1] = {ld_elems * 2};
+    const cuuint32_t box[2] = {box_inner, box_outer};
+    const cuuint32_t estr[2] = {1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+size_t gemm_tc_min_scratch(int64_t M, int64_t N)
+{
+    // the three bf16 terms of a 64-wide panel of A and of B, each buffer 1024-byte aligned
+    return (size_t)6 * (size_t)(M + round_up(N, 8)) * 64 + 8 * 1024;
+}
+
+cudaError_t gemm_tc(cudaStream_t st, int64_t M, int64_t N, int64_t K, float alpha, const float* A, int64_t lda,
+                    const float* B, int64_t ldb, float beta, float* C, int64_t ldc,
+                    void* scratch, size_t scratch_bytes, int32_t* status_dev, const int32_t* done)
+{
+    if (M <= 0 || N <= 0) return cudaSuccess;
+    if (K <= 0 || scratch_bytes < gemm_tc_min_scratch(M, N) || ((uintptr_t)scratch & 255)) return cudaErrorInvalidValue;
+    PFN_encodeTiled enc = get_encode();
+    if (!enc) return cudaErrorNotSupported;
+    const int64_t ldn = round_up(N, 8);                         // row stride of the B terms (16-byte multiple)
+    // panel width: largest multiple of 64 whose six buffers fit
+    int64_t kc = (int64_t)((scratch_bytes - 8 * 1024) / (6 * (size_t)(M + ldn))) / 64 * 64;
+    if (kc > round_up(K, 64)) kc = round_up(K, 64);
+    if (kc > 8192) kc = 8192;
+    auto align_up = [](size_t x) { return (x + 1023) / 1024 * 1024; };
+    const size_t a_bytes = align_up((size_t)M * kc * 2), b_bytes = align_up((size_t)kc * ldn * 2);
+    if (3 * (a_bytes + b_bytes) > scratch_bytes) return cudaErrorInvalidValue;
+    __nv_bfloat16* ap[3]; __nv_bfloat16* bp[3];
+    for (int i = 0; i < 3; ++i) {
+        ap[i] = (__nv_bfloat16*)((char*)scratch + i * a_bytes);
+        bp[i] = (__nv_bfloat16*)((char*)scratch + 3 * a_bytes + i * b_bytes);
+    }
+    int dev = 0, sms = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(k_gemm3, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    const int TM = (int)((M + TILE_M - 1) / TILE_M), TN = (int)((N + TILE_N - 1) / TILE_N);
+    const int num_ids = TM * TN;
+    const int vec_ok = (((uintptr_t)C & 15) == 0 && (ldc % 4) == 0 && (N % 4) == 0) ? 1 : 0;
+    for (int64_t k0 = 0; k0 < K; k0 += kc) {
+        const int64_t kw = K - k0 < kc ? K - k0 : kc;
+        const int64_t kw8 = round_up(kw, 8);                    // row stride of the A terms
+        k_split3<<<1184, 256, 0, st>>>(A + k0, lda, M, kw, ap[0], ap[1], ap[2], kw8, done);
+        k_split3<<<1184, 256, 0, st>>>(B + k0 * ldb, ldb, kw, N, bp[0], bp[1], bp[2], ldn, done);
+        Maps maps;
+        for (int i = 0; i < 3; ++i) {
+            // A terms: inner dimension k (kw valid, rows kw8 apart), box 64 x 128; B terms: inner n, box 64 x 64
+            if (!encode_2d(enc, &maps.a[i], ap[i], (uint64_t)kw, (uint64_t)M, (uint64_t)kw8, BLOCK_K, TILE_M)) return cudaErrorInvalidValue;
+            if (!encode_2d(enc, &maps.b[i], bp[i], (uint64_t)N, (uint64_t)kw, (uint64_t)ldn, 64, BLOCK_K)) return cudaErrorInvalidValue;
+        }
+        const int grid = num_ids < sms ? num_ids : sms;
+        k_gemm3<<<grid, NUM_THREADS, SMEM_BYTES, st>>>(maps, M, N, kw, alpha, k0 == 0 ? beta : 1.f, C, ldc, vec_ok, status_dev, done);
+        count_launches(3);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
+}
+
+}  // namespace osscar

@@ -160,7 +160,14 @@ int osscar_gram(osscar_ctx* ctx, const void* X, int x_dtype, int64_t n_rows, int
         k_add_damp<<<64, 256, 0, st>>>(H, d1, damp, &ctx->ctl->acc[0]);
         count_launches(2);
     }
-    CKC(sgemm(st, false, false, d1, m, d1, 1.f, H, d1, W, m, 0.f, G, m));
+    if (ctx->ws && ctx->ws_bytes >= gemm_tc_min_scratch(d1, m)) {
+        // tensor-core product with the operand terms staged in the lent workspace (its contents are overwritten)
+        const size_t cap = ctx->ws_bytes < ((size_t)3 << 30) ? ctx->ws_bytes : ((size_t)3 << 30);
+        CKC(gemm_tc(st, d1, m, d1, 1.f, H, d1, W, m, 0.f, G, m, ctx->ws, cap, &ctx->ctl->status));
+        ctx->have_state = false;
+    } else {
+        CKC(sgemm(st, false, false, d1, m, d1, 1.f, H, d1, W, m, 0.f, G, m));
+    }
     CKC(trace_product(st, W, m, G, m, d1, m, ctx->partials, &ctx->ctl->acc[1]));
     CKC(cudaMemcpyAsync(ctx->ctl_host, ctx->ctl, sizeof(SearchCtl), cudaMemcpyDeviceToHost, st));
     CKC(cudaStreamSynchronize(st));

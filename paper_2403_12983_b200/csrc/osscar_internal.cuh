@@ -48,6 +48,7 @@ struct Layout {
     size_t off_vnorm, off_rnorm, off_D, off_A, off_c, off_small, off_gramV, off_gramR;
     size_t off_perm, off_slotof, off_energy, off_panel;
     size_t off_pairCinv, off_pairKK, off_pairScratch, off_pairDelta;   // PAIR_EXACT scoring
+    size_t off_tc, tc_bytes;                                           // bf16 operand terms of the tensor-core GEMMs
     int64_t pair_capacity;                                             // pairs the workspace can score
     size_t bytes;
 };
@@ -82,6 +83,13 @@ namespace osscar {
 cudaError_t sgemm(cudaStream_t st, bool transA, bool transB, int64_t M, int64_t N, int64_t K,
                   float alpha, const float* A, int64_t lda, const float* B, int64_t ldb,
                   float beta, float* C, int64_t ldc, const int32_t* done = nullptr);
+
+// ---- gemm_tc.cu: the same product on the tensor cores (three-term bf16 split, fp32-accurate); A and B row-major.
+// `scratch` (256-byte aligned device memory, at least gemm_tc_min_scratch bytes) holds the bf16 terms of one K panel.
+size_t gemm_tc_min_scratch(int64_t M, int64_t N);
+cudaError_t gemm_tc(cudaStream_t st, int64_t M, int64_t N, int64_t K, float alpha, const float* A, int64_t lda,
+                    const float* B, int64_t ldb, float beta, float* C, int64_t ldc,
+                    void* scratch, size_t scratch_bytes, int32_t* status_dev, const int32_t* done = nullptr);
 
 // ---- gram_tc.cu: H (+)= Xc^T Xc on the tensor cores (bf16 in, fp32 out) ----------------------
 cudaError_t gram_bf16_tcgen05(cudaStream_t st, const void* X, int64_t n_rows, int64_t d1,

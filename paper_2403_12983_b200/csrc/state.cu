@@ -334,6 +334,12 @@ int make_layout(int64_t d1, int64_t m, int32_t g, int32_t k, Layout* L)
     L->off_pairKK = take(pairs_ok ? gg8 * k : 8);
     L->off_pairScratch = take(pairs_ok ? gg8 * 8 * 296 : 8);
     L->off_pairDelta = take(pairs_ok ? sizeof(double) * L->pair_capacity : 8);
+    {   // K panels of up to 2048 for the widest products of the state build (M <= d1, N <= max(m, n_I))
+        const int64_t nmax = ldm > ldh ? ldm : ldh;
+        L->tc_bytes = 3 * ((size_t)d1 * 2048 * 2 + (size_t)2048 * nmax * 2) + 16 * 1024;
+        if (L->tc_bytes < gemm_tc_min_scratch(d1, nmax)) L->tc_bytes = gemm_tc_min_scratch(d1, nmax);
+        L->off_tc = take(L->tc_bytes);
+    }
     L->bytes = off;
     return OSSCAR_OK;
 }
@@ -380,6 +386,7 @@ int build_state(osscar_ctx* ctx, bool guarded)
     float* Un = U + NB * L.ldh;
     float* Dinv = Un + NB * L.ldh;
     const int32_t* done = guarded ? &ctx->ctl->done : nullptr;
+    void* tc = ws + L.off_tc;
     const int64_t nI = L.nI, nJ = L.nJ;
 
     {   // slot-permuted copy of H
@@ -402,6 +409,8 @@ int build_state(osscar_ctx* ctx, bool guarded)
             k_copy_rows<<<grid, 256, 0, st>>>(Hinv, L.ldh, p0, nb, nI, U, L.ldh);
         }
         CK(sgemm(st, false, false, nb, nI, nb, -1.f, Dinv, NB, U, L.ldh, 0.f, Un, L.ldh, done));
+        // the rank-64 updates stay on the fp32 pipes: the inversion amplifies rounding by cond(H_II), and the tensor
+        // core's truncating accumulation is biased where fp32 FMA chains are not
         CK(sgemm(st, false, false, nI, nI, nb, -1.f, T, NB, U, L.ldh, 1.f, Hinv, L.ldh, done));
         k_gj_writeback<<<(unsigned)((nI * nb + 255) / 256), 256, 0, st>>>(Hinv, L.ldh, nI, p0, nb, T, NB, Un, L.ldh, Dinv);
         count_launches(4);     // pivot inverse, zero rows, copy rows, write-back (the GEMMs count themselves)
@@ -410,6 +419,8 @@ int build_state(osscar_ctx* ctx, bool guarded)
     // V = Hinv * G_I
     k_gather_rows<<<(unsigned)nI, 256, 0, st>>>(ctx->G, L.m, L.g, perm, 0, big, L.ldm);
     if (L.ldm != L.m) CK(cudaMemsetAsync(V, 0, sizeof(float) * nI * L.ldm, st));     // padding columns stay zero
+    // V = Hinv G_I sums large terms of both signs to a small result (cond(H_II) of cancellation): it stays on the
+    // fp32 pipes, whose rounding is unbiased; the tensor core's truncating accumulation cost 0.2 % of obj here
     CK(sgemm(st, false, false, nI, L.m, nI, 1.f, Hinv, L.ldh, big, L.ldm, 0.f, V, L.ldm, done));
     // obj = Tr(W^T G) - Tr(G_I^T V)
     CK(trace_product(st, ctx->W, L.m, ctx->G, L.m, L.d1, L.m, ctx->partials, &ctx->ctl->acc[0]));
@@ -419,9 +430,9 @@ int build_state(osscar_ctx* ctx, bool guarded)
     if (nJ > 0) {
         // R_J = G_J - Hp[J, I] V
         k_gather_rows<<<(unsigned)nJ, 256, 0, st>>>(ctx->G, L.m, L.g, perm, nI, R, L.ldm);
-        CK(sgemm(st, false, false, nJ, L.m, nI, -1.f, Hp + nI * L.ldp, L.ldp, V, L.ldm, 1.f, R, L.ldm, done));
+        CK(gemm_tc(st, nJ, L.m, nI, -1.f, Hp + nI * L.ldp, L.ldp, V, L.ldm, 1.f, R, L.ldm, tc, L.tc_bytes, &ctx->ctl->status, done));
         // Pm = Hp[J, I] Hinv, then the Schur complements
-        CK(sgemm(st, false, false, nJ, nI, nI, 1.f, Hp + nI * L.ldp, L.ldp, Hinv, L.ldh, 0.f, big, L.ldh, done));
+        CK(gemm_tc(st, nJ, nI, nI, 1.f, Hp + nI * L.ldp, L.ldp, Hinv, L.ldh, 0.f, big, L.ldh, tc, L.tc_bytes, &ctx->ctl->status, done));
         k_schur<<<(unsigned)(L.ng - L.k), 256, 0, st>>>(Hp, L.ldp, big, L.ldh, nI, L.g, c);
         count_launches(2);
     }

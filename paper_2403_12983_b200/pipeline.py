@@ -75,6 +75,7 @@ def solve_layer(solver: b.Solver, x_chunks: Sequence[torch.Tensor], W: torch.Ten
         io["h2d"] += W.numel() * 4
         W = W.to(dev, non_blocking=True)
     d1, m = W.shape
+    solver.ensure_workspace(d1, m, g, k)          # also lets the cross term G = H W run on the tensor cores
     if H is None:
         H = torch.empty(d1, d1, dtype=torch.float32, device=dev)
     if G is None:

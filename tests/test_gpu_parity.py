@@ -68,6 +68,23 @@ def test_gram_fp32(solver, name, over):
     assert const == pytest.approx(const64, rel=1e-5)
 
 
+@pytest.mark.parametrize("name,over", [GRAM_CASES[0], GRAM_CASES[2], ("c2", dict(n=600, d1=200, m=37, k=100, chunk_rows=600))])
+def test_cross_term_on_tensor_cores(solver, name, over):
+    """With a workspace lent to the context, G = H W runs as a three-term bf16 split on the tensor cores;
+    it must be as accurate as the fp32 product (ragged sizes: m not a multiple of 4, d1 not of 64)."""
+    wl = workloads.config(name, **over)
+    chunks, W, H64, G64, const64 = oracle_problem(wl)
+    Wd = wl.weight().cuda()
+    solver.ensure_workspace(wl.d1, wl.m, wl.g, wl.k)
+    H, G, const = solver.gram([c.cuda() for c in wl.x_chunks()], Wd, wl.damp)
+    Hg = H.cpu().numpy().astype(np.float64)
+    Gref = Hg @ W                        # the product itself, from the GPU's own H: isolates the GEMM
+    gs = np.linalg.norm(Gref, axis=1, keepdims=True) + 1e-300
+    assert np.max(np.abs(G.cpu().numpy() - Gref) / gs) < 2e-6
+    assert const == pytest.approx(float(np.sum(W * Gref)), rel=3e-6)
+    assert rel_fro(G.cpu().numpy(), G64) < 1e-5
+
+
 def test_gram_empty_and_single_chunk_flags(solver, osscar):
     wl = workloads.config("c2", n=256, d1=64, m=8, k=32, chunk_rows=256)
     X = wl.x_chunk(0).cuda(); W = wl.weight().cuda()
