@@ -929,8 +929,7 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
         mark();
         if (fast) {
             // single-row groups: decide, {H pass || V}, {R || slot exchange}, next entering group, {Hinv + next y}
-            const unsigned nbV = (unsigned)((L.nI + 7) / 8), nbH = (unsigned)((L.nJ + 1 + 7) / 8);
-            const unsigned nbR = (unsigned)((L.nJ + 7) / 8);
+            const unsigned nbV = (unsigned)L.nI, nbH = (unsigned)(L.nJ + 1), nbR = (unsigned)L.nJ;   // one row per block
             k_decide_g1<<<1, 1024, 0, st>>>(p, prm->accept_mode, tol, obj_trace, swap_trace);   mark();
             k_l1_g1<<<nbV + nbH, 256, 0, st>>>(p, nbV);                                          mark();
             k_l2_g1<<<nbR + 32, 256, 0, st>>>(p, nbR);                                           mark();
