@@ -292,7 +292,7 @@ def run_ours(args):
     dom = max(shares, key=shares.get) if shares else "gram_tcgen05"
     # dram bytes / algorithmic bytes measured with ncu on a mid-size case (profiles/swap_step_g1_kernels_mid_size.md);
     # traffic grows in proportion to the rows streamed, so the ratio carries over to a full-size launch
-    traffic_ratio = {"l1_hpass_update_v": 1.010, "l2_update_r_swap": 0.915, "l4_update_hinv_y": 0.807}
+    traffic_ratio = {"l1_hpass_update_v": 1.010, "l2_update_r_swap": 0.915, "l4_update_hinv_y": 0.793}
     if dom in KERNEL_BYTES and kern_avg.get(dom, 0) > 0:
         bytes_per_launch = KERNEL_BYTES[dom](nI, nJ, m)
         ach = bytes_per_launch / (kern_avg[dom] * 1e-3) / 1e9
