@@ -488,6 +488,37 @@ def lowrank_swap(H, st: State, g: int, slot: int, q: int) -> State:
     return State(S=S2, Hinv=Hinv2, V=V2, R=R2, c=c2, obj=obj2)
 
 
+# --------------------------------------------------------------------------- nested (greedy) phase
+def greedy_prune(H, G, const, g, k, t_hat=1):
+    """Nested phase of Algorithm 1 (t_i = p_i = t_hat): start from all groups kept (S_0 in the paper is the empty
+    pruned set, with H^-1 and W* = H^-1 G) and, per iteration, prune the t_hat kept groups whose removal costs
+    least (Eq. impact by Case 1 / Lemma A.1), all chosen from the scores at the current support, until k remain;
+    the last iteration prunes only what is left to prune.  Everything is recomputed by fresh solves.
+
+    Returns (kept groups sorted, list of the group tuples pruned per iteration in order of increasing score,
+    objective after each iteration with entry 0 = obj of the full support).
+    """
+    H = np.asarray(H, np.float64); G = np.asarray(G, np.float64)
+    ng = H.shape[0] // g
+    S = np.arange(ng)
+    obj = [solve_support(H, G, const, S, g)[1]]
+    dropped = []
+    while len(S) > k:
+        I = rows_of(S, g)
+        L = sla.cho_factor(H[np.ix_(I, I)], lower=True, check_finite=False)
+        Hinv = sla.cho_solve(L, np.eye(len(I)), check_finite=False)
+        V = sla.cho_solve(L, G[I], check_finite=False)
+        st = State(S=S, Hinv=0.5 * (Hinv + Hinv.T), V=V, R=None, c={}, obj=obj[-1])
+        D = drop_scores(st, g)
+        t = min(t_hat, len(S) - k)
+        order = np.lexsort((S, D))[:t]            # smallest score first, ties -> smaller id
+        out = tuple(int(S[i]) for i in order)
+        dropped.append(out)
+        S = np.array([q for q in S if q not in set(out)])
+        obj.append(solve_support(H, G, const, S, g)[1])
+    return np.sort(S), dropped, np.array(obj)
+
+
 # --------------------------------------------------------------------------- exhaustive reference
 def brute_force(H, G, const, g, k):
     """Objective of every support of k groups (Eq. struc by enumeration).  Tiny inputs only."""

@@ -396,3 +396,41 @@ def test_workloads_are_reproducible_and_shaped():
     assert np.mean(x4[:, 4] == 0) == pytest.approx(0.5, abs=0.12)
     # zero padding: the top-left tap of the first patch of an image is outside the map
     assert x4[0, 0] == 0 and x4[49, 0] == 0
+
+
+# ----------------------------------------------------------------------------- nested (greedy) phase
+@pytest.mark.parametrize("g,t_hat", [(1, 1), (1, 3), (2, 2)])
+def test_greedy_phase_prunes_the_cheapest_groups(g, t_hat):
+    """Each iteration of the nested phase removes the kept groups whose individual removal raises the
+    reconstruction error least, as re-solved from X; the objective is non-decreasing and ends at obj of the result."""
+    p, k = 9, 4
+    wl = workloads.tiny(p=p, m=4, g=g, k=k, n=80, seed=13)
+    X, W, H, G, const = problem(wl)
+    S, dropped, obj = orc.greedy_prune(H, G, const, g, k, t_hat)
+    assert len(S) == k and sum(len(d) for d in dropped) == p - k
+    assert abs(obj[0]) < 1e-8 * const                      # full support reproduces the dense layer
+    assert np.all(np.diff(obj) >= -1e-9 * const)
+    cur = list(range(p))
+    for out in dropped:
+        base = orc.solve_support_lstsq(X, W, cur, g)[1]
+        cost = {i: orc.solve_support_lstsq(X, W, [x for x in cur if x != i], g)[1] - base for i in cur}
+        expect = sorted(cur, key=lambda i: (cost[i], i))[:len(out)]
+        assert list(out) == expect
+        cur = [x for x in cur if x not in out]
+    assert sorted(cur) == list(S)
+    assert obj[-1] == pytest.approx(orc.solve_support_lstsq(X, W, list(S), g)[1], rel=1e-8)
+
+
+def test_greedy_phase_on_orthogonal_columns_keeps_the_largest_energies():
+    rng = np.random.default_rng(8)
+    n, p, m, k = 30, 8, 2, 3
+    Q, _ = np.linalg.qr(rng.standard_normal((n, p)))
+    sc = rng.uniform(0.5, 3.0, p)
+    X = Q * sc
+    W = rng.standard_normal((p, m))
+    H, G, const = orc.gram(X, W)
+    e = sc ** 2 * np.sum(W * W, axis=1)
+    S, dropped, obj = orc.greedy_prune(H, G, const, 1, k, 2)
+    assert set(S) == set(np.argsort(-e)[:k])
+    assert [q for d in dropped for q in d] == list(np.argsort(e)[:p - k])
+    assert obj[-1] == pytest.approx(float(np.sum(np.sort(e)[:p - k])), rel=1e-9)
