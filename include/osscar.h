@@ -97,6 +97,22 @@ int osscar_init_support(osscar_ctx* ctx, const float* H, const float* G, const f
                         int64_t d1, int64_t m, int32_t g, int32_t k, int mode,
                         int32_t* support, double* obj0);
 
+/*
+ * Starting support by the nested (greedy) phase of Algorithm 1 (t_i = p_i = t_hat; the paper's own schedule:
+ * Appendix B.1 uses t_hat = 2 for channels and heads, 10 for FC neurons).  All d1/g groups start kept, with
+ * H^-1 and W* = H^-1 G (Algorithm 1, line 1); each iteration prunes the t_hat kept groups whose removal raises
+ * obj least (Eq. impact, evaluated by Case 1 of Proposition 1 / Lemma A.1), all chosen from the scores of the
+ * current support, and moves H_II^-1 and W^(S) with the joint Case-1 downdate; the last iteration prunes only
+ * what is left.  When k groups remain the search state is built as in osscar_init_support, so
+ * osscar_local_search can follow (the paper's "non-nested" refinement).
+ * t_hat * g <= 256, else OSSCAR_E_SHAPE.  support: device int32[k] (sorted ids on return).  drop_trace: device
+ * int32[d1/g - k] or NULL, the pruned groups in pruning order (inside an iteration by increasing score).
+ * obj0: host, obj of the k-group support.  n_iters: host or NULL.  Needs the workspace; synchronises once.
+ */
+int osscar_init_support_greedy(osscar_ctx* ctx, const float* H, const float* G, const float* W,
+                               int64_t d1, int64_t m, int32_t g, int32_t k, int32_t t_hat,
+                               int32_t* support, int32_t* drop_trace, double* obj0, int32_t* n_iters);
+
 typedef struct {
     int32_t max_swaps;        /* >= 0                                                        */
     int32_t score_mode;       /* OSSCAR_SCORE_*                                              */

@@ -22,7 +22,7 @@ STOP_NAMES = {0: "max_swaps", 1: "no_improvement", 2: "guard"}
 
 EXPORTS = ["osscar_create", "osscar_destroy", "osscar_workspace_bytes", "osscar_set_workspace",
            "osscar_gram", "osscar_init_support", "osscar_local_search", "osscar_objective",
-           "osscar_debug_get_state", "osscar_status_string", "osscar_launch_count", "osscar_trace_noalloc"]
+           "osscar_debug_get_state", "osscar_status_string", "osscar_launch_count", "osscar_trace_noalloc", "osscar_init_support_greedy"]
 
 
 class SearchParams(C.Structure):
@@ -74,6 +74,7 @@ def lib() -> C.CDLL:
     L.osscar_set_workspace.argtypes = [vp, vp, C.c_size_t]
     L.osscar_gram.argtypes = [vp, vp, C.c_int, i64, i64, vp, i64, C.c_int, C.c_float, vp, vp, C.POINTER(C.c_double)]
     L.osscar_init_support.argtypes = [vp, vp, vp, vp, i64, i64, i32, i32, C.c_int, vp, C.POINTER(C.c_double)]
+    L.osscar_init_support_greedy.argtypes = [vp, vp, vp, vp, i64, i64, i32, i32, i32, vp, vp, C.POINTER(C.c_double), C.POINTER(i32)]
     L.osscar_local_search.argtypes = [vp, C.POINTER(SearchParams), vp, vp, vp, vp, C.POINTER(SearchResult)]
     L.osscar_objective.argtypes = [vp, vp, vp, vp, i64, i64, C.POINTER(C.c_double)]
     L.osscar_debug_get_state.argtypes = [vp, C.c_int, vp]
@@ -224,6 +225,21 @@ class Solver:
         _check(lib().osscar_init_support(self._h, _ptr(H), _ptr(G), _ptr(W), d1, m, g, k, mode, _ptr(support), C.byref(obj0)),
                "osscar_init_support")
         return support, obj0.value
+
+    def init_support_greedy(self, H, G, W, g: int, k: int, t_hat: int = 1):
+        """Nested (greedy) phase of Algorithm 1 down to k groups, then the search state.  Returns
+        (support int32[k] sorted, drop_trace int32[d1/g - k], obj0, iterations)."""
+        _dev_f32(H, "H"); _dev_f32(G, "G"); _dev_f32(W, "W")
+        d1, m = W.shape
+        self.ensure_workspace(d1, m, g, k)
+        support = torch.empty(k, dtype=torch.int32, device=W.device)
+        drops = torch.empty(max(1, d1 // g - k), dtype=torch.int32, device=W.device)
+        obj0, iters = C.c_double(0.0), C.c_int32(0)
+        self._keep = [H, G, W]
+        self._shape = (d1, m, g, k)
+        _check(lib().osscar_init_support_greedy(self._h, _ptr(H), _ptr(G), _ptr(W), d1, m, g, k, t_hat, _ptr(support),
+                                                _ptr(drops), C.byref(obj0), C.byref(iters)), "osscar_init_support_greedy")
+        return support, drops[:d1 // g - k], obj0.value, iters.value
 
     def local_search(self, max_swaps: int, score_mode: int = SCORE_INDEPENDENT, accept_mode: int = ACCEPT_IMPROVING,
                      refresh_every: int = 0, accept_rel_tol: float = -1.0, profile_samples: int = 0) -> SearchOutput:

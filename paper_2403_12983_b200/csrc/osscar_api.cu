@@ -203,6 +203,35 @@ int osscar_init_support(osscar_ctx* ctx, const float* H, const float* G, const f
     return OSSCAR_OK;
 }
 
+int osscar_init_support_greedy(osscar_ctx* ctx, const float* H, const float* G, const float* W,
+                               int64_t d1, int64_t m, int32_t g, int32_t k, int32_t t_hat,
+                               int32_t* support, int32_t* drop_trace, double* obj0, int32_t* n_iters)
+{
+    if (!ctx || !H || !G || !W || !support || !obj0) return OSSCAR_E_ARG;
+    Layout L;
+    const int rc0 = make_layout(d1, m, g, k, &L);
+    if (rc0 != OSSCAR_OK) return rc0;
+    if (t_hat < 1 || (int64_t)t_hat * g > 256) return OSSCAR_E_SHAPE;
+    if (!ctx->ws || ctx->ws_bytes < L.bytes) return OSSCAR_E_WORKSPACE;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return OSSCAR_E_CUDA;
+    ctx->L = L; ctx->H = H; ctx->G = G; ctx->W = W; ctx->have_state = false;
+    cudaStream_t st = ctx->stream;
+    k_clear_status<<<1, 1, 0, st>>>(ctx->ctl);
+    int iters = 0;
+    int rc = greedy_support(ctx, t_hat, support, drop_trace, &iters);
+    if (rc == OSSCAR_OK) rc = build_state(ctx, false);
+    if (rc == OSSCAR_OK && score_pass(ctx) != cudaSuccess) rc = OSSCAR_E_CUDA;
+    if (rc != OSSCAR_OK) { cudaStreamSynchronize(st); return rc; }
+    CKC(cudaMemcpyAsync(ctx->ctl_host, ctx->ctl, sizeof(SearchCtl), cudaMemcpyDeviceToHost, st));
+    CKC(cudaStreamSynchronize(st));
+    if (ctx->ctl_host->status != OSSCAR_OK) return ctx->ctl_host->status;
+    *obj0 = ctx->ctl_host->obj;
+    if (n_iters) *n_iters = iters;
+    ctx->have_state = true;
+    return OSSCAR_OK;
+}
+
 int osscar_local_search(osscar_ctx* ctx, const osscar_search_params* params,
                         int32_t* support_out, float* W_out, double* obj_trace, int32_t* swap_trace,
                         osscar_search_result* result)

@@ -48,6 +48,7 @@ struct Layout {
     size_t off_vnorm, off_rnorm, off_D, off_A, off_c, off_small, off_gramV, off_gramR;
     size_t off_perm, off_slotof, off_energy, off_panel;
     size_t off_pairCinv, off_pairKK, off_pairScratch, off_pairDelta;   // PAIR_EXACT scoring
+    size_t off_greedy;                                                 // scratch of the nested (greedy) phase
     size_t off_tc, tc_bytes;                                           // bf16 operand terms of the tensor-core GEMMs
     int64_t pair_capacity;                                             // pairs the workspace can score
     size_t bytes;
@@ -99,10 +100,15 @@ cudaError_t gram_mirror(cudaStream_t st, float* H, int64_t d1);   // copy upper 
 // ---- state.cu: support selection and state construction --------------------------------------
 int select_support(osscar_ctx* ctx, int mode, int32_t* support);
 int build_state(osscar_ctx* ctx, bool guarded);
+int invert_spd_inplace(osscar_ctx* ctx, float* A, int64_t lda, int64_t n, const float* ref, int64_t ldref, const int32_t* done);
 cudaError_t gather_rows(cudaStream_t st, const float* src, int64_t m, int g, const int32_t* perm,
                         int64_t slot_row0, int64_t nrows, float* dst, int64_t ld);
 cudaError_t trace_product(cudaStream_t st, const float* A, int64_t lda, const float* B, int64_t ldb,
                           int64_t rows, int64_t cols, double* partials, double* out_dev);   // *out = sum A.*B
+
+// ---- greedy.cu: nested phase of Algorithm 1 down to L.k groups (leaves the slot permutation in the workspace) -----
+size_t greedy_scratch_bytes(int64_t d1, int64_t m, int g);
+int greedy_support(osscar_ctx* ctx, int t_hat, int32_t* support, int32_t* drop_trace, int32_t* n_iters_out);
 
 // ---- search.cu -------------------------------------------------------------------------------
 int run_search(osscar_ctx* ctx, const osscar_search_params* p, int32_t* support_out, float* W_out,

@@ -300,6 +300,10 @@ int make_layout(int64_t d1, int64_t m, int32_t g, int32_t k, Layout* L)
     const int64_t npairs = (int64_t)k * (ng - k);
     L->pair_capacity = npairs <= kMaxPairs ? npairs : 0;
     if (L->pair_capacity > 0 && nJ * ldh + nI * round_up(nJ, kPadF) > big) big = nJ * ldh + nI * round_up(nJ, kPadF);
+    {   // the nested phase keeps V of all rows plus up to 256 staged rows of Hinv (twice) and of V in `big`
+        const int64_t gneed = d1 * ldm + 2 * 256 * L->ldp + 256 * ldm;
+        if (gneed > big) big = gneed;
+    }
     L->off_big = take(sizeof(float) * big);
     L->off_Hp = take(sizeof(float) * d1 * L->ldp);
     L->off_Hinv = take(sizeof(float) * nI * ldh);
@@ -327,13 +331,14 @@ int make_layout(int64_t d1, int64_t m, int32_t g, int32_t k, Layout* L)
     L->off_perm = take(sizeof(int32_t) * ng);
     L->off_slotof = take(sizeof(int32_t) * ng);
     L->off_energy = take(sizeof(double) * ng + sizeof(int32_t) * ng);
-    L->off_panel = take(sizeof(float) * (nI * NB + 2 * NB * ldh + NB * NB));
+    L->off_panel = take(sizeof(float) * (d1 * NB + 2 * NB * L->ldp + NB * NB));
     const size_t gg8 = sizeof(double) * g * g;
     const bool pairs_ok = L->pair_capacity > 0;
     L->off_pairCinv = take(pairs_ok ? gg8 * k : 8);
     L->off_pairKK = take(pairs_ok ? gg8 * k : 8);
     L->off_pairScratch = take(pairs_ok ? gg8 * 8 * 296 : 8);
     L->off_pairDelta = take(pairs_ok ? sizeof(double) * L->pair_capacity : 8);
+    L->off_greedy = take(greedy_scratch_bytes(d1, m, g));
     {   // K panels of up to 2048 for the widest products of the state build (M <= d1, N <= max(m, n_I))
         const int64_t nmax = ldm > ldh ? ldm : ldh;
         L->tc_bytes = 3 * ((size_t)d1 * 2048 * 2 + (size_t)2048 * nmax * 2) + 16 * 1024;
@@ -367,6 +372,39 @@ int select_support(osscar_ctx* ctx, int mode, int32_t* support)
     return OSSCAR_OK;
 }
 
+// In-place inverse of the n x n SPD matrix A (row stride lda) by the blocked exchange (Gauss-Jordan) scheme:
+// per 64-wide pivot block an fp64 Cholesky inverse, then one rank-64 update of the whole matrix in a GEMM.
+// `ref` (row stride ldref) supplies the original diagonal, the scale of the positive-definiteness test.
+int invert_spd_inplace(osscar_ctx* ctx, float* A, int64_t lda, int64_t n, const float* ref, int64_t ldref, const int32_t* done)
+{
+    const Layout& L = ctx->L;
+    cudaStream_t st = ctx->stream;
+    float* T = (float*)((char*)ctx->ws + L.off_panel);
+    float* U = T + L.d1 * NB;
+    float* Un = U + NB * L.ldp;
+    float* Dinv = Un + NB * L.ldp;
+    CK(cudaFuncSetAttribute(k_pivot_inverse, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * NB * NB * (int)sizeof(double)));
+    for (int64_t p0 = 0; p0 < n; p0 += NB) {
+        const int nb = (int)(n - p0 < NB ? n - p0 : NB);
+        k_pivot_inverse<<<1, 256, 2 * NB * NB * sizeof(double), st>>>(A, lda, p0, nb, Dinv, ref, ldref, ctx->ctl);
+        // T = A[:, P] * Dinv
+        CK(sgemm(st, false, false, n, nb, nb, 1.f, A + p0, lda, Dinv, NB, 0.f, T, NB, done));
+        k_zero_rows<<<(nb * nb + 255) / 256, 256, 0, st>>>(T, NB, p0, nb, nb);
+        {
+            dim3 grid((unsigned)((n + 255) / 256 < 32 ? (n + 255) / 256 : 32), (unsigned)nb);
+            k_copy_rows<<<grid, 256, 0, st>>>(A, lda, p0, nb, n, U, lda);
+        }
+        CK(sgemm(st, false, false, nb, n, nb, -1.f, Dinv, NB, U, lda, 0.f, Un, lda, done));
+        // the rank-64 updates stay on the fp32 pipes: the inversion amplifies rounding by cond(A), and the tensor
+        // core's truncating accumulation is biased where fp32 FMA chains are not
+        CK(sgemm(st, false, false, n, n, nb, -1.f, T, NB, U, lda, 1.f, A, lda, done));
+        k_gj_writeback<<<(unsigned)((n * nb + 255) / 256), 256, 0, st>>>(A, lda, n, p0, nb, T, NB, Un, lda, Dinv);
+        count_launches(4);     // pivot inverse, zero rows, copy rows, write-back (the GEMMs count themselves)
+    }
+    CK(cudaGetLastError());
+    return OSSCAR_OK;
+}
+
 // Rebuilds every piece of the search state from H, G and the current slot permutation.
 // With `guarded`, the kernels that can be skipped return at once when the loop has stopped.
 int build_state(osscar_ctx* ctx, bool guarded)
@@ -381,10 +419,6 @@ int build_state(osscar_ctx* ctx, bool guarded)
     float* big = (float*)(ws + L.off_big);
     double* c = (double*)(ws + L.off_c);
     const int32_t* perm = (const int32_t*)(ws + L.off_perm);
-    float* T = (float*)(ws + L.off_panel);
-    float* U = T + L.nI * NB;
-    float* Un = U + NB * L.ldh;
-    float* Dinv = Un + NB * L.ldh;
     const int32_t* done = guarded ? &ctx->ctl->done : nullptr;
     void* tc = ws + L.off_tc;
     const int64_t nI = L.nI, nJ = L.nJ;
@@ -397,25 +431,7 @@ int build_state(osscar_ctx* ctx, bool guarded)
     k_copy_pad<<<(unsigned)nI, 256, 0, st>>>(Hp, L.ldp, nI, nI, Hinv, L.ldh);
     count_launches(2);
     CK(cudaGetLastError());
-    CK(cudaFuncSetAttribute(k_pivot_inverse, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * NB * NB * (int)sizeof(double)));
-    for (int64_t p0 = 0; p0 < nI; p0 += NB) {
-        const int nb = (int)(nI - p0 < NB ? nI - p0 : NB);
-        k_pivot_inverse<<<1, 256, 2 * NB * NB * sizeof(double), st>>>(Hinv, L.ldh, p0, nb, Dinv, Hp, L.ldp, ctx->ctl);
-        // T = A[:, P] * Dinv
-        CK(sgemm(st, false, false, nI, nb, nb, 1.f, Hinv + p0, L.ldh, Dinv, NB, 0.f, T, NB, done));
-        k_zero_rows<<<(nb * nb + 255) / 256, 256, 0, st>>>(T, NB, p0, nb, nb);
-        {
-            dim3 grid((unsigned)((nI + 255) / 256 < 32 ? (nI + 255) / 256 : 32), (unsigned)nb);
-            k_copy_rows<<<grid, 256, 0, st>>>(Hinv, L.ldh, p0, nb, nI, U, L.ldh);
-        }
-        CK(sgemm(st, false, false, nb, nI, nb, -1.f, Dinv, NB, U, L.ldh, 0.f, Un, L.ldh, done));
-        // the rank-64 updates stay on the fp32 pipes: the inversion amplifies rounding by cond(H_II), and the tensor
-        // core's truncating accumulation is biased where fp32 FMA chains are not
-        CK(sgemm(st, false, false, nI, nI, nb, -1.f, T, NB, U, L.ldh, 1.f, Hinv, L.ldh, done));
-        k_gj_writeback<<<(unsigned)((nI * nb + 255) / 256), 256, 0, st>>>(Hinv, L.ldh, nI, p0, nb, T, NB, Un, L.ldh, Dinv);
-        count_launches(4);     // pivot inverse, zero rows, copy rows, write-back (the GEMMs count themselves)
-    }
-    CK(cudaGetLastError());
+    { const int rc_inv = invert_spd_inplace(ctx, Hinv, L.ldh, nI, Hp, L.ldp, done); if (rc_inv != OSSCAR_OK) return rc_inv; }
     // V = Hinv * G_I
     k_gather_rows<<<(unsigned)nI, 256, 0, st>>>(ctx->G, L.m, L.g, perm, 0, big, L.ldm);
     if (L.ldm != L.m) CK(cudaMemsetAsync(V, 0, sizeof(float) * nI * L.ldm, st));     // padding columns stay zero

@@ -74,3 +74,32 @@ def follow_trace(H, G, const, g, S0, swaps, gpu_obj, score_mode="independent", a
 def rel_fro(a, b):
     a = np.asarray(a, np.float64); b = np.asarray(b, np.float64)
     return float(np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-300))
+
+
+def follow_greedy(H, G, const, g, k, t_hat, drops):
+    """Walks the GPU's nested (greedy) phase with the oracle: per iteration the groups the GPU pruned must be the
+    t cheapest by the oracle's fresh scores, up to ties within GAP; the oracle then continues from the GPU's set."""
+    import scipy.linalg as sla
+    ng = H.shape[0] // g
+    S = np.arange(ng)
+    pos = 0
+    while len(S) > k:
+        t = min(t_hat, len(S) - k)
+        I = orc.rows_of(S, g)
+        L = sla.cho_factor(H[np.ix_(I, I)], lower=True, check_finite=False)
+        Hinv = sla.cho_solve(L, np.eye(len(I)), check_finite=False)
+        V = sla.cho_solve(L, G[I], check_finite=False)
+        D = orc.drop_scores(orc.State(S=S, Hinv=0.5 * (Hinv + Hinv.T), V=V, R=None, c={}, obj=0.0), g)
+        out = [int(q) for q in drops[pos:pos + t]]
+        assert len(set(out)) == t and all(q in S for q in out), f"iteration at {pos}: bad drop set {out}"
+        thr = np.sort(D)[t - 1]
+        idx = {int(q): i for i, q in enumerate(S)}
+        for q in out:
+            assert D[idx[q]] <= thr * (1 + GAP) + 1e-300, f"pruned group {q} is not among the {t} cheapest"
+        for q in S:
+            if int(q) not in out:
+                assert D[idx[int(q)]] >= thr * (1 - GAP) - 1e-300, f"group {q} is cheaper than the pruned ones"
+        keep = np.array([q for q in S if int(q) not in set(out)])
+        S = keep
+        pos += t
+    return np.sort(S)

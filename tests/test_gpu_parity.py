@@ -5,7 +5,7 @@ import torch
 
 import workloads
 from oracle import osscar_oracle as orc
-from tests.parity import GAP, follow_trace, oracle_problem, rel_fro
+from tests.parity import GAP, follow_greedy, follow_trace, oracle_problem, rel_fro
 
 pytestmark = pytest.mark.gpu
 
@@ -328,6 +328,40 @@ def test_state_after_search_is_consistent(solver):
     assert rel_fro(solver.debug_state(2).cpu().numpy(), st.R[perm[wl.k:]]) < 1e-4
     c = solver.debug_state(3).cpu().numpy().reshape(-1)
     assert np.allclose(c, [st.c[int(q)][0, 0] for q in perm[wl.k:]], rtol=1e-3)
+
+
+# ------------------------------------------------------------------------------------ nested (greedy) phase
+GREEDY_CASES = [
+    ("c1", {}, 1),
+    ("c1", {}, 5),
+    ("c2", dict(n=4096, d1=520, m=150, k=207, chunk_rows=4096), 10),
+    ("c5", dict(n=4096, d1=264, m=72, k=80, chunk_rows=4096), 7),
+    ("c4", dict(n=49 * 40, d1=9 * 60, m=130, k=25, chunk_rows=49 * 40), 2),
+    ("c3", dict(n=8192, d1=12 * 40, m=200, g=40, k=6, chunk_rows=8192), 2),
+]
+
+
+@pytest.mark.parametrize("name,over,t_hat", GREEDY_CASES)
+def test_greedy_phase_matches_oracle(solver, name, over, t_hat):
+    """Nested phase of Algorithm 1 from the dense layer down to k groups, then the swap search from there."""
+    wl = workloads.config(name, **over)
+    chunks, W, H64, G64, const64 = oracle_problem(wl)
+    H, G, Wd = dev(H64), dev(G64), dev(W)
+    Hr, Gr = H.cpu().numpy().astype(np.float64), G.cpu().numpy().astype(np.float64)
+    const_r = float(np.sum(W * Gr))
+    support, drops, obj0, iters = solver.init_support_greedy(H, G, Wd, wl.g, wl.k, t_hat)
+    npr = wl.ngroups - wl.k
+    assert iters == -(-npr // t_hat) and len(drops) == npr
+    S_or = follow_greedy(Hr, Gr, const_r, wl.g, wl.k, t_hat, drops.cpu().numpy())
+    assert np.array_equal(support.cpu().numpy(), S_or)
+    assert obj0 == pytest.approx(orc.solve_support(Hr, Gr, const_r, S_or, wl.g)[1], rel=1e-4)
+    # the state handed over is the regular one: the swap search continues from it and follows the oracle
+    out = solver.local_search(20, accept_rel_tol=wl.eps_acc)
+    swaps = [tuple(int(v) for v in r) for r in out.swap_trace.cpu().numpy()]
+    srch, _ = follow_trace(Hr, Gr, const_r, wl.g, S_or, swaps, out.obj_trace.cpu().numpy(), gpu_stop=out.stop_reason,
+                           max_swaps=20, eps_acc=wl.eps_acc)
+    assert np.array_equal(out.support.cpu().numpy(), srch.result()[0])
+    assert out.obj_final == pytest.approx(srch.st.obj, rel=1e-4)
 
 
 # ------------------------------------------------------------------------------------ edge cases and errors
