@@ -212,7 +212,7 @@ def run_ours(args):
     def step(x_chunks, W_in, prof=0):
         return pkg.solve_layer(solver, x_chunks, W_in, wl.g, wl.k, max_swaps, damp=wl.damp, accept_mode=accept, accept_rel_tol=wl.eps_acc,
                                score_mode=b.SCORE_PAIR_EXACT if wl.score_mode == "pair_exact" else b.SCORE_INDEPENDENT,
-                               profile_samples=prof, H=H, G=G)
+                               profile_samples=prof, H=H, G=G, greedy_t_hat=args.greedy)
 
     def barrier():
         if world > 1:
@@ -319,7 +319,8 @@ def run_ours(args):
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32 (bf16 tensor-core Gram, fp32 accumulate)", "data": "synthetic",
         "config": {"workload": f"{wl.name}: d1={wl.d1} m={wl.m} g={wl.g} k={wl.k} n={wl.n} in {wl.n_chunks} chunks, "
-                               f"max_swaps={max_swaps}, accept={'always' if args.accept_always else 'improving'} (eps {wl.eps_acc:g}), damp={wl.damp}",
+                               f"max_swaps={max_swaps}, accept={'always' if args.accept_always else 'improving'} (eps {wl.eps_acc:g}), damp={wl.damp}, "
+                               f"init={'greedy t_hat=%d' % args.greedy if args.greedy else 'energy'}",
                    "l2": "inputs larger than L2 (X, H and the search state are each > 126 MB)" if wl.d1 >= 8192 else
                          "state smaller than L2; numbers are cache-resident",
                    "replicas": world},
@@ -363,6 +364,7 @@ def main():
     ap.add_argument("--m", type=int, default=None)
     ap.add_argument("--k", type=int, default=None)
     ap.add_argument("--max-swaps", type=int, default=None)
+    ap.add_argument("--greedy", type=int, default=0, help="start from the nested phase of Algorithm 1 with this t_hat")
     ap.add_argument("--accept-always", action="store_true", help="paper-literal fixed number of iterations")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")

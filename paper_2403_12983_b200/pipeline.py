@@ -63,9 +63,11 @@ def solve_layer(solver: b.Solver, x_chunks: Sequence[torch.Tensor], W: torch.Ten
                 max_swaps: int, damp: float = 0.0, init_mode: int = b.INIT_ENERGY,
                 score_mode: int = b.SCORE_INDEPENDENT, accept_mode: int = b.ACCEPT_IMPROVING,
                 refresh_every: int = 0, profile_samples: int = 0, accept_rel_tol: float = -1.0,
-                H: Optional[torch.Tensor] = None, G: Optional[torch.Tensor] = None) -> LayerResult:
+                H: Optional[torch.Tensor] = None, G: Optional[torch.Tensor] = None,
+                greedy_t_hat: int = 0) -> LayerResult:
     """Prunes one layer to k groups of g rows.  W: d1 x m fp32 (device or host); x_chunks: row blocks of X
-    (bf16 or fp32; all on the device, or all on the host)."""
+    (bf16 or fp32; all on the device, or all on the host).  greedy_t_hat > 0 starts from the nested phase with
+    that many groups pruned per iteration instead of the energy ranking."""
     dev = torch.device("cuda", solver.device)
     host_x = not x_chunks[0].is_cuda
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(5)]
@@ -88,7 +90,10 @@ def solve_layer(solver: b.Solver, x_chunks: Sequence[torch.Tensor], W: torch.Ten
     ev[1].record()
     const = solver.gram_chunk(x_chunks[0][:0] if not host_x else solver._stage[0][:0], H, b.GRAM_END, W, G, damp)
     ev[2].record()
-    support0, obj0 = solver.init_support(H, G, W, g, k, init_mode)
+    if greedy_t_hat > 0:          # the paper's own start: nested phase of Algorithm 1 from the dense layer
+        support0, _, obj0, _ = solver.init_support_greedy(H, G, W, g, k, greedy_t_hat)
+    else:
+        support0, obj0 = solver.init_support(H, G, W, g, k, init_mode)
     ev[3].record()
     out = solver.local_search(max_swaps, score_mode, accept_mode, refresh_every, accept_rel_tol=accept_rel_tol,
                               profile_samples=profile_samples)
