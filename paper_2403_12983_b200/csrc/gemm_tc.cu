@@ -10,6 +10,10 @@
 // chains would cost accuracy; the register sums are round-to-nearest.
 //   warp 0: TMA producer     warp 1: MMA issuer     warps 2-9: accumulate (TMEM -> registers) and write C
 // K is processed in panels sized to the caller's scratch (the bf16 terms of one panel of A and B live there).
+//
+// The same pipeline, instantiated with an MN-major A operand and a single bf16 term, is the Gram kernel
+// H (+)= Xc^T Xc over the upper-triangle tiles (chains of 32 k-blocks between drains), and with B taken from a
+// second matrix the cross term G (+)= Xc^T Yc (Y in bf16, or fp32 split into three terms).
 #include "osscar_internal.cuh"
 #include <cuda_bf16.h>
 #include "tc_common.cuh"
@@ -27,13 +31,23 @@ constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256;
 constexpr int NUM_THREADS = 320;                              // 10 warps
 constexpr int TMEM_COLS = 512;
-constexpr int kFlush = 2;                                     // k-blocks (x 6 term pairs) per TMEM accumulation chain
-constexpr int kTerms = 6;
-constexpr int BAND = 8;                                       // tile rows per raster band
+constexpr int BAND = 8;                                       // tile rows per raster band (full rasters)
+constexpr int TRI_BAND = 16;                                  // same for the upper-triangle raster
 
-// kind::f16, D fp32, A/B bf16, A K-major, B MN-major, M = 128, N = 256.
-constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16)
-                          | ((uint32_t)(TILE_N >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
+// Variants of the pipeline.
+enum { MODE_GEMM3 = 0,      // A fp32 split, K-major; B fp32 split; six term pairs; all tiles
+       MODE_GRAM = 1,       // A = B = X (bf16, MN-major); one term; upper-triangle tiles
+       MODE_CROSS = 2,      // A = X (MN-major), B = Y bf16; one term; all tiles
+       MODE_CROSS3 = 3 };   // A = X (MN-major), B = Y fp32 split in three terms
+template <int MODE> struct Traits {
+    static constexpr bool kAMN = MODE != MODE_GEMM3;
+    static constexpr int kTerms = MODE == MODE_GEMM3 ? 6 : (MODE == MODE_CROSS3 ? 3 : 1);
+    static constexpr bool kUpper = MODE == MODE_GRAM;
+    // k-blocks per TMEM accumulation chain: short where small terms ride on large ones, 32 (128 MMAs) for plain bf16
+    static constexpr int kFlush = MODE == MODE_GEMM3 ? 2 : (MODE == MODE_CROSS3 ? 4 : 32);
+    static constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((kAMN ? 1u : 0u) << 15) | (1u << 16)
+                                     | ((uint32_t)(TILE_N >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
+};
 
 // A tile: K-major, SWIZZLE_128B: rows of 128 bytes, 8-row swizzle atoms 1024 bytes apart (stride byte offset);
 // the leading byte offset is not used by swizzled K-major layouts.
@@ -47,18 +61,45 @@ __device__ __forceinline__ uint64_t desc_b(uint32_t saddr) {
 
 struct Maps { CUtensorMap a[3]; CUtensorMap b[3]; };
 
-__device__ __forceinline__ void tile_of(int id, int TM, int TN, int* tm, int* tn) {
+__device__ __forceinline__ void tile_full(int id, int TM, int TN, int* tm, int* tn) {
     // bands of BAND tile rows, column-major inside a band: concurrent CTAs share A rows and B columns in L2
     const int per_band = BAND * TN;
     const int b = id / per_band, r = id % per_band;
     const int rows = min(BAND, TM - b * BAND);
     *tn = r / rows; *tm = b * BAND + r % rows;
 }
+// Upper-triangle tiles of a symmetric result (tile (tm, tn) exists iff tn >= tm / 2), bands of TRI_BAND rows.
+__device__ __forceinline__ void tile_upper(int id, int TM, int TN, int* tm_out, int* tn_out) {
+    int b = 0;
+    while (true) {
+        int cnt = 0;
+        const int r1 = min(TM, (b + 1) * TRI_BAND);
+        for (int tm = b * TRI_BAND; tm < r1; ++tm) cnt += TN - tm / 2;
+        if (id < cnt) break;
+        id -= cnt; ++b;
+    }
+    const int r0 = b * TRI_BAND, r1 = min(TM, r0 + TRI_BAND);
+    for (int tn = r0 / 2; tn < TN; ++tn) {
+        const int last = min(r1 - 1, 2 * tn + 1);
+        const int cnt = last - r0 + 1;
+        if (id < cnt) { *tm_out = r0 + id; *tn_out = tn; return; }
+        id -= cnt;
+    }
+    *tm_out = r0; *tn_out = TN - 1;
+}
+template <bool UPPER> __device__ __forceinline__ void tile_of(int id, int TM, int TN, int* tm, int* tn) {
+    if (UPPER) tile_upper(id, TM, TN, tm, tn); else tile_full(id, TM, TN, tm, tn);
+}
 
+template <int MODE>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-k_gemm3(const __grid_constant__ Maps maps, int64_t M, int64_t N, int64_t K, float alpha, float beta,
-        float* __restrict__ C, int64_t ldc, int vec_ok, int32_t* __restrict__ status, const int32_t* __restrict__ done)
+k_mma_pipe(const __grid_constant__ Maps maps, int64_t M, int64_t N, int64_t K, float alpha, float beta,
+           float* __restrict__ C, int64_t ldc, int vec_ok, int num_ids, int32_t* __restrict__ status,
+           const int32_t* __restrict__ done)
 {
+    using TR = Traits<MODE>;
+    constexpr int kTerms = TR::kTerms, kFlush = TR::kFlush;
+    constexpr uint32_t kIdesc = TR::kIdesc;
     if (done && *done) return;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -74,9 +115,6 @@ k_gemm3(const __grid_constant__ Maps maps, int64_t M, int64_t N, int64_t K, floa
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int TM = (int)((M + TILE_M - 1) / TILE_M), TN = (int)((N + TILE_N - 1) / TILE_N);
-    // the band raster enumerates BAND * TN ids per band; the last band may be short
-    const int full_bands = TM / BAND, rem_rows = TM % BAND;
-    const int num_ids = full_bands * BAND * TN + rem_rows * TN;
     const int nkb = (int)((K + BLOCK_K - 1) / BLOCK_K);
     const int nflush = (nkb + kFlush - 1) / kFlush;
 
@@ -101,19 +139,26 @@ k_gemm3(const __grid_constant__ Maps maps, int64_t M, int64_t N, int64_t K, floa
             bool ok = true;
             for (int id = blockIdx.x; id < num_ids && ok; id += gridDim.x) {
                 int tm, tn;
-                tile_of(id, TM, TN, &tm, &tn);
+                tile_of<TR::kUpper>(id, TM, TN, &tm, &tn);
                 for (int kb = 0; kb < nkb && ok; ++kb) {
                     for (int term = 0; term < kTerms; ++term, ++it) {
                         // term pairs, small products first: (3,1) (2,2) (1,3) (2,1) (1,2) (1,1)
-                        const int pa = (0x001012 >> (4 * term)) & 0xF;      // index of the A term: 2,1,0,1,0,0
-                        const int pb = (0x010210 >> (4 * term)) & 0xF;      // index of the B term: 0,1,2,0,1,0
+                        const int pa = MODE == MODE_GEMM3 ? (0x001012 >> (4 * term)) & 0xF : 0;     // A term: 2,1,0,1,0,0
+                        const int pb = MODE == MODE_GEMM3 ? (0x010210 >> (4 * term)) & 0xF          // B term: 0,1,2,0,1,0
+                                     : (MODE == MODE_CROSS3 ? 2 - term : 0);
                         const int s = it % STAGES;
                         const uint32_t ph = (it / STAGES) & 1;
                         if (!mbar_wait(empty_bar(s), ph ^ 1, abort_flag)) { ok = false; break; }
                         mbar_expect_tx(full_bar(s), STAGE_BYTES);
                         const uint32_t a_dst = tiles_base + s * STAGE_BYTES;
                         const uint32_t b_dst = a_dst + A_BYTES;
-                        tma_load_2d(a_dst, &maps.a[pa], full_bar(s), kb * BLOCK_K, tm * TILE_M);
+                        if (TR::kAMN) {         // A^T tile: two boxes of 64 columns x 64 k-rows
+#pragma unroll
+                            for (int i = 0; i < TILE_M / 64; ++i)
+                                tma_load_2d(a_dst + i * BOX_BYTES, &maps.a[pa], full_bar(s), tm * TILE_M + i * 64, kb * BLOCK_K);
+                        } else {
+                            tma_load_2d(a_dst, &maps.a[pa], full_bar(s), kb * BLOCK_K, tm * TILE_M);
+                        }
 #pragma unroll
                         for (int i = 0; i < TILE_N / 64; ++i)
                             tma_load_2d(b_dst + i * BOX_BYTES, &maps.b[pb], full_bar(s), tn * TILE_N + i * 64, kb * BLOCK_K);
@@ -151,8 +196,9 @@ k_gemm3(const __grid_constant__ Maps maps, int64_t M, int64_t N, int64_t K, floa
                             const uint32_t b_src = a_src + A_BYTES;
 #pragma unroll
                             for (int j = 0; j < BLOCK_K / UMMA_K; ++j) {
-                                // A: +32 bytes per 16 k inside the 128-byte row; B: +16 k-rows of 128 bytes
-                                umma_f16(d_tmem, desc_a(a_src + j * 32), desc_b(b_src + j * (UMMA_K * 128)), kIdesc, first ? 0u : 1u);
+                                // K-major A: +32 bytes per 16 k inside the 128-byte row; MN-major: +16 k-rows of 128 bytes
+                                const uint64_t ad = TR::kAMN ? desc_b(a_src + j * (UMMA_K * 128)) : desc_a(a_src + j * 32);
+                                umma_f16(d_tmem, ad, desc_b(b_src + j * (UMMA_K * 128)), kIdesc, first ? 0u : 1u);
                                 first = false;
                             }
                             umma_commit(empty_bar(s));
@@ -169,7 +215,7 @@ k_gemm3(const __grid_constant__ Maps maps, int64_t M, int64_t N, int64_t K, floa
         bool ok = true;
         for (int id = blockIdx.x; id < num_ids && ok; id += gridDim.x) {
             int tm, tn;
-            tile_of(id, TM, TN, &tm, &tn);
+            tile_of<TR::kUpper>(id, TM, TN, &tm, &tn);
             float acc[128];
 #pragma unroll
             for (int j = 0; j < 128; ++j) acc[j] = 0.f;
@@ -294,7 +340,7 @@ cudaError_t gemm_tc(cudaStream_t st, int64_t M, int64_t N, int64_t K, float alph
     if (e != cudaSuccess) return e;
     e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(k_gemm3, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    e = cudaFuncSetAttribute(k_mma_pipe<MODE_GEMM3>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e != cudaSuccess) return e;
     const int TM = (int)((M + TILE_M - 1) / TILE_M), TN = (int)((N + TILE_N - 1) / TILE_N);
     const int num_ids = TM * TN;
@@ -311,12 +357,76 @@ cudaError_t gemm_tc(cudaStream_t st, int64_t M, int64_t N, int64_t K, float alph
             if (!encode_2d(enc, &maps.b[i], bp[i], (uint64_t)N, (uint64_t)kw, (uint64_t)ldn, 64, BLOCK_K)) return cudaErrorInvalidValue;
         }
         const int grid = num_ids < sms ? num_ids : sms;
-        k_gemm3<<<grid, NUM_THREADS, SMEM_BYTES, st>>>(maps, M, N, kw, alpha, k0 == 0 ? beta : 1.f, C, ldc, vec_ok, status_dev, done);
+        k_mma_pipe<MODE_GEMM3><<<grid, NUM_THREADS, SMEM_BYTES, st>>>(maps, M, N, kw, alpha, k0 == 0 ? beta : 1.f, C, ldc, vec_ok,
+                                                                      num_ids, status_dev, done);
         count_launches(3);
         e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }
     return cudaSuccess;
+}
+
+// H (+)= Xc^T Xc over the upper-triangle tiles (Yc == nullptr), or G (+)= Xc^T Yc over all tiles.
+// Xc: n_rows x d1 bf16.  Yc: n_rows x m, bf16 (y_fp32 == 0) or fp32, which is split into three bf16 terms in
+// `scratch` (3 * n_rows * round_up(m, 8) * 2 bytes, 1024-byte aligned pieces).
+cudaError_t gram_tc2(cudaStream_t st, const void* X, int64_t n_rows, int64_t d1, const void* Y, int y_fp32, int64_t m,
+                     float* C, bool accumulate, void* scratch, size_t scratch_bytes, int32_t* status_dev)
+{
+    if (n_rows <= 0) return cudaSuccess;
+    if (((uintptr_t)X & 15) || (d1 % 8) != 0) return cudaErrorInvalidValue;
+    PFN_encodeTiled enc = get_encode();
+    if (!enc) return cudaErrorNotSupported;
+    int dev = 0, sms = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    Maps maps;
+    if (!encode_2d(enc, &maps.a[0], X, (uint64_t)d1, (uint64_t)n_rows, (uint64_t)d1, 64, BLOCK_K)) return cudaErrorInvalidValue;
+    maps.a[1] = maps.a[2] = maps.a[0];
+    const float beta = accumulate ? 1.f : 0.f;
+    const int TM = (int)((d1 + TILE_M - 1) / TILE_M);
+    if (!Y) {
+        for (int i = 0; i < 3; ++i) maps.b[i] = maps.a[0];
+        const int TN = (int)((d1 + TILE_N - 1) / TILE_N);
+        int num_ids = 0;
+        for (int tm = 0; tm < TM; ++tm) num_ids += TN - tm / 2;
+        const int vec_ok = (((uintptr_t)C & 15) == 0 && (d1 % 4) == 0) ? 1 : 0;
+        e = cudaFuncSetAttribute(k_mma_pipe<MODE_GRAM>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        k_mma_pipe<MODE_GRAM><<<num_ids < sms ? num_ids : sms, NUM_THREADS, SMEM_BYTES, st>>>(
+            maps, d1, d1, n_rows, 1.f, beta, C, d1, vec_ok, num_ids, status_dev, nullptr);
+        count_launches(1);
+        return cudaGetLastError();
+    }
+    const int TN = (int)((m + TILE_N - 1) / TILE_N);
+    const int num_ids = TM * TN;
+    const int vec_ok = (((uintptr_t)C & 15) == 0 && (m % 4) == 0) ? 1 : 0;
+    if (!y_fp32) {
+        if (((uintptr_t)Y & 15) || (m % 8) != 0) return cudaErrorInvalidValue;
+        if (!encode_2d(enc, &maps.b[0], Y, (uint64_t)m, (uint64_t)n_rows, (uint64_t)m, 64, BLOCK_K)) return cudaErrorInvalidValue;
+        maps.b[1] = maps.b[2] = maps.b[0];
+        e = cudaFuncSetAttribute(k_mma_pipe<MODE_CROSS>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        k_mma_pipe<MODE_CROSS><<<num_ids < sms ? num_ids : sms, NUM_THREADS, SMEM_BYTES, st>>>(
+            maps, d1, m, n_rows, 1.f, beta, C, m, vec_ok, num_ids, status_dev, nullptr);
+        count_launches(1);
+        return cudaGetLastError();
+    }
+    const int64_t ldn = round_up(m, 8);
+    const size_t piece = ((size_t)n_rows * ldn * 2 + 1023) / 1024 * 1024;
+    if (!scratch || scratch_bytes < 3 * piece || ((uintptr_t)scratch & 255)) return cudaErrorInvalidValue;
+    __nv_bfloat16* yp[3];
+    for (int i = 0; i < 3; ++i) yp[i] = (__nv_bfloat16*)((char*)scratch + i * piece);
+    k_split3<<<1184, 256, 0, st>>>((const float*)Y, m, n_rows, m, yp[0], yp[1], yp[2], ldn, nullptr);
+    for (int i = 0; i < 3; ++i)
+        if (!encode_2d(enc, &maps.b[i], yp[i], (uint64_t)m, (uint64_t)n_rows, (uint64_t)ldn, 64, BLOCK_K)) return cudaErrorInvalidValue;
+    e = cudaFuncSetAttribute(k_mma_pipe<MODE_CROSS3>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    k_mma_pipe<MODE_CROSS3><<<num_ids < sms ? num_ids : sms, NUM_THREADS, SMEM_BYTES, st>>>(
+        maps, d1, m, n_rows, 1.f, beta, C, m, vec_ok, num_ids, status_dev, nullptr);
+    count_launches(2);
+    return cudaGetLastError();
 }
 
 }  // namespace osscar

@@ -145,7 +145,7 @@ int osscar_gram(osscar_ctx* ctx, const void* X, int x_dtype, int64_t n_rows, int
     if (n_rows > 0) {
         if (x_dtype == OSSCAR_BF16) {
             // upper-triangle tiles only; the lower triangle is filled on END
-            CKC(gram_bf16_tcgen05(st, X, n_rows, d1, H, !begin, &ctx->ctl->status));
+            CKC(gram_tc2(st, X, n_rows, d1, nullptr, 0, 0, H, !begin, nullptr, 0, &ctx->ctl->status));
         } else {
             CKC(sgemm(st, true, false, d1, d1, n_rows, 1.f, (const float*)X, d1, (const float*)X, d1,
                       begin ? 0.f : 1.f, H, d1));

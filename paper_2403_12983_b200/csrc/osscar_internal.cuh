@@ -92,9 +92,11 @@ cudaError_t gemm_tc(cudaStream_t st, int64_t M, int64_t N, int64_t K, float alph
                     const float* B, int64_t ldb, float beta, float* C, int64_t ldc,
                     void* scratch, size_t scratch_bytes, int32_t* status_dev, const int32_t* done = nullptr);
 
-// ---- gram_tc.cu: H (+)= Xc^T Xc on the tensor cores (bf16 in, fp32 out) ----------------------
-cudaError_t gram_bf16_tcgen05(cudaStream_t st, const void* X, int64_t n_rows, int64_t d1,
-                              float* H, bool accumulate, int32_t* status_dev);
+// H (+)= Xc^T Xc (upper-triangle tiles; Y null) or G (+)= Xc^T Yc with the drained-accumulator pipeline of gemm_tc.cu.
+cudaError_t gram_tc2(cudaStream_t st, const void* X, int64_t n_rows, int64_t d1, const void* Y, int y_fp32, int64_t m,
+                     float* C, bool accumulate, void* scratch, size_t scratch_bytes, int32_t* status_dev);
+
+// ---- gram_tc.cu ---------------------------------------------------------------------------------------------
 cudaError_t gram_mirror(cudaStream_t st, float* H, int64_t d1);   // copy upper triangle to lower
 
 // ---- state.cu: support selection and state construction --------------------------------------

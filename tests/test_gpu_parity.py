@@ -46,9 +46,9 @@ def test_gram_bf16_tensor_core(solver, name, over):
     H, G, const = solver.gram([c.cuda() for c in wl.x_chunks()], wl.weight().cuda(), wl.damp)
     Hg, Gg = H.cpu().numpy().astype(np.float64), G.cpu().numpy().astype(np.float64)
     scale = np.sqrt(np.outer(np.diag(H64), np.diag(H64)))
-    # bf16 products are exact in fp32; the tensor core adds each 16-token partial sum to its fp32
-    # accumulator with truncation, so the error grows with the number of accumulation steps per call
-    assert np.max(np.abs(Hg - H64) / scale) < 1e-6 + 6e-8 * (wl.chunk_rows / 16)
+    # bf16 products are exact in fp32; the tensor core adds each 16-token partial sum to its fp32 accumulator
+    # with truncation, so chains are cut at 2048 tokens (128 MMAs, bias <= ~2e-6) and summed in registers
+    assert np.max(np.abs(Hg - H64) / scale) < 4e-6
     assert np.array_equal(Hg, Hg.T)
     gs = np.linalg.norm(G64, axis=1, keepdims=True) + 1e-300
     assert np.max(np.abs(Gg - G64) / gs) < 1e-5
