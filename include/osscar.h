@@ -83,6 +83,23 @@ int osscar_gram(osscar_ctx* ctx, const void* X, int x_dtype, int64_t n_rows, int
                 float* H, float* G, double* const_term);
 
 /*
+ * Gram and cross term for sequential layer-wise pruning (Appendix B.1, "Pruning strategies": the layer's target is
+ * the DENSE model's output, its input the PRUNED model's activations): with X the pruned model's input block and
+ * Y = X_hat W_hat the dense model's output block (n_rows x m),
+ *     H (+)= Xc^T Xc,   G (+)= Xc^T Yc,   const (+)= ||Yc||_F^2,
+ * so that obj(S) = min_W ||Y - X W||_F^2 = const - Tr(G_I^T (H_II)^-1 G_I).  Flags and damp as in osscar_gram (damping
+ * touches H only).  X: bf16 (d1 % 8 == 0, 16-byte aligned) or fp32; Y: bf16 (m % 8 == 0) or fp32 (fp32 Y with bf16 X
+ * is split into three bf16 terms in the workspace, which must hold 6 * n_rows * round_up(m, 8) bytes and is
+ * overwritten); fp32 X requires fp32 Y.  On END *const_term is written and remembered by the context: the following
+ * init / search calls use it in place of Tr(W_hat^T G).  osscar_set_const_term sets or clears that value by hand
+ * (e.g. when H and G come from elsewhere).
+ */
+int osscar_gram_cross(osscar_ctx* ctx, const void* X, int x_dtype, const void* Y, int y_dtype,
+                      int64_t n_rows, int64_t d1, int64_t m, int flags, float damp,
+                      float* H, float* G, double* const_term);
+int osscar_set_const_term(osscar_ctx* ctx, double const_term, int enabled);
+
+/*
  * Starting support and search state (Algorithm 1, line 1, for a k-group support instead of
  * the dense start).  mode ENERGY keeps the k groups with the largest Tr(W_q^T H_qq W_q),
  * MAGNITUDE the k largest ||W_q||_F^2 (the paper's MP rule, Appendix B.1), ties to the

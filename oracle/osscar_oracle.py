@@ -64,6 +64,17 @@ def gram(X: np.ndarray, W_hat: np.ndarray, damp: float = 0.0):
     return H, G, const
 
 
+def gram_cross(X, Y, damp: float = 0.0):
+    """Sequential layer-wise objective (Appendix B.1, "Pruning strategies"): the target is the dense model's output
+    Y = X_hat W_hat, the input the pruned model's activations X, so L(W) = ||Y - X W||_F^2 and
+    H = X^T X (+ damping), G = X^T Y, const = ||Y||_F^2."""
+    X = np.asarray(X, np.float64); Y = np.asarray(Y, np.float64)
+    H = X.T @ X
+    if damp:
+        H = H + damp * np.mean(np.diag(H)) * np.eye(H.shape[0])
+    return H, X.T @ Y, float(np.sum(Y * Y))
+
+
 def gram_chunked(chunks: Iterable[np.ndarray], W_hat: np.ndarray, damp: float = 0.0):
     """Same as `gram` with X given as an iterable of row blocks."""
     H = None

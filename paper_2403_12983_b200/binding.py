@@ -22,7 +22,7 @@ STOP_NAMES = {0: "max_swaps", 1: "no_improvement", 2: "guard"}
 
 EXPORTS = ["osscar_create", "osscar_destroy", "osscar_workspace_bytes", "osscar_set_workspace",
            "osscar_gram", "osscar_init_support", "osscar_local_search", "osscar_objective",
-           "osscar_debug_get_state", "osscar_status_string", "osscar_launch_count", "osscar_trace_noalloc", "osscar_init_support_greedy"]
+           "osscar_debug_get_state", "osscar_status_string", "osscar_launch_count", "osscar_trace_noalloc", "osscar_init_support_greedy", "osscar_gram_cross", "osscar_set_const_term"]
 
 
 class SearchParams(C.Structure):
@@ -75,6 +75,8 @@ def lib() -> C.CDLL:
     L.osscar_gram.argtypes = [vp, vp, C.c_int, i64, i64, vp, i64, C.c_int, C.c_float, vp, vp, C.POINTER(C.c_double)]
     L.osscar_init_support.argtypes = [vp, vp, vp, vp, i64, i64, i32, i32, C.c_int, vp, C.POINTER(C.c_double)]
     L.osscar_init_support_greedy.argtypes = [vp, vp, vp, vp, i64, i64, i32, i32, i32, vp, vp, C.POINTER(C.c_double), C.POINTER(i32)]
+    L.osscar_gram_cross.argtypes = [vp, vp, C.c_int, vp, C.c_int, i64, i64, i64, C.c_int, C.c_float, vp, vp, C.POINTER(C.c_double)]
+    L.osscar_set_const_term.argtypes = [vp, C.c_double, C.c_int]
     L.osscar_local_search.argtypes = [vp, C.POINTER(SearchParams), vp, vp, vp, vp, C.POINTER(SearchResult)]
     L.osscar_objective.argtypes = [vp, vp, vp, vp, i64, i64, C.POINTER(C.c_double)]
     L.osscar_debug_get_state.argtypes = [vp, C.c_int, vp]
@@ -210,6 +212,32 @@ class Solver:
             flags = (GRAM_BEGIN if i == 0 else 0) | (GRAM_END if i == len(chunks) - 1 else 0)
             const = self.gram_chunk(Xc, H, flags, W, G, damp)
         return H, G, const
+
+    def gram_cross(self, x_chunks, y_chunks, damp: float = 0.0):
+        """H = X^T X, G = X^T Y, const = ||Y||_F^2 from row blocks of the pruned model's input X and the dense
+        model's output Y (CUDA tensors; X bf16 or fp32, Y bf16 or fp32)."""
+        x_chunks, y_chunks = list(x_chunks), list(y_chunks)
+        d1, m = x_chunks[0].shape[1], y_chunks[0].shape[1]
+        dev = x_chunks[0].device
+        H = torch.empty(d1, d1, dtype=torch.float32, device=dev)
+        G = torch.empty(d1, m, dtype=torch.float32, device=dev)
+        code = {torch.bfloat16: BF16, torch.float32: FP32}
+        const = C.c_double(0.0)
+        if x_chunks[0].dtype == torch.bfloat16 and y_chunks[0].dtype == torch.float32:
+            need = 6 * max(c.shape[0] for c in x_chunks) * ((m + 7) // 8 * 8) + 4096
+            if self._ws is None or self._ws.numel() < need:
+                self._ws = torch.empty(need, dtype=torch.uint8, device=dev)
+            _check(lib().osscar_set_workspace(self._h, _ptr(self._ws), self._ws.numel()), "osscar_set_workspace")
+        for i, (Xc, Yc) in enumerate(zip(x_chunks, y_chunks)):
+            if not (Xc.is_cuda and Yc.is_cuda and Xc.is_contiguous() and Yc.is_contiguous() and Xc.shape[0] == Yc.shape[0]):
+                raise ValueError("X and Y blocks must be contiguous CUDA tensors with equal row counts")
+            flags = (GRAM_BEGIN if i == 0 else 0) | (GRAM_END if i == len(x_chunks) - 1 else 0)
+            _check(lib().osscar_gram_cross(self._h, _ptr(Xc), code[Xc.dtype], _ptr(Yc), code[Yc.dtype], Xc.shape[0], d1, m,
+                                           flags, damp, _ptr(H), _ptr(G), C.byref(const)), "osscar_gram_cross")
+        return H, G, const.value
+
+    def set_const_term(self, value: float, enabled: bool = True):
+        _check(lib().osscar_set_const_term(self._h, float(value), int(enabled)), "osscar_set_const_term")
 
     def init_support(self, H, G, W, g: int, k: int, mode: int = INIT_ENERGY, support: Optional[torch.Tensor] = None):
         _dev_f32(H, "H"); _dev_f32(G, "G"); _dev_f32(W, "W")

@@ -356,7 +356,8 @@ int greedy_support(osscar_ctx* ctx, int t_hat, int32_t* support, int32_t* drop_t
     // W* = H^-1 G (Algorithm 1, line 1)
     if (L.ldm != L.m) CK(cudaMemsetAsync(p.V, 0, sizeof(float) * d1 * L.ldm, st));
     CK(sgemm(st, false, false, d1, L.m, d1, 1.f, p.A, p.lda, ctx->G, L.m, 0.f, p.V, L.ldm));
-    CK(trace_product(st, ctx->W, L.m, ctx->G, L.m, d1, L.m, ctx->partials, &ctx->ctl->acc[0]));
+    if (ctx->have_const) CK(set_device_double(st, &ctx->ctl->acc[0], ctx->user_const));
+    else CK(trace_product(st, ctx->W, L.m, ctx->G, L.m, d1, L.m, ctx->partials, &ctx->ctl->acc[0]));
     CK(trace_product(st, ctx->G, L.m, p.V, L.ldm, d1, L.m, ctx->partials, &ctx->ctl->acc[1]));
     k_set_obj0<<<1, 1, 0, st>>>(ctx->ctl);
     count_launches(1);

@@ -2,6 +2,7 @@
 #include "osscar_internal.cuh"
 #include <new>
 #include <string.h>
+#include <cuda_bf16.h>
 
 using namespace osscar;
 
@@ -41,6 +42,31 @@ __global__ void k_sub(const float* __restrict__ A, const float* __restrict__ B, 
 {
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
         C[i] = A[i] - B[i];
+}
+
+// sum of squares of a row block of Y (bf16 or fp32) in two deterministic stages, added to *acc
+__global__ void k_sumsq(const void* __restrict__ Y, int is_fp32, int64_t n, double* __restrict__ partial)
+{
+    __shared__ double red[32];
+    double acc = 0.0;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+        const double v = is_fp32 ? (double)((const float*)Y)[i] : (double)__bfloat162float(((const __nv_bfloat16*)Y)[i]);
+        acc += v * v;
+    }
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = acc;
+    __syncthreads();
+    if (threadIdx.x == 0) { double s = 0.0; for (int i = 0; i < (int)(blockDim.x >> 5); ++i) s += red[i]; partial[blockIdx.x] = s; }
+}
+__global__ void k_add_partials(const double* __restrict__ partial, int n, double* __restrict__ acc, int reset)
+{
+    __shared__ double red[32];
+    double a = 0.0;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) a += partial[i];
+    for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = a;
+    __syncthreads();
+    if (threadIdx.x == 0) { double s = 0.0; for (int i = 0; i < (int)(blockDim.x >> 5); ++i) s += red[i]; *acc = reset ? s : *acc + s; }
 }
 
 }  // namespace
@@ -153,6 +179,7 @@ int osscar_gram(osscar_ctx* ctx, const void* X, int x_dtype, int64_t n_rows, int
         ctx->gram_rows += (double)n_rows;
     }
     if (!end) { CKC(cudaGetLastError()); return OSSCAR_OK; }
+    ctx->have_const = false;
     CKC(gram_mirror(st, H, d1));
     if (damp > 0.f) {
         CKC(cudaMemsetAsync(&ctx->ctl->acc[0], 0, sizeof(double), st));
@@ -173,6 +200,73 @@ int osscar_gram(osscar_ctx* ctx, const void* X, int x_dtype, int64_t n_rows, int
     CKC(cudaStreamSynchronize(st));
     if (ctx->ctl_host->status != OSSCAR_OK) return ctx->ctl_host->status;
     *const_term = ctx->ctl_host->acc[1];
+    return OSSCAR_OK;
+}
+
+int osscar_gram_cross(osscar_ctx* ctx, const void* X, int x_dtype, const void* Y, int y_dtype,
+                      int64_t n_rows, int64_t d1, int64_t m, int flags, float damp,
+                      float* H, float* G, double* const_term)
+{
+    if (!ctx || !H || !G || (n_rows > 0 && (!X || !Y))) return OSSCAR_E_ARG;
+    if ((x_dtype != OSSCAR_BF16 && x_dtype != OSSCAR_FP32) || (y_dtype != OSSCAR_BF16 && y_dtype != OSSCAR_FP32)) return OSSCAR_E_ARG;
+    if (x_dtype == OSSCAR_FP32 && y_dtype != OSSCAR_FP32) return OSSCAR_E_ARG;
+    if (flags & ~(OSSCAR_GRAM_BEGIN | OSSCAR_GRAM_END)) return OSSCAR_E_ARG;
+    if (d1 <= 0 || m <= 0 || n_rows < 0 || !(damp >= 0.f)) return OSSCAR_E_SHAPE;
+    const bool begin = flags & OSSCAR_GRAM_BEGIN, end = flags & OSSCAR_GRAM_END;
+    if (end && !const_term) return OSSCAR_E_ARG;
+    if (x_dtype == OSSCAR_BF16 && n_rows > 0) {
+        if ((d1 % 8) != 0 || ((uintptr_t)X & 15)) return OSSCAR_E_SHAPE;
+        if (y_dtype == OSSCAR_BF16 && ((m % 8) != 0 || ((uintptr_t)Y & 15))) return OSSCAR_E_SHAPE;
+    }
+    const size_t need = y_dtype == OSSCAR_FP32 && x_dtype == OSSCAR_BF16
+                      ? 3 * (((size_t)n_rows * round_up(m, 8) * 2 + 1023) / 1024 * 1024) : 0;
+    if (need > 0 && (!ctx->ws || ctx->ws_bytes < need)) return OSSCAR_E_WORKSPACE;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return OSSCAR_E_CUDA;
+    cudaStream_t st = ctx->stream;
+    k_clear_status<<<1, 1, 0, st>>>(ctx->ctl);
+    count_launches(1);
+    if (begin && n_rows == 0) {
+        CKC(cudaMemsetAsync(H, 0, sizeof(float) * d1 * d1, st));
+        CKC(cudaMemsetAsync(G, 0, sizeof(float) * d1 * m, st));
+        CKC(cudaMemsetAsync(&ctx->ctl->acc[2], 0, sizeof(double), st));
+    }
+    if (n_rows > 0) {
+        if (x_dtype == OSSCAR_BF16) {
+            CKC(gram_tc2(st, X, n_rows, d1, nullptr, 0, 0, H, !begin, nullptr, 0, &ctx->ctl->status));
+            CKC(gram_tc2(st, X, n_rows, d1, Y, y_dtype == OSSCAR_FP32, m, G, !begin, ctx->ws, ctx->ws_bytes, &ctx->ctl->status));
+            if (need > 0) ctx->have_state = false;
+        } else {
+            CKC(sgemm(st, true, false, d1, d1, n_rows, 1.f, (const float*)X, d1, (const float*)X, d1, begin ? 0.f : 1.f, H, d1));
+            CKC(sgemm(st, true, false, d1, m, n_rows, 1.f, (const float*)X, d1, (const float*)Y, m, begin ? 0.f : 1.f, G, m));
+        }
+        const int nblk = kTracePartials;
+        k_sumsq<<<nblk, 256, 0, st>>>(Y, y_dtype == OSSCAR_FP32, n_rows * m, ctx->partials);
+        k_add_partials<<<1, 256, 0, st>>>(ctx->partials, nblk, &ctx->ctl->acc[2], begin ? 1 : 0);
+        count_launches(2);
+    }
+    if (!end) { CKC(cudaGetLastError()); return OSSCAR_OK; }
+    CKC(gram_mirror(st, H, d1));
+    if (damp > 0.f) {
+        CKC(cudaMemsetAsync(&ctx->ctl->acc[0], 0, sizeof(double), st));
+        k_diag_sum<<<64, 256, 0, st>>>(H, d1, &ctx->ctl->acc[0]);
+        k_add_damp<<<64, 256, 0, st>>>(H, d1, damp, &ctx->ctl->acc[0]);
+        count_launches(2);
+    }
+    CKC(cudaMemcpyAsync(ctx->ctl_host, ctx->ctl, sizeof(SearchCtl), cudaMemcpyDeviceToHost, st));
+    CKC(cudaStreamSynchronize(st));
+    if (ctx->ctl_host->status != OSSCAR_OK) return ctx->ctl_host->status;
+    *const_term = ctx->ctl_host->acc[2];
+    ctx->have_const = true;
+    ctx->user_const = *const_term;
+    return OSSCAR_OK;
+}
+
+int osscar_set_const_term(osscar_ctx* ctx, double const_term, int enabled)
+{
+    if (!ctx) return OSSCAR_E_ARG;
+    ctx->have_const = enabled != 0;
+    ctx->user_const = const_term;
     return OSSCAR_OK;
 }
 

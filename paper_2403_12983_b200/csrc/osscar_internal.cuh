@@ -74,6 +74,8 @@ struct osscar_ctx {
     const float* W;
     cudaEvent_t ev0, ev1;
     double gram_rows;                // rows accumulated since GRAM_BEGIN (bookkeeping only)
+    bool have_const;                 // const term supplied by the caller (cross-term problems) instead of Tr(W^T G)
+    double user_const;
 };
 
 namespace osscar {
@@ -97,6 +99,7 @@ cudaError_t gram_tc2(cudaStream_t st, const void* X, int64_t n_rows, int64_t d1,
                      float* C, bool accumulate, void* scratch, size_t scratch_bytes, int32_t* status_dev);
 
 // ---- gram_tc.cu ---------------------------------------------------------------------------------------------
+cudaError_t set_device_double(cudaStream_t st, double* dst, double v);          // *dst = v on the stream
 cudaError_t gram_mirror(cudaStream_t st, float* H, int64_t d1);   // copy upper triangle to lower
 
 // ---- state.cu: support selection and state construction --------------------------------------

@@ -264,6 +264,13 @@ __global__ void k_set_obj(SearchCtl* ctl)   // obj = const - Tr(G_I^T V), with a
 
 }  // namespace
 
+__global__ void k_set_double(double* dst, double v) { *dst = v; }
+cudaError_t set_device_double(cudaStream_t st, double* dst, double v)
+{
+    k_set_double<<<1, 1, 0, st>>>(dst, v);
+    count_launches(1);
+    return cudaGetLastError();
+}
 cudaError_t gather_rows(cudaStream_t st, const float* src, int64_t m, int g, const int32_t* perm,
                         int64_t slot_row0, int64_t nrows, float* dst, int64_t ld)
 {
@@ -439,7 +446,8 @@ int build_state(osscar_ctx* ctx, bool guarded)
     // fp32 pipes, whose rounding is unbiased; the tensor core's truncating accumulation cost 0.2 % of obj here
     CK(sgemm(st, false, false, nI, L.m, nI, 1.f, Hinv, L.ldh, big, L.ldm, 0.f, V, L.ldm, done));
     // obj = Tr(W^T G) - Tr(G_I^T V)
-    CK(trace_product(st, ctx->W, L.m, ctx->G, L.m, L.d1, L.m, ctx->partials, &ctx->ctl->acc[0]));
+    if (ctx->have_const) CK(set_device_double(st, &ctx->ctl->acc[0], ctx->user_const));
+    else CK(trace_product(st, ctx->W, L.m, ctx->G, L.m, L.d1, L.m, ctx->partials, &ctx->ctl->acc[0]));
     CK(trace_product(st, big, L.ldm, V, L.ldm, nI, L.m, ctx->partials, &ctx->ctl->acc[1]));
     k_set_obj<<<1, 1, 0, st>>>(ctx->ctl);
     count_launches(2);

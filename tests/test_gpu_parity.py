@@ -364,6 +364,39 @@ def test_greedy_phase_matches_oracle(solver, name, over, t_hat):
     assert out.obj_final == pytest.approx(srch.st.obj, rel=1e-4)
 
 
+# ------------------------------------------------------------------------------------ cross term (sequential layer-wise form)
+@pytest.mark.parametrize("name,over,ydt", [
+    ("c2", dict(n=3000, d1=520, m=152, k=207, chunk_rows=1024), torch.bfloat16),
+    ("c2", dict(n=3000, d1=520, m=150, k=207, chunk_rows=1024), torch.float32),
+    ("c4", dict(n=49 * 30, d1=9 * 37, m=50, k=12, chunk_rows=49 * 10), torch.float32),
+])
+def test_cross_term_gram_and_search(solver, name, over, ydt):
+    """Pruned-model inputs X, dense-model outputs Y: H = X^T X, G = X^T Y, const = ||Y||^2, then init and search."""
+    wl = workloads.config(name, **over)
+    W = wl.weight().numpy().astype(np.float64)
+    xs = [wl.x_pruned_chunk(c) for c in range(wl.n_chunks)]
+    ys = [wl.dense_output_chunk(c, dtype=ydt) for c in range(wl.n_chunks)]
+    H64, G64, const64 = orc.gram_cross(np.concatenate([x.float().numpy() for x in xs]),
+                                       np.concatenate([y.float().numpy() for y in ys]), wl.damp)
+    H, G, const = solver.gram_cross([x.cuda() for x in xs], [y.cuda() for y in ys], wl.damp)
+    scale = np.sqrt(np.outer(np.diag(H64), np.diag(H64)))
+    assert np.max(np.abs(H.cpu().numpy() - H64) / scale) < 5e-6
+    gs = np.linalg.norm(G64, axis=1, keepdims=True) + 1e-300
+    assert np.max(np.abs(G.cpu().numpy() - G64) / gs) < 5e-6
+    assert const == pytest.approx(const64, rel=1e-9)
+    Wd = wl.weight().cuda()
+    support, obj0 = solver.init_support(H, G, Wd, wl.g, wl.k)
+    S0 = support.cpu().numpy()
+    assert obj0 == pytest.approx(orc.solve_support(H64, G64, const64, S0, wl.g)[1], rel=1e-4)
+    out = solver.local_search(40, accept_rel_tol=wl.eps_acc)
+    swaps = [tuple(int(v) for v in r) for r in out.swap_trace.cpu().numpy()]
+    srch, _ = follow_trace(H64, G64, const64, wl.g, S0, swaps, out.obj_trace.cpu().numpy(), gpu_stop=out.stop_reason,
+                           max_swaps=40, eps_acc=wl.eps_acc)
+    assert np.array_equal(out.support.cpu().numpy(), srch.result()[0])
+    assert out.obj_final == pytest.approx(srch.st.obj, rel=1e-4)
+    assert rel_fro(out.W.cpu().numpy(), srch.result()[1]) < 1e-3
+
+
 # ------------------------------------------------------------------------------------ edge cases and errors
 def test_edge_cases(solver, osscar):
     b = osscar.binding

@@ -434,3 +434,25 @@ def test_greedy_phase_on_orthogonal_columns_keeps_the_largest_energies():
     assert set(S) == set(np.argsort(-e)[:k])
     assert [q for d in dropped for q in d] == list(np.argsort(e)[:p - k])
     assert obj[-1] == pytest.approx(float(np.sum(np.sort(e)[:p - k])), rel=1e-9)
+
+
+# ----------------------------------------------------------------------------- cross term (sequential layer-wise form)
+def test_cross_term_objective_is_least_squares_against_dense_output():
+    wl = workloads.tiny(p=9, m=4, g=1, k=4, n=70, seed=21)
+    Xd = wl.x_chunk(0).numpy().astype(np.float64)
+    Xp = wl.x_pruned_chunk(0, noise=0.3).numpy().astype(np.float64)
+    W = wl.weight().numpy().astype(np.float64)
+    Y = wl.dense_output_chunk(0).numpy().astype(np.float64)
+    assert np.allclose(Y, Xd @ W, rtol=1e-6, atol=1e-6) and not np.allclose(Xp, Xd)
+    H, G, const = orc.gram_cross(Xp, Y)
+    for S in [(0, 2, 5, 8), (1, 3, 4, 6), tuple(range(9))]:
+        W_S, obj = orc.solve_support(H, G, const, S, 1)
+        V, res, *_ = np.linalg.lstsq(Xp[:, list(S)], Y, rcond=None)
+        assert obj == pytest.approx(float(np.sum((Y - Xp[:, list(S)] @ V) ** 2)), rel=1e-8)
+        assert np.allclose(W_S[list(S)], V, rtol=1e-6, atol=1e-9)
+    # the search works on (H, G, const) unchanged: every accepted swap lowers ||Y - X W||^2
+    S0, _ = orc.init_support(H, W, 1, 4)
+    run = orc.Search(H, G, const, 1, S0).run(20)
+    assert np.all(np.diff(run.obj_trace) < 0)
+    Wf = run.result()[1]
+    assert run.obj_trace[-1] == pytest.approx(float(np.sum((Y - Xp @ Wf) ** 2)), rel=1e-8)

@@ -134,6 +134,24 @@ class Workload:
             X = X * sh["scale"]
         return X.to(self.x_dtype).contiguous()
 
+    # ------------------------------------------------------------------ sequential layer-wise setting
+    def x_pruned_chunk(self, c: int, device: str = "cpu", noise: float = 0.1) -> torch.Tensor:
+        """Input block as the already-pruned upstream model would produce it: the dense block plus a seeded
+        perturbation of relative size `noise` (same dtype and sign structure)."""
+        X = self.x_chunk(c, device).float()
+        gdev = "cuda" if str(device).startswith("cuda") else "cpu"
+        gen = torch.Generator(device=gdev).manual_seed(self.seed * 1_000_003 + 104729 * (c + 1))
+        E = torch.randn(X.shape, generator=gen, dtype=torch.float32, device=device)
+        Xp = X + noise * X.abs().mean() * E
+        if self.kind in ("fc2_relu", "conv_unfold"):
+            Xp = torch.relu_(Xp)
+        return Xp.to(self.x_dtype).contiguous()
+
+    def dense_output_chunk(self, c: int, device: str = "cpu", dtype: torch.dtype = torch.float32) -> torch.Tensor:
+        """Y block = dense-model input block times the dense weight (the layer's target output)."""
+        Y = self.x_chunk(c, device).double() @ self.weight(device).double()
+        return Y.to(dtype).contiguous()
+
     def x_chunks(self, device: str = "cpu") -> Iterator[torch.Tensor]:
         for c in range(self.n_chunks):
             yield self.x_chunk(c, device)
