@@ -306,7 +306,7 @@ def run_ours(args):
         tiles = sum(tn_ - t // 2 for t in range(tm_))
         flops = 2.0 * 128 * 256 * tiles * wl.n
         ach = flops / (phase["gram"] / K * 1e-3) / 1e12
-        roof = {"kernel": "k_gram_tcgen05", "bound": "tensor", "achieved": ach, "peak": pk["bf16_tflops_sustained"],
+        roof = {"kernel": "k_mma_pipe<GRAM>", "bound": "tensor", "achieved": ach, "peak": pk["bf16_tflops_sustained"],
                 "unit": "TFLOP/s", "frac": ach / pk["bf16_tflops_sustained"], "traffic": None,
                 "flops_per_step": flops, "peak_source": pk["source"] + " (sustained)"}
     tm_, tn_ = -(-wl.d1 // 128), -(-wl.d1 // 256)
