@@ -29,6 +29,8 @@ Readings of the paper taken here (each pinned by a CPU test)
 * Selection (text after Eq. impact, with t_hat = 2, p_hat = 0 so s1 = s2 = 1):
   the kept group whose removal costs least leaves, the pruned group whose
   return gains most enters.  Ties go to the smallest group id.
+* Larger local-search steps (t_hat = 2 s, p_hat = 0, `BlockSearch`): s_1 = s_2 = s groups are exchanged per
+  iteration, all chosen from the scores at the current support; the acceptance test applies to the whole exchange.
 * The paper has no acceptance test; `accept="improving"` (stop at the first swap
   that does not lower obj by more than eps_acc * obj) and damping of H are
   choices of this build: parity unpinned by the paper.
@@ -428,6 +430,86 @@ class Search:
         W = np.zeros_like(self.G)
         W[rows_of(self.st.S, self.g)] = self.st.V
         return np.sort(self.st.S), W, np.array(self.obj_trace), list(self.swap_trace)
+
+
+@dataclass
+class BlockStepInfo:
+    slots: List[int]          # slots of the leaving groups, cheapest first
+    out: List[int]            # leaving group ids (same order)
+    inn: List[int]            # entering group ids, most valuable first; inn[t] takes slots[t]
+    delta: float              # exact change of obj for the whole exchange (fresh evaluation)
+    obj_before: float
+    accepted: bool
+    D: np.ndarray             # drop scores by slot
+    A: np.ndarray             # add scores by group id (-inf for kept / ineligible groups)
+
+
+class BlockSearch:
+    """Local-search iterations of Algorithm 1 with p_hat = 0 and t_hat = 2 s (Eq. local, Eq. impact): the s kept
+    groups with the lowest impact leave and the s pruned groups with the highest impact enter, all scored at the
+    current support (s_1 = s_2 = s).  The exchange is kept iff it lowers obj by more than eps_acc * obj (or always).
+    s = 1 is `Search` with independent scores.  Everything is recomputed from H, G at each iteration."""
+
+    def __init__(self, H, G, const, g, S0, s, accept="improving", eps_acc=EPS_ACC):
+        self.H = np.asarray(H, np.float64)
+        self.G = np.asarray(G, np.float64)
+        self.const = float(const)
+        self.g, self.s = int(g), int(s)
+        self.ngroups = self.H.shape[0] // self.g
+        self.accept, self.eps_acc = accept, eps_acc
+        S0 = np.asarray(S0, np.int64)
+        if not (1 <= self.s <= min(len(S0), self.ngroups - len(S0))):
+            raise ValueError("block size must be between 1 and min(k, ngroups - k)")
+        self.st = fresh_state(self.H, self.G, self.const, S0, self.g)
+        self.obj_trace = [self.st.obj]
+        self.block_trace: List[Tuple[Tuple[int, ...], Tuple[int, ...]]] = []
+        self.stop_reason: Optional[str] = None
+
+    def exchange_delta(self, slots, inn) -> float:
+        S_new = self.st.S.copy()
+        S_new[np.asarray(slots)] = np.asarray(inn)
+        return solve_support(self.H, self.G, self.const, S_new, self.g)[1] - \
+            solve_support(self.H, self.G, self.const, self.st.S, self.g)[1]
+
+    def propose(self) -> Optional[BlockStepInfo]:
+        st = self.st
+        D = drop_scores(st, self.g)
+        A = add_scores(st, self.g, self.ngroups, self.H)
+        slots = np.lexsort((st.S, D))[: self.s]
+        inn = np.lexsort((np.arange(self.ngroups), -A))[: self.s]
+        if not (np.all(np.isfinite(D[slots])) and np.all(np.isfinite(A[inn]))):
+            return None
+        delta = self.exchange_delta(slots, inn)
+        accepted = True if self.accept == "always" else bool(delta <= -self.eps_acc * st.obj)
+        return BlockStepInfo([int(v) for v in slots], [int(st.S[v]) for v in slots], [int(v) for v in inn],
+                             float(delta), st.obj, accepted, D, A)
+
+    def apply(self, slots, inn):
+        out = tuple(int(self.st.S[v]) for v in slots)
+        S_new = self.st.S.copy()
+        S_new[np.asarray(slots)] = np.asarray(inn)
+        self.st = fresh_state(self.H, self.G, self.const, S_new, self.g)
+        self.obj_trace.append(self.st.obj)
+        self.block_trace.append((out, tuple(int(v) for v in inn)))
+
+    def run(self, max_iters: int):
+        while len(self.block_trace) < max_iters:
+            info = self.propose()
+            if info is None:
+                self.stop_reason = "guard"
+                break
+            if not info.accepted:
+                self.stop_reason = "no_improvement"
+                break
+            self.apply(info.slots, info.inn)
+        else:
+            self.stop_reason = "max_swaps"
+        return self
+
+    def result(self):
+        W = np.zeros_like(self.G)
+        W[rows_of(self.st.S, self.g)] = self.st.V
+        return np.sort(self.st.S), W, np.array(self.obj_trace), list(self.block_trace)
 
 
 def lowrank_swap(H, st: State, g: int, slot: int, q: int) -> State:

@@ -456,3 +456,78 @@ def test_cross_term_objective_is_least_squares_against_dense_output():
     assert np.all(np.diff(run.obj_trace) < 0)
     Wf = run.result()[1]
     assert run.obj_trace[-1] == pytest.approx(float(np.sum((Y - Xp @ Wf) ** 2)), rel=1e-8)
+
+
+# ----------------------------------------------------------------------------- block exchanges (t_hat = 2 s, p_hat = 0)
+def _tiny_problem(p=14, m=4, g=1, k=6, n=90, seed=5):
+    wl = workloads.tiny(p=p, m=m, g=g, k=k, n=n, seed=seed)
+    X = wl.x_chunk(0).numpy().astype(np.float64)
+    W = wl.weight().numpy().astype(np.float64)
+    H, G, const = orc.gram(X, W)
+    return X, W, H, G, const
+
+
+def test_block_search_with_one_pair_is_the_swap_search():
+    X, W, H, G, const = _tiny_problem()
+    S0, _ = orc.init_support(H, W, 1, 6)
+    a = orc.Search(H, G, const, 1, S0, mode="strict").run(20)
+    b = orc.BlockSearch(H, G, const, 1, S0, 1).run(20)
+    assert [(o[0], i[0]) for o, i in b.block_trace] == a.swap_trace and len(a.swap_trace) > 0
+    assert np.allclose(a.obj_trace, b.obj_trace, rtol=1e-12)
+    assert a.stop_reason == b.stop_reason
+
+
+@pytest.mark.parametrize("g,s", [(1, 2), (1, 3), (2, 2)])
+def test_block_exchange_takes_the_s_lowest_and_highest_impacts_from_definitions(g, s):
+    """Eq. impact by brute force: B_j from re-solved supports; the exchange is the s extremes on each side and its
+    change of obj is the re-solved difference measured on X."""
+    X, W, H, G, const = _tiny_problem(p=10, m=3, g=g, k=5, n=80, seed=8)
+    S0, _ = orc.init_support(H, W, g, 5)
+    srch = orc.BlockSearch(H, G, const, g, S0, s, accept="always")
+    for _ in range(3):
+        S = [int(v) for v in srch.st.S]
+        obj = orc.solve_support_lstsq(X, W, S, g)[1]
+        drop = {i: orc.solve_support_lstsq(X, W, [j for j in S if j != i], g)[1] - obj for i in S}
+        add = {q: obj - orc.solve_support_lstsq(X, W, S + [q], g)[1] for q in range(10) if q not in S}
+        want_out = sorted(drop, key=lambda i: (drop[i], i))[:s]
+        want_in = sorted(add, key=lambda q: (-add[q], q))[:s]
+        info = srch.propose()
+        assert info.out == want_out and info.inn == want_in
+        S_new = sorted(set(S) - set(want_out) | set(want_in))
+        assert info.delta == pytest.approx(orc.solve_support_lstsq(X, W, S_new, g)[1] - obj, rel=1e-7, abs=1e-9)
+        srch.apply(info.slots, info.inn)
+        assert sorted(int(v) for v in srch.st.S) == S_new
+        assert srch.st.obj == pytest.approx(orc.solve_support_lstsq(X, W, S_new, g)[1], rel=1e-8)
+
+
+def test_block_exchange_on_orthogonal_columns_adds_up():
+    """H diagonal: impacts do not interact, so the exchange changes obj by sum(D_out) - sum(A_in) and the search
+    reaches the top-k energies in one iteration when s covers every misplaced group."""
+    rng = np.random.default_rng(3)
+    h = rng.uniform(0.5, 2.0, 12)
+    W = rng.normal(size=(12, 3))
+    H = np.diag(h); G = H @ W; const = float(np.sum(W * G))
+    e = h * np.sum(W * W, axis=1)
+    best = np.argsort(-e)[:6]
+    S0 = np.sort(np.concatenate([best[:3], np.argsort(-e)[9:]]))       # three right, three wrong
+    srch = orc.BlockSearch(H, G, const, 1, S0, 3)
+    info = srch.propose()
+    assert sorted(info.out) == sorted(int(v) for v in np.argsort(-e)[9:])
+    assert sorted(info.inn) == sorted(int(v) for v in best[3:])
+    assert info.delta == pytest.approx(np.sum(e[info.out]) - np.sum(e[info.inn]), rel=1e-10)
+    srch.run(5)
+    assert sorted(int(v) for v in srch.st.S) == sorted(int(v) for v in best)
+    assert srch.stop_reason == "no_improvement" and len(srch.block_trace) == 1
+
+
+def test_block_search_stops_when_the_exchange_does_not_improve_and_rejects_bad_sizes():
+    X, W, H, G, const = _tiny_problem(p=12, m=4, g=1, k=6, n=100, seed=11)
+    S0, _ = orc.init_support(H, W, 1, 6)
+    run = orc.BlockSearch(H, G, const, 1, S0, 2).run(50)
+    assert run.stop_reason == "no_improvement" and np.all(np.diff(run.obj_trace) < 0)
+    info = run.propose()
+    assert info.delta > -run.eps_acc * run.st.obj
+    with pytest.raises(ValueError):
+        orc.BlockSearch(H, G, const, 1, S0, 7)
+    with pytest.raises(ValueError):
+        orc.BlockSearch(H, G, const, 1, S0, 0)
