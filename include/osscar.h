@@ -137,7 +137,7 @@ typedef struct {
     int32_t refresh_every;    /* rebuild the state from H every this many swaps; 0 = never   */
     double  accept_rel_tol;   /* IMPROVING: accept iff delta <= -tol * obj (1e-5 if < 0)     */
     int32_t profile_samples;  /* time each kernel of this many evenly spaced steps (0..8)    */
-    int32_t reserved;         /* must be 0                                                   */
+    int32_t block_pairs;      /* s: groups exchanged per iteration (0 or 1: one swap per step) */
 } osscar_search_params;
 
 #define OSSCAR_NUM_STEP_KERNELS 12   /* select, pair Grams, y pass, small algebra, staging, H pass,
@@ -163,6 +163,13 @@ typedef struct {
  * zero.  obj_trace: device double[max_swaps+1], entry 0 = starting obj.  swap_trace: device
  * int32[2*max_swaps], (group out, group in) per accepted swap.  result: host.
  * Synchronises once at the end.
+ * block_pairs = s > 1 (Eq. local with t_hat = 2 s, p_hat = 0, so s_1 = s_2 = s in the rule after Eq. impact;
+ * Appendix B.1 uses t_hat up to 100 for FC neurons): each iteration takes the s cheapest drops and the s most
+ * valuable adds, all from the scores at the current support, and moves the state with one rank-(2 s g) update;
+ * the accept rule applies to the exact change of the whole exchange.  INDEPENDENT scores only; needs
+ * s <= min(k, d1/g - k) and s * g <= OSSCAR_MAX_GROUP (else OSSCAR_E_ARG).  floor(max_swaps / s) iterations at
+ * most; n_swaps counts groups (s per iteration), swap_trace lists the s pairs of an iteration in order
+ * (cheapest drop with best add first) and obj_trace has one entry per ITERATION after entry 0.
  */
 int osscar_local_search(osscar_ctx* ctx, const osscar_search_params* params,
                         int32_t* support_out, float* W_out,

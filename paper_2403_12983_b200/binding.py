@@ -27,7 +27,7 @@ EXPORTS = ["osscar_create", "osscar_destroy", "osscar_workspace_bytes", "osscar_
 
 class SearchParams(C.Structure):
     _fields_ = [("max_swaps", C.c_int32), ("score_mode", C.c_int32), ("accept_mode", C.c_int32),
-                ("refresh_every", C.c_int32), ("accept_rel_tol", C.c_double), ("profile_samples", C.c_int32), ("reserved", C.c_int32)]
+                ("refresh_every", C.c_int32), ("accept_rel_tol", C.c_double), ("profile_samples", C.c_int32), ("block_pairs", C.c_int32)]
 
 
 class SearchResult(C.Structure):
@@ -40,6 +40,9 @@ STEP_KERNELS = ["select", "pair_grams", "y_pass", "small_algebra", "staging", "h
                 "update_r", "group_scores", "h_swap_rows", "h_swap_cols"]
 # single-row groups run a fused five-launch step
 STEP_KERNELS_G1 = ["decide", "l1_hpass_update_v", "l2_update_r_swap", "select_in", "l4_update_hinv_y"]
+# block exchanges (block_pairs > 1): stages of one iteration
+STEP_KERNELS_BLOCK = ["select", "gather_y", "grams_algebra_staging", "h_pass", "update_hinv", "update_v", "update_r",
+                      "update_c_fix", "h_swap", "scores"]
 
 
 class OsscarError(RuntimeError):
@@ -270,22 +273,24 @@ class Solver:
         return support, drops[:d1 // g - k], obj0.value, iters.value
 
     def local_search(self, max_swaps: int, score_mode: int = SCORE_INDEPENDENT, accept_mode: int = ACCEPT_IMPROVING,
-                     refresh_every: int = 0, accept_rel_tol: float = -1.0, profile_samples: int = 0) -> SearchOutput:
+                     refresh_every: int = 0, accept_rel_tol: float = -1.0, profile_samples: int = 0,
+                     block_pairs: int = 0) -> SearchOutput:
         d1, m, g, k = self._shape
         dev = self._keep[0].device
         support = torch.empty(k, dtype=torch.int32, device=dev)
         W_out = torch.empty(d1, m, dtype=torch.float32, device=dev)
         obj_trace = torch.zeros(max_swaps + 1, dtype=torch.float64, device=dev)
         swap_trace = torch.zeros(max(1, 2 * max_swaps), dtype=torch.int32, device=dev)
-        prm = SearchParams(max_swaps, score_mode, accept_mode, refresh_every, accept_rel_tol, profile_samples, 0)
+        prm = SearchParams(max_swaps, score_mode, accept_mode, refresh_every, accept_rel_tol, profile_samples, block_pairs)
         res = SearchResult()
         _check(lib().osscar_local_search(self._h, C.byref(prm), _ptr(support), _ptr(W_out), _ptr(obj_trace), _ptr(swap_trace),
                                          C.byref(res)), "osscar_local_search")
         n = res.n_swaps
-        return SearchOutput(support, W_out, obj_trace[:n + 1], swap_trace[:2 * n].view(n, 2), n,
+        n_obj = n // block_pairs if block_pairs > 1 else n      # one objective per iteration
+        return SearchOutput(support, W_out, obj_trace[:n_obj + 1], swap_trace[:2 * n].view(n, 2), n,
                             STOP_NAMES.get(res.stop_reason, str(res.stop_reason)), res.n_refresh,
                             res.obj_init, res.obj_final, res.ms_search,
-                            {n: res.ms_kernel[i] for i, n in enumerate(STEP_KERNELS_G1 if g == 1 else STEP_KERNELS)}
+                            {n: res.ms_kernel[i] for i, n in enumerate(STEP_KERNELS_BLOCK if block_pairs > 1 else STEP_KERNELS_G1 if g == 1 else STEP_KERNELS)}
                             if res.n_profiled > 0 else {})
 
     def objective(self, H, W, Wt) -> float:

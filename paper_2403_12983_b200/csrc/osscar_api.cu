@@ -334,9 +334,14 @@ int osscar_local_search(osscar_ctx* ctx, const osscar_search_params* params,
     if (params->max_swaps < 0 || (params->max_swaps > 0 && !swap_trace)) return OSSCAR_E_ARG;
     if (params->score_mode != OSSCAR_SCORE_INDEPENDENT && params->score_mode != OSSCAR_SCORE_PAIR_EXACT) return OSSCAR_E_ARG;
     if (params->accept_mode != OSSCAR_ACCEPT_IMPROVING && params->accept_mode != OSSCAR_ACCEPT_ALWAYS) return OSSCAR_E_ARG;
-    if (params->refresh_every < 0 || params->profile_samples < 0 || params->profile_samples > 8 || params->reserved != 0) return OSSCAR_E_ARG;
+    if (params->refresh_every < 0 || params->profile_samples < 0 || params->profile_samples > 8 || params->block_pairs < 0) return OSSCAR_E_ARG;
     if (!ctx->have_state) return OSSCAR_E_STATE;
     if (params->score_mode == OSSCAR_SCORE_PAIR_EXACT && ctx->L.nJ > 0 && ctx->L.pair_capacity == 0) return OSSCAR_E_SHAPE;
+    if (params->block_pairs > 1) {      // block exchanges: independent scores, s <= min(k, pruned groups), s g rows fit the panels
+        const osscar::Layout& L = ctx->L;
+        const int64_t s = params->block_pairs;
+        if (params->score_mode != OSSCAR_SCORE_INDEPENDENT || s * L.g > L.block_rows_max || s > L.k || s > L.ng - L.k) return OSSCAR_E_ARG;
+    }
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return OSSCAR_E_CUDA;
     memset(result, 0, sizeof(*result));

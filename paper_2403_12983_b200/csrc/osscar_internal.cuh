@@ -50,6 +50,8 @@ struct Layout {
     size_t off_pairCinv, off_pairKK, off_pairScratch, off_pairDelta;   // PAIR_EXACT scoring
     size_t off_greedy;                                                 // scratch of the nested (greedy) phase
     size_t off_tc, tc_bytes;                                           // bf16 operand terms of the tensor-core GEMMs
+    size_t off_block, block_bytes;                                     // panels of the block exchange (search_block.cuh)
+    int32_t block_rows_max;                                            // largest s*g the block region holds
     int64_t pair_capacity;                                             // pairs the workspace can score
     size_t bytes;
 };

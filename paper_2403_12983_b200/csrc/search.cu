@@ -752,6 +752,8 @@ cudaError_t enqueue_scores(osscar_ctx* ctx, const Ptrs& p, bool norms, bool gene
     return cudaGetLastError();
 }
 
+#include "search_block.cuh"
+
 }  // namespace
 
 cudaError_t score_pass(osscar_ctx* ctx)
@@ -772,14 +774,22 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
     Ptrs p = make_ptrs(ctx);
     const int g = L.g;
     const double tol = prm->accept_rel_tol < 0 ? 1e-5 : prm->accept_rel_tol;
-    const int max_swaps = (L.nJ > 0) ? prm->max_swaps : 0;
+    int max_swaps = (L.nJ > 0) ? prm->max_swaps : 0;
 
     k_begin<<<1, 1, 0, st>>>(ctx->ctl, obj_trace, ctx->done_flag_dev);
     count_launches(1);
     CK(cudaGetLastError());
     CK(cudaEventRecord(ctx->ev0, st));
     const bool pair = prm->score_mode == OSSCAR_SCORE_PAIR_EXACT;
-    const bool fast = g == 1 && !pair;            // fused five-launch step for single-row groups
+    const int bs = prm->block_pairs > 1 ? prm->block_pairs : 1;     // groups exchanged per iteration
+    const bool block = bs > 1;
+    if (block) {
+        if (pair || (int64_t)bs * g > L.block_rows_max || bs > L.k || bs > L.ng - L.k) return OSSCAR_E_ARG;
+        if (block_region_bytes(L, bs * g) > L.block_bytes) return OSSCAR_E_WORKSPACE;
+    }
+    BlockPtrs bp = make_block_ptrs(ctx, bs);
+    const bool fast = g == 1 && !pair && !block;  // fused five-launch step for single-row groups
+    if (block) max_swaps /= bs;                   // from here on: iterations
     const int64_t npairs = (int64_t)L.k * (L.ng - L.k);
     if (max_swaps > 0) CK(enqueue_scores(ctx, p, true, pair));
     auto pair_scores = [&]() -> cudaError_t {      // PAIR_EXACT: exact change of obj of every (kept, pruned) pair
@@ -809,6 +819,11 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
     };
     if (max_swaps > 0 && fast) CK(bootstrap_g1());
 
+    if (block) {
+        CK(cudaMemsetAsync((char*)ctx->ws + L.off_block, 0, block_region_bytes(L, bs * g), st));
+        const size_t smem = 2 * (size_t)g * bs * g * sizeof(double);
+        if (smem > 48 * 1024) CK(cudaFuncSetAttribute(k_blk_update_c, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    }
     if (g > 1) CK(cudaFuncSetAttribute(k_update_c, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(2 * (size_t)g * g * sizeof(double))));
     const int batch = 32;
     cudaEvent_t evb[2];
@@ -851,7 +866,9 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
         int slot = 0;
         auto mark = [&]() { if (pe) cudaEventRecord(pe[slot], st); ++slot; };
         mark();
-        if (fast) {
+        if (block) {
+            if (enqueue_block_step(ctx, p, bp, prm->accept_mode, tol, obj_trace, swap_trace, mark) != cudaSuccess) { rc = OSSCAR_E_CUDA; break; }
+        } else if (fast) {
             // single-row groups: decide, {H pass || V}, {R || slot exchange}, next entering group, {Hinv + next y}
             const unsigned nbV = (unsigned)L.nI, nbH = (unsigned)(L.nJ + 1), nbR = (unsigned)L.nJ;   // one row per block
             k_decide_g1<<<1, 1024, 0, st>>>(p, prm->accept_mode, tol, obj_trace, swap_trace);   mark();
@@ -928,7 +945,7 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
     // kernel times of the sampled steps that really swapped (a stopped loop runs empty kernels)
     int used = 0;
     for (int i = 0; i < nprof; ++i) {
-        if (i < next_prof && prof_it[i] < res->n_swaps) {
+        if (i < next_prof && prof_it[i] < res->n_swaps / bs) {
             for (int j = 0; j + 1 < nmarks && j < NK; ++j) {
                 float t = 0.f;
                 if (cudaEventElapsedTime(&t, evp[i][j], evp[i][j + 1]) == cudaSuccess) res->ms_kernel[j] += t;

@@ -1,0 +1,444 @@
+// Block exchanges: local-search iterations of Algorithm 1 with p_hat = 0 and t_hat = 2 s (Eq. local, Eq. impact).
+// The s kept groups with the lowest drop score leave and the s pruned groups with the highest add score enter in ONE
+// rank-2G update (G = s g rows on each side), so every matrix of the state is streamed once per s swaps.
+// Included by search.cu (same translation unit: uses its Ptrs, small-matrix slots and reductions).
+//
+// The algebra is that of a single swap (header of search.cu) with r = the G leaving rows and q = the G entering
+// rows, given by index lists instead of one contiguous group; the joint Schur complement of the entering rows,
+// c_qq = H_qq - H_qI Hinv H_Iq, is formed from y because the state only carries its diagonal blocks.
+// Panels (row-major, one staged vector per row):
+//   hT, yT (G x ldh)   h = Hp[q, 0:n_I],  y = Hinv h
+//   PB (2G x ldh)      [ b ; u2 ]          b = rows r of Hinv
+//   PA (2G x ldh)      [ b C^-1 ; -u2 c1^-1 ]
+//   KV (2G x ldm)      [ K ; Vq ]
+//   UD ((n_J+G) x 2G)  [ u | -d ] for the pruned rows, then the leaving rows
+//   Hinv' = Hinv - PA^T PB,   V' = V - PB^T KV,   R' = R + UD KV      (three GEMMs with inner dimension 2G)
+#pragma once
+
+struct BlockPtrs {
+    int32_t *rslot, *tslot;        // kept slots that leave (cheapest first), pruned slots that enter (best first)
+    float *hT, *yT, *HrT, *PB, *PA, *KV, *Vr, *Rq, *UD;
+    double* small;                 // kBlockSmall matrices of G x G doubles
+    int s, G;
+};
+constexpr int kBlockSmall = 18;
+enum { B_CQ = 16, B_HY = 17 };     // joint Schur complement of the entering rows, h^T y
+
+size_t block_region_bytes(const Layout& L, int G)
+{
+    auto al = [](size_t b) { return (b + 255) / 256 * 256; };
+    size_t n = 2 * al(sizeof(int32_t) * (size_t)G);
+    n += 3 * al(sizeof(float) * (size_t)G * L.ldh);          // hT, yT, HrT
+    n += 2 * al(sizeof(float) * 2 * (size_t)G * L.ldh);      // PB, PA
+    n += al(sizeof(float) * 2 * (size_t)G * L.ldm);          // KV
+    n += 2 * al(sizeof(float) * (size_t)G * L.ldm);          // Vr, Rq
+    n += al(sizeof(float) * (size_t)(L.nJ + G) * 2 * G);     // UD
+    n += al(sizeof(double) * kBlockSmall * (size_t)G * G);
+    return n;
+}
+
+BlockPtrs make_block_ptrs(osscar_ctx* ctx, int s)
+{
+    const Layout& L = ctx->L;
+    const int G = s * L.g;
+    char* base = (char*)ctx->ws + L.off_block;
+    size_t off = 0;
+    auto take = [&](size_t b) { char* q = base + off; off += (b + 255) / 256 * 256; return q; };
+    BlockPtrs bp;
+    bp.s = s; bp.G = G;
+    bp.rslot = (int32_t*)take(sizeof(int32_t) * (size_t)G);
+    bp.tslot = (int32_t*)take(sizeof(int32_t) * (size_t)G);
+    bp.hT = (float*)take(sizeof(float) * (size_t)G * L.ldh);
+    bp.yT = (float*)take(sizeof(float) * (size_t)G * L.ldh);
+    bp.HrT = (float*)take(sizeof(float) * (size_t)G * L.ldh);
+    bp.PB = (float*)take(sizeof(float) * 2 * (size_t)G * L.ldh);
+    bp.PA = (float*)take(sizeof(float) * 2 * (size_t)G * L.ldh);
+    bp.KV = (float*)take(sizeof(float) * 2 * (size_t)G * L.ldm);
+    bp.Vr = (float*)take(sizeof(float) * (size_t)G * L.ldm);
+    bp.Rq = (float*)take(sizeof(float) * (size_t)G * L.ldm);
+    bp.UD = (float*)take(sizeof(float) * (size_t)(L.nJ + G) * 2 * G);
+    bp.small = (double*)take(sizeof(double) * kBlockSmall * (size_t)G * G);
+    return bp;
+}
+
+// row of the e-th leaving row among the kept slots / of the e-th entering row among the pruned slots
+__device__ __forceinline__ int64_t blk_rrow(const Ptrs& p, const BlockPtrs& bp, int e) { return (int64_t)bp.rslot[e / p.g] * p.g + e % p.g; }
+__device__ __forceinline__ int64_t blk_qrow(const Ptrs& p, const BlockPtrs& bp, int e) { return (int64_t)bp.tslot[e / p.g] * p.g + e % p.g; }
+
+// Arg-min over val[0..n) (negate: arg-max), ties to the smaller id; the array is rewritten between calls, so it is
+// read through a plain pointer.  Result in every thread.
+__device__ void blk_argmin(double* val, const int32_t* ids, int n, bool negate, double* best_out, int* idx_out)
+{
+    __shared__ double sv[32]; __shared__ int sid[32]; __shared__ int sidx[32];
+    const int t = threadIdx.x, lane = t & 31, w = t >> 5;
+    double best = INFINITY; int bid = INT_MAX, bidx = -1;
+    for (int i = t; i < n; i += blockDim.x) {
+        const double v = negate ? -val[i] : val[i];
+        const int id = ids[i];
+        if (v < best || (v == best && id < bid)) { best = v; bid = id; bidx = i; }
+    }
+    for (int o = 16; o > 0; o >>= 1) {
+        const double ov = __shfl_xor_sync(0xffffffffu, best, o);
+        const int oid = __shfl_xor_sync(0xffffffffu, bid, o);
+        const int oidx = __shfl_xor_sync(0xffffffffu, bidx, o);
+        if (ov < best || (ov == best && oid < bid)) { best = ov; bid = oid; bidx = oidx; }
+    }
+    __syncthreads();
+    if (lane == 0) { sv[w] = best; sid[w] = bid; sidx[w] = bidx; }
+    __syncthreads();
+    if (t == 0) {
+        for (int i = 1; i < (int)(blockDim.x >> 5); ++i)
+            if (sv[i] < best || (sv[i] == best && sid[i] < bid)) { best = sv[i]; bid = sid[i]; bidx = sidx[i]; }
+        sv[0] = best; sidx[0] = bidx;
+    }
+    __syncthreads();
+    *best_out = negate ? -sv[0] : sv[0];
+    *idx_out = sidx[0];
+    __syncthreads();
+}
+
+// The s cheapest kept slots and the s most valuable pruned slots (scores at the current support; ties -> smaller id).
+// Chosen entries of D and A are overwritten with +-inf while the lists are drawn.
+__global__ void __launch_bounds__(1024) k_blk_select(Ptrs p, BlockPtrs bp)
+{
+    SearchCtl* ctl = p.ctl;
+    if (ctl->done) return;
+    const int npr = (int)(p.ng - p.k);
+    if (p.g == 1) {
+        for (int i = threadIdx.x; i < p.k; i += blockDim.x) {
+            const double hd = p.Hinv[(int64_t)i * p.ldh + i];
+            p.D[i] = hd > 0.0 ? (double)p.vnorm[i] / hd : INFINITY;
+        }
+        for (int i = threadIdx.x; i < npr; i += blockDim.x) {
+            const double cc = p.c[i];
+            const double hd = p.Hp[(p.nI + i) * p.ldp + p.nI + i];
+            p.A[i] = cc > kAddPivotTol * hd ? (double)p.rnorm[i] / cc : -INFINITY;
+        }
+        __syncthreads();
+    }
+    bool ok = true;
+    for (int t = 0; t < bp.s; ++t) {
+        double best; int idx;
+        blk_argmin(p.D, p.perm, p.k, false, &best, &idx);
+        if (idx < 0 || !isfinite(best)) { ok = false; break; }
+        if (threadIdx.x == 0) { bp.rslot[t] = idx; p.D[idx] = INFINITY; }
+        __syncthreads();
+    }
+    for (int t = 0; ok && t < bp.s; ++t) {
+        double best; int idx;
+        blk_argmin(p.A, p.perm + p.k, npr, true, &best, &idx);
+        if (idx < 0 || !isfinite(best)) { ok = false; break; }
+        if (threadIdx.x == 0) { bp.tslot[t] = idx; p.A[idx] = -INFINITY; }
+        __syncthreads();
+    }
+    if (!ok && threadIdx.x == 0) { ctl->done = 1; ctl->stop_reason = OSSCAR_STOP_GUARD; *p.done_host = 1; }
+}
+
+// Rows of the exchange copied into the panels: hT, HrT (rows of Hp), b (rows of Hinv), V_r, R_q.  grid (G, 5).
+__global__ void __launch_bounds__(256) k_blk_gather(Ptrs p, BlockPtrs bp)
+{
+    if (p.ctl->done) return;
+    const int e = blockIdx.x, which = blockIdx.y;
+    const int64_t rrow = blk_rrow(p, bp, e), qrow = blk_qrow(p, bp, e);
+    const float* src; float* dst; int64_t n, valid;
+    switch (which) {
+    case 0:  src = p.Hp + (p.nI + qrow) * p.ldp; dst = bp.hT + (int64_t)e * p.ldh;  n = p.ldh; valid = p.nI; break;
+    case 1:  src = p.Hp + rrow * p.ldp;          dst = bp.HrT + (int64_t)e * p.ldh; n = p.ldh; valid = p.nI; break;
+    case 2:  src = p.Hinv + rrow * p.ldh;        dst = bp.PB + (int64_t)e * p.ldh;  n = p.ldh; valid = p.nI; break;
+    case 3:  src = p.V + rrow * p.ldm;           dst = bp.Vr + (int64_t)e * p.ldm;  n = p.ldm; valid = p.m; break;
+    default: src = p.R + qrow * p.ldm;           dst = bp.Rq + (int64_t)e * p.ldm;  n = p.ldm; valid = p.m; break;
+    }
+    for (int64_t x = threadIdx.x; x < n; x += blockDim.x) dst[x] = x < valid ? src[x] : 0.f;
+}
+
+// G x G Grams of the panels, one warp per entry: GV = V_r V_r^T, GX = V_r R_q^T, GR = R_q R_q^T, HY = h^T y.
+__global__ void __launch_bounds__(256) k_blk_gram(Ptrs p, BlockPtrs bp)
+{
+    if (p.ctl->done) return;
+    const int G = bp.G;
+    const int64_t wid = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (wid >= 4LL * G * G) return;
+    const int which = (int)(wid / (G * G)), a = (int)((wid / G) % G), b = (int)(wid % G);
+    const int lane = threadIdx.x & 31;
+    const float *x, *z; int64_t n;
+    if (which == 3) { x = bp.hT + (int64_t)a * p.ldh; z = bp.yT + (int64_t)b * p.ldh; n = p.ldh; }
+    else {
+        x = (which == 2 ? bp.Rq : bp.Vr) + (int64_t)a * p.ldm;
+        z = (which == 0 ? bp.Vr : bp.Rq) + (int64_t)b * p.ldm;
+        n = p.ldm;
+    }
+    const float4* x4 = reinterpret_cast<const float4*>(x);
+    const float4* z4 = reinterpret_cast<const float4*>(z);
+    float s0 = 0.f, s1 = 0.f;
+    int64_t c = lane;
+    for (; c + 32 < n / 4; c += 64) {
+        const float4 xa = x4[c], zb = z4[c], xc = x4[c + 32], zd = z4[c + 32];
+        s0 += xa.x * zb.x + xa.y * zb.y + xa.z * zb.z + xa.w * zb.w;
+        s1 += xc.x * zd.x + xc.y * zd.y + xc.z * zd.z + xc.w * zd.w;
+    }
+    for (; c < n / 4; c += 32) {
+        const float4 xa = x4[c], zb = z4[c];
+        s0 += xa.x * zb.x + xa.y * zb.y + xa.z * zb.z + xa.w * zb.w;
+    }
+    s0 = warp_sum(s0 + s1);
+    const int slot = which == 0 ? S_GV : which == 1 ? S_GX : which == 2 ? S_GR : B_HY;
+    if (lane == 0) bp.small[(int64_t)slot * G * G + a * G + b] = (double)s0;
+}
+
+// One block: the G x G algebra of the exchange, its exact change of obj and the accept decision.
+__global__ void __launch_bounds__(256)
+k_blk_small(Ptrs p, BlockPtrs bp, int accept_mode, double accept_tol, double* __restrict__ obj_trace, int32_t* __restrict__ swap_trace)
+{
+    SearchCtl* ctl = p.ctl;
+    if (ctl->done) return;
+    __shared__ double red[32];
+    const int g = bp.G, gg = g * g;
+    double* S = bp.small;
+    double *Cinv = S + S_CINV * gg, *c1inv = S + S_C1INV * gg, *Q1 = S + S_Q1 * gg, *Q1c = S + S_Q1C * gg, *M2 = S + S_M2 * gg;
+    double *GV = S + S_GV * gg, *GX = S + S_GX * gg, *GR = S + S_GR * gg, *C = S + S_C * gg, *P = S + S_P * gg;
+    double *T1 = S + S_T1 * gg, *T2 = S + S_T2 * gg, *T3 = S + S_T3 * gg, *c1 = S + S_C1 * gg, *Lw = S + S_L * gg;
+    double *cq = S + B_CQ * gg, *HY = S + B_HY * gg;
+    for (int idx = threadIdx.x; idx < gg; idx += blockDim.x) {
+        const int i = idx / g, j = idx % g;
+        const int64_t ri = blk_rrow(p, bp, i), rj = blk_rrow(p, bp, j);
+        const int64_t qi = p.nI + blk_qrow(p, bp, i), qj = p.nI + blk_qrow(p, bp, j);
+        C[idx] = 0.5 * ((double)bp.PB[(int64_t)i * p.ldh + rj] + (double)bp.PB[(int64_t)j * p.ldh + ri]);
+        P[idx] = (double)bp.yT[(int64_t)i * p.ldh + rj];                  // P[a][b] = y_a[r_b]
+        cq[idx] = (double)p.Hp[qi * p.ldp + qj] - 0.5 * (HY[idx] + HY[j * g + i]);
+    }
+    __syncthreads();
+    const double pivC = chol_inverse(C, Lw, Cinv, g);
+    const double Ds = mat_trace_prod(Cinv, GV, g, red);               // Tr(C^-1 V_r V_r^T)
+    mat_mul(Cinv, false, GX, false, T1, g);                           // K R_q^T
+    mat_mul(P, false, T1, false, T2, g);                              // P K R_q^T
+    mat_mul(P, false, Cinv, false, T1, g);                            // P Cinv
+    mat_mul(T1, false, GV, false, T3, g);                             // P Cinv GV
+    mat_mul(T3, false, T1, true, Lw, g);                              // P Cinv GV Cinv P^T
+    for (int idx = threadIdx.x; idx < gg; idx += blockDim.x) {
+        const int i = idx / g, j = idx % g;
+        T3[idx] = GR[idx] + T2[idx] + T2[j * g + i] + Lw[idx];        // R1 R1^T
+    }
+    __syncthreads();
+    mat_mul(T1, false, P, true, T2, g);                               // P Cinv P^T
+    for (int idx = threadIdx.x; idx < gg; idx += blockDim.x) {
+        const int i = idx / g, j = idx % g;
+        c1[idx] = cq[idx] + 0.5 * (T2[idx] + T2[j * g + i]);
+    }
+    __syncthreads();
+    // the smallest pivot of c1 is compared with the diagonal of H on the entering rows (eligibility of the joint add)
+    double scale = 0.0;
+    for (int i = 0; i < g; ++i) {
+        const int64_t qi = p.nI + blk_qrow(p, bp, i);
+        const double hd = p.Hp[qi * p.ldp + qi];
+        if (hd > scale) scale = hd;
+    }
+    const double pivc1 = chol_inverse(c1, Lw, c1inv, g);
+    const double gain = mat_trace_prod(c1inv, T3, g, red);
+    const double delta = Ds - gain;
+    mat_mul(Cinv, false, P, true, Q1, g);                             // Q1 = Cinv P^T
+    mat_mul(Q1, false, c1inv, false, Q1c, g);                         // Q1 c1inv
+    mat_mul(c1inv, false, T1, false, M2, g);                          // c1inv P Cinv
+    if (threadIdx.x == 0) {
+        const double obj = ctl->obj;
+        bool stop = false; int reason = 0;
+        if (!(pivC > 0.0) || !(pivc1 > kAddPivotTol * scale) || !isfinite(delta)) { stop = true; reason = OSSCAR_STOP_GUARD; }
+        else if (accept_mode == OSSCAR_ACCEPT_IMPROVING && !(delta <= -accept_tol * obj)) { stop = true; reason = OSSCAR_STOP_NO_IMPROVEMENT; }
+        ctl->delta = delta;
+        if (stop) { ctl->done = 1; ctl->stop_reason = reason; *p.done_host = 1; }
+        else {
+            const int n = ctl->n_swaps;
+            for (int t = 0; t < bp.s; ++t) {
+                swap_trace[2 * (n + t)] = p.perm[bp.rslot[t]];
+                swap_trace[2 * (n + t) + 1] = p.perm[p.k + bp.tslot[t]];
+            }
+            obj_trace[n / bp.s + 1] = obj + delta;
+            ctl->obj = obj + delta;
+            ctl->n_swaps = n + bp.s;
+        }
+    }
+}
+
+// Staged panels.  Part A (kept rows i): b C^-1, u2 = y - b Q1 (0 on r), -u2 c1^-1.  Part B (columns): K, Vq.
+__global__ void __launch_bounds__(256) k_blk_prep(Ptrs p, BlockPtrs bp)
+{
+    if (p.ctl->done) return;
+    const int G = bp.G, gg = G * G;
+    const double* S = bp.small;
+    const double *Cinv = S + S_CINV * gg, *c1inv = S + S_C1INV * gg, *Q1 = S + S_Q1 * gg, *Q1c = S + S_Q1C * gg, *M2 = S + S_M2 * gg;
+    const int64_t nA = p.ldh * G, nB = p.ldm * G;
+    for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < nA + nB; idx += (int64_t)gridDim.x * blockDim.x) {
+        if (idx < nA) {
+            const int e = (int)(idx / p.ldh); const int64_t i = idx % p.ldh;
+            float vbc = 0.f, vu2 = 0.f, vnu = 0.f;
+            if (i < p.nI) {
+                double bc = 0.0, bq = 0.0, bqc = 0.0, yc = 0.0;
+                for (int f = 0; f < G; ++f) {
+                    const double bf = (double)bp.PB[(int64_t)f * p.ldh + i];
+                    bc += bf * Cinv[f * G + e];
+                    bq += bf * Q1[f * G + e];
+                    bqc += bf * Q1c[f * G + e];
+                    yc += (double)bp.yT[(int64_t)f * p.ldh + i] * c1inv[f * G + e];
+                }
+                bool in_r = false;
+                const int slot = (int)(i / p.g);
+                for (int t = 0; t < bp.s; ++t) in_r |= bp.rslot[t] == slot;
+                vbc = (float)bc;
+                if (!in_r) { vu2 = (float)((double)bp.yT[(int64_t)e * p.ldh + i] - bq); vnu = (float)(bqc - yc); }
+            }
+            bp.PA[(int64_t)e * p.ldh + i] = vbc;
+            bp.PB[(int64_t)(G + e) * p.ldh + i] = vu2;
+            bp.PA[(int64_t)(G + e) * p.ldh + i] = vnu;
+        } else {
+            const int64_t j = idx - nA;
+            const int e = (int)(j / p.ldm); const int64_t c = j % p.ldm;
+            double kk = 0.0, vq = 0.0;
+            for (int f = 0; f < G; ++f) {
+                const double vr = (double)bp.Vr[(int64_t)f * p.ldm + c];
+                const double rq = (double)bp.Rq[(int64_t)f * p.ldm + c];
+                kk += Cinv[e * G + f] * vr;
+                vq += c1inv[e * G + f] * rq + M2[e * G + f] * vr;
+            }
+            bp.KV[(int64_t)e * p.ldm + c] = (float)kk;
+            bp.KV[(int64_t)(G + e) * p.ldm + c] = (float)vq;
+        }
+    }
+}
+
+// After the H pass: UD[l][G+e] = Hp[l, I] u2_e  ->  -(d_l)_e = that - Hp[l, q_e]; the u part of a leaving row is e_l.
+__global__ void __launch_bounds__(256) k_blk_finish_d(Ptrs p, BlockPtrs bp)
+{
+    if (p.ctl->done) return;
+    const int G = bp.G;
+    const int64_t n = (p.nJ + G) * G;
+    for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < n; idx += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t l = idx / G; const int e = (int)(idx % G);
+        const int64_t row = l < p.nJ ? p.nI + l : blk_rrow(p, bp, (int)(l - p.nJ));
+        float* ud = bp.UD + l * 2 * G;
+        ud[G + e] -= p.Hp[row * p.ldp + p.nI + blk_qrow(p, bp, e)];
+        if (l >= p.nJ) ud[e] = (l - p.nJ == e) ? 1.f : 0.f;
+    }
+}
+
+// Rows and columns r of Hinv' = -u2 c1^-1 (block rr: c1^-1), rows r of V' = Vq, rows q of R' = the leaving rows'
+// residual (staged in Rq).  One launch: blocks [0, G) per leaving row.
+__global__ void __launch_bounds__(256) k_blk_fix(Ptrs p, BlockPtrs bp)
+{
+    if (p.ctl->done) return;
+    const int G = bp.G, t = blockIdx.x;
+    const double* c1inv = bp.small + (int64_t)S_C1INV * G * G;
+    const int64_t row = blk_rrow(p, bp, t), qrow = blk_qrow(p, bp, t);
+    const float* nu = bp.PA + (int64_t)(G + t) * p.ldh;
+    for (int64_t i = threadIdx.x; i < p.nI; i += blockDim.x) {
+        float v = nu[i];
+        const int slot = (int)(i / p.g);
+        for (int a = 0; a < bp.s; ++a)
+            if (bp.rslot[a] == slot) { const int ea = a * p.g + (int)(i % p.g); v = (float)(0.5 * (c1inv[ea * G + t] + c1inv[t * G + ea])); }
+        p.Hinv[i * p.ldh + row] = v;
+        p.Hinv[row * p.ldh + i] = v;
+    }
+    const float* vq = bp.KV + (int64_t)(G + t) * p.ldm;
+    const float* rn = bp.Rq + (int64_t)t * p.ldm;
+    for (int64_t c = threadIdx.x; c < p.m; c += blockDim.x) {
+        p.V[row * p.ldm + c] = vq[c];
+        p.R[qrow * p.ldm + c] = rn[c];
+    }
+}
+
+// c_l' = c_l + u_l C^-1 u_l^T - d_l c1^-1 d_l^T for every pruned slot; an entering slot receives the leaving group
+// (old c = 0, u_l = unit rows).  One block per pruned slot; dynamic shared memory 2 g G doubles.
+__global__ void __launch_bounds__(128) k_blk_update_c(Ptrs p, BlockPtrs bp)
+{
+    if (p.ctl->done) return;
+    extern __shared__ double smc[];
+    const int g = p.g, G = bp.G;
+    double* TU = smc; double* TD = smc + g * G;
+    const int64_t t = blockIdx.x;
+    int pos = -1;
+    for (int a = 0; a < bp.s; ++a) if (bp.tslot[a] == t) pos = a;
+    const int64_t base = pos >= 0 ? p.nJ + (int64_t)pos * g : t * g;
+    const double* Cinv = bp.small + (int64_t)S_CINV * G * G;
+    const double* c1inv = bp.small + (int64_t)S_C1INV * G * G;
+    const float* ud = bp.UD + base * 2 * G;
+    for (int idx = threadIdx.x; idx < g * G; idx += blockDim.x) {
+        const int a = idx / G, f = idx % G;
+        double tu = 0.0, td = 0.0;
+        for (int e = 0; e < G; ++e) {
+            tu += (double)ud[a * 2 * G + e] * Cinv[e * G + f];
+            td += (double)ud[a * 2 * G + G + e] * c1inv[e * G + f];
+        }
+        TU[idx] = tu; TD[idx] = td;
+    }
+    __syncthreads();
+    for (int idx = threadIdx.x; idx < g * g; idx += blockDim.x) {
+        const int a = idx / g, b2 = idx % g;
+        double s = pos >= 0 ? 0.0 : p.c[t * g * g + idx];
+        for (int f = 0; f < G; ++f)
+            s += TU[a * G + f] * (double)ud[b2 * 2 * G + f] - TD[a * G + f] * (double)ud[b2 * 2 * G + G + f];
+        p.c[t * g * g + idx] = s;
+    }
+}
+
+// Exchange the rows (phase 0) or columns (phase 1) of Hp of every leaving / entering pair; phase 1 also exchanges
+// the groups in the slot permutation.
+__global__ void __launch_bounds__(256) k_blk_hswap(Ptrs p, BlockPtrs bp, int phase)
+{
+    if (p.ctl->done) return;
+    const int G = bp.G;
+    const int64_t n = p.ldp * G;
+    for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < n; idx += (int64_t)gridDim.x * blockDim.x) {
+        const int e = (int)(idx / p.ldp); const int64_t x = idx % p.ldp;
+        const int64_t a = blk_rrow(p, bp, e), b = p.nI + blk_qrow(p, bp, e);
+        float *pa, *pb;
+        if (phase == 0) { pa = p.Hp + a * p.ldp + x; pb = p.Hp + b * p.ldp + x; }
+        else {
+            if (x >= p.nI + p.nJ) continue;
+            pa = p.Hp + x * p.ldp + a; pb = p.Hp + x * p.ldp + b;
+        }
+        const float va = *pa, vb = *pb;
+        *pa = vb; *pb = va;
+    }
+    if (phase == 1 && blockIdx.x == 0 && threadIdx.x == 0) {
+        for (int t = 0; t < bp.s; ++t) {
+            const int s = bp.rslot[t], u = p.k + bp.tslot[t];
+            const int gi = p.perm[s], gj = p.perm[u];
+            p.perm[s] = gj; p.perm[u] = gi;
+            p.slotof[gj] = s; p.slotof[gi] = u;
+        }
+    }
+}
+
+// One iteration of the block exchange on the stream; `mark` records an event after each stage when profiling.
+template <class Mark>
+cudaError_t enqueue_block_step(osscar_ctx* ctx, const Ptrs& p, const BlockPtrs& bp, int accept_mode, double tol,
+                               double* obj_trace, int32_t* swap_trace, Mark&& mark)
+{
+    const Layout& L = ctx->L;
+    cudaStream_t st = ctx->stream;
+    const int G = bp.G;
+    const int32_t* done = &ctx->ctl->done;
+    cudaError_t e;
+#define BK(x) do { e = (x); if (e != cudaSuccess) return e; } while (0)
+    k_blk_select<<<1, 1024, 0, st>>>(p, bp);                                                    mark();
+    k_blk_gather<<<dim3((unsigned)G, 5), 256, 0, st>>>(p, bp);
+    BK(sgemm(st, false, false, G, L.nI, L.nI, 1.f, bp.hT, L.ldh, p.Hinv, L.ldh, 0.f, bp.yT, L.ldh, done));   mark();
+    k_blk_gram<<<(unsigned)((4 * G * G + 7) / 8), 256, 0, st>>>(p, bp);
+    k_blk_small<<<1, 256, 0, st>>>(p, bp, accept_mode, tol, obj_trace, swap_trace);
+    k_blk_prep<<<(unsigned)(((L.ldh + L.ldm) * G + 255) / 256), 256, 0, st>>>(p, bp);           mark();
+    // H pass: [u | H u2] for the pruned rows and the leaving rows, then -d
+    BK(sgemm(st, false, true, L.nJ, 2 * G, L.nI, 1.f, p.Hp + L.nI * L.ldp, L.ldp, bp.PB, L.ldh, 0.f, bp.UD, 2 * G, done));
+    BK(sgemm(st, false, true, G, 2 * G, L.nI, 1.f, bp.HrT, L.ldh, bp.PB, L.ldh, 0.f, bp.UD + L.nJ * 2 * G, 2 * G, done));
+    k_blk_finish_d<<<(unsigned)(((L.nJ + G) * G + 255) / 256), 256, 0, st>>>(p, bp);            mark();
+    // the three rank-2G updates; the residual rows of the leaving groups go through the Rq panel
+    BK(sgemm(st, true, false, L.nI, L.nI, 2 * G, -1.f, bp.PA, L.ldh, bp.PB, L.ldh, 1.f, p.Hinv, L.ldh, done));   mark();
+    BK(sgemm(st, true, false, L.nI, L.m, 2 * G, -1.f, bp.PB, L.ldh, bp.KV, L.ldm, 1.f, p.V, L.ldm, done));        mark();
+    BK(sgemm(st, false, false, L.nJ, L.m, 2 * G, 1.f, bp.UD, 2 * G, bp.KV, L.ldm, 1.f, p.R, L.ldm, done));
+    BK(sgemm(st, false, false, G, L.m, 2 * G, 1.f, bp.UD + L.nJ * 2 * G, 2 * G, bp.KV, L.ldm, 0.f, bp.Rq, L.ldm, done));   mark();
+    k_blk_update_c<<<(unsigned)(L.ng - L.k), 128, 2 * (size_t)L.g * G * sizeof(double), st>>>(p, bp);
+    k_blk_fix<<<(unsigned)G, 256, 0, st>>>(p, bp);                                              mark();
+    k_blk_hswap<<<(unsigned)((L.ldp * G + 255) / 256), 256, 0, st>>>(p, bp, 0);
+    k_blk_hswap<<<(unsigned)((L.ldp * G + 255) / 256), 256, 0, st>>>(p, bp, 1);                 mark();
+    count_launches(10);
+    BK(enqueue_scores(ctx, p, true, false));                                                   mark();
+#undef BK
+    return cudaGetLastError();
+}

@@ -352,6 +352,22 @@ int make_layout(int64_t d1, int64_t m, int32_t g, int32_t k, Layout* L)
         if (L->tc_bytes < gemm_tc_min_scratch(d1, nmax)) L->tc_bytes = gemm_tc_min_scratch(d1, nmax);
         L->off_tc = take(L->tc_bytes);
     }
+    {   // block exchange: panels for up to min(OSSCAR_MAX_GROUP, n_I, n_J) rows on each side (a multiple of g)
+        int64_t G = OSSCAR_MAX_GROUP;
+        if (nI < G) G = nI;
+        if (nJ < G) G = nJ;
+        G = G / g * g;
+        L->block_rows_max = (int32_t)G;
+        auto al = [](size_t b) { return (b + 255) / 256 * 256; };
+        size_t n = 256;
+        if (G > 0) {
+            n = 2 * al(sizeof(int32_t) * (size_t)G) + 3 * al(sizeof(float) * (size_t)G * ldh) + 2 * al(sizeof(float) * 2 * (size_t)G * ldh)
+              + al(sizeof(float) * 2 * (size_t)G * ldm) + 2 * al(sizeof(float) * (size_t)G * ldm)
+              + al(sizeof(float) * (size_t)(nJ + G) * 2 * G) + al(sizeof(double) * 18 * (size_t)G * G);
+        }
+        L->block_bytes = n;
+        L->off_block = take(n);
+    }
     L->bytes = off;
     return OSSCAR_OK;
 }

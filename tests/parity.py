@@ -71,6 +71,61 @@ def follow_trace(H, G, const, g, S0, swaps, gpu_obj, score_mode="independent", a
     return srch, rebased
 
 
+def follow_block(H, G, const, g, S0, s, swaps, gpu_obj, accept="improving", gpu_stop=None, max_iters=None,
+                 obj_rtol=1e-4, eps_acc=orc.EPS_ACC):
+    """Walks the GPU's block exchanges (s pairs per iteration) with the oracle.  Per iteration the groups the GPU took
+    out must be the s cheapest drops and the groups it brought in the s best adds by the oracle's fresh scores, up
+    to ties within GAP at the cut; the oracle then makes the GPU's exchange and the objectives must agree."""
+    import pytest
+    srch = orc.BlockSearch(H, G, const, g, S0, s, accept=accept, eps_acc=eps_acc)
+    assert gpu_obj[0] == pytest.approx(srch.st.obj, rel=obj_rtol)
+    assert len(swaps) % s == 0 and len(gpu_obj) == len(swaps) // s + 1
+    for it in range(len(swaps) // s):
+        out = [o for o, _ in swaps[it * s:(it + 1) * s]]
+        inn = [i for _, i in swaps[it * s:(it + 1) * s]]
+        info = srch.propose()
+        assert info is not None, f"iteration {it}: oracle has no candidate"
+        assert len(set(out)) == s and len(set(inn)) == s, f"iteration {it}: repeated group"
+        S = srch.st.S
+        assert all(o in S for o in out) and all(i in srch.st.c for i in inn), f"iteration {it}: impossible exchange"
+        slots = [int(np.nonzero(S == o)[0][0]) for o in out]
+        thrD = np.sort(info.D)[s - 1]
+        finiteA = info.A[np.isfinite(info.A)]
+        thrA = np.sort(finiteA)[::-1][s - 1]
+        for sl in slots:
+            assert info.D[sl] <= thrD * (1 + GAP) + 1e-300, f"iteration {it}: group {S[sl]} is not among the {s} cheapest"
+        for sl in range(len(S)):
+            if sl not in slots:
+                assert info.D[sl] >= thrD * (1 - GAP) - 1e-300, f"iteration {it}: kept group {S[sl]} is cheaper than a dropped one"
+        for q in inn:
+            assert info.A[q] >= thrA * (1 - GAP) - 1e-300, f"iteration {it}: group {q} is not among the {s} best adds"
+        for q in srch.st.c:
+            if q not in inn and np.isfinite(info.A[q]):
+                assert info.A[q] <= thrA * (1 + GAP) + 1e-300, f"iteration {it}: pruned group {q} beats an added one"
+        same = sorted(out) == sorted(info.out) and sorted(inn) == sorted(info.inn)
+        delta = info.delta if same else srch.exchange_delta(slots, inn)
+        if accept == "improving":
+            thr = -srch.eps_acc * srch.st.obj
+            Dsum = float(np.sum(info.D[slots]))
+            band = GAP * (abs(Dsum) + abs(Dsum - delta))
+            assert delta <= thr or abs(delta - thr) <= band, f"iteration {it}: accepted a non-improving exchange"
+        srch.apply(slots, inn)
+        assert gpu_obj[it + 1] == pytest.approx(srch.st.obj, rel=obj_rtol), f"iteration {it}: objective drifted"
+    if gpu_stop == "no_improvement":
+        info = srch.propose()
+        if info is not None and info.accepted:
+            Dsum = float(np.sum(info.D[info.slots]))
+            band = GAP * (abs(Dsum) + abs(Dsum - info.delta))
+            sD = np.sort(info.D); sA = np.sort(info.A[np.isfinite(info.A)])[::-1]
+            tie = (len(sD) > s and sD[s] - sD[s - 1] <= GAP * abs(sD[s - 1])) or \
+                  (len(sA) > s and sA[s - 1] - sA[s] <= GAP * abs(sA[s - 1]))
+            assert abs(info.delta + srch.eps_acc * srch.st.obj) <= band or tie, \
+                f"GPU stopped but the oracle would go on (delta {info.delta}, obj {srch.st.obj})"
+    elif gpu_stop == "max_swaps":
+        assert len(swaps) // s == max_iters
+    return srch
+
+
 def rel_fro(a, b):
     a = np.asarray(a, np.float64); b = np.asarray(b, np.float64)
     return float(np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-300))

@@ -5,7 +5,7 @@ import torch
 
 import workloads
 from oracle import osscar_oracle as orc
-from tests.parity import GAP, follow_greedy, follow_trace, oracle_problem, rel_fro
+from tests.parity import GAP, follow_block, follow_greedy, follow_trace, oracle_problem, rel_fro
 
 pytestmark = pytest.mark.gpu
 
@@ -328,6 +328,78 @@ def test_state_after_search_is_consistent(solver):
     assert rel_fro(solver.debug_state(2).cpu().numpy(), st.R[perm[wl.k:]]) < 1e-4
     c = solver.debug_state(3).cpu().numpy().reshape(-1)
     assert np.allclose(c, [st.c[int(q)][0, 0] for q in perm[wl.k:]], rtol=1e-3)
+
+
+# ------------------------------------------------------------------------------------ block exchanges (t_hat = 2 s, p_hat = 0)
+BLOCK_CASES = [
+    # name, overrides, seed, pairs per iteration, max_swaps, accept always
+    ("c1", {}, 0, 2, 50, False),
+    ("c1", {}, 1, 5, 50, True),
+    ("c2", dict(n=4096, d1=520, m=150, k=207, chunk_rows=4096), 1, 4, 200, False),
+    ("c2", dict(n=4096, d1=520, m=150, k=207, chunk_rows=4096), 0, 16, 160, False),
+    ("c5", dict(n=8192, d1=1000, m=300, k=300, chunk_rows=4096), 0, 50, 500, False),
+    ("c5", dict(n=4096, d1=520, m=150, k=156, chunk_rows=4096), 2, 96, 960, True),
+    ("c4", dict(n=49 * 40, d1=9 * 100, m=130, k=50, chunk_rows=49 * 40), 0, 2, 60, False),
+    ("c4", dict(n=49 * 40, d1=9 * 100, m=130, k=50, chunk_rows=49 * 40), 1, 5, 40, True),
+    ("c3", dict(n=8192, d1=12 * 40, m=200, g=40, k=6, chunk_rows=8192, score_mode="independent"), 0, 2, 12, True),
+]
+
+
+@pytest.mark.parametrize("name,over,seed,s,max_swaps,always", BLOCK_CASES)
+def test_block_exchange_matches_oracle(solver, name, over, seed, s, max_swaps, always):
+    """s groups out and s groups in per iteration: sets, exact change, objective, final support and weights."""
+    import paper_2403_12983_b200.binding as b
+    wl = workloads.config(name, seed=seed, **over)
+    chunks, W, H64, G64, const64 = oracle_problem(wl)
+    H, G, Wd = dev(H64), dev(G64), dev(W)
+    Hr, Gr = H.cpu().numpy().astype(np.float64), G.cpu().numpy().astype(np.float64)
+    const_r = float(np.sum(W * Gr))
+    support, obj0 = solver.init_support(H, G, Wd, wl.g, wl.k)
+    S0 = support.cpu().numpy()
+    max_swaps = min(max_swaps, 6 * s) if always else max_swaps
+    out = solver.local_search(max_swaps, accept_mode=b.ACCEPT_ALWAYS if always else b.ACCEPT_IMPROVING,
+                              accept_rel_tol=wl.eps_acc, block_pairs=s)
+    swaps = [tuple(int(v) for v in r) for r in out.swap_trace.cpu().numpy()]
+    gobj = out.obj_trace.cpu().numpy()
+    assert out.n_swaps % s == 0 and (out.n_swaps >= s or not always)
+    srch = follow_block(Hr, Gr, const_r, wl.g, S0, s, swaps, gobj, accept="always" if always else "improving",
+                        gpu_stop=out.stop_reason, max_iters=max_swaps // s, eps_acc=wl.eps_acc)
+    S_or, W_or, _, _ = srch.result()
+    assert np.array_equal(out.support.cpu().numpy(), S_or)
+    assert out.obj_final == pytest.approx(srch.st.obj, rel=1e-4)
+    assert gobj[-1] == pytest.approx(out.obj_final, rel=1e-4)
+    assert rel_fro(out.W.cpu().numpy(), W_or) < 1e-3
+    # the maintained state against a fresh solve of the final support (slot order of the device)
+    perm = solver.debug_state(4).cpu().numpy()
+    st = orc.fresh_state(Hr, Gr, const_r, perm[:wl.k], wl.g)
+    assert rel_fro(solver.debug_state(0).cpu().numpy(), st.Hinv) < 1e-3
+    assert rel_fro(solver.debug_state(1).cpu().numpy(), st.V) < 1e-3
+    pr = orc.rows_of(perm[wl.k:], wl.g)
+    assert rel_fro(solver.debug_state(2).cpu().numpy(), st.R[pr]) < 1e-3
+    c = solver.debug_state(3).cpu().numpy()
+    cref = np.stack([st.c[int(q)] for q in perm[wl.k:]])
+    assert np.allclose(c, cref, rtol=2e-3, atol=2e-3 * np.abs(cref).max())
+
+
+def test_block_exchange_argument_checks(solver, osscar):
+    import paper_2403_12983_b200.binding as b
+    wl = workloads.config("c1")
+    chunks, W, H64, G64, _ = oracle_problem(wl)
+    H, G, Wd = dev(H64), dev(G64), dev(W)
+    solver.init_support(H, G, Wd, 1, wl.k)
+    for bad in (33, 97):                      # more pairs than pruned / kept groups, more rows than the limit
+        with pytest.raises(osscar.OsscarError) as ei:
+            solver.local_search(100, block_pairs=bad)
+        assert ei.value.status == b.E_ARG
+    with pytest.raises(osscar.OsscarError):
+        solver.local_search(10, score_mode=b.SCORE_PAIR_EXACT, block_pairs=2)
+    out = solver.local_search(3, block_pairs=4)           # fewer swaps allowed than one iteration exchanges
+    assert out.n_swaps == 0 and out.stop_reason == "max_swaps"
+    out = solver.local_search(50, block_pairs=1)          # one pair per iteration is the plain swap search
+    ref = orc.Search(H.cpu().numpy().astype(np.float64), G.cpu().numpy().astype(np.float64),
+                     float(np.sum(W * G.cpu().numpy().astype(np.float64))), 1,
+                     orc.init_support(H.cpu().numpy().astype(np.float64), W, 1, wl.k)[0]).run(50)
+    assert out.n_swaps == len(ref.swap_trace)
 
 
 # ------------------------------------------------------------------------------------ nested (greedy) phase
