@@ -28,7 +28,9 @@ constexpr int A_BYTES = TILE_M * BLOCK_K * 2;                 // 16384: one box 
 constexpr int BOX_BYTES = 64 * BLOCK_K * 2;                   // 8192: 64 columns of B x 64 k-rows
 constexpr int B_BYTES = (TILE_N / 64) * BOX_BYTES;            // 32768
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256;
+constexpr int EPI_LD = 33;                                    // row stride (floats) of an epilogue staging block
+constexpr int EPI_BYTES = 8 * 32 * EPI_LD * 4;                // one 32 x 32 block per accumulate warp
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256 + EPI_BYTES;
 constexpr int NUM_THREADS = 320;                              // 10 warps
 constexpr int TMEM_COLS = 512;
 constexpr int BAND = 8;                                       // tile rows per raster band (full rasters)
@@ -112,6 +114,7 @@ k_mma_pipe(const __grid_constant__ Maps maps, int64_t M, int64_t N, int64_t K, f
     auto tempty_bar = [&](int b) { return bars + 8u * (2 * STAGES + 2 + b); };
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_ptr + 8 * (2 * STAGES + 4));
     volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_ptr + 8 * (2 * STAGES + 4) + 8);
+    float* epi = reinterpret_cast<float*>(bar_ptr + 256);      // staging blocks of the accumulate warps
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int TM = (int)((M + TILE_M - 1) / TILE_M), TN = (int)((N + TILE_N - 1) / TILE_N);
@@ -238,25 +241,47 @@ k_mma_pipe(const __grid_constant__ Maps maps, int64_t M, int64_t N, int64_t K, f
             if (!ok) break;
             const int64_t grow = (int64_t)tm * TILE_M + lg * 32 + lane;
             const int64_t gcol0 = (int64_t)tn * TILE_N + half * 128;
-            if (grow < M) {
+            {
                 float* crow = C + grow * ldc;
                 if (vec_ok) {
+                    // 32 x 32 blocks go through shared memory so that a warp touches whole 128-byte lines of C:
+                    // 8 lanes per row, 4 rows per instruction, the 8 row groups of a block in flight together
+                    float* stg = epi + (warp - 2) * 32 * EPI_LD;
+                    const int64_t grow0 = (int64_t)tm * TILE_M + lg * 32;
+                    const int rsub = lane >> 3, c4 = (lane & 7) * 4;
 #pragma unroll
-                    for (int j = 0; j < 128; j += 4) {
-                        if (gcol0 + j < N) {        // N is a multiple of 4 on this path
-                            float4* dst = reinterpret_cast<float4*>(crow + gcol0 + j);
-                            float4 v = make_float4(alpha * acc[j], alpha * acc[j + 1], alpha * acc[j + 2], alpha * acc[j + 3]);
-                            if (beta != 0.f) {
-                                const float4 o = *dst;
-                                v.x = fmaf(beta, o.x, v.x); v.y = fmaf(beta, o.y, v.y); v.z = fmaf(beta, o.z, v.z); v.w = fmaf(beta, o.w, v.w);
+                    for (int c = 0; c < 4; ++c) {
+                        const int64_t gc = gcol0 + c * 32 + c4;
+                        __syncwarp();
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) stg[lane * EPI_LD + j] = alpha * acc[c * 32 + j];
+                        __syncwarp();
+                        float4 o[8];
+                        if (beta != 0.f) {
+#pragma unroll
+                            for (int q = 0; q < 8; ++q) {
+                                const int64_t gr = grow0 + q * 4 + rsub;
+                                o[q] = (gr < M && gc < N) ? __ldcs(reinterpret_cast<const float4*>(C + gr * ldc + gc))
+                                                          : make_float4(0.f, 0.f, 0.f, 0.f);
                             }
-                            *dst = v;
+                        }
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) {
+                            const int r = q * 4 + rsub;
+                            const int64_t gr = grow0 + r;
+                            const float* sp = stg + r * EPI_LD + c4;
+                            float4 v = make_float4(sp[0], sp[1], sp[2], sp[3]);
+                            if (beta != 0.f) {
+                                v.x = fmaf(beta, o[q].x, v.x); v.y = fmaf(beta, o[q].y, v.y);
+                                v.z = fmaf(beta, o[q].z, v.z); v.w = fmaf(beta, o[q].w, v.w);
+                            }
+                            if (gr < M && gc < N) *reinterpret_cast<float4*>(C + gr * ldc + gc) = v;
                         }
                     }
                 } else {
 #pragma unroll
                     for (int j = 0; j < 128; ++j) {
-                        if (gcol0 + j < N) {
+                        if (grow < M && gcol0 + j < N) {
                             float v = alpha * acc[j];
                             if (beta != 0.f) v = fmaf(beta, crow[gcol0 + j], v);
                             crow[gcol0 + j] = v;

@@ -55,6 +55,19 @@ struct Layout {
     int64_t pair_capacity;                                             // pairs the workspace can score
     size_t bytes;
 };
+// bytes of the block-exchange panels for G rows on each side (layout in search_block.cuh)
+static inline size_t block_region_bytes(int64_t ldh, int64_t ldm, int64_t nJ, int64_t G)
+{
+    auto al = [](size_t b) { return (b + 255) / 256 * 256; };
+    size_t n = 2 * al(sizeof(int32_t) * (size_t)G);
+    n += 3 * al(sizeof(float) * (size_t)G * ldh);            // hT, yT, HrT
+    n += 4 * al(sizeof(float) * 2 * (size_t)G * ldh);        // PB, PA and their transposes
+    n += al(sizeof(float) * 2 * (size_t)G * ldm);            // KV
+    n += 2 * al(sizeof(float) * (size_t)G * ldm);            // Vr, Rq
+    n += al(sizeof(float) * (size_t)(nJ + G) * 2 * G);       // UD
+    n += al(sizeof(double) * 18 * (size_t)G * G);            // small matrices
+    return n;
+}
 int make_layout(int64_t d1, int64_t m, int32_t g, int32_t k, Layout* L);
 
 }  // namespace osscar
@@ -88,6 +101,12 @@ namespace osscar {
 cudaError_t sgemm(cudaStream_t st, bool transA, bool transB, int64_t M, int64_t N, int64_t K,
                   float alpha, const float* A, int64_t lda, const float* B, int64_t ldb,
                   float beta, float* C, int64_t ldc, const int32_t* done = nullptr);
+
+// ---- panel.cu: Y[i*so_row + e*so_col] = sum_k A[i][k] * P[e][k]; A is M x K (streamed once), P an N x K panel --------
+// `scratch` (may be null) holds partial sums when the k range is split to fill the machine.
+cudaError_t panel_dot(cudaStream_t st, int64_t M, int64_t N, int64_t K, const float* A, int64_t lda,
+                      const float* P, int64_t ldp, float* Y, int64_t so_row, int64_t so_col,
+                      float* scratch, size_t scratch_floats, const int32_t* done = nullptr);
 
 // ---- gemm_tc.cu: the same product on the tensor cores (three-term bf16 split, fp32-accurate); A and B row-major.
 // `scratch` (256-byte aligned device memory, at least gemm_tc_min_scratch bytes) holds the bf16 terms of one K panel.

@@ -785,7 +785,7 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
     const bool block = bs > 1;
     if (block) {
         if (pair || (int64_t)bs * g > L.block_rows_max || bs > L.k || bs > L.ng - L.k) return OSSCAR_E_ARG;
-        if (block_region_bytes(L, bs * g) > L.block_bytes) return OSSCAR_E_WORKSPACE;
+        if (block_bytes_for(L, bs * g) > L.block_bytes) return OSSCAR_E_WORKSPACE;
     }
     BlockPtrs bp = make_block_ptrs(ctx, bs);
     const bool fast = g == 1 && !pair && !block;  // fused five-launch step for single-row groups
@@ -820,7 +820,7 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
     if (max_swaps > 0 && fast) CK(bootstrap_g1());
 
     if (block) {
-        CK(cudaMemsetAsync((char*)ctx->ws + L.off_block, 0, block_region_bytes(L, bs * g), st));
+        CK(cudaMemsetAsync((char*)ctx->ws + L.off_block, 0, block_bytes_for(L, bs * g), st));
         const size_t smem = 2 * (size_t)g * bs * g * sizeof(double);
         if (smem > 48 * 1024) CK(cudaFuncSetAttribute(k_blk_update_c, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     }

@@ -11,31 +11,21 @@
 //   PB (2G x ldh)      [ b ; u2 ]          b = rows r of Hinv
 //   PA (2G x ldh)      [ b C^-1 ; -u2 c1^-1 ]
 //   KV (2G x ldm)      [ K ; Vq ]
+//   PBT, PAT (n_I x 2G) the transposes of PB and PA (left operands of the update GEMMs)
 //   UD ((n_J+G) x 2G)  [ u | -d ] for the pruned rows, then the leaving rows
 //   Hinv' = Hinv - PA^T PB,   V' = V - PB^T KV,   R' = R + UD KV      (three GEMMs with inner dimension 2G)
 #pragma once
 
 struct BlockPtrs {
     int32_t *rslot, *tslot;        // kept slots that leave (cheapest first), pruned slots that enter (best first)
-    float *hT, *yT, *HrT, *PB, *PA, *KV, *Vr, *Rq, *UD;
+    float *hT, *yT, *HrT, *PB, *PA, *PBT, *PAT, *KV, *Vr, *Rq, *UD;
     double* small;                 // kBlockSmall matrices of G x G doubles
     int s, G;
 };
 constexpr int kBlockSmall = 18;
 enum { B_CQ = 16, B_HY = 17 };     // joint Schur complement of the entering rows, h^T y
 
-size_t block_region_bytes(const Layout& L, int G)
-{
-    auto al = [](size_t b) { return (b + 255) / 256 * 256; };
-    size_t n = 2 * al(sizeof(int32_t) * (size_t)G);
-    n += 3 * al(sizeof(float) * (size_t)G * L.ldh);          // hT, yT, HrT
-    n += 2 * al(sizeof(float) * 2 * (size_t)G * L.ldh);      // PB, PA
-    n += al(sizeof(float) * 2 * (size_t)G * L.ldm);          // KV
-    n += 2 * al(sizeof(float) * (size_t)G * L.ldm);          // Vr, Rq
-    n += al(sizeof(float) * (size_t)(L.nJ + G) * 2 * G);     // UD
-    n += al(sizeof(double) * kBlockSmall * (size_t)G * G);
-    return n;
-}
+size_t block_bytes_for(const Layout& L, int G) { return osscar::block_region_bytes(L.ldh, L.ldm, L.nJ, G); }
 
 BlockPtrs make_block_ptrs(osscar_ctx* ctx, int s)
 {
@@ -53,6 +43,8 @@ BlockPtrs make_block_ptrs(osscar_ctx* ctx, int s)
     bp.HrT = (float*)take(sizeof(float) * (size_t)G * L.ldh);
     bp.PB = (float*)take(sizeof(float) * 2 * (size_t)G * L.ldh);
     bp.PA = (float*)take(sizeof(float) * 2 * (size_t)G * L.ldh);
+    bp.PBT = (float*)take(sizeof(float) * 2 * (size_t)G * L.ldh);
+    bp.PAT = (float*)take(sizeof(float) * 2 * (size_t)G * L.ldh);
     bp.KV = (float*)take(sizeof(float) * 2 * (size_t)G * L.ldm);
     bp.Vr = (float*)take(sizeof(float) * (size_t)G * L.ldm);
     bp.Rq = (float*)take(sizeof(float) * (size_t)G * L.ldm);
@@ -65,73 +57,74 @@ BlockPtrs make_block_ptrs(osscar_ctx* ctx, int s)
 __device__ __forceinline__ int64_t blk_rrow(const Ptrs& p, const BlockPtrs& bp, int e) { return (int64_t)bp.rslot[e / p.g] * p.g + e % p.g; }
 __device__ __forceinline__ int64_t blk_qrow(const Ptrs& p, const BlockPtrs& bp, int e) { return (int64_t)bp.tslot[e / p.g] * p.g + e % p.g; }
 
-// Arg-min over val[0..n) (negate: arg-max), ties to the smaller id; the array is rewritten between calls, so it is
-// read through a plain pointer.  Result in every thread.
-__device__ void blk_argmin(double* val, const int32_t* ids, int n, bool negate, double* best_out, int* idx_out)
-{
-    __shared__ double sv[32]; __shared__ int sid[32]; __shared__ int sidx[32];
-    const int t = threadIdx.x, lane = t & 31, w = t >> 5;
-    double best = INFINITY; int bid = INT_MAX, bidx = -1;
-    for (int i = t; i < n; i += blockDim.x) {
-        const double v = negate ? -val[i] : val[i];
-        const int id = ids[i];
-        if (v < best || (v == best && id < bid)) { best = v; bid = id; bidx = i; }
-    }
-    for (int o = 16; o > 0; o >>= 1) {
-        const double ov = __shfl_xor_sync(0xffffffffu, best, o);
-        const int oid = __shfl_xor_sync(0xffffffffu, bid, o);
-        const int oidx = __shfl_xor_sync(0xffffffffu, bidx, o);
-        if (ov < best || (ov == best && oid < bid)) { best = ov; bid = oid; bidx = oidx; }
-    }
-    __syncthreads();
-    if (lane == 0) { sv[w] = best; sid[w] = bid; sidx[w] = bidx; }
-    __syncthreads();
-    if (t == 0) {
-        for (int i = 1; i < (int)(blockDim.x >> 5); ++i)
-            if (sv[i] < best || (sv[i] == best && sid[i] < bid)) { best = sv[i]; bid = sid[i]; bidx = sidx[i]; }
-        sv[0] = best; sidx[0] = bidx;
-    }
-    __syncthreads();
-    *best_out = negate ? -sv[0] : sv[0];
-    *idx_out = sidx[0];
-    __syncthreads();
-}
-
-// The s cheapest kept slots and the s most valuable pruned slots (scores at the current support; ties -> smaller id).
-// Chosen entries of D and A are overwritten with +-inf while the lists are drawn.
+// The s cheapest kept slots (block 0) and the s most valuable pruned slots (block 1), from the scores at the current
+// support; ties go to the smaller group id.  Every thread keeps the best of its own strided share of the scores;
+// a round reduces those over the block, and only the winner's owner rescans its share.  Chosen entries of D and A
+// are overwritten with +-inf while the lists are drawn.
 __global__ void __launch_bounds__(1024) k_blk_select(Ptrs p, BlockPtrs bp)
 {
     SearchCtl* ctl = p.ctl;
     if (ctl->done) return;
-    const int npr = (int)(p.ng - p.k);
-    if (p.g == 1) {
-        for (int i = threadIdx.x; i < p.k; i += blockDim.x) {
-            const double hd = p.Hinv[(int64_t)i * p.ldh + i];
-            p.D[i] = hd > 0.0 ? (double)p.vnorm[i] / hd : INFINITY;
+    __shared__ double sv[32]; __shared__ int sid[32]; __shared__ int sidx[32];
+    const int side = blockIdx.x;
+    const int n = side == 0 ? p.k : (int)(p.ng - p.k);
+    double* val = side == 0 ? p.D : p.A;
+    const int32_t* ids = side == 0 ? p.perm : p.perm + p.k;
+    int32_t* out = side == 0 ? bp.rslot : bp.tslot;
+    const int t = threadIdx.x, lane = t & 31, w = t >> 5, nt = blockDim.x;
+    if (p.g == 1) {                       // single-row groups: scores from the row norms
+        for (int i = t; i < n; i += nt) {
+            if (side == 0) {
+                const double hd = p.Hinv[(int64_t)i * p.ldh + i];
+                val[i] = hd > 0.0 ? (double)p.vnorm[i] / hd : INFINITY;
+            } else {
+                const double cc = p.c[i];
+                const double hd = p.Hp[(p.nI + i) * p.ldp + p.nI + i];
+                val[i] = cc > kAddPivotTol * hd ? (double)p.rnorm[i] / cc : -INFINITY;
+            }
         }
-        for (int i = threadIdx.x; i < npr; i += blockDim.x) {
-            const double cc = p.c[i];
-            const double hd = p.Hp[(p.nI + i) * p.ldp + p.nI + i];
-            p.A[i] = cc > kAddPivotTol * hd ? (double)p.rnorm[i] / cc : -INFINITY;
+    }
+    const double sign = side == 0 ? 1.0 : -1.0;
+    double best; int bid, bidx;
+    auto rescan = [&]() {                 // a thread only ever reads entries it wrote or that no thread writes
+        best = INFINITY; bid = INT_MAX; bidx = -1;
+        for (int i = t; i < n; i += nt) {
+            const double v = sign * val[i];
+            const int id = ids[i];
+            if (v < best || (v == best && id < bid)) { best = v; bid = id; bidx = i; }
+        }
+    };
+    rescan();
+    for (int round = 0; round < bp.s; ++round) {
+        double rv = best; int rid = bid, rix = bidx;
+        for (int o = 16; o > 0; o >>= 1) {
+            const double ov = __shfl_xor_sync(0xffffffffu, rv, o);
+            const int oid = __shfl_xor_sync(0xffffffffu, rid, o);
+            const int oix = __shfl_xor_sync(0xffffffffu, rix, o);
+            if (ov < rv || (ov == rv && oid < rid)) { rv = ov; rid = oid; rix = oix; }
+        }
+        if (lane == 0) { sv[w] = rv; sid[w] = rid; sidx[w] = rix; }
+        __syncthreads();
+        if (w == 0) {
+            rv = lane < (nt >> 5) ? sv[lane] : INFINITY; rid = lane < (nt >> 5) ? sid[lane] : INT_MAX; rix = lane < (nt >> 5) ? sidx[lane] : -1;
+            for (int o = 16; o > 0; o >>= 1) {
+                const double ov = __shfl_xor_sync(0xffffffffu, rv, o);
+                const int oid = __shfl_xor_sync(0xffffffffu, rid, o);
+                const int oix = __shfl_xor_sync(0xffffffffu, rix, o);
+                if (ov < rv || (ov == rv && oid < rid)) { rv = ov; rid = oid; rix = oix; }
+            }
+            if (lane == 0) { sv[0] = rv; sidx[0] = rix; }
         }
         __syncthreads();
-    }
-    bool ok = true;
-    for (int t = 0; t < bp.s; ++t) {
-        double best; int idx;
-        blk_argmin(p.D, p.perm, p.k, false, &best, &idx);
-        if (idx < 0 || !isfinite(best)) { ok = false; break; }
-        if (threadIdx.x == 0) { bp.rslot[t] = idx; p.D[idx] = INFINITY; }
+        const double wv = sv[0]; const int wix = sidx[0];
         __syncthreads();
+        if (wix < 0 || !isfinite(wv)) {
+            if (t == 0) { ctl->done = 1; ctl->stop_reason = OSSCAR_STOP_GUARD; *p.done_host = 1; }
+            return;
+        }
+        if (t == 0) out[round] = wix;
+        if (wix % nt == t) { val[wix] = sign * INFINITY; rescan(); }
     }
-    for (int t = 0; ok && t < bp.s; ++t) {
-        double best; int idx;
-        blk_argmin(p.A, p.perm + p.k, npr, true, &best, &idx);
-        if (idx < 0 || !isfinite(best)) { ok = false; break; }
-        if (threadIdx.x == 0) { bp.tslot[t] = idx; p.A[idx] = -INFINITY; }
-        __syncthreads();
-    }
-    if (!ok && threadIdx.x == 0) { ctl->done = 1; ctl->stop_reason = OSSCAR_STOP_GUARD; *p.done_host = 1; }
 }
 
 // Rows of the exchange copied into the panels: hT, HrT (rows of Hp), b (rows of Hinv), V_r, R_q.  grid (G, 5).
@@ -186,7 +179,7 @@ __global__ void __launch_bounds__(256) k_blk_gram(Ptrs p, BlockPtrs bp)
 }
 
 // One block: the G x G algebra of the exchange, its exact change of obj and the accept decision.
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(1024)
 k_blk_small(Ptrs p, BlockPtrs bp, int accept_mode, double accept_tol, double* __restrict__ obj_trace, int32_t* __restrict__ swap_trace)
 {
     SearchCtl* ctl = p.ctl;
@@ -288,6 +281,12 @@ __global__ void __launch_bounds__(256) k_blk_prep(Ptrs p, BlockPtrs bp)
             bp.PA[(int64_t)e * p.ldh + i] = vbc;
             bp.PB[(int64_t)(G + e) * p.ldh + i] = vu2;
             bp.PA[(int64_t)(G + e) * p.ldh + i] = vnu;
+            if (i < p.nI) {
+                bp.PBT[i * 2 * G + e] = bp.PB[(int64_t)e * p.ldh + i];
+                bp.PBT[i * 2 * G + G + e] = vu2;
+                bp.PAT[i * 2 * G + e] = vbc;
+                bp.PAT[i * 2 * G + G + e] = vnu;
+            }
         } else {
             const int64_t j = idx - nA;
             const int e = (int)(j / p.ldm); const int64_t c = j % p.ldm;
@@ -302,6 +301,31 @@ __global__ void __launch_bounds__(256) k_blk_prep(Ptrs p, BlockPtrs bp)
             bp.KV[(int64_t)(G + e) * p.ldm + c] = (float)vq;
         }
     }
+}
+
+// H pass of the G leaving rows: UD[n_J + a][G + e] = Hp[r_a, 0:n_I] . u2_e, one warp per entry.
+__global__ void __launch_bounds__(256) k_blk_leave_d(Ptrs p, BlockPtrs bp)
+{
+    if (p.ctl->done) return;
+    const int G = bp.G;
+    const int64_t wid = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (wid >= (int64_t)G * G) return;
+    const int a = (int)(wid / G), e = (int)(wid % G), lane = threadIdx.x & 31;
+    const float4* x4 = reinterpret_cast<const float4*>(bp.HrT + (int64_t)a * p.ldh);
+    const float4* z4 = reinterpret_cast<const float4*>(bp.PB + (int64_t)(G + e) * p.ldh);
+    float s0 = 0.f, s1 = 0.f;
+    int64_t c = lane;
+    for (; c + 32 < p.ldh / 4; c += 64) {
+        const float4 xa = x4[c], zb = z4[c], xc = x4[c + 32], zd = z4[c + 32];
+        s0 += xa.x * zb.x + xa.y * zb.y + xa.z * zb.z + xa.w * zb.w;
+        s1 += xc.x * zd.x + xc.y * zd.y + xc.z * zd.z + xc.w * zd.w;
+    }
+    for (; c < p.ldh / 4; c += 32) {
+        const float4 xa = x4[c], zb = z4[c];
+        s0 += xa.x * zb.x + xa.y * zb.y + xa.z * zb.z + xa.w * zb.w;
+    }
+    s0 = warp_sum(s0 + s1);
+    if (lane == 0) bp.UD[(p.nJ + a) * 2 * G + G + e] = s0;
 }
 
 // After the H pass: UD[l][G+e] = Hp[l, I] u2_e  ->  -(d_l)_e = that - Hp[l, q_e]; the u part of a leaving row is e_l.
@@ -418,26 +442,30 @@ cudaError_t enqueue_block_step(osscar_ctx* ctx, const Ptrs& p, const BlockPtrs& 
     const int32_t* done = &ctx->ctl->done;
     cudaError_t e;
 #define BK(x) do { e = (x); if (e != cudaSuccess) return e; } while (0)
-    k_blk_select<<<1, 1024, 0, st>>>(p, bp);                                                    mark();
+    k_blk_select<<<2, 1024, 0, st>>>(p, bp);                                                    mark();
     k_blk_gather<<<dim3((unsigned)G, 5), 256, 0, st>>>(p, bp);
-    BK(sgemm(st, false, false, G, L.nI, L.nI, 1.f, bp.hT, L.ldh, p.Hinv, L.ldh, 0.f, bp.yT, L.ldh, done));   mark();
+    float* big = (float*)((char*)ctx->ws + L.off_big);          // free between refreshes: partial sums of split products
+    const size_t big_floats = (L.off_Hp - L.off_big) / sizeof(float);
+    BK(panel_dot(st, L.nI, G, L.nI, p.Hinv, L.ldh, bp.hT, L.ldh, bp.yT, 1, L.ldh, big, big_floats, done));     mark();   // y^T (Hinv symmetric)
     k_blk_gram<<<(unsigned)((4 * G * G + 7) / 8), 256, 0, st>>>(p, bp);
-    k_blk_small<<<1, 256, 0, st>>>(p, bp, accept_mode, tol, obj_trace, swap_trace);
+    k_blk_small<<<1, 1024, 0, st>>>(p, bp, accept_mode, tol, obj_trace, swap_trace);
     k_blk_prep<<<(unsigned)(((L.ldh + L.ldm) * G + 255) / 256), 256, 0, st>>>(p, bp);           mark();
     // H pass: [u | H u2] for the pruned rows and the leaving rows, then -d
-    BK(sgemm(st, false, true, L.nJ, 2 * G, L.nI, 1.f, p.Hp + L.nI * L.ldp, L.ldp, bp.PB, L.ldh, 0.f, bp.UD, 2 * G, done));
-    BK(sgemm(st, false, true, G, 2 * G, L.nI, 1.f, bp.HrT, L.ldh, bp.PB, L.ldh, 0.f, bp.UD + L.nJ * 2 * G, 2 * G, done));
+    BK(panel_dot(st, L.nJ, 2 * G, L.nI, p.Hp + L.nI * L.ldp, L.ldp, bp.PB, L.ldh, bp.UD, 2 * G, 1, big, big_floats, done));
+    k_blk_leave_d<<<(unsigned)((G * G + 7) / 8), 256, 0, st>>>(p, bp);
     k_blk_finish_d<<<(unsigned)(((L.nJ + G) * G + 255) / 256), 256, 0, st>>>(p, bp);            mark();
     // the three rank-2G updates; the residual rows of the leaving groups go through the Rq panel
-    BK(sgemm(st, true, false, L.nI, L.nI, 2 * G, -1.f, bp.PA, L.ldh, bp.PB, L.ldh, 1.f, p.Hinv, L.ldh, done));   mark();
-    BK(sgemm(st, true, false, L.nI, L.m, 2 * G, -1.f, bp.PB, L.ldh, bp.KV, L.ldm, 1.f, p.V, L.ldm, done));        mark();
-    BK(sgemm(st, false, false, L.nJ, L.m, 2 * G, 1.f, bp.UD, 2 * G, bp.KV, L.ldm, 1.f, p.R, L.ldm, done));
+    void* tc = (char*)ctx->ws + L.off_tc;
+    int32_t* stat = &ctx->ctl->status;
+    BK(gemm_tc(st, L.nI, L.ldh, 2 * G, -1.f, bp.PAT, 2 * G, bp.PB, L.ldh, 1.f, p.Hinv, L.ldh, tc, L.tc_bytes, stat, done));   mark();
+    BK(gemm_tc(st, L.nI, L.m, 2 * G, -1.f, bp.PBT, 2 * G, bp.KV, L.ldm, 1.f, p.V, L.ldm, tc, L.tc_bytes, stat, done));        mark();
+    BK(gemm_tc(st, L.nJ, L.m, 2 * G, 1.f, bp.UD, 2 * G, bp.KV, L.ldm, 1.f, p.R, L.ldm, tc, L.tc_bytes, stat, done));
     BK(sgemm(st, false, false, G, L.m, 2 * G, 1.f, bp.UD + L.nJ * 2 * G, 2 * G, bp.KV, L.ldm, 0.f, bp.Rq, L.ldm, done));   mark();
     k_blk_update_c<<<(unsigned)(L.ng - L.k), 128, 2 * (size_t)L.g * G * sizeof(double), st>>>(p, bp);
     k_blk_fix<<<(unsigned)G, 256, 0, st>>>(p, bp);                                              mark();
     k_blk_hswap<<<(unsigned)((L.ldp * G + 255) / 256), 256, 0, st>>>(p, bp, 0);
     k_blk_hswap<<<(unsigned)((L.ldp * G + 255) / 256), 256, 0, st>>>(p, bp, 1);                 mark();
-    count_launches(10);
+    count_launches(11);
     BK(enqueue_scores(ctx, p, true, false));                                                   mark();
 #undef BK
     return cudaGetLastError();

@@ -358,13 +358,7 @@ int make_layout(int64_t d1, int64_t m, int32_t g, int32_t k, Layout* L)
         if (nJ < G) G = nJ;
         G = G / g * g;
         L->block_rows_max = (int32_t)G;
-        auto al = [](size_t b) { return (b + 255) / 256 * 256; };
-        size_t n = 256;
-        if (G > 0) {
-            n = 2 * al(sizeof(int32_t) * (size_t)G) + 3 * al(sizeof(float) * (size_t)G * ldh) + 2 * al(sizeof(float) * 2 * (size_t)G * ldh)
-              + al(sizeof(float) * 2 * (size_t)G * ldm) + 2 * al(sizeof(float) * (size_t)G * ldm)
-              + al(sizeof(float) * (size_t)(nJ + G) * 2 * G) + al(sizeof(double) * 18 * (size_t)G * G);
-        }
+        const size_t n = G > 0 ? block_region_bytes(ldh, ldm, nJ, G) : 256;
         L->block_bytes = n;
         L->off_block = take(n);
     }
