@@ -222,6 +222,15 @@ k_mma_pipe(const __grid_constant__ Maps maps, int64_t M, int64_t N, int64_t K, f
             float acc[128];
 #pragma unroll
             for (int j = 0; j < 128; ++j) acc[j] = 0.f;
+            if (beta != 0.f) {      // bring this thread's part of the old C row towards L2 while the tile is computed
+                const int64_t prow = (int64_t)tm * TILE_M + lg * 32 + lane;
+                const int64_t pcol = (int64_t)tn * TILE_N + half * 128;
+                if (prow < M) {
+#pragma unroll
+                    for (int j = 0; j < 128; j += 32)
+                        if (pcol + j < N) asm volatile("prefetch.global.L2 [%0];" ::"l"(C + prow * ldc + pcol + j));
+                }
+            }
             for (int f = 0; f < nflush && ok; ++f, ++fl) {
                 const int buf = fl & 1;
                 if (!mbar_wait(tfull_bar(buf), (fl >> 1) & 1, abort_flag)) { ok = false; break; }

@@ -108,6 +108,13 @@ cudaError_t panel_dot(cudaStream_t st, int64_t M, int64_t N, int64_t K, const fl
                       const float* P, int64_t ldp, float* Y, int64_t so_row, int64_t so_col,
                       float* scratch, size_t scratch_floats, const int32_t* done = nullptr);
 
+// ---- panel_tc.cu: the same product on the tensor cores; A is split into bf16 terms on the way (fp32-accurate) -------
+// A 16-byte aligned with lda % 4 == 0; scratch at least panel_dot_tc_scratch bytes.
+size_t panel_dot_tc_scratch(int64_t M, int64_t N, int64_t K);
+cudaError_t panel_dot_tc(cudaStream_t st, int64_t M, int64_t N, int64_t K, const float* A, int64_t lda,
+                         const float* P, int64_t ldp, float* Y, int64_t so_row, int64_t so_col,
+                         void* scratch, size_t scratch_bytes, int32_t* status_dev, const int32_t* done = nullptr);
+
 // ---- gemm_tc.cu: the same product on the tensor cores (three-term bf16 split, fp32-accurate); A and B row-major.
 // `scratch` (256-byte aligned device memory, at least gemm_tc_min_scratch bytes) holds the bf16 terms of one K panel.
 size_t gemm_tc_min_scratch(int64_t M, int64_t N);

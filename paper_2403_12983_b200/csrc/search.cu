@@ -823,6 +823,9 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
         CK(cudaMemsetAsync((char*)ctx->ws + L.off_block, 0, block_bytes_for(L, bs * g), st));
         const size_t smem = 2 * (size_t)g * bs * g * sizeof(double);
         if (smem > 48 * 1024) CK(cudaFuncSetAttribute(k_blk_update_c, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        const size_t smem2 = 2 * (size_t)bs * g * bs * g * sizeof(double);
+        if (smem2 > 48 * 1024) CK(cudaFuncSetAttribute(k_blk_small, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2));
+        if (smem2 / 2 > 48 * 1024) CK(cudaFuncSetAttribute(k_blk_update_c_g1, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(smem2 / 2)));
     }
     if (g > 1) CK(cudaFuncSetAttribute(k_update_c, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(2 * (size_t)g * g * sizeof(double))));
     const int batch = 32;

@@ -178,6 +178,26 @@ __global__ void __launch_bounds__(256) k_blk_gram(Ptrs p, BlockPtrs bp)
     if (lane == 0) bp.small[(int64_t)slot * G * G + a * G + b] = (double)s0;
 }
 
+// C = op(A) * op(B) (G x G, fp64) with both operands staged in shared memory (2 G^2 doubles at `sm`).
+__device__ void blk_mat_mul(const double* A, bool tA, const double* B, bool tB, double* C, int g, double* sm)
+{
+    const int gg = g * g;
+    __syncthreads();
+    for (int idx = threadIdx.x; idx < gg; idx += blockDim.x) { sm[idx] = A[idx]; sm[gg + idx] = B[idx]; }
+    __syncthreads();
+    const double* As = sm; const double* Bs = sm + gg;
+    for (int idx = threadIdx.x; idx < gg; idx += blockDim.x) {
+        const int i = idx / g, j = idx % g;
+        double s = 0.0;
+        if (!tA && !tB)     for (int kx = 0; kx < g; ++kx) s += As[i * g + kx] * Bs[kx * g + j];
+        else if (!tA && tB) for (int kx = 0; kx < g; ++kx) s += As[i * g + kx] * Bs[j * g + kx];
+        else if (tA && !tB) for (int kx = 0; kx < g; ++kx) s += As[kx * g + i] * Bs[kx * g + j];
+        else                for (int kx = 0; kx < g; ++kx) s += As[kx * g + i] * Bs[j * g + kx];
+        C[idx] = s;
+    }
+    __syncthreads();
+}
+
 // One block: the G x G algebra of the exchange, its exact change of obj and the accept decision.
 __global__ void __launch_bounds__(1024)
 k_blk_small(Ptrs p, BlockPtrs bp, int accept_mode, double accept_tol, double* __restrict__ obj_trace, int32_t* __restrict__ swap_trace)
@@ -185,6 +205,7 @@ k_blk_small(Ptrs p, BlockPtrs bp, int accept_mode, double accept_tol, double* __
     SearchCtl* ctl = p.ctl;
     if (ctl->done) return;
     __shared__ double red[32];
+    extern __shared__ double smw[];          // 2 G^2 doubles: the matrix being factorised and its work array
     const int g = bp.G, gg = g * g;
     double* S = bp.small;
     double *Cinv = S + S_CINV * gg, *c1inv = S + S_C1INV * gg, *Q1 = S + S_Q1 * gg, *Q1c = S + S_Q1C * gg, *M2 = S + S_M2 * gg;
@@ -200,19 +221,21 @@ k_blk_small(Ptrs p, BlockPtrs bp, int accept_mode, double accept_tol, double* __
         cq[idx] = (double)p.Hp[qi * p.ldp + qj] - 0.5 * (HY[idx] + HY[j * g + i]);
     }
     __syncthreads();
-    const double pivC = chol_inverse(C, Lw, Cinv, g);
+    for (int idx = threadIdx.x; idx < gg; idx += blockDim.x) smw[idx] = C[idx];
+    __syncthreads();
+    const double pivC = chol_inverse(smw, smw + gg, Cinv, g);
     const double Ds = mat_trace_prod(Cinv, GV, g, red);               // Tr(C^-1 V_r V_r^T)
-    mat_mul(Cinv, false, GX, false, T1, g);                           // K R_q^T
-    mat_mul(P, false, T1, false, T2, g);                              // P K R_q^T
-    mat_mul(P, false, Cinv, false, T1, g);                            // P Cinv
-    mat_mul(T1, false, GV, false, T3, g);                             // P Cinv GV
-    mat_mul(T3, false, T1, true, Lw, g);                              // P Cinv GV Cinv P^T
+    blk_mat_mul(Cinv, false, GX, false, T1, g, smw);                           // K R_q^T
+    blk_mat_mul(P, false, T1, false, T2, g, smw);                              // P K R_q^T
+    blk_mat_mul(P, false, Cinv, false, T1, g, smw);                            // P Cinv
+    blk_mat_mul(T1, false, GV, false, T3, g, smw);                             // P Cinv GV
+    blk_mat_mul(T3, false, T1, true, Lw, g, smw);                              // P Cinv GV Cinv P^T
     for (int idx = threadIdx.x; idx < gg; idx += blockDim.x) {
         const int i = idx / g, j = idx % g;
         T3[idx] = GR[idx] + T2[idx] + T2[j * g + i] + Lw[idx];        // R1 R1^T
     }
     __syncthreads();
-    mat_mul(T1, false, P, true, T2, g);                               // P Cinv P^T
+    blk_mat_mul(T1, false, P, true, T2, g, smw);                               // P Cinv P^T
     for (int idx = threadIdx.x; idx < gg; idx += blockDim.x) {
         const int i = idx / g, j = idx % g;
         c1[idx] = cq[idx] + 0.5 * (T2[idx] + T2[j * g + i]);
@@ -220,30 +243,43 @@ k_blk_small(Ptrs p, BlockPtrs bp, int accept_mode, double accept_tol, double* __
     __syncthreads();
     // the smallest pivot of c1 is compared with the diagonal of H on the entering rows (eligibility of the joint add)
     double scale = 0.0;
-    for (int i = 0; i < g; ++i) {
-        const int64_t qi = p.nI + blk_qrow(p, bp, i);
-        const double hd = p.Hp[qi * p.ldp + qi];
-        if (hd > scale) scale = hd;
+    {
+        double hd = 0.0;
+        for (int i = threadIdx.x; i < g; i += blockDim.x) {
+            const int64_t qi = p.nI + blk_qrow(p, bp, i);
+            hd = fmax(hd, (double)p.Hp[qi * p.ldp + qi]);
+        }
+        for (int o = 16; o > 0; o >>= 1) hd = fmax(hd, __shfl_xor_sync(0xffffffffu, hd, o));
+        __syncthreads();
+        if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = hd;
+        __syncthreads();
+        for (int i = 0; i < (int)(blockDim.x >> 5); ++i) scale = fmax(scale, red[i]);
+        __syncthreads();
     }
-    const double pivc1 = chol_inverse(c1, Lw, c1inv, g);
+    for (int idx = threadIdx.x; idx < gg; idx += blockDim.x) smw[idx] = c1[idx];
+    __syncthreads();
+    const double pivc1 = chol_inverse(smw, smw + gg, c1inv, g);
     const double gain = mat_trace_prod(c1inv, T3, g, red);
     const double delta = Ds - gain;
-    mat_mul(Cinv, false, P, true, Q1, g);                             // Q1 = Cinv P^T
-    mat_mul(Q1, false, c1inv, false, Q1c, g);                         // Q1 c1inv
-    mat_mul(c1inv, false, T1, false, M2, g);                          // c1inv P Cinv
+    blk_mat_mul(Cinv, false, P, true, Q1, g, smw);                             // Q1 = Cinv P^T
+    blk_mat_mul(Q1, false, c1inv, false, Q1c, g, smw);                         // Q1 c1inv
+    blk_mat_mul(c1inv, false, T1, false, M2, g, smw);                          // c1inv P Cinv
+    const double obj = ctl->obj;
+    const int n = ctl->n_swaps;
+    bool stop = false; int reason = 0;
+    if (!(pivC > 0.0) || !(pivc1 > kAddPivotTol * scale) || !isfinite(delta)) { stop = true; reason = OSSCAR_STOP_GUARD; }
+    else if (accept_mode == OSSCAR_ACCEPT_IMPROVING && !(delta <= -accept_tol * obj)) { stop = true; reason = OSSCAR_STOP_NO_IMPROVEMENT; }
+    if (!stop) {
+        for (int t = threadIdx.x; t < bp.s; t += blockDim.x) {
+            swap_trace[2 * (n + t)] = p.perm[bp.rslot[t]];
+            swap_trace[2 * (n + t) + 1] = p.perm[p.k + bp.tslot[t]];
+        }
+    }
+    __syncthreads();                     // every thread has read obj and n_swaps
     if (threadIdx.x == 0) {
-        const double obj = ctl->obj;
-        bool stop = false; int reason = 0;
-        if (!(pivC > 0.0) || !(pivc1 > kAddPivotTol * scale) || !isfinite(delta)) { stop = true; reason = OSSCAR_STOP_GUARD; }
-        else if (accept_mode == OSSCAR_ACCEPT_IMPROVING && !(delta <= -accept_tol * obj)) { stop = true; reason = OSSCAR_STOP_NO_IMPROVEMENT; }
         ctl->delta = delta;
         if (stop) { ctl->done = 1; ctl->stop_reason = reason; *p.done_host = 1; }
         else {
-            const int n = ctl->n_swaps;
-            for (int t = 0; t < bp.s; ++t) {
-                swap_trace[2 * (n + t)] = p.perm[bp.rslot[t]];
-                swap_trace[2 * (n + t) + 1] = p.perm[p.k + bp.tslot[t]];
-            }
             obj_trace[n / bp.s + 1] = obj + delta;
             ctl->obj = obj + delta;
             ctl->n_swaps = n + bp.s;
@@ -272,11 +308,8 @@ __global__ void __launch_bounds__(256) k_blk_prep(Ptrs p, BlockPtrs bp)
                     bqc += bf * Q1c[f * G + e];
                     yc += (double)bp.yT[(int64_t)f * p.ldh + i] * c1inv[f * G + e];
                 }
-                bool in_r = false;
-                const int slot = (int)(i / p.g);
-                for (int t = 0; t < bp.s; ++t) in_r |= bp.rslot[t] == slot;
-                vbc = (float)bc;
-                if (!in_r) { vu2 = (float)((double)bp.yT[(int64_t)e * p.ldh + i] - bq); vnu = (float)(bqc - yc); }
+                vbc = (float)bc;                 // the entries of u2 on the leaving rows are cleared by k_blk_zero_r
+                vu2 = (float)((double)bp.yT[(int64_t)e * p.ldh + i] - bq); vnu = (float)(bqc - yc);
             }
             bp.PA[(int64_t)e * p.ldh + i] = vbc;
             bp.PB[(int64_t)(G + e) * p.ldh + i] = vu2;
@@ -301,6 +334,24 @@ __global__ void __launch_bounds__(256) k_blk_prep(Ptrs p, BlockPtrs bp)
             bp.KV[(int64_t)(G + e) * p.ldm + c] = (float)vq;
         }
     }
+}
+
+// u2 vanishes on the leaving rows (y_r - C C^-1 y_r = 0): make the zeros exact, and put the block c1^-1 there in
+// the -u2 c1^-1 panel.  G x G entries.
+__global__ void __launch_bounds__(256) k_blk_zero_r(Ptrs p, BlockPtrs bp)
+{
+    if (p.ctl->done) return;
+    const int G = bp.G;
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= G * G) return;
+    const int e = idx / G, a = idx % G;
+    const int64_t i = blk_rrow(p, bp, a);
+    const double* c1inv = bp.small + (int64_t)S_C1INV * G * G;
+    bp.PB[(int64_t)(G + e) * p.ldh + i] = 0.f;
+    // this row of PA doubles as the new rows / columns r of Hinv (k_blk_fix): -u2 c1^-1 off r, c1^-1 on r
+    bp.PA[(int64_t)(G + e) * p.ldh + i] = (float)(0.5 * (c1inv[a * G + e] + c1inv[e * G + a]));
+    bp.PBT[i * 2 * G + G + e] = 0.f;
+    bp.PAT[i * 2 * G + G + e] = 0.f;
 }
 
 // H pass of the G leaving rows: UD[n_J + a][G + e] = Hp[r_a, 0:n_I] . u2_e, one warp per entry.
@@ -349,14 +400,10 @@ __global__ void __launch_bounds__(256) k_blk_fix(Ptrs p, BlockPtrs bp)
 {
     if (p.ctl->done) return;
     const int G = bp.G, t = blockIdx.x;
-    const double* c1inv = bp.small + (int64_t)S_C1INV * G * G;
     const int64_t row = blk_rrow(p, bp, t), qrow = blk_qrow(p, bp, t);
     const float* nu = bp.PA + (int64_t)(G + t) * p.ldh;
-    for (int64_t i = threadIdx.x; i < p.nI; i += blockDim.x) {
-        float v = nu[i];
-        const int slot = (int)(i / p.g);
-        for (int a = 0; a < bp.s; ++a)
-            if (bp.rslot[a] == slot) { const int ea = a * p.g + (int)(i % p.g); v = (float)(0.5 * (c1inv[ea * G + t] + c1inv[t * G + ea])); }
+    for (int64_t i = threadIdx.x; i < p.nI; i += blockDim.x) {       // on the leaving rows the panel holds c1^-1 (symmetric)
+        const float v = nu[i];
         p.Hinv[i * p.ldh + row] = v;
         p.Hinv[row * p.ldh + i] = v;
     }
@@ -399,6 +446,50 @@ __global__ void __launch_bounds__(128) k_blk_update_c(Ptrs p, BlockPtrs bp)
         for (int f = 0; f < G; ++f)
             s += TU[a * G + f] * (double)ud[b2 * 2 * G + f] - TD[a * G + f] * (double)ud[b2 * 2 * G + G + f];
         p.c[t * g * g + idx] = s;
+    }
+}
+
+// Single-row groups: c_l' = c_l + u_l C^-1 u_l^T - d_l c1^-1 d_l^T, one warp per four pruned rows; C^-1 and c1^-1
+// sit in shared memory as fp32 (u and d are fp32 values already) and the sums run in fp32, the update of c in fp64.
+__global__ void __launch_bounds__(256) k_blk_update_c_g1(Ptrs p, BlockPtrs bp)
+{
+    if (p.ctl->done) return;
+    extern __shared__ float smf[];
+    const int G = bp.G, gg = G * G;
+    float* Ci = smf; float* c1i = smf + gg;
+    for (int idx = threadIdx.x; idx < gg; idx += blockDim.x) {
+        Ci[idx] = (float)bp.small[(int64_t)S_CINV * gg + idx];
+        c1i[idx] = (float)bp.small[(int64_t)S_C1INV * gg + idx];
+    }
+    __syncthreads();
+    const int lane = threadIdx.x & 31;
+    const int64_t nw = (int64_t)gridDim.x * (blockDim.x >> 5);
+    for (int64_t t0 = ((int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * 4; t0 < p.nJ; t0 += nw * 4) {
+        const float* ud[4]; bool enter[4];
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            const int64_t t = t0 + r < p.nJ ? t0 + r : p.nJ - 1;
+            int pos = -1;
+            for (int a = 0; a < bp.s; ++a) if (bp.tslot[a] == t) pos = a;
+            enter[r] = pos >= 0;
+            ud[r] = bp.UD + (pos >= 0 ? p.nJ + pos : t) * 2 * G;
+        }
+        float s[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int e = lane; e < G; e += 32) {
+            float tu[4] = {0.f, 0.f, 0.f, 0.f}, td[4] = {0.f, 0.f, 0.f, 0.f};
+            for (int f = 0; f < G; ++f) {
+                const float ci = Ci[f * G + e], c1 = c1i[f * G + e];
+#pragma unroll
+                for (int r = 0; r < 4; ++r) { tu[r] = fmaf(ud[r][f], ci, tu[r]); td[r] = fmaf(ud[r][G + f], c1, td[r]); }
+            }
+#pragma unroll
+            for (int r = 0; r < 4; ++r) s[r] += tu[r] * ud[r][e] - td[r] * ud[r][G + e];
+        }
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            const float v = warp_sum(s[r]);
+            if (lane == 0 && t0 + r < p.nJ) p.c[t0 + r] = (enter[r] ? 0.0 : p.c[t0 + r]) + (double)v;
+        }
     }
 }
 
@@ -446,26 +537,31 @@ cudaError_t enqueue_block_step(osscar_ctx* ctx, const Ptrs& p, const BlockPtrs& 
     k_blk_gather<<<dim3((unsigned)G, 5), 256, 0, st>>>(p, bp);
     float* big = (float*)((char*)ctx->ws + L.off_big);          // free between refreshes: partial sums of split products
     const size_t big_floats = (L.off_Hp - L.off_big) / sizeof(float);
-    BK(panel_dot(st, L.nI, G, L.nI, p.Hinv, L.ldh, bp.hT, L.ldh, bp.yT, 1, L.ldh, big, big_floats, done));     mark();   // y^T (Hinv symmetric)
+    void* tc = (char*)ctx->ws + L.off_tc;
+    int32_t* stat = &ctx->ctl->status;
+    const bool use_tc = L.tc_bytes >= panel_dot_tc_scratch(L.nJ > L.nI ? L.nJ : L.nI, 2 * G, L.nI);
+    if (use_tc) BK(panel_dot_tc(st, L.nI, G, L.nI, p.Hinv, L.ldh, bp.hT, L.ldh, bp.yT, 1, L.ldh, tc, L.tc_bytes, stat, done));
+    else BK(panel_dot(st, L.nI, G, L.nI, p.Hinv, L.ldh, bp.hT, L.ldh, bp.yT, 1, L.ldh, big, big_floats, done));     mark();   // y^T (Hinv symmetric)
     k_blk_gram<<<(unsigned)((4 * G * G + 7) / 8), 256, 0, st>>>(p, bp);
-    k_blk_small<<<1, 1024, 0, st>>>(p, bp, accept_mode, tol, obj_trace, swap_trace);
-    k_blk_prep<<<(unsigned)(((L.ldh + L.ldm) * G + 255) / 256), 256, 0, st>>>(p, bp);           mark();
+    k_blk_small<<<1, 1024, 2 * (size_t)G * G * sizeof(double), st>>>(p, bp, accept_mode, tol, obj_trace, swap_trace);
+    k_blk_prep<<<(unsigned)(((L.ldh + L.ldm) * G + 255) / 256), 256, 0, st>>>(p, bp);
+    k_blk_zero_r<<<(unsigned)((G * G + 255) / 256), 256, 0, st>>>(p, bp);                        mark();
     // H pass: [u | H u2] for the pruned rows and the leaving rows, then -d
-    BK(panel_dot(st, L.nJ, 2 * G, L.nI, p.Hp + L.nI * L.ldp, L.ldp, bp.PB, L.ldh, bp.UD, 2 * G, 1, big, big_floats, done));
+    if (use_tc) BK(panel_dot_tc(st, L.nJ, 2 * G, L.nI, p.Hp + L.nI * L.ldp, L.ldp, bp.PB, L.ldh, bp.UD, 2 * G, 1, tc, L.tc_bytes, stat, done));
+    else BK(panel_dot(st, L.nJ, 2 * G, L.nI, p.Hp + L.nI * L.ldp, L.ldp, bp.PB, L.ldh, bp.UD, 2 * G, 1, big, big_floats, done));
     k_blk_leave_d<<<(unsigned)((G * G + 7) / 8), 256, 0, st>>>(p, bp);
     k_blk_finish_d<<<(unsigned)(((L.nJ + G) * G + 255) / 256), 256, 0, st>>>(p, bp);            mark();
     // the three rank-2G updates; the residual rows of the leaving groups go through the Rq panel
-    void* tc = (char*)ctx->ws + L.off_tc;
-    int32_t* stat = &ctx->ctl->status;
     BK(gemm_tc(st, L.nI, L.ldh, 2 * G, -1.f, bp.PAT, 2 * G, bp.PB, L.ldh, 1.f, p.Hinv, L.ldh, tc, L.tc_bytes, stat, done));   mark();
     BK(gemm_tc(st, L.nI, L.m, 2 * G, -1.f, bp.PBT, 2 * G, bp.KV, L.ldm, 1.f, p.V, L.ldm, tc, L.tc_bytes, stat, done));        mark();
     BK(gemm_tc(st, L.nJ, L.m, 2 * G, 1.f, bp.UD, 2 * G, bp.KV, L.ldm, 1.f, p.R, L.ldm, tc, L.tc_bytes, stat, done));
     BK(sgemm(st, false, false, G, L.m, 2 * G, 1.f, bp.UD + L.nJ * 2 * G, 2 * G, bp.KV, L.ldm, 0.f, bp.Rq, L.ldm, done));   mark();
-    k_blk_update_c<<<(unsigned)(L.ng - L.k), 128, 2 * (size_t)L.g * G * sizeof(double), st>>>(p, bp);
+    if (L.g == 1) k_blk_update_c_g1<<<296, 256, 2 * (size_t)G * G * sizeof(float), st>>>(p, bp);
+    else k_blk_update_c<<<(unsigned)(L.ng - L.k), 128, 2 * (size_t)L.g * G * sizeof(double), st>>>(p, bp);
     k_blk_fix<<<(unsigned)G, 256, 0, st>>>(p, bp);                                              mark();
     k_blk_hswap<<<(unsigned)((L.ldp * G + 255) / 256), 256, 0, st>>>(p, bp, 0);
     k_blk_hswap<<<(unsigned)((L.ldp * G + 255) / 256), 256, 0, st>>>(p, bp, 1);                 mark();
-    count_launches(11);
+    count_launches(12);
     BK(enqueue_scores(ctx, p, true, false));                                                   mark();
 #undef BK
     return cudaGetLastError();

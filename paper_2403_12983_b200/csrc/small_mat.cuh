@@ -16,45 +16,40 @@ static __device__ __forceinline__ double warp_sum(double v) {
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
     return v;
 }
-// Block-cooperative Cholesky inverse of the g x g SPD matrix M (ld g, overwritten by its factor).
-// Lw, Out: g x g work / result.  Returns the smallest pivot (<= 0 when not positive definite).
+// Block-cooperative inverse of the g x g SPD matrix M (ld g) by in-place Gauss-Jordan elimination without pivoting:
+// g steps of one rank-1 update over all g^2 entries, so every thread of the block works in every step.
+// M is overwritten (keep it in shared memory where possible); Out receives the symmetrised inverse; Lw: scratch of
+// at least 2 g doubles.  Returns the smallest pivot, i.e. the smallest diagonal entry of the successive Schur
+// complements = the squared diagonal of the Cholesky factor (<= 0 when M is not positive definite).
 static __device__ double chol_inverse(double* M, double* Lw, double* Out, int g)
 {
     __shared__ double minpiv;
     const int t = threadIdx.x, nt = blockDim.x;
+    double* colj = Lw; double* rowj = Lw + g;
+    __syncthreads();
     if (t == 0) minpiv = DBL_MAX;
     __syncthreads();
     for (int j = 0; j < g; ++j) {
-        if (t == 0) {
-            double dd = M[j * g + j];
-            if (dd < minpiv) minpiv = dd;
-            if (!(dd > 0.0)) { minpiv = -1.0; dd = 1.0; }
-            M[j * g + j] = sqrt(dd);
-        }
+        double d = M[j * g + j];
+        const bool bad = !(d > 0.0);
+        if (t == 0) { if (bad) minpiv = -1.0; else if (d < minpiv) minpiv = d; }
+        if (bad) d = 1.0;
+        const double pinv = 1.0 / d;
+        for (int i = t; i < g; i += nt) { colj[i] = M[i * g + j]; rowj[i] = M[j * g + i] * pinv; }
         __syncthreads();
-        const double djj = M[j * g + j];
-        for (int i = j + 1 + t; i < g; i += nt) M[i * g + j] /= djj;
-        __syncthreads();
-        const int rem = g - j - 1;
-        for (int idx = t; idx < rem * rem; idx += nt) {
-            const int i = j + 1 + idx / rem, c = j + 1 + idx % rem;
-            if (c <= i) M[i * g + c] -= M[i * g + j] * M[c * g + j];
+        for (int idx = t; idx < g * g; idx += nt) {
+            const int i = idx / g, c = idx % g;
+            double v;
+            if (i == j) v = (c == j) ? pinv : rowj[c];
+            else if (c == j) v = -colj[i] * pinv;
+            else v = M[idx] - colj[i] * rowj[c];
+            M[idx] = v;
         }
         __syncthreads();
     }
-    for (int c = t; c < g; c += nt) {
-        for (int i = 0; i < g; ++i) {
-            double s = (i == c) ? 1.0 : 0.0;
-            for (int kx = c; kx < i; ++kx) s -= M[i * g + kx] * Lw[kx * g + c];
-            Lw[i * g + c] = (i < c) ? 0.0 : s / M[i * g + i];
-        }
-    }
-    __syncthreads();
-    for (int idx = t; idx < g * g; idx += nt) {
-        const int i = idx / g, j = idx % g;
-        double s = 0.0;
-        for (int kx = (i > j ? i : j); kx < g; ++kx) s += Lw[kx * g + i] * Lw[kx * g + j];
-        Out[idx] = s;
+    for (int idx = t; idx < g * g; idx += nt) {          // the two triangles differ by rounding only
+        const int i = idx / g, c = idx % g;
+        Out[idx] = 0.5 * (M[idx] + M[c * g + i]);
     }
     __syncthreads();
     return minpiv;
