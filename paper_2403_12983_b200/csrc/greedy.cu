@@ -25,6 +25,7 @@ struct GPtrs {
     float* B;                       // T x lda: rows r of A (= columns, A symmetric)
     float* BC;                      // T x lda: C^-1 B
     float* KT;                      // T x ldv: C^-1 V_r
+    float* BCT; float* BT;          // n x T: transposes of BC and B (left operands of the tensor-core downdates)
     double* gram;                   // ngroups x g x g
     double* D;                      // ngroups
     double* Cm;                     // 3 x T x T doubles: C, work, C^-1
@@ -103,12 +104,19 @@ __global__ void __launch_bounds__(1024) k_gr_select(GPtrs p, int n_live, int t, 
     __shared__ double sv[32]; __shared__ int sid[32], sidx[32];
     __shared__ int chosen[kMaxT];
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
-    for (int round = 0; round < t; ++round) {
-        double best = INFINITY; int bid = INT_MAX, bidx = -1;
+    // every thread keeps the best of its own strided share; only the owner of a round's winner rescans its share
+    double mine = INFINITY; int mid = INT_MAX, midx = -1;
+    auto rescan = [&]() {
+        mine = INFINITY; mid = INT_MAX; midx = -1;
         for (int i = tid; i < n_live; i += blockDim.x) {
             const double v = p.D[i]; const int id = p.perm[i];
-            if (v < best || (v == best && id < bid)) { best = v; bid = id; bidx = i; }
+            if (v < mine || (v == mine && id < mid)) { mine = v; mid = id; midx = i; }
         }
+    };
+    rescan();
+    __shared__ int winner;
+    for (int round = 0; round < t; ++round) {
+        double best = mine; int bid = mid, bidx = midx;
         for (int o = 16; o > 0; o >>= 1) {
             const double ov = __shfl_xor_sync(0xffffffffu, best, o);
             const int oid = __shfl_xor_sync(0xffffffffu, bid, o), oidx = __shfl_xor_sync(0xffffffffu, bidx, o);
@@ -124,8 +132,10 @@ __global__ void __launch_bounds__(1024) k_gr_select(GPtrs p, int n_live, int t, 
             chosen[round] = bidx;
             if (p.drop_trace) p.drop_trace[trace_pos + round] = p.perm[bidx];
             p.D[bidx] = INFINITY;                 // not again in this iteration
+            winner = bidx;
         }
         __syncthreads();
+        if (winner % (int)blockDim.x == tid) rescan();
     }
     if (tid == 0) {
         // refill plan: the new live range is [0, n_new); every chosen slot below n_new is a hole, every slot of
@@ -159,10 +169,11 @@ __global__ void k_gr_stage_b(GPtrs p, int n_live)
     const int64_t n = (int64_t)n_live * g;
     for (int64_t c = threadIdx.x; c < p.lda; c += blockDim.x) p.B[(int64_t)e * p.lda + c] = c < n ? p.A[r * p.lda + c] : 0.f;
 }
-__global__ void __launch_bounds__(256) k_gr_cinv(GPtrs p)
+__global__ void __launch_bounds__(1024) k_gr_cinv(GPtrs p, int in_smem)
 {
+    extern __shared__ double smg[];           // T^2 + 2 T doubles when the matrix fits
     const int g = p.g, t = p.sel[0], T = t * g;
-    double* C = p.Cm; double* Lw = p.Cm + kMaxT * kMaxT; double* Cinv = p.Cm + 2 * kMaxT * kMaxT;
+    double* C = in_smem ? smg : p.Cm; double* Lw = in_smem ? smg + T * T : p.Cm + kMaxT * kMaxT; double* Cinv = p.Cm + 2 * kMaxT * kMaxT;
     for (int idx = threadIdx.x; idx < T * T; idx += blockDim.x) {
         const int a = idx / T, b = idx % T;
         const int64_t ra = (int64_t)p.sel[1 + a / g] * g + a % g, rb = (int64_t)p.sel[1 + b / g] * g + b % g;
@@ -184,6 +195,7 @@ __global__ void k_gr_stage_bc(GPtrs p, int n_live)
             double acc = 0.0;
             for (int f = 0; f < T; ++f) acc += Cinv[e * T + f] * (double)p.B[(int64_t)f * p.lda + s];
             p.BC[idx] = (float)acc;
+            if (s < (int64_t)n_live * g) { p.BCT[s * T + e] = (float)acc; p.BT[s * T + e] = p.B[(int64_t)e * p.lda + s]; }
         } else {
             const int64_t j = idx - nA;
             const int e = (int)(j / p.ldv); const int64_t c = j % p.ldv;
@@ -196,12 +208,12 @@ __global__ void k_gr_stage_bc(GPtrs p, int n_live)
         }
     }
 }
-__global__ void __launch_bounds__(1024) k_gr_obj(GPtrs p)
+__global__ void __launch_bounds__(256) k_gr_obj(GPtrs p, double* __restrict__ partial)
 {
     __shared__ double red[32];
     const int g = p.g, t = p.sel[0], T = t * g;
     double acc = 0.0;
-    for (int64_t idx = threadIdx.x; idx < (int64_t)T * p.ldv; idx += blockDim.x) {
+    for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < (int64_t)T * p.ldv; idx += (int64_t)gridDim.x * blockDim.x) {
         const int e = (int)(idx / p.ldv); const int64_t c = idx % p.ldv;
         const int64_t re = (int64_t)p.sel[1 + e / g] * g + e % g;
         acc += (double)p.KT[idx] * (double)p.V[re * p.ldv + c];
@@ -209,7 +221,13 @@ __global__ void __launch_bounds__(1024) k_gr_obj(GPtrs p)
     acc = warp_sum(acc);
     if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = acc;
     __syncthreads();
-    if (threadIdx.x == 0) { double s = 0.0; for (int i = 0; i < 32; ++i) s += red[i]; p.ctl->obj += s; }
+    if (threadIdx.x == 0) { double s = 0.0; for (int i = 0; i < (int)(blockDim.x >> 5); ++i) s += red[i]; partial[blockIdx.x] = s; }
+}
+__global__ void k_gr_obj_add(SearchCtl* ctl, const double* __restrict__ partial, int n)
+{
+    double s = 0.0;
+    for (int i = 0; i < n; ++i) s += partial[i];      // fixed order
+    ctl->obj += s;
 }
 
 // M[s][c] -= sum_e left[e][s] * right[e][c] for live rows s and columns c < ncols (M = A with right = B, or
@@ -333,12 +351,13 @@ int greedy_support(osscar_ctx* ctx, int t_hat, int32_t* support, int32_t* drop_t
     // scratch carved from `big` (2 d1 ldm floats at least): V of all rows, then B, BC (T x ldp each), KT (T x ldm)
     float* big = (float*)(ws + L.off_big);
     const size_t big_floats = (L.off_Hp - L.off_big) / sizeof(float);
-    const size_t need = (size_t)d1 * L.ldm + 2 * (size_t)T * L.ldp + (size_t)T * L.ldm;
+    const size_t need = (size_t)d1 * L.ldm + 2 * (size_t)T * L.ldp + (size_t)T * L.ldm + 2 * (size_t)d1 * T;
     if (need > big_floats) return OSSCAR_E_WORKSPACE;
     GPtrs p;
     p.A = (float*)(ws + L.off_Hp); p.lda = L.ldp;
     p.V = big; p.ldv = L.ldm; p.m = L.m;
     p.B = big + (size_t)d1 * L.ldm; p.BC = p.B + (size_t)T * L.ldp; p.KT = p.BC + (size_t)T * L.ldp;
+    p.BCT = p.KT + (size_t)T * L.ldm; p.BT = p.BCT + (size_t)d1 * T;
     char* gs = ws + L.off_greedy;
     p.gram = (double*)gs; p.D = p.gram + ng * g * g; p.Cm = p.D + ng;
     p.sel = (int32_t*)(p.Cm + 3 * kMaxT * kMaxT);
@@ -364,6 +383,7 @@ int greedy_support(osscar_ctx* ctx, int t_hat, int32_t* support, int32_t* drop_t
 
     const size_t smem_score = 3 * (size_t)g * g * sizeof(double);
     CK(cudaFuncSetAttribute(k_gr_score, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_score));
+    CK(cudaFuncSetAttribute(k_gr_cinv, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
     int n_live = (int)ng, iters = 0, trace_pos = 0;
     while (n_live > L.k) {
         const int t = n_live - L.k < t_hat ? n_live - L.k : t_hat;
@@ -372,10 +392,23 @@ int greedy_support(osscar_ctx* ctx, int t_hat, int32_t* support, int32_t* drop_t
         k_gr_score<<<(unsigned)n_live, g == 1 ? 32 : 256, smem_score, st>>>(p);
         k_gr_select<<<1, 1024, 0, st>>>(p, n_live, t, trace_pos);
         k_gr_stage_b<<<(unsigned)(t * g), 256, 0, st>>>(p, n_live);
-        k_gr_cinv<<<1, 256, 0, st>>>(p);
-        k_gr_stage_bc<<<(unsigned)(((int64_t)t * g * (p.lda + p.ldv) + 255) / 256 < 2368 ? ((int64_t)t * g * (p.lda + p.ldv) + 255) / 256 : 2368), 256, 0, st>>>(p, n_live);
-        k_gr_obj<<<1, 1024, 0, st>>>(p);
         {
+            const size_t cs = ((size_t)t * g * t * g + 2 * (size_t)t * g) * sizeof(double);
+            const bool fits = cs <= 200 * 1024;
+            k_gr_cinv<<<1, fits ? 1024 : 256, fits ? cs : 0, st>>>(p, fits ? 1 : 0);
+        }
+        k_gr_stage_bc<<<(unsigned)(((int64_t)t * g * (p.lda + p.ldv) + 255) / 256 < 2368 ? ((int64_t)t * g * (p.lda + p.ldv) + 255) / 256 : 2368), 256, 0, st>>>(p, n_live);
+        k_gr_obj<<<128, 256, 0, st>>>(p, ctx->partials);
+        k_gr_obj_add<<<1, 1, 0, st>>>(ctx->ctl, ctx->partials, 128);
+        const int64_t Tt = (int64_t)t * g;
+        if (Tt >= 32) {
+            // wide downdates: A -= BC^T B and V -= B^T KT as products with inner dimension T on the tensor cores
+            void* tc = ws + L.off_tc;
+            if (gemm_tc(st, nrows, round_up(nrows, 4), Tt, -1.f, p.BCT, Tt, p.B, p.lda, 1.f, p.A, p.lda, tc, L.tc_bytes, &ctx->ctl->status)
+                    != cudaSuccess) return OSSCAR_E_CUDA;
+            if (gemm_tc(st, nrows, p.ldv, Tt, -1.f, p.BT, Tt, p.KT, p.ldv, 1.f, p.V, p.ldv, tc, L.tc_bytes, &ctx->ctl->status)
+                    != cudaSuccess) return OSSCAR_E_CUDA;
+        } else {
             const int64_t nc4 = (round_up(nrows, 4)) / 4;
             dim3 ga((unsigned)((nc4 + 255) / 256), (unsigned)((nrows + UT_ROWS - 1) / UT_ROWS));
             k_gr_update<<<ga, 256, 0, st>>>(p.A, p.lda, nc4, nrows, p.BC, p.lda, p.B, p.lda, p.sel, g);
@@ -386,7 +419,7 @@ int greedy_support(osscar_ctx* ctx, int t_hat, int32_t* support, int32_t* drop_t
         const int n_new = n_live - t;
         k_gr_compact<<<dim3(64, (unsigned)t), 256, 0, st>>>(p, 0, (int64_t)n_new);
         k_gr_compact<<<dim3(64, (unsigned)t), 256, 0, st>>>(p, 1, (int64_t)n_new);
-        count_launches(11);
+        count_launches(12);
         CK(cudaGetLastError());
         n_live = n_new; trace_pos += t; ++iters;
     }

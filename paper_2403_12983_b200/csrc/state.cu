@@ -307,8 +307,8 @@ int make_layout(int64_t d1, int64_t m, int32_t g, int32_t k, Layout* L)
     const int64_t npairs = (int64_t)k * (ng - k);
     L->pair_capacity = npairs <= kMaxPairs ? npairs : 0;
     if (L->pair_capacity > 0 && nJ * ldh + nI * round_up(nJ, kPadF) > big) big = nJ * ldh + nI * round_up(nJ, kPadF);
-    {   // the nested phase keeps V of all rows plus up to 256 staged rows of Hinv (twice) and of V in `big`
-        const int64_t gneed = d1 * ldm + 2 * 256 * L->ldp + 256 * ldm;
+    {   // the nested phase keeps V of all rows plus up to 256 staged rows of Hinv (twice, and their transposes) and of V in `big`
+        const int64_t gneed = d1 * ldm + 2 * 256 * L->ldp + 256 * ldm + 2 * 256 * d1;
         if (gneed > big) big = gneed;
     }
     L->off_big = take(sizeof(float) * big);

@@ -410,6 +410,8 @@ GREEDY_CASES = [
     ("c5", dict(n=4096, d1=264, m=72, k=80, chunk_rows=4096), 7),
     ("c4", dict(n=49 * 40, d1=9 * 60, m=130, k=25, chunk_rows=49 * 40), 2),
     ("c3", dict(n=8192, d1=12 * 40, m=200, g=40, k=6, chunk_rows=8192), 2),
+    ("c2", dict(n=4096, d1=520, m=150, k=207, chunk_rows=4096), 64),          # wide steps: tensor-core downdates
+    ("c5", dict(n=8192, d1=1000, m=300, k=300, chunk_rows=4096), 100),
 ]
 
 
