@@ -20,25 +20,30 @@ import workloads
 pytestmark = [pytest.mark.gpu, pytest.mark.slow]
 
 
-def _run(name, n_cols, max_swaps):
+def _run(name, n_cols, max_swaps, block_pairs=0):
     import paper_2403_12983_b200 as pkg
     wl = workloads.config(name)
     dev = torch.device("cuda", 0)
     solver = pkg.Solver(0)
     W = wl.weight(dev)
     x_dev = [wl.x_chunk(c, dev) for c in range(wl.n_chunks)]
-    res = pkg.solve_layer(solver, x_dev, W, wl.g, wl.k, max_swaps, damp=wl.damp, accept_rel_tol=wl.eps_acc)
+    res = pkg.solve_layer(solver, x_dev, W, wl.g, wl.k, max_swaps, damp=wl.damp, accept_rel_tol=wl.eps_acc,
+                          block_pairs=block_pairs)
     rng = np.random.default_rng(0)
     support = res.support.cpu().numpy()
     assert len(np.unique(support)) == wl.k and support.min() >= 0 and support.max() < wl.ngroups
     assert np.all(np.diff(support) > 0)
     obj = res.obj_trace.cpu().numpy()
-    assert len(obj) == res.n_swaps + 1 and res.n_swaps > 0
+    per_it = max(block_pairs, 1)                 # block exchanges record one objective per iteration
+    assert res.n_swaps % per_it == 0 and len(obj) == res.n_swaps // per_it + 1 and res.n_swaps > 0
     assert np.all(np.diff(obj) <= -wl.eps_acc * obj[:-1] * (1 - 1e-6))
     assert obj[-1] == pytest.approx(res.obj_final, rel=1e-4)
     swaps = res.swap_trace.cpu().numpy()
     kept = set(int(s) for s in support)
     assert all(int(j) != int(i) for i, j in swaps)
+    for it in range(res.n_swaps // per_it):       # an exchange moves distinct groups
+        blk = swaps[it * per_it:(it + 1) * per_it]
+        assert len(set(int(v) for v in blk.reshape(-1))) == 2 * per_it
     Wout = res.W
     pruned_mask = torch.ones(wl.d1, dtype=torch.bool, device=dev)
     pruned_mask[res.support.long()] = False
@@ -94,3 +99,13 @@ def test_c2_full_size_properties():
 def test_c5_full_size_properties():
     res = _run("c5", n_cols=2, max_swaps=300)
     assert res.n_swaps == 300 or res.stop_reason == "no_improvement"
+
+
+def test_c2_full_size_block_exchange_properties():
+    res = _run("c2", n_cols=4, max_swaps=2000, block_pairs=50)
+    assert res.stop_reason in ("no_improvement", "max_swaps")
+
+
+def test_c5_full_size_block_exchange_properties():
+    res = _run("c5", n_cols=2, max_swaps=600, block_pairs=50)
+    assert res.n_swaps == 600 or res.stop_reason == "no_improvement"
