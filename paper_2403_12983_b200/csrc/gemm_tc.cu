@@ -328,6 +328,205 @@ __global__ void k_split3(const float* __restrict__ src, int64_t lds, int64_t row
     }
 }
 
+// ---------------------------------------------------------------------------------------------------------------
+// Rank-K update C += alpha * U * W with a short inner dimension (K <= 128): U (M x K) and W (K x N) are panels, C is
+// large and streamed once.  The generic pipeline above re-reads the operand terms for every output tile, which for
+// K ~ 100 is more L2 traffic than the tile of C itself; here a CTA keeps the three bf16 terms of its 128-row band
+// of U in shared memory (up to 96 KB) across a run of 128-column tiles and only the terms of W stream through a
+// two-stage ring (48 KB per 64-wide k-block).  One TMEM accumulator chain per tile (at most 48 MMAs), drained by
+// eight accumulate warps that do the read-modify-write of C through the shared-memory staging blocks.
+constexpr int RU_TN = 128;                                   // columns per tile
+constexpr int RU_W_BYTES = 3 * (RU_TN / 64) * BOX_BYTES;     // 49152: three terms of a 64 x 128 block of W
+constexpr int RU_U_BYTES = 3 * 2 * A_BYTES;                  // 98304: three terms x two k-blocks of the U band
+constexpr int RU_SMEM = RU_U_BYTES + 2 * RU_W_BYTES + 1024 + 256 + EPI_BYTES;
+constexpr uint32_t kRuIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(RU_TN >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
+
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+k_rank_update(const __grid_constant__ Maps maps, int64_t M, int64_t N, int nkb, float alpha, float* __restrict__ C, int64_t ldc,
+              int TN, int nchunk, int num_items, int32_t* __restrict__ status, const int32_t* __restrict__ done)
+{
+    if (done && *done) return;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t* base_ptr = smem_raw + (base - raw);
+    const uint32_t u_base = base, w_base = base + RU_U_BYTES;
+    uint8_t* bar_ptr = base_ptr + RU_U_BYTES + 2 * RU_W_BYTES;
+    const uint32_t bars = base + RU_U_BYTES + 2 * RU_W_BYTES;
+    auto w_full = [&](int s) { return bars + 8u * s; };
+    auto w_empty = [&](int s) { return bars + 8u * (2 + s); };
+    auto tfull_bar = [&](int b) { return bars + 8u * (4 + b); };
+    auto tempty_bar = [&](int b) { return bars + 8u * (6 + b); };
+    const uint32_t u_full = bars + 8u * 8, u_empty = bars + 8u * 9;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_ptr + 8 * 10);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_ptr + 8 * 10 + 8);
+    float* epi = reinterpret_cast<float*>(bar_ptr + 256);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < 2; ++i) { mbar_init(w_full(i), 1); mbar_init(w_empty(i), 1); mbar_init(tfull_bar(i), 1); mbar_init(tempty_bar(i), 8); }
+        mbar_init(u_full, 1); mbar_init(u_empty, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "n"(256) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = *tmem_slot;
+
+    // item = (row band, run of column tiles)
+    auto item_of = [&](int id, int* tm, int* tn0, int* tn1) {
+        *tm = id / nchunk;
+        const int c = id % nchunk, per = (TN + nchunk - 1) / nchunk;
+        *tn0 = c * per; *tn1 = min(TN, *tn0 + per);
+    };
+
+    if (warp == 0) {
+        if (lane == 0) {
+            uint32_t it = 0, item = 0;          // item counts the bands this CTA has loaded
+            bool ok = true;
+            for (int id = blockIdx.x; id < num_items && ok; id += gridDim.x) {
+                int tm, tn0, tn1;
+                item_of(id, &tm, &tn0, &tn1);
+                if (tn0 >= tn1) continue;
+                if (!mbar_wait(u_empty, (item & 1) ^ 1, abort_flag)) { ok = false; break; }
+                ++item;
+                mbar_expect_tx(u_full, (uint32_t)(3 * nkb * A_BYTES));
+                for (int kb = 0; kb < nkb; ++kb)
+#pragma unroll
+                    for (int term = 0; term < 3; ++term)
+                        tma_load_2d(u_base + (term * 2 + kb) * A_BYTES, &maps.a[term], u_full, kb * BLOCK_K, tm * TILE_M);
+                for (int tn = tn0; tn < tn1 && ok; ++tn) {
+                    for (int kb = 0; kb < nkb; ++kb, ++it) {
+                        const int s = it & 1;
+                        if (!mbar_wait(w_empty(s), ((it >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
+                        mbar_expect_tx(w_full(s), RU_W_BYTES);
+#pragma unroll
+                        for (int term = 0; term < 3; ++term)
+#pragma unroll
+                            for (int i = 0; i < RU_TN / 64; ++i)
+                                tma_load_2d(w_base + s * RU_W_BYTES + (term * (RU_TN / 64) + i) * BOX_BYTES, &maps.b[term], w_full(s),
+                                            tn * RU_TN + i * 64, kb * BLOCK_K);
+                    }
+                }
+            }
+            if (*abort_flag) {                    // let the copies in flight land before the CTA exits
+                const long long t0 = clock64();
+                while (it > 0 && !mbar_try_wait(w_full((it - 1) & 1), ((it - 1) >> 1) & 1))
+                    if (clock64() - t0 > kWaitLimitCycles) break;
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            uint32_t it = 0, tile = 0, item = 0;
+            bool ok = true;
+            for (int id = blockIdx.x; id < num_items && ok; id += gridDim.x) {
+                int tm, tn0, tn1;
+                item_of(id, &tm, &tn0, &tn1);
+                if (tn0 >= tn1) continue;
+                if (!mbar_wait(u_full, item & 1, abort_flag)) { ok = false; break; }
+                ++item;
+                for (int tn = tn0; tn < tn1 && ok; ++tn, ++tile) {
+                    const int buf = tile & 1;
+                    if (!mbar_wait(tempty_bar(buf), ((tile >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint32_t d_tmem = tmem_base + (uint32_t)(buf * RU_TN);
+                    bool first = true;
+                    for (int kb = 0; kb < nkb && ok; ++kb, ++it) {
+                        const int s = it & 1;
+                        if (!mbar_wait(w_full(s), (it >> 1) & 1, abort_flag)) { ok = false; break; }
+                        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll
+                        for (int term = 0; term < 6; ++term) {
+                            const int pa = (0x001012 >> (4 * term)) & 0xF;      // small products first
+                            const int pb = (0x010210 >> (4 * term)) & 0xF;
+                            const uint32_t a_src = u_base + (pa * 2 + kb) * A_BYTES;
+                            const uint32_t b_src = w_base + s * RU_W_BYTES + pb * (RU_TN / 64) * BOX_BYTES;
+#pragma unroll
+                            for (int j = 0; j < BLOCK_K / UMMA_K; ++j) {
+                                umma_f16(d_tmem, desc_a(a_src + j * 32), desc_b(b_src + j * (UMMA_K * 128)), kRuIdesc, first ? 0u : 1u);
+                                first = false;
+                            }
+                        }
+                        umma_commit(w_empty(s));
+                    }
+                    if (ok) umma_commit(tfull_bar(buf));
+                }
+                if (ok) umma_commit(u_empty);        // the band's terms may be replaced once these MMAs are done
+            }
+        }
+    } else {
+        const int lg = warp & 3, half = (warp - 2) >> 2;       // 32 rows x 64 columns per warp
+        uint32_t tile = 0;
+        bool ok = true;
+        float* stg = epi + (warp - 2) * 32 * EPI_LD;
+        const int rsub = lane >> 3, c4 = (lane & 7) * 4;
+        for (int id = blockIdx.x; id < num_items && ok; id += gridDim.x) {
+            int tm, tn0, tn1;
+            item_of(id, &tm, &tn0, &tn1);
+            for (int tn = tn0; tn < tn1 && ok; ++tn, ++tile) {
+                const int buf = tile & 1;
+                const int64_t grow0 = (int64_t)tm * TILE_M + lg * 32;
+                const int64_t gcol0 = (int64_t)tn * RU_TN + half * 64;
+                if (grow0 + lane < M) {          // bring the old values of this thread's row segment towards L2
+#pragma unroll
+                    for (int j = 0; j < 64; j += 32)
+                        if (gcol0 + j < N) asm volatile("prefetch.global.L2 [%0];" ::"l"(C + (grow0 + lane) * ldc + gcol0 + j));
+                }
+                if (!mbar_wait(tfull_bar(buf), (tile >> 1) & 1, abort_flag)) { ok = false; break; }
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                float acc[64];
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    uint32_t r[32];
+                    tmem_ld32(tmem_base + ((uint32_t)(lg * 32) << 16) + (uint32_t)(buf * RU_TN + half * 64 + c * 32), r);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) acc[c * 32 + j] = alpha * __uint_as_float(r[j]);
+                }
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) mbar_arrive(tempty_bar(buf));
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    const int64_t gc = gcol0 + c * 32 + c4;
+                    __syncwarp();
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) stg[lane * EPI_LD + j] = acc[c * 32 + j];
+                    __syncwarp();
+                    float4 o[8];
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        const int64_t gr = grow0 + q * 4 + rsub;
+                        o[q] = (gr < M && gc < N) ? __ldcs(reinterpret_cast<const float4*>(C + gr * ldc + gc)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        const int r = q * 4 + rsub;
+                        const int64_t gr = grow0 + r;
+                        const float* sp = stg + r * EPI_LD + c4;
+                        if (gr < M && gc < N)
+                            *reinterpret_cast<float4*>(C + gr * ldc + gc) =
+                                make_float4(o[q].x + sp[0], o[q].y + sp[1], o[q].z + sp[2], o[q].w + sp[3]);
+                    }
+                }
+            }
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "n"(256) : "memory");
+    }
+    if (threadIdx.x == 0 && *abort_flag) *status = OSSCAR_E_TIMEOUT;
+}
+
 bool encode_2d(PFN_encodeTiled enc, CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer, uint64_t ld_elems,
                uint32_t box_inner, uint32_t box_outer)
 {
@@ -398,6 +597,54 @@ cudaError_t gemm_tc(cudaStream_t st, int64_t M, int64_t N, int64_t K, float alph
         if (e != cudaSuccess) return e;
     }
     return cudaSuccess;
+}
+
+// C += alpha * U * W for a short inner dimension (see k_rank_update); falls back to the generic product otherwise.
+cudaError_t rank_update_tc(cudaStream_t st, int64_t M, int64_t N, int64_t K, float alpha, const float* U, int64_t ldu,
+                           const float* W, int64_t ldw, float* C, int64_t ldc,
+                           void* scratch, size_t scratch_bytes, int32_t* status_dev, const int32_t* done)
+{
+    if (M <= 0 || N <= 0 || K <= 0) return cudaSuccess;
+    const bool fits = K <= 2 * BLOCK_K && (N % 4) == 0 && (ldc % 4) == 0 && (((uintptr_t)C & 15) == 0);
+    if (!fits) return gemm_tc(st, M, N, K, alpha, U, ldu, W, ldw, 1.f, C, ldc, scratch, scratch_bytes, status_dev, done);
+    PFN_encodeTiled enc = get_encode();
+    if (!enc) return cudaErrorNotSupported;
+    if ((uintptr_t)scratch & 255) return cudaErrorInvalidValue;
+    const int64_t k8 = round_up(K, 8), ldn = round_up(N, 8);
+    auto align_up = [](size_t x) { return (x + 1023) / 1024 * 1024; };
+    const size_t u_bytes = align_up((size_t)M * k8 * 2), w_bytes = align_up((size_t)K * ldn * 2);
+    if (3 * (u_bytes + w_bytes) > scratch_bytes) return cudaErrorInvalidValue;
+    __nv_bfloat16* up[3]; __nv_bfloat16* wp[3];
+    for (int i = 0; i < 3; ++i) {
+        up[i] = (__nv_bfloat16*)((char*)scratch + i * u_bytes);
+        wp[i] = (__nv_bfloat16*)((char*)scratch + 3 * u_bytes + i * w_bytes);
+    }
+    int dev = 0, sms = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(k_rank_update, cudaFuncAttributeMaxDynamicSharedMemorySize, RU_SMEM);
+    if (e != cudaSuccess) return e;
+    k_split3<<<1184, 256, 0, st>>>(U, ldu, M, K, up[0], up[1], up[2], k8, done);
+    k_split3<<<1184, 256, 0, st>>>(W, ldw, K, N, wp[0], wp[1], wp[2], ldn, done);
+    Maps maps;
+    for (int i = 0; i < 3; ++i) {
+        if (!encode_2d(enc, &maps.a[i], up[i], (uint64_t)K, (uint64_t)M, (uint64_t)k8, BLOCK_K, TILE_M)) return cudaErrorInvalidValue;
+        if (!encode_2d(enc, &maps.b[i], wp[i], (uint64_t)N, (uint64_t)K, (uint64_t)ldn, 64, BLOCK_K)) return cudaErrorInvalidValue;
+    }
+    const int TM = (int)((M + TILE_M - 1) / TILE_M), TN = (int)((N + RU_TN - 1) / RU_TN);
+    int nchunk = (4 * sms + TM - 1) / TM;                 // runs of column tiles per band: about four items per SM
+    if (nchunk > TN) nchunk = TN;
+    if (nchunk < 1) nchunk = 1;
+    const int per = (TN + nchunk - 1) / nchunk;
+    nchunk = (TN + per - 1) / per;                        // no empty runs
+    const int num_items = TM * nchunk;
+    const int nkb = (int)((K + BLOCK_K - 1) / BLOCK_K);
+    k_rank_update<<<num_items < sms ? num_items : sms, NUM_THREADS, RU_SMEM, st>>>(maps, M, N, nkb, alpha, C, ldc, TN, nchunk, num_items,
+                                                                                  status_dev, done);
+    count_launches(3);
+    return cudaGetLastError();
 }
 
 // H (+)= Xc^T Xc over the upper-triangle tiles (Yc == nullptr), or G (+)= Xc^T Yc over all tiles.

@@ -552,9 +552,9 @@ cudaError_t enqueue_block_step(osscar_ctx* ctx, const Ptrs& p, const BlockPtrs& 
     k_blk_leave_d<<<(unsigned)((G * G + 7) / 8), 256, 0, st>>>(p, bp);
     k_blk_finish_d<<<(unsigned)(((L.nJ + G) * G + 255) / 256), 256, 0, st>>>(p, bp);            mark();
     // the three rank-2G updates; the residual rows of the leaving groups go through the Rq panel
-    BK(gemm_tc(st, L.nI, L.ldh, 2 * G, -1.f, bp.PAT, 2 * G, bp.PB, L.ldh, 1.f, p.Hinv, L.ldh, tc, L.tc_bytes, stat, done));   mark();
-    BK(gemm_tc(st, L.nI, L.m, 2 * G, -1.f, bp.PBT, 2 * G, bp.KV, L.ldm, 1.f, p.V, L.ldm, tc, L.tc_bytes, stat, done));        mark();
-    BK(gemm_tc(st, L.nJ, L.m, 2 * G, 1.f, bp.UD, 2 * G, bp.KV, L.ldm, 1.f, p.R, L.ldm, tc, L.tc_bytes, stat, done));
+    BK(rank_update_tc(st, L.nI, L.ldh, 2 * G, -1.f, bp.PAT, 2 * G, bp.PB, L.ldh, p.Hinv, L.ldh, tc, L.tc_bytes, stat, done));   mark();
+    BK(rank_update_tc(st, L.nI, L.ldm, 2 * G, -1.f, bp.PBT, 2 * G, bp.KV, L.ldm, p.V, L.ldm, tc, L.tc_bytes, stat, done));       mark();
+    BK(rank_update_tc(st, L.nJ, L.ldm, 2 * G, 1.f, bp.UD, 2 * G, bp.KV, L.ldm, p.R, L.ldm, tc, L.tc_bytes, stat, done));
     BK(sgemm(st, false, false, G, L.m, 2 * G, 1.f, bp.UD + L.nJ * 2 * G, 2 * G, bp.KV, L.ldm, 0.f, bp.Rq, L.ldm, done));   mark();
     if (L.g == 1) k_blk_update_c_g1<<<296, 256, 2 * (size_t)G * G * sizeof(float), st>>>(p, bp);
     else k_blk_update_c<<<(unsigned)(L.ng - L.k), 128, 2 * (size_t)L.g * G * sizeof(double), st>>>(p, bp);
