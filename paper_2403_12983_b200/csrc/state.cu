@@ -127,59 +127,47 @@ __global__ void k_copy_pad(const float* __restrict__ src, int64_t lds, int64_t r
 constexpr int NB = 64;
 constexpr double kPivotRelTol = 1e-7;
 
-// Inverse of the nb x nb pivot block A[p0:p0+nb, p0:p0+nb] by Cholesky in fp64 (one block).
+// Inverse of the nb x nb pivot block A[p0:p0+nb, p0:p0+nb] in fp64 (one block): in-place Gauss-Jordan elimination
+// without pivoting, one rank-1 update over the whole block per step, so every thread works in every step.  The
+// pivots are the diagonal of the successive Schur complements (the squared diagonal of the Cholesky factor).
 // Raises OSSCAR_E_NOTPD in ctl->status when a pivot is not positive.
 __global__ void __launch_bounds__(256)
 k_pivot_inverse(const float* __restrict__ A, int64_t lda, int64_t p0, int nb, float* __restrict__ Dinv,
                 const float* __restrict__ Hp, int64_t ldp, SearchCtl* ctl)
 {
     extern __shared__ double sm[];
-    double* L = sm;                 // nb x nb, lower Cholesky factor, then its inverse
-    double* R = sm + NB * NB;       // result
+    double* L = sm;                 // nb x nb (ld NB): the block, overwritten by its inverse
+    double* colj = sm + NB * NB;    // column j and scaled row j of the current step
+    double* rowj = colj + NB;
     const int t = threadIdx.x;
     for (int idx = t; idx < nb * nb; idx += blockDim.x) {
         int i = idx / nb, j = idx % nb;
         // symmetrise: the two triangles can differ in the last bits
         L[i * NB + j] = 0.5 * ((double)A[(p0 + i) * lda + p0 + j] + (double)A[(p0 + j) * lda + p0 + i]);
     }
-    __syncthreads();
     __shared__ int bad;
     if (t == 0) bad = 0;
     __syncthreads();
     for (int j = 0; j < nb; ++j) {
-        if (t == 0) {
-            double d = L[j * NB + j];
-            // a pivot that fp32 data cannot tell from zero counts as not positive
-            if (!(d > kPivotRelTol * (double)Hp[(p0 + j) * ldp + p0 + j])) { bad = 1; d = 1.0; }
-            L[j * NB + j] = sqrt(d);
-        }
+        double d = L[j * NB + j];
+        // a pivot that fp32 data cannot tell from zero counts as not positive
+        if (!(d > kPivotRelTol * (double)Hp[(p0 + j) * ldp + p0 + j])) { if (t == 0) bad = 1; d = 1.0; }
+        const double pinv = 1.0 / d;
+        for (int i = t; i < nb; i += blockDim.x) { colj[i] = L[i * NB + j]; rowj[i] = L[j * NB + i] * pinv; }
         __syncthreads();
-        const double djj = L[j * NB + j];
-        for (int i = j + 1 + t; i < nb; i += blockDim.x) L[i * NB + j] /= djj;
-        __syncthreads();
-        // trailing update of the lower triangle
-        const int rem = nb - j - 1;
-        for (int idx = t; idx < rem * rem; idx += blockDim.x) {
-            int i = j + 1 + idx / rem, c = j + 1 + idx % rem;
-            if (c <= i) L[i * NB + c] -= L[i * NB + j] * L[c * NB + j];
+        for (int idx = t; idx < nb * nb; idx += blockDim.x) {
+            const int i = idx / nb, c = idx % nb;
+            double v;
+            if (i == j) v = (c == j) ? pinv : rowj[c];
+            else if (c == j) v = -colj[i] * pinv;
+            else v = L[i * NB + c] - colj[i] * rowj[c];
+            L[i * NB + c] = v;
         }
         __syncthreads();
     }
-    // R = L^-1 (lower): column by column forward substitution, one thread per column
-    for (int c = t; c < nb; c += blockDim.x) {
-        for (int i = 0; i < nb; ++i) {
-            double s = (i == c) ? 1.0 : 0.0;
-            for (int kx = c; kx < i; ++kx) s -= L[i * NB + kx] * R[kx * NB + c];
-            R[i * NB + c] = (i < c) ? 0.0 : s / L[i * NB + i];
-        }
-    }
-    __syncthreads();
-    // Dinv = R^T R
-    for (int idx = t; idx < nb * nb; idx += blockDim.x) {
+    for (int idx = t; idx < nb * nb; idx += blockDim.x) {       // the two triangles differ by rounding only
         int i = idx / nb, j = idx % nb;
-        double s = 0.0;
-        for (int kx = (i > j ? i : j); kx < nb; ++kx) s += R[kx * NB + i] * R[kx * NB + j];
-        Dinv[i * NB + j] = (float)s;
+        Dinv[i * NB + j] = (float)(0.5 * (L[i * NB + j] + L[j * NB + i]));
     }
     if (t == 0 && bad) ctl->status = OSSCAR_E_NOTPD;
 }
