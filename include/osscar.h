@@ -134,7 +134,7 @@ typedef struct {
     int32_t max_swaps;        /* >= 0                                                        */
     int32_t score_mode;       /* OSSCAR_SCORE_*                                              */
     int32_t accept_mode;      /* OSSCAR_ACCEPT_*                                             */
-    int32_t refresh_every;    /* rebuild the state from H every this many swaps; 0 = never   */
+    int32_t refresh_every;    /* rebuild the state from H every this many steps (swaps, or iterations of a block exchange); 0 = never */
     double  accept_rel_tol;   /* IMPROVING: accept iff delta <= -tol * obj (1e-5 if < 0)     */
     int32_t profile_samples;  /* time each kernel of this many evenly spaced steps (0..8)    */
     int32_t block_pairs;      /* s: groups exchanged per iteration (0 or 1: one swap per step) */

@@ -381,6 +381,35 @@ def test_block_exchange_matches_oracle(solver, name, over, seed, s, max_swaps, a
     assert np.allclose(c, cref, rtol=2e-3, atol=2e-3 * np.abs(cref).max())
 
 
+@pytest.mark.parametrize("name,over,s,greedy", [
+    ("c2", dict(n=4096, d1=520, m=150, k=207, chunk_rows=4096), 8, 0),
+    ("c4", dict(n=49 * 40, d1=9 * 100, m=130, k=50, chunk_rows=49 * 40), 3, 0),
+    ("c2", dict(n=4096, d1=520, m=150, k=207, chunk_rows=4096), 8, 16),
+])
+def test_block_exchange_with_refresh_and_greedy_start(solver, osscar, name, over, s, greedy):
+    """Block exchanges with the state rebuilt from H every second iteration, from the energy start and after the
+    nested phase: the rebuilt state must continue the same walk."""
+    b = osscar.binding
+    wl = workloads.config(name, **over)
+    chunks, W, H64, G64, const64 = oracle_problem(wl)
+    H, G, Wd = dev(H64), dev(G64), dev(W)
+    Hr, Gr = H.cpu().numpy().astype(np.float64), G.cpu().numpy().astype(np.float64)
+    const_r = float(np.sum(W * Gr))
+    if greedy:
+        support, _, obj0, _ = solver.init_support_greedy(H, G, Wd, wl.g, wl.k, greedy)
+    else:
+        support, obj0 = solver.init_support(H, G, Wd, wl.g, wl.k)
+    S0 = support.cpu().numpy()
+    out = solver.local_search(5 * s, accept_mode=b.ACCEPT_ALWAYS, refresh_every=2, block_pairs=s)
+    assert out.n_swaps == 5 * s and out.n_refresh == 2          # before iterations 2 and 4
+    swaps = [tuple(int(v) for v in r) for r in out.swap_trace.cpu().numpy()]
+    srch = follow_block(Hr, Gr, const_r, wl.g, S0, s, swaps, out.obj_trace.cpu().numpy(), accept="always",
+                        gpu_stop=out.stop_reason, max_iters=5, eps_acc=wl.eps_acc)
+    assert np.array_equal(out.support.cpu().numpy(), srch.result()[0])
+    assert out.obj_final == pytest.approx(srch.st.obj, rel=1e-4)
+    assert rel_fro(out.W.cpu().numpy(), srch.result()[1]) < 1e-3
+
+
 def test_block_exchange_argument_checks(solver, osscar):
     import paper_2403_12983_b200.binding as b
     wl = workloads.config("c1")
