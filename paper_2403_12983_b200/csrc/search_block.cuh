@@ -185,17 +185,7 @@ __device__ void blk_mat_mul(const double* A, bool tA, const double* B, bool tB, 
     __syncthreads();
     for (int idx = threadIdx.x; idx < gg; idx += blockDim.x) { sm[idx] = A[idx]; sm[gg + idx] = B[idx]; }
     __syncthreads();
-    const double* As = sm; const double* Bs = sm + gg;
-    for (int idx = threadIdx.x; idx < gg; idx += blockDim.x) {
-        const int i = idx / g, j = idx % g;
-        double s = 0.0;
-        if (!tA && !tB)     for (int kx = 0; kx < g; ++kx) s += As[i * g + kx] * Bs[kx * g + j];
-        else if (!tA && tB) for (int kx = 0; kx < g; ++kx) s += As[i * g + kx] * Bs[j * g + kx];
-        else if (tA && !tB) for (int kx = 0; kx < g; ++kx) s += As[kx * g + i] * Bs[kx * g + j];
-        else                for (int kx = 0; kx < g; ++kx) s += As[kx * g + i] * Bs[j * g + kx];
-        C[idx] = s;
-    }
-    __syncthreads();
+    mat_mul(sm, tA, sm + gg, tB, C, g);
 }
 
 // One block: the G x G algebra of the exchange, its exact change of obj and the accept decision.

@@ -54,15 +54,32 @@ static __device__ double chol_inverse(double* M, double* Lw, double* Out, int g)
     __syncthreads();
     return minpiv;
 }
-// C = op(A) * op(B), all g x g, block-cooperative.
+// C = op(A) * op(B), all g x g (ld g), block-cooperative, on the fp64 tensor-core path: every warp of the block takes
+// 8 x 8 tiles of C in turn and runs g / 4 steps of mma.m8n8k4 (A fragment: row lane / 4, column lane % 4; B fragment:
+// row lane % 4, column lane / 4; C fragment: row lane / 4, columns 2 (lane % 4) and + 1).  Entries beyond g read as 0.
+// C must not overlap A or B.  blockDim.x must be a multiple of 32.
 static __device__ void mat_mul(const double* A, bool tA, const double* B, bool tB, double* C, int g)
 {
-    for (int idx = threadIdx.x; idx < g * g; idx += blockDim.x) {
-        const int i = idx / g, j = idx % g;
-        double s = 0.0;
-        for (int kx = 0; kx < g; ++kx)
-            s += (tA ? A[kx * g + i] : A[i * g + kx]) * (tB ? B[j * g + kx] : B[kx * g + j]);
-        C[idx] = s;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    const int nt = (g + 7) >> 3;
+    const int r4 = lane >> 2, c4 = lane & 3;
+    for (int tile = warp; tile < nt * nt; tile += nwarps) {
+        const int i0 = (tile / nt) * 8, j0 = (tile % nt) * 8;
+        const int ai = i0 + r4, bj = j0 + r4;
+        double d0 = 0.0, d1 = 0.0;
+        for (int k0 = 0; k0 < g; k0 += 4) {
+            const int kk = k0 + c4;
+            const bool ka = kk < g;
+            const double a = (ka && ai < g) ? (tA ? A[kk * g + ai] : A[ai * g + kk]) : 0.0;
+            const double b = (ka && bj < g) ? (tB ? B[bj * g + kk] : B[kk * g + bj]) : 0.0;
+            asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0, %1}, {%2}, {%3}, {%0, %1};"
+                         : "+d"(d0), "+d"(d1) : "d"(a), "d"(b));
+        }
+        const int ci = i0 + r4, cj = j0 + 2 * c4;
+        if (ci < g) {
+            if (cj < g) C[ci * g + cj] = d0;
+            if (cj + 1 < g) C[ci * g + cj + 1] = d1;
+        }
     }
     __syncthreads();
 }
