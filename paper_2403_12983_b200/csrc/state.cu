@@ -146,12 +146,14 @@ k_pivot_inverse(const float* __restrict__ A, int64_t lda, int64_t p0, int nb, fl
         L[i * NB + j] = 0.5 * ((double)A[(p0 + i) * lda + p0 + j] + (double)A[(p0 + j) * lda + p0 + i]);
     }
     __shared__ int bad;
+    __shared__ double hdiag[NB];         // diagonal of the original matrix: scale of the pivot test
     if (t == 0) bad = 0;
+    for (int j = t; j < nb; j += blockDim.x) hdiag[j] = (double)Hp[(p0 + j) * ldp + p0 + j];
     __syncthreads();
     for (int j = 0; j < nb; ++j) {
         double d = L[j * NB + j];
         // a pivot that fp32 data cannot tell from zero counts as not positive
-        if (!(d > kPivotRelTol * (double)Hp[(p0 + j) * ldp + p0 + j])) { if (t == 0) bad = 1; d = 1.0; }
+        if (!(d > kPivotRelTol * hdiag[j])) { if (t == 0) bad = 1; d = 1.0; }
         const double pinv = 1.0 / d;
         for (int i = t; i < nb; i += blockDim.x) { colj[i] = L[i * NB + j]; rowj[i] = L[j * NB + i] * pinv; }
         __syncthreads();
