@@ -245,6 +245,25 @@ def run_ours(args):
     total_ms = e0.elapsed_time(e1)
     K = max(args.steps, 1)
 
+    # ---------------- the same layer with the paper's larger local-search steps (outside the timed region above)
+    block_extra = None
+    if world == 1 and args.block_pairs <= 1 and not args.no_block_extra and wl.g * 16 <= 96 and wl.score_mode != "pair_exact":
+        block_extra = []
+        for s_pairs in (16, 50):
+            if s_pairs * wl.g > 96 or s_pairs > min(wl.k, wl.ngroups - wl.k):
+                continue
+            f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            f0.record()
+            rb = pkg.solve_layer(solver, x_dev, W, wl.g, wl.k, max_swaps, damp=wl.damp, accept_mode=accept, accept_rel_tol=wl.eps_acc,
+                                 H=H, G=G, block_pairs=s_pairs)
+            f1.record()
+            torch.cuda.synchronize()
+            block_extra.append({"pairs_per_iteration": s_pairs, "swaps": rb.n_swaps, "iterations": rb.n_swaps // s_pairs,
+                                "layer_solve_s": f0.elapsed_time(f1) / 1e3, "search_ms": rb.ms["search"],
+                                "swaps_per_s": rb.n_swaps / max(rb.ms["search"] * 1e-3, 1e-9),
+                                "obj_init": rb.obj_init, "obj_final": rb.obj_final, "stop_reason": rb.stop_reason})
+
     # ---------------- end to end: host buffers, copies inside the timed region
     e2e = None
     if not args.no_e2e:
@@ -350,6 +369,8 @@ def run_ours(args):
     else:
         out["e2e"] = {"value": None, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0,
                       "note": (e2e or {}).get("error", "skipped")}
+    if block_extra:
+        out["block_exchange"] = block_extra
     if world == 1 and not args.no_cpu:
         out["cpu_baseline"] = cpu_baseline()
     print(json.dumps(out))
@@ -371,6 +392,7 @@ def main():
     ap.add_argument("--max-swaps", type=int, default=None)
     ap.add_argument("--greedy", type=int, default=0, help="start from the nested phase of Algorithm 1 with this t_hat")
     ap.add_argument("--block-pairs", type=int, default=0, help="groups exchanged per iteration (t_hat = 2 s, p_hat = 0); 0 = single swaps")
+    ap.add_argument("--no-block-extra", action="store_true", help="skip the extra solves with block exchanges of 16 and 50 groups")
     ap.add_argument("--accept-always", action="store_true", help="paper-literal fixed number of iterations")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
