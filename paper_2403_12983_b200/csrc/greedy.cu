@@ -92,7 +92,7 @@ __global__ void k_gr_score(GPtrs p)
         M[idx] = 0.5 * ((double)p.A[(grp * g + i) * p.lda + grp * g + j] + (double)p.A[(grp * g + j) * p.lda + grp * g + i]);
     }
     __syncthreads();
-    const double piv = chol_inverse(M, Lw, Out, g);
+    const double piv = spd_inverse(M, Lw, Out, g);
     const double tr = mat_trace_prod(Out, p.gram + grp * gg, g, red);
     if (threadIdx.x == 0) p.D[grp] = piv > 0.0 ? tr : INFINITY;
 }
@@ -180,7 +180,7 @@ __global__ void __launch_bounds__(1024) k_gr_cinv(GPtrs p, int in_smem)
         C[idx] = 0.5 * ((double)p.A[ra * p.lda + rb] + (double)p.A[rb * p.lda + ra]);
     }
     __syncthreads();
-    const double piv = chol_inverse(C, Lw, Cinv, T);
+    const double piv = spd_inverse(C, Lw, Cinv, T);
     if (threadIdx.x == 0 && !(piv > 0.0)) p.ctl->status = OSSCAR_E_NOTPD;
 }
 // BC[e][s] = sum_f Cinv[e][f] B[f][s]  and  KT[e][c] = sum_f Cinv[e][f] V[r_f][c];  obj += sum_e KT[e] . V[r_e].

@@ -108,7 +108,7 @@ __global__ void k_scores_general(Ptrs p, int kind)
         }
     }
     __syncthreads();
-    const double piv = chol_inverse(M, Lw, Out, g);
+    const double piv = spd_inverse(M, Lw, Out, g);
     const double* gram = (kind == 0 ? p.gramV : p.gramR) + grp * g * g;
     const double tr = mat_trace_prod(Out, gram, g, red);
     if (threadIdx.x == 0) {
@@ -239,7 +239,7 @@ k_small(Ptrs p, int accept_mode, double accept_tol, int max_swaps, double* __res
         P[idx] = (double)p.y[(int64_t)i * p.ldh + r0 + j];           // P[a][b] = y_a[r_b]
     }
     __syncthreads();
-    const double pivC = chol_inverse(C, Lw, Cinv, g);
+    const double pivC = spd_inverse(C, Lw, Cinv, g);
     const double Ds = mat_trace_prod(Cinv, GV, g, red);               // Tr(C^-1 V_r V_r^T)
     // R1 R1^T = GR + P (Cinv GX) + (P Cinv GX)^T + P Cinv GV Cinv P^T
     mat_mul(Cinv, false, GX, false, T1, g);                           // K R_q^T
@@ -259,7 +259,7 @@ k_small(Ptrs p, int accept_mode, double accept_tol, int max_swaps, double* __res
         c1[idx] = cq + 0.5 * (T2[idx] + T2[j * g + i]);
     }
     __syncthreads();
-    const double pivc1 = chol_inverse(c1, Lw, c1inv, g);
+    const double pivc1 = spd_inverse(c1, Lw, c1inv, g);
     const double gain = mat_trace_prod(c1inv, T3, g, red);
     const double delta = Ds - gain;
     mat_mul(Cinv, false, P, true, Q1, g);                             // Q1 = Cinv y_r = Cinv P^T
@@ -613,7 +613,7 @@ __global__ void k_pair_slots(Ptrs p)
         M[idx] = 0.5 * ((double)p.Hinv[(s * g + i) * p.ldh + s * g + j] + (double)p.Hinv[(s * g + j) * p.ldh + s * g + i]);
     }
     __syncthreads();
-    const double piv = chol_inverse(M, Lw, Cinv, g);
+    const double piv = spd_inverse(M, Lw, Cinv, g);
     const double* GV = p.gramV + s * gg;
     mat_mul(Cinv, false, GV, false, T, g);
     mat_mul(T, false, Cinv, false, KK, g);
@@ -660,7 +660,7 @@ k_pair_delta(Ptrs p, const float* __restrict__ Pm, int64_t ldpm, const float* __
             RR[idx] += p.gramR[t * gg + idx] + TMP[idx] + TMP[j * g + i];
         }
         __syncthreads();
-        const double piv = chol_inverse(c1, Lw, OUT, g);
+        const double piv = spd_inverse(c1, Lw, OUT, g);
         const double gain = mat_trace_prod(OUT, RR, g, red);
         if (threadIdx.x == 0) p.pairDelta[pair] = piv > 0.0 ? Ds - gain : INFINITY;
         __syncthreads();

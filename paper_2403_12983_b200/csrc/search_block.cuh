@@ -213,7 +213,7 @@ k_blk_small(Ptrs p, BlockPtrs bp, int accept_mode, double accept_tol, double* __
     __syncthreads();
     for (int idx = threadIdx.x; idx < gg; idx += blockDim.x) smw[idx] = C[idx];
     __syncthreads();
-    const double pivC = chol_inverse(smw, smw + gg, Cinv, g);
+    const double pivC = spd_inverse(smw, smw + gg, Cinv, g);
     const double Ds = mat_trace_prod(Cinv, GV, g, red);               // Tr(C^-1 V_r V_r^T)
     blk_mat_mul(Cinv, false, GX, false, T1, g, smw);                           // K R_q^T
     blk_mat_mul(P, false, T1, false, T2, g, smw);                              // P K R_q^T
@@ -248,7 +248,7 @@ k_blk_small(Ptrs p, BlockPtrs bp, int accept_mode, double accept_tol, double* __
     }
     for (int idx = threadIdx.x; idx < gg; idx += blockDim.x) smw[idx] = c1[idx];
     __syncthreads();
-    const double pivc1 = chol_inverse(smw, smw + gg, c1inv, g);
+    const double pivc1 = spd_inverse(smw, smw + gg, c1inv, g);
     const double gain = mat_trace_prod(c1inv, T3, g, red);
     const double delta = Ds - gain;
     blk_mat_mul(Cinv, false, P, true, Q1, g, smw);                             // Q1 = Cinv P^T

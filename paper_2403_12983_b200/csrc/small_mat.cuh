@@ -21,7 +21,7 @@ static __device__ __forceinline__ double warp_sum(double v) {
 // M is overwritten (keep it in shared memory where possible); Out receives the symmetrised inverse; Lw: scratch of
 // at least 2 g doubles.  Returns the smallest pivot, i.e. the smallest diagonal entry of the successive Schur
 // complements = the squared diagonal of the Cholesky factor (<= 0 when M is not positive definite).
-static __device__ double chol_inverse(double* M, double* Lw, double* Out, int g)
+static __device__ double spd_inverse(double* M, double* Lw, double* Out, int g)
 {
     __shared__ double minpiv;
     const int t = threadIdx.x, nt = blockDim.x;

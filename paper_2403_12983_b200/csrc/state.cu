@@ -380,7 +380,7 @@ int select_support(osscar_ctx* ctx, int mode, int32_t* support)
 }
 
 // In-place inverse of the n x n SPD matrix A (row stride lda) by the blocked exchange (Gauss-Jordan) scheme:
-// per 64-wide pivot block an fp64 Cholesky inverse, then one rank-64 update of the whole matrix in a GEMM.
+// per 64-wide pivot block an fp64 Gauss-Jordan inverse in shared memory, then one rank-64 update of the whole matrix in a GEMM.
 // `ref` (row stride ldref) supplies the original diagonal, the scale of the positive-definiteness test.
 int invert_spd_inplace(osscar_ctx* ctx, float* A, int64_t lda, int64_t n, const float* ref, int64_t ldref, const int32_t* done)
 {
