@@ -102,13 +102,8 @@ cudaError_t sgemm(cudaStream_t st, bool transA, bool transB, int64_t M, int64_t 
                   float alpha, const float* A, int64_t lda, const float* B, int64_t ldb,
                   float beta, float* C, int64_t ldc, const int32_t* done = nullptr);
 
-// ---- panel.cu: Y[i*so_row + e*so_col] = sum_k A[i][k] * P[e][k]; A is M x K (streamed once), P an N x K panel --------
-// `scratch` (may be null) holds partial sums when the k range is split to fill the machine.
-cudaError_t panel_dot(cudaStream_t st, int64_t M, int64_t N, int64_t K, const float* A, int64_t lda,
-                      const float* P, int64_t ldp, float* Y, int64_t so_row, int64_t so_col,
-                      float* scratch, size_t scratch_floats, const int32_t* done = nullptr);
-
-// ---- panel_tc.cu: the same product on the tensor cores; A is split into bf16 terms on the way (fp32-accurate) -------
+// ---- panel_tc.cu: Y[i*so_row + e*so_col] = sum_k A[i][k] * P[e][k] on the tensor cores; A (M x K, streamed once) is split
+// into bf16 terms on the way (fp32-accurate); P is an N x K panel
 // A 16-byte aligned with lda % 4 == 0; scratch at least panel_dot_tc_scratch bytes.
 size_t panel_dot_tc_scratch(int64_t M, int64_t N, int64_t K);
 cudaError_t panel_dot_tc(cudaStream_t st, int64_t M, int64_t N, int64_t K, const float* A, int64_t lda,

@@ -786,6 +786,7 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
     if (block) {
         if (pair || (int64_t)bs * g > L.block_rows_max || bs > L.k || bs > L.ng - L.k) return OSSCAR_E_ARG;
         if (block_bytes_for(L, bs * g) > L.block_bytes) return OSSCAR_E_WORKSPACE;
+        if (panel_dot_tc_scratch(L.nJ > L.nI ? L.nJ : L.nI, 2 * bs * g, L.nI) + 1024 > L.tc_bytes) return OSSCAR_E_WORKSPACE;
     }
     BlockPtrs bp = make_block_ptrs(ctx, bs);
     const bool fast = g == 1 && !pair && !block;  // fused five-launch step for single-row groups

@@ -525,20 +525,15 @@ cudaError_t enqueue_block_step(osscar_ctx* ctx, const Ptrs& p, const BlockPtrs& 
 #define BK(x) do { e = (x); if (e != cudaSuccess) return e; } while (0)
     k_blk_select<<<2, 1024, 0, st>>>(p, bp);                                                    mark();
     k_blk_gather<<<dim3((unsigned)G, 5), 256, 0, st>>>(p, bp);
-    float* big = (float*)((char*)ctx->ws + L.off_big);          // free between refreshes: partial sums of split products
-    const size_t big_floats = (L.off_Hp - L.off_big) / sizeof(float);
-    void* tc = (char*)ctx->ws + L.off_tc;
+    void* tc = (char*)ctx->ws + L.off_tc;                       // free between state builds: bf16 terms and partial sums
     int32_t* stat = &ctx->ctl->status;
-    const bool use_tc = L.tc_bytes >= panel_dot_tc_scratch(L.nJ > L.nI ? L.nJ : L.nI, 2 * G, L.nI);
-    if (use_tc) BK(panel_dot_tc(st, L.nI, G, L.nI, p.Hinv, L.ldh, bp.hT, L.ldh, bp.yT, 1, L.ldh, tc, L.tc_bytes, stat, done));
-    else BK(panel_dot(st, L.nI, G, L.nI, p.Hinv, L.ldh, bp.hT, L.ldh, bp.yT, 1, L.ldh, big, big_floats, done));     mark();   // y^T (Hinv symmetric)
+    BK(panel_dot_tc(st, L.nI, G, L.nI, p.Hinv, L.ldh, bp.hT, L.ldh, bp.yT, 1, L.ldh, tc, L.tc_bytes, stat, done));     mark();   // y^T (Hinv symmetric)
     k_blk_gram<<<(unsigned)((4 * G * G + 7) / 8), 256, 0, st>>>(p, bp);
     k_blk_small<<<1, 1024, 2 * (size_t)G * G * sizeof(double), st>>>(p, bp, accept_mode, tol, obj_trace, swap_trace);
     k_blk_prep<<<(unsigned)(((L.ldh + L.ldm) * G + 255) / 256), 256, 0, st>>>(p, bp);
     k_blk_zero_r<<<(unsigned)((G * G + 255) / 256), 256, 0, st>>>(p, bp);                        mark();
     // H pass: [u | H u2] for the pruned rows and the leaving rows, then -d
-    if (use_tc) BK(panel_dot_tc(st, L.nJ, 2 * G, L.nI, p.Hp + L.nI * L.ldp, L.ldp, bp.PB, L.ldh, bp.UD, 2 * G, 1, tc, L.tc_bytes, stat, done));
-    else BK(panel_dot(st, L.nJ, 2 * G, L.nI, p.Hp + L.nI * L.ldp, L.ldp, bp.PB, L.ldh, bp.UD, 2 * G, 1, big, big_floats, done));
+    BK(panel_dot_tc(st, L.nJ, 2 * G, L.nI, p.Hp + L.nI * L.ldp, L.ldp, bp.PB, L.ldh, bp.UD, 2 * G, 1, tc, L.tc_bytes, stat, done));
     k_blk_leave_d<<<(unsigned)((G * G + 7) / 8), 256, 0, st>>>(p, bp);
     k_blk_finish_d<<<(unsigned)(((L.nJ + G) * G + 255) / 256), 256, 0, st>>>(p, bp);            mark();
     // the three rank-2G updates; the residual rows of the leaving groups go through the Rq panel
