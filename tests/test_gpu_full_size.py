@@ -109,3 +109,8 @@ def test_c2_full_size_block_exchange_properties():
 def test_c5_full_size_block_exchange_properties():
     res = _run("c5", n_cols=2, max_swaps=600, block_pairs=50)
     assert res.n_swaps == 600 or res.stop_reason == "no_improvement"
+
+
+def test_c6_pointwise_conv_full_size_properties():
+    res = _run("c6", n_cols=4, max_swaps=500)
+    assert res.stop_reason in ("no_improvement", "max_swaps")

@@ -322,6 +322,7 @@ def test_dropped_rows_vanish_case1():
     ("c2", dict(n=2048, d1=256, m=64, k=128, chunk_rows=2048)),
     ("c5", dict(n=2048, d1=256, m=64, k=77, chunk_rows=2048)),
     ("c4", dict(n=49 * 16, d1=9 * 48, m=32, k=24, chunk_rows=49 * 16)),
+    ("c6", dict(n=49 * 40, d1=128, m=48, k=64, chunk_rows=49 * 10)),
 ])
 def test_strict_and_lowrank_follow_the_same_sequence(name, over):
     wl = workloads.config(name, **over)
@@ -396,6 +397,10 @@ def test_workloads_are_reproducible_and_shaped():
     assert np.mean(x4[:, 4] == 0) == pytest.approx(0.5, abs=0.12)
     # zero padding: the top-left tap of the first patch of an image is outside the map
     assert x4[0, 0] == 0 and x4[49, 0] == 0
+    c6 = workloads.config("c6", n=49 * 6, d1=32, m=8, k=16, chunk_rows=49 * 2)
+    x6 = c6.x_full().numpy()
+    assert x6.shape == (294, 32) and x6.min() >= 0 and 0.3 < np.mean(x6 == 0) < 0.7 and c6.n_chunks == 3
+    assert np.array_equal(x6[98:196], c6.x_chunk(1).numpy())
 
 
 # ----------------------------------------------------------------------------- nested (greedy) phase

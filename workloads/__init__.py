@@ -33,7 +33,7 @@ class Workload:
     """Description of one synthetic layer; activations come from `x_chunks()`."""
 
     name: str
-    kind: str                 # "dense_mix" | "fc2_relu" | "attn_heads" | "conv_unfold"
+    kind: str                 # "dense_mix" | "fc2_relu" | "attn_heads" | "conv_unfold" | "conv1x1"
     n: int                    # calibration rows (tokens / patches)
     d1: int                   # rows of W (inputs)
     m: int                    # columns of W (outputs)
@@ -70,7 +70,7 @@ class Workload:
             return self._shared_cache[1]
         gen = torch.Generator(device="cpu").manual_seed(self.seed * 1_000_003 + 23)
         out = {}
-        if self.kind == "dense_mix":
+        if self.kind in ("dense_mix", "conv1x1"):
             E = torch.randn(self.d1, self.d1, generator=gen, dtype=torch.float32) / math.sqrt(self.d1)
             out["A"] = (torch.eye(self.d1) + self.params.get("mix", 0.3) * E).to(device)
         elif self.kind == "fc2_relu":
@@ -128,6 +128,13 @@ class Workload:
             cols = torch.nn.functional.unfold(F, (kh, kw), padding=self.params["pad"], stride=1)
             # cols: imgs x (cin*kh*kw) x (fh*fw), row index of the middle axis = c*kh*kw + i*kw + j
             X = cols.transpose(1, 2).reshape(imgs * fh * fw, self.d1)
+        elif self.kind == "conv1x1":
+            # pointwise convolution: every pixel of the cin-channel feature map is one row; channels are mixed by a
+            # fixed random matrix before the ReLU so that they are correlated, as the outputs of a depthwise stage are
+            cin, fh, fw = self.d1, self.params["fh"], self.params["fw"]
+            imgs = rows // (fh * fw)
+            F = torch.relu_(randn(imgs * fh * fw, cin) @ sh["A"])
+            X = F
         else:
             raise ValueError(self.kind)
         if "scale" in sh:
@@ -162,7 +169,7 @@ class Workload:
 
 # ---------------------------------------------------------------------- named configurations
 def config(name: str, seed: int = 0, **over) -> Workload:
-    """The five named layer shapes (c1..c5) and scaled-down relatives.
+    """The named layer shapes (c1..c5 of the headline set, c6 a pointwise convolution) and scaled-down relatives.
 
     `over` replaces any Workload field (e.g. n=4096, d1=1024) to get a smaller
     problem with the same value structure.
@@ -186,6 +193,10 @@ def config(name: str, seed: int = 0, **over) -> Workload:
         wl = Workload("c5", "fc2_relu", n=262144, d1=28672, m=7168, g=1, k=8602, max_swaps=5000,
                       x_dtype=torch.bfloat16, damp=1e-2, eps_acc=1e-7,
                       params={"rank": 64, "rho": 1.0, "outlier_frac": 0.005, "outlier_scale": 30.0})
+    elif name == "c6":    # MobileNetV1-shaped pointwise (1x1) convolution: input channels, 500 images of 7 x 7
+        wl = Workload("c6", "conv1x1", n=500 * 49, d1=1024, m=1024, g=1, k=512, max_swaps=500,
+                      x_dtype=torch.float32, w_std=math.sqrt(2.0 / 1024.0), chunk_rows=100 * 49,
+                      params={"mix": 0.5, "fh": 7, "fw": 7})
     else:
         raise ValueError(name)
     wl.seed = seed
@@ -194,6 +205,9 @@ def config(name: str, seed: int = 0, **over) -> Workload:
             wl.params.update(val)
         else:
             setattr(wl, key, val)
+    if wl.kind == "conv1x1":
+        hw = wl.params["fh"] * wl.params["fw"]
+        assert wl.n % hw == 0 and wl.chunk_rows % hw == 0, "conv chunks must hold whole images"
     if wl.kind == "conv_unfold":
         hw = wl.params["fh"] * wl.params["fw"]
         assert wl.n % hw == 0 and wl.chunk_rows % hw == 0, "conv chunks must hold whole images"
