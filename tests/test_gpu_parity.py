@@ -341,6 +341,8 @@ BLOCK_CASES = [
     ("c5", dict(n=8192, d1=1000, m=300, k=300, chunk_rows=4096), 0, 50, 500, False),
     ("c5", dict(n=4096, d1=520, m=150, k=156, chunk_rows=4096), 2, 96, 960, True),
     ("c6", dict(n=49 * 60, d1=320, m=136, k=160, chunk_rows=49 * 20), 0, 8, 160, False),
+    ("c2", dict(n=1024, d1=64, m=16, k=60, chunk_rows=1024), 0, 4, 8, True),        # every pruned group enters
+    ("c2", dict(n=1024, d1=64, m=16, k=3, chunk_rows=1024), 0, 3, 6, True),         # every kept group leaves
     ("c4", dict(n=49 * 40, d1=9 * 100, m=130, k=50, chunk_rows=49 * 40), 0, 2, 60, False),
     ("c4", dict(n=49 * 40, d1=9 * 100, m=130, k=50, chunk_rows=49 * 40), 1, 5, 40, True),
     ("c3", dict(n=8192, d1=12 * 40, m=200, g=40, k=6, chunk_rows=8192, score_mode="independent"), 0, 2, 12, True),
