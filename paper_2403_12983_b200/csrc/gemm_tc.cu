@@ -317,8 +317,11 @@ __global__ void k_split3(const float* __restrict__ src, int64_t lds, int64_t row
 {
     if (done && *done) return;
     const int64_t total = rows * ldd;
+    const bool small = total < (int64_t)0x7fffffff;          // 32-bit index arithmetic where it fits (64-bit division is slow)
     for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
-        const int64_t r = idx / ldd, c = idx % ldd;
+        int64_t r, c;
+        if (small) { const uint32_t i32 = (uint32_t)idx, l32 = (uint32_t)ldd; r = i32 / l32; c = i32 % l32; }
+        else { r = idx / ldd; c = idx % ldd; }
         float x = c < cols ? src[r * lds + c] : 0.f;
         const __nv_bfloat16 a = __float2bfloat16_rn(x);
         x -= __bfloat162float(a);
