@@ -1,4 +1,4 @@
-"""Full-size checks (BASELINE c2 and c5 shapes, the launch configuration bench.py times).
+"""Full-size checks (the c2, c5 and c6 shapes, in the launch configuration bench.py times).
 
 The oracle cannot form H at these sizes in test time, so the checks are properties that hold at any size,
 evaluated on the oracle side from X itself on sampled outputs:
