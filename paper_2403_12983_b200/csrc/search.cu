@@ -501,40 +501,60 @@ __global__ void __launch_bounds__(256) k_update_rows(Ptrs p, int kind)
     }
 }
 
+// C += sign * A * B^T (all g x g, ld g) on the fp64 tensor-core path; each entry of C is owned by one lane.
+__device__ void mat_mul_nt_acc(const double* A, const double* B, double* C, int g, double sign)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    const int nt = (g + 7) >> 3, r4 = lane >> 2, c4 = lane & 3;
+    for (int tile = warp; tile < nt * nt; tile += nwarps) {
+        const int i0 = (tile / nt) * 8, j0 = (tile % nt) * 8;
+        const int ai = i0 + r4, bj = j0 + r4;
+        double d0 = 0.0, d1 = 0.0;
+        for (int k0 = 0; k0 < g; k0 += 4) {
+            const int kk = k0 + c4;
+            const double a = (kk < g && ai < g) ? A[ai * g + kk] : 0.0;
+            const double b = (kk < g && bj < g) ? B[bj * g + kk] : 0.0;
+            asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0, %1}, {%2}, {%3}, {%0, %1};"
+                         : "+d"(d0), "+d"(d1) : "d"(a), "d"(b));
+        }
+        const int ci = i0 + r4, cj = j0 + 2 * c4;
+        if (ci < g) {
+            if (cj < g) C[ci * g + cj] += sign * d0;
+            if (cj + 1 < g) C[ci * g + cj + 1] += sign * d1;
+        }
+    }
+    __syncthreads();
+}
+
 // c_l' = c_l + u_l C^-1 u_l^T - d_l c1^-1 d_l^T for every pruned slot (g > 1); the entering slot receives
-// the leaving group: c' = C^-1 - d_r c1^-1 d_r^T.  One block per pruned slot; T = u_l C^-1 and d_l c1^-1 are
-// staged in shared memory (2 g^2 doubles) so the work is O(g^3) per slot.
+// the leaving group: c' = C^-1 - d_r c1^-1 d_r^T.  One block per pruned slot; u_l (then d_l) and its product
+// with C^-1 (c1^-1) sit in shared memory (2 g^2 doubles), the four g x g products run on the fp64 tensor-core path.
 __global__ void __launch_bounds__(256) k_update_c(Ptrs p)
 {
     if (p.ctl->done) return;
     extern __shared__ double smc[];
     const int g = p.g, gg = g * g;
-    double* TU = smc; double* TD = smc + gg;
+    double* X = smc; double* T = smc + gg;
     const int64_t t = blockIdx.x;
     const bool special = t == p.ctl->sel_t;
     const double* Cinv = p.small + S_CINV * gg;
     const double* c1inv = p.small + S_C1INV * gg;
     const float* ul = p.u + (special ? p.nJ : t * g) * g;     // g x g, row a = row of the group
     const float* dl = p.d + (special ? p.nJ : t * g) * g;
-    for (int idx = threadIdx.x; idx < gg; idx += blockDim.x) {
-        const int a = idx / g, f = idx % g;
-        double tu = 0.0, td = 0.0;
-        for (int e = 0; e < g; ++e) {
-            if (!special) tu += (double)ul[a * g + e] * Cinv[e * g + f];
-            td += (double)dl[a * g + e] * c1inv[e * g + f];
-        }
-        TU[idx] = tu; TD[idx] = td;
+    double* c = p.c + t * gg;
+    if (special) {
+        for (int idx = threadIdx.x; idx < gg; idx += blockDim.x) c[idx] = Cinv[idx];
+    } else {
+        for (int idx = threadIdx.x; idx < gg; idx += blockDim.x) X[idx] = (double)ul[idx];
+        __syncthreads();
+        mat_mul(X, false, Cinv, false, T, g);                 // u_l C^-1
+        mat_mul_nt_acc(T, X, c, g, 1.0);
     }
     __syncthreads();
-    for (int idx = threadIdx.x; idx < gg; idx += blockDim.x) {
-        const int a = idx / g, b2 = idx % g;
-        double s = special ? Cinv[idx] : p.c[t * gg + idx];
-        for (int f = 0; f < g; ++f) {
-            if (!special) s += TU[a * g + f] * (double)ul[b2 * g + f];
-            s -= TD[a * g + f] * (double)dl[b2 * g + f];
-        }
-        p.c[t * gg + idx] = s;      // each thread reads only its own old entry
-    }
+    for (int idx = threadIdx.x; idx < gg; idx += blockDim.x) X[idx] = (double)dl[idx];
+    __syncthreads();
+    mat_mul(X, false, c1inv, false, T, g);                    // d_l c1^-1
+    mat_mul_nt_acc(T, X, c, g, -1.0);
 }
 
 // Exchange the rows (phase 0) or columns (phase 1) of Hp that belong to the leaving and entering groups;
