@@ -346,7 +346,8 @@ constexpr uint32_t kRuIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | 
 
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 k_rank_update(const __grid_constant__ Maps maps, int64_t M, int64_t N, int nkb, float alpha, float* __restrict__ C, int64_t ldc,
-              int TN, int nchunk, int num_items, int32_t* __restrict__ status, const int32_t* __restrict__ done)
+              int TN, int nchunk, int num_items, float* __restrict__ sq_part, int32_t* __restrict__ status,
+              const int32_t* __restrict__ done)
 {
     if (done && *done) return;
     extern __shared__ uint8_t smem_raw[];
@@ -494,6 +495,9 @@ k_rank_update(const __grid_constant__ Maps maps, int64_t M, int64_t N, int nkb, 
                 asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
                 __syncwarp();
                 if (lane == 0) mbar_arrive(tempty_bar(buf));
+                float sq[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) sq[q] = 0.f;
 #pragma unroll
                 for (int c = 0; c < 2; ++c) {
                     const int64_t gc = gcol0 + c * 32 + c4;
@@ -512,9 +516,20 @@ k_rank_update(const __grid_constant__ Maps maps, int64_t M, int64_t N, int nkb, 
                         const int r = q * 4 + rsub;
                         const int64_t gr = grow0 + r;
                         const float* sp = stg + r * EPI_LD + c4;
-                        if (gr < M && gc < N)
-                            *reinterpret_cast<float4*>(C + gr * ldc + gc) =
-                                make_float4(o[q].x + sp[0], o[q].y + sp[1], o[q].z + sp[2], o[q].w + sp[3]);
+                        const float4 v = make_float4(o[q].x + sp[0], o[q].y + sp[1], o[q].z + sp[2], o[q].w + sp[3]);
+                        if (gr < M && gc < N) {
+                            *reinterpret_cast<float4*>(C + gr * ldc + gc) = v;
+                            sq[q] += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+                        }
+                    }
+                }
+                if (sq_part) {           // squared norm of the new row segment (64 columns): one partial per row and segment
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        float v = sq[q];
+                        v += __shfl_xor_sync(0xffffffffu, v, 1); v += __shfl_xor_sync(0xffffffffu, v, 2); v += __shfl_xor_sync(0xffffffffu, v, 4);
+                        const int64_t gr = grow0 + q * 4 + rsub;
+                        if ((lane & 7) == 0 && gr < M) sq_part[gr * (2 * TN) + 2 * tn + half] = v;
                     }
                 }
             }
@@ -602,13 +617,32 @@ cudaError_t gemm_tc(cudaStream_t st, int64_t M, int64_t N, int64_t K, float alph
     return cudaSuccess;
 }
 
+}  // namespace osscar (reopened below)
+namespace osscar {
+namespace {
+// norm[row] = sum of the row's partials, in segment order.
+__global__ void k_rownorm_sum(const float* __restrict__ part, int64_t rows, int nseg, float* __restrict__ norm, const int32_t* __restrict__ done)
+{
+    if (done && *done) return;
+    const int64_t r = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= rows) return;
+    float s = 0.f;
+    for (int j = 0; j < nseg; ++j) s += part[r * nseg + j];
+    norm[r] = s;
+}
+}  // namespace
+
 // C += alpha * U * W for a short inner dimension (see k_rank_update); falls back to the generic product otherwise.
+// With `row_sq` (M floats) and `sq_scratch` (M * 2 * ceil(N / 128) floats) the squared norms of the updated rows come
+// out of the same pass (short-dimension path only; returns cudaErrorInvalidValue otherwise).
 cudaError_t rank_update_tc(cudaStream_t st, int64_t M, int64_t N, int64_t K, float alpha, const float* U, int64_t ldu,
                            const float* W, int64_t ldw, float* C, int64_t ldc,
-                           void* scratch, size_t scratch_bytes, int32_t* status_dev, const int32_t* done)
+                           void* scratch, size_t scratch_bytes, int32_t* status_dev, const int32_t* done,
+                           float* row_sq, float* sq_scratch)
 {
     if (M <= 0 || N <= 0 || K <= 0) return cudaSuccess;
     const bool fits = K <= 2 * BLOCK_K && (N % 4) == 0 && (ldc % 4) == 0 && (((uintptr_t)C & 15) == 0);
+    if (!fits && row_sq) return cudaErrorInvalidValue;
     if (!fits) return gemm_tc(st, M, N, K, alpha, U, ldu, W, ldw, 1.f, C, ldc, scratch, scratch_bytes, status_dev, done);
     PFN_encodeTiled enc = get_encode();
     if (!enc) return cudaErrorNotSupported;
@@ -645,8 +679,12 @@ cudaError_t rank_update_tc(cudaStream_t st, int64_t M, int64_t N, int64_t K, flo
     const int num_items = TM * nchunk;
     const int nkb = (int)((K + BLOCK_K - 1) / BLOCK_K);
     k_rank_update<<<num_items < sms ? num_items : sms, NUM_THREADS, RU_SMEM, st>>>(maps, M, N, nkb, alpha, C, ldc, TN, nchunk, num_items,
-                                                                                  status_dev, done);
+                                                                                  row_sq ? sq_scratch : nullptr, status_dev, done);
     count_launches(3);
+    if (row_sq) {
+        k_rownorm_sum<<<(unsigned)((M + 255) / 256), 256, 0, st>>>(sq_scratch, M, 2 * TN, row_sq, done);
+        count_launches(1);
+    }
     return cudaGetLastError();
 }
 

@@ -118,10 +118,12 @@ cudaError_t gemm_tc(cudaStream_t st, int64_t M, int64_t N, int64_t K, float alph
                     void* scratch, size_t scratch_bytes, int32_t* status_dev, const int32_t* done = nullptr);
 
 // C += alpha * A * B for a short inner dimension (K <= 128 keeps the terms of A's row band in shared memory across a run
-// of column tiles; larger K goes through gemm_tc).  Same operands and scratch as gemm_tc.
+// of column tiles; larger K goes through gemm_tc).  Same operands and scratch as gemm_tc.  With row_sq (M floats) and
+// sq_scratch (M * 2 * ceil(N / 128) floats) the squared norms of the updated rows are produced in the same pass (K <= 128 only).
 cudaError_t rank_update_tc(cudaStream_t st, int64_t M, int64_t N, int64_t K, float alpha, const float* A, int64_t lda,
                            const float* B, int64_t ldb, float* C, int64_t ldc,
-                           void* scratch, size_t scratch_bytes, int32_t* status_dev, const int32_t* done = nullptr);
+                           void* scratch, size_t scratch_bytes, int32_t* status_dev, const int32_t* done = nullptr,
+                           float* row_sq = nullptr, float* sq_scratch = nullptr);
 
 // H (+)= Xc^T Xc (upper-triangle tiles; Y null) or G (+)= Xc^T Yc with the drained-accumulator pipeline of gemm_tc.cu.
 cudaError_t gram_tc2(cudaStream_t st, const void* X, int64_t n_rows, int64_t d1, const void* Y, int y_fp32, int64_t m,

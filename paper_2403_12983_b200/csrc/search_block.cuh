@@ -399,9 +399,18 @@ __global__ void __launch_bounds__(256) k_blk_fix(Ptrs p, BlockPtrs bp)
     }
     const float* vq = bp.KV + (int64_t)(G + t) * p.ldm;
     const float* rn = bp.Rq + (int64_t)t * p.ldm;
+    float sv = 0.f, sr = 0.f;
     for (int64_t c = threadIdx.x; c < p.m; c += blockDim.x) {
-        p.V[row * p.ldm + c] = vq[c];
-        p.R[qrow * p.ldm + c] = rn[c];
+        const float a = vq[c], b = rn[c];
+        p.V[row * p.ldm + c] = a;
+        p.R[qrow * p.ldm + c] = b;
+        sv = fmaf(a, a, sv); sr = fmaf(b, b, sr);
+    }
+    if (p.g == 1) {                      // single-row groups are scored from the row norms
+        __shared__ float red[32];
+        sv = block_sum_f(sv, red);
+        sr = block_sum_f(sr, red);
+        if (threadIdx.x == 0) { p.vnorm[row] = sv; p.rnorm[qrow] = sr; }
     }
 }
 
@@ -538,8 +547,15 @@ cudaError_t enqueue_block_step(osscar_ctx* ctx, const Ptrs& p, const BlockPtrs& 
     k_blk_finish_d<<<(unsigned)(((L.nJ + G) * G + 255) / 256), 256, 0, st>>>(p, bp);            mark();
     // the three rank-2G updates; the residual rows of the leaving groups go through the Rq panel
     BK(rank_update_tc(st, L.nI, L.ldh, 2 * G, -1.f, bp.PAT, 2 * G, bp.PB, L.ldh, p.Hinv, L.ldh, tc, L.tc_bytes, stat, done));   mark();
-    BK(rank_update_tc(st, L.nI, L.ldm, 2 * G, -1.f, bp.PBT, 2 * G, bp.KV, L.ldm, p.V, L.ldm, tc, L.tc_bytes, stat, done));       mark();
-    BK(rank_update_tc(st, L.nJ, L.ldm, 2 * G, 1.f, bp.UD, 2 * G, bp.KV, L.ldm, p.R, L.ldm, tc, L.tc_bytes, stat, done));
+    // single-row groups: the squared row norms of V' and R' (the next scores) come out of the update passes
+    float* sq = (float*)((char*)tc + (L.tc_bytes / 2 / 1024) * 1024);
+    const size_t sq_floats = (L.tc_bytes - (L.tc_bytes / 2 / 1024) * 1024) / sizeof(float);
+    const int64_t nseg = 2 * ((L.ldm + 127) / 128);
+    const bool fused_norms = L.g == 1 && 2 * G <= 128 && (size_t)((L.nJ > L.nI ? L.nJ : L.nI) * nseg) <= sq_floats;
+    BK(rank_update_tc(st, L.nI, L.ldm, 2 * G, -1.f, bp.PBT, 2 * G, bp.KV, L.ldm, p.V, L.ldm, tc, L.tc_bytes / 2, stat, done,
+                      fused_norms ? p.vnorm : nullptr, sq));                                                              mark();
+    BK(rank_update_tc(st, L.nJ, L.ldm, 2 * G, 1.f, bp.UD, 2 * G, bp.KV, L.ldm, p.R, L.ldm, tc, L.tc_bytes / 2, stat, done,
+                      fused_norms ? p.rnorm : nullptr, sq));
     BK(sgemm(st, false, false, G, L.m, 2 * G, 1.f, bp.UD + L.nJ * 2 * G, 2 * G, bp.KV, L.ldm, 0.f, bp.Rq, L.ldm, done));   mark();
     if (L.g == 1) k_blk_update_c_g1<<<296, 256, 2 * (size_t)G * G * sizeof(float), st>>>(p, bp);
     else k_blk_update_c<<<(unsigned)(L.ng - L.k), 128, 2 * (size_t)L.g * G * sizeof(double), st>>>(p, bp);
@@ -547,7 +563,7 @@ cudaError_t enqueue_block_step(osscar_ctx* ctx, const Ptrs& p, const BlockPtrs& 
     k_blk_hswap<<<(unsigned)((L.ldp * G + 255) / 256), 256, 0, st>>>(p, bp, 0);
     k_blk_hswap<<<(unsigned)((L.ldp * G + 255) / 256), 256, 0, st>>>(p, bp, 1);                 mark();
     count_launches(12);
-    BK(enqueue_scores(ctx, p, true, false));                                                   mark();
+    BK(enqueue_scores(ctx, p, !fused_norms, false));                                           mark();
 #undef BK
     return cudaGetLastError();
 }
