@@ -33,6 +33,10 @@ __device__ float block_sum_f(float v, float* red) {      // result in every thre
     return s;
 }
 
+__device__ __forceinline__ float dot4f(const float4& a, const float4& b) {
+    return a.x * b.x + a.y * b.y + a.z * b.z + a.w * b.w;
+}
+
 struct Ptrs {
     float *Hp, *Hinv, *V, *R, *y, *b, *u2, *bC, *u2c, *u, *d, *K, *Vq, *vnorm, *rnorm;
     double *D, *A, *c, *small, *gramV, *gramR;
@@ -62,36 +66,55 @@ __global__ void k_row_norms(const float* __restrict__ M, int64_t ld, float* __re
     if (threadIdx.x == 0) norm[blockIdx.x] = acc;
 }
 
-// gram[grp][a][b] = M[grp*g+a,:] . M[grp*g+b,:]; grid (groups, g), warps loop over b.
-__global__ void k_group_gram(const float* __restrict__ M, int64_t ld, int g, double* __restrict__ gram, const SearchCtl* ctl)
+// gram[grp][a][b] = M[grp*g+a,:] . M[grp*g+b,:] for the kept groups (rows of V -> gramV) and the pruned groups (rows of
+// R -> gramR) in one launch.  Grid (ng, ceil(g / GG_AT)): blocks [0, k) take kept slots, the rest pruned slots; a block
+// owns GG_AT rows a of its group, its warps loop over the rows b >= the first of them, and each streamed piece of row b
+// meets the GG_AT rows a (cache resident) at once; the lower triangle is written as the mirror image.
+constexpr int GG_AT = 4;
+__global__ void __launch_bounds__(256) k_group_gram(Ptrs p)
 {
-    if (ctl->done) return;
-    const int64_t grp = blockIdx.x;
-    const int a = blockIdx.y;
+    if (p.ctl->done) return;
+    const int g = p.g;
+    const bool kept = (int)blockIdx.x < p.k;
+    const int64_t grp = kept ? blockIdx.x : blockIdx.x - p.k;
+    const float* M = (kept ? p.V : p.R) + grp * g * p.ldm;
+    double* gram = (kept ? p.gramV : p.gramR) + grp * g * g;
+    const int64_t n4 = p.ldm / 4;
+    const int a0 = blockIdx.y * GG_AT;
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
-    const float4* ra = reinterpret_cast<const float4*>(M + (grp * g + a) * ld);
-    for (int b = w; b < g; b += nw) {
-        const float4* rb = reinterpret_cast<const float4*>(M + (grp * g + b) * ld);
-        float s = 0.f;
-        for (int64_t c = lane; c < ld / 4; c += 32) {
-            const float4 x = ra[c], z = rb[c];
-            s += x.x * z.x + x.y * z.y + x.z * z.z + x.w * z.w;
+    const float4* ra[GG_AT];
+#pragma unroll
+    for (int i = 0; i < GG_AT; ++i) ra[i] = reinterpret_cast<const float4*>(M + (int64_t)(a0 + i < g ? a0 + i : a0) * p.ldm);
+    for (int b = a0 + w; b < g; b += nw) {
+        const float4* rb = reinterpret_cast<const float4*>(M + (int64_t)b * p.ldm);
+        float s[GG_AT];
+#pragma unroll
+        for (int i = 0; i < GG_AT; ++i) s[i] = 0.f;
+        for (int64_t c = lane; c < n4; c += 32) {
+            const float4 z = rb[c];
+#pragma unroll
+            for (int i = 0; i < GG_AT; ++i) s[i] += dot4f(ra[i][c], z);
         }
-        s = warp_sum(s);
-        if (lane == 0) gram[(grp * g + a) * g + b] = (double)s;
+#pragma unroll
+        for (int i = 0; i < GG_AT; ++i) {
+            const float t = warp_sum(s[i]);
+            const int a = a0 + i;
+            if (lane == 0 && a <= b) { gram[a * g + b] = (double)t; gram[b * g + a] = (double)t; }
+        }
     }
 }
 
 // Scores of groups of more than one row: score = Tr(M^-1 Gram); one block per group.
-// kind 0: kept slots (M = Hinv_rr, Gram of V rows) -> D; kind 1: pruned slots (M = c, Gram of R rows) -> A.
-__global__ void k_scores_general(Ptrs p, int kind)
+// Blocks [0, k): kept slots (M = Hinv_rr, Gram of V rows) -> D; the rest: pruned slots (M = c, Gram of R rows) -> A.
+__global__ void __launch_bounds__(1024) k_scores_general(Ptrs p)
 {
     if (p.ctl->done) return;
     extern __shared__ double smd[];
     const int g = p.g;
     double* M = smd; double* Lw = smd + g * g; double* Out = Lw + g * g;
     __shared__ double red[32];
-    const int64_t grp = blockIdx.x;
+    const int kind = (int)blockIdx.x < p.k ? 0 : 1;
+    const int64_t grp = kind == 0 ? blockIdx.x : blockIdx.x - p.k;
     double scale = 0.0;
     for (int idx = threadIdx.x; idx < g * g; idx += blockDim.x) {
         const int i = idx / g, j = idx % g;
@@ -220,26 +243,28 @@ __global__ void __launch_bounds__(256) k_pairgram(Ptrs p)
 }
 
 // One block: the g x g algebra of the step, the exact change of obj and the accept decision.
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(1024)
 k_small(Ptrs p, int accept_mode, double accept_tol, int max_swaps, double* __restrict__ obj_trace, int32_t* __restrict__ swap_trace)
 {
     SearchCtl* ctl = p.ctl;
     if (ctl->done) return;
     __shared__ double red[32];
+    extern __shared__ double smd[];             // g^2 + 2 g doubles: the matrix being inverted and the pivot row/column
     const int g = p.g, gg = g * g;
+    double* Ms = smd; double* Lws = smd + gg;
     double* S = p.small;
     double *Cinv = S + S_CINV * gg, *c1inv = S + S_C1INV * gg, *Q1 = S + S_Q1 * gg, *Q1c = S + S_Q1C * gg, *M2 = S + S_M2 * gg;
-    double *GV = S + S_GV * gg, *GX = S + S_GX * gg, *GR = S + S_GR * gg, *C = S + S_C * gg, *P = S + S_P * gg;
-    double *T1 = S + S_T1 * gg, *T2 = S + S_T2 * gg, *T3 = S + S_T3 * gg, *c1 = S + S_C1 * gg, *Lw = S + S_L * gg;
+    double *GV = S + S_GV * gg, *GX = S + S_GX * gg, *GR = S + S_GR * gg, *P = S + S_P * gg;
+    double *T1 = S + S_T1 * gg, *T2 = S + S_T2 * gg, *T3 = S + S_T3 * gg, *Lw = S + S_L * gg;
     const int64_t r0 = (int64_t)ctl->sel_slot * g;
     const int64_t tq = ctl->sel_t;
     for (int idx = threadIdx.x; idx < gg; idx += blockDim.x) {
         const int i = idx / g, j = idx % g;
-        C[idx] = 0.5 * ((double)p.Hinv[(r0 + i) * p.ldh + r0 + j] + (double)p.Hinv[(r0 + j) * p.ldh + r0 + i]);
+        Ms[idx] = 0.5 * ((double)p.Hinv[(r0 + i) * p.ldh + r0 + j] + (double)p.Hinv[(r0 + j) * p.ldh + r0 + i]);
         P[idx] = (double)p.y[(int64_t)i * p.ldh + r0 + j];           // P[a][b] = y_a[r_b]
     }
     __syncthreads();
-    const double pivC = spd_inverse(C, Lw, Cinv, g);
+    const double pivC = spd_inverse(Ms, Lws, Cinv, g);
     const double Ds = mat_trace_prod(Cinv, GV, g, red);               // Tr(C^-1 V_r V_r^T)
     // R1 R1^T = GR + P (Cinv GX) + (P Cinv GX)^T + P Cinv GV Cinv P^T
     mat_mul(Cinv, false, GX, false, T1, g);                           // K R_q^T
@@ -256,10 +281,10 @@ k_small(Ptrs p, int accept_mode, double accept_tol, int max_swaps, double* __res
     for (int idx = threadIdx.x; idx < gg; idx += blockDim.x) {
         const int i = idx / g, j = idx % g;
         const double cq = 0.5 * (p.c[tq * gg + idx] + p.c[tq * gg + j * g + i]);
-        c1[idx] = cq + 0.5 * (T2[idx] + T2[j * g + i]);
+        Ms[idx] = cq + 0.5 * (T2[idx] + T2[j * g + i]);
     }
     __syncthreads();
-    const double pivc1 = spd_inverse(c1, Lw, c1inv, g);
+    const double pivc1 = spd_inverse(Ms, Lws, c1inv, g);
     const double gain = mat_trace_prod(c1inv, T3, g, red);
     const double delta = Ds - gain;
     mat_mul(Cinv, false, P, true, Q1, g);                             // Q1 = Cinv y_r = Cinv P^T
@@ -371,134 +396,307 @@ __global__ void __launch_bounds__(256) k_hpass(Ptrs p)
     }
 }
 
-// Hinv' = Hinv - bC b^T + u2c u2^T; rows/columns of r take -u2c, the rr block c1^-1.
+// Single-row groups outside the fused five-launch step (exhaustive pair scoring with g = 1):
+// Hinv' = Hinv - bC b^T + u2c u2^T; row/column r takes -u2c, the corner 1/c1.
 // Block: 256 threads x float4 = 1024 columns, RT rows.
 constexpr int HI_RT = 8;
 __global__ void __launch_bounds__(256) k_update_hinv(Ptrs p)
 {
     if (p.ctl->done) return;
-    const int g = p.g;
     const int64_t c4 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;     // float4 column index
     if (c4 * 4 >= p.ldh) return;
     const int64_t col = c4 * 4;
-    const int64_t r0 = (int64_t)p.ctl->sel_slot * g;
+    const int64_t r0 = p.ctl->sel_slot;
     const int64_t row0 = (int64_t)blockIdx.y * HI_RT;
-    const double* c1inv = p.small + S_C1INV * g * g;
-    if (g == 1) {
-        const float4 bb = reinterpret_cast<const float4*>(p.b)[c4];
-        const float4 uu = reinterpret_cast<const float4*>(p.u2)[c4];
-        const float4 uc = reinterpret_cast<const float4*>(p.u2c)[c4];
+    const double* c1inv = p.small + S_C1INV;
+    const float4 bb = reinterpret_cast<const float4*>(p.b)[c4];
+    const float4 uu = reinterpret_cast<const float4*>(p.u2)[c4];
+    const float4 uc = reinterpret_cast<const float4*>(p.u2c)[c4];
 #pragma unroll
-        for (int i = 0; i < HI_RT; ++i) {
-            const int64_t s = row0 + i;
-            if (s >= p.nI) break;
-            float4* ptr = reinterpret_cast<float4*>(p.Hinv + s * p.ldh) + c4;
-            float4 h = *ptr;
-            if (s == r0) {
-                h.x = -uc.x; h.y = -uc.y; h.z = -uc.z; h.w = -uc.w;
-            } else {
-                const float nb = -p.bC[s], us = p.u2c[s];
-                h.x = fmaf(us, uu.x, fmaf(nb, bb.x, h.x));
-                h.y = fmaf(us, uu.y, fmaf(nb, bb.y, h.y));
-                h.z = fmaf(us, uu.z, fmaf(nb, bb.z, h.z));
-                h.w = fmaf(us, uu.w, fmaf(nb, bb.w, h.w));
-            }
-            float* hf = reinterpret_cast<float*>(&h);
-            if (r0 >= col && r0 < col + 4) hf[r0 - col] = (s == r0) ? (float)c1inv[0] : -p.u2c[s];
-            *ptr = h;
-        }
-        return;
-    }
     for (int i = 0; i < HI_RT; ++i) {
         const int64_t s = row0 + i;
         if (s >= p.nI) break;
         float4* ptr = reinterpret_cast<float4*>(p.Hinv + s * p.ldh) + c4;
         float4 h = *ptr;
-        float* hf = reinterpret_cast<float*>(&h);
-        const bool srow = s >= r0 && s < r0 + g;
-        for (int j = 0; j < 4; ++j) {
-            const int64_t sc = col + j;
-            const bool scol = sc >= r0 && sc < r0 + g;
-            float v;
-            if (srow && scol) v = (float)c1inv[(s - r0) * g + (sc - r0)];
-            else if (srow) v = -p.u2c[(s - r0) * p.ldh + sc];
-            else if (scol) v = -p.u2c[(sc - r0) * p.ldh + s];
-            else {
-                v = hf[j];
-                for (int e = 0; e < g; ++e) {
-                    v = fmaf(-p.bC[(int64_t)e * p.ldh + s], p.b[(int64_t)e * p.ldh + sc], v);
-                    v = fmaf(p.u2c[(int64_t)e * p.ldh + s], p.u2[(int64_t)e * p.ldh + sc], v);
-                }
-            }
-            hf[j] = v;
+        if (s == r0) {
+            h.x = -uc.x; h.y = -uc.y; h.z = -uc.z; h.w = -uc.w;
+        } else {
+            const float nb = -p.bC[s], us = p.u2c[s];
+            h.x = fmaf(us, uu.x, fmaf(nb, bb.x, h.x));
+            h.y = fmaf(us, uu.y, fmaf(nb, bb.y, h.y));
+            h.z = fmaf(us, uu.z, fmaf(nb, bb.z, h.z));
+            h.w = fmaf(us, uu.w, fmaf(nb, bb.w, h.w));
         }
+        float* hf = reinterpret_cast<float*>(&h);
+        if (r0 >= col && r0 < col + 4) hf[r0 - col] = (s == r0) ? (float)c1inv[0] : -p.u2c[s];
         *ptr = h;
     }
 }
 
-// Row updates of V (kind 0) and R (kind 1) with the squared row norm of the result (g = 1 scoring).
-//   V'[s] = V[s] - sum_e b[e][s] K[e] - sum_e u2[e][s] Vq[e]         (rows of r: Vq)
-//   R'[l] = R[l] + sum_e u[l][e] K[e] - sum_e d[l][e] Vq[e]          (rows of q: K[e] - sum_f d[nJ+e][f] Vq[f])
-// For g = 1 the R pass also moves c and the kept pass nothing else.  One block per ROWS rows.
+// Single-row groups outside the fused five-launch step: row updates of V (kind 0) and R (kind 1) with the squared
+// row norm of the result (the next scores).
+//   V'[s] = V[s] - b[s] K - u2[s] Vq   (row r: Vq)        R'[l] = R[l] + u[l] K - d[l] Vq   (row q: K - d[nJ] Vq)
+// The R pass also moves c.  One block per UP_ROWS rows.
 constexpr int UP_ROWS = 4;
 __global__ void __launch_bounds__(256) k_update_rows(Ptrs p, int kind)
 {
     if (p.ctl->done) return;
     __shared__ float red[32];
-    const int g = p.g;
     float* M = kind == 0 ? p.V : p.R;
     const int64_t nrows = kind == 0 ? p.nI : p.nJ;
-    const int64_t special0 = (kind == 0 ? (int64_t)p.ctl->sel_slot : (int64_t)p.ctl->sel_t) * g;
+    const int64_t special0 = kind == 0 ? (int64_t)p.ctl->sel_slot : (int64_t)p.ctl->sel_t;
     const int64_t n4 = p.ldm / 4;
     const int64_t row0 = (int64_t)blockIdx.x * UP_ROWS;
+    const float4* K4 = reinterpret_cast<const float4*>(p.K);
+    const float4* Q4 = reinterpret_cast<const float4*>(p.Vq);
     for (int i = 0; i < UP_ROWS; ++i) {
         const int64_t s = row0 + i;
         if (s >= nrows) break;
-        const bool special = s >= special0 && s < special0 + g;
+        const bool special = s == special0;
+        float ck, cq;
+        if (special) { ck = kind == 0 ? 0.f : 1.f; cq = kind == 0 ? 1.f : -p.d[p.nJ]; }
+        else { ck = kind == 0 ? -p.b[s] : p.u[s]; cq = kind == 0 ? -p.u2[s] : -p.d[s]; }
         float4* row = reinterpret_cast<float4*>(M + s * p.ldm);
         float nrm = 0.f;
         for (int64_t c = threadIdx.x; c < n4; c += blockDim.x) {
-            float4 v;
-            if (special) {
-                const int e = (int)(s - special0);
-                if (kind == 0) v = reinterpret_cast<const float4*>(p.Vq + (int64_t)e * p.ldm)[c];
-                else {
-                    v = reinterpret_cast<const float4*>(p.K + (int64_t)e * p.ldm)[c];
-                    for (int f = 0; f < g; ++f) {
-                        const float df = -p.d[(p.nJ + e) * g + f];
-                        const float4 q = reinterpret_cast<const float4*>(p.Vq + (int64_t)f * p.ldm)[c];
-                        v.x = fmaf(df, q.x, v.x); v.y = fmaf(df, q.y, v.y); v.z = fmaf(df, q.z, v.z); v.w = fmaf(df, q.w, v.w);
-                    }
-                }
-            } else {
-                v = row[c];
-                for (int e = 0; e < g; ++e) {
-                    const float ck = kind == 0 ? -p.b[(int64_t)e * p.ldh + s] : p.u[s * g + e];
-                    const float cq = kind == 0 ? -p.u2[(int64_t)e * p.ldh + s] : -p.d[s * g + e];
-                    const float4 kk = reinterpret_cast<const float4*>(p.K + (int64_t)e * p.ldm)[c];
-                    const float4 q = reinterpret_cast<const float4*>(p.Vq + (int64_t)e * p.ldm)[c];
-                    v.x = fmaf(cq, q.x, fmaf(ck, kk.x, v.x));
-                    v.y = fmaf(cq, q.y, fmaf(ck, kk.y, v.y));
-                    v.z = fmaf(cq, q.z, fmaf(ck, kk.z, v.z));
-                    v.w = fmaf(cq, q.w, fmaf(ck, kk.w, v.w));
-                }
-            }
+            float4 v = special ? make_float4(0.f, 0.f, 0.f, 0.f) : row[c];
+            const float4 kk = K4[c], q = Q4[c];
+            v.x = fmaf(cq, q.x, fmaf(ck, kk.x, v.x));
+            v.y = fmaf(cq, q.y, fmaf(ck, kk.y, v.y));
+            v.z = fmaf(cq, q.z, fmaf(ck, kk.z, v.z));
+            v.w = fmaf(cq, q.w, fmaf(ck, kk.w, v.w));
             row[c] = v;
             nrm += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
         }
-        if (g == 1) {
-            nrm = block_sum_f(nrm, red);
-            if (threadIdx.x == 0) {
-                if (kind == 0) p.vnorm[s] = nrm;
-                else {
-                    p.rnorm[s] = nrm;
-                    const double Cinv = p.small[S_CINV], c1inv = p.small[S_C1INV];
-                    if (special) { const double dd = p.d[p.nJ]; p.c[s] = Cinv - dd * dd * c1inv; }
-                    else { const double uu = p.u[s], dd = p.d[s]; p.c[s] += uu * uu * Cinv - dd * dd * c1inv; }
-                }
+        nrm = block_sum_f(nrm, red);
+        if (threadIdx.x == 0) {
+            if (kind == 0) p.vnorm[s] = nrm;
+            else {
+                p.rnorm[s] = nrm;
+                const double Cinv = p.small[S_CINV], c1inv = p.small[S_C1INV];
+                if (special) { const double dd = p.d[p.nJ]; p.c[s] = Cinv - dd * dd * c1inv; }
+                else { const double uu = p.u[s], dd = p.d[s]; p.c[s] += uu * uu * Cinv - dd * dd * c1inv; }
             }
         }
     }
+}
+
+// Groups of more than one row: y = Hinv h and the H pass as warp tiles of TP_R rows x TP_E right-hand sides, so that a
+// streamed piece of a matrix row meets TP_E vectors and a piece of a vector TP_R rows (the per-(row, vector) kernels
+// above re-read every row g times from L2).  Blocks of TP_W warps; grid (row tiles, ceil(g / TP_E)); TP_R is chosen per
+// launch so that small layers still fill the machine.
+constexpr int TP_E = 4, TP_W = 4;
+
+// y[e][s] = Hinv[s, :] . Hp[q_e, 0:n_I]
+template <int TP_R>
+__global__ void __launch_bounds__(32 * TP_W) k_ypass_g(Ptrs p)
+{
+    if (p.ctl->done) return;
+    const int g = p.g, e0 = blockIdx.y * TP_E;
+    const int lane = threadIdx.x & 31;
+    const int64_t s0 = ((int64_t)blockIdx.x * TP_W + (threadIdx.x >> 5)) * TP_R;
+    if (s0 >= p.nI) return;
+    const float4 *arow[TP_R], *hrow[TP_E];
+#pragma unroll
+    for (int i = 0; i < TP_R; ++i) arow[i] = reinterpret_cast<const float4*>(p.Hinv + (s0 + i < p.nI ? s0 + i : p.nI - 1) * p.ldh);
+#pragma unroll
+    for (int j = 0; j < TP_E; ++j)
+        hrow[j] = reinterpret_cast<const float4*>(p.Hp + (p.nI + (int64_t)p.ctl->sel_t * g + (e0 + j < g ? e0 + j : g - 1)) * p.ldp);
+    float acc[TP_R][TP_E];
+#pragma unroll
+    for (int i = 0; i < TP_R; ++i)
+#pragma unroll
+        for (int j = 0; j < TP_E; ++j) acc[i][j] = 0.f;
+    for (int64_t c = lane; c < p.ldh / 4; c += 32) {
+        float4 x[TP_R], h[TP_E];
+#pragma unroll
+        for (int i = 0; i < TP_R; ++i) x[i] = arow[i][c];
+#pragma unroll
+        for (int j = 0; j < TP_E; ++j) h[j] = __ldg(hrow[j] + c);
+#pragma unroll
+        for (int i = 0; i < TP_R; ++i)
+#pragma unroll
+            for (int j = 0; j < TP_E; ++j) acc[i][j] += dot4f(x[i], h[j]);
+    }
+#pragma unroll
+    for (int i = 0; i < TP_R; ++i)
+#pragma unroll
+        for (int j = 0; j < TP_E; ++j) {
+            const float t = warp_sum(acc[i][j]);
+            if (lane == 0 && s0 + i < p.nI && e0 + j < g) p.y[(int64_t)(e0 + j) * p.ldh + s0 + i] = t;
+        }
+}
+
+// u_l = Hp[l, 0:n_I] b,  d_l = Hp[l, q] - Hp[l, 0:n_I] u2   for the pruned rows and the g leaving rows.
+template <int TP_R>
+__global__ void __launch_bounds__(32 * TP_W) k_hpass_g(Ptrs p)
+{
+    if (p.ctl->done) return;
+    const int g = p.g, e0 = blockIdx.y * TP_E;
+    const int lane = threadIdx.x & 31;
+    const int64_t nrows = p.nJ + g;
+    const int64_t l0 = ((int64_t)blockIdx.x * TP_W + (threadIdx.x >> 5)) * TP_R;
+    if (l0 >= nrows) return;
+    const int64_t r0 = (int64_t)p.ctl->sel_slot * g;
+    const int64_t qcol0 = p.nI + (int64_t)p.ctl->sel_t * g;
+    const float4 *rows[TP_R], *bv[TP_E], *uv[TP_E];
+#pragma unroll
+    for (int i = 0; i < TP_R; ++i) {
+        const int64_t l = l0 + i < nrows ? l0 + i : nrows - 1;
+        rows[i] = reinterpret_cast<const float4*>(p.Hp + (l < p.nJ ? p.nI + l : r0 + (l - p.nJ)) * p.ldp);
+    }
+#pragma unroll
+    for (int j = 0; j < TP_E; ++j) {
+        const int64_t e = e0 + j < g ? e0 + j : g - 1;
+        bv[j] = reinterpret_cast<const float4*>(p.b + e * p.ldh);
+        uv[j] = reinterpret_cast<const float4*>(p.u2 + e * p.ldh);
+    }
+    float au[TP_R][TP_E], ad[TP_R][TP_E];
+#pragma unroll
+    for (int i = 0; i < TP_R; ++i)
+#pragma unroll
+        for (int j = 0; j < TP_E; ++j) { au[i][j] = 0.f; ad[i][j] = 0.f; }
+    for (int64_t c = lane; c < p.ldh / 4; c += 32) {
+        float4 x[TP_R];
+#pragma unroll
+        for (int i = 0; i < TP_R; ++i) x[i] = rows[i][c];
+#pragma unroll
+        for (int j = 0; j < TP_E; ++j) {
+            const float4 bb = __ldg(bv[j] + c), uu = __ldg(uv[j] + c);
+#pragma unroll
+            for (int i = 0; i < TP_R; ++i) { au[i][j] += dot4f(x[i], bb); ad[i][j] += dot4f(x[i], uu); }
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < TP_R; ++i)
+#pragma unroll
+        for (int j = 0; j < TP_E; ++j) {
+            const float su = warp_sum(au[i][j]), sd = warp_sum(ad[i][j]);
+            const int64_t l = l0 + i;
+            if (lane == 0 && l < nrows && e0 + j < g) {
+                p.u[l * g + e0 + j] = su;
+                p.d[l * g + e0 + j] = reinterpret_cast<const float*>(rows[i])[qcol0 + e0 + j] - sd;
+            }
+        }
+}
+
+// Groups of more than one row: the rank-2g updates as register tiles.  A block owns TG_RT rows x (TG_T float4) columns;
+// the 2 g coefficients of its rows sit in shared memory, every streamed piece of the g-row panels (b, u2 / K, Vq) is
+// used by all TG_RT rows, and the rows and columns that the formulas replace are patched before the store.
+constexpr int TG_RT = 8;
+constexpr int TG_T = 128;
+
+// Hinv' = Hinv - bC b^T + u2c u2^T; rows/columns of r take -u2c, the rr block c1^-1.  Grid (column tiles, row tiles),
+// dynamic shared memory 2 g TG_RT floats.
+__global__ void __launch_bounds__(TG_T) k_update_hinv_g(Ptrs p)
+{
+    if (p.ctl->done) return;
+    extern __shared__ float smf[];
+    const int g = p.g;
+    float* nbs = smf;                       // [e][i] = -bC[e][row0 + i]
+    float* ucs = smf + g * TG_RT;           // [e][i] = u2c[e][row0 + i]
+    const int64_t row0 = (int64_t)blockIdx.y * TG_RT;
+    const int64_t r0 = (int64_t)p.ctl->sel_slot * g;
+    for (int idx = threadIdx.x; idx < g * TG_RT; idx += TG_T) {
+        const int e = idx / TG_RT; const int64_t s = row0 + idx % TG_RT;
+        const bool ok = s < p.nI;
+        nbs[idx] = ok ? -p.bC[(int64_t)e * p.ldh + s] : 0.f;
+        ucs[idx] = ok ? p.u2c[(int64_t)e * p.ldh + s] : 0.f;
+    }
+    __syncthreads();
+    const int64_t n4 = p.ldh / 4;
+    const int64_t c4 = (int64_t)blockIdx.x * TG_T + threadIdx.x;
+    if (c4 >= n4) return;
+    float4 h[TG_RT];
+#pragma unroll
+    for (int i = 0; i < TG_RT; ++i)
+        h[i] = row0 + i < p.nI ? reinterpret_cast<const float4*>(p.Hinv + (row0 + i) * p.ldh)[c4] : make_float4(0.f, 0.f, 0.f, 0.f);
+    const float4* b4 = reinterpret_cast<const float4*>(p.b) + c4;
+    const float4* u4 = reinterpret_cast<const float4*>(p.u2) + c4;
+    for (int e = 0; e < g; ++e) {
+        const float4 bb = __ldg(b4 + (int64_t)e * n4), uu = __ldg(u4 + (int64_t)e * n4);
+#pragma unroll
+        for (int i = 0; i < TG_RT; ++i) {
+            const float nb = nbs[e * TG_RT + i], us = ucs[e * TG_RT + i];
+            h[i].x = fmaf(us, uu.x, fmaf(nb, bb.x, h[i].x)); h[i].y = fmaf(us, uu.y, fmaf(nb, bb.y, h[i].y));
+            h[i].z = fmaf(us, uu.z, fmaf(nb, bb.z, h[i].z)); h[i].w = fmaf(us, uu.w, fmaf(nb, bb.w, h[i].w));
+        }
+    }
+    const int64_t col = c4 * 4;
+    const bool col_hit = col + 4 > r0 && col < r0 + g;
+    const double* c1inv = p.small + S_C1INV * g * g;
+#pragma unroll
+    for (int i = 0; i < TG_RT; ++i) {
+        const int64_t s = row0 + i;
+        if (s >= p.nI) break;
+        const bool srow = s >= r0 && s < r0 + g;
+        if (srow || col_hit) {
+            float* hf = reinterpret_cast<float*>(&h[i]);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int64_t sc = col + j;
+                const bool scol = sc >= r0 && sc < r0 + g;
+                if (srow && scol) hf[j] = (float)c1inv[(s - r0) * g + (sc - r0)];
+                else if (srow) hf[j] = -p.u2c[(s - r0) * p.ldh + sc];
+                else if (scol) hf[j] = -p.u2c[(sc - r0) * p.ldh + s];
+            }
+        }
+        reinterpret_cast<float4*>(p.Hinv + s * p.ldh)[c4] = h[i];
+    }
+}
+
+// V'[s] = V[s] - sum_e b[e][s] K[e] - sum_e u2[e][s] Vq[e] (rows of r: Vq) for kind 0,
+// R'[l] = R[l] + sum_e u[l][e] K[e] - sum_e d[l][e] Vq[e] (rows of q: K[e] - sum_f d[nJ+e][f] Vq[f]) for kind 1.
+// The replaced rows are the same sum started from zero with their own coefficients.
+__global__ void __launch_bounds__(TG_T) k_update_rows_g(Ptrs p, int kind)
+{
+    if (p.ctl->done) return;
+    extern __shared__ float smf[];
+    const int g = p.g;
+    float* cks = smf;                       // coefficient of K[e] for row i
+    float* cqs = smf + g * TG_RT;           // coefficient of Vq[e]
+    float* M = kind == 0 ? p.V : p.R;
+    const int64_t nrows = kind == 0 ? p.nI : p.nJ;
+    const int64_t special0 = (kind == 0 ? (int64_t)p.ctl->sel_slot : (int64_t)p.ctl->sel_t) * g;
+    const int64_t row0 = (int64_t)blockIdx.y * TG_RT;
+    for (int idx = threadIdx.x; idx < g * TG_RT; idx += TG_T) {
+        const int e = idx / TG_RT; const int64_t s = row0 + idx % TG_RT;
+        float ck = 0.f, cq = 0.f;
+        if (s < nrows) {
+            if (s >= special0 && s < special0 + g) {
+                const int ee = (int)(s - special0);
+                if (kind == 0) cq = e == ee ? 1.f : 0.f;
+                else { ck = e == ee ? 1.f : 0.f; cq = -p.d[(p.nJ + ee) * g + e]; }
+            } else if (kind == 0) { ck = -p.b[(int64_t)e * p.ldh + s]; cq = -p.u2[(int64_t)e * p.ldh + s]; }
+            else { ck = p.u[s * g + e]; cq = -p.d[s * g + e]; }
+        }
+        cks[idx] = ck; cqs[idx] = cq;
+    }
+    __syncthreads();
+    const int64_t n4 = p.ldm / 4;
+    const int64_t c4 = (int64_t)blockIdx.x * TG_T + threadIdx.x;
+    if (c4 >= n4) return;
+    float4 v[TG_RT];
+#pragma unroll
+    for (int i = 0; i < TG_RT; ++i) {
+        const int64_t s = row0 + i;
+        const bool keep = s < nrows && !(s >= special0 && s < special0 + g);
+        v[i] = keep ? reinterpret_cast<const float4*>(M + s * p.ldm)[c4] : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    const float4* K4 = reinterpret_cast<const float4*>(p.K) + c4;
+    const float4* Q4 = reinterpret_cast<const float4*>(p.Vq) + c4;
+    for (int e = 0; e < g; ++e) {
+        const float4 kk = __ldg(K4 + (int64_t)e * n4), q = __ldg(Q4 + (int64_t)e * n4);
+#pragma unroll
+        for (int i = 0; i < TG_RT; ++i) {
+            const float ck = cks[e * TG_RT + i], cq = cqs[e * TG_RT + i];
+            v[i].x = fmaf(cq, q.x, fmaf(ck, kk.x, v[i].x)); v[i].y = fmaf(cq, q.y, fmaf(ck, kk.y, v[i].y));
+            v[i].z = fmaf(cq, q.z, fmaf(ck, kk.z, v[i].z)); v[i].w = fmaf(cq, q.w, fmaf(ck, kk.w, v[i].w));
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < TG_RT; ++i)
+        if (row0 + i < nrows) reinterpret_cast<float4*>(M + (row0 + i) * p.ldm)[c4] = v[i];
 }
 
 // C += sign * A * B^T (all g x g, ld g) on the fp64 tensor-core path; each entry of C is owned by one lane.
@@ -529,7 +727,7 @@ __device__ void mat_mul_nt_acc(const double* A, const double* B, double* C, int 
 // c_l' = c_l + u_l C^-1 u_l^T - d_l c1^-1 d_l^T for every pruned slot (g > 1); the entering slot receives
 // the leaving group: c' = C^-1 - d_r c1^-1 d_r^T.  One block per pruned slot; u_l (then d_l) and its product
 // with C^-1 (c1^-1) sit in shared memory (2 g^2 doubles), the four g x g products run on the fp64 tensor-core path.
-__global__ void __launch_bounds__(256) k_update_c(Ptrs p)
+__global__ void __launch_bounds__(1024) k_update_c(Ptrs p)
 {
     if (p.ctl->done) return;
     extern __shared__ double smc[];
@@ -618,7 +816,7 @@ constexpr int kPairBlocks = 296;
 constexpr int kPairTemps = 8;
 
 // Per kept slot: C_s^-1, KK_s = C_s^-1 GV_s C_s^-1 and D_s (block per slot; dynamic smem 3 g^2 doubles).
-__global__ void k_pair_slots(Ptrs p)
+__global__ void __launch_bounds__(1024) k_pair_slots(Ptrs p)
 {
     if (p.ctl->done) return;
     extern __shared__ double smd[];
@@ -641,15 +839,17 @@ __global__ void k_pair_slots(Ptrs p)
     if (threadIdx.x == 0) p.D[s] = piv > 0.0 ? tr : INFINITY;
 }
 
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(1024)
 k_pair_delta(Ptrs p, const float* __restrict__ Pm, int64_t ldpm, const float* __restrict__ XG, int64_t ldxg, int64_t npairs)
 {
     if (p.ctl->done) return;
     __shared__ double red[32];
+    extern __shared__ double smd[];             // g^2 + 2 g doubles: c1 while it is inverted
     const int g = p.g, gg = g * g;
+    double* Ms = smd; double* Lws = smd + gg;
     const int64_t npr = p.ng - p.k;
     double* S = p.pairScratch + (int64_t)blockIdx.x * kPairTemps * gg;
-    double *P = S, *GX = S + gg, *T1 = S + 2 * gg, *c1 = S + 3 * gg, *RR = S + 4 * gg, *TMP = S + 5 * gg, *Lw = S + 6 * gg, *OUT = S + 7 * gg;
+    double *P = S, *GX = S + gg, *T1 = S + 2 * gg, *RR = S + 4 * gg, *TMP = S + 5 * gg, *OUT = S + 7 * gg;
     for (int64_t pair = blockIdx.x; pair < npairs; pair += gridDim.x) {
         const int64_t s = pair / npr, t = pair % npr;
         const double Ds = p.D[s], At = p.A[t];
@@ -669,7 +869,7 @@ k_pair_delta(Ptrs p, const float* __restrict__ Pm, int64_t ldpm, const float* __
         mat_mul(T1, false, P, true, TMP, g);                     // P C^-1 P^T
         for (int idx = threadIdx.x; idx < gg; idx += blockDim.x) {
             const int i = idx / g, j = idx % g;
-            c1[idx] = 0.5 * (p.c[t * gg + idx] + p.c[t * gg + j * g + i]) + 0.5 * (TMP[idx] + TMP[j * g + i]);
+            Ms[idx] = 0.5 * (p.c[t * gg + idx] + p.c[t * gg + j * g + i]) + 0.5 * (TMP[idx] + TMP[j * g + i]);
         }
         __syncthreads();
         mat_mul(T1, false, GX, false, TMP, g);                   // P C^-1 V_s R_t^T
@@ -680,7 +880,7 @@ k_pair_delta(Ptrs p, const float* __restrict__ Pm, int64_t ldpm, const float* __
             RR[idx] += p.gramR[t * gg + idx] + TMP[idx] + TMP[j * g + i];
         }
         __syncthreads();
-        const double piv = spd_inverse(c1, Lw, OUT, g);
+        const double piv = spd_inverse(Ms, Lws, OUT, g);
         const double gain = mat_trace_prod(OUT, RR, g, red);
         if (threadIdx.x == 0) p.pairDelta[pair] = piv > 0.0 ? Ds - gain : INFINITY;
         __syncthreads();
@@ -745,6 +945,9 @@ Ptrs make_ptrs(osscar_ctx* ctx)
     return p;
 }
 
+// Threads of the one-block-per-matrix kernels of the g x g algebra: a thread per entry up to the block limit.
+static unsigned small_threads(int g) { return g * g >= 1024 ? 1024u : 256u; }
+
 #define CK(x) do { cudaError_t e_ = (x); if (e_ != cudaSuccess) return OSSCAR_E_CUDA; } while (0)
 
 // Everything the selection needs from a freshly built or freshly updated state.
@@ -761,13 +964,9 @@ cudaError_t enqueue_scores(osscar_ctx* ctx, const Ptrs& p, bool norms, bool gene
         const size_t smem = 3 * (size_t)p.g * p.g * sizeof(double);
         cudaError_t e = cudaFuncSetAttribute(k_scores_general, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        k_group_gram<<<dim3((unsigned)p.k, (unsigned)p.g), 256, 0, st>>>(p.V, p.ldm, p.g, p.gramV, p.ctl);
-        k_scores_general<<<(unsigned)p.k, 256, smem, st>>>(p, 0);
-        count_launches(p.nJ > 0 ? 4 : 2);
-        if (p.nJ > 0) {
-            k_group_gram<<<dim3((unsigned)(p.ng - p.k), (unsigned)p.g), 256, 0, st>>>(p.R, p.ldm, p.g, p.gramR, p.ctl);
-            k_scores_general<<<(unsigned)(p.ng - p.k), 256, smem, st>>>(p, 1);
-        }
+        k_group_gram<<<dim3((unsigned)p.ng, (unsigned)((p.g + GG_AT - 1) / GG_AT)), 256, 0, st>>>(p);      // kept and pruned groups together
+        k_scores_general<<<(unsigned)p.ng, small_threads(p.g), smem, st>>>(p);
+        count_launches(2);
     }
     return cudaGetLastError();
 }
@@ -813,6 +1012,11 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
     if (block) max_swaps /= bs;                   // from here on: iterations
     const int64_t npairs = (int64_t)L.k * (L.ng - L.k);
     if (max_swaps > 0) CK(enqueue_scores(ctx, p, true, pair));
+    const size_t inv_smem = ((size_t)g * g + 2 * (size_t)g) * sizeof(double);      // matrix under inversion + pivot row/column
+    if (inv_smem > 48 * 1024) {
+        CK(cudaFuncSetAttribute(k_small, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)inv_smem));
+        CK(cudaFuncSetAttribute(k_pair_delta, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)inv_smem));
+    }
     auto pair_scores = [&]() -> cudaError_t {      // PAIR_EXACT: exact change of obj of every (kept, pruned) pair
         float* Pm = (float*)((char*)ctx->ws + L.off_big);
         const int64_t ldj = round_up(L.nJ, kPadF);
@@ -825,8 +1029,8 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
         const size_t smem = 3 * (size_t)g * g * sizeof(double);
         e = cudaFuncSetAttribute(k_pair_slots, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        k_pair_slots<<<(unsigned)L.k, 256, smem, st>>>(p);
-        k_pair_delta<<<(unsigned)(npairs < kPairBlocks ? npairs : kPairBlocks), 256, 0, st>>>(p, Pm, L.ldh, XG, ldj, npairs);
+        k_pair_slots<<<(unsigned)L.k, small_threads(g), smem, st>>>(p);
+        k_pair_delta<<<(unsigned)(npairs < kPairBlocks ? npairs : kPairBlocks), small_threads(g), inv_smem, st>>>(p, Pm, L.ldh, XG, ldj, npairs);
         k_pair_select<<<1, 1024, 0, st>>>(p, npairs);
         count_launches(3);
         return cudaGetLastError();
@@ -849,6 +1053,7 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
         if (smem2 / 2 > 48 * 1024) CK(cudaFuncSetAttribute(k_blk_update_c_g1, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(smem2 / 2)));
     }
     if (g > 1) CK(cudaFuncSetAttribute(k_update_c, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(2 * (size_t)g * g * sizeof(double))));
+
     const int batch = 32;
     cudaEvent_t evb[2];
     CK(cudaEventCreateWithFlags(&evb[0], cudaEventDisableTiming));
@@ -866,6 +1071,12 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
     const unsigned yblocks = (unsigned)((L.nI + 7) / 8);
     constexpr int RPW = 4;
     const unsigned hblocks = (unsigned)((L.nJ + g + 8 * RPW - 1) / (8 * RPW));
+    const unsigned gtiles = (unsigned)((g + TP_E - 1) / TP_E);
+    auto tile_blocks = [](int64_t rows, int R) { return (unsigned)((rows + TP_W * R - 1) / (TP_W * R)); };
+    auto tile_rows = [&](int64_t rows) {           // rows per warp: as many as still leave about 4096 warps in flight
+        for (int R = 4; R > 1; R >>= 1) if ((rows + R - 1) / R * gtiles >= 4096) return R;
+        return 1;
+    };
     const unsigned prep_blocks = (unsigned)(((L.nI + L.ldm) * g + 255) / 256);
     int next_prof = 0;
     int nmarks = 0;                 // events recorded per profiled step (depends on the step variant)
@@ -906,17 +1117,41 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
             else k_select<<<1, 1024, 0, st>>>(p);
             mark();
             k_pairgram<<<(unsigned)((3 * g * g + 7) / 8), 256, 0, st>>>(p);                          mark();
-            k_ypass<<<dim3(yblocks, g), 256, 0, st>>>(p);                                            mark();
-            k_small<<<1, 256, 0, st>>>(p, prm->accept_mode, tol, max_swaps, obj_trace, swap_trace);  mark();
-            k_prep<<<prep_blocks, 256, 0, st>>>(p);                                                  mark();
-            k_hpass<RPW><<<dim3(hblocks, g), 256, 0, st>>>(p);                                       mark();
-            k_update_hinv<<<dim3((unsigned)((L.ldh / 4 + 255) / 256), (unsigned)((L.nI + HI_RT - 1) / HI_RT)), 256, 0, st>>>(p);
+            if (g > 1) {
+                const int R = tile_rows(L.nI);
+                if (R == 4) k_ypass_g<4><<<dim3(tile_blocks(L.nI, 4), gtiles), 32 * TP_W, 0, st>>>(p);
+                else if (R == 2) k_ypass_g<2><<<dim3(tile_blocks(L.nI, 2), gtiles), 32 * TP_W, 0, st>>>(p);
+                else k_ypass_g<1><<<dim3(tile_blocks(L.nI, 1), gtiles), 32 * TP_W, 0, st>>>(p);
+            }
+            else k_ypass<<<dim3(yblocks, 1), 256, 0, st>>>(p);
             mark();
-            k_update_rows<<<(unsigned)((L.nI + UP_ROWS - 1) / UP_ROWS), 256, 0, st>>>(p, 0);          mark();
-            k_update_rows<<<(unsigned)((L.nJ + UP_ROWS - 1) / UP_ROWS), 256, 0, st>>>(p, 1);          mark();
+            k_small<<<1, small_threads(g), inv_smem, st>>>(p, prm->accept_mode, tol, max_swaps, obj_trace, swap_trace);
+            mark();
+            k_prep<<<prep_blocks, 256, 0, st>>>(p);                                                  mark();
+            if (g > 1) {
+                const int R = tile_rows(L.nJ + g);
+                if (R == 4) k_hpass_g<4><<<dim3(tile_blocks(L.nJ + g, 4), gtiles), 32 * TP_W, 0, st>>>(p);
+                else if (R == 2) k_hpass_g<2><<<dim3(tile_blocks(L.nJ + g, 2), gtiles), 32 * TP_W, 0, st>>>(p);
+                else k_hpass_g<1><<<dim3(tile_blocks(L.nJ + g, 1), gtiles), 32 * TP_W, 0, st>>>(p);
+            }
+            else k_hpass<RPW><<<dim3(hblocks, 1), 256, 0, st>>>(p);
+            mark();
+            if (g > 1) {
+                const size_t sm_t = 2 * (size_t)g * TG_RT * sizeof(float);
+                k_update_hinv_g<<<dim3((unsigned)((L.ldh / 4 + TG_T - 1) / TG_T), (unsigned)((L.nI + TG_RT - 1) / TG_RT)), TG_T, sm_t, st>>>(p);
+                mark();
+                const unsigned ctiles = (unsigned)((L.ldm / 4 + TG_T - 1) / TG_T);
+                k_update_rows_g<<<dim3(ctiles, (unsigned)((L.nI + TG_RT - 1) / TG_RT)), TG_T, sm_t, st>>>(p, 0);     mark();
+                k_update_rows_g<<<dim3(ctiles, (unsigned)((L.nJ + TG_RT - 1) / TG_RT)), TG_T, sm_t, st>>>(p, 1);     mark();
+            } else {
+                k_update_hinv<<<dim3((unsigned)((L.ldh / 4 + 255) / 256), (unsigned)((L.nI + HI_RT - 1) / HI_RT)), 256, 0, st>>>(p);
+                mark();
+                k_update_rows<<<(unsigned)((L.nI + UP_ROWS - 1) / UP_ROWS), 256, 0, st>>>(p, 0);          mark();
+                k_update_rows<<<(unsigned)((L.nJ + UP_ROWS - 1) / UP_ROWS), 256, 0, st>>>(p, 1);          mark();
+            }
             count_launches(9);
             if (g > 1) {
-                k_update_c<<<(unsigned)(L.ng - L.k), 256, 2 * (size_t)g * g * sizeof(double), st>>>(p);
+                k_update_c<<<(unsigned)(L.ng - L.k), small_threads(g), 2 * (size_t)g * g * sizeof(double), st>>>(p);
                 count_launches(1);
             }
             if (g > 1 || pair) {
