@@ -74,7 +74,10 @@ int osscar_set_workspace(osscar_ctx* ctx, void* dev_ptr, size_t bytes);
  *                   With a workspace set, G is formed on the tensor cores (three-term bf16 split, fp32-accurate)
  *                   and the workspace contents are overwritten; without one it runs on the fp32 pipes.
  * X: device, n_rows x d1, bf16 (tensor cores, fp32 accumulation) or fp32.  For bf16 the
- * pointer must be 16-byte aligned and d1 a multiple of 8.  W: device d1 x m fp32 (read on END).
+ * pointer must be 16-byte aligned and d1 a multiple of 8.  fp32 X with a workspace set is split into three bf16
+ * terms there (row panels of 6 * round_up(d1, 8) bytes per row, workspace contents overwritten) and accumulated on
+ * the tensor cores to fp32 accuracy; without a workspace it runs on the fp32 pipes.
+ * W: device d1 x m fp32 (read on END).
  * H: device d1 x d1 fp32, G: device d1 x m fp32, const_term: host (written on END).
  * n_rows may be 0 (nothing is added).
  */

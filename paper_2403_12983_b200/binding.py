@@ -183,6 +183,12 @@ class Solver:
         _check(lib().osscar_set_workspace(self._h, _ptr(self._ws), self._ws.numel()), "osscar_set_workspace")
         return need
 
+    def lend_workspace(self, nbytes: int):
+        """Lends a workspace of exactly `nbytes` (staging room for the tensor-core products before a state exists)."""
+        self._ws = None
+        self._ws = torch.empty(int(nbytes), dtype=torch.uint8, device=f"cuda:{self.device}")
+        _check(lib().osscar_set_workspace(self._h, _ptr(self._ws), self._ws.numel()), "osscar_set_workspace")
+
     # -------------------------------------------------------------- calls of include/osscar.h
     def gram_chunk(self, X: torch.Tensor, H: torch.Tensor, flags: int, W=None, G=None, damp: float = 0.0) -> Optional[float]:
         if X.dtype == torch.bfloat16:

@@ -40,13 +40,15 @@ constexpr int TRI_BAND = 16;                                  // same for the up
 enum { MODE_GEMM3 = 0,      // A fp32 split, K-major; B fp32 split; six term pairs; all tiles
        MODE_GRAM = 1,       // A = B = X (bf16, MN-major); one term; upper-triangle tiles
        MODE_CROSS = 2,      // A = X (MN-major), B = Y bf16; one term; all tiles
-       MODE_CROSS3 = 3 };   // A = X (MN-major), B = Y fp32 split in three terms
+       MODE_CROSS3 = 3,     // A = X (MN-major), B = Y fp32 split in three terms
+       MODE_GRAM3 = 4 };    // A = B = X fp32 split in three terms (MN-major); six term pairs; upper-triangle tiles
 template <int MODE> struct Traits {
     static constexpr bool kAMN = MODE != MODE_GEMM3;
-    static constexpr int kTerms = MODE == MODE_GEMM3 ? 6 : (MODE == MODE_CROSS3 ? 3 : 1);
-    static constexpr bool kUpper = MODE == MODE_GRAM;
+    static constexpr bool kSixPairs = MODE == MODE_GEMM3 || MODE == MODE_GRAM3;
+    static constexpr int kTerms = kSixPairs ? 6 : (MODE == MODE_CROSS3 ? 3 : 1);
+    static constexpr bool kUpper = MODE == MODE_GRAM || MODE == MODE_GRAM3;
     // k-blocks per TMEM accumulation chain: short where small terms ride on large ones, 32 (128 MMAs) for plain bf16
-    static constexpr int kFlush = MODE == MODE_GEMM3 ? 2 : (MODE == MODE_CROSS3 ? 4 : 32);
+    static constexpr int kFlush = kSixPairs ? 2 : (MODE == MODE_CROSS3 ? 4 : 32);
     static constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((kAMN ? 1u : 0u) << 15) | (1u << 16)
                                      | ((uint32_t)(TILE_N >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
 };
@@ -146,8 +148,8 @@ k_mma_pipe(const __grid_constant__ Maps maps, int64_t M, int64_t N, int64_t K, f
                 for (int kb = 0; kb < nkb && ok; ++kb) {
                     for (int term = 0; term < kTerms; ++term, ++it) {
                         // term pairs, small products first: (3,1) (2,2) (1,3) (2,1) (1,2) (1,1)
-                        const int pa = MODE == MODE_GEMM3 ? (0x001012 >> (4 * term)) & 0xF : 0;     // A term: 2,1,0,1,0,0
-                        const int pb = MODE == MODE_GEMM3 ? (0x010210 >> (4 * term)) & 0xF          // B term: 0,1,2,0,1,0
+                        const int pa = TR::kSixPairs ? (0x001012 >> (4 * term)) & 0xF : 0;          // A term: 2,1,0,1,0,0
+                        const int pb = TR::kSixPairs ? (0x010210 >> (4 * term)) & 0xF               // B term: 0,1,2,0,1,0
                                      : (MODE == MODE_CROSS3 ? 2 - term : 0);
                         const int s = it % STAGES;
                         const uint32_t ph = (it / STAGES) & 1;
@@ -748,6 +750,51 @@ cudaError_t gram_tc2(cudaStream_t st, const void* X, int64_t n_rows, int64_t d1,
     k_mma_pipe<MODE_CROSS3><<<num_ids < sms ? num_ids : sms, NUM_THREADS, SMEM_BYTES, st>>>(
         maps, d1, m, n_rows, 1.f, beta, C, m, vec_ok, num_ids, status_dev, nullptr);
     count_launches(2);
+    return cudaGetLastError();
+}
+
+// H (+)= Xc^T Xc for fp32 Xc (n_rows x d1, row-major) on the tensor cores: Xc is split into three bf16 terms in
+// `scratch` and the six term pairs down to 2^-24 relative are accumulated over the upper-triangle tiles, in row panels
+// sized to the scratch (each panel needs 6 * rows * round_up(d1, 8) bytes).  Returns cudaErrorMemoryAllocation when
+// the scratch cannot hold a panel of 64 rows, so that the caller can take another path.
+cudaError_t gram_tc3(cudaStream_t st, const float* X, int64_t n_rows, int64_t d1, float* C, bool accumulate,
+                     void* scratch, size_t scratch_bytes, int32_t* status_dev)
+{
+    if (n_rows <= 0) return cudaSuccess;
+    const int64_t ldn = round_up(d1, 8);
+    if (!scratch || ((uintptr_t)scratch & 255)) return cudaErrorMemoryAllocation;
+    const size_t usable = scratch_bytes > 4096 ? scratch_bytes - 4096 : 0;
+    int64_t panel = (int64_t)(usable / (6 * (size_t)ldn));
+    if (panel >= n_rows) panel = n_rows; else panel = panel / 64 * 64;
+    if (panel < 64 && panel < n_rows) return cudaErrorMemoryAllocation;
+    PFN_encodeTiled enc = get_encode();
+    if (!enc) return cudaErrorNotSupported;
+    int dev = 0, sms = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(k_mma_pipe<MODE_GRAM3>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    const size_t piece = ((size_t)panel * ldn * 2 + 1023) / 1024 * 1024;
+    __nv_bfloat16* xp[3];
+    for (int i = 0; i < 3; ++i) xp[i] = (__nv_bfloat16*)((char*)scratch + i * piece);
+    const int TM = (int)((d1 + TILE_M - 1) / TILE_M), TN = (int)((d1 + TILE_N - 1) / TILE_N);
+    int num_ids = 0;
+    for (int tm = 0; tm < TM; ++tm) num_ids += TN - tm / 2;
+    const int vec_ok = (((uintptr_t)C & 15) == 0 && (d1 % 4) == 0) ? 1 : 0;
+    for (int64_t r0 = 0; r0 < n_rows; r0 += panel) {
+        const int64_t rows = n_rows - r0 < panel ? n_rows - r0 : panel;
+        k_split3<<<1184, 256, 0, st>>>(X + r0 * d1, d1, rows, d1, xp[0], xp[1], xp[2], ldn, nullptr);
+        Maps maps;
+        for (int i = 0; i < 3; ++i) {
+            if (!encode_2d(enc, &maps.a[i], xp[i], (uint64_t)d1, (uint64_t)rows, (uint64_t)ldn, 64, BLOCK_K)) return cudaErrorInvalidValue;
+            maps.b[i] = maps.a[i];
+        }
+        k_mma_pipe<MODE_GRAM3><<<num_ids < sms ? num_ids : sms, NUM_THREADS, SMEM_BYTES, st>>>(
+            maps, d1, d1, rows, 1.f, (accumulate || r0 > 0) ? 1.f : 0.f, C, d1, vec_ok, num_ids, status_dev, nullptr);
+        count_launches(2);
+    }
     return cudaGetLastError();
 }
 

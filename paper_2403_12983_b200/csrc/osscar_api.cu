@@ -173,8 +173,16 @@ int osscar_gram(osscar_ctx* ctx, const void* X, int x_dtype, int64_t n_rows, int
             // upper-triangle tiles only; the lower triangle is filled on END
             CKC(gram_tc2(st, X, n_rows, d1, nullptr, 0, 0, H, !begin, nullptr, 0, &ctx->ctl->status));
         } else {
-            CKC(sgemm(st, true, false, d1, d1, n_rows, 1.f, (const float*)X, d1, (const float*)X, d1,
-                      begin ? 0.f : 1.f, H, d1));
+            // fp32 activations: three-term bf16 split on the tensor cores when a workspace is lent (its contents are
+            // overwritten), else (or when it cannot hold a 64-row panel of the terms) the fp32 pipes
+            cudaError_t ge = cudaErrorMemoryAllocation;
+            if (ctx->ws) {
+                ge = gram_tc3(st, (const float*)X, n_rows, d1, H, !begin, ctx->ws, ctx->ws_bytes, &ctx->ctl->status);
+                if (ge == cudaSuccess) ctx->have_state = false;
+            }
+            if (ge == cudaErrorMemoryAllocation)
+                ge = sgemm(st, true, false, d1, d1, n_rows, 1.f, (const float*)X, d1, (const float*)X, d1, begin ? 0.f : 1.f, H, d1);
+            CKC(ge);
         }
         ctx->gram_rows += (double)n_rows;
     }

@@ -128,6 +128,10 @@ cudaError_t rank_update_tc(cudaStream_t st, int64_t M, int64_t N, int64_t K, flo
 // H (+)= Xc^T Xc (upper-triangle tiles; Y null) or G (+)= Xc^T Yc with the drained-accumulator pipeline of gemm_tc.cu.
 cudaError_t gram_tc2(cudaStream_t st, const void* X, int64_t n_rows, int64_t d1, const void* Y, int y_fp32, int64_t m,
                      float* C, bool accumulate, void* scratch, size_t scratch_bytes, int32_t* status_dev);
+// H (+)= Xc^T Xc for fp32 Xc on the tensor cores (three-term bf16 split staged in `scratch`, row panels sized to it);
+// cudaErrorMemoryAllocation when the scratch is too small for one panel.
+cudaError_t gram_tc3(cudaStream_t st, const float* X, int64_t n_rows, int64_t d1, float* C, bool accumulate,
+                     void* scratch, size_t scratch_bytes, int32_t* status_dev);
 
 // ---- gram_tc.cu ---------------------------------------------------------------------------------------------
 cudaError_t set_device_double(cudaStream_t st, double* dst, double v);          // *dst = v on the stream

@@ -68,6 +68,34 @@ def test_gram_fp32(solver, name, over):
     assert const == pytest.approx(const64, rel=1e-5)
 
 
+@pytest.mark.parametrize("name,over,ws_rows", [
+    ("c1", {}, None),
+    ("c4", dict(n=49 * 12, d1=9 * 37, m=50, k=12, chunk_rows=49 * 5), None),         # d1 = 333: ragged tiles, odd row length
+    ("c4", dict(n=49 * 24, d1=9 * 64, m=64, k=20, chunk_rows=49 * 10), 200),          # workspace holds 192-row panels only
+    ("c6", dict(n=49 * 40, d1=520, m=96, k=260, chunk_rows=49 * 16), None),
+])
+def test_gram_fp32_on_tensor_cores(solver, osscar, name, over, ws_rows):
+    """With a workspace lent to the context, fp32 activations are split into three bf16 terms and accumulated on the
+    tensor cores (in row panels when the workspace is small); the result must be as accurate as the fp32 product."""
+    wl = workloads.config(name, **over)
+    chunks, W, H64, G64, const64 = oracle_problem(wl)
+    if ws_rows is None:
+        solver.ensure_workspace(wl.d1, wl.m, wl.g, wl.k)
+    else:
+        solver.lend_workspace(6 * ws_rows * ((wl.d1 + 7) // 8 * 8) + 4096)
+    launches0 = osscar.binding.launch_count()
+    H, G, const = solver.gram([c.cuda() for c in wl.x_chunks()], wl.weight().cuda(), wl.damp)
+    Hg = H.cpu().numpy().astype(np.float64)
+    scale = np.sqrt(np.outer(np.diag(H64), np.diag(H64)))
+    assert np.max(np.abs(Hg - H64) / scale) < 5e-6
+    assert np.array_equal(Hg, Hg.T)
+    assert rel_fro(G.cpu().numpy(), G64) < 1e-5
+    assert const == pytest.approx(const64, rel=1e-5)
+    if ws_rows is not None:       # panels of 192 rows (whole multiples of 64 that fit): one split and one product each
+        panels = sum(-(-c.shape[0] // (ws_rows // 64 * 64)) for c in chunks)
+        assert panels > len(chunks) and osscar.binding.launch_count() - launches0 >= 2 * panels
+
+
 @pytest.mark.parametrize("name,over", [GRAM_CASES[0], GRAM_CASES[2], ("c2", dict(n=600, d1=200, m=37, k=100, chunk_rows=600))])
 def test_cross_term_on_tensor_cores(solver, name, over):
     """With a workspace lent to the context, G = H W runs as a three-term bf16 split on the tensor cores;
