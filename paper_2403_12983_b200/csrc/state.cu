@@ -127,49 +127,70 @@ __global__ void k_copy_pad(const float* __restrict__ src, int64_t lds, int64_t r
 constexpr int NB = 64;
 constexpr double kPivotRelTol = 1e-7;
 
-// Inverse of the nb x nb pivot block A[p0:p0+nb, p0:p0+nb] in fp64 (one block): in-place Gauss-Jordan elimination
-// without pivoting, one rank-1 update over the whole block per step, so every thread works in every step.  The
-// pivots are the diagonal of the successive Schur complements (the squared diagonal of the Cholesky factor).
-// Raises OSSCAR_E_NOTPD in ctl->status when a pivot is not positive.
-__global__ void __launch_bounds__(256)
+// Inverse of the nb x nb pivot block A[p0:p0+nb, p0:p0+nb] in fp64 (one block of 1024 threads): Gauss-Jordan
+// elimination without pivoting with the block held in registers.  Thread (i, cb) = (t / 16, t % 16) owns the entries
+// (i, cb + 16 k), k = 0..3.  In step j every thread fetches its row's entry of column j by a shuffle inside its
+// half-warp, the threads of row j publish the scaled pivot row through shared memory (double-buffered: one barrier per
+// step), and every entry takes its rank-1 update.  The pivots are the diagonal of the successive Schur complements
+// (the squared diagonal of the Cholesky factor).  Raises OSSCAR_E_NOTPD in ctl->status when a pivot is not positive.
+__global__ void __launch_bounds__(1024)
 k_pivot_inverse(const float* __restrict__ A, int64_t lda, int64_t p0, int nb, float* __restrict__ Dinv,
                 const float* __restrict__ Hp, int64_t ldp, SearchCtl* ctl)
 {
-    extern __shared__ double sm[];
-    double* L = sm;                 // nb x nb (ld NB): the block, overwritten by its inverse
-    double* colj = sm + NB * NB;    // column j and scaled row j of the current step
-    double* rowj = colj + NB;
-    const int t = threadIdx.x;
-    for (int idx = t; idx < nb * nb; idx += blockDim.x) {
-        int i = idx / nb, j = idx % nb;
-        // symmetrise: the two triangles can differ in the last bits
-        L[i * NB + j] = 0.5 * ((double)A[(p0 + i) * lda + p0 + j] + (double)A[(p0 + j) * lda + p0 + i]);
-    }
-    __shared__ int bad;
+    static_assert(NB == 64, "thread layout of the pivot inverse");
+    __shared__ double rowj[2][NB];
+    __shared__ double pinv_s[2];
     __shared__ double hdiag[NB];         // diagonal of the original matrix: scale of the pivot test
-    if (t == 0) bad = 0;
-    for (int j = t; j < nb; j += blockDim.x) hdiag[j] = (double)Hp[(p0 + j) * ldp + p0 + j];
-    __syncthreads();
-    for (int j = 0; j < nb; ++j) {
-        double d = L[j * NB + j];
-        // a pivot that fp32 data cannot tell from zero counts as not positive
-        if (!(d > kPivotRelTol * hdiag[j])) { if (t == 0) bad = 1; d = 1.0; }
-        const double pinv = 1.0 / d;
-        for (int i = t; i < nb; i += blockDim.x) { colj[i] = L[i * NB + j]; rowj[i] = L[j * NB + i] * pinv; }
-        __syncthreads();
-        for (int idx = t; idx < nb * nb; idx += blockDim.x) {
-            const int i = idx / nb, c = idx % nb;
-            double v;
-            if (i == j) v = (c == j) ? pinv : rowj[c];
-            else if (c == j) v = -colj[i] * pinv;
-            else v = L[i * NB + c] - colj[i] * rowj[c];
-            L[i * NB + c] = v;
-        }
-        __syncthreads();
+    __shared__ double Ls[NB][NB + 1];    // the finished inverse, for the symmetrised write
+    __shared__ int bad;
+    const int t = threadIdx.x, i = t >> 4, cb = t & 15, lane = t & 31;
+    double Lr[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const int c = cb + 16 * k;
+        // symmetrise: the two triangles can differ in the last bits
+        Lr[k] = (i < nb && c < nb) ? 0.5 * ((double)A[(p0 + i) * lda + p0 + c] + (double)A[(p0 + c) * lda + p0 + i]) : 0.0;
     }
-    for (int idx = t; idx < nb * nb; idx += blockDim.x) {       // the two triangles differ by rounding only
-        int i = idx / nb, j = idx % nb;
-        Dinv[i * NB + j] = (float)(0.5 * (L[i * NB + j] + L[j * NB + i]));
+    if (t == 0) bad = 0;
+    if (t < nb) hdiag[t] = (double)Hp[(p0 + t) * ldp + p0 + t];
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < 4; ++kk) {
+        for (int jj = 0; jj < 16; ++jj) {
+            const int j = kk * 16 + jj;
+            if (j >= nb) break;
+            const int buf = j & 1;
+            const double x = __shfl_sync(0xffffffffu, Lr[kk], (lane & 16) | jj);     // entry (i, j) of this thread's row
+            if (i == j) {
+                double d = x;
+                // a pivot that fp32 data cannot tell from zero counts as not positive
+                if (!(d > kPivotRelTol * hdiag[j])) { if (cb == 0) bad = 1; d = 1.0; }
+                const double pinv = 1.0 / d;
+#pragma unroll
+                for (int k = 0; k < 4; ++k) rowj[buf][cb + 16 * k] = Lr[k] * pinv;
+                if (cb == 0) pinv_s[buf] = pinv;
+            }
+            __syncthreads();
+            const double pinv = pinv_s[buf];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int c = cb + 16 * k;
+                const double r = rowj[buf][c];
+                double v;
+                if (i == j) v = (c == j) ? pinv : r;
+                else if (c == j) v = -x * pinv;
+                else v = Lr[k] - x * r;
+                Lr[k] = v;
+            }
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < 4; ++k) Ls[i][cb + 16 * k] = Lr[k];
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {                  // the two triangles differ by rounding only
+        const int c = cb + 16 * k;
+        if (i < nb && c < nb) Dinv[i * NB + c] = (float)(0.5 * (Ls[i][c] + Ls[c][i]));
     }
     if (t == 0 && bad) ctl->status = OSSCAR_E_NOTPD;
 }
@@ -390,10 +411,9 @@ int invert_spd_inplace(osscar_ctx* ctx, float* A, int64_t lda, int64_t n, const 
     float* U = T + L.d1 * NB;
     float* Un = U + NB * L.ldp;
     float* Dinv = Un + NB * L.ldp;
-    CK(cudaFuncSetAttribute(k_pivot_inverse, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * NB * NB * (int)sizeof(double)));
     for (int64_t p0 = 0; p0 < n; p0 += NB) {
         const int nb = (int)(n - p0 < NB ? n - p0 : NB);
-        k_pivot_inverse<<<1, 256, 2 * NB * NB * sizeof(double), st>>>(A, lda, p0, nb, Dinv, ref, ldref, ctx->ctl);
+        k_pivot_inverse<<<1, 1024, 0, st>>>(A, lda, p0, nb, Dinv, ref, ldref, ctx->ctl);
         // T = A[:, P] * Dinv
         CK(sgemm(st, false, false, n, nb, nb, 1.f, A + p0, lda, Dinv, NB, 0.f, T, NB, done));
         k_zero_rows<<<(nb * nb + 255) / 256, 256, 0, st>>>(T, NB, p0, nb, nb);
