@@ -1105,12 +1105,13 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
             if (enqueue_block_step(ctx, p, bp, prm->accept_mode, tol, obj_trace, swap_trace, mark) != cudaSuccess) { rc = OSSCAR_E_CUDA; break; }
         } else if (fast) {
             // single-row groups: decide, {H pass || V}, {R || slot exchange}, next entering group, {Hinv + next y}
-            const unsigned nbV = (unsigned)L.nI, nbH = (unsigned)(L.nJ + 1), nbR = (unsigned)L.nJ;   // one row per block
+            // G1_RB rows per block; the H pass has one more block for the leaving row
+            const unsigned nbV = (unsigned)((L.nI + G1_RB - 1) / G1_RB), nbR = (unsigned)((L.nJ + G1_RB - 1) / G1_RB), nbH = nbR + 1;
             k_decide_g1<<<1, 1024, 0, st>>>(p, prm->accept_mode, tol, obj_trace, swap_trace);   mark();
             k_l1_g1<<<nbV + nbH, 256, 0, st>>>(p, nbV);                                          mark();
             k_l2_g1<<<nbR + 32, 256, 0, st>>>(p, nbR);                                           mark();
             k_select_in_g1<<<1, 1024, 0, st>>>(p);                                               mark();
-            k_l4_g1<<<nbV, 256, 0, st>>>(p);                                                     mark();
+            k_l4_g1<G1_RB4><<<(unsigned)((L.nI + G1_RB4 - 1) / G1_RB4), 256, 0, st>>>(p);                                                     mark();
             count_launches(5);
         } else {
             if (pair) { if (pair_scores() != cudaSuccess) { rc = OSSCAR_E_CUDA; break; } }

@@ -171,9 +171,12 @@ k_decide_g1(Ptrs p, int accept_mode, double accept_tol, double* __restrict__ obj
     }
 }
 
-// Streaming layout of the three big kernels: ONE ROW PER BLOCK of 256 threads, every thread requests its (up to)
-// eight 16-byte pieces of the row at once, one block-wide reduction at the end.  Measured on the R update shape
-// (20070 x 7168): 6.7 TB/s against 5.7 TB/s for a warp per row and 6.0 TB/s for a plain copy.
+// Streaming layout of the three big kernels: a block of 256 threads owns whole rows, every thread requests its (up to)
+// eight or nine 16-byte pieces of a row at once, one block-wide reduction per row at the end.  Measured on the R update
+// shape (20070 x 7168): 6.7 TB/s for a row per block against 5.7 TB/s for a warp per row and 6.0 TB/s for a plain copy.
+// Two rows per block halve the L2 reads of the step's vectors: measured at the OPT-30B FC2 shape that pays for the Hinv
+// update with its three vectors (0.122 -> 0.115 ms) and costs the V / R updates and the H pass 12-17 % (half as many
+// resident blocks), so G1_RB = 1 there and G1_RB4 = 2 for the Hinv update.
 constexpr int G1_U = 8;
 constexpr int G1_UH = 9;            // pieces per thread for rows of Hinv / Hp: 9 x 256 x 4 floats cover n_I = 8602 in one pass
 constexpr int G1_T = 256;
@@ -190,118 +193,168 @@ __device__ __forceinline__ float block_sum_256(float v, float* red /*[8]*/)
     return t;
 }
 
-// Row update M'[s] = M[s] + ck_s K + cq_s Vq with the squared norm of the new row.  kind 0: V (ck = -b_s,
-// cq = -u2_s, row r0 := Vq, D' written), kind 1: R (ck = u_l, cq = -d_l, row of the entering slot := K - d_r Vq,
-// c' and A' written).
-__device__ __forceinline__ void update_row_g1(const Ptrs& p, int kind, int64_t s, float* red)
+// Row update M'[s] = M[s] + ck_s K + cq_s Vq with the squared norm of the new row, RB rows per block (every piece of
+// K and Vq fetched from L2 serves the RB rows).  kind 0: V (ck = -b_s, cq = -u2_s, row r0 := Vq, D' written),
+// kind 1: R (ck = u_l, cq = -d_l, row of the entering slot := K - d_r Vq, c' and A' written).
+template <int RB>
+__device__ __forceinline__ void update_row_g1(const Ptrs& p, int kind, int64_t s0, float* red)
 {
     float* M = kind == 0 ? p.V : p.R;
+    const int64_t nrows = kind == 0 ? p.nI : p.nJ;
     const int64_t n4 = p.ldm / 4;
     const float4* K4 = reinterpret_cast<const float4*>(p.K);
     const float4* Q4 = reinterpret_cast<const float4*>(p.Vq);
-    float4* row = reinterpret_cast<float4*>(M + s * p.ldm);
-    float nrm = 0.f;
-    bool sp = false;
-    float ck = 0.f, cq = 0.f, dr = 0.f;
-    for (int64_t base = threadIdx.x; base < n4; base += (int64_t)G1_T * G1_U) {
-        float4 v[G1_U];
+    float4* row[RB];
+    int64_t srow[RB];
 #pragma unroll
-        for (int j = 0; j < G1_U; ++j) {
-            const int64_t c = base + G1_T * j;
-            v[j] = c < n4 ? row[c] : make_float4(0.f, 0.f, 0.f, 0.f);     // requested before the step's scalars arrive
-        }
-        if (base == threadIdx.x) {           // first pass: the scalars of this row, loaded behind the row itself
+    for (int r = 0; r < RB; ++r) {
+        srow[r] = s0 + r < nrows ? s0 + r : nrows - 1;
+        row[r] = reinterpret_cast<float4*>(M + srow[r] * p.ldm);
+    }
+    float nrm[RB], ck[RB], cq[RB];
+    bool sp[RB];
+    float dr = 0.f;
+#pragma unroll
+    for (int r = 0; r < RB; ++r) { nrm[r] = 0.f; ck[r] = 0.f; cq[r] = 0.f; sp[r] = false; }
+    for (int64_t base = threadIdx.x; base < n4; base += (int64_t)G1_T * G1_U) {
+        float4 v[RB][G1_U];
+#pragma unroll
+        for (int r = 0; r < RB; ++r)
+#pragma unroll
+            for (int j = 0; j < G1_U; ++j) {
+                const int64_t c = base + G1_T * j;
+                v[r][j] = c < n4 ? row[r][c] : make_float4(0.f, 0.f, 0.f, 0.f);     // requested before the step's scalars arrive
+            }
+        if (base == threadIdx.x) {           // first pass: the scalars of these rows, loaded behind the rows themselves
             if (p.ctl->done) return;             // a stopped loop only read; nothing is written
             const int64_t special = kind == 0 ? (int64_t)p.ctl->sel_slot : (int64_t)p.ctl->sel_t;
-            sp = s == special;
-            if (kind == 0) { ck = -p.b[s]; cq = -p.u2[s]; }
-            else { ck = p.u[s]; cq = -p.d[s]; dr = p.d[p.nJ]; }
-            if (sp) { ck = kind == 0 ? 0.f : 1.f; cq = kind == 0 ? 1.f : -dr; }      // new row = ck K + cq Vq
+            if (kind == 1) dr = p.d[p.nJ];
+#pragma unroll
+            for (int r = 0; r < RB; ++r) {
+                const int64_t s = srow[r];
+                sp[r] = s == special;
+                if (kind == 0) { ck[r] = -p.b[s]; cq[r] = -p.u2[s]; }
+                else { ck[r] = p.u[s]; cq[r] = -p.d[s]; }
+                if (sp[r]) { ck[r] = kind == 0 ? 0.f : 1.f; cq[r] = kind == 0 ? 1.f : -dr; }      // new row = ck K + cq Vq
+            }
         }
 #pragma unroll
         for (int j = 0; j < G1_U; ++j) {
             const int64_t c = base + G1_T * j;
             if (c < n4) {
-                if (sp) v[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-                fma4(v[j], ck, __ldg(K4 + c));
-                fma4(v[j], cq, __ldg(Q4 + c));
-                row[c] = v[j];
-                nrm += dot4(v[j], v[j]);
+                const float4 kk = __ldg(K4 + c), qq = __ldg(Q4 + c);
+#pragma unroll
+                for (int r = 0; r < RB; ++r) {
+                    if (sp[r]) v[r][j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    fma4(v[r][j], ck[r], kk);
+                    fma4(v[r][j], cq[r], qq);
+                    if (s0 + r < nrows) row[r][c] = v[r][j];
+                    nrm[r] += dot4(v[r][j], v[r][j]);
+                }
             }
         }
     }
-    nrm = block_sum_256(nrm, red);
-    if (threadIdx.x == 0) {
-        const double Cinv = p.small[S_CINV], c1inv = p.small[S_C1INV];
-        if (kind == 0) {
-            p.vnorm[s] = nrm;
-            double hd;
-            if (sp) hd = c1inv;
-            else {
-                const double bs = p.b[s], us = p.u2[s];
-                hd = (double)p.Hinv[s * p.ldh + s] - bs * bs * Cinv + us * us * c1inv;
+#pragma unroll
+    for (int r = 0; r < RB; ++r) {
+        const float nr = block_sum_256(nrm[r], red);
+        if (threadIdx.x == 0 && s0 + r < nrows) {
+            const int64_t s = s0 + r;
+            const double Cinv = p.small[S_CINV], c1inv = p.small[S_C1INV];
+            if (kind == 0) {
+                p.vnorm[s] = nr;
+                double hd;
+                if (sp[r]) hd = c1inv;
+                else {
+                    const double bs = p.b[s], us = p.u2[s];
+                    hd = (double)p.Hinv[s * p.ldh + s] - bs * bs * Cinv + us * us * c1inv;
+                }
+                p.D[s] = hd > 0.0 ? (double)nr / hd : INFINITY;
+            } else {
+                p.rnorm[s] = nr;
+                double cc, hd;
+                if (sp[r]) { cc = Cinv - (double)dr * (double)dr * c1inv; hd = p.small[G1_HDIAG]; }
+                else {
+                    const double uu = p.u[s], dd = p.d[s];
+                    cc = p.c[s] + uu * uu * Cinv - dd * dd * c1inv;
+                    hd = p.Hp[(p.nI + s) * p.ldp + p.nI + s];
+                }
+                p.c[s] = cc;
+                p.A[s] = cc > kAddPivotTol * hd ? (double)nr / cc : -INFINITY;
             }
-            p.D[s] = hd > 0.0 ? (double)nrm / hd : INFINITY;
-        } else {
-            p.rnorm[s] = nrm;
-            double cc, hd;
-            if (sp) { cc = Cinv - (double)dr * (double)dr * c1inv; hd = p.small[G1_HDIAG]; }
-            else {
-                const double uu = p.u[s], dd = p.d[s];
-                cc = p.c[s] + uu * uu * Cinv - dd * dd * c1inv;
-                hd = p.Hp[(p.nI + s) * p.ldp + p.nI + s];
-            }
-            p.c[s] = cc;
-            p.A[s] = cc > kAddPivotTol * hd ? (double)nrm / cc : -INFINITY;
         }
     }
 }
 
-// u_l = Hp[l, 0:n_I] . b and d_l = Hp[l, q] - Hp[l, 0:n_I] . u2 for pruned row l (l = n_J: the leaving row).
-__device__ __forceinline__ void hpass_stream(const Ptrs& p, const float4* __restrict__ row, int64_t l, float* red /*[16]*/)
+// u_l = Hp[l, 0:n_I] . b and d_l = Hp[l, q] - Hp[l, 0:n_I] . u2 for RB rows (pruned rows l0.., or the single leaving
+// row, l = n_J); every piece of b and u2 serves the RB rows.
+template <int RB>
+__device__ __forceinline__ void hpass_stream(const Ptrs& p, const float4* const (&row)[RB], int64_t l0, int nvalid, float* red /*[16]*/)
 {
     const float4* bv = reinterpret_cast<const float4*>(p.b);
     const float4* uv = reinterpret_cast<const float4*>(p.u2);
     const int64_t n4 = p.ldh / 4;
-    float au = 0.f, ad = 0.f;
+    float au[RB], ad[RB];
+#pragma unroll
+    for (int r = 0; r < RB; ++r) { au[r] = 0.f; ad[r] = 0.f; }
     for (int64_t base = threadIdx.x; base < n4; base += (int64_t)G1_T * G1_UH) {
-        float4 x[G1_UH];
+        float4 x[RB][G1_UH];
+#pragma unroll
+        for (int r = 0; r < RB; ++r)
+#pragma unroll
+            for (int j = 0; j < G1_UH; ++j) {
+                const int64_t c = base + G1_T * j;
+                x[r][j] = c < n4 ? row[r][c] : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
 #pragma unroll
         for (int j = 0; j < G1_UH; ++j) {
             const int64_t c = base + G1_T * j;
-            x[j] = c < n4 ? row[c] : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
+            if (c < n4) {
+                const float4 bb = __ldg(bv + c), uu = __ldg(uv + c);
 #pragma unroll
-        for (int j = 0; j < G1_UH; ++j) {
-            const int64_t c = base + G1_T * j;
-            if (c < n4) { au += dot4(x[j], __ldg(bv + c)); ad += dot4(x[j], __ldg(uv + c)); }
+                for (int r = 0; r < RB; ++r) { au[r] += dot4(x[r][j], bb); ad[r] += dot4(x[r][j], uu); }
+            }
         }
     }
-    au = warp_sum(au); ad = warp_sum(ad);
-    if ((threadIdx.x & 31) == 0) { red[threadIdx.x >> 5] = au; red[8 + (threadIdx.x >> 5)] = ad; }
-    __syncthreads();
-    if (threadIdx.x == 0 && !p.ctl->done) {
-        float su = 0.f, sd = 0.f;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) { su += red[i]; sd += red[8 + i]; }
-        const int64_t qcol = p.nI + (int64_t)p.ctl->sel_t;
-        p.u[l] = su;
-        p.d[l] = reinterpret_cast<const float*>(row)[qcol] - sd;
+    for (int r = 0; r < RB; ++r) {
+        const float a = warp_sum(au[r]), d = warp_sum(ad[r]);
+        __syncthreads();
+        if ((threadIdx.x & 31) == 0) { red[threadIdx.x >> 5] = a; red[8 + (threadIdx.x >> 5)] = d; }
+        __syncthreads();
+        if (threadIdx.x == 0 && r < nvalid && !p.ctl->done) {
+            float su = 0.f, sd = 0.f;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) { su += red[i]; sd += red[8 + i]; }
+            const int64_t qcol = p.nI + (int64_t)p.ctl->sel_t;
+            p.u[l0 + r] = su;
+            p.d[l0 + r] = reinterpret_cast<const float*>(row[r])[qcol] - sd;
+        }
     }
-}
-__device__ __forceinline__ void hpass_row_g1(const Ptrs& p, int64_t l, float* red)
-{
-    // pruned rows know their address without reading the control block, so their stream starts at once
-    if (l < p.nJ) hpass_stream(p, reinterpret_cast<const float4*>(p.Hp + (p.nI + l) * p.ldp), l, red);
-    else hpass_stream(p, reinterpret_cast<const float4*>(p.Hp + (int64_t)p.ctl->sel_slot * p.ldp), l, red);
 }
 
-// L1: blocks [0, n_I) update one row of V each, the rest run the H pass (one row each).
-__global__ void __launch_bounds__(G1_T) k_l1_g1(Ptrs p, unsigned nbV)
+// L1: blocks [0, nbV) update G1_RB rows of V each; then one block per G1_RB pruned rows of the H pass (their addresses
+// need no control-block read, so their streams start at once) and a last block for the leaving row.
+constexpr int G1_RB = 1;            // rows per block of the V / R updates and the H pass
+constexpr int G1_RB4 = 2;           // rows per block of the Hinv update
+__global__ void __launch_bounds__(G1_T, 4) k_l1_g1(Ptrs p, unsigned nbV)      // 64 registers: four resident blocks per SM
 {
     __shared__ float red[16];
-    if (blockIdx.x < nbV) update_row_g1(p, 0, (int64_t)blockIdx.x, red);
-    else hpass_row_g1(p, (int64_t)(blockIdx.x - nbV), red);
+    if (blockIdx.x < nbV) { update_row_g1<G1_RB>(p, 0, (int64_t)blockIdx.x * G1_RB, red); return; }
+    const int64_t l0 = (int64_t)(blockIdx.x - nbV) * G1_RB;
+    if (l0 < p.nJ) {
+        const float4* rows[G1_RB];
+        int nvalid = 0;
+#pragma unroll
+        for (int r = 0; r < G1_RB; ++r) {
+            const int64_t l = l0 + r < p.nJ ? l0 + r : p.nJ - 1;
+            rows[r] = reinterpret_cast<const float4*>(p.Hp + (p.nI + l) * p.ldp);
+            nvalid += l0 + r < p.nJ;
+        }
+        hpass_stream<G1_RB>(p, rows, l0, nvalid, red);
+    } else {
+        const float4* rows[1] = { reinterpret_cast<const float4*>(p.Hp + (int64_t)p.ctl->sel_slot * p.ldp) };
+        hpass_stream<1>(p, rows, p.nJ, 1, red);
+    }
 }
 
 // Exchange of the leaving kept slot a and the entering pruned slot b in Hp (rows and columns) and in the
@@ -330,11 +383,11 @@ __device__ __forceinline__ void hswap_g1(const Ptrs& p, int64_t idx, int64_t str
     }
 }
 
-// L2: blocks [0, n_J) update one row of R each (+ c, A); the remaining blocks exchange the two slots in Hp.
-__global__ void __launch_bounds__(G1_T) k_l2_g1(Ptrs p, unsigned nbR)
+// L2: blocks [0, nbR) update G1_RB rows of R each (+ c, A); the remaining blocks exchange the two slots in Hp.
+__global__ void __launch_bounds__(G1_T, 4) k_l2_g1(Ptrs p, unsigned nbR)
 {
     __shared__ float red[8];
-    if (blockIdx.x < nbR) { update_row_g1(p, 1, (int64_t)blockIdx.x, red); return; }
+    if (blockIdx.x < nbR) { update_row_g1<G1_RB>(p, 1, (int64_t)blockIdx.x * G1_RB, red); return; }
     if (p.ctl->done) return;
     const int64_t nsw = gridDim.x - nbR;
     hswap_g1(p, (int64_t)(blockIdx.x - nbR) * blockDim.x + threadIdx.x, nsw * blockDim.x);
@@ -347,52 +400,71 @@ __global__ void __launch_bounds__(G1_T) k_l2_g1(Ptrs p, unsigned nbR)
 }
 
 // L4: Hinv' = Hinv - (b/C) b^T + (u2/c1) u2^T (row and column r0: -u2/c1, corner 1/c1) and, in the same pass,
-// y_next = Hinv' h with h = Hp[row of the next entering group, 0:n_I].  One row per block.
+// y_next = Hinv' h with h = Hp[row of the next entering group, 0:n_I].  RB rows per block: every piece of b, u2 and h
+// fetched from L2 serves the RB rows.
+template <int RB>
 __global__ void __launch_bounds__(G1_T) k_l4_g1(Ptrs p)
 {
     __shared__ float red[8];
-    const int64_t s = blockIdx.x;
+    const int64_t s0 = (int64_t)blockIdx.x * RB;
     const float4* b4 = reinterpret_cast<const float4*>(p.b);
     const float4* u4 = reinterpret_cast<const float4*>(p.u2);
-    float4* row = reinterpret_cast<float4*>(p.Hinv + s * p.ldh);
     const int64_t n4 = p.ldh / 4;
+    float4* row[RB];
+#pragma unroll
+    for (int r = 0; r < RB; ++r) row[r] = reinterpret_cast<float4*>(p.Hinv + (s0 + r < p.nI ? s0 + r : p.nI - 1) * p.ldh);
     int64_t r0 = 0;
     const float4* h4 = nullptr;
-    bool srow = false;
-    float nb = 0.f, us = 0.f, corner = 0.f, yacc = 0.f;
-    for (int64_t base = threadIdx.x; base < n4; base += (int64_t)G1_T * G1_UH) {
-        float4 h[G1_UH];
+    bool srow[RB];
+    float nb[RB], us[RB], corner[RB], yacc[RB];
 #pragma unroll
-        for (int j = 0; j < G1_UH; ++j) {
-            const int64_t c = base + G1_T * j;
-            h[j] = c < n4 ? row[c] : make_float4(0.f, 0.f, 0.f, 0.f);       // requested before the step's scalars arrive
-        }
+    for (int r = 0; r < RB; ++r) { srow[r] = false; nb[r] = 0.f; us[r] = 0.f; corner[r] = 0.f; yacc[r] = 0.f; }
+    for (int64_t base = threadIdx.x; base < n4; base += (int64_t)G1_T * G1_UH) {
+        float4 h[RB][G1_UH];
+#pragma unroll
+        for (int r = 0; r < RB; ++r)
+#pragma unroll
+            for (int j = 0; j < G1_UH; ++j) {
+                const int64_t c = base + G1_T * j;
+                h[r][j] = c < n4 ? row[r][c] : make_float4(0.f, 0.f, 0.f, 0.f);   // requested before the step's scalars arrive
+            }
         if (base == threadIdx.x) {
             if (p.ctl->done) return;
             r0 = p.ctl->sel_slot;
             const float Cinv = (float)p.small[S_CINV], c1inv = (float)p.small[S_C1INV];
             h4 = reinterpret_cast<const float4*>(p.Hp + (p.nI + (int64_t)p.ctl->sel_t) * p.ldp);
-            srow = s == r0;
-            // row r0 becomes -u2/c1: treat it as 0 * old - 0 * b + (-1/c1) * u2
-            nb = srow ? 0.f : -p.b[s] * Cinv;
-            us = srow ? -c1inv : p.u2[s] * c1inv;
-            corner = srow ? c1inv : -us;                                     // value of column r0 in this row
+#pragma unroll
+            for (int r = 0; r < RB; ++r) {
+                const int64_t s = s0 + r < p.nI ? s0 + r : p.nI - 1;
+                srow[r] = s == r0;
+                // row r0 becomes -u2/c1: treat it as 0 * old - 0 * b + (-1/c1) * u2
+                nb[r] = srow[r] ? 0.f : -p.b[s] * Cinv;
+                us[r] = srow[r] ? -c1inv : p.u2[s] * c1inv;
+                corner[r] = srow[r] ? c1inv : -us[r];                            // value of column r0 in this row
+            }
         }
 #pragma unroll
         for (int j = 0; j < G1_UH; ++j) {
             const int64_t c = base + G1_T * j;
             if (c < n4) {
-                if (srow) h[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-                fma4(h[j], nb, __ldg(b4 + c));
-                fma4(h[j], us, __ldg(u4 + c));
+                const float4 bb = __ldg(b4 + c), uu = __ldg(u4 + c), hh = __ldg(h4 + c);
                 const int64_t rc = r0 - c * 4;           // position of column r0 inside this float4, if any
-                h[j].x = rc == 0 ? corner : h[j].x; h[j].y = rc == 1 ? corner : h[j].y;
-                h[j].z = rc == 2 ? corner : h[j].z; h[j].w = rc == 3 ? corner : h[j].w;
-                row[c] = h[j];
-                yacc += dot4(h[j], __ldg(h4 + c));
+#pragma unroll
+                for (int r = 0; r < RB; ++r) {
+                    if (srow[r]) h[r][j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    fma4(h[r][j], nb[r], bb);
+                    fma4(h[r][j], us[r], uu);
+                    h[r][j].x = rc == 0 ? corner[r] : h[r][j].x; h[r][j].y = rc == 1 ? corner[r] : h[r][j].y;
+                    h[r][j].z = rc == 2 ? corner[r] : h[r][j].z; h[r][j].w = rc == 3 ? corner[r] : h[r][j].w;
+                    if (s0 + r < p.nI) row[r][c] = h[r][j];
+                    yacc[r] += dot4(h[r][j], hh);
+                }
             }
         }
     }
-    yacc = block_sum_256(yacc, red);
-    if (threadIdx.x == 0) p.y[s] = yacc;
+#pragma unroll
+    for (int r = 0; r < RB; ++r) {
+        const float t = block_sum_256(yacc[r], red);
+        if (threadIdx.x == 0 && s0 + r < p.nI) p.y[s0 + r] = t;
+    }
 }
