@@ -64,6 +64,21 @@ sgemm_kernel(int64_t M, int64_t N, int64_t K, float alpha, const float* __restri
         }
     };
 
+    // the old tile of C is wanted only at the very end: ask for its lines now (one 128-byte line per 32 columns), so
+    // that the read-modify-write of a short product (rank-64 updates of the exchange inversion) finds them in L2
+    if (beta != 0.f && (tx & 7) == 0) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int64_t gm = m0 + (i < 4 ? ty * 4 + i : 64 + ty * 4 + (i - 4));
+            if (gm >= M) continue;
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int64_t gn = n0 + h * 64 + tx * 4;
+                if (gn < N) asm volatile("prefetch.global.L2 [%0];" ::"l"(C + gm * ldc + gn));
+            }
+        }
+    }
+
     load_tiles(0);
     store_tiles(0);
     __syncthreads();
