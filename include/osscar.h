@@ -93,7 +93,8 @@ int osscar_gram(osscar_ctx* ctx, const void* X, int x_dtype, int64_t n_rows, int
  * so that obj(S) = min_W ||Y - X W||_F^2 = const - Tr(G_I^T (H_II)^-1 G_I).  Flags and damp as in osscar_gram (damping
  * touches H only).  X: bf16 (d1 % 8 == 0, 16-byte aligned) or fp32; Y: bf16 (m % 8 == 0) or fp32 (fp32 Y with bf16 X
  * is split into three bf16 terms in the workspace, which must hold 6 * n_rows * round_up(m, 8) bytes and is
- * overwritten); fp32 X requires fp32 Y.  On END *const_term is written and remembered by the context: the following
+ * overwritten); fp32 X requires fp32 Y, and with a workspace set its H runs on the tensor cores as in osscar_gram
+ * (workspace contents overwritten), G on the fp32 pipes.  On END *const_term is written and remembered by the context: the following
  * init / search calls use it in place of Tr(W_hat^T G).  osscar_set_const_term sets or clears that value by hand
  * (e.g. when H and G come from elsewhere).
  */

@@ -245,7 +245,15 @@ int osscar_gram_cross(osscar_ctx* ctx, const void* X, int x_dtype, const void* Y
             CKC(gram_tc2(st, X, n_rows, d1, Y, y_dtype == OSSCAR_FP32, m, G, !begin, ctx->ws, ctx->ws_bytes, &ctx->ctl->status));
             if (need > 0) ctx->have_state = false;
         } else {
-            CKC(sgemm(st, true, false, d1, d1, n_rows, 1.f, (const float*)X, d1, (const float*)X, d1, begin ? 0.f : 1.f, H, d1));
+            // H as in osscar_gram: on the tensor cores when a workspace can stage the bf16 terms, else the fp32 pipes
+            cudaError_t ge = cudaErrorMemoryAllocation;
+            if (ctx->ws) {
+                ge = gram_tc3(st, (const float*)X, n_rows, d1, H, !begin, ctx->ws, ctx->ws_bytes, &ctx->ctl->status);
+                if (ge == cudaSuccess) ctx->have_state = false;
+            }
+            if (ge == cudaErrorMemoryAllocation)
+                ge = sgemm(st, true, false, d1, d1, n_rows, 1.f, (const float*)X, d1, (const float*)X, d1, begin ? 0.f : 1.f, H, d1);
+            CKC(ge);
             CKC(sgemm(st, true, false, d1, m, n_rows, 1.f, (const float*)X, d1, (const float*)Y, m, begin ? 0.f : 1.f, G, m));
         }
         const int nblk = kTracePartials;

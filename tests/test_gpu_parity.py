@@ -500,14 +500,17 @@ def test_greedy_phase_matches_oracle(solver, name, over, t_hat):
 
 
 # ------------------------------------------------------------------------------------ cross term (sequential layer-wise form)
-@pytest.mark.parametrize("name,over,ydt", [
-    ("c2", dict(n=3000, d1=520, m=152, k=207, chunk_rows=1024), torch.bfloat16),
-    ("c2", dict(n=3000, d1=520, m=150, k=207, chunk_rows=1024), torch.float32),
-    ("c4", dict(n=49 * 30, d1=9 * 37, m=50, k=12, chunk_rows=49 * 10), torch.float32),
+@pytest.mark.parametrize("name,over,ydt,lend", [
+    ("c2", dict(n=3000, d1=520, m=152, k=207, chunk_rows=1024), torch.bfloat16, False),
+    ("c2", dict(n=3000, d1=520, m=150, k=207, chunk_rows=1024), torch.float32, False),
+    ("c4", dict(n=49 * 30, d1=9 * 37, m=50, k=12, chunk_rows=49 * 10), torch.float32, False),
+    ("c4", dict(n=49 * 30, d1=9 * 37, m=50, k=12, chunk_rows=49 * 10), torch.float32, True),    # fp32 X: H on the tensor cores
 ])
-def test_cross_term_gram_and_search(solver, name, over, ydt):
+def test_cross_term_gram_and_search(solver, name, over, ydt, lend):
     """Pruned-model inputs X, dense-model outputs Y: H = X^T X, G = X^T Y, const = ||Y||^2, then init and search."""
     wl = workloads.config(name, **over)
+    if lend:
+        solver.ensure_workspace(wl.d1, wl.m, wl.g, wl.k)
     W = wl.weight().numpy().astype(np.float64)
     xs = [wl.x_pruned_chunk(c) for c in range(wl.n_chunks)]
     ys = [wl.dense_output_chunk(c, dtype=ydt) for c in range(wl.n_chunks)]
