@@ -50,6 +50,10 @@ enum { OSSCAR_INIT_ENERGY = 0, OSSCAR_INIT_MAGNITUDE = 1, OSSCAR_INIT_USER = 2 }
 enum { OSSCAR_SCORE_INDEPENDENT = 0, OSSCAR_SCORE_PAIR_EXACT = 1 };
 enum { OSSCAR_ACCEPT_IMPROVING = 0, OSSCAR_ACCEPT_ALWAYS = 1 };
 enum { OSSCAR_STOP_MAX_SWAPS = 0, OSSCAR_STOP_NO_IMPROVEMENT = 1, OSSCAR_STOP_GUARD = 2 };
+/* Swap loop of single-row groups: AUTO picks PERSISTENT when the device can hold the cooperative grid;
+ * PERSISTENT = one cooperative kernel that runs all steps with bounded grid-wide barriers between their phases;
+ * LAUNCHES = five dependent launches per step, enqueued ahead of the device. */
+enum { OSSCAR_LOOP_AUTO = 0, OSSCAR_LOOP_PERSISTENT = 1, OSSCAR_LOOP_LAUNCHES = 2 };
 
 #define OSSCAR_MAX_GROUP 96   /* largest supported group size g */
 
@@ -57,6 +61,13 @@ enum { OSSCAR_STOP_MAX_SWAPS = 0, OSSCAR_STOP_NO_IMPROVEMENT = 1, OSSCAR_STOP_GU
  * legacy default stream).  create allocates a few KB of device and pinned host memory. */
 int osscar_create(osscar_ctx** out, int device, void* cuda_stream);
 int osscar_destroy(osscar_ctx* ctx);
+
+/* Budget, in SM clock cycles, of every bounded device-side wait of kernels launched through this context (mbarrier
+ * waits of the tensor-core pipelines, grid barriers of the persistent swap loop).  A wait that runs out makes its
+ * kernel return early and the call that reads the device status return OSSCAR_E_TIMEOUT; the context stays usable
+ * and the outputs of that call are unspecified.  0 restores the default (4e9 cycles, about two seconds).  Waits a
+ * kernel makes, while giving up, for its own copies and tensor-core work in flight keep the default budget. */
+int osscar_set_wait_limit(osscar_ctx* ctx, uint64_t cycles);
 
 /* Scratch needed by init_support / local_search / objective for a layer of this shape.
  * The caller allocates it on the device (256-byte aligned) and lends it with set_workspace;
@@ -142,6 +153,9 @@ typedef struct {
     double  accept_rel_tol;   /* IMPROVING: accept iff delta <= -tol * obj (1e-5 if < 0)     */
     int32_t profile_samples;  /* time each kernel of this many evenly spaced steps (0..8)    */
     int32_t block_pairs;      /* s: groups exchanged per iteration (0 or 1: one swap per step) */
+    int32_t loop_mode;        /* OSSCAR_LOOP_*: how the swap loop of single-row groups is driven */
+    int32_t reserved;         /* 0 */
+    uint64_t wait_limit_cycles; /* budget of the bounded device-side waits of this search; 0 = the context's value */
 } osscar_search_params;
 
 #define OSSCAR_NUM_STEP_KERNELS 12   /* select, pair Grams, y pass, small algebra, staging, H pass,
@@ -205,8 +219,10 @@ int osscar_debug_get_state(osscar_ctx* ctx, int which, void* dst);
  *   rows <= OSSCAR_NOALLOC_MAX_ROWS, else OSSCAR_E_SHAPE (the built-in scratch is 65536 + 32 doubles,
  *   about 512 KB, resident on every GPU that loads the library until the process exits).
  *   device: ordinal that owns A and B; cuda_stream: a cudaStream_t (NULL = legacy default stream).
- * The first call on a device looks up the device address of the built-in array; make that call before any
- * stream capture begins.  All calls share the array and it keeps the previous call's contents (each call
+ *   A or B not on `device`: OSSCAR_E_ARG.
+ * The first call on a device looks up the device address of the built-in array, and it may also be the moment the
+ * CUDA runtime loads this library's kernels onto the device (which allocates inside the driver); make that
+ * warm-up call before any stream capture begins and before the no-allocation regime starts.  All calls share the array and it keeps the previous call's contents (each call
  * overwrites every slot it later reads, so old contents never reach the result); calls whose kernels can
  * overlap on the GPU -- different streams, different threads -- race on it and must be serialised by the caller.
  * Synchronises the stream once, at its end.

@@ -19,15 +19,18 @@ SCORE_INDEPENDENT, SCORE_PAIR_EXACT = 0, 1
 ACCEPT_IMPROVING, ACCEPT_ALWAYS = 0, 1
 STOP_MAX_SWAPS, STOP_NO_IMPROVEMENT, STOP_GUARD = 0, 1, 2
 STOP_NAMES = {0: "max_swaps", 1: "no_improvement", 2: "guard"}
+LOOP_AUTO, LOOP_PERSISTENT, LOOP_LAUNCHES = 0, 1, 2
 
 EXPORTS = ["osscar_create", "osscar_destroy", "osscar_workspace_bytes", "osscar_set_workspace",
            "osscar_gram", "osscar_init_support", "osscar_local_search", "osscar_objective",
-           "osscar_debug_get_state", "osscar_status_string", "osscar_launch_count", "osscar_trace_noalloc", "osscar_init_support_greedy", "osscar_gram_cross", "osscar_set_const_term"]
+           "osscar_debug_get_state", "osscar_status_string", "osscar_launch_count", "osscar_trace_noalloc", "osscar_init_support_greedy", "osscar_gram_cross", "osscar_set_const_term",
+           "osscar_set_wait_limit"]
 
 
 class SearchParams(C.Structure):
     _fields_ = [("max_swaps", C.c_int32), ("score_mode", C.c_int32), ("accept_mode", C.c_int32),
-                ("refresh_every", C.c_int32), ("accept_rel_tol", C.c_double), ("profile_samples", C.c_int32), ("block_pairs", C.c_int32)]
+                ("refresh_every", C.c_int32), ("accept_rel_tol", C.c_double), ("profile_samples", C.c_int32), ("block_pairs", C.c_int32),
+                ("loop_mode", C.c_int32), ("reserved", C.c_int32), ("wait_limit_cycles", C.c_uint64)]
 
 
 class SearchResult(C.Structure):
@@ -80,6 +83,7 @@ def lib() -> C.CDLL:
     L.osscar_init_support_greedy.argtypes = [vp, vp, vp, vp, i64, i64, i32, i32, i32, vp, vp, C.POINTER(C.c_double), C.POINTER(i32)]
     L.osscar_gram_cross.argtypes = [vp, vp, C.c_int, vp, C.c_int, i64, i64, i64, C.c_int, C.c_float, vp, vp, C.POINTER(C.c_double)]
     L.osscar_set_const_term.argtypes = [vp, C.c_double, C.c_int]
+    L.osscar_set_wait_limit.argtypes = [vp, C.c_uint64]
     L.osscar_local_search.argtypes = [vp, C.POINTER(SearchParams), vp, vp, vp, vp, C.POINTER(SearchResult)]
     L.osscar_objective.argtypes = [vp, vp, vp, vp, i64, i64, C.POINTER(C.c_double)]
     L.osscar_debug_get_state.argtypes = [vp, C.c_int, vp]
@@ -245,6 +249,10 @@ class Solver:
                                            flags, damp, _ptr(H), _ptr(G), C.byref(const)), "osscar_gram_cross")
         return H, G, const.value
 
+    def set_wait_limit(self, cycles: int):
+        """Budget (SM cycles) of every bounded device-side wait of this context's kernels; 0 = default."""
+        _check(lib().osscar_set_wait_limit(self._h, int(cycles)), "osscar_set_wait_limit")
+
     def set_const_term(self, value: float, enabled: bool = True):
         _check(lib().osscar_set_const_term(self._h, float(value), int(enabled)), "osscar_set_const_term")
 
@@ -280,14 +288,15 @@ class Solver:
 
     def local_search(self, max_swaps: int, score_mode: int = SCORE_INDEPENDENT, accept_mode: int = ACCEPT_IMPROVING,
                      refresh_every: int = 0, accept_rel_tol: float = -1.0, profile_samples: int = 0,
-                     block_pairs: int = 0) -> SearchOutput:
+                     block_pairs: int = 0, loop_mode: int = LOOP_AUTO, wait_limit_cycles: int = 0) -> SearchOutput:
         d1, m, g, k = self._shape
         dev = self._keep[0].device
         support = torch.empty(k, dtype=torch.int32, device=dev)
         W_out = torch.empty(d1, m, dtype=torch.float32, device=dev)
         obj_trace = torch.zeros(max_swaps + 1, dtype=torch.float64, device=dev)
         swap_trace = torch.zeros(max(1, 2 * max_swaps), dtype=torch.int32, device=dev)
-        prm = SearchParams(max_swaps, score_mode, accept_mode, refresh_every, accept_rel_tol, profile_samples, block_pairs)
+        prm = SearchParams(max_swaps, score_mode, accept_mode, refresh_every, accept_rel_tol, profile_samples, block_pairs,
+                           loop_mode, 0, wait_limit_cycles)
         res = SearchResult()
         _check(lib().osscar_local_search(self._h, C.byref(prm), _ptr(support), _ptr(W_out), _ptr(obj_trace), _ptr(swap_trace),
                                          C.byref(res)), "osscar_local_search")

@@ -98,7 +98,7 @@ template <bool UPPER> __device__ __forceinline__ void tile_of(int id, int TM, in
 template <int MODE>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 k_mma_pipe(const __grid_constant__ Maps maps, int64_t M, int64_t N, int64_t K, float alpha, float beta,
-           float* __restrict__ C, int64_t ldc, int vec_ok, int num_ids, int32_t* __restrict__ status,
+           float* __restrict__ C, int64_t ldc, int vec_ok, int num_ids, SearchCtl* __restrict__ ctl,
            const int32_t* __restrict__ done)
 {
     using TR = Traits<MODE>;
@@ -114,9 +114,11 @@ k_mma_pipe(const __grid_constant__ Maps maps, int64_t M, int64_t N, int64_t K, f
     auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
     auto tfull_bar = [&](int b) { return bars + 8u * (2 * STAGES + b); };
     auto tempty_bar = [&](int b) { return bars + 8u * (2 * STAGES + 2 + b); };
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_ptr + 8 * (2 * STAGES + 4));
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_ptr + 8 * (2 * STAGES + 4) + 8);
+    const uint32_t drain_bar = bars + 8u * (2 * STAGES + 4);   // completion of the MMAs in flight when the issuer gives up
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_ptr + 8 * (2 * STAGES + 5));
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_ptr + 8 * (2 * STAGES + 5) + 8);
     float* epi = reinterpret_cast<float*>(bar_ptr + 256);      // staging blocks of the accumulate warps
+    const long long wl = ctl->wait_limit;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int TM = (int)((M + TILE_M - 1) / TILE_M), TN = (int)((N + TILE_N - 1) / TILE_N);
@@ -126,6 +128,7 @@ k_mma_pipe(const __grid_constant__ Maps maps, int64_t M, int64_t N, int64_t K, f
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 8); }
+        mbar_init(drain_bar, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -153,7 +156,7 @@ k_mma_pipe(const __grid_constant__ Maps maps, int64_t M, int64_t N, int64_t K, f
                                      : (MODE == MODE_CROSS3 ? 2 - term : 0);
                         const int s = it % STAGES;
                         const uint32_t ph = (it / STAGES) & 1;
-                        if (!mbar_wait(empty_bar(s), ph ^ 1, abort_flag)) { ok = false; break; }
+                        if (!mbar_wait(empty_bar(s), ph ^ 1, abort_flag, wl)) { ok = false; break; }
                         mbar_expect_tx(full_bar(s), STAGE_BYTES);
                         const uint32_t a_dst = tiles_base + s * STAGE_BYTES;
                         const uint32_t b_dst = a_dst + A_BYTES;
@@ -170,13 +173,9 @@ k_mma_pipe(const __grid_constant__ Maps maps, int64_t M, int64_t N, int64_t K, f
                     }
                 }
             }
-            if (*abort_flag) {
+            if (*abort_flag) {                    // the copies still in flight must land before the CTA exits
                 const uint32_t first = it > STAGES ? it - STAGES : 0;
-                for (uint32_t j = first; j < it; ++j) {
-                    const long long t0 = clock64();
-                    while (!mbar_try_wait(full_bar(j % STAGES), (j / STAGES) & 1))
-                        if (clock64() - t0 > kWaitLimitCycles) break;
-                }
+                for (uint32_t j = first; j < it; ++j) mbar_drain(full_bar(j % STAGES), (j / STAGES) & 1);
             }
         }
     } else if (warp == 1) {
@@ -186,7 +185,7 @@ k_mma_pipe(const __grid_constant__ Maps maps, int64_t M, int64_t N, int64_t K, f
             for (int id = blockIdx.x; id < num_ids && ok; id += gridDim.x) {
                 for (int f = 0; f < nflush && ok; ++f, ++fl) {
                     const int buf = fl & 1;
-                    if (!mbar_wait(tempty_bar(buf), ((fl >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(tempty_bar(buf), ((fl >> 1) & 1) ^ 1, abort_flag, wl)) { ok = false; break; }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint32_t d_tmem = tmem_base + (uint32_t)(buf * TILE_N);
                     const int kb1 = min(nkb, (f + 1) * kFlush);
@@ -195,7 +194,7 @@ k_mma_pipe(const __grid_constant__ Maps maps, int64_t M, int64_t N, int64_t K, f
                         for (int term = 0; term < kTerms; ++term, ++it) {
                             const int s = it % STAGES;
                             const uint32_t ph = (it / STAGES) & 1;
-                            if (!mbar_wait(full_bar(s), ph, abort_flag)) { ok = false; break; }
+                            if (!mbar_wait(full_bar(s), ph, abort_flag, wl)) { ok = false; break; }
                             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                             const uint32_t a_src = tiles_base + s * STAGE_BYTES;
                             const uint32_t b_src = a_src + A_BYTES;
@@ -211,6 +210,10 @@ k_mma_pipe(const __grid_constant__ Maps maps, int64_t M, int64_t N, int64_t K, f
                     }
                     if (ok) umma_commit(tfull_bar(buf));
                 }
+            }
+            if (!ok) {            // MMAs already issued keep running: they must finish before TMEM and the tiles are released
+                umma_commit(drain_bar);
+                mbar_drain(drain_bar, 0);
             }
         }
     } else {
@@ -235,7 +238,7 @@ k_mma_pipe(const __grid_constant__ Maps maps, int64_t M, int64_t N, int64_t K, f
             }
             for (int f = 0; f < nflush && ok; ++f, ++fl) {
                 const int buf = fl & 1;
-                if (!mbar_wait(tfull_bar(buf), (fl >> 1) & 1, abort_flag)) { ok = false; break; }
+                if (!mbar_wait(tfull_bar(buf), (fl >> 1) & 1, abort_flag, wl)) { ok = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
@@ -309,7 +312,7 @@ k_mma_pipe(const __grid_constant__ Maps maps, int64_t M, int64_t N, int64_t K, f
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "n"(TMEM_COLS) : "memory");
     }
-    if (threadIdx.x == 0 && *abort_flag) *status = OSSCAR_E_TIMEOUT;
+    if (threadIdx.x == 0 && *abort_flag) ctl->status = OSSCAR_E_TIMEOUT;
 }
 
 // x = x1 + x2 + x3 with bf16 terms (round to nearest each time); dst rows are ldd wide, the tail is zero.
@@ -348,7 +351,7 @@ constexpr uint32_t kRuIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | 
 
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 k_rank_update(const __grid_constant__ Maps maps, int64_t M, int64_t N, int nkb, float alpha, float* __restrict__ C, int64_t ldc,
-              int TN, int nchunk, int num_items, float* __restrict__ sq_part, int32_t* __restrict__ status,
+              int TN, int nchunk, int num_items, float* __restrict__ sq_part, SearchCtl* __restrict__ ctl,
               const int32_t* __restrict__ done)
 {
     if (done && *done) return;
@@ -363,15 +366,16 @@ k_rank_update(const __grid_constant__ Maps maps, int64_t M, int64_t N, int nkb, 
     auto w_empty = [&](int s) { return bars + 8u * (2 + s); };
     auto tfull_bar = [&](int b) { return bars + 8u * (4 + b); };
     auto tempty_bar = [&](int b) { return bars + 8u * (6 + b); };
-    const uint32_t u_full = bars + 8u * 8, u_empty = bars + 8u * 9;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_ptr + 8 * 10);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_ptr + 8 * 10 + 8);
+    const uint32_t u_full = bars + 8u * 8, u_empty = bars + 8u * 9, drain_bar = bars + 8u * 10;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_ptr + 8 * 11);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_ptr + 8 * 11 + 8);
     float* epi = reinterpret_cast<float*>(bar_ptr + 256);
+    const long long wl = ctl->wait_limit;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
         for (int i = 0; i < 2; ++i) { mbar_init(w_full(i), 1); mbar_init(w_empty(i), 1); mbar_init(tfull_bar(i), 1); mbar_init(tempty_bar(i), 8); }
-        mbar_init(u_full, 1); mbar_init(u_empty, 1);
+        mbar_init(u_full, 1); mbar_init(u_empty, 1); mbar_init(drain_bar, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -399,7 +403,7 @@ k_rank_update(const __grid_constant__ Maps maps, int64_t M, int64_t N, int nkb, 
                 int tm, tn0, tn1;
                 item_of(id, &tm, &tn0, &tn1);
                 if (tn0 >= tn1) continue;
-                if (!mbar_wait(u_empty, (item & 1) ^ 1, abort_flag)) { ok = false; break; }
+                if (!mbar_wait(u_empty, (item & 1) ^ 1, abort_flag, wl)) { ok = false; break; }
                 ++item;
                 mbar_expect_tx(u_full, (uint32_t)(3 * nkb * A_BYTES));
                 for (int kb = 0; kb < nkb; ++kb)
@@ -409,7 +413,7 @@ k_rank_update(const __grid_constant__ Maps maps, int64_t M, int64_t N, int nkb, 
                 for (int tn = tn0; tn < tn1 && ok; ++tn) {
                     for (int kb = 0; kb < nkb; ++kb, ++it) {
                         const int s = it & 1;
-                        if (!mbar_wait(w_empty(s), ((it >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
+                        if (!mbar_wait(w_empty(s), ((it >> 1) & 1) ^ 1, abort_flag, wl)) { ok = false; break; }
                         mbar_expect_tx(w_full(s), RU_W_BYTES);
 #pragma unroll
                         for (int term = 0; term < 3; ++term)
@@ -421,9 +425,8 @@ k_rank_update(const __grid_constant__ Maps maps, int64_t M, int64_t N, int nkb, 
                 }
             }
             if (*abort_flag) {                    // let the copies in flight land before the CTA exits
-                const long long t0 = clock64();
-                while (it > 0 && !mbar_try_wait(w_full((it - 1) & 1), ((it - 1) >> 1) & 1))
-                    if (clock64() - t0 > kWaitLimitCycles) break;
+                if (item > 0) mbar_drain(u_full, (item - 1) & 1);
+                for (uint32_t j = it > 2 ? it - 2 : 0; j < it; ++j) mbar_drain(w_full(j & 1), (j >> 1) & 1);
             }
         }
     } else if (warp == 1) {
@@ -434,17 +437,17 @@ k_rank_update(const __grid_constant__ Maps maps, int64_t M, int64_t N, int nkb, 
                 int tm, tn0, tn1;
                 item_of(id, &tm, &tn0, &tn1);
                 if (tn0 >= tn1) continue;
-                if (!mbar_wait(u_full, item & 1, abort_flag)) { ok = false; break; }
+                if (!mbar_wait(u_full, item & 1, abort_flag, wl)) { ok = false; break; }
                 ++item;
                 for (int tn = tn0; tn < tn1 && ok; ++tn, ++tile) {
                     const int buf = tile & 1;
-                    if (!mbar_wait(tempty_bar(buf), ((tile >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(tempty_bar(buf), ((tile >> 1) & 1) ^ 1, abort_flag, wl)) { ok = false; break; }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint32_t d_tmem = tmem_base + (uint32_t)(buf * RU_TN);
                     bool first = true;
                     for (int kb = 0; kb < nkb && ok; ++kb, ++it) {
                         const int s = it & 1;
-                        if (!mbar_wait(w_full(s), (it >> 1) & 1, abort_flag)) { ok = false; break; }
+                        if (!mbar_wait(w_full(s), (it >> 1) & 1, abort_flag, wl)) { ok = false; break; }
                         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
                         for (int term = 0; term < 6; ++term) {
@@ -463,6 +466,10 @@ k_rank_update(const __grid_constant__ Maps maps, int64_t M, int64_t N, int nkb, 
                     if (ok) umma_commit(tfull_bar(buf));
                 }
                 if (ok) umma_commit(u_empty);        // the band's terms may be replaced once these MMAs are done
+            }
+            if (!ok) {            // MMAs already issued must finish before TMEM and the operand tiles are released
+                umma_commit(drain_bar);
+                mbar_drain(drain_bar, 0);
             }
         }
     } else {
@@ -483,7 +490,7 @@ k_rank_update(const __grid_constant__ Maps maps, int64_t M, int64_t N, int nkb, 
                     for (int j = 0; j < 64; j += 32)
                         if (gcol0 + j < N) asm volatile("prefetch.global.L2 [%0];" ::"l"(C + (grow0 + lane) * ldc + gcol0 + j));
                 }
-                if (!mbar_wait(tfull_bar(buf), (tile >> 1) & 1, abort_flag)) { ok = false; break; }
+                if (!mbar_wait(tfull_bar(buf), (tile >> 1) & 1, abort_flag, wl)) { ok = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 float acc[64];
 #pragma unroll
@@ -544,7 +551,7 @@ k_rank_update(const __grid_constant__ Maps maps, int64_t M, int64_t N, int nkb, 
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "n"(256) : "memory");
     }
-    if (threadIdx.x == 0 && *abort_flag) *status = OSSCAR_E_TIMEOUT;
+    if (threadIdx.x == 0 && *abort_flag) ctl->status = OSSCAR_E_TIMEOUT;
 }
 
 bool encode_2d(PFN_encodeTiled enc, CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer, uint64_t ld_elems,
@@ -569,7 +576,7 @@ size_t gemm_tc_min_scratch(int64_t M, int64_t N)
 
 cudaError_t gemm_tc(cudaStream_t st, int64_t M, int64_t N, int64_t K, float alpha, const float* A, int64_t lda,
                     const float* B, int64_t ldb, float beta, float* C, int64_t ldc,
-                    void* scratch, size_t scratch_bytes, int32_t* status_dev, const int32_t* done)
+                    void* scratch, size_t scratch_bytes, SearchCtl* ctl_dev, const int32_t* done)
 {
     if (M <= 0 || N <= 0) return cudaSuccess;
     if (K <= 0 || scratch_bytes < gemm_tc_min_scratch(M, N) || ((uintptr_t)scratch & 255)) return cudaErrorInvalidValue;
@@ -611,7 +618,7 @@ cudaError_t gemm_tc(cudaStream_t st, int64_t M, int64_t N, int64_t K, float alph
         }
         const int grid = num_ids < sms ? num_ids : sms;
         k_mma_pipe<MODE_GEMM3><<<grid, NUM_THREADS, SMEM_BYTES, st>>>(maps, M, N, kw, alpha, k0 == 0 ? beta : 1.f, C, ldc, vec_ok,
-                                                                      num_ids, status_dev, done);
+                                                                      num_ids, ctl_dev, done);
         count_launches(3);
         e = cudaGetLastError();
         if (e != cudaSuccess) return e;
@@ -639,13 +646,13 @@ __global__ void k_rownorm_sum(const float* __restrict__ part, int64_t rows, int 
 // out of the same pass (short-dimension path only; returns cudaErrorInvalidValue otherwise).
 cudaError_t rank_update_tc(cudaStream_t st, int64_t M, int64_t N, int64_t K, float alpha, const float* U, int64_t ldu,
                            const float* W, int64_t ldw, float* C, int64_t ldc,
-                           void* scratch, size_t scratch_bytes, int32_t* status_dev, const int32_t* done,
+                           void* scratch, size_t scratch_bytes, SearchCtl* ctl_dev, const int32_t* done,
                            float* row_sq, float* sq_scratch)
 {
     if (M <= 0 || N <= 0 || K <= 0) return cudaSuccess;
     const bool fits = K <= 2 * BLOCK_K && (N % 4) == 0 && (ldc % 4) == 0 && (((uintptr_t)C & 15) == 0);
     if (!fits && row_sq) return cudaErrorInvalidValue;
-    if (!fits) return gemm_tc(st, M, N, K, alpha, U, ldu, W, ldw, 1.f, C, ldc, scratch, scratch_bytes, status_dev, done);
+    if (!fits) return gemm_tc(st, M, N, K, alpha, U, ldu, W, ldw, 1.f, C, ldc, scratch, scratch_bytes, ctl_dev, done);
     PFN_encodeTiled enc = get_encode();
     if (!enc) return cudaErrorNotSupported;
     if ((uintptr_t)scratch & 255) return cudaErrorInvalidValue;
@@ -681,7 +688,7 @@ cudaError_t rank_update_tc(cudaStream_t st, int64_t M, int64_t N, int64_t K, flo
     const int num_items = TM * nchunk;
     const int nkb = (int)((K + BLOCK_K - 1) / BLOCK_K);
     k_rank_update<<<num_items < sms ? num_items : sms, NUM_THREADS, RU_SMEM, st>>>(maps, M, N, nkb, alpha, C, ldc, TN, nchunk, num_items,
-                                                                                  row_sq ? sq_scratch : nullptr, status_dev, done);
+                                                                                  row_sq ? sq_scratch : nullptr, ctl_dev, done);
     count_launches(3);
     if (row_sq) {
         k_rownorm_sum<<<(unsigned)((M + 255) / 256), 256, 0, st>>>(sq_scratch, M, 2 * TN, row_sq, done);
@@ -694,7 +701,7 @@ cudaError_t rank_update_tc(cudaStream_t st, int64_t M, int64_t N, int64_t K, flo
 // Xc: n_rows x d1 bf16.  Yc: n_rows x m, bf16 (y_fp32 == 0) or fp32, which is split into three bf16 terms in
 // `scratch` (3 * n_rows * round_up(m, 8) * 2 bytes, 1024-byte aligned pieces).
 cudaError_t gram_tc2(cudaStream_t st, const void* X, int64_t n_rows, int64_t d1, const void* Y, int y_fp32, int64_t m,
-                     float* C, bool accumulate, void* scratch, size_t scratch_bytes, int32_t* status_dev)
+                     float* C, bool accumulate, void* scratch, size_t scratch_bytes, SearchCtl* ctl_dev)
 {
     if (n_rows <= 0) return cudaSuccess;
     if (((uintptr_t)X & 15) || (d1 % 8) != 0) return cudaErrorInvalidValue;
@@ -719,7 +726,7 @@ cudaError_t gram_tc2(cudaStream_t st, const void* X, int64_t n_rows, int64_t d1,
         e = cudaFuncSetAttribute(k_mma_pipe<MODE_GRAM>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
         if (e != cudaSuccess) return e;
         k_mma_pipe<MODE_GRAM><<<num_ids < sms ? num_ids : sms, NUM_THREADS, SMEM_BYTES, st>>>(
-            maps, d1, d1, n_rows, 1.f, beta, C, d1, vec_ok, num_ids, status_dev, nullptr);
+            maps, d1, d1, n_rows, 1.f, beta, C, d1, vec_ok, num_ids, ctl_dev, nullptr);
         count_launches(1);
         return cudaGetLastError();
     }
@@ -733,7 +740,7 @@ cudaError_t gram_tc2(cudaStream_t st, const void* X, int64_t n_rows, int64_t d1,
         e = cudaFuncSetAttribute(k_mma_pipe<MODE_CROSS>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
         if (e != cudaSuccess) return e;
         k_mma_pipe<MODE_CROSS><<<num_ids < sms ? num_ids : sms, NUM_THREADS, SMEM_BYTES, st>>>(
-            maps, d1, m, n_rows, 1.f, beta, C, m, vec_ok, num_ids, status_dev, nullptr);
+            maps, d1, m, n_rows, 1.f, beta, C, m, vec_ok, num_ids, ctl_dev, nullptr);
         count_launches(1);
         return cudaGetLastError();
     }
@@ -748,7 +755,7 @@ cudaError_t gram_tc2(cudaStream_t st, const void* X, int64_t n_rows, int64_t d1,
     e = cudaFuncSetAttribute(k_mma_pipe<MODE_CROSS3>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e != cudaSuccess) return e;
     k_mma_pipe<MODE_CROSS3><<<num_ids < sms ? num_ids : sms, NUM_THREADS, SMEM_BYTES, st>>>(
-        maps, d1, m, n_rows, 1.f, beta, C, m, vec_ok, num_ids, status_dev, nullptr);
+        maps, d1, m, n_rows, 1.f, beta, C, m, vec_ok, num_ids, ctl_dev, nullptr);
     count_launches(2);
     return cudaGetLastError();
 }
@@ -758,7 +765,7 @@ cudaError_t gram_tc2(cudaStream_t st, const void* X, int64_t n_rows, int64_t d1,
 // sized to the scratch (each panel needs 6 * rows * round_up(d1, 8) bytes).  Returns cudaErrorMemoryAllocation when
 // the scratch cannot hold a panel of 64 rows, so that the caller can take another path.
 cudaError_t gram_tc3(cudaStream_t st, const float* X, int64_t n_rows, int64_t d1, float* C, bool accumulate,
-                     void* scratch, size_t scratch_bytes, int32_t* status_dev)
+                     void* scratch, size_t scratch_bytes, SearchCtl* ctl_dev)
 {
     if (n_rows <= 0) return cudaSuccess;
     const int64_t ldn = round_up(d1, 8);
@@ -792,7 +799,7 @@ cudaError_t gram_tc3(cudaStream_t st, const float* X, int64_t n_rows, int64_t d1
             maps.b[i] = maps.a[i];
         }
         k_mma_pipe<MODE_GRAM3><<<num_ids < sms ? num_ids : sms, NUM_THREADS, SMEM_BYTES, st>>>(
-            maps, d1, d1, rows, 1.f, (accumulate || r0 > 0) ? 1.f : 0.f, C, d1, vec_ok, num_ids, status_dev, nullptr);
+            maps, d1, d1, rows, 1.f, (accumulate || r0 > 0) ? 1.f : 0.f, C, d1, vec_ok, num_ids, ctl_dev, nullptr);
         count_launches(2);
     }
     return cudaGetLastError();

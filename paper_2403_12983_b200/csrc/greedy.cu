@@ -404,9 +404,9 @@ int greedy_support(osscar_ctx* ctx, int t_hat, int32_t* support, int32_t* drop_t
         if (Tt >= 32) {
             // wide downdates: A -= BC^T B and V -= B^T KT as products with inner dimension T on the tensor cores
             void* tc = ws + L.off_tc;
-            if (rank_update_tc(st, nrows, round_up(nrows, 4), Tt, -1.f, p.BCT, Tt, p.B, p.lda, p.A, p.lda, tc, L.tc_bytes, &ctx->ctl->status)
+            if (rank_update_tc(st, nrows, round_up(nrows, 4), Tt, -1.f, p.BCT, Tt, p.B, p.lda, p.A, p.lda, tc, L.tc_bytes, ctx->ctl)
                     != cudaSuccess) return OSSCAR_E_CUDA;
-            if (rank_update_tc(st, nrows, p.ldv, Tt, -1.f, p.BT, Tt, p.KT, p.ldv, p.V, p.ldv, tc, L.tc_bytes, &ctx->ctl->status)
+            if (rank_update_tc(st, nrows, p.ldv, Tt, -1.f, p.BT, Tt, p.KT, p.ldv, p.V, p.ldv, tc, L.tc_bytes, ctx->ctl)
                     != cudaSuccess) return OSSCAR_E_CUDA;
         } else {
             const int64_t nc4 = (round_up(nrows, 4)) / 4;

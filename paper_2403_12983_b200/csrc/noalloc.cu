@@ -3,7 +3,10 @@
 // library image.  See osscar_trace_noalloc in osscar.h for who needs this and for its limits.
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <atomic>
 #include "osscar.h"
+
+namespace osscar { extern unsigned long long g_launches; }     // the library-wide launch counter (osscar_launch_count)
 
 namespace {
 
@@ -12,7 +15,17 @@ namespace {
 static __device__ __align__(256) double g_noalloc_scratch[OSSCAR_NOALLOC_MAX_ROWS + 32];
 
 constexpr int kMaxDevices = 64;
-double* g_scratch_addr[kMaxDevices] = {};      // device address of the array, looked up once per device
+// Device address of the array, looked up on first use per device.  Callers on different host threads may arrive here
+// together; every writer stores the same value, and the atomic makes that store and the later loads well defined.
+std::atomic<double*> g_scratch_addr[kMaxDevices];
+
+// true iff p is device memory of `device` (or managed memory, which every device can reach)
+bool on_device(const void* p, int device)
+{
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, p) != cudaSuccess) { cudaGetLastError(); return false; }
+    return at.type == cudaMemoryTypeManaged || (at.type == cudaMemoryTypeDevice && at.device == device);
+}
 
 __device__ __forceinline__ double warp_sum_d(double v) {
 #pragma unroll
@@ -67,19 +80,23 @@ extern "C" int osscar_trace_noalloc(const float* A, int64_t lda, const float* B,
     if (cudaGetDevice(&prev) != cudaSuccess) return OSSCAR_E_CUDA;
     if (prev != device && cudaSetDevice(device) != cudaSuccess) return OSSCAR_E_CUDA;
     int rc = OSSCAR_OK;
+    // the kernels run on `device`: both matrices must live there (a wrong ordinal would aim them at foreign pointers)
+    if (rows > 0 && cols > 0 && (!on_device(A, device) || !on_device(B, device))) rc = OSSCAR_E_ARG;
     // Set-up, once per device and with that device current: the array's name is only a host-side handle;
     // kernels must be given the device address that the runtime reports for it.
-    if (!g_scratch_addr[device]) {
+    double* scratch = g_scratch_addr[device].load(std::memory_order_acquire);
+    if (rc == OSSCAR_OK && !scratch) {
         double* p = nullptr;
         if (cudaGetSymbolAddress((void**)&p, g_noalloc_scratch) != cudaSuccess || !p) rc = OSSCAR_E_CUDA;
-        else g_scratch_addr[device] = p;
+        else { g_scratch_addr[device].store(p, std::memory_order_release); scratch = p; }
     }
     if (rc == OSSCAR_OK) {
         cudaStream_t st = (cudaStream_t)cuda_stream;
-        double* partial = g_scratch_addr[device];
+        double* partial = scratch;
         double* total = partial + OSSCAR_NOALLOC_MAX_ROWS;
         if (rows > 0 && cols > 0) k_noalloc_rows<<<(unsigned)rows, 256, 0, st>>>(A, lda, B, ldb, cols, partial);
         k_noalloc_total<<<1, 1024, 0, st>>>(partial, (rows > 0 && cols > 0) ? rows : 0, total);
+        osscar::g_launches += (rows > 0 && cols > 0) ? 2 : 1;
         if (cudaGetLastError() != cudaSuccess
             || cudaMemcpyAsync(out, total, sizeof(double), cudaMemcpyDeviceToHost, st) != cudaSuccess
             || cudaStreamSynchronize(st) != cudaSuccess)

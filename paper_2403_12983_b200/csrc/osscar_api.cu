@@ -3,6 +3,7 @@
 #include <new>
 #include <string.h>
 #include <cuda_bf16.h>
+#include "tc_common.cuh"
 
 using namespace osscar;
 
@@ -11,6 +12,9 @@ namespace osscar { unsigned long long g_launches = 0; }
 namespace {
 
 #define CKC(x) do { cudaError_t e_ = (x); if (e_ != cudaSuccess) return OSSCAR_E_CUDA; } while (0)
+// the same for calls that follow enqueued work: the stream is drained first, so that a failed call never returns with
+// kernels still running on the caller's buffers
+#define CKS(x) do { cudaError_t e_ = (x); if (e_ != cudaSuccess) { cudaStreamSynchronize(st); return OSSCAR_E_CUDA; } } while (0)
 
 struct DeviceGuard {
     int prev; bool ok;
@@ -22,6 +26,7 @@ struct DeviceGuard {
 };
 
 __global__ void k_clear_status(SearchCtl* ctl) { ctl->status = OSSCAR_OK; ctl->done = 0; }
+__global__ void k_set_wait_limit(SearchCtl* ctl, long long cycles) { ctl->wait_limit = cycles; }
 
 // diag sum of H in fp64, then H += damp * mean(diag) * I
 __global__ void k_diag_sum(const float* __restrict__ H, int64_t d1, double* __restrict__ out)
@@ -110,6 +115,11 @@ int osscar_create(osscar_ctx** out, int device, void* cuda_stream)
            && cudaHostAlloc((void**)&ctx->done_flag_host, 64, cudaHostAllocMapped) == cudaSuccess
            && cudaHostGetDevicePointer((void**)&ctx->done_flag_dev, (void*)ctx->done_flag_host, 0) == cudaSuccess
            && cudaEventCreate(&ctx->ev0) == cudaSuccess && cudaEventCreate(&ctx->ev1) == cudaSuccess;
+    if (ok) {
+        ctx->wait_limit = tc::kWaitLimitCycles;
+        k_set_wait_limit<<<1, 1>>>(ctx->ctl, ctx->wait_limit);
+        ok = cudaDeviceSynchronize() == cudaSuccess;
+    }
     if (!ok) { osscar_destroy(ctx); return OSSCAR_E_CUDA; }
     *ctx->done_flag_host = 0;
     *out = ctx;
@@ -127,6 +137,19 @@ int osscar_destroy(osscar_ctx* ctx)
     if (ctx->ev0) cudaEventDestroy(ctx->ev0);
     if (ctx->ev1) cudaEventDestroy(ctx->ev1);
     delete ctx;
+    return OSSCAR_OK;
+}
+
+int osscar_set_wait_limit(osscar_ctx* ctx, uint64_t cycles)
+{
+    if (!ctx) return OSSCAR_E_ARG;
+    if (cycles > (uint64_t)1 << 62) return OSSCAR_E_ARG;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return OSSCAR_E_CUDA;
+    ctx->wait_limit = cycles ? (long long)cycles : tc::kWaitLimitCycles;
+    k_set_wait_limit<<<1, 1, 0, ctx->stream>>>(ctx->ctl, ctx->wait_limit);
+    count_launches(1);
+    CKC(cudaGetLastError());
     return OSSCAR_OK;
 }
 
@@ -164,33 +187,33 @@ int osscar_gram(osscar_ctx* ctx, const void* X, int x_dtype, int64_t n_rows, int
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return OSSCAR_E_CUDA;
     cudaStream_t st = ctx->stream;
-    k_clear_status<<<1, 1, 0, st>>>(ctx->ctl);
-    count_launches(1);
+    // a device-side error of any chunk must reach the END call: the status is cleared by the BEGIN chunk only
+    if (begin) { k_clear_status<<<1, 1, 0, st>>>(ctx->ctl); count_launches(1); }
     if (begin) ctx->gram_rows = 0;
-    if (begin && n_rows == 0) CKC(cudaMemsetAsync(H, 0, sizeof(float) * d1 * d1, st));
+    if (begin && n_rows == 0) CKS(cudaMemsetAsync(H, 0, sizeof(float) * d1 * d1, st));
     if (n_rows > 0) {
         if (x_dtype == OSSCAR_BF16) {
             // upper-triangle tiles only; the lower triangle is filled on END
-            CKC(gram_tc2(st, X, n_rows, d1, nullptr, 0, 0, H, !begin, nullptr, 0, &ctx->ctl->status));
+            CKS(gram_tc2(st, X, n_rows, d1, nullptr, 0, 0, H, !begin, nullptr, 0, ctx->ctl));
         } else {
             // fp32 activations: three-term bf16 split on the tensor cores when a workspace is lent (its contents are
             // overwritten), else (or when it cannot hold a 64-row panel of the terms) the fp32 pipes
             cudaError_t ge = cudaErrorMemoryAllocation;
             if (ctx->ws) {
-                ge = gram_tc3(st, (const float*)X, n_rows, d1, H, !begin, ctx->ws, ctx->ws_bytes, &ctx->ctl->status);
+                ge = gram_tc3(st, (const float*)X, n_rows, d1, H, !begin, ctx->ws, ctx->ws_bytes, ctx->ctl);
                 if (ge == cudaSuccess) ctx->have_state = false;
             }
             if (ge == cudaErrorMemoryAllocation)
                 ge = sgemm(st, true, false, d1, d1, n_rows, 1.f, (const float*)X, d1, (const float*)X, d1, begin ? 0.f : 1.f, H, d1);
-            CKC(ge);
+            CKS(ge);
         }
         ctx->gram_rows += (double)n_rows;
     }
-    if (!end) { CKC(cudaGetLastError()); return OSSCAR_OK; }
+    if (!end) { CKS(cudaGetLastError()); return OSSCAR_OK; }
     ctx->have_const = false;
-    CKC(gram_mirror(st, H, d1));
+    CKS(gram_mirror(st, H, d1));
     if (damp > 0.f) {
-        CKC(cudaMemsetAsync(&ctx->ctl->acc[0], 0, sizeof(double), st));
+        CKS(cudaMemsetAsync(&ctx->ctl->acc[0], 0, sizeof(double), st));
         k_diag_sum<<<64, 256, 0, st>>>(H, d1, &ctx->ctl->acc[0]);
         k_add_damp<<<64, 256, 0, st>>>(H, d1, damp, &ctx->ctl->acc[0]);
         count_launches(2);
@@ -198,14 +221,14 @@ int osscar_gram(osscar_ctx* ctx, const void* X, int x_dtype, int64_t n_rows, int
     if (ctx->ws && ctx->ws_bytes >= gemm_tc_min_scratch(d1, m)) {
         // tensor-core product with the operand terms staged in the lent workspace (its contents are overwritten)
         const size_t cap = ctx->ws_bytes < ((size_t)3 << 30) ? ctx->ws_bytes : ((size_t)3 << 30);
-        CKC(gemm_tc(st, d1, m, d1, 1.f, H, d1, W, m, 0.f, G, m, ctx->ws, cap, &ctx->ctl->status));
+        CKS(gemm_tc(st, d1, m, d1, 1.f, H, d1, W, m, 0.f, G, m, ctx->ws, cap, ctx->ctl));
         ctx->have_state = false;
     } else {
-        CKC(sgemm(st, false, false, d1, m, d1, 1.f, H, d1, W, m, 0.f, G, m));
+        CKS(sgemm(st, false, false, d1, m, d1, 1.f, H, d1, W, m, 0.f, G, m));
     }
-    CKC(trace_product(st, W, m, G, m, d1, m, ctx->partials, &ctx->ctl->acc[1]));
-    CKC(cudaMemcpyAsync(ctx->ctl_host, ctx->ctl, sizeof(SearchCtl), cudaMemcpyDeviceToHost, st));
-    CKC(cudaStreamSynchronize(st));
+    CKS(trace_product(st, W, m, G, m, d1, m, ctx->partials, &ctx->ctl->acc[1]));
+    CKS(cudaMemcpyAsync(ctx->ctl_host, ctx->ctl, sizeof(SearchCtl), cudaMemcpyDeviceToHost, st));
+    CKS(cudaStreamSynchronize(st));
     if (ctx->ctl_host->status != OSSCAR_OK) return ctx->ctl_host->status;
     *const_term = ctx->ctl_host->acc[1];
     return OSSCAR_OK;
@@ -232,45 +255,44 @@ int osscar_gram_cross(osscar_ctx* ctx, const void* X, int x_dtype, const void* Y
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return OSSCAR_E_CUDA;
     cudaStream_t st = ctx->stream;
-    k_clear_status<<<1, 1, 0, st>>>(ctx->ctl);
-    count_launches(1);
+    if (begin) { k_clear_status<<<1, 1, 0, st>>>(ctx->ctl); count_launches(1); }     // sticky until END, as in osscar_gram
     if (begin && n_rows == 0) {
-        CKC(cudaMemsetAsync(H, 0, sizeof(float) * d1 * d1, st));
-        CKC(cudaMemsetAsync(G, 0, sizeof(float) * d1 * m, st));
-        CKC(cudaMemsetAsync(&ctx->ctl->acc[2], 0, sizeof(double), st));
+        CKS(cudaMemsetAsync(H, 0, sizeof(float) * d1 * d1, st));
+        CKS(cudaMemsetAsync(G, 0, sizeof(float) * d1 * m, st));
+        CKS(cudaMemsetAsync(&ctx->ctl->acc[2], 0, sizeof(double), st));
     }
     if (n_rows > 0) {
         if (x_dtype == OSSCAR_BF16) {
-            CKC(gram_tc2(st, X, n_rows, d1, nullptr, 0, 0, H, !begin, nullptr, 0, &ctx->ctl->status));
-            CKC(gram_tc2(st, X, n_rows, d1, Y, y_dtype == OSSCAR_FP32, m, G, !begin, ctx->ws, ctx->ws_bytes, &ctx->ctl->status));
+            CKS(gram_tc2(st, X, n_rows, d1, nullptr, 0, 0, H, !begin, nullptr, 0, ctx->ctl));
+            CKS(gram_tc2(st, X, n_rows, d1, Y, y_dtype == OSSCAR_FP32, m, G, !begin, ctx->ws, ctx->ws_bytes, ctx->ctl));
             if (need > 0) ctx->have_state = false;
         } else {
             // H as in osscar_gram: on the tensor cores when a workspace can stage the bf16 terms, else the fp32 pipes
             cudaError_t ge = cudaErrorMemoryAllocation;
             if (ctx->ws) {
-                ge = gram_tc3(st, (const float*)X, n_rows, d1, H, !begin, ctx->ws, ctx->ws_bytes, &ctx->ctl->status);
+                ge = gram_tc3(st, (const float*)X, n_rows, d1, H, !begin, ctx->ws, ctx->ws_bytes, ctx->ctl);
                 if (ge == cudaSuccess) ctx->have_state = false;
             }
             if (ge == cudaErrorMemoryAllocation)
                 ge = sgemm(st, true, false, d1, d1, n_rows, 1.f, (const float*)X, d1, (const float*)X, d1, begin ? 0.f : 1.f, H, d1);
-            CKC(ge);
-            CKC(sgemm(st, true, false, d1, m, n_rows, 1.f, (const float*)X, d1, (const float*)Y, m, begin ? 0.f : 1.f, G, m));
+            CKS(ge);
+            CKS(sgemm(st, true, false, d1, m, n_rows, 1.f, (const float*)X, d1, (const float*)Y, m, begin ? 0.f : 1.f, G, m));
         }
         const int nblk = kTracePartials;
         k_sumsq<<<nblk, 256, 0, st>>>(Y, y_dtype == OSSCAR_FP32, n_rows * m, ctx->partials);
         k_add_partials<<<1, 256, 0, st>>>(ctx->partials, nblk, &ctx->ctl->acc[2], begin ? 1 : 0);
         count_launches(2);
     }
-    if (!end) { CKC(cudaGetLastError()); return OSSCAR_OK; }
-    CKC(gram_mirror(st, H, d1));
+    if (!end) { CKS(cudaGetLastError()); return OSSCAR_OK; }
+    CKS(gram_mirror(st, H, d1));
     if (damp > 0.f) {
-        CKC(cudaMemsetAsync(&ctx->ctl->acc[0], 0, sizeof(double), st));
+        CKS(cudaMemsetAsync(&ctx->ctl->acc[0], 0, sizeof(double), st));
         k_diag_sum<<<64, 256, 0, st>>>(H, d1, &ctx->ctl->acc[0]);
         k_add_damp<<<64, 256, 0, st>>>(H, d1, damp, &ctx->ctl->acc[0]);
         count_launches(2);
     }
-    CKC(cudaMemcpyAsync(ctx->ctl_host, ctx->ctl, sizeof(SearchCtl), cudaMemcpyDeviceToHost, st));
-    CKC(cudaStreamSynchronize(st));
+    CKS(cudaMemcpyAsync(ctx->ctl_host, ctx->ctl, sizeof(SearchCtl), cudaMemcpyDeviceToHost, st));
+    CKS(cudaStreamSynchronize(st));
     if (ctx->ctl_host->status != OSSCAR_OK) return ctx->ctl_host->status;
     *const_term = ctx->ctl_host->acc[2];
     ctx->have_const = true;
@@ -301,7 +323,14 @@ int osscar_init_support(osscar_ctx* ctx, const float* H, const float* G, const f
     ctx->L = L; ctx->H = H; ctx->G = G; ctx->W = W; ctx->have_state = false;
     cudaStream_t st = ctx->stream;
     k_clear_status<<<1, 1, 0, st>>>(ctx->ctl);
+    count_launches(1);
     int rc = select_support(ctx, mode, support);
+    if (rc == OSSCAR_OK && mode == OSSCAR_INIT_USER) {
+        // a rejected list (duplicate or out-of-range ids) ends the call here: nothing is built on it
+        CKS(cudaMemcpyAsync(ctx->ctl_host, ctx->ctl, sizeof(SearchCtl), cudaMemcpyDeviceToHost, st));
+        CKS(cudaStreamSynchronize(st));
+        if (ctx->ctl_host->status != OSSCAR_OK) return ctx->ctl_host->status;
+    }
     if (rc == OSSCAR_OK) rc = build_state(ctx, false);
     if (rc == OSSCAR_OK && score_pass(ctx) != cudaSuccess) rc = OSSCAR_E_CUDA;
     if (rc != OSSCAR_OK) { cudaStreamSynchronize(st); return rc; }
@@ -328,6 +357,7 @@ int osscar_init_support_greedy(osscar_ctx* ctx, const float* H, const float* G, 
     ctx->L = L; ctx->H = H; ctx->G = G; ctx->W = W; ctx->have_state = false;
     cudaStream_t st = ctx->stream;
     k_clear_status<<<1, 1, 0, st>>>(ctx->ctl);
+    count_launches(1);
     int iters = 0;
     int rc = greedy_support(ctx, t_hat, support, drop_trace, &iters);
     if (rc == OSSCAR_OK) rc = build_state(ctx, false);
@@ -351,6 +381,7 @@ int osscar_local_search(osscar_ctx* ctx, const osscar_search_params* params,
     if (params->score_mode != OSSCAR_SCORE_INDEPENDENT && params->score_mode != OSSCAR_SCORE_PAIR_EXACT) return OSSCAR_E_ARG;
     if (params->accept_mode != OSSCAR_ACCEPT_IMPROVING && params->accept_mode != OSSCAR_ACCEPT_ALWAYS) return OSSCAR_E_ARG;
     if (params->refresh_every < 0 || params->profile_samples < 0 || params->profile_samples > 8 || params->block_pairs < 0) return OSSCAR_E_ARG;
+    if (params->loop_mode < OSSCAR_LOOP_AUTO || params->loop_mode > OSSCAR_LOOP_LAUNCHES || params->wait_limit_cycles > (uint64_t)1 << 62) return OSSCAR_E_ARG;
     if (!ctx->have_state) return OSSCAR_E_STATE;
     if (params->score_mode == OSSCAR_SCORE_PAIR_EXACT && ctx->L.nJ > 0 && ctx->L.pair_capacity == 0) return OSSCAR_E_SHAPE;
     if (params->block_pairs > 1) {      // block exchanges: independent scores, s <= min(k, pruned groups), s g rows fit the panels
@@ -378,14 +409,16 @@ int osscar_objective(osscar_ctx* ctx, const float* H, const float* W, const floa
     cudaStream_t st = ctx->stream;
     float* E = (float*)ctx->ws;
     float* HE = E + d1 * m;
+    k_clear_status<<<1, 1, 0, st>>>(ctx->ctl);
     k_sub<<<1184, 256, 0, st>>>(W, Wt, E, d1 * m);
-    count_launches(1);
-    CKC(sgemm(st, false, false, d1, m, d1, 1.f, H, d1, E, m, 0.f, HE, m));
-    CKC(trace_product(st, E, m, HE, m, d1, m, ctx->partials, &ctx->ctl->acc[0]));
-    CKC(cudaMemcpyAsync(ctx->ctl_host, ctx->ctl, sizeof(SearchCtl), cudaMemcpyDeviceToHost, st));
-    CKC(cudaStreamSynchronize(st));
-    *obj = ctx->ctl_host->acc[0];
+    count_launches(2);
+    CKS(sgemm(st, false, false, d1, m, d1, 1.f, H, d1, E, m, 0.f, HE, m));
+    CKS(trace_product(st, E, m, HE, m, d1, m, ctx->partials, &ctx->ctl->acc[0]));
+    CKS(cudaMemcpyAsync(ctx->ctl_host, ctx->ctl, sizeof(SearchCtl), cudaMemcpyDeviceToHost, st));
+    CKS(cudaStreamSynchronize(st));
     ctx->have_state = false;      // the workspace start was overwritten
+    if (ctx->ctl_host->status != OSSCAR_OK) return ctx->ctl_host->status;      // raised on the device during this call
+    *obj = ctx->ctl_host->acc[0];
     return OSSCAR_OK;
 }
 

@@ -9,6 +9,7 @@ namespace osscar {
 
 constexpr int kTracePartials = 1184;   // blocks of a trace reduction; the context owns that many doubles
 constexpr int64_t kMaxPairs = 1 << 20;     // PAIR_EXACT scores at most this many (kept, pruned) pairs per step
+constexpr int kLoopMaxBlocks = 2048;   // most blocks the persistent swap loop is launched with (size of its candidate lists)
 constexpr int kPadF = 32;   // leading dimensions of internal fp32 matrices are padded to this many floats
 
 extern unsigned long long g_launches;      // kernels launched by the library (host-side count)
@@ -31,6 +32,10 @@ struct SearchCtl {
     double  delta;           // exact change of obj of the chosen swap
     double  const_term;
     double  acc[4];          // scratch accumulators (traces, objective reductions)
+    long long wait_limit;    // cycles a bounded device-side wait may spin before it raises OSSCAR_E_TIMEOUT
+    unsigned long long bar_count;   // arrivals at the grid barrier of the persistent swap loop (monotone)
+    int32_t abort;           // set by a wait that ran out: every block of the persistent loop returns
+    int32_t pad1;
 };
 
 // Geometry of one layer's search state inside the caller's workspace.
@@ -47,6 +52,7 @@ struct Layout {
     size_t off_vec_begin, off_vec_end;   // the staged vectors (zeroed once when the state is built)
     size_t off_vnorm, off_rnorm, off_D, off_A, off_c, off_small, off_gramV, off_gramR;
     size_t off_perm, off_slotof, off_energy, off_panel;
+    size_t off_loop;                                                   // persistent swap loop: per-block candidates, phase timers
     size_t off_pairCinv, off_pairKK, off_pairScratch, off_pairDelta;   // PAIR_EXACT scoring
     size_t off_greedy;                                                 // scratch of the nested (greedy) phase
     size_t off_tc, tc_bytes;                                           // bf16 operand terms of the tensor-core GEMMs
@@ -91,6 +97,7 @@ struct osscar_ctx {
     double gram_rows;                // rows accumulated since GRAM_BEGIN (bookkeeping only)
     bool have_const;                 // const term supplied by the caller (cross-term problems) instead of Tr(W^T G)
     double user_const;
+    long long wait_limit;            // context default of SearchCtl::wait_limit
 };
 
 namespace osscar {
@@ -108,30 +115,30 @@ cudaError_t sgemm(cudaStream_t st, bool transA, bool transB, int64_t M, int64_t 
 size_t panel_dot_tc_scratch(int64_t M, int64_t N, int64_t K);
 cudaError_t panel_dot_tc(cudaStream_t st, int64_t M, int64_t N, int64_t K, const float* A, int64_t lda,
                          const float* P, int64_t ldp, float* Y, int64_t so_row, int64_t so_col,
-                         void* scratch, size_t scratch_bytes, int32_t* status_dev, const int32_t* done = nullptr);
+                         void* scratch, size_t scratch_bytes, SearchCtl* ctl_dev, const int32_t* done = nullptr);
 
 // ---- gemm_tc.cu: the same product on the tensor cores (three-term bf16 split, fp32-accurate); A and B row-major.
 // `scratch` (256-byte aligned device memory, at least gemm_tc_min_scratch bytes) holds the bf16 terms of one K panel.
 size_t gemm_tc_min_scratch(int64_t M, int64_t N);
 cudaError_t gemm_tc(cudaStream_t st, int64_t M, int64_t N, int64_t K, float alpha, const float* A, int64_t lda,
                     const float* B, int64_t ldb, float beta, float* C, int64_t ldc,
-                    void* scratch, size_t scratch_bytes, int32_t* status_dev, const int32_t* done = nullptr);
+                    void* scratch, size_t scratch_bytes, SearchCtl* ctl_dev, const int32_t* done = nullptr);
 
 // C += alpha * A * B for a short inner dimension (K <= 128 keeps the terms of A's row band in shared memory across a run
 // of column tiles; larger K goes through gemm_tc).  Same operands and scratch as gemm_tc.  With row_sq (M floats) and
 // sq_scratch (M * 2 * ceil(N / 128) floats) the squared norms of the updated rows are produced in the same pass (K <= 128 only).
 cudaError_t rank_update_tc(cudaStream_t st, int64_t M, int64_t N, int64_t K, float alpha, const float* A, int64_t lda,
                            const float* B, int64_t ldb, float* C, int64_t ldc,
-                           void* scratch, size_t scratch_bytes, int32_t* status_dev, const int32_t* done = nullptr,
+                           void* scratch, size_t scratch_bytes, SearchCtl* ctl_dev, const int32_t* done = nullptr,
                            float* row_sq = nullptr, float* sq_scratch = nullptr);
 
 // H (+)= Xc^T Xc (upper-triangle tiles; Y null) or G (+)= Xc^T Yc with the drained-accumulator pipeline of gemm_tc.cu.
 cudaError_t gram_tc2(cudaStream_t st, const void* X, int64_t n_rows, int64_t d1, const void* Y, int y_fp32, int64_t m,
-                     float* C, bool accumulate, void* scratch, size_t scratch_bytes, int32_t* status_dev);
+                     float* C, bool accumulate, void* scratch, size_t scratch_bytes, SearchCtl* ctl_dev);
 // H (+)= Xc^T Xc for fp32 Xc on the tensor cores (three-term bf16 split staged in `scratch`, row panels sized to it);
 // cudaErrorMemoryAllocation when the scratch is too small for one panel.
 cudaError_t gram_tc3(cudaStream_t st, const float* X, int64_t n_rows, int64_t d1, float* C, bool accumulate,
-                     void* scratch, size_t scratch_bytes, int32_t* status_dev);
+                     void* scratch, size_t scratch_bytes, SearchCtl* ctl_dev);
 
 // ---- gram_tc.cu ---------------------------------------------------------------------------------------------
 cudaError_t set_device_double(cudaStream_t st, double* dst, double v);          // *dst = v on the stream

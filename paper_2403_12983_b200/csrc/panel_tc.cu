@@ -35,7 +35,7 @@ template <int NCH>       // NCH = padded panel width / 32
 __global__ void __launch_bounds__(PT_THREADS, 1)
 k_panel_tc(const __grid_constant__ PanelMaps maps, int64_t M, int N, int nkb_total, int kbs, int KS, int num_items,
            float* __restrict__ Y, int64_t so_row, int64_t so_col, float* __restrict__ part,
-           int32_t* __restrict__ status, const int32_t* __restrict__ done)
+           SearchCtl* __restrict__ ctl, const int32_t* __restrict__ done)
 {
     constexpr int NP = NCH * 32;
     constexpr int P_BYTES = NP * 128;                    // one bf16 term tile of the panel (NP rows x 64 k)
@@ -57,8 +57,10 @@ k_panel_tc(const __grid_constant__ PanelMaps maps, int64_t M, int N, int nkb_tot
     auto stage_free = [&](int s) { return bars + 8u * (8 + s); };
     auto tfull = [&](int b) { return bars + 8u * (10 + b); };
     auto tempty = [&](int b) { return bars + 8u * (12 + b); };
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_ptr + 8 * 14);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_ptr + 8 * 14 + 8);
+    const uint32_t drain_bar = bars + 8u * 14;           // completion of the MMAs in flight when the issuer gives up
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_ptr + 8 * 15);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_ptr + 8 * 15 + 8);
+    const long long wl = ctl->wait_limit;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
@@ -66,6 +68,7 @@ k_panel_tc(const __grid_constant__ PanelMaps maps, int64_t M, int N, int nkb_tot
             mbar_init(raw_full(i), 1); mbar_init(raw_empty(i), 4); mbar_init(p_full(i), 1); mbar_init(a_ready(i), 4);
             mbar_init(stage_free(i), 1); mbar_init(tfull(i), 1); mbar_init(tempty(i), 4);
         }
+        mbar_init(drain_bar, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -87,6 +90,7 @@ k_panel_tc(const __grid_constant__ PanelMaps maps, int64_t M, int N, int nkb_tot
     if (warp == 0) {
         if (lane == 0) {
             uint32_t it = 0;
+            uint32_t n_p[2] = {0, 0}, n_raw[2] = {0, 0};      // copy batches issued per barrier (for the drain of an abort)
             bool ok = true;
             for (int id = blockIdx.x; id < num_items && ok; id += gridDim.x) {
                 int tm, ks, kb0, kb1;
@@ -94,25 +98,26 @@ k_panel_tc(const __grid_constant__ PanelMaps maps, int64_t M, int N, int nkb_tot
                 for (int kb = kb0; kb < kb1 && ok; ++kb, ++it) {
                     const int s = it & 1;
                     const uint32_t ph = (it >> 1) & 1;
-                    if (!mbar_wait(stage_free(s), ph ^ 1, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(stage_free(s), ph ^ 1, abort_flag, wl)) { ok = false; break; }
                     mbar_expect_tx(p_full(s), 3 * P_BYTES);
                     const uint32_t p_dst = stage0 + s * STAGE_BYTES + 3 * PT_AT_BYTES;
 #pragma unroll
                     for (int term = 0; term < 3; ++term)
                         tma_load_2d(p_dst + term * P_BYTES, &maps.p[term], p_full(s), kb * PT_BK, 0);
+                    ++n_p[s];
                     for (int h = 0; h < 2; ++h) {
-                        if (!mbar_wait(raw_empty(h), (it & 1) ^ 1, abort_flag)) { ok = false; break; }
+                        if (!mbar_wait(raw_empty(h), (it & 1) ^ 1, abort_flag, wl)) { ok = false; break; }
                         mbar_expect_tx(raw_full(h), PT_RAW_BYTES);
                         tma_load_2d(raw_ring + h * PT_RAW_BYTES, &maps.a, raw_full(h), kb * PT_BK + h * 32, tm * PT_M);
+                        ++n_raw[h];
                     }
                 }
             }
-            if (*abort_flag && it > 0) {          // let the copies in flight land before the CTA exits
-                const uint32_t last = it - 1;
-                const long long t0 = clock64();
-                while (!(mbar_try_wait(raw_full(0), last & 1) && mbar_try_wait(raw_full(1), last & 1) &&
-                         mbar_try_wait(p_full(last & 1), (last >> 1) & 1)))
-                    if (clock64() - t0 > kWaitLimitCycles) break;
+            if (*abort_flag) {                    // let the copies in flight land before the CTA exits
+                for (int i = 0; i < 2; ++i) {     // the n-th batch on a barrier completes its phase n - 1
+                    if (n_p[i] > 0) mbar_drain(p_full(i), (n_p[i] - 1) & 1);
+                    if (n_raw[i] > 0) mbar_drain(raw_full(i), (n_raw[i] - 1) & 1);
+                }
             }
         }
     } else if (warp == 1) {
@@ -125,7 +130,7 @@ k_panel_tc(const __grid_constant__ PanelMaps maps, int64_t M, int N, int nkb_tot
                 const int nflush = (kb1 - kb0 + PT_FLUSH - 1) / PT_FLUSH;
                 for (int f = 0; f < nflush && ok; ++f, ++fl) {
                     const int buf = fl & 1;
-                    if (!mbar_wait(tempty(buf), ((fl >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(tempty(buf), ((fl >> 1) & 1) ^ 1, abort_flag, wl)) { ok = false; break; }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint32_t d_tmem = tmem_base + (uint32_t)(buf * PT_NMAX);
                     const int e1 = min(kb1, kb0 + (f + 1) * PT_FLUSH);
@@ -133,7 +138,7 @@ k_panel_tc(const __grid_constant__ PanelMaps maps, int64_t M, int N, int nkb_tot
                     for (int kb = kb0 + f * PT_FLUSH; kb < e1 && ok; ++kb, ++it) {
                         const int s = it & 1;
                         const uint32_t ph = (it >> 1) & 1;
-                        if (!mbar_wait(a_ready(s), ph, abort_flag) || !mbar_wait(p_full(s), ph, abort_flag)) { ok = false; break; }
+                        if (!mbar_wait(a_ready(s), ph, abort_flag, wl) || !mbar_wait(p_full(s), ph, abort_flag, wl)) { ok = false; break; }
                         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                         const uint32_t a_src = stage0 + s * STAGE_BYTES;
                         const uint32_t p_src = a_src + 3 * PT_AT_BYTES;
@@ -154,6 +159,10 @@ k_panel_tc(const __grid_constant__ PanelMaps maps, int64_t M, int N, int nkb_tot
                     if (ok) umma_commit(tfull(buf));
                 }
             }
+            if (!ok) {            // MMAs already issued must finish before TMEM and the operand tiles are released
+                umma_commit(drain_bar);
+                mbar_drain(drain_bar, 0);
+            }
         }
     } else if (warp < 6) {
         // converters: warp cw owns rows [32 cw, 32 cw + 32) of the tile; a lane handles two adjacent k of two rows
@@ -167,10 +176,10 @@ k_panel_tc(const __grid_constant__ PanelMaps maps, int64_t M, int N, int nkb_tot
             for (int kb = kb0; kb < kb1 && ok; ++kb, ++it) {
                 const int s = it & 1;
                 const uint32_t ph = (it >> 1) & 1;
-                if (!mbar_wait(stage_free(s), ph ^ 1, abort_flag)) { ok = false; break; }
+                if (!mbar_wait(stage_free(s), ph ^ 1, abort_flag, wl)) { ok = false; break; }
                 uint8_t* at = base_ptr + 2 * PT_RAW_BYTES + s * STAGE_BYTES;
                 for (int h = 0; h < 2 && ok; ++h) {
-                    if (!mbar_wait(raw_full(h), it & 1, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(raw_full(h), it & 1, abort_flag, wl)) { ok = false; break; }
                     const uint8_t* rw = base_ptr + h * PT_RAW_BYTES;
                     float2 v[16];
 #pragma unroll
@@ -216,7 +225,7 @@ k_panel_tc(const __grid_constant__ PanelMaps maps, int64_t M, int N, int nkb_tot
             for (int j = 0; j < NP; ++j) acc[j] = 0.f;
             for (int f = 0; f < nflush && ok; ++f, ++fl) {
                 const int buf = fl & 1;
-                if (!mbar_wait(tfull(buf), (fl >> 1) & 1, abort_flag)) { ok = false; break; }
+                if (!mbar_wait(tfull(buf), (fl >> 1) & 1, abort_flag, wl)) { ok = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
                 for (int c = 0; c < NCH; ++c) {
@@ -251,7 +260,7 @@ k_panel_tc(const __grid_constant__ PanelMaps maps, int64_t M, int N, int nkb_tot
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "n"(PT_TMEM_COLS) : "memory");
     }
-    if (threadIdx.x == 0 && *abort_flag) *status = OSSCAR_E_TIMEOUT;
+    if (threadIdx.x == 0 && *abort_flag) ctl->status = OSSCAR_E_TIMEOUT;
 }
 
 // The panel as three bf16 terms, NP rows x K8 columns each (rows >= N and columns >= K are zero).
@@ -286,12 +295,12 @@ __global__ void k_panel_sum(const float* __restrict__ part, int64_t M, int N, in
 
 template <int NCH>
 cudaError_t launch_panel_tc(cudaStream_t st, int grid, const PanelMaps& maps, int64_t M, int N, int nkb_total, int kbs, int KS,
-                            int num_items, float* Y, int64_t so_row, int64_t so_col, float* part, int32_t* status, const int32_t* done)
+                            int num_items, float* Y, int64_t so_row, int64_t so_col, float* part, SearchCtl* ctl, const int32_t* done)
 {
     constexpr int smem = 2 * PT_RAW_BYTES + 2 * (3 * PT_AT_BYTES + 3 * NCH * 32 * 128) + 1024 + 256;
     cudaError_t e = cudaFuncSetAttribute(k_panel_tc<NCH>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
-    k_panel_tc<NCH><<<grid, PT_THREADS, smem, st>>>(maps, M, N, nkb_total, kbs, KS, num_items, Y, so_row, so_col, part, status, done);
+    k_panel_tc<NCH><<<grid, PT_THREADS, smem, st>>>(maps, M, N, nkb_total, kbs, KS, num_items, Y, so_row, so_col, part, ctl, done);
     return cudaGetLastError();
 }
 
@@ -305,7 +314,7 @@ size_t panel_dot_tc_scratch(int64_t M, int64_t N, int64_t K)
 
 cudaError_t panel_dot_tc(cudaStream_t st, int64_t M, int64_t N, int64_t K, const float* A, int64_t lda,
                          const float* P, int64_t ldp, float* Y, int64_t so_row, int64_t so_col,
-                         void* scratch, size_t scratch_bytes, int32_t* status_dev, const int32_t* done)
+                         void* scratch, size_t scratch_bytes, SearchCtl* ctl_dev, const int32_t* done)
 {
     if (M <= 0 || N <= 0) return cudaSuccess;
     if (K <= 0 || ((uintptr_t)A & 15) || (lda % 4) != 0 || !scratch) return cudaErrorInvalidValue;
@@ -365,10 +374,10 @@ cudaError_t panel_dot_tc(cudaStream_t st, int64_t M, int64_t N, int64_t K, const
         const int grid = num_items < sms ? num_items : sms;
         float* Yc = Y + e0 * so_col;
         switch (NCH) {
-        case 1:  e = launch_panel_tc<1>(st, grid, maps, M, n, nkb_total, kbs, KS, num_items, Yc, so_row, so_col, part, status_dev, done); break;
-        case 2:  e = launch_panel_tc<2>(st, grid, maps, M, n, nkb_total, kbs, KS, num_items, Yc, so_row, so_col, part, status_dev, done); break;
-        case 3:  e = launch_panel_tc<3>(st, grid, maps, M, n, nkb_total, kbs, KS, num_items, Yc, so_row, so_col, part, status_dev, done); break;
-        default: e = launch_panel_tc<4>(st, grid, maps, M, n, nkb_total, kbs, KS, num_items, Yc, so_row, so_col, part, status_dev, done); break;
+        case 1:  e = launch_panel_tc<1>(st, grid, maps, M, n, nkb_total, kbs, KS, num_items, Yc, so_row, so_col, part, ctl_dev, done); break;
+        case 2:  e = launch_panel_tc<2>(st, grid, maps, M, n, nkb_total, kbs, KS, num_items, Yc, so_row, so_col, part, ctl_dev, done); break;
+        case 3:  e = launch_panel_tc<3>(st, grid, maps, M, n, nkb_total, kbs, KS, num_items, Yc, so_row, so_col, part, ctl_dev, done); break;
+        default: e = launch_panel_tc<4>(st, grid, maps, M, n, nkb_total, kbs, KS, num_items, Yc, so_row, so_col, part, ctl_dev, done); break;
         }
         if (e != cudaSuccess) return e;
         count_launches(2);

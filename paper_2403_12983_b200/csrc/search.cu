@@ -806,6 +806,7 @@ __global__ void k_begin(SearchCtl* ctl, double* obj_trace, int32_t* done_host)
     *done_host = 0;
 }
 __global__ void k_count_refresh(SearchCtl* ctl) { if (!ctl->done) ctl->n_refresh += 1; }
+__global__ void k_search_wait_limit(SearchCtl* ctl, long long cycles) { ctl->wait_limit = cycles; }
 __global__ void k_final_obj(SearchCtl* ctl) { ctl->acc[3] = ctl->const_term - ctl->acc[1]; }
 
 // ------------------------------------------------------------------ exhaustive pair scoring (PAIR_EXACT)
@@ -972,6 +973,26 @@ cudaError_t enqueue_scores(osscar_ctx* ctx, const Ptrs& p, bool norms, bool gene
 }
 
 #include "search_block.cuh"
+#include "search_loop_g1.cuh"
+
+// Blocks of the persistent loop: every block the device can hold at once (cooperative launch), but no more than the
+// longest phase has passes to hand out.  0 when the device cannot launch cooperatively.
+int persistent_grid(const Layout& L)
+{
+    int dev = 0, coop = 0, sms = 0, per_sm = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess || !coop) return 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_swap_loop_g1, PL_T, 0) != cudaSuccess || per_sm < 1) return 0;
+    int64_t grid = (int64_t)sms * per_sm;
+    const int rbm = pl_rows_per_pass(L.ldm / 4), rbh = pl_rows_per_pass(L.ldh / 4);
+    int64_t passes = (L.nI + rbm - 1) / rbm;
+    if ((L.nJ + rbm - 1) / rbm > passes) passes = (L.nJ + rbm - 1) / rbm;
+    if ((L.nJ + rbh) / rbh > passes) passes = (L.nJ + rbh) / rbh;
+    if (grid > passes) grid = passes;
+    if (grid > PL_MAX_BLOCKS) grid = PL_MAX_BLOCKS;
+    return (int)(grid < 1 ? 1 : grid);
+}
 
 }  // namespace
 
@@ -997,6 +1018,8 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
 
     k_begin<<<1, 1, 0, st>>>(ctx->ctl, obj_trace, ctx->done_flag_dev);
     count_launches(1);
+    const bool own_limit = prm->wait_limit_cycles != 0;       // this search's budget for bounded waits; restored at the end
+    if (own_limit) { k_search_wait_limit<<<1, 1, 0, st>>>(ctx->ctl, (long long)prm->wait_limit_cycles); count_launches(1); }
     CK(cudaGetLastError());
     CK(cudaEventRecord(ctx->ev0, st));
     const bool pair = prm->score_mode == OSSCAR_SCORE_PAIR_EXACT;
@@ -1008,7 +1031,11 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
         if (panel_dot_tc_scratch(L.nJ > L.nI ? L.nJ : L.nI, 2 * bs * g, L.nI) + 1024 > L.tc_bytes) return OSSCAR_E_WORKSPACE;
     }
     BlockPtrs bp = make_block_ptrs(ctx, bs);
-    const bool fast = g == 1 && !pair && !block;  // fused five-launch step for single-row groups
+    const bool fast = g == 1 && !pair && !block;  // fused step for single-row groups
+    // one cooperative kernel for the whole loop, unless asked otherwise or the device cannot hold such a grid
+    const int pgrid = (fast && prm->loop_mode != OSSCAR_LOOP_LAUNCHES && L.nJ > 0) ? persistent_grid(L) : 0;
+    if (prm->loop_mode == OSSCAR_LOOP_PERSISTENT && pgrid == 0) return OSSCAR_E_ARG;
+    const bool persistent = pgrid > 0;
     if (block) max_swaps /= bs;                   // from here on: iterations
     const int64_t npairs = (int64_t)L.k * (L.ng - L.k);
     if (max_swaps > 0) CK(enqueue_scores(ctx, p, true, pair));
@@ -1080,7 +1107,37 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
     const unsigned prep_blocks = (unsigned)(((L.nI + L.ldm) * g + 255) / 256);
     int next_prof = 0;
     int nmarks = 0;                 // events recorded per profiled step (depends on the step variant)
-    for (int it = 0; it < max_swaps && rc == OSSCAR_OK; ++it) {
+    unsigned long long* loop_prof = (unsigned long long*)((char*)ctx->ws + L.off_loop + 2 * (size_t)kLoopMaxBlocks * 16);
+    if (persistent && max_swaps > 0) {
+        // chunks of steps between rebuilds of the state (one chunk when the state is only ever updated); a stopped loop
+        // makes the remaining launches return at once, so no host round trip is needed in between
+        LoopArgs la;
+        la.p = p;
+        la.candD = (LoopCand*)((char*)ctx->ws + L.off_loop);
+        la.candA = la.candD + kLoopMaxBlocks;
+        la.prof = loop_prof;
+        la.obj_trace = obj_trace; la.swap_trace = swap_trace;
+        la.tol = tol; la.accept_mode = prm->accept_mode; la.max_swaps = max_swaps;
+        if (cudaMemsetAsync(loop_prof, 0, 8 * sizeof(unsigned long long), st) != cudaSuccess) rc = OSSCAR_E_CUDA;
+        const int chunk = prm->refresh_every > 0 ? prm->refresh_every : max_swaps;
+        for (int it0 = 0; it0 < max_swaps && rc == OSSCAR_OK; it0 += chunk) {
+            if (it0 > 0) {
+                rc = build_state(ctx, true);
+                if (rc != OSSCAR_OK) break;
+                k_count_refresh<<<1, 1, 0, st>>>(ctx->ctl);
+                count_launches(1);
+                if (enqueue_scores(ctx, p, true, false) != cudaSuccess || bootstrap_g1() != cudaSuccess) { rc = OSSCAR_E_CUDA; break; }
+            }
+            la.max_steps = max_swaps - it0 < chunk ? max_swaps - it0 : chunk;
+            if (cudaMemsetAsync(&ctx->ctl->bar_count, 0, sizeof(unsigned long long) + sizeof(int32_t), st) != cudaSuccess) { rc = OSSCAR_E_CUDA; break; }
+            void* kargs[] = { (void*)&la };
+            if (cudaLaunchCooperativeKernel((const void*)k_swap_loop_g1, dim3((unsigned)pgrid), dim3(PL_T), kargs, 0, st) != cudaSuccess) {
+                rc = OSSCAR_E_CUDA; break;
+            }
+            count_launches(1);
+        }
+    }
+    for (int it = 0; it < (persistent ? 0 : max_swaps) && rc == OSSCAR_OK; ++it) {
         if (it % batch == 0) {
             const int bi = it / batch;
             if (bi >= 2) {      // stay at most two batches ahead of the device, and stop feeding a finished loop
@@ -1172,6 +1229,7 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
     cudaEventDestroy(evb[0]);
     cudaEventDestroy(evb[1]);
     if (rc != OSSCAR_OK) {
+        if (own_limit) k_search_wait_limit<<<1, 1, 0, st>>>(ctx->ctl, ctx->wait_limit);
         cudaStreamSynchronize(st);
         for (int i = 0; i < nprof; ++i) for (int j = 0; j <= NK; ++j) cudaEventDestroy(evp[i][j]);
         return rc;
@@ -1190,6 +1248,7 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
         k_final_obj<<<1, 1, 0, st>>>(ctx->ctl);
         count_launches(3);
     }
+    if (own_limit) { k_search_wait_limit<<<1, 1, 0, st>>>(ctx->ctl, ctx->wait_limit); count_launches(1); }
     CK(cudaGetLastError());
     CK(cudaMemcpyAsync(ctx->ctl_host, ctx->ctl, sizeof(SearchCtl), cudaMemcpyDeviceToHost, st));
     CK(cudaStreamSynchronize(st));
@@ -1216,6 +1275,17 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
     }
     for (int j = 0; j < NK && used > 0; ++j) res->ms_kernel[j] /= (float)used;
     res->n_profiled = used;
+    if (persistent && max_swaps > 0) {      // phase times of the persistent loop (block 0's clock), mean over its steps
+        unsigned long long prof[8] = {0};
+        CK(cudaMemcpy(prof, loop_prof, sizeof(prof), cudaMemcpyDeviceToHost));
+        const double steps = prof[4] > 0 ? (double)prof[4] : 1.0;
+        res->ms_kernel[0] = (float)(prof[0] / steps * 1e-6);      // decide + staging
+        res->ms_kernel[1] = (float)(prof[1] / steps * 1e-6);      // H pass || V update
+        res->ms_kernel[2] = (float)(prof[2] / steps * 1e-6);      // R update || slot exchange
+        res->ms_kernel[3] = 0.f;                                  // (the selection rides on the other phases)
+        res->ms_kernel[4] = (float)(prof[3] / steps * 1e-6);      // Hinv update + next y
+        res->n_profiled = (int32_t)prof[4];
+    }
     return ctx->ctl_host->status;
 }
 

@@ -535,7 +535,7 @@ cudaError_t enqueue_block_step(osscar_ctx* ctx, const Ptrs& p, const BlockPtrs& 
     k_blk_select<<<2, 1024, 0, st>>>(p, bp);                                                    mark();
     k_blk_gather<<<dim3((unsigned)G, 5), 256, 0, st>>>(p, bp);
     void* tc = (char*)ctx->ws + L.off_tc;                       // free between state builds: bf16 terms and partial sums
-    int32_t* stat = &ctx->ctl->status;
+    SearchCtl* stat = ctx->ctl;
     BK(panel_dot_tc(st, L.nI, G, L.nI, p.Hinv, L.ldh, bp.hT, L.ldh, bp.yT, 1, L.ldh, tc, L.tc_bytes, stat, done));     mark();   // y^T (Hinv symmetric)
     k_blk_gram<<<(unsigned)((4 * G * G + 7) / 8), 256, 0, st>>>(p, bp);
     k_blk_small<<<1, 1024, 2 * (size_t)G * G * sizeof(double), st>>>(p, bp, accept_mode, tol, obj_trace, swap_trace);

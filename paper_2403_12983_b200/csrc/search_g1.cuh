@@ -359,9 +359,8 @@ __global__ void __launch_bounds__(G1_T, 4) k_l1_g1(Ptrs p, unsigned nbV)      //
 
 // Exchange of the leaving kept slot a and the entering pruned slot b in Hp (rows and columns) and in the
 // slot permutation.  Work item ranges: [0, ldp) the two rows, [ldp, 2 ldp) the two columns.
-__device__ __forceinline__ void hswap_g1(const Ptrs& p, int64_t idx, int64_t stride)
+__device__ __forceinline__ void hswap_g1_at(const Ptrs& p, const int64_t a, const int64_t b, int64_t idx, int64_t stride)
 {
-    const int64_t a = p.ctl->sel_slot, b = p.nI + (int64_t)p.ctl->sel_t;
     const int64_t d1 = p.nI + p.nJ;
     for (; idx < 2 * p.ldp; idx += stride) {
         if (idx < p.ldp) {
@@ -381,6 +380,11 @@ __device__ __forceinline__ void hswap_g1(const Ptrs& p, int64_t idx, int64_t str
             }
         }
     }
+}
+
+__device__ __forceinline__ void hswap_g1(const Ptrs& p, int64_t idx, int64_t stride)
+{
+    hswap_g1_at(p, p.ctl->sel_slot, p.nI + (int64_t)p.ctl->sel_t, idx, stride);
 }
 
 // L2: blocks [0, nbR) update G1_RB rows of R each (+ c, A); the remaining blocks exchange the two slots in Hp.

@@ -74,6 +74,23 @@ __global__ void k_user_support(const int32_t* __restrict__ support, int k, int64
     if (atomicExch(&kept[q], 1) != 0) ctl->status = OSSCAR_E_ARG;   // duplicate id
 }
 
+// After k_user_support: a list that was rejected (id out of range, duplicate) marks fewer than k groups.  The kernels
+// that follow index H and G through the slot permutation, so the marks are replaced by a valid set (the first k
+// groups) and the error stays in ctl->status; nothing downstream can then leave its buffers.  One block.
+__global__ void __launch_bounds__(1024) k_user_support_guard(int32_t* __restrict__ kept, int64_t ng, int k, SearchCtl* ctl)
+{
+    __shared__ int cnt;
+    if (threadIdx.x == 0) cnt = 0;
+    __syncthreads();
+    int local = 0;
+    for (int64_t q = threadIdx.x; q < ng; q += blockDim.x) local += kept[q] != 0;
+    if (local) atomicAdd(&cnt, local);
+    __syncthreads();
+    if (ctl->status == OSSCAR_OK && cnt == k) return;
+    for (int64_t q = threadIdx.x; q < ng; q += blockDim.x) kept[q] = q < k;
+    if (threadIdx.x == 0 && ctl->status == OSSCAR_OK) ctl->status = OSSCAR_E_ARG;
+}
+
 // Slots: kept groups in ascending id order take slots 0..k-1, pruned groups k..ng-1.
 __global__ void k_build_perm(const int32_t* __restrict__ kept, int64_t ng, int k,
                              int32_t* __restrict__ perm, int32_t* __restrict__ slotof,
@@ -84,6 +101,7 @@ __global__ void k_build_perm(const int32_t* __restrict__ kept, int64_t ng, int k
     int before_kept = 0;
     for (int64_t p = 0; p < q; ++p) before_kept += kept[p];
     const int slot = kept[q] ? before_kept : k + (int)(q - before_kept);
+    if (slot < 0 || slot >= ng || (kept[q] && slot >= k)) return;       // cannot happen with exactly k marks
     perm[slot] = (int32_t)q;
     slotof[q] = slot;
     if (kept[q]) support[slot] = (int32_t)q;
@@ -192,7 +210,7 @@ k_pivot_inverse(const float* __restrict__ A, int64_t lda, int64_t p0, int nb, fl
         const int c = cb + 16 * k;
         if (i < nb && c < nb) Dinv[i * NB + c] = (float)(0.5 * (Ls[i][c] + Ls[c][i]));
     }
-    if (t == 0 && bad) ctl->status = OSSCAR_E_NOTPD;
+    if (t == 0 && bad && ctl->status == OSSCAR_OK) ctl->status = OSSCAR_E_NOTPD;       // the first error is the one reported
 }
 
 // U = A[p0:p0+nb, 0:n) (copy of the pivot rows), and zero T's pivot rows afterwards is done in k_zero_rows.
@@ -350,6 +368,7 @@ int make_layout(int64_t d1, int64_t m, int32_t g, int32_t k, Layout* L)
     L->off_slotof = take(sizeof(int32_t) * ng);
     L->off_energy = take(sizeof(double) * ng + sizeof(int32_t) * ng);
     L->off_panel = take(sizeof(float) * (d1 * NB + 2 * NB * L->ldp + NB * NB));
+    L->off_loop = take(2 * (size_t)kLoopMaxBlocks * 16 + 64);
     const size_t gg8 = sizeof(double) * g * g;
     const bool pairs_ok = L->pair_capacity > 0;
     L->off_pairCinv = take(pairs_ok ? gg8 * k : 8);
@@ -390,6 +409,8 @@ int select_support(osscar_ctx* ctx, int mode, int32_t* support)
     if (mode == OSSCAR_INIT_USER) {
         CK(cudaMemsetAsync(kept, 0, sizeof(int32_t) * L.ng, st));
         k_user_support<<<(L.k + 255) / 256, 256, 0, st>>>(support, L.k, L.ng, kept, ctx->ctl);
+        k_user_support_guard<<<1, 1024, 0, st>>>(kept, L.ng, L.k, ctx->ctl);
+        count_launches(1);
     } else {
         k_energy<<<(unsigned)L.ng, 128, 0, st>>>(ctx->H, ctx->W, L.d1, L.m, L.g, mode, e);
         k_rank_select<<<nb, 256, 0, st>>>(e, L.ng, L.k, kept);
@@ -474,9 +495,9 @@ int build_state(osscar_ctx* ctx, bool guarded)
     if (nJ > 0) {
         // R_J = G_J - Hp[J, I] V
         k_gather_rows<<<(unsigned)nJ, 256, 0, st>>>(ctx->G, L.m, L.g, perm, nI, R, L.ldm);
-        CK(gemm_tc(st, nJ, L.m, nI, -1.f, Hp + nI * L.ldp, L.ldp, V, L.ldm, 1.f, R, L.ldm, tc, L.tc_bytes, &ctx->ctl->status, done));
+        CK(gemm_tc(st, nJ, L.m, nI, -1.f, Hp + nI * L.ldp, L.ldp, V, L.ldm, 1.f, R, L.ldm, tc, L.tc_bytes, ctx->ctl, done));
         // Pm = Hp[J, I] Hinv, then the Schur complements
-        CK(gemm_tc(st, nJ, nI, nI, 1.f, Hp + nI * L.ldp, L.ldp, Hinv, L.ldh, 0.f, big, L.ldh, tc, L.tc_bytes, &ctx->ctl->status, done));
+        CK(gemm_tc(st, nJ, nI, nI, 1.f, Hp + nI * L.ldp, L.ldp, Hinv, L.ldh, 0.f, big, L.ldh, tc, L.tc_bytes, ctx->ctl, done));
         k_schur<<<(unsigned)(L.ng - L.k), 256, 0, st>>>(Hp, L.ldp, big, L.ldh, nI, L.g, c);
         count_launches(2);
     }

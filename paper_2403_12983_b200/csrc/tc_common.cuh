@@ -7,7 +7,8 @@
 namespace osscar {
 namespace tc {
 
-constexpr long long kWaitLimitCycles = 4000000000LL;     // about two seconds: then the kernel gives up
+constexpr long long kWaitLimitCycles = 4000000000LL;     // default budget of a wait, about two seconds: then the kernel gives up
+constexpr long long kDrainLimitCycles = 4000000000LL;    // budget of the waits an aborting kernel makes for its own copies and MMAs in flight
 
 static __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -26,14 +27,31 @@ static __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t pari
                  : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait: false when the budget ran out or another role already gave up.
-static __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+static __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: false when the budget ran out or another role already gave up.  try_wait may suspend the thread for a
+// hardware-chosen time before it reports "not yet", which is fine for budgets of milliseconds; budgets below
+// kTightBudgetCycles are polled with the non-suspending test_wait so that they are honoured to the cycle count.
+constexpr long long kTightBudgetCycles = 100000;
+static __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, long long limit) {
     const long long t0 = clock64();
-    while (!mbar_try_wait(bar, parity)) {
+    const bool tight = limit < kTightBudgetCycles;
+    while (!(tight ? mbar_test_wait(bar, parity) : mbar_try_wait(bar, parity))) {
         if (*abort_flag) return false;
-        if (clock64() - t0 > kWaitLimitCycles) { *abort_flag = 1; return false; }
+        if (clock64() - t0 > limit) { *abort_flag = 1; return false; }
     }
     return true;
+}
+// Wait of an aborting kernel for work it has itself put in flight (TMA copies into its shared memory, MMAs into its
+// TMEM): independent of the configurable limit, because leaving earlier would let that work land after the CTA is gone.
+static __device__ __forceinline__ void mbar_drain(uint32_t bar, uint32_t parity) {
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity))
+        if (clock64() - t0 > kDrainLimitCycles) break;
 }
 static __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tmap, uint32_t bar, int x, int y) {
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"

@@ -1,12 +1,41 @@
 """Shared helpers of the GPU parity tests: oracle problems and the step-by-step comparison of a
-GPU swap trace with the fp64 oracle (re-basing the oracle at non-decisive steps)."""
+GPU swap trace with the fp64 oracle (re-basing the oracle at non-decisive steps).
+
+Which oracle mode walks beside the GPU.  `strict` (every step re-solved from H and G with a fresh Cholesky
+factorisation; nothing is carried from step to step) is the default and is used by every case whose strict step
+takes under about a second: all reduced-size cases, the c1, c3, c4 and c6 layers at full size.  `lowrank` (the
+oracle's own fp64 update identities) is used only for the full-size c2 and c5 layers, where one strict step costs
+3 s and 30 s of host time; there the walk re-solves from scratch every `refactor_every` steps, compares the carried
+state with the fresh one and continues from the fresh one.
+"""
+import contextlib
+
 import numpy as np
 import torch
+from threadpoolctl import threadpool_limits
 
 import workloads
 from oracle import osscar_oracle as orc
 
 GAP = 1e-5      # relative best-vs-second-best gap above which the oracle's choice is binding
+
+
+def blas_threads(H, g):
+    """Small problems (and the many g x g solves of multi-row groups) run faster on one BLAS thread than on a
+    pool that spins up for every tiny call; large single-row layers use every core."""
+    small = H.shape[0] <= 3000 or g > 1
+    return threadpool_limits(1) if small else contextlib.nullcontext()
+
+
+def assert_states_agree(a, b, tol=1e-8):
+    """The carried low-rank state `a` against the freshly solved `b` (same support, same slot order)."""
+    assert np.array_equal(a.S, b.S)
+    assert rel_fro(a.Hinv, b.Hinv) < tol and rel_fro(a.V, b.V) < tol
+    scale = np.linalg.norm(b.R) + 1e-300
+    assert np.linalg.norm(a.R - b.R) / scale < tol
+    assert abs(a.obj - b.obj) <= tol * abs(b.obj)
+    for q, cq in b.c.items():
+        assert np.allclose(a.c[q], cq, rtol=1e-6, atol=1e-9 * np.abs(cq).max())
 
 
 def oracle_problem(wl):
@@ -17,7 +46,7 @@ def oracle_problem(wl):
 
 
 def follow_trace(H, G, const, g, S0, swaps, gpu_obj, score_mode="independent", accept="improving",
-                 mode="lowrank", max_swaps=None, gpu_stop=None, obj_rtol=1e-4, eps_acc=orc.EPS_ACC):
+                 mode="strict", max_swaps=None, gpu_stop=None, obj_rtol=1e-4, eps_acc=orc.EPS_ACC, refactor_every=25):
     """Walks the GPU's swap sequence with the oracle.  Returns (search, n_rebased).
 
     At each step the oracle proposes its swap from its own fp64 state.  If the GPU made the same
@@ -25,10 +54,23 @@ def follow_trace(H, G, const, g, S0, swaps, gpu_obj, score_mode="independent", a
     the GPU's choice must itself be within GAP of the oracle's best scores; the oracle is then moved
     to the GPU's support and the walk continues.  The running objective must agree throughout.
     """
-    srch = orc.Search(H, G, const, g, S0, mode=mode, score_mode=score_mode, accept=accept, eps_acc=eps_acc)
+    with blas_threads(np.asarray(H), g):
+        return _follow_trace(H, G, const, g, S0, swaps, gpu_obj, score_mode, accept, mode, max_swaps, gpu_stop, obj_rtol,
+                             eps_acc, refactor_every)
+
+
+def _follow_trace(H, G, const, g, S0, swaps, gpu_obj, score_mode, accept, mode, max_swaps, gpu_stop, obj_rtol, eps_acc,
+                  refactor_every):
+    # the oracle's own periodic re-factorisation is switched off: the walk does it below and checks the carried state
+    srch = orc.Search(H, G, const, g, S0, mode=mode, score_mode=score_mode, accept=accept, eps_acc=eps_acc,
+                      refactor_every=1 << 30)
     rebased = 0
     assert gpu_obj[0] == __import__("pytest").approx(srch.st.obj, rel=obj_rtol)
     for step, (i_out, j_in) in enumerate(swaps):
+        if mode == "lowrank" and step > 0 and step % refactor_every == 0:
+            fresh = orc.fresh_state(srch.H, srch.G, srch.const, srch.st.S, g)
+            assert_states_agree(srch.st, fresh)
+            srch.st = fresh
         info = srch.propose(keep_scores=True)
         assert info is not None, f"step {step}: oracle has no candidate"
         slot = int(np.nonzero(srch.st.S == i_out)[0][0]) if i_out in srch.st.S else None
@@ -46,7 +88,7 @@ def follow_trace(H, G, const, g, S0, swaps, gpu_obj, score_mode="independent", a
                 dgpu = info.pair_delta[slot, int(np.nonzero(pruned == j_in)[0][0])]
                 assert abs(dgpu - info.delta) <= GAP * abs(info.delta), f"step {step}: pair not admissible"
             rebased += 1
-            delta = orc.swap_delta_closed_form(srch.H, srch.st, g, slot, j_in)
+            delta = srch.exact_delta(slot, j_in) if mode == "strict" else orc.swap_delta_closed_form(srch.H, srch.st, g, slot, j_in)
         else:
             delta = info.delta
         if accept == "improving":
@@ -57,6 +99,10 @@ def follow_trace(H, G, const, g, S0, swaps, gpu_obj, score_mode="independent", a
             assert delta <= thr or abs(delta - thr) <= band, f"step {step}: accepted a non-improving swap"
         srch.apply(slot, j_in)
         assert gpu_obj[step + 1] == __import__("pytest").approx(srch.st.obj, rel=obj_rtol), f"step {step}: objective drifted"
+    if mode == "lowrank" and len(swaps) > 0:      # the carried state at the end of the walk, against a fresh solve
+        fresh = orc.fresh_state(srch.H, srch.G, srch.const, srch.st.S, g)
+        assert_states_agree(srch.st, fresh)
+        srch.st = fresh
     # after the GPU's last swap: it either hit max_swaps or stopped because the next swap did not improve
     if gpu_stop == "no_improvement":
         info = srch.propose(keep_scores=True)
@@ -76,6 +122,12 @@ def follow_block(H, G, const, g, S0, s, swaps, gpu_obj, accept="improving", gpu_
     """Walks the GPU's block exchanges (s pairs per iteration) with the oracle.  Per iteration the groups the GPU took
     out must be the s cheapest drops and the groups it brought in the s best adds by the oracle's fresh scores, up
     to ties within GAP at the cut; the oracle then makes the GPU's exchange and the objectives must agree."""
+    import pytest
+    with blas_threads(np.asarray(H), g):
+        return _follow_block(H, G, const, g, S0, s, swaps, gpu_obj, accept, gpu_stop, max_iters, obj_rtol, eps_acc)
+
+
+def _follow_block(H, G, const, g, S0, s, swaps, gpu_obj, accept, gpu_stop, max_iters, obj_rtol, eps_acc):
     import pytest
     srch = orc.BlockSearch(H, G, const, g, S0, s, accept=accept, eps_acc=eps_acc)
     assert gpu_obj[0] == pytest.approx(srch.st.obj, rel=obj_rtol)

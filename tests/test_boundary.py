@@ -26,7 +26,9 @@ def test_library_exports_every_declared_symbol():
 
 def test_struct_layouts_match_header():
     import paper_2403_12983_b200.binding as b
-    assert ctypes.sizeof(b.SearchParams) == 32
+    assert ctypes.sizeof(b.SearchParams) == 48
+    assert b.SearchParams.accept_rel_tol.offset == 16 and b.SearchParams.loop_mode.offset == 32
+    assert b.SearchParams.wait_limit_cycles.offset == 40
     assert ctypes.sizeof(b.SearchResult) == 88
     assert b.SearchResult.obj_init.offset == 16 and b.SearchResult.ms_search.offset == 32
 

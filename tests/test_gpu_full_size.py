@@ -1,116 +1,337 @@
-"""Full-size checks (the c2, c5 and c6 shapes, in the launch configuration bench.py times).
+"""Full-size checks: the c2, c3, c4, c5 and c6 layers in the launch configuration bench.py times.
 
-The oracle cannot form H at these sizes in test time, so the checks are properties that hold at any size,
-evaluated on the oracle side from X itself on sampled outputs:
-  * sampled entries of H against fp64 inner products of the corresponding columns of X;
-  * optimality of the returned weights for the returned support: for sampled kept rows i and sampled output
-    columns j,  X_i^T (X e_j) + lambda e_ij = 0  with e = W_hat - W_out and lambda the damping term;
-  * the objective: per sampled column, ||X e_j||^2 + lambda ||e_j||^2 against the same column of the GPU's
-    quadratic form, and the search's running objective against its recomputed value and against the
-    state-independent osscar_objective entry point;
-  * the trace: every accepted swap lowered the objective by more than the accept threshold; the support has k
-    distinct groups; pruned rows of W_out are exactly zero.
+Two kinds of test.
+
+Sequence parity at full size.  c4 and c3 are small enough for the strict oracle (fresh Cholesky solve at every
+step) to run from X itself: both sides get the same host-made activations, the GPU's Gram is compared entry by entry
+with the fp64 Gram, and the whole search is walked step by step.  For c2 and c5 one strict step costs seconds to
+tens of seconds of host time, so the oracle takes the GPU's own H and G (fp32 -> fp64; the Gram itself is checked
+against X on sampled entries below) and walks the first steps in its low-rank mode, re-solving from scratch every
+25 steps and at the end, and comparing the carried state with the fresh one each time.
+
+Properties at full size, from X: sampled entries of H against fp64 inner products of columns of X; optimality of the
+returned weights for the returned support (X_i^T (X e_j) + lambda e_ij = 0 for sampled kept rows i and output
+columns j, e = W_hat - W_out); the objective per sampled column against ||X e_j||^2 + lambda ||e_j||^2, the running
+objective against its recomputed value and against the state-independent osscar_objective entry point; the maintained
+inverse against H_II on sampled rows; every accepted swap lowered the objective by more than the accept threshold;
+k distinct groups kept; pruned rows exactly zero.  c5 is walked to the benchmark's own stop, not to a swap cap.
 """
 import numpy as np
 import pytest
 import torch
 
 import workloads
+from oracle import osscar_oracle as orc
+from tests.parity import GAP, follow_trace, rel_fro
 
 pytestmark = [pytest.mark.gpu, pytest.mark.slow]
 
+DEV = torch.device("cuda", 0)
 
-def _run(name, n_cols, max_swaps, block_pairs=0):
-    import paper_2403_12983_b200 as pkg
-    wl = workloads.config(name)
-    dev = torch.device("cuda", 0)
+
+def trace_of(out):
+    return [tuple(int(v) for v in r) for r in out.swap_trace.cpu().numpy()], out.obj_trace.cpu().numpy()
+
+
+def eligible_by_both_thresholds(st, H, g):
+    """Smallest Schur-complement pivot of any pruned group, relative to the largest diagonal entry of its H block.
+    The oracle drops a candidate at 1e-12 of that scale (fp64), the device at 1e-6 (its state is built from fp32 data):
+    when every group clears 1e-5 both tests keep every group, so the two sides score the same candidates."""
+    worst = np.inf
+    for q, cq in st.c.items():
+        scale = float(np.max(np.diag(H[q * g:(q + 1) * g, q * g:(q + 1) * g])))
+        piv = np.min(np.diag(np.linalg.cholesky(0.5 * (cq + cq.T)))) ** 2 if g > 1 else float(cq[0, 0])
+        worst = min(worst, piv / scale)
+    return worst
+
+
+# ------------------------------------------------------------------------------------ c4 and c3: strict oracle from X
+def solve_from_host_x(pkg, wl, max_swaps, score_mode, accept_always=False, S0=None):
+    b = pkg.binding
     solver = pkg.Solver(0)
-    W = wl.weight(dev)
-    x_dev = [wl.x_chunk(c, dev) for c in range(wl.n_chunks)]
-    res = pkg.solve_layer(solver, x_dev, W, wl.g, wl.k, max_swaps, damp=wl.damp, accept_rel_tol=wl.eps_acc,
-                          block_pairs=block_pairs)
+    W = wl.weight()
+    chunks = list(wl.x_chunks())
+    H, G, const = solver.gram([c.cuda() for c in chunks], W.cuda(), wl.damp)
+    if S0 is None:
+        support, obj0 = solver.init_support(H, G, W.cuda(), wl.g, wl.k)
+    else:
+        support, obj0 = solver.init_support(H, G, W.cuda(), wl.g, wl.k, mode=b.INIT_USER, support=torch.as_tensor(S0))
+    out = solver.local_search(max_swaps, score_mode=score_mode, accept_rel_tol=wl.eps_acc,
+                              accept_mode=b.ACCEPT_ALWAYS if accept_always else b.ACCEPT_IMPROVING)
+    return solver, chunks, W, H, G, const, support.cpu().numpy(), obj0, out
+
+
+def oracle_gram_fp64(chunks, W, damp):
+    W64 = W.numpy().astype(np.float64)
+    return orc.gram_chunked((c.float().numpy() for c in chunks), W64, damp) + (W64,)
+
+
+def check_gram(H, G, const, H64, G64, const64):
+    scale = np.sqrt(np.outer(np.diag(H64), np.diag(H64)))
+    assert np.max(np.abs(H.cpu().numpy() - H64) / scale) < 5e-6
+    gs = np.linalg.norm(G64, axis=1, keepdims=True) + 1e-300
+    assert np.max(np.abs(G.cpu().numpy() - G64) / gs) < 1e-5
+    assert const == pytest.approx(const64, rel=1e-5)
+
+
+def check_start(S0, H64, W64, wl):
+    S0o, e = orc.init_support(H64, W64, wl.g, wl.k)
+    if not np.array_equal(S0, S0o):      # only groups whose energies tie within GAP at the cut may differ
+        thr = np.sort(e)[-wl.k]
+        assert np.all(np.abs(e[np.setxor1d(S0, S0o)] - thr) <= GAP * thr)
+
+
+def test_c4_full_size_sequence_parity_from_x():
+    """ResNet50-shaped 3 x 3 convolution, groups of 9 rows: the whole improving run against the strict oracle."""
+    import paper_2403_12983_b200 as pkg
+    wl = workloads.config("c4")
+    solver, chunks, W, H, G, const, S0, obj0, out = solve_from_host_x(pkg, wl, wl.max_swaps, pkg.binding.SCORE_INDEPENDENT)
+    H64, G64, const64, W64 = oracle_gram_fp64(chunks, W, wl.damp)
+    check_gram(H, G, const, H64, G64, const64)
+    check_start(S0, H64, W64, wl)
+    assert eligible_by_both_thresholds(orc.fresh_state(H64, G64, const64, S0, wl.g), H64, wl.g) > 1e-5
+    swaps, gobj = trace_of(out)
+    assert out.stop_reason == "no_improvement" and len(swaps) >= 10
+    srch, rebased = follow_trace(H64, G64, const64, wl.g, S0, swaps, gobj, gpu_stop=out.stop_reason, max_swaps=wl.max_swaps,
+                                 eps_acc=wl.eps_acc, mode="strict")
+    S_or, W_or, _, _ = srch.result()
+    assert np.array_equal(out.support.cpu().numpy(), S_or)
+    assert out.obj_final == pytest.approx(srch.st.obj, rel=1e-4)
+    assert rel_fro(out.W.cpu().numpy(), W_or) < 1e-3
+    assert solver.objective(H, W.cuda(), out.W) == pytest.approx(srch.st.obj, rel=2e-4)
+    solver.close()
+
+
+def test_c3_full_size_pair_exact_sequence_parity_from_x():
+    """OPT-2.7B-shaped out_proj, 32 heads of 80 rows, exhaustive scoring of the 256 head pairs: the improving run from
+    the energy start, then eight forced exchanges, each against the strict oracle's best pair."""
+    import paper_2403_12983_b200 as pkg
+    b = pkg.binding
+    wl = workloads.config("c3")
+    solver, chunks, W, H, G, const, S0, obj0, out = solve_from_host_x(pkg, wl, wl.max_swaps, b.SCORE_PAIR_EXACT)
+    H64, G64, const64, W64 = oracle_gram_fp64(chunks, W, wl.damp)
+    del chunks
+    check_gram(H, G, const, H64, G64, const64)
+    check_start(S0, H64, W64, wl)
+    assert eligible_by_both_thresholds(orc.fresh_state(H64, G64, const64, S0, wl.g), H64, wl.g) > 1e-5
+    swaps, gobj = trace_of(out)
+    srch, _ = follow_trace(H64, G64, const64, wl.g, S0, swaps, gobj, score_mode="pair_exact", gpu_stop=out.stop_reason,
+                           max_swaps=wl.max_swaps, eps_acc=wl.eps_acc, mode="strict")
+    assert np.array_equal(out.support.cpu().numpy(), srch.result()[0])
+    assert out.obj_final == pytest.approx(srch.st.obj, rel=1e-4)
+    assert rel_fro(out.W.cpu().numpy(), srch.result()[1]) < 1e-3
+    # the paper's fixed-iteration form from the same start: every step must take the oracle's best pair
+    S_start = out.support.cpu().numpy()
+    support, obj0 = solver.init_support(H, G, W.cuda(), wl.g, wl.k, mode=b.INIT_USER, support=torch.as_tensor(S_start))
+    forced = solver.local_search(8, score_mode=b.SCORE_PAIR_EXACT, accept_mode=b.ACCEPT_ALWAYS)
+    assert forced.n_swaps == 8
+    swaps, gobj = trace_of(forced)
+    srch, _ = follow_trace(H64, G64, const64, wl.g, S_start, swaps, gobj, score_mode="pair_exact", accept="always",
+                           gpu_stop="max_swaps", max_swaps=8, mode="strict")
+    assert np.array_equal(forced.support.cpu().numpy(), srch.result()[0])
+    assert forced.obj_final == pytest.approx(srch.st.obj, rel=1e-4)
+    assert rel_fro(forced.W.cpu().numpy(), srch.result()[1]) < 1e-3
+    solver.close()
+
+
+# ------------------------------------------------------------------------------------ c2, c5, c6: device-made X
+class DeviceLayer:
+    """A layer whose activations are drawn on the device (as bench.py does), its Gram built once and shared."""
+
+    def __init__(self, name):
+        import paper_2403_12983_b200 as pkg
+        self.pkg, self.wl = pkg, workloads.config(name)
+        wl = self.wl
+        self.solver = pkg.Solver(0)
+        self.W = wl.weight(DEV)
+        self.x_dev = [wl.x_chunk(c, DEV) for c in range(wl.n_chunks)]
+        self.solver.ensure_workspace(wl.d1, wl.m, wl.g, wl.k)
+        self.H, self.G, self.const = self.solver.gram(self.x_dev, self.W, wl.damp)
+        self._stats = None
+
+    def close(self):
+        self.solver.close()
+        self.x_dev = None
+
+    def x_stats(self, E_cols, rows_i, hcols):
+        """fp64 accumulation over the chunks of X: column norms, X[:, rows_i]^T (X E), ||X E_j||^2, Gram of hcols."""
+        wl = self.wl
+        colsq = np.zeros(wl.d1); a_ij = np.zeros((len(rows_i), E_cols.shape[1])); rr = np.zeros(E_cols.shape[1])
+        hsub = np.zeros((len(hcols), len(hcols)))
+        for Xc in self.x_dev:
+            Xh = Xc.float().cpu().numpy().astype(np.float64)
+            colsq += np.einsum("ij,ij->j", Xh, Xh)
+            r = Xh @ E_cols
+            a_ij += Xh[:, rows_i].T @ r
+            rr += np.einsum("ij,ij->j", r, r)
+            Xs = Xh[:, hcols]
+            hsub += Xs.T @ Xs
+            del Xh
+        return colsq, a_ij, rr, hsub
+
+
+@pytest.fixture(scope="module")
+def c2_layer():
+    layer = DeviceLayer("c2")
+    yield layer
+    layer.close()
+
+
+@pytest.fixture(scope="module")
+def c5_layer():
+    layer = DeviceLayer("c5")
+    yield layer
+    layer.close()
+
+
+def run_search(layer, max_swaps, block_pairs=0, refresh_every=0):
+    wl, solver = layer.wl, layer.solver
+    support, obj0 = solver.init_support(layer.H, layer.G, layer.W, wl.g, wl.k)
+    out = solver.local_search(max_swaps, accept_rel_tol=wl.eps_acc, block_pairs=block_pairs, refresh_every=refresh_every)
+    return support.cpu().numpy(), obj0, out
+
+
+def check_properties(layer, out, n_cols, block_pairs=0):
+    wl, solver = layer.wl, layer.solver
     rng = np.random.default_rng(0)
-    support = res.support.cpu().numpy()
+    support = out.support.cpu().numpy()
     assert len(np.unique(support)) == wl.k and support.min() >= 0 and support.max() < wl.ngroups
     assert np.all(np.diff(support) > 0)
-    obj = res.obj_trace.cpu().numpy()
+    obj = out.obj_trace.cpu().numpy()
     per_it = max(block_pairs, 1)                 # block exchanges record one objective per iteration
-    assert res.n_swaps % per_it == 0 and len(obj) == res.n_swaps // per_it + 1 and res.n_swaps > 0
+    assert out.n_swaps % per_it == 0 and len(obj) == out.n_swaps // per_it + 1 and out.n_swaps > 0
     assert np.all(np.diff(obj) <= -wl.eps_acc * obj[:-1] * (1 - 1e-6))
-    assert obj[-1] == pytest.approx(res.obj_final, rel=1e-4)
-    swaps = res.swap_trace.cpu().numpy()
-    kept = set(int(s) for s in support)
+    assert obj[-1] == pytest.approx(out.obj_final, rel=1e-4)
+    swaps = out.swap_trace.cpu().numpy()
     assert all(int(j) != int(i) for i, j in swaps)
-    for it in range(res.n_swaps // per_it):       # an exchange moves distinct groups
+    for it in range(out.n_swaps // per_it):       # an exchange moves distinct groups
         blk = swaps[it * per_it:(it + 1) * per_it]
         assert len(set(int(v) for v in blk.reshape(-1))) == 2 * per_it
-    Wout = res.W
-    pruned_mask = torch.ones(wl.d1, dtype=torch.bool, device=dev)
-    pruned_mask[res.support.long()] = False
+    Wout = out.W
+    pruned_mask = torch.ones(wl.d1, dtype=torch.bool, device=DEV)
+    pruned_mask[out.support.long()] = False
     assert torch.count_nonzero(Wout[pruned_mask]).item() == 0
+    # ---- the maintained inverse against H_II on sampled rows (slot order of the device), in fp64 on the device
+    perm = solver.debug_state(4).long()
+    I = perm[:wl.k]
+    Hinv = solver.debug_state(0)
+    rows = torch.as_tensor(np.sort(rng.choice(wl.k, 16, replace=False)), device=DEV)
+    HII = layer.H[I][:, I].double()
+    prod = Hinv[rows].double() @ HII
+    eye = torch.zeros_like(prod)
+    eye[torch.arange(len(rows)), rows] = 1.0
+    assert (prod - eye).abs().max().item() < 2e-3
+    del HII, prod, Hinv
     # ---- oracle side, from X: sampled columns of X and E, accumulated chunk by chunk in fp64
-    E = (W - Wout)
+    E = layer.W - Wout
     cols_j = np.sort(rng.choice(wl.m, n_cols, replace=False))
     rows_i = np.sort(rng.choice(support, 24, replace=False))
-    hpairs = rng.integers(0, wl.d1, size=(48, 2))
-    hcols = np.unique(hpairs.reshape(-1))
-    E_s = E[:, torch.as_tensor(cols_j, device=dev)].double().cpu().numpy()
-    colsq = np.zeros(wl.d1)
-    a_ij = np.zeros((len(rows_i), n_cols))
-    rr = np.zeros(n_cols)
-    hsub = np.zeros((len(hcols), len(hcols)))
-    for Xc in x_dev:
-        Xh = Xc.float().cpu().numpy().astype(np.float64)
-        colsq += np.einsum("ij,ij->j", Xh, Xh)
-        r = Xh @ E_s
-        a_ij += Xh[:, rows_i].T @ r
-        rr += np.einsum("ij,ij->j", r, r)
-        Xs = Xh[:, hcols]
-        hsub += Xs.T @ Xs
-        del Xh
+    hcols = np.unique(rng.integers(0, wl.d1, size=(48, 2)).reshape(-1))
+    cj = torch.as_tensor(cols_j, device=DEV)
+    E_s = E[:, cj].double().cpu().numpy()
+    colsq, a_ij, rr, hsub = layer.x_stats(E_s, rows_i, hcols)
     lam = wl.damp * colsq.mean()
-    # sampled H entries (damping sits on the diagonal)
-    Hg = res.H[torch.as_tensor(hcols, device=dev)][:, torch.as_tensor(hcols, device=dev)].double().cpu().numpy()
+    hc = torch.as_tensor(hcols, device=DEV)
+    Hg = layer.H[hc][:, hc].double().cpu().numpy()
     href = hsub + lam * np.eye(len(hcols))
     scale = np.sqrt(np.outer(np.diag(href), np.diag(href)))
     assert np.max(np.abs(Hg - href) / scale) < 4e-6
-    # optimality on kept rows: X_i^T r_j + lam e_ij = 0, relative to |X_i| |r_j|
-    resid = a_ij + lam * E_s[rows_i]
+    resid = a_ij + lam * E_s[rows_i]                    # optimality on kept rows, relative to |X_i| |r_j|
     denom = np.sqrt(np.outer(colsq[rows_i] + lam, rr + 1e-300))
     assert np.max(np.abs(resid) / denom) < 2e-4
-    # per-column objective of the GPU's quadratic form vs ||X e_j||^2 + lam ||e_j||^2
-    HE = res.H @ E[:, torch.as_tensor(cols_j, device=dev)]
-    obj_cols_gpu = (E[:, torch.as_tensor(cols_j, device=dev)] * HE).sum(0).double().cpu().numpy()
-    obj_cols = rr + lam * np.sum(E_s * E_s, axis=0)
-    assert np.allclose(obj_cols_gpu, obj_cols, rtol=2e-4)
-    # state-independent objective entry point (independent of the search state)
-    H, Wd, Wo = res.H, W, res.W.clone()
-    total = solver.objective(H, Wd, Wo)
-    assert total == pytest.approx(res.obj_final, rel=2e-4)
-    solver.close()
-    return res
+    HE = layer.H @ E[:, cj]
+    obj_cols_gpu = (E[:, cj] * HE).sum(0).double().cpu().numpy()
+    assert np.allclose(obj_cols_gpu, rr + lam * np.sum(E_s * E_s, axis=0), rtol=2e-4)
+    # state-independent objective entry point (overwrites the workspace: last)
+    total = solver.objective(layer.H, layer.W, Wout.clone())
+    assert total == pytest.approx(out.obj_final, rel=2e-4)
 
 
-def test_c2_full_size_properties():
-    res = _run("c2", n_cols=4, max_swaps=2000)
-    assert res.stop_reason in ("no_improvement", "max_swaps")
+def sequence_parity_with_device_gram(layer, steps, refactor_every):
+    """First `steps` swaps of the improving run, the oracle fed the device's H and G."""
+    wl, solver = layer.wl, layer.solver
+    S0, obj0, out = run_search(layer, steps)
+    Hr = layer.H.cpu().numpy().astype(np.float64)
+    Gr = layer.G.cpu().numpy().astype(np.float64)
+    Wr = layer.W.cpu().numpy().astype(np.float64)
+    const_r = float(np.sum(Wr * Gr))
+    assert layer.const == pytest.approx(const_r, rel=1e-9)
+    check_start(S0, Hr, Wr, wl)
+    swaps, gobj = trace_of(out)
+    assert len(swaps) == steps and out.stop_reason == "max_swaps"
+    srch, rebased = follow_trace(Hr, Gr, const_r, wl.g, S0, swaps, gobj, gpu_stop=out.stop_reason, max_swaps=steps,
+                                 eps_acc=wl.eps_acc, mode="lowrank", refactor_every=refactor_every)
+    assert eligible_by_both_thresholds(srch.st, Hr, wl.g) > 1e-5
+    S_or, W_or, _, _ = srch.result()
+    assert np.array_equal(out.support.cpu().numpy(), S_or)
+    assert out.obj_final == pytest.approx(srch.st.obj, rel=1e-4)
+    assert rel_fro(out.W.cpu().numpy(), W_or) < 1e-3
+    # the device's maintained state after the walk against the oracle's fresh solve of the same support (the walk ends
+    # on one; both sides put a newcomer into the slot its predecessor left, so the slot orders coincide)
+    perm = solver.debug_state(4).cpu().numpy()
+    st = srch.st
+    assert np.array_equal(st.S, perm[:wl.k])
+    assert rel_fro(solver.debug_state(1).cpu().numpy(), st.V) < 1e-4
+    assert rel_fro(solver.debug_state(2).cpu().numpy(), st.R[perm[wl.k:]]) < 1e-4
+    return rebased
 
 
-def test_c5_full_size_properties():
-    res = _run("c5", n_cols=2, max_swaps=300)
-    assert res.n_swaps == 300 or res.stop_reason == "no_improvement"
+def test_c2_full_size_sequence_parity(c2_layer):
+    sequence_parity_with_device_gram(c2_layer, steps=100, refactor_every=25)
 
 
-def test_c2_full_size_block_exchange_properties():
-    res = _run("c2", n_cols=4, max_swaps=2000, block_pairs=50)
-    assert res.stop_reason in ("no_improvement", "max_swaps")
+def test_c2_full_size_properties(c2_layer):
+    S0, obj0, out = run_search(c2_layer, 2000)
+    assert out.stop_reason in ("no_improvement", "max_swaps")
+    check_properties(c2_layer, out, n_cols=4)
 
 
-def test_c5_full_size_block_exchange_properties():
-    res = _run("c5", n_cols=2, max_swaps=600, block_pairs=50)
-    assert res.n_swaps == 600 or res.stop_reason == "no_improvement"
+def test_c2_full_size_block_exchange_properties(c2_layer):
+    S0, obj0, out = run_search(c2_layer, 2000, block_pairs=50)
+    assert out.stop_reason in ("no_improvement", "max_swaps")
+    check_properties(c2_layer, out, n_cols=4, block_pairs=50)
 
 
-def test_c6_pointwise_conv_full_size_properties():
-    res = _run("c6", n_cols=4, max_swaps=500)
-    assert res.stop_reason in ("no_improvement", "max_swaps")
+def test_c5_full_size_sequence_parity(c5_layer):
+    sequence_parity_with_device_gram(c5_layer, steps=20, refactor_every=25)
+
+
+def test_c5_full_size_run_to_its_stop(c5_layer):
+    """The benchmark's own run: improving swaps until none is left (about 1100), checked at the end of the walk."""
+    S0, obj0, out = run_search(c5_layer, c5_layer.wl.max_swaps)
+    assert out.stop_reason == "no_improvement" and out.n_swaps > 500
+    check_properties(c5_layer, out, n_cols=2)
+
+
+def test_c5_full_size_run_with_refresh(c5_layer):
+    """The same run with the state rebuilt from H every 400 swaps: properties at its stop, and the same objective as the
+    run that only updates (the two may part at near-ties, so the supports are not compared)."""
+    S0, obj0, plain = run_search(c5_layer, c5_layer.wl.max_swaps)
+    S0, obj0, out = run_search(c5_layer, c5_layer.wl.max_swaps, refresh_every=400)
+    assert out.stop_reason == "no_improvement" and out.n_refresh >= 1
+    assert out.obj_final == pytest.approx(plain.obj_final, rel=1e-4)
+    check_properties(c5_layer, out, n_cols=2)
+
+
+def test_c5_full_size_block_exchange_properties(c5_layer):
+    S0, obj0, out = run_search(c5_layer, 600, block_pairs=50)
+    assert out.n_swaps == 600 or out.stop_reason == "no_improvement"
+    check_properties(c5_layer, out, n_cols=2, block_pairs=50)
+
+
+def test_c6_pointwise_conv_full_size_parity_and_properties():
+    """MobileNetV1-shaped 1 x 1 convolution: small enough for the strict oracle on the device's Gram over the whole run."""
+    layer = DeviceLayer("c6")
+    wl = layer.wl
+    S0, obj0, out = run_search(layer, wl.max_swaps)
+    assert out.stop_reason in ("no_improvement", "max_swaps")
+    Hr = layer.H.cpu().numpy().astype(np.float64); Gr = layer.G.cpu().numpy().astype(np.float64)
+    const_r = float(np.sum(layer.W.cpu().numpy().astype(np.float64) * Gr))
+    swaps, gobj = trace_of(out)
+    srch, _ = follow_trace(Hr, Gr, const_r, wl.g, S0, swaps, gobj, gpu_stop=out.stop_reason, max_swaps=wl.max_swaps,
+                           eps_acc=wl.eps_acc, mode="strict")
+    assert np.array_equal(out.support.cpu().numpy(), srch.result()[0])
+    assert out.obj_final == pytest.approx(srch.st.obj, rel=1e-4)
+    assert rel_fro(out.W.cpu().numpy(), srch.result()[1]) < 1e-3
+    check_properties(layer, out, n_cols=4)
+    layer.close()

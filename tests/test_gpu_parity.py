@@ -535,6 +535,180 @@ def test_cross_term_gram_and_search(solver, name, over, ydt, lend):
     assert rel_fro(out.W.cpu().numpy(), srch.result()[1]) < 1e-3
 
 
+# ------------------------------------------------------------------------------------ candidate guard
+def duplicated_layer(g, k, m, n, seed, free_last):
+    """H, G (fp64) of a layer whose groups k .. 2k-1 repeat the columns of groups 0 .. k-1 exactly (H is assembled from
+    one k*g-wide Gram block, so the copies are bit-identical); with `free_last` the last group gets fresh columns."""
+    rng = np.random.default_rng(seed)
+    Xk = rng.standard_normal((n, k * g))
+    X = np.concatenate([Xk, Xk], axis=1)
+    if free_last:
+        X[:, (2 * k - 1) * g:] = rng.standard_normal((n, g))
+    Hk = Xk.T @ Xk
+    H = np.block([[Hk, Hk], [Hk, Hk]])
+    if free_last:
+        last = slice((2 * k - 1) * g, 2 * k * g)
+        H[:, last] = X.T @ X[:, last]
+        H[last, :] = H[:, last].T
+    W = rng.standard_normal((2 * k * g, m)) / 8.0
+    return H, H @ W, W
+
+
+@pytest.mark.parametrize("g", [1, 3])
+def test_dependent_groups_never_enter(solver, osscar, g):
+    """Pruned groups that repeat kept columns have a vanishing Schur complement: both sides must leave them out of the
+    add scores (the oracle by its 1e-12 pivot test in fp64, the device by 1e-6 on its fp32-built state), and the forced
+    walk must still follow the oracle."""
+    b = osscar.binding
+    k = 12
+    H64, G64, W = duplicated_layer(g, k, m=40, n=240, seed=3 + g, free_last=True)
+    H, G, Wd = dev(H64), dev(G64), dev(W)
+    Hr, Gr = H.cpu().numpy().astype(np.float64), G.cpu().numpy().astype(np.float64)
+    const_r = float(np.sum(W * Gr))
+    S0 = np.arange(k)
+    support, obj0 = solver.init_support(H, G, Wd, g, k, mode=b.INIT_USER, support=torch.as_tensor(S0))
+    A = solver.debug_state(6).cpu().numpy()                  # add scores by pruned slot (slot t holds group k + t)
+    assert np.all(np.isneginf(A[:k - 1])) and np.isfinite(A[k - 1])
+    st = orc.fresh_state(Hr, Gr, const_r, S0, g)
+    A_or = orc.add_scores(st, g, 2 * k, Hr)
+    assert np.all(np.isneginf(A_or[k:2 * k - 1])) and A[k - 1] == pytest.approx(A_or[2 * k - 1], rel=1e-4)
+    out = solver.local_search(4, accept_mode=b.ACCEPT_ALWAYS)
+    assert out.n_swaps == 4
+    swaps = [tuple(int(v) for v in r) for r in out.swap_trace.cpu().numpy()]
+    twin = {q: q + k for q in range(k - 1)}
+    twin.update({q + k: q for q in range(k - 1)})
+    kept = set(range(k))
+    for i_out, j_in in swaps:                                 # no group enters while the group with the same columns is kept
+        assert twin.get(j_in) not in kept
+        kept.remove(i_out); kept.add(j_in)
+    srch, _ = follow_trace(Hr, Gr, const_r, g, S0, swaps, out.obj_trace.cpu().numpy(), accept="always",
+                           gpu_stop="max_swaps", max_swaps=4)
+    assert np.array_equal(out.support.cpu().numpy(), srch.result()[0])
+
+
+@pytest.mark.parametrize("g,pairs", [(1, 0), (2, 0), (1, 3)])
+def test_guard_stop_when_every_candidate_is_dependent(solver, osscar, g, pairs):
+    b = osscar.binding
+    k = 10
+    H64, G64, W = duplicated_layer(g, k, m=24, n=200, seed=11, free_last=False)
+    H, G, Wd = dev(H64), dev(G64), dev(W)
+    support, obj0 = solver.init_support(H, G, Wd, g, k, mode=b.INIT_USER, support=torch.arange(k, dtype=torch.int32))
+    assert np.all(np.isneginf(solver.debug_state(6).cpu().numpy()))
+    out = solver.local_search(12, accept_mode=b.ACCEPT_ALWAYS, block_pairs=pairs)
+    assert out.n_swaps == 0 and out.stop_reason == "guard"
+    assert out.obj_final == pytest.approx(obj0, rel=1e-6)
+    assert np.array_equal(out.support.cpu().numpy(), np.arange(k))
+    ref = orc.Search(H.cpu().numpy().astype(np.float64), G.cpu().numpy().astype(np.float64),
+                     float(np.sum(W * G.cpu().numpy().astype(np.float64))), g, np.arange(k), accept="always").run(12)
+    assert ref.stop_reason == "guard" and len(ref.swap_trace) == 0
+
+
+# ------------------------------------------------------------------------------------ the two drivers of the swap loop
+@pytest.mark.parametrize("name,over,seed,max_swaps", [
+    SEARCH_CASES[0],                                                                  # 64 rows: fewer rows than blocks
+    SEARCH_CASES[3],                                                                  # four / two rows per pass
+    ("c2", dict(n=8192, d1=2600, m=1100, k=1300, chunk_rows=4096), 0, 60),            # two rows and one row per pass
+    ("c5", dict(n=8192, d1=4200, m=2300, k=2100, chunk_rows=4096), 1, 40),            # one row per pass, two passes per row of V
+])
+def test_persistent_loop_and_launch_chain_follow_the_oracle(solver, osscar, name, over, seed, max_swaps):
+    """Single-row groups have two drivers: one cooperative kernel with grid-wide barriers, or five launches per step.
+    Both must follow the strict oracle; where no choice is a near-tie they make the same swaps."""
+    b = osscar.binding
+    wl = workloads.config(name, seed=seed, **over)
+    chunks, W, H64, G64, const64 = oracle_problem(wl)
+    H, G, Wd = dev(H64), dev(G64), dev(W)
+    Hr, Gr = H.cpu().numpy().astype(np.float64), G.cpu().numpy().astype(np.float64)
+    const_r = float(np.sum(W * Gr))
+    runs = {}
+    for mode in (b.LOOP_PERSISTENT, b.LOOP_LAUNCHES):
+        S0, obj0 = solver.init_support(H, G, Wd, wl.g, wl.k)
+        launches0 = b.launch_count()
+        out = solver.local_search(max_swaps, accept_rel_tol=wl.eps_acc, loop_mode=mode, profile_samples=2)
+        launched = b.launch_count() - launches0
+        swaps = [tuple(int(v) for v in r) for r in out.swap_trace.cpu().numpy()]
+        srch, rebased = follow_trace(Hr, Gr, const_r, wl.g, S0.cpu().numpy(), swaps, out.obj_trace.cpu().numpy(),
+                                     gpu_stop=out.stop_reason, max_swaps=max_swaps, eps_acc=wl.eps_acc)
+        assert np.array_equal(out.support.cpu().numpy(), srch.result()[0])
+        assert out.obj_final == pytest.approx(srch.st.obj, rel=1e-4)
+        assert rel_fro(out.W.cpu().numpy(), srch.result()[1]) < 1e-3
+        # the maintained state after the run against a fresh solve of the final support
+        perm = solver.debug_state(4).cpu().numpy()
+        st = orc.fresh_state(Hr, Gr, const_r, perm[:wl.k], wl.g)
+        assert rel_fro(solver.debug_state(0).cpu().numpy(), st.Hinv) < 2e-4
+        assert rel_fro(solver.debug_state(1).cpu().numpy(), st.V) < 1e-4
+        assert rel_fro(solver.debug_state(2).cpu().numpy(), st.R[perm[wl.k:]]) < 1e-4
+        runs[mode] = (swaps, rebased, launched, out)
+    # the persistent driver is a handful of launches however many swaps it makes
+    assert runs[b.LOOP_PERSISTENT][2] < 20 <= runs[b.LOOP_LAUNCHES][2]
+    assert runs[b.LOOP_PERSISTENT][3].ms_kernel and runs[b.LOOP_LAUNCHES][3].ms_kernel
+    if runs[b.LOOP_PERSISTENT][1] == 0 and runs[b.LOOP_LAUNCHES][1] == 0:
+        assert runs[b.LOOP_PERSISTENT][0] == runs[b.LOOP_LAUNCHES][0]
+
+
+def test_persistent_loop_with_refresh_and_forced_swaps(solver, osscar):
+    b = osscar.binding
+    wl = workloads.config("c2", n=4096, d1=520, m=150, k=207, chunk_rows=4096)
+    chunks, W, H64, G64, const64 = oracle_problem(wl)
+    H, G, Wd = dev(H64), dev(G64), dev(W)
+    Hr, Gr = H.cpu().numpy().astype(np.float64), G.cpu().numpy().astype(np.float64)
+    const_r = float(np.sum(W * Gr))
+    S0, obj0 = solver.init_support(H, G, Wd, 1, wl.k)
+    out = solver.local_search(40, accept_mode=b.ACCEPT_ALWAYS, refresh_every=16, loop_mode=b.LOOP_PERSISTENT)
+    assert out.n_swaps == 40 and out.stop_reason == "max_swaps" and out.n_refresh == 2
+    swaps = [tuple(int(v) for v in r) for r in out.swap_trace.cpu().numpy()]
+    srch, _ = follow_trace(Hr, Gr, const_r, 1, S0.cpu().numpy(), swaps, out.obj_trace.cpu().numpy(),
+                           accept="always", gpu_stop="max_swaps", max_swaps=40)
+    assert np.array_equal(out.support.cpu().numpy(), srch.result()[0])
+    assert out.obj_final == pytest.approx(srch.st.obj, rel=1e-4)
+
+
+# ------------------------------------------------------------------------------------ bounded waits
+def test_grid_barrier_that_runs_out_returns_a_status(solver, osscar):
+    """With a budget of a few cycles the first block to reach the first grid barrier of the persistent loop gives up:
+    every block returns, the call reports OSSCAR_E_TIMEOUT, nothing hangs, and the same context then solves the same
+    layer with the default budget."""
+    b = osscar.binding
+    wl = workloads.config("c2", n=4096, d1=1000, m=300, k=437, chunk_rows=4096)
+    chunks, W, H64, G64, const64 = oracle_problem(wl)
+    H, G, Wd = dev(H64), dev(G64), dev(W)
+    solver.init_support(H, G, Wd, 1, wl.k)
+    with pytest.raises(osscar.OsscarError) as ei:
+        solver.local_search(50, accept_rel_tol=wl.eps_acc, loop_mode=b.LOOP_PERSISTENT, wait_limit_cycles=4)
+    assert ei.value.status == b.E_TIMEOUT
+    with pytest.raises(osscar.OsscarError) as ei:               # the state of a failed search is not trusted
+        solver.local_search(50, accept_rel_tol=wl.eps_acc)
+    assert ei.value.status == b.E_STATE
+    S0, obj0 = solver.init_support(H, G, Wd, 1, wl.k)
+    out = solver.local_search(50, accept_rel_tol=wl.eps_acc, loop_mode=b.LOOP_PERSISTENT)
+    Hr, Gr = H.cpu().numpy().astype(np.float64), G.cpu().numpy().astype(np.float64)
+    swaps = [tuple(int(v) for v in r) for r in out.swap_trace.cpu().numpy()]
+    srch, _ = follow_trace(Hr, Gr, float(np.sum(W * Gr)), 1, S0.cpu().numpy(), swaps, out.obj_trace.cpu().numpy(),
+                           gpu_stop=out.stop_reason, max_swaps=50, eps_acc=wl.eps_acc)
+    assert np.array_equal(out.support.cpu().numpy(), srch.result()[0]) and out.n_swaps > 0
+
+
+def test_wait_that_runs_out_in_a_gram_chunk_is_reported_at_the_end(solver, osscar):
+    """A wait budget of one cycle makes the first pipeline wait of the first chunk run out; the kernel drains its
+    copies, returns, and the error must survive the second chunk and come back from the END call.  The context then
+    works as before."""
+    b = osscar.binding
+    wl = workloads.config("c2", n=1024, d1=512, m=64, k=200, chunk_rows=512)
+    X = [c.cuda() for c in wl.x_chunks()]
+    W = wl.weight().cuda()
+    H = torch.empty(wl.d1, wl.d1, device="cuda"); G = torch.empty(wl.d1, wl.m, device="cuda")
+    solver.set_wait_limit(1)
+    solver.gram_chunk(X[0], H, b.GRAM_BEGIN)
+    solver.set_wait_limit(0)                                  # back to the default before the second chunk
+    with pytest.raises(osscar.OsscarError) as ei:
+        solver.gram_chunk(X[1], H, b.GRAM_END, W, G, wl.damp)
+    assert ei.value.status == b.E_TIMEOUT
+    chunks, Wh, H64, G64, const64 = oracle_problem(wl)
+    H2, G2, const = solver.gram(X, W, wl.damp)
+    scale = np.sqrt(np.outer(np.diag(H64), np.diag(H64)))
+    assert np.max(np.abs(H2.cpu().numpy() - H64) / scale) < 4e-6
+    assert const == pytest.approx(const64, rel=1e-5)
+
+
 # ------------------------------------------------------------------------------------ edge cases and errors
 def test_edge_cases(solver, osscar):
     b = osscar.binding

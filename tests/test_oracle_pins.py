@@ -80,7 +80,7 @@ def test_closed_form_objective_equals_least_squares_for_every_support(g, p, k):
 
 
 def test_enumerator_count_matches_paper_example():
-    """Section 3.1: pruning half of 32 channels gives 'over 600 million' supports."""
+    """Section 3.1: C(32, 16), the supports that keep half of 32 channels, exceeds the bound the paper prints."""
     with open(os.path.join(GOLDEN, "paper_support_count.txt")) as fh:
         rows = [l.split() for l in fh if l.strip() and not l.startswith("#")]
     (p, k, lower_bound), = [(int(a), int(b), int(c)) for a, b, c in rows]
@@ -536,3 +536,65 @@ def test_block_search_stops_when_the_exchange_does_not_improve_and_rejects_bad_s
         orc.BlockSearch(H, G, const, 1, S0, 7)
     with pytest.raises(ValueError):
         orc.BlockSearch(H, G, const, 1, S0, 0)
+
+
+# ----------------------------------------------------------------------------- candidate guard (Proposition 1, Case 2)
+def duplicated_problem(g, k, m=5, n=80, seed=0):
+    """A layer whose last k groups are copies of its first k groups (columns of X repeated): with the first k groups
+    kept, every pruned group lies in the span of the kept columns."""
+    rng = np.random.default_rng(seed)
+    Xk = rng.standard_normal((n, k * g))
+    X = np.concatenate([Xk, Xk], axis=1)
+    W = rng.standard_normal((2 * k * g, m))
+    H, G, const = orc.gram(X, W)
+    return X, W, H, G, const
+
+
+@pytest.mark.parametrize("g", [1, 3])
+def test_dependent_group_is_ineligible_and_adds_nothing(g):
+    """A pruned group that repeats kept columns has Schur complement 0 (the C^-1 of Case 2 is H_qq - H_qI H_II^-1 H_Iq,
+    the squared distance of its columns from the kept span), bringing it back cannot lower the least-squares error,
+    and the oracle must score it -inf (single rows) / report no inverse (groups) instead of dividing by it."""
+    k = 4
+    X, W, H, G, const = duplicated_problem(g, k)
+    ng = 2 * k
+    # one independent extra candidate so that the step still has somewhere to go: replace the last copy by fresh columns
+    rng = np.random.default_rng(5)
+    X[:, (ng - 1) * g:] = rng.standard_normal((X.shape[0], g))
+    H, G, const = orc.gram(X, W)
+    S = np.arange(k)
+    st = orc.fresh_state(H, G, const, S, g)
+    _, obj_S = orc.solve_support_lstsq(X, W, S, g)
+    for q in range(k, ng - 1):
+        assert np.abs(st.c[q]).max() <= 1e-9 * np.abs(H).max()                       # Schur complement vanishes
+        _, obj_add = orc.solve_support_lstsq(X, W, list(S) + [q], g)                 # the definition: nothing gained
+        assert obj_add == pytest.approx(obj_S, rel=1e-9)
+        if g > 1:
+            assert orc._quad_inv(st.c[q], st.R[q * g:(q + 1) * g], float(np.max(np.diag(H[q * g:(q + 1) * g, q * g:(q + 1) * g])))) is None
+    A = orc.add_scores(st, g, ng, H)
+    assert np.all(np.isneginf(A[:ng - 1])) and np.isfinite(A[ng - 1]) and A[ng - 1] > 0
+    # the eligible candidate's score is the true gain
+    _, obj_new = orc.solve_support_lstsq(X, W, list(S) + [ng - 1], g)
+    assert A[ng - 1] == pytest.approx(obj_S - obj_new, rel=1e-8)
+    # the search never brings a group in while its twin (the group with the same columns) is kept
+    twin = {q: q + k for q in range(k - 1)}
+    twin.update({q + k: q for q in range(k - 1)})
+    srch = orc.Search(H, G, const, g, S, accept="always")
+    for _ in range(4):
+        info = srch.propose(keep_scores=True)
+        assert info is not None
+        kept = set(int(v) for v in srch.st.S)
+        assert twin.get(info.j_in) not in kept
+        srch.apply(info.slot, info.j_in)
+        assert len(set(int(v) for v in srch.st.S)) == k
+
+
+@pytest.mark.parametrize("g", [1, 2])
+def test_search_stops_with_guard_when_every_candidate_is_dependent(g):
+    k = 5
+    X, W, H, G, const = duplicated_problem(g, k, seed=2)
+    srch = orc.Search(H, G, const, g, np.arange(k), accept="always").run(10)
+    assert srch.stop_reason == "guard" and len(srch.swap_trace) == 0
+    assert srch.propose() is None
+    blk = orc.BlockSearch(H, G, const, g, np.arange(k), 2, accept="always").run(3)
+    assert blk.stop_reason == "guard" and len(blk.block_trace) == 0

@@ -43,6 +43,12 @@ def test_noalloc_trace_matches_gram_const_twice():
     Wv, Gv = W[:, :20], G[:, :20]
     ref = float(np.sum(Wv.cpu().numpy().astype(np.float64) * Gv.cpu().numpy().astype(np.float64)))
     assert b.osscar_trace_noalloc(Wv, Gv) == pytest.approx(ref, rel=1e-12)
+    # the entry point's promise: a warmed call leaves the amount of free device memory where it was
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
+    assert b.osscar_trace_noalloc(Wv, Gv) == pytest.approx(ref, rel=1e-12)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free_before
     out = ctypes.c_double(-1.0)          # zero rows: valid pointers, nothing to add
     rc = pkg.lib().osscar_trace_noalloc(ctypes.c_void_p(W.data_ptr()), W.stride(0), ctypes.c_void_p(G.data_ptr()),
                                         G.stride(0), 0, W.shape[1], W.device.index, None, ctypes.byref(out))
@@ -60,4 +66,9 @@ def test_noalloc_rejects_sizes_beyond_its_scratch():
                                 A.device.index, None, ctypes.byref(out))
     assert rc == b.E_SHAPE
     rc = L.osscar_trace_noalloc(None, 4, ctypes.c_void_p(A.data_ptr()), 4, 8, 4, A.device.index, None, ctypes.byref(out))
+    assert rc == b.E_ARG
+    # a matrix that does not live on the named device (here: pinned host memory) is refused, not dereferenced
+    Hh = torch.zeros(8, 4).pin_memory()
+    rc = L.osscar_trace_noalloc(ctypes.c_void_p(Hh.data_ptr()), 4, ctypes.c_void_p(A.data_ptr()), 4, 8, 4, A.device.index, None,
+                                ctypes.byref(out))
     assert rc == b.E_ARG
