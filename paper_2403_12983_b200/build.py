@@ -9,7 +9,7 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libosscar.so")
-SOURCES = ["osscar_api.cu", "sgemm.cu", "gram_tc.cu", "gemm_tc.cu", "state.cu", "search.cu", "greedy.cu", "panel_tc.cu", "noalloc.cu"]
+SOURCES = ["osscar_api.cu", "sgemm.cu", "gram_tc.cu", "gemm_tc.cu", "state.cu", "search.cu", "greedy.cu", "panel_tc.cu", "noalloc.cu", "dgemm.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 

@@ -109,6 +109,12 @@ cudaError_t sgemm(cudaStream_t st, bool transA, bool transB, int64_t M, int64_t 
                   float alpha, const float* A, int64_t lda, const float* B, int64_t ldb,
                   float beta, float* C, int64_t ldc, const int32_t* done = nullptr);
 
+// ---- dgemm.cu: C = beta * C0 + alpha * A * B (or I + alpha * A * B) with fp32 operands, products and sums in fp64;
+// A (M x K) and B (K x N) row-major, C0 may alias C.
+cudaError_t gemm_f64acc(cudaStream_t st, int64_t M, int64_t N, int64_t K, double alpha, const float* A, int64_t lda,
+                        const float* B, int64_t ldb, double beta, const float* C0, int64_t ldc0, float* C, int64_t ldc,
+                        bool identity_plus, const int32_t* done = nullptr);
+
 // ---- panel_tc.cu: Y[i*so_row + e*so_col] = sum_k A[i][k] * P[e][k] on the tensor cores; A (M x K, streamed once) is split
 // into bf16 terms on the way (fp32-accurate); P is an N x K panel
 // A 16-byte aligned with lda % 4 == 0; scratch at least panel_dot_tc_scratch bytes.

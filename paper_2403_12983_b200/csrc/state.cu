@@ -283,6 +283,23 @@ __global__ void k_sum_partials(const double* __restrict__ partial, int n, double
     if (threadIdx.x == 0) *out = acc;
 }
 
+// A := sym(A + D) on the n x n leading block: the blocked inversion leaves its two triangles different in the last bits
+// times cond, and the correction of that difference is the antisymmetric part of D, so both are symmetrised together.
+// A thread owns the pair (r, c), (c, r) with c >= r; tiles below the diagonal have nothing to do.
+__global__ void k_add_sym(float* __restrict__ A, int64_t lda, const float* __restrict__ D, int64_t ldd, int64_t n,
+                          const int32_t* __restrict__ done)
+{
+    if (done && *done) return;
+    if (blockIdx.x < blockIdx.y) return;
+    const int64_t c = (int64_t)blockIdx.x * 32 + threadIdx.x;
+    for (int64_t r = (int64_t)blockIdx.y * 32 + threadIdx.y; r < (int64_t)blockIdx.y * 32 + 32 && r < n; r += 8) {
+        if (c >= n || c < r) continue;
+        const float v = 0.5f * ((A[r * lda + c] + A[c * lda + r]) + (D[r * ldd + c] + D[c * ldd + r]));
+        A[r * lda + c] = v;
+        A[c * lda + r] = v;
+    }
+}
+
 __global__ void k_set_obj(SearchCtl* ctl)   // obj = const - Tr(G_I^T V), with acc[0] = const, acc[1] = trace
 {
     ctl->const_term = ctl->acc[0];
@@ -333,6 +350,7 @@ int make_layout(int64_t d1, int64_t m, int32_t g, int32_t k, Layout* L)
     int64_t big = nI * ldm;
     if (nJ * ldh > big) big = nJ * ldh;
     if (2 * d1 * ldm > big) big = 2 * d1 * ldm;
+    if (2 * nI * ldh > big) big = 2 * nI * ldh;             // residual and correction of the refinement step on Hinv
     const int64_t npairs = (int64_t)k * (ng - k);
     L->pair_capacity = npairs <= kMaxPairs ? npairs : 0;
     if (L->pair_capacity > 0 && nJ * ldh + nI * round_up(nJ, kPadF) > big) big = nJ * ldh + nI * round_up(nJ, kPadF);
@@ -480,24 +498,36 @@ int build_state(osscar_ctx* ctx, bool guarded)
     count_launches(2);
     CK(cudaGetLastError());
     { const int rc_inv = invert_spd_inplace(ctx, Hinv, L.ldh, nI, Hp, L.ldp, done); if (rc_inv != OSSCAR_OK) return rc_inv; }
-    // V = Hinv * G_I
-    k_gather_rows<<<(unsigned)nI, 256, 0, st>>>(ctx->G, L.m, L.g, perm, 0, big, L.ldm);
+    // Every product below that forms a small difference of large sums is accumulated in fp64 (gemm_f64acc): the scores
+    // of Eq. impact are compared at 1e-5 relative, and fp32 accumulation leaves cond(H_II) * 2^-24 in them.
+    // (1) one Newton-Schulz step on the inverse: E = I - H_II Hinv in fp64, Hinv += Hinv E (E is tiny: any product will do)
+    float* E = big;
+    float* Dlt = big + nI * L.ldh;
+    CK(gemm_f64acc(st, nI, nI, nI, -1.0, Hp, L.ldp, Hinv, L.ldh, 0.0, nullptr, 0, E, L.ldh, true, done));
+    CK(gemm_tc(st, nI, nI, nI, 1.f, Hinv, L.ldh, E, L.ldh, 0.f, Dlt, L.ldh, tc, L.tc_bytes, ctx->ctl, done));
+    k_add_sym<<<dim3((unsigned)((nI + 31) / 32), (unsigned)((nI + 31) / 32)), dim3(32, 8), 0, st>>>(Hinv, L.ldh, Dlt, L.ldh, nI, done);
+    count_launches(1);
+    // (2) V = Hinv G_I on the tensor cores, then one refinement step with the residual G_I - H_II V in fp64
+    float* GI = big;
+    float* rV = big + nI * L.ldm;
+    k_gather_rows<<<(unsigned)nI, 256, 0, st>>>(ctx->G, L.m, L.g, perm, 0, GI, L.ldm);
+    count_launches(1);
     if (L.ldm != L.m) CK(cudaMemsetAsync(V, 0, sizeof(float) * nI * L.ldm, st));     // padding columns stay zero
-    // V = Hinv G_I sums large terms of both signs to a small result (cond(H_II) of cancellation): it stays on the
-    // fp32 pipes, whose rounding is unbiased; the tensor core's truncating accumulation cost 0.2 % of obj here
-    CK(sgemm(st, false, false, nI, L.m, nI, 1.f, Hinv, L.ldh, big, L.ldm, 0.f, V, L.ldm, done));
+    CK(gemm_tc(st, nI, L.m, nI, 1.f, Hinv, L.ldh, GI, L.ldm, 0.f, V, L.ldm, tc, L.tc_bytes, ctx->ctl, done));
+    CK(gemm_f64acc(st, nI, L.m, nI, -1.0, Hp, L.ldp, V, L.ldm, 1.0, GI, L.ldm, rV, L.ldm, false, done));
+    CK(gemm_tc(st, nI, L.m, nI, 1.f, Hinv, L.ldh, rV, L.ldm, 1.f, V, L.ldm, tc, L.tc_bytes, ctx->ctl, done));
     // obj = Tr(W^T G) - Tr(G_I^T V)
     if (ctx->have_const) CK(set_device_double(st, &ctx->ctl->acc[0], ctx->user_const));
     else CK(trace_product(st, ctx->W, L.m, ctx->G, L.m, L.d1, L.m, ctx->partials, &ctx->ctl->acc[0]));
-    CK(trace_product(st, big, L.ldm, V, L.ldm, nI, L.m, ctx->partials, &ctx->ctl->acc[1]));
+    CK(trace_product(st, GI, L.ldm, V, L.ldm, nI, L.m, ctx->partials, &ctx->ctl->acc[1]));
     k_set_obj<<<1, 1, 0, st>>>(ctx->ctl);
-    count_launches(2);
+    count_launches(1);
     if (nJ > 0) {
-        // R_J = G_J - Hp[J, I] V
+        // (3) R_J = G_J - Hp[J, I] V, accumulated in fp64
         k_gather_rows<<<(unsigned)nJ, 256, 0, st>>>(ctx->G, L.m, L.g, perm, nI, R, L.ldm);
-        CK(gemm_tc(st, nJ, L.m, nI, -1.f, Hp + nI * L.ldp, L.ldp, V, L.ldm, 1.f, R, L.ldm, tc, L.tc_bytes, ctx->ctl, done));
-        // Pm = Hp[J, I] Hinv, then the Schur complements
-        CK(gemm_tc(st, nJ, nI, nI, 1.f, Hp + nI * L.ldp, L.ldp, Hinv, L.ldh, 0.f, big, L.ldh, tc, L.tc_bytes, ctx->ctl, done));
+        CK(gemm_f64acc(st, nJ, L.m, nI, -1.0, Hp + nI * L.ldp, L.ldp, V, L.ldm, 1.0, R, L.ldm, R, L.ldm, false, done));
+        // (4) Pm = Hp[J, I] Hinv in fp64, then the Schur complements (fp64 dot products)
+        CK(gemm_f64acc(st, nJ, nI, nI, 1.0, Hp + nI * L.ldp, L.ldp, Hinv, L.ldh, 0.0, nullptr, 0, big, L.ldh, false, done));
         k_schur<<<(unsigned)(L.ng - L.k), 256, 0, st>>>(Hp, L.ldp, big, L.ldh, nI, L.g, c);
         count_launches(2);
     }
