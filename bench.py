@@ -110,20 +110,23 @@ def reduce_over_ranks(values: dict, world: int, backend_device):
 
 
 def swap_bytes(nI, nJ, m, fused_y=False):
-    """Algorithmic HBM bytes of one swap (fp32): Hinv read+write, V and R_J read+write, H[J,I] read once, and
-    the y = Hinv h pass (n_I^2 more) unless it is fused into the Hinv update."""
-    return 4 * ((2 if fused_y else 3) * nI * nI + 2 * nI * m + 2 * nJ * m + nJ * nI)
+    """Algorithmic HBM bytes of one swap: V and R_J read+write and H[J,I] read once in fp32; the inverse read+write
+    in fp64 with the next y fused into that pass (single-row groups), or in fp32 with a separate y pass."""
+    if fused_y:
+        return 16 * nI * nI + 4 * (2 * nI * m + 2 * nJ * m + nJ * nI)
+    return 4 * (3 * nI * nI + 2 * nI * m + 2 * nJ * m + nJ * nI)
 
 
 KERNEL_BYTES = {   # algorithmic bytes per launch of the streaming kernels of a step
     "y_pass": lambda nI, nJ, m: 4 * nI * nI,
     "h_pass": lambda nI, nJ, m: 4 * nJ * nI,
     "update_hinv": lambda nI, nJ, m: 8 * nI * nI,
+    "swap_loop": lambda nI, nJ, m: swap_bytes(nI, nJ, m, True),
     "update_v": lambda nI, nJ, m: 8 * nI * m,
     "update_r": lambda nI, nJ, m: 8 * nJ * m,
     "l1_hpass_update_v": lambda nI, nJ, m: 4 * nJ * nI + 8 * nI * m,
     "l2_update_r_swap": lambda nI, nJ, m: 8 * nJ * m,
-    "l4_update_hinv_y": lambda nI, nJ, m: 8 * nI * nI,
+    "l4_update_hinv_y": lambda nI, nJ, m: 16 * nI * nI,
 }
 
 
@@ -212,7 +215,8 @@ def run_ours(args):
     def step(x_chunks, W_in, prof=0):
         return pkg.solve_layer(solver, x_chunks, W_in, wl.g, wl.k, max_swaps, damp=wl.damp, accept_mode=accept, accept_rel_tol=wl.eps_acc,
                                score_mode=b.SCORE_PAIR_EXACT if wl.score_mode == "pair_exact" else b.SCORE_INDEPENDENT,
-                               profile_samples=prof, H=H, G=G, greedy_t_hat=args.greedy, block_pairs=args.block_pairs)
+                               profile_samples=prof, H=H, G=G, greedy_t_hat=args.greedy, block_pairs=args.block_pairs,
+                               loop_mode=args.loop_mode)
 
     def barrier():
         if world > 1:
@@ -398,6 +402,7 @@ def main():
     ap.add_argument("--block-pairs", type=int, default=0, help="groups exchanged per iteration (t_hat = 2 s, p_hat = 0); 0 = single swaps")
     ap.add_argument("--no-block-extra", action="store_true", help="skip the extra solves with block exchanges of 16 and 50 groups")
     ap.add_argument("--accept-always", action="store_true", help="paper-literal fixed number of iterations")
+    ap.add_argument("--loop-mode", type=int, default=0, help="0 auto, 1 persistent cooperative loop, 2 five launches per step (single-row groups)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()

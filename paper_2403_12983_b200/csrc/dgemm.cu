@@ -37,11 +37,12 @@ __device__ __forceinline__ float4 load4_guard(const float* __restrict__ row, int
     return v;
 }
 
-// mode 0: C = beta * C0 + alpha * A B (C0 may alias C);  mode 1: C = I + alpha * A B (C0 unused)
+// mode 0: C = beta * C0 + alpha * A B (C0 may alias C);  mode 1: C = I + alpha * A B (C0 unused).  OutT float or double.
+template <typename OutT>
 __global__ void __launch_bounds__(DG_T, 2)
 k_gemm_f64acc(int64_t M, int64_t N, int64_t K, double alpha, const float* __restrict__ A, int64_t lda,
               const float* __restrict__ B, int64_t ldb, double beta, const float* C0, int64_t ldc0,
-              float* C, int64_t ldc, int mode, int vecA, int vecB, const int32_t* __restrict__ done)
+              OutT* C, int64_t ldc, int mode, int vecA, int vecB, const int32_t* __restrict__ done)
 {
     if (done && *done) return;
     extern __shared__ double dg_smem[];
@@ -120,7 +121,7 @@ k_gemm_f64acc(int64_t M, int64_t N, int64_t K, double alpha, const float* __rest
                 double v = alpha * acc[i][j][e];
                 if (mode == 1) v += (row == col + e) ? 1.0 : 0.0;
                 else if (beta != 0.0) v += beta * (double)C0[row * ldc0 + col + e];
-                C[row * ldc + col + e] = (float)v;
+                C[row * ldc + col + e] = (OutT)v;
             }
         }
     }
@@ -137,9 +138,25 @@ cudaError_t gemm_f64acc(cudaStream_t st, int64_t M, int64_t N, int64_t K, double
     const int vecB = (((uintptr_t)B & 15) == 0 && (ldb % 4) == 0) ? 1 : 0;
     dim3 grid((unsigned)((N + DG_BN - 1) / DG_BN), (unsigned)((M + DG_BM - 1) / DG_BM));
     constexpr int smem = (2 * DG_BM * DG_AS + 2 * DG_BK * DG_BS) * (int)sizeof(double);
-    cudaError_t e = cudaFuncSetAttribute(k_gemm_f64acc, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    cudaError_t e = cudaFuncSetAttribute(k_gemm_f64acc<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
-    k_gemm_f64acc<<<grid, DG_T, smem, st>>>(M, N, K, alpha, A, lda, B, ldb, beta, C0, ldc0, C, ldc, identity_plus ? 1 : 0, vecA, vecB, done);
+    k_gemm_f64acc<float><<<grid, DG_T, smem, st>>>(M, N, K, alpha, A, lda, B, ldb, beta, C0, ldc0, C, ldc, identity_plus ? 1 : 0, vecA, vecB, done);
+    count_launches(1);
+    return cudaGetLastError();
+}
+
+// The plain product with the result kept in fp64: C (M x N doubles, row stride ldc) = A * B.
+cudaError_t gemm_f64out(cudaStream_t st, int64_t M, int64_t N, int64_t K, const float* A, int64_t lda,
+                        const float* B, int64_t ldb, double* C, int64_t ldc, const int32_t* done)
+{
+    if (M <= 0 || N <= 0) return cudaSuccess;
+    const int vecA = (((uintptr_t)A & 15) == 0 && (lda % 4) == 0) ? 1 : 0;
+    const int vecB = (((uintptr_t)B & 15) == 0 && (ldb % 4) == 0) ? 1 : 0;
+    dim3 grid((unsigned)((N + DG_BN - 1) / DG_BN), (unsigned)((M + DG_BM - 1) / DG_BM));
+    constexpr int smem = (2 * DG_BM * DG_AS + 2 * DG_BK * DG_BS) * (int)sizeof(double);
+    cudaError_t e = cudaFuncSetAttribute(k_gemm_f64acc<double>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    k_gemm_f64acc<double><<<grid, DG_T, smem, st>>>(M, N, K, 1.0, A, lda, B, ldb, 0.0, nullptr, 0, C, ldc, 0, vecA, vecB, done);
     count_launches(1);
     return cudaGetLastError();
 }

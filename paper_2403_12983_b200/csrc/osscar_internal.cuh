@@ -48,6 +48,7 @@ struct Layout {
     int64_t ldm;             // leading dimension of V, R, K, Vq
     // offsets in bytes from the workspace base
     size_t off_Hp, off_Hinv, off_V, off_R, off_big;
+    size_t off_Hd;                                                     // fp64 copy of the inverse (g = 1 only, else a stub)
     size_t off_y, off_b, off_u2, off_bC, off_u2c, off_u, off_d, off_K, off_Vq;
     size_t off_vec_begin, off_vec_end;   // the staged vectors (zeroed once when the state is built)
     size_t off_vnorm, off_rnorm, off_D, off_A, off_c, off_small, off_gramV, off_gramR;
@@ -98,6 +99,7 @@ struct osscar_ctx {
     bool have_const;                 // const term supplied by the caller (cross-term problems) instead of Tr(W^T G)
     double user_const;
     long long wait_limit;            // context default of SearchCtl::wait_limit
+    bool hd_valid;                   // the fp64 copy of the inverse matches the state
 };
 
 namespace osscar {
@@ -114,6 +116,8 @@ cudaError_t sgemm(cudaStream_t st, bool transA, bool transB, int64_t M, int64_t 
 cudaError_t gemm_f64acc(cudaStream_t st, int64_t M, int64_t N, int64_t K, double alpha, const float* A, int64_t lda,
                         const float* B, int64_t ldb, double beta, const float* C0, int64_t ldc0, float* C, int64_t ldc,
                         bool identity_plus, const int32_t* done = nullptr);
+cudaError_t gemm_f64out(cudaStream_t st, int64_t M, int64_t N, int64_t K, const float* A, int64_t lda,
+                        const float* B, int64_t ldb, double* C, int64_t ldc, const int32_t* done = nullptr);
 
 // ---- panel_tc.cu: Y[i*so_row + e*so_col] = sum_k A[i][k] * P[e][k] on the tensor cores; A (M x K, streamed once) is split
 // into bf16 terms on the way (fp32-accurate); P is an N x K panel
@@ -167,5 +171,7 @@ int greedy_support(osscar_ctx* ctx, int t_hat, int32_t* support, int32_t* drop_t
 int run_search(osscar_ctx* ctx, const osscar_search_params* p, int32_t* support_out, float* W_out,
                double* obj_trace, int32_t* swap_trace, osscar_search_result* res);
 cudaError_t score_pass(osscar_ctx* ctx);   // full scoring pass from the current state (fills D, A)
+// fp64 copy of the inverse from the fp32 one by a Newton-Schulz step summed in fp64 (single-row groups; uses `big`)
+int build_hinv64(osscar_ctx* ctx, bool guarded);
 
 }  // namespace osscar

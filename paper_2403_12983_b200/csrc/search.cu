@@ -40,6 +40,7 @@ __device__ __forceinline__ float dot4f(const float4& a, const float4& b) {
 struct Ptrs {
     float *Hp, *Hinv, *V, *R, *y, *b, *u2, *bC, *u2c, *u, *d, *K, *Vq, *vnorm, *rnorm;
     double *D, *A, *c, *small, *gramV, *gramR;
+    double *Hd;                                              // fp64 copy of the inverse (single-row groups, independent scores)
     double *pairCinv, *pairKK, *pairScratch, *pairDelta;     // PAIR_EXACT scoring
     int32_t *perm, *slotof;
     SearchCtl* ctl;
@@ -937,6 +938,7 @@ Ptrs make_ptrs(osscar_ctx* ctx)
     p.vnorm = (float*)(ws + L.off_vnorm); p.rnorm = (float*)(ws + L.off_rnorm);
     p.D = (double*)(ws + L.off_D); p.A = (double*)(ws + L.off_A); p.c = (double*)(ws + L.off_c);
     p.small = (double*)(ws + L.off_small); p.gramV = (double*)(ws + L.off_gramV); p.gramR = (double*)(ws + L.off_gramR);
+    p.Hd = (double*)(ws + L.off_Hd);
     p.perm = (int32_t*)(ws + L.off_perm); p.slotof = (int32_t*)(ws + L.off_slotof);
     p.pairCinv = (double*)(ws + L.off_pairCinv); p.pairKK = (double*)(ws + L.off_pairKK);
     p.pairScratch = (double*)(ws + L.off_pairScratch); p.pairDelta = (double*)(ws + L.off_pairDelta);
@@ -995,6 +997,27 @@ int persistent_grid(const Layout& L)
 }
 
 }  // namespace
+
+int build_hinv64(osscar_ctx* ctx, bool guarded)
+{
+    const Layout& L = ctx->L;
+    cudaStream_t st = ctx->stream;
+    char* ws = (char*)ctx->ws;
+    float* Hp = (float*)(ws + L.off_Hp);
+    float* Hinv = (float*)(ws + L.off_Hinv);
+    double* Hd = (double*)(ws + L.off_Hd);
+    float* E = (float*)(ws + L.off_big);
+    float* Dlt = E + L.nI * L.ldh;
+    const int32_t* done = guarded ? &ctx->ctl->done : nullptr;
+    // E = I - H_II Hinv with fp64 sums; Hd = Hinv + Hinv E, the sum taken in fp64 (the correction is below 2^-24 of Hinv)
+    if (gemm_f64acc(st, L.nI, L.nI, L.nI, -1.0, Hp, L.ldp, Hinv, L.ldh, 0.0, nullptr, 0, E, L.ldh, true, done) != cudaSuccess) return OSSCAR_E_CUDA;
+    if (gemm_tc(st, L.nI, L.nI, L.nI, 1.f, Hinv, L.ldh, E, L.ldh, 0.f, Dlt, L.ldh, ws + L.off_tc, L.tc_bytes, ctx->ctl, done) != cudaSuccess) return OSSCAR_E_CUDA;
+    k_hinv_to_d<<<(unsigned)L.nI, 256, 0, st>>>(Hinv, Dlt, Hd, L.ldh, L.nI, done);
+    count_launches(1);
+    if (cudaGetLastError() != cudaSuccess) return OSSCAR_E_CUDA;
+    ctx->hd_valid = true;
+    return OSSCAR_OK;
+}
 
 cudaError_t score_pass(osscar_ctx* ctx)
 {
@@ -1065,11 +1088,15 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
     auto bootstrap_g1 = [&]() -> cudaError_t {       // score vectors, first entering group and its y from the current state
         k_scores_g1<<<(unsigned)((L.d1 + 255) / 256), 256, 0, st>>>(p);
         k_select_in_g1<<<1, 1024, 0, st>>>(p);
-        k_ypass<<<dim3((unsigned)((L.nI + 7) / 8), 1), 256, 0, st>>>(p);
+        k_ypass_d<<<dim3((unsigned)((L.nI + 7) / 8), 1), 256, 0, st>>>(p);
         count_launches(3);
         return cudaGetLastError();
     };
-    if (max_swaps > 0 && fast) CK(bootstrap_g1());
+    if (g == 1 && !fast) ctx->hd_valid = false;          // these drivers move the fp32 inverse only
+    if (max_swaps > 0 && fast) {
+        if (!ctx->hd_valid) { const int rcd = build_hinv64(ctx, false); if (rcd != OSSCAR_OK) return rcd; }
+        CK(bootstrap_g1());
+    }
 
     if (block) {
         CK(cudaMemsetAsync((char*)ctx->ws + L.off_block, 0, block_bytes_for(L, bs * g), st));
@@ -1235,6 +1262,10 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
         return rc;
     }
     CK(cudaEventRecord(ctx->ev1, st));
+    if (fast && max_swaps > 0) {       // the fp32 inverse follows its fp64 copy (state reader, other drivers)
+        k_hinv_from_d<<<(unsigned)L.nI, 256, 0, st>>>(p.Hd, p.Hinv, L.ldh);
+        count_launches(1);
+    }
 
     // results: weights, support, objective recomputed from the final state
     CK(cudaMemsetAsync(W_out, 0, sizeof(float) * L.d1 * L.m, st));

@@ -26,7 +26,7 @@ __global__ void k_scores_g1(Ptrs p)
     if (p.ctl->done) return;
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i < p.nI) {
-        const double hd = p.Hinv[i * p.ldh + i];
+        const double hd = p.Hd[i * p.ldh + i];
         p.D[i] = hd > 0.0 ? (double)p.vnorm[i] / hd : INFINITY;
     } else if (i < p.nI + p.nJ) {
         const int64_t t = i - p.nI;
@@ -114,7 +114,7 @@ k_decide_g1(Ptrs p, int accept_mode, double accept_tol, double* __restrict__ obj
     for (int64_t c = threadIdx.x; c < p.ldm / 4; c += blockDim.x) acc += dot4(vr[c], rq[c]);
     const double GX = (double)block_sum_f(acc, redf);
     if (threadIdx.x == 0) {
-        const double C = p.Hinv[r0 * p.ldh + r0], P = p.y[r0], cq = p.c[t];
+        const double C = p.Hd[r0 * p.ldh + r0], P = p.y[r0], cq = p.c[t];
         const double GV = p.vnorm[r0], GR = p.rnorm[t];
         const double Cinv = 1.0 / C;
         const double Ds = GV * Cinv;
@@ -145,14 +145,14 @@ k_decide_g1(Ptrs p, int accept_mode, double accept_tol, double* __restrict__ obj
     if (s_stop) return;
     const float Q1 = (float)p.small[G1_Q1];
     const double Cinv = p.small[S_CINV], c1inv = p.small[S_C1INV], M2 = p.small[G1_M2];
-    const float* hrow = p.Hinv + r0 * p.ldh;
-    // float4 wide (pads of Hinv rows, y, V, R are zero, so the padded tails stay zero)
-    const float4* hrow4 = reinterpret_cast<const float4*>(hrow);
+    // float4 wide (pads of Hinv rows, y, V, R are zero, so the padded tails stay zero); the inverse is kept in fp64
+    const double2* hrow2 = reinterpret_cast<const double2*>(p.Hd + r0 * p.ldh);
     const float4* y4 = reinterpret_cast<const float4*>(p.y);
     float4* b4 = reinterpret_cast<float4*>(p.b);
     float4* u4 = reinterpret_cast<float4*>(p.u2);
     for (int64_t c = threadIdx.x; c < p.ldh / 4; c += blockDim.x) {
-        const float4 bs = hrow4[c], yy = y4[c];
+        const double2 h0 = hrow2[2 * c], h1 = hrow2[2 * c + 1];
+        const float4 bs = make_float4((float)h0.x, (float)h0.y, (float)h1.x, (float)h1.y), yy = y4[c];
         float4 uu = make_float4(fmaf(-bs.x, Q1, yy.x), fmaf(-bs.y, Q1, yy.y), fmaf(-bs.z, Q1, yy.z), fmaf(-bs.w, Q1, yy.w));
         const int64_t rc = r0 - c * 4;
         uu.x = rc == 0 ? 0.f : uu.x; uu.y = rc == 1 ? 0.f : uu.y; uu.z = rc == 2 ? 0.f : uu.z; uu.w = rc == 3 ? 0.f : uu.w;
@@ -266,7 +266,7 @@ __device__ __forceinline__ void update_row_g1(const Ptrs& p, int kind, int64_t s
                 if (sp[r]) hd = c1inv;
                 else {
                     const double bs = p.b[s], us = p.u2[s];
-                    hd = (double)p.Hinv[s * p.ldh + s] - bs * bs * Cinv + us * us * c1inv;
+                    hd = p.Hd[s * p.ldh + s] - bs * bs * Cinv + us * us * c1inv;
                 }
                 p.D[s] = hd > 0.0 ? (double)nr / hd : INFINITY;
             } else {
@@ -335,7 +335,7 @@ __device__ __forceinline__ void hpass_stream(const Ptrs& p, const float4* const 
 // L1: blocks [0, nbV) update G1_RB rows of V each; then one block per G1_RB pruned rows of the H pass (their addresses
 // need no control-block read, so their streams start at once) and a last block for the leaving row.
 constexpr int G1_RB = 1;            // rows per block of the V / R updates and the H pass
-constexpr int G1_RB4 = 2;           // rows per block of the Hinv update
+constexpr int G1_RB4 = 1;           // rows per block of the Hinv update
 __global__ void __launch_bounds__(G1_T, 4) k_l1_g1(Ptrs p, unsigned nbV)      // 64 registers: four resident blocks per SM
 {
     __shared__ float red[16];
@@ -403,72 +403,113 @@ __global__ void __launch_bounds__(G1_T, 4) k_l2_g1(Ptrs p, unsigned nbR)
     }
 }
 
-// L4: Hinv' = Hinv - (b/C) b^T + (u2/c1) u2^T (row and column r0: -u2/c1, corner 1/c1) and, in the same pass,
-// y_next = Hinv' h with h = Hp[row of the next entering group, 0:n_I].  RB rows per block: every piece of b, u2 and h
-// fetched from L2 serves the RB rows.
+// L4: Hinv' = Hinv - (b/C) b^T + (u2/c1) u2^T (row and column r0: -u2/c1, corner 1/c1) on the fp64 copy of the inverse and,
+// in the same pass, y_next = Hinv' h with h = Hp[row of the next entering group, 0:n_I].  RB rows per block; a piece is a
+// double2, nine pieces per thread and pass.
 template <int RB>
 __global__ void __launch_bounds__(G1_T) k_l4_g1(Ptrs p)
 {
-    __shared__ float red[8];
+    __shared__ double red[8];
     const int64_t s0 = (int64_t)blockIdx.x * RB;
-    const float4* b4 = reinterpret_cast<const float4*>(p.b);
-    const float4* u4 = reinterpret_cast<const float4*>(p.u2);
-    const int64_t n4 = p.ldh / 4;
-    float4* row[RB];
+    const float2* b2 = reinterpret_cast<const float2*>(p.b);
+    const float2* u2v = reinterpret_cast<const float2*>(p.u2);
+    const int64_t n2 = p.ldh / 2;
+    double2* row[RB];
 #pragma unroll
-    for (int r = 0; r < RB; ++r) row[r] = reinterpret_cast<float4*>(p.Hinv + (s0 + r < p.nI ? s0 + r : p.nI - 1) * p.ldh);
+    for (int r = 0; r < RB; ++r) row[r] = reinterpret_cast<double2*>(p.Hd + (s0 + r < p.nI ? s0 + r : p.nI - 1) * p.ldh);
     int64_t r0 = 0;
-    const float4* h4 = nullptr;
+    const float2* h2 = nullptr;
     bool srow[RB];
-    float nb[RB], us[RB], corner[RB], yacc[RB];
+    double nb[RB], us[RB], corner[RB], yacc[RB];
 #pragma unroll
-    for (int r = 0; r < RB; ++r) { srow[r] = false; nb[r] = 0.f; us[r] = 0.f; corner[r] = 0.f; yacc[r] = 0.f; }
-    for (int64_t base = threadIdx.x; base < n4; base += (int64_t)G1_T * G1_UH) {
-        float4 h[RB][G1_UH];
+    for (int r = 0; r < RB; ++r) { srow[r] = false; nb[r] = 0.0; us[r] = 0.0; corner[r] = 0.0; yacc[r] = 0.0; }
+    for (int64_t base = threadIdx.x; base < n2; base += (int64_t)G1_T * G1_UH) {
+        double2 h[RB][G1_UH];
 #pragma unroll
         for (int r = 0; r < RB; ++r)
 #pragma unroll
             for (int j = 0; j < G1_UH; ++j) {
                 const int64_t c = base + G1_T * j;
-                h[r][j] = c < n4 ? row[r][c] : make_float4(0.f, 0.f, 0.f, 0.f);   // requested before the step's scalars arrive
+                h[r][j] = c < n2 ? row[r][c] : make_double2(0.0, 0.0);    // requested before the step's scalars arrive
             }
         if (base == threadIdx.x) {
             if (p.ctl->done) return;
             r0 = p.ctl->sel_slot;
-            const float Cinv = (float)p.small[S_CINV], c1inv = (float)p.small[S_C1INV];
-            h4 = reinterpret_cast<const float4*>(p.Hp + (p.nI + (int64_t)p.ctl->sel_t) * p.ldp);
+            const double Cinv = p.small[S_CINV], c1inv = p.small[S_C1INV];
+            h2 = reinterpret_cast<const float2*>(p.Hp + (p.nI + (int64_t)p.ctl->sel_t) * p.ldp);
 #pragma unroll
             for (int r = 0; r < RB; ++r) {
                 const int64_t s = s0 + r < p.nI ? s0 + r : p.nI - 1;
                 srow[r] = s == r0;
                 // row r0 becomes -u2/c1: treat it as 0 * old - 0 * b + (-1/c1) * u2
-                nb[r] = srow[r] ? 0.f : -p.b[s] * Cinv;
-                us[r] = srow[r] ? -c1inv : p.u2[s] * c1inv;
+                nb[r] = srow[r] ? 0.0 : -(double)p.b[s] * Cinv;
+                us[r] = srow[r] ? -c1inv : (double)p.u2[s] * c1inv;
                 corner[r] = srow[r] ? c1inv : -us[r];                            // value of column r0 in this row
             }
         }
 #pragma unroll
         for (int j = 0; j < G1_UH; ++j) {
             const int64_t c = base + G1_T * j;
-            if (c < n4) {
-                const float4 bb = __ldg(b4 + c), uu = __ldg(u4 + c), hh = __ldg(h4 + c);
-                const int64_t rc = r0 - c * 4;           // position of column r0 inside this float4, if any
+            if (c < n2) {
+                const float2 bb = __ldg(b2 + c), uu = __ldg(u2v + c), hh = __ldg(h2 + c);
+                const int64_t rc = r0 - c * 2;           // position of column r0 inside this piece, if any
 #pragma unroll
                 for (int r = 0; r < RB; ++r) {
-                    if (srow[r]) h[r][j] = make_float4(0.f, 0.f, 0.f, 0.f);
-                    fma4(h[r][j], nb[r], bb);
-                    fma4(h[r][j], us[r], uu);
-                    h[r][j].x = rc == 0 ? corner[r] : h[r][j].x; h[r][j].y = rc == 1 ? corner[r] : h[r][j].y;
-                    h[r][j].z = rc == 2 ? corner[r] : h[r][j].z; h[r][j].w = rc == 3 ? corner[r] : h[r][j].w;
-                    if (s0 + r < p.nI) row[r][c] = h[r][j];
-                    yacc[r] += dot4(h[r][j], hh);
+                    double2 v = srow[r] ? make_double2(0.0, 0.0) : h[r][j];
+                    v.x = fma(us[r], (double)uu.x, fma(nb[r], (double)bb.x, v.x));
+                    v.y = fma(us[r], (double)uu.y, fma(nb[r], (double)bb.y, v.y));
+                    v.x = rc == 0 ? corner[r] : v.x;
+                    v.y = rc == 1 ? corner[r] : v.y;
+                    if (s0 + r < p.nI) row[r][c] = v;
+                    yacc[r] = fma(v.x, (double)hh.x, fma(v.y, (double)hh.y, yacc[r]));
                 }
             }
         }
     }
 #pragma unroll
     for (int r = 0; r < RB; ++r) {
-        const float t = block_sum_256(yacc[r], red);
-        if (threadIdx.x == 0 && s0 + r < p.nI) p.y[s0 + r] = t;
+        double t = warp_sum(yacc[r]);
+        __syncthreads();
+        if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = t;
+        __syncthreads();
+        if (threadIdx.x == 0 && s0 + r < p.nI) {
+            double sum = 0.0;
+#pragma unroll
+            for (int i = 0; i < G1_T / 32; ++i) sum += red[i];
+            p.y[s0 + r] = (float)sum;
+        }
     }
+}
+
+// y = Hd h for the entering group chosen by the bootstrap (one warp per row; runs once per state build).
+__global__ void __launch_bounds__(256) k_ypass_d(Ptrs p)
+{
+    if (p.ctl->done) return;
+    const int lane = threadIdx.x & 31;
+    const int64_t s = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (s >= p.nI) return;
+    const float* hrow = p.Hp + (p.nI + (int64_t)p.ctl->sel_t) * p.ldp;
+    const double* arow = p.Hd + s * p.ldh;
+    double acc = 0.0;
+    for (int64_t c = lane; c < p.nI; c += 32) acc = fma(arow[c], (double)hrow[c], acc);
+    acc = warp_sum(acc);
+    if (lane == 0) p.y[s] = (float)acc;
+}
+
+// Hd := (double) Hinv + (double) Dlt, symmetrised (second Newton-Schulz step, summed in fp64), and the reverse copy.
+__global__ void k_hinv_to_d(const float* __restrict__ Hinv, const float* __restrict__ Dlt, double* __restrict__ Hd, int64_t ldh, int64_t n,
+                            const int32_t* __restrict__ done)
+{
+    if (done && *done) return;
+    const int64_t r = blockIdx.x;
+    for (int64_t c = threadIdx.x; c < ldh; c += blockDim.x) {
+        double v = 0.0;
+        if (c < n) v = 0.5 * (((double)Hinv[r * ldh + c] + (double)Hinv[c * ldh + r]) + ((double)Dlt[r * ldh + c] + (double)Dlt[c * ldh + r]));
+        Hd[r * ldh + c] = v;
+    }
+}
+__global__ void k_hinv_from_d(const double* __restrict__ Hd, float* __restrict__ Hinv, int64_t ldh)
+{
+    const int64_t r = blockIdx.x;
+    for (int64_t c = threadIdx.x; c < ldh; c += blockDim.x) Hinv[r * ldh + c] = (float)Hd[r * ldh + c];
 }

@@ -131,6 +131,26 @@ __device__ __forceinline__ void block_sums(float (&v)[RB], float* red /*[RB * 8]
     }
 }
 
+template <int RB>
+__device__ __forceinline__ void block_sums_d(double (&v)[RB], double* red /*[RB * 8]*/)
+{
+#pragma unroll
+    for (int r = 0; r < RB; ++r) v[r] = warp_sum(v[r]);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) {
+#pragma unroll
+        for (int r = 0; r < RB; ++r) red[r * 8 + (threadIdx.x >> 5)] = v[r];
+    }
+    __syncthreads();
+#pragma unroll
+    for (int r = 0; r < RB; ++r) {
+        double t = 0.0;
+#pragma unroll
+        for (int i = 0; i < PL_T / 32; ++i) t += red[r * 8 + i];
+        v[r] = t;
+    }
+}
+
 // P1 / P2 row updates.  kind 0: V'[s] = V[s] - b[s] K - u2[s] Vq (row r0 := Vq), D'[s];
 // kind 1: R'[l] = R[l] + u[l] K - d[l] Vq (row t := K - d_r Vq), c'[l], A'[l].  RB rows per pass, grid stride.
 template <int RB>
@@ -179,7 +199,7 @@ __device__ __noinline__ void pl_update_rows(const Ptrs& p, const int kind, const
                 }
                 if (tid < RB && rows0 + tid < nrows) {
                     const int64_t s = rows0 + tid;
-                    if (kind == 0) { e0 = (double)p.Hinv[s * p.ldh + s]; e1 = (double)p.b[s]; e2 = (double)p.u2[s]; }
+                    if (kind == 0) { e0 = p.Hd[s * p.ldh + s]; e1 = (double)p.b[s]; e2 = (double)p.u2[s]; }
                     else { e0 = p.c[s]; e1 = (double)p.Hp[(p.nI + s) * p.ldp + p.nI + s]; }
                 }
             }
@@ -287,32 +307,35 @@ __device__ __noinline__ void pl_hpass(const Ptrs& p, const StepScal& sc, unsigne
     }
 }
 
-// P3: Hinv' rows (row and column r0 replaced) and y_next = Hinv' h, RB rows per pass.
+// P3: rows of the inverse, kept in fp64 (row and column r0 replaced), and y_next = Hinv' h; RB rows per pass.
+// The inverse is the one piece of the state that fp32 cannot carry: y = Hinv h cancels the common component of the
+// rows of H to a few parts in 10^4, so an entry rounded to 2^-24 shows up in y, then in u2, and from there in every
+// matrix (measured: the scores drift 3e-7 per swap with an fp32 inverse, 5e-9 with this one).  A piece is a double2.
 template <int RB>
 __device__ __noinline__ void pl_update_hinv(const Ptrs& p, const StepScal& sc, int64_t t_next, unsigned nblocks, float* red)
 {
     constexpr int PP = PlPieces<RB>::value;
-    const float4* b4 = reinterpret_cast<const float4*>(p.b);
-    const float4* u4 = reinterpret_cast<const float4*>(p.u2);
-    const float4* h4 = reinterpret_cast<const float4*>(p.Hp + (p.nI + t_next) * p.ldp);
-    const int64_t n4 = p.ldh / 4;
+    const float2* b2 = reinterpret_cast<const float2*>(p.b);
+    const float2* u2v = reinterpret_cast<const float2*>(p.u2);
+    const float2* h2 = reinterpret_cast<const float2*>(p.Hp + (p.nI + t_next) * p.ldp);
+    const int64_t n2 = p.ldh / 2;
     const int tid = threadIdx.x;
     for (int64_t s0 = (int64_t)blockIdx.x * RB; s0 < p.nI; s0 += (int64_t)nblocks * RB) {
-        float4* row[RB];
+        double2* row[RB];
 #pragma unroll
-        for (int r = 0; r < RB; ++r) row[r] = reinterpret_cast<float4*>(p.Hinv + (s0 + r < p.nI ? s0 + r : p.nI - 1) * p.ldh);
+        for (int r = 0; r < RB; ++r) row[r] = reinterpret_cast<double2*>(p.Hd + (s0 + r < p.nI ? s0 + r : p.nI - 1) * p.ldh);
         bool srow[RB];
-        float nb[RB], us[RB], corner[RB], yacc[RB];
+        double nb[RB], us[RB], corner[RB], yacc[RB];
 #pragma unroll
-        for (int r = 0; r < RB; ++r) yacc[r] = 0.f;
-        for (int64_t base = tid; base < n4; base += (int64_t)PL_T * PP) {
-            float4 h[RB][PP];
+        for (int r = 0; r < RB; ++r) { yacc[r] = 0.0; srow[r] = false; nb[r] = 0.0; us[r] = 0.0; corner[r] = 0.0; }
+        for (int64_t base = tid; base < n2; base += (int64_t)PL_T * PP) {
+            double2 h[RB][PP];
 #pragma unroll
             for (int r = 0; r < RB; ++r)
 #pragma unroll
                 for (int j = 0; j < PP; ++j) {
                     const int64_t c = base + PL_T * j;
-                    h[r][j] = c < n4 ? row[r][c] : make_float4(0.f, 0.f, 0.f, 0.f);
+                    h[r][j] = c < n2 ? row[r][c] : make_double2(0.0, 0.0);
                 }
             if (base == tid) {
 #pragma unroll
@@ -320,36 +343,36 @@ __device__ __noinline__ void pl_update_hinv(const Ptrs& p, const StepScal& sc, i
                     const int64_t s = s0 + r < p.nI ? s0 + r : p.nI - 1;
                     srow[r] = s == sc.r0;
                     // row r0 becomes -u2 / c1: 0 * old - 0 * b + (-1 / c1) * u2
-                    nb[r] = srow[r] ? 0.f : -p.b[s] * sc.Cinv;
-                    us[r] = srow[r] ? -sc.c1inv : p.u2[s] * sc.c1inv;
-                    corner[r] = srow[r] ? sc.c1inv : -us[r];         // value of column r0 in this row
+                    nb[r] = srow[r] ? 0.0 : -(double)p.b[s] * sc.Cinv_d;
+                    us[r] = srow[r] ? -sc.c1inv_d : (double)p.u2[s] * sc.c1inv_d;
+                    corner[r] = srow[r] ? sc.c1inv_d : -us[r];       // value of column r0 in this row
                 }
             }
 #pragma unroll
             for (int j = 0; j < PP; ++j) {
                 const int64_t c = base + PL_T * j;
-                if (c < n4) {
-                    const float4 bb = __ldg(b4 + c), uu = __ldg(u4 + c), hh = __ldg(h4 + c);
-                    const int64_t rc = sc.r0 - c * 4;                // position of column r0 inside this float4, if any
+                if (c < n2) {
+                    const float2 bb = __ldg(b2 + c), uu = __ldg(u2v + c), hh = __ldg(h2 + c);
+                    const int64_t rc = sc.r0 - c * 2;                // position of column r0 inside this piece, if any
 #pragma unroll
                     for (int r = 0; r < RB; ++r) {
-                        if (srow[r]) h[r][j] = make_float4(0.f, 0.f, 0.f, 0.f);
-                        fma4(h[r][j], nb[r], bb);
-                        fma4(h[r][j], us[r], uu);
-                        h[r][j].x = rc == 0 ? corner[r] : h[r][j].x; h[r][j].y = rc == 1 ? corner[r] : h[r][j].y;
-                        h[r][j].z = rc == 2 ? corner[r] : h[r][j].z; h[r][j].w = rc == 3 ? corner[r] : h[r][j].w;
-                        if (s0 + r < p.nI) row[r][c] = h[r][j];
-                        yacc[r] += dot4(h[r][j], hh);
+                        double2 v = srow[r] ? make_double2(0.0, 0.0) : h[r][j];
+                        v.x = fma(us[r], (double)uu.x, fma(nb[r], (double)bb.x, v.x));
+                        v.y = fma(us[r], (double)uu.y, fma(nb[r], (double)bb.y, v.y));
+                        v.x = rc == 0 ? corner[r] : v.x;
+                        v.y = rc == 1 ? corner[r] : v.y;
+                        if (s0 + r < p.nI) row[r][c] = v;
+                        yacc[r] = fma(v.x, (double)hh.x, fma(v.y, (double)hh.y, yacc[r]));
                     }
                 }
             }
         }
-        block_sums<RB>(yacc, red);
+        block_sums_d<RB>(yacc, reinterpret_cast<double*>(red));
         if (tid < RB && s0 + tid < p.nI) {
-            float t = yacc[0];
+            double t = yacc[0];
 #pragma unroll
             for (int r = 1; r < RB; ++r) t = tid == r ? yacc[r] : t;
-            p.y[s0 + tid] = t;
+            p.y[s0 + tid] = (float)t;
         }
     }
 }
@@ -378,7 +401,7 @@ __global__ void __launch_bounds__(PL_T, 3) k_swap_loop_g1(LoopArgs a)
     __syncthreads();
     const Ptrs& p = s_p;
     SearchCtl* ctl = a.p.ctl;
-    __shared__ float red[8 * 8];
+    __shared__ __align__(16) float red[8 * 8];
     __shared__ LoopCand s_best[4];
     __shared__ StepScal s_sc;
     __shared__ int s_flag, s_stop, s_idx;
@@ -390,7 +413,7 @@ __global__ void __launch_bounds__(PL_T, 3) k_swap_loop_g1(LoopArgs a)
     unsigned long long epoch = 0;
     double obj = ctl->obj;
     int n_swaps = ctl->n_swaps;
-    const int rbm = pl_rows_per_pass(p.ldm / 4), rbh = pl_rows_per_pass(p.ldh / 4);
+    const int rbm = pl_rows_per_pass(p.ldm / 4), rbh = pl_rows_per_pass(p.ldh / 4), rbd = pl_rows_per_pass(p.ldh / 2);
 
     // candidates from the score vectors that the host-side bootstrap left (D, A of the current state)
     if (tid < 4) s_best[tid].idx = -1;
@@ -452,7 +475,7 @@ __global__ void __launch_bounds__(PL_T, 3) k_swap_loop_g1(LoopArgs a)
             block_sums<1>(gx, red);
             if (tid == 0) {
                 const double GX = (double)gx[0];
-                const double C = p.Hinv[r0 * p.ldh + r0], P = p.y[r0], cq = p.c[t];
+                const double C = p.Hd[r0 * p.ldh + r0], P = p.y[r0], cq = p.c[t];
                 const double GV = p.vnorm[r0], GR = p.rnorm[t];
                 const double Cinv = 1.0 / C;
                 const double Ds = GV * Cinv;
@@ -498,12 +521,13 @@ __global__ void __launch_bounds__(PL_T, 3) k_swap_loop_g1(LoopArgs a)
         StepScal sc = s_sc;
         {   // staged vectors, a slice per block
             const int64_t gidx = (int64_t)blockIdx.x * PL_T + tid, gstride = (int64_t)nblocks * PL_T;
-            const float4* hrow4 = reinterpret_cast<const float4*>(p.Hinv + r0 * p.ldh);
+            const double2* hrow2 = reinterpret_cast<const double2*>(p.Hd + r0 * p.ldh);
             const float4* y4 = reinterpret_cast<const float4*>(p.y);
             float4* b4 = reinterpret_cast<float4*>(p.b);
             float4* u4 = reinterpret_cast<float4*>(p.u2);
             for (int64_t c = gidx; c < p.ldh / 4; c += gstride) {
-                const float4 bs = hrow4[c], yy = y4[c];
+                const double2 h0 = hrow2[2 * c], h1 = hrow2[2 * c + 1];
+                const float4 bs = make_float4((float)h0.x, (float)h0.y, (float)h1.x, (float)h1.y), yy = y4[c];
                 float4 uu = make_float4(fmaf(-bs.x, sc.Q1, yy.x), fmaf(-bs.y, sc.Q1, yy.y), fmaf(-bs.z, sc.Q1, yy.z), fmaf(-bs.w, sc.Q1, yy.w));
                 const int64_t rc = r0 - c * 4;
                 uu.x = rc == 0 ? 0.f : uu.x; uu.y = rc == 1 ? 0.f : uu.y; uu.z = rc == 2 ? 0.f : uu.z; uu.w = rc == 3 ? 0.f : uu.w;
@@ -561,8 +585,8 @@ __global__ void __launch_bounds__(PL_T, 3) k_swap_loop_g1(LoopArgs a)
         __syncthreads();
         const int64_t t_next = s_idx >= 0 ? s_idx : 0;
         const bool no_add = s_idx < 0;
-        if (rbh == 4) pl_update_hinv<4>(p, sc, t_next, nblocks, red);
-        else if (rbh == 2) pl_update_hinv<2>(p, sc, t_next, nblocks, red);
+        if (rbd == 4) pl_update_hinv<4>(p, sc, t_next, nblocks, red);
+        else if (rbd == 2) pl_update_hinv<2>(p, sc, t_next, nblocks, red);
         else pl_update_hinv<1>(p, sc, t_next, nblocks, red);
         t_cur = t_next;
         if (timer) a.prof[4] += 1;

@@ -248,17 +248,19 @@ __global__ void k_gj_writeback(float* __restrict__ A, int64_t lda, int64_t n, in
 }
 
 // c_t[a][b] = Hp[J_ta][J_tb] - sum_s Pm[ta][s] * Hp[J_tb][s]  for pruned slot t; one block per t.
-__global__ void k_schur(const float* __restrict__ Hp, int64_t ldp, const float* __restrict__ Pm, int64_t ldpm,
-                        int64_t nI, int g, double* __restrict__ c)
+// Pm holds the rows of the pruned slots [t0, t0 + gridDim.x) in fp64 (row stride ldpm).
+__global__ void k_schur(const float* __restrict__ Hp, int64_t ldp, const double* __restrict__ Pm, int64_t ldpm,
+                        int64_t nI, int g, double* __restrict__ c, int64_t t0, const int32_t* __restrict__ done)
 {
-    const int64_t t = blockIdx.x;
+    if (done && *done) return;
+    const int64_t t = t0 + blockIdx.x;
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
     for (int pair = w; pair < g * g; pair += nw) {
         const int a = pair / g, b = pair % g;
-        const float* pr = Pm + (t * g + a) * ldpm;
+        const double* pr = Pm + ((t - t0) * g + a) * ldpm;
         const float* hr = Hp + (nI + t * g + b) * ldp;
         double s = 0.0;
-        for (int64_t x = lane; x < nI; x += 32) s += (double)pr[x] * (double)hr[x];
+        for (int64_t x = lane; x < nI; x += 32) s = fma(pr[x], (double)hr[x], s);
         s = warp_sum(s);
         if (lane == 0) c[(t * g + a) * g + b] = (double)Hp[(nI + t * g + a) * ldp + nI + t * g + b] - s;
     }
@@ -361,6 +363,7 @@ int make_layout(int64_t d1, int64_t m, int32_t g, int32_t k, Layout* L)
     L->off_big = take(sizeof(float) * big);
     L->off_Hp = take(sizeof(float) * d1 * L->ldp);
     L->off_Hinv = take(sizeof(float) * nI * ldh);
+    L->off_Hd = take(g == 1 ? sizeof(double) * nI * ldh : 256);
     L->off_V = take(sizeof(float) * nI * ldm);
     L->off_R = take(sizeof(float) * (nJ > 0 ? nJ : 1) * ldm);
     L->off_y = take(sizeof(float) * ldh * g);
@@ -507,6 +510,8 @@ int build_state(osscar_ctx* ctx, bool guarded)
     CK(gemm_tc(st, nI, nI, nI, 1.f, Hinv, L.ldh, E, L.ldh, 0.f, Dlt, L.ldh, tc, L.tc_bytes, ctx->ctl, done));
     k_add_sym<<<dim3((unsigned)((nI + 31) / 32), (unsigned)((nI + 31) / 32)), dim3(32, 8), 0, st>>>(Hinv, L.ldh, Dlt, L.ldh, nI, done);
     count_launches(1);
+    ctx->hd_valid = false;
+    if (L.g == 1) { const int rc_d = build_hinv64(ctx, guarded); if (rc_d != OSSCAR_OK) return rc_d; }
     // (2) V = Hinv G_I on the tensor cores, then one refinement step with the residual G_I - H_II V in fp64
     float* GI = big;
     float* rV = big + nI * L.ldm;
@@ -526,10 +531,19 @@ int build_state(osscar_ctx* ctx, bool guarded)
         // (3) R_J = G_J - Hp[J, I] V, accumulated in fp64
         k_gather_rows<<<(unsigned)nJ, 256, 0, st>>>(ctx->G, L.m, L.g, perm, nI, R, L.ldm);
         CK(gemm_f64acc(st, nJ, L.m, nI, -1.0, Hp + nI * L.ldp, L.ldp, V, L.ldm, 1.0, R, L.ldm, R, L.ldm, false, done));
-        // (4) Pm = Hp[J, I] Hinv in fp64, then the Schur complements (fp64 dot products)
-        CK(gemm_f64acc(st, nJ, nI, nI, 1.0, Hp + nI * L.ldp, L.ldp, Hinv, L.ldh, 0.0, nullptr, 0, big, L.ldh, false, done));
-        k_schur<<<(unsigned)(L.ng - L.k), 256, 0, st>>>(Hp, L.ldp, big, L.ldh, nI, L.g, c);
-        count_launches(2);
+        // (4) Pm = Hp[J, I] Hinv kept in fp64, in panels of whole pruned groups that fit the scratch, then the Schur
+        // complements H_qq - Pm_q . H_qI as fp64 dot products
+        count_launches(1);
+        double* Pm = (double*)big;
+        const int64_t big_floats = (int64_t)((L.off_Hp - L.off_big) / sizeof(float));
+        int64_t gpp = (big_floats / 2) / (L.ldh * L.g);                 // pruned groups per panel
+        if (gpp < 1) return OSSCAR_E_WORKSPACE;
+        for (int64_t t0 = 0; t0 < L.ng - L.k; t0 += gpp) {
+            const int64_t ngr = L.ng - L.k - t0 < gpp ? L.ng - L.k - t0 : gpp;
+            CK(gemm_f64out(st, ngr * L.g, nI, nI, Hp + (nI + t0 * L.g) * L.ldp, L.ldp, Hinv, L.ldh, Pm, L.ldh, done));
+            k_schur<<<(unsigned)ngr, 256, 0, st>>>(Hp, L.ldp, Pm, L.ldh, nI, L.g, c, t0, done);
+            count_launches(1);
+        }
     }
     CK(cudaGetLastError());
     return OSSCAR_OK;

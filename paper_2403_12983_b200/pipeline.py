@@ -64,7 +64,7 @@ def solve_layer(solver: b.Solver, x_chunks: Sequence[torch.Tensor], W: torch.Ten
                 score_mode: int = b.SCORE_INDEPENDENT, accept_mode: int = b.ACCEPT_IMPROVING,
                 refresh_every: int = 0, profile_samples: int = 0, accept_rel_tol: float = -1.0,
                 H: Optional[torch.Tensor] = None, G: Optional[torch.Tensor] = None,
-                greedy_t_hat: int = 0, block_pairs: int = 0) -> LayerResult:
+                greedy_t_hat: int = 0, block_pairs: int = 0, loop_mode: int = b.LOOP_AUTO) -> LayerResult:
     """Prunes one layer to k groups of g rows.  W: d1 x m fp32 (device or host); x_chunks: row blocks of X
     (bf16 or fp32; all on the device, or all on the host).  block_pairs > 1 exchanges that many groups per iteration.  greedy_t_hat > 0 starts from the nested phase with
     that many groups pruned per iteration instead of the energy ranking."""
@@ -96,7 +96,7 @@ def solve_layer(solver: b.Solver, x_chunks: Sequence[torch.Tensor], W: torch.Ten
         support0, obj0 = solver.init_support(H, G, W, g, k, init_mode)
     ev[3].record()
     out = solver.local_search(max_swaps, score_mode, accept_mode, refresh_every, accept_rel_tol=accept_rel_tol,
-                              profile_samples=profile_samples, block_pairs=block_pairs)
+                              profile_samples=profile_samples, block_pairs=block_pairs, loop_mode=loop_mode)
     ev[4].record()
     ev[4].synchronize()
     names = ["gram", "gram_end", "init", "search"]

@@ -21,9 +21,9 @@ GAP = 1e-5      # relative best-vs-second-best gap above which the oracle's choi
 
 
 def blas_threads(H, g):
-    """Small problems (and the many g x g solves of multi-row groups) run faster on one BLAS thread than on a
-    pool that spins up for every tiny call; large single-row layers use every core."""
-    small = H.shape[0] <= 3000 or g > 1
+    """Small problems run faster on one BLAS thread than on a pool that spins up for every tiny call; large layers
+    use every core."""
+    small = H.shape[0] <= 3000
     return threadpool_limits(1) if small else contextlib.nullcontext()
 
 

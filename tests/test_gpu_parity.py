@@ -607,8 +607,8 @@ def test_guard_stop_when_every_candidate_is_dependent(solver, osscar, g, pairs):
 @pytest.mark.parametrize("name,over,seed,max_swaps", [
     SEARCH_CASES[0],                                                                  # 64 rows: fewer rows than blocks
     SEARCH_CASES[3],                                                                  # four / two rows per pass
-    ("c2", dict(n=8192, d1=2600, m=1100, k=1300, chunk_rows=4096), 0, 60),            # two rows and one row per pass
-    ("c5", dict(n=8192, d1=4200, m=2300, k=2100, chunk_rows=4096), 1, 40),            # one row per pass, two passes per row of V
+    ("c2", dict(n=8192, d1=2600, m=1100, k=1300, chunk_rows=4096), 0, 10),            # two rows and one row per pass
+    ("c5", dict(n=8192, d1=4200, m=2300, k=2100, chunk_rows=4096), 1, 8),            # one row per pass, two passes per row of V
 ])
 def test_persistent_loop_and_launch_chain_follow_the_oracle(solver, osscar, name, over, seed, max_swaps):
     """Single-row groups have two drivers: one cooperative kernel with grid-wide barriers, or five launches per step.
