@@ -28,7 +28,6 @@ import workloads  # noqa: E402
 
 METRIC = "swaps/s of the device-resident swap search (layer-solve seconds in ms_per_step)"
 UNIT = "swaps/s"
-CPU_SAMPLE = dict(n=4096, d1=2048, m=512, k=614, chunk_rows=4096)    # same value structure as c5, 1/14 of its width
 
 
 def peaks():
@@ -130,56 +129,165 @@ KERNEL_BYTES = {   # algorithmic bytes per launch of the streaming kernels of a 
 }
 
 
-# ------------------------------------------------------------------------------------------ reference arm (CPU oracle)
-def oracle_step(wl, max_swaps):
+# ------------------------------------------------------------------------------------------ CPU oracle legs
+def workload_label(wl, max_swaps, accept_always=False, greedy=0, block_pairs=0):
+    return (f"{wl.name}: d1={wl.d1} m={wl.m} g={wl.g} k={wl.k} n={wl.n} in {wl.n_chunks} chunks, "
+            f"max_swaps={max_swaps}, accept={'always' if accept_always else 'improving'} (eps {wl.eps_acc:g}), damp={wl.damp}, "
+            f"init={'greedy t_hat=%d' % greedy if greedy else 'energy'}"
+            + (f", block exchanges of {block_pairs} groups" if block_pairs > 1 else ""))
+
+
+def oracle_swaps_at_size(H, G, const, wl, n_swaps):
+    """Times the oracle's low-rank mode on a layer of the workload's own size: the fresh solve that starts it (set-up)
+    and `n_swaps` steps (propose + apply).  H, G are fp64 arrays of the full layer."""
     import numpy as np
     from oracle import osscar_oracle as orc
     t0 = time.perf_counter()
-    chunks = [c.float().numpy() for c in wl.x_chunks()]
-    W = wl.weight().numpy().astype(np.float64)
+    S0, _ = orc.init_support(H, wl.weight().numpy().astype(np.float64), wl.g, wl.k)
+    srch = orc.Search(H, G, const, wl.g, S0, mode="lowrank", eps_acc=wl.eps_acc, accept="always")
     t1 = time.perf_counter()
-    H, G, const = orc.gram_chunked(chunks, W, wl.damp)
+    per = []
+    for _ in range(n_swaps):
+        ts = time.perf_counter()
+        info = srch.propose()
+        if info is None:
+            break
+        srch.apply(info.slot, info.j_in)
+        per.append(time.perf_counter() - ts)
+    return {"setup_s": t1 - t0, "swap_s": per}
+
+
+def synthetic_spd_layer(wl, tokens=512):
+    """A full-width SPD H for the CPU legs that have no device: the Gram of `tokens` calibration rows plus the damping
+    term (full rank through the damping; the oracle's cost per swap does not depend on the values), and G = H W."""
+    import numpy as np
+    keep = wl.chunk_rows
+    wl.chunk_rows = tokens
+    X = wl.x_chunk(0).float().numpy().astype(np.float64)
+    wl.chunk_rows = keep
+    H = X.T @ X
+    H += max(wl.damp, 1e-2) * np.mean(np.diag(H)) * np.eye(wl.d1)
+    W = wl.weight().numpy().astype(np.float64)
+    G = H @ W
+    return H, G, float(np.sum(W * G))
+
+
+def strict_step_seconds(H, G, const, wl, steps, score_mode="independent"):
+    """Seconds per step of the strict oracle (fresh Cholesky solve per step) on fp64 H, G of a whole layer."""
+    import numpy as np
+    from oracle import osscar_oracle as orc
+    W = wl.weight().numpy().astype(np.float64)
     S0, _ = orc.init_support(H, W, wl.g, wl.k)
-    srch = orc.Search(H, G, const, wl.g, S0, mode="lowrank", eps_acc=wl.eps_acc)
-    t2 = time.perf_counter()
-    srch.run(max_swaps)
-    t3 = time.perf_counter()
-    return {"solve_s": t3 - t1, "search_s": t3 - t2, "swaps": len(srch.swap_trace), "gen_s": t1 - t0}
-
-
-def cpu_baseline(max_swaps=250):
-    wl = workloads.config("c5", **CPU_SAMPLE)
-    r = oracle_step(wl, max_swaps)
-    cores = torch.get_num_threads()
-    return {"value": r["swaps"] / max(r["search_s"], 1e-9), "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": (f"fp64 NumPy oracle (low-rank-update mode) on a c5-structured layer cut to d1={wl.d1}, m={wl.m}, "
-                       f"k={wl.k}, n={wl.n}: {r['swaps']} swaps in {r['search_s']:.2f} s, whole solve {r['solve_s']:.2f} s"),
-            "layer_solve_s": r["solve_s"]}
+    srch = orc.Search(H, G, const, wl.g, S0, mode="strict", score_mode=score_mode, accept="always")
+    per = []
+    for _ in range(steps):
+        ts = time.perf_counter()
+        info = srch.propose()
+        if info is None:
+            break
+        srch.apply(info.slot, info.j_in)
+        per.append(time.perf_counter() - ts)
+    return per
 
 
 def run_reference(args):
+    """The oracle as it stands, on the host cores, on the benchmark's own layer size: one step = one swap of its
+    low-rank mode (propose + apply) on a full-width layer; the fresh solve that starts it is set-up, outside the steps."""
     rank, world, _ = dist_env()
     if rank != 0:
         return
-    wl = workloads.config("c5", **CPU_SAMPLE)
-    for _ in range(args.warmup):
-        oracle_step(wl, 5)
-    tot, swaps, search = 0.0, 0, 0.0
-    for _ in range(args.steps):
-        r = oracle_step(wl, 40)
-        tot += r["solve_s"]; swaps += r["swaps"]; search += r["search_s"]
-    value = swaps / max(search, 1e-9)
+    wl = workloads.config(args.workload)
+    max_swaps = args.max_swaps if args.max_swaps is not None else wl.max_swaps
+    H, G, const = synthetic_spd_layer(wl)
+    r = oracle_swaps_at_size(H, G, const, wl, args.warmup + args.steps)
+    timed = r["swap_s"][args.warmup:]
+    tot = sum(timed)
+    value = len(timed) / max(tot, 1e-9)
     cores = torch.get_num_threads()
-    sample = (f"fp64 NumPy oracle on a c5-structured layer cut to d1={wl.d1}, m={wl.m}, k={wl.k}, n={wl.n}, "
-              f"at most 40 swaps per step")
+    sample = (f"fp64 NumPy oracle (low-rank-update mode) at the layer's own size d1={wl.d1}, m={wl.m}, k={wl.k}: one swap per step, "
+              f"{len(timed)} timed swaps after {args.warmup} warm-up swaps; H = Gram of 512 synthetic tokens + damping, G = H W; "
+              f"set-up (fresh fp64 solve) {r['setup_s']:.1f} s outside the steps")
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": 1e3 * tot / max(args.steps, 1), "higher_is_better": True,
+        "warmup": args.warmup, "ms_per_step": 1e3 * tot / max(len(timed), 1), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": "c5 (OPT-30B-shaped FC2) bounded sample: " + sample},
+        "config": {"workload": workload_label(wl, max_swaps)},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0}))
+
+
+def cpu_baseline_at_size(wl, H_dev, G_dev, const, n_swaps=3):
+    """The oracle on the host cores at the benchmark layer's own size, fed the device's H and G (fp32 -> fp64):
+    `n_swaps` steps of its low-rank mode after the fresh fp64 solve that starts it, plus the fp64 Gram of a slice of
+    one token chunk (the Gram is linear in tokens, so the slice scales to the layer)."""
+    import numpy as np
+    H = H_dev.cpu().numpy().astype(np.float64)
+    G = G_dev.cpu().numpy().astype(np.float64)
+    r = oracle_swaps_at_size(H, G, const, wl, n_swaps)
+    del H, G
+    rows = max(64, min(wl.chunk_rows, int(2.0e12 / (2.0 * wl.d1 * wl.d1))))        # about 2 TFLOP of fp64 work
+    keep = wl.chunk_rows
+    wl.chunk_rows = rows
+    X = wl.x_chunk(0).float().numpy().astype(np.float64)
+    wl.chunk_rows = keep
+    t0 = time.perf_counter()
+    Hs = X.T @ X
+    gram_s = time.perf_counter() - t0
+    del Hs, X
+    per = r["swap_s"]
+    s_per_swap = sum(per) / max(len(per), 1)
+    return {"value": 1.0 / max(s_per_swap, 1e-9), "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
+            "sample": (f"fp64 NumPy oracle (low-rank-update mode) at the layer's own size (d1={wl.d1}, m={wl.m}, k={wl.k}) on the device's H and G: "
+                       f"{len(per)} swaps, {s_per_swap:.2f} s per swap, after a fresh fp64 solve of the start state ({r['setup_s']:.1f} s, not counted)"),
+            "s_per_swap": s_per_swap, "setup_s": r["setup_s"],
+            "gram_fp64": {"rows": rows, "seconds": gram_s, "scale_to_layer": wl.n / rows,
+                          "layer_seconds_extrapolated": gram_s * wl.n / rows}}
+
+
+def other_configs(pkg, b, solver, dev, with_cpu):
+    """The other named layers, one warm-up and one timed solve each (outside the headline's timed region), and, with
+    `with_cpu`, seconds per step of the strict oracle (fresh Cholesky solve per step) on the device's H and G."""
+    import numpy as np
+    from threadpoolctl import threadpool_limits
+    import contextlib
+    out = {}
+    for name, strict_steps in (("c1", 4), ("c2", 1), ("c3", 2), ("c4", 2), ("c6", 4)):
+        wl = workloads.config(name)
+        W = wl.weight(dev)
+        x = [wl.x_chunk(c, dev) for c in range(wl.n_chunks)]
+        pair = wl.score_mode == "pair_exact"
+        kw = dict(damp=wl.damp, accept_rel_tol=wl.eps_acc, score_mode=b.SCORE_PAIR_EXACT if pair else b.SCORE_INDEPENDENT)
+        pkg.solve_layer(solver, x, W, wl.g, wl.k, wl.max_swaps, **kw)
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        f0.record()
+        r = pkg.solve_layer(solver, x, W, wl.g, wl.k, wl.max_swaps, **kw)
+        f1.record()
+        torch.cuda.synchronize()
+        nI, nJ = wl.k * wl.g, wl.d1 - wl.k * wl.g
+        fused = wl.g == 1 and not pair
+        loop_s = r.ms["search_loop"] * 1e-3
+        rec = {"workload": workload_label(wl, wl.max_swaps), "layer_solve_s": f0.elapsed_time(f1) / 1e3, "swaps": r.n_swaps,
+               "stop_reason": r.stop_reason, "phases_ms": r.ms, "loop_driver": r.loop_driver,
+               "swaps_per_s": r.n_swaps / max(loop_s, 1e-9) if r.n_swaps else 0.0,
+               "loop_gbs": swap_bytes(nI, nJ, wl.m, fused) * r.n_swaps / max(loop_s, 1e-9) / 1e9 if r.n_swaps else 0.0}
+        if name == "c3":        # no improving swap from the energy start: the paper's fixed-iteration form gives the step time
+            rf = pkg.solve_layer(solver, x, W, wl.g, wl.k, 8, accept_mode=b.ACCEPT_ALWAYS, **kw)
+            rec["forced_swaps"] = {"swaps": rf.n_swaps, "ms_per_swap": rf.ms["search_loop"] / max(rf.n_swaps, 1)}
+        if with_cpu:
+            H64 = r.H.cpu().numpy().astype(np.float64); G64 = r.G.cpu().numpy().astype(np.float64)
+            ctxm = threadpool_limits(1) if wl.d1 <= 3000 else contextlib.nullcontext()
+            with ctxm:
+                per = strict_step_seconds(H64, G64, r.const_term, wl, strict_steps, "pair_exact" if pair else "independent")
+            rec["cpu_strict_oracle"] = {"steps": len(per), "s_per_step": sum(per) / max(len(per), 1),
+                                        "cores": 1 if wl.d1 <= 3000 else torch.get_num_threads(),
+                                        "what": "strict fp64 oracle (fresh Cholesky solve per step) on the device's H and G"}
+            del H64, G64
+        out[name] = rec
+        del x, W, r
+        torch.cuda.empty_cache()
+    return out
 
 
 # ------------------------------------------------------------------------------------------ our arm
@@ -236,11 +344,9 @@ def run_ours(args):
     swaps = 0
     e0.record()
     for _ in range(args.steps):
-        res = step(x_dev, W, prof=8)
+        res = step(x_dev, W)
         for key in phase:
             phase[key] += res.ms[key]
-        for key, val in res.ms_kernel.items():
-            kern[key] = kern.get(key, 0.0) + val
         swaps += res.n_swaps
     e1.record()
     barrier()
@@ -248,6 +354,11 @@ def run_ours(args):
     clocks = sampler.stop()
     total_ms = e0.elapsed_time(e1)
     K = max(args.steps, 1)
+    # phase / kernel times of a step come from one more solve outside the timed region (the launch-chain driver records
+    # events around sampled steps; the persistent loop reads the device clock at its barriers)
+    prof_res = step(x_dev, W, prof=8)
+    for key, val in prof_res.ms_kernel.items():
+        kern[key] = val * K
 
     # ---------------- the same layer with the paper's larger local-search steps (outside the timed region above)
     block_extra = None
@@ -315,15 +426,24 @@ def run_ours(args):
     shares = {k2: v * per_step_swaps / max(args.block_pairs, 1) for k2, v in kern_avg.items()}
     shares["gram_tcgen05"] = phase["gram"] / K
     dom = max(shares, key=shares.get) if shares else "gram_tcgen05"
-    # dram bytes / algorithmic bytes measured with ncu on a mid-size case (profiles/swap_step_g1_kernels_mid_size.md);
-    # traffic grows in proportion to the rows streamed, so the ratio carries over to a full-size launch
-    traffic_ratio = {"l1_hpass_update_v": 1.010, "l2_update_r_swap": 0.915, "l4_update_hinv_y": 0.793}
-    if dom in KERNEL_BYTES and kern_avg.get(dom, 0) > 0:
+    fused_path = wl.g == 1 and wl.score_mode != "pair_exact" and args.block_pairs <= 1
+    loop_ms = phase["search_loop"] / K
+    if fused_path and loop_ms > 0 and loop_ms >= phase["gram"] / K:
+        # the swap loop is the dominant kernel: one cooperative launch per solve (or its five-launch-per-step form),
+        # timed by the library with CUDA events on its own stream around the loop
+        persistent = res.loop_driver == "persistent"
+        bytes_per_launch = swap_bytes(nI, nJ, m, True) * (swaps / K)
+        ach = bytes_per_launch / (loop_ms * 1e-3) / 1e9
+        roof = {"kernel": "k_swap_loop_g1 (persistent cooperative loop, one launch per solve)" if persistent
+                          else "swap loop as five launches per step (k_decide_g1, k_l1_g1, k_l2_g1, k_select_in_g1, k_l4_g1)",
+                "bound": "hbm", "achieved": ach, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": ach / pk["hbm_gbs"],
+                "traffic": None, "bytes_per_launch": int(bytes_per_launch), "ms_per_launch": loop_ms,
+                "bytes_per_swap": swap_bytes(nI, nJ, m, True), "peak_source": pk["source"]}
+    elif dom in KERNEL_BYTES and kern_avg.get(dom, 0) > 0:
         bytes_per_launch = KERNEL_BYTES[dom](nI, nJ, m)
         ach = bytes_per_launch / (kern_avg[dom] * 1e-3) / 1e9
         roof = {"kernel": dom, "bound": "hbm", "achieved": ach, "peak": pk["hbm_gbs"], "unit": "GB/s",
-                "frac": ach / pk["hbm_gbs"],
-                "traffic": int(traffic_ratio[dom] * bytes_per_launch) if dom in traffic_ratio else None,
+                "frac": ach / pk["hbm_gbs"], "traffic": None,
                 "bytes_per_launch": bytes_per_launch,
                 "ms_per_launch": kern_avg[dom], "peak_source": pk["source"]}
     else:
@@ -348,13 +468,11 @@ def run_ours(args):
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32 (bf16 tensor-core Gram, fp32 accumulate)" if wl.x_dtype == torch.bfloat16
                  else "f32 (Gram as a three-term bf16 split on the tensor cores, fp32 accumulate)", "data": "synthetic",
-        "config": {"workload": f"{wl.name}: d1={wl.d1} m={wl.m} g={wl.g} k={wl.k} n={wl.n} in {wl.n_chunks} chunks, "
-                               f"max_swaps={max_swaps}, accept={'always' if args.accept_always else 'improving'} (eps {wl.eps_acc:g}), damp={wl.damp}, "
-                               f"init={'greedy t_hat=%d' % args.greedy if args.greedy else 'energy'}"
-                               + (f", block exchanges of {args.block_pairs} groups" if args.block_pairs > 1 else ""),
-                   "l2": "inputs larger than L2 (X, H and the search state are each > 126 MB)" if wl.d1 >= 8192 else
-                         "state smaller than L2; numbers are cache-resident",
-                   "replicas": world},
+        "config": {"workload": workload_label(wl, max_swaps, args.accept_always, args.greedy, args.block_pairs),
+                   },
+        "notes": {"l2": "inputs larger than L2 (X, H and the search state are each > 126 MB)" if wl.d1 >= 8192 else
+                        "state smaller than L2; numbers are cache-resident",
+                  "replicas": world, "loop_driver": res.loop_driver},
         "clocks": clocks,
         "layer_solve_s": ms_step / 1e3,
         "swaps_per_step": per_step_swaps, "stop_reason": res.stop_reason,
@@ -372,15 +490,17 @@ def run_ours(args):
     }
     if e2e and "ms_per_step" in e2e:
         e_val = red["sum_e2e_swaps"] / max(min(K, 2), 1) / max(red["max_e2e_ms"] * 1e-3, 1e-9)
-        out["e2e"] = {"value": e_val, "unit": "swaps per second of whole-solve time, host buffers", "ms_per_step": red["max_e2e_ms"],
+        out["e2e"] = {"value": e_val, "unit": UNIT, "what": "swaps per second of whole-solve time, host buffers", "ms_per_step": red["max_e2e_ms"],
                       "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"]}
     else:
         out["e2e"] = {"value": None, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0,
                       "note": (e2e or {}).get("error", "skipped")}
     if block_extra:
         out["block_exchange"] = block_extra
+    if world == 1 and not args.no_other_configs and args.workload == "c5":
+        out["other_configs"] = other_configs(pkg, b, solver, dev, with_cpu=not args.no_cpu)
     if world == 1 and not args.no_cpu:
-        out["cpu_baseline"] = cpu_baseline()
+        out["cpu_baseline"] = cpu_baseline_at_size(wl, H, G, res.const_term)
     print(json.dumps(out))
     if world > 1:
         torch.distributed.destroy_process_group()
@@ -405,6 +525,7 @@ def main():
     ap.add_argument("--loop-mode", type=int, default=0, help="0 auto, 1 persistent cooperative loop, 2 five launches per step (single-row groups)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-other-configs", action="store_true", help="skip the extra solves of c1, c2, c3, c4 and c6")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

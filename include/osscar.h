@@ -50,9 +50,10 @@ enum { OSSCAR_INIT_ENERGY = 0, OSSCAR_INIT_MAGNITUDE = 1, OSSCAR_INIT_USER = 2 }
 enum { OSSCAR_SCORE_INDEPENDENT = 0, OSSCAR_SCORE_PAIR_EXACT = 1 };
 enum { OSSCAR_ACCEPT_IMPROVING = 0, OSSCAR_ACCEPT_ALWAYS = 1 };
 enum { OSSCAR_STOP_MAX_SWAPS = 0, OSSCAR_STOP_NO_IMPROVEMENT = 1, OSSCAR_STOP_GUARD = 2 };
-/* Swap loop of single-row groups: AUTO picks PERSISTENT when the device can hold the cooperative grid;
- * PERSISTENT = one cooperative kernel that runs all steps with bounded grid-wide barriers between their phases;
- * LAUNCHES = five dependent launches per step, enqueued ahead of the device. */
+/* Swap loop of single-row groups.  PERSISTENT = one cooperative kernel that runs all steps with bounded grid-wide
+ * barriers between their phases (OSSCAR_E_ARG if the device cannot launch cooperatively); LAUNCHES = five dependent
+ * launches per step, enqueued ahead of the device; AUTO = PERSISTENT for states that fit the L2 cache (under 96 MB),
+ * LAUNCHES for states streamed from HBM. */
 enum { OSSCAR_LOOP_AUTO = 0, OSSCAR_LOOP_PERSISTENT = 1, OSSCAR_LOOP_LAUNCHES = 2 };
 
 #define OSSCAR_MAX_GROUP 96   /* largest supported group size g */
@@ -167,6 +168,7 @@ typedef struct {
     float   ms_search;               /* device time of the swap loop                         */
     int32_t n_profiled;              /* steps that were timed kernel by kernel and did a swap */
     float   ms_kernel[OSSCAR_NUM_STEP_KERNELS]; /* mean device time of each kernel over those steps */
+    int32_t loop_driver;             /* OSSCAR_LOOP_PERSISTENT or OSSCAR_LOOP_LAUNCHES: what drove the loop  */
 } osscar_search_result;
 
 /*

@@ -36,7 +36,7 @@ class SearchParams(C.Structure):
 class SearchResult(C.Structure):
     _fields_ = [("n_swaps", C.c_int32), ("stop_reason", C.c_int32), ("n_refresh", C.c_int32), ("status", C.c_int32),
                 ("obj_init", C.c_double), ("obj_final", C.c_double), ("ms_search", C.c_float),
-                ("n_profiled", C.c_int32), ("ms_kernel", C.c_float * 12)]
+                ("n_profiled", C.c_int32), ("ms_kernel", C.c_float * 12), ("loop_driver", C.c_int32)]
 
 
 STEP_KERNELS = ["select", "pair_grams", "y_pass", "small_algebra", "staging", "h_pass", "update_hinv", "update_v",
@@ -149,6 +149,7 @@ class SearchOutput:
     obj_final: float
     ms_search: float
     ms_kernel: dict              # mean device ms per kernel of a step over the profiled steps ({} if none)
+    loop_driver: str = "launches"  # "persistent" (one cooperative kernel) or "launches"
 
 
 class Solver:
@@ -306,7 +307,7 @@ class Solver:
                             STOP_NAMES.get(res.stop_reason, str(res.stop_reason)), res.n_refresh,
                             res.obj_init, res.obj_final, res.ms_search,
                             {n: res.ms_kernel[i] for i, n in enumerate(STEP_KERNELS_BLOCK if block_pairs > 1 else STEP_KERNELS_G1 if g == 1 else STEP_KERNELS)}
-                            if res.n_profiled > 0 else {})
+                            if res.n_profiled > 0 else {}, "persistent" if res.loop_driver == LOOP_PERSISTENT else "launches")
 
     def objective(self, H, W, Wt) -> float:
         _dev_f32(H, "H"); _dev_f32(W, "W"); _dev_f32(Wt, "Wt")

@@ -1056,7 +1056,13 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
     BlockPtrs bp = make_block_ptrs(ctx, bs);
     const bool fast = g == 1 && !pair && !block;  // fused step for single-row groups
     // one cooperative kernel for the whole loop, unless asked otherwise or the device cannot hold such a grid
-    const int pgrid = (fast && prm->loop_mode != OSSCAR_LOOP_LAUNCHES && L.nJ > 0) ? persistent_grid(L) : 0;
+    // AUTO: the cooperative loop for states that stay in L2 (its barriers cost less than five launches per step: 2-8 x
+    // the swaps per second measured on the small layers); the launch chain for states streamed from HBM, where four
+    // resident blocks per SM of one-row kernels keep more loads in flight than the loop's blocks do (measured 0.81
+    // against 0.71 of copy bandwidth on the OPT-30B-shaped FC2 layer)
+    const double state_bytes = 8.0 * L.nI * L.ldh + 4.0 * (L.nI + L.nJ) * L.ldm + 4.0 * L.nJ * L.ldh;
+    const bool want_persistent = prm->loop_mode == OSSCAR_LOOP_PERSISTENT || (prm->loop_mode == OSSCAR_LOOP_AUTO && state_bytes <= 96.0e6);
+    const int pgrid = (fast && want_persistent && L.nJ > 0) ? persistent_grid(L) : 0;
     if (prm->loop_mode == OSSCAR_LOOP_PERSISTENT && pgrid == 0) return OSSCAR_E_ARG;
     const bool persistent = pgrid > 0;
     if (block) max_swaps /= bs;                   // from here on: iterations
@@ -1292,6 +1298,7 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
     res->obj_init = ctx->ctl_host->acc[2];
     res->obj_final = ctx->ctl_host->acc[3];
     res->ms_search = ms;
+    res->loop_driver = persistent ? OSSCAR_LOOP_PERSISTENT : OSSCAR_LOOP_LAUNCHES;
     // kernel times of the sampled steps that really swapped (a stopped loop runs empty kernels)
     int used = 0;
     for (int i = 0; i < nprof; ++i) {

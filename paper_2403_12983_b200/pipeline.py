@@ -105,6 +105,7 @@ def solve_layer(solver: b.Solver, x_chunks: Sequence[torch.Tensor], W: torch.Ten
     res = LayerResult(out.support, out.W, out.obj_trace, out.swap_trace, out.n_swaps, out.stop_reason,
                       out.obj_init, out.obj_final, const, ms, out.ms_kernel, H, G)
     res.io = io
+    res.loop_driver = out.loop_driver
     return res
 
 

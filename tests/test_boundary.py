@@ -29,7 +29,7 @@ def test_struct_layouts_match_header():
     assert ctypes.sizeof(b.SearchParams) == 48
     assert b.SearchParams.accept_rel_tol.offset == 16 and b.SearchParams.loop_mode.offset == 32
     assert b.SearchParams.wait_limit_cycles.offset == 40
-    assert ctypes.sizeof(b.SearchResult) == 88
+    assert ctypes.sizeof(b.SearchResult) == 96 and b.SearchResult.loop_driver.offset == 88
     assert b.SearchResult.obj_init.offset == 16 and b.SearchResult.ms_search.offset == 32
 
 
