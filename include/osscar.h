@@ -70,6 +70,27 @@ int osscar_destroy(osscar_ctx* ctx);
  * kernel makes, while giving up, for its own copies and tensor-core work in flight keep the default budget. */
 int osscar_set_wait_limit(osscar_ctx* ctx, uint64_t cycles);
 
+/*
+ * Column shards (Section 2, convolutional-layer paragraph: the outputs of two filters are independent given the
+ * kept set, so the columns of W_hat -- and with them G, the optimal weights and the residual -- split across devices).
+ * A context that has a reduce hook holds the columns [c0, c0 + m) of one layer: it is given its own m columns of
+ * W_hat and G and the whole of H.  The kept set, (H_II)^-1, the slot-permuted H and the Schur complements are then
+ * replicated (every shard computes the same values), while the row norms of the weights and of the residual, the
+ * cross term of the chosen pair, the group energies and the objective are sums over columns: the library leaves each
+ * shard's partial sums in a buffer inside the caller's workspace and calls
+ *     reduce(user, dev_buf, count, dtype, cuda_stream)        dtype: OSSCAR_FP32 or OSSCAR_FP64 (doubles)
+ * from the host thread of the API call, in stream order; the hook must enqueue on `cuda_stream` an in-place sum of
+ * dev_buf over all shards (ncclAllReduce, or torch.distributed.all_reduce on a view of the workspace) and return 0.
+ * Two calls per swap (one double; d1 floats), none of them synchronises the host.  Every shard must make the same
+ * calls in the same order.  Supported: single-row groups (g = 1), OSSCAR_SCORE_INDEPENDENT, one swap per step,
+ * OSSCAR_INIT_ENERGY / MAGNITUDE / USER; anything else returns OSSCAR_E_ARG while a hook is set.  Results: support and
+ * traces are identical on every shard, W_out holds the shard's columns, objectives are those of the whole layer.
+ * fn = NULL removes the hook.
+ */
+typedef int (*osscar_reduce_fn)(void* user, void* dev_buf, int64_t count, int dtype, void* cuda_stream);
+enum { OSSCAR_FP64 = 2 };
+int osscar_set_shard_reduce(osscar_ctx* ctx, osscar_reduce_fn fn, void* user);
+
 /* Scratch needed by init_support / local_search / objective for a layer of this shape.
  * The caller allocates it on the device (256-byte aligned) and lends it with set_workspace;
  * it must stay alive, and untouched by others, from init_support to the end of local_search. */

@@ -12,7 +12,7 @@ from . import build as _build
 
 OK = 0
 E_ARG, E_SHAPE, E_NOTPD, E_WORKSPACE, E_CUDA, E_TIMEOUT, E_STATE = -1, -2, -3, -4, -5, -6, -7
-BF16, FP32 = 0, 1
+BF16, FP32, FP64 = 0, 1, 2
 GRAM_BEGIN, GRAM_END = 1, 2
 INIT_ENERGY, INIT_MAGNITUDE, INIT_USER = 0, 1, 2
 SCORE_INDEPENDENT, SCORE_PAIR_EXACT = 0, 1
@@ -24,7 +24,7 @@ LOOP_AUTO, LOOP_PERSISTENT, LOOP_LAUNCHES = 0, 1, 2
 EXPORTS = ["osscar_create", "osscar_destroy", "osscar_workspace_bytes", "osscar_set_workspace",
            "osscar_gram", "osscar_init_support", "osscar_local_search", "osscar_objective",
            "osscar_debug_get_state", "osscar_status_string", "osscar_launch_count", "osscar_trace_noalloc", "osscar_init_support_greedy", "osscar_gram_cross", "osscar_set_const_term",
-           "osscar_set_wait_limit"]
+           "osscar_set_wait_limit", "osscar_set_shard_reduce"]
 
 
 class SearchParams(C.Structure):
@@ -46,6 +46,10 @@ STEP_KERNELS_G1 = ["decide", "l1_hpass_update_v", "l2_update_r_swap", "select_in
 # block exchanges (block_pairs > 1): stages of one iteration
 STEP_KERNELS_BLOCK = ["select", "gather_y", "grams_algebra_staging", "h_pass", "update_hinv", "update_v", "update_r",
                       "update_c_fix", "h_swap", "scores"]
+
+
+# int reduce(void* user, void* dev_buf, int64_t count, int dtype, void* cuda_stream)
+REDUCE_FN = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_void_p, C.c_int64, C.c_int, C.c_void_p)
 
 
 class OsscarError(RuntimeError):
@@ -84,6 +88,7 @@ def lib() -> C.CDLL:
     L.osscar_gram_cross.argtypes = [vp, vp, C.c_int, vp, C.c_int, i64, i64, i64, C.c_int, C.c_float, vp, vp, C.POINTER(C.c_double)]
     L.osscar_set_const_term.argtypes = [vp, C.c_double, C.c_int]
     L.osscar_set_wait_limit.argtypes = [vp, C.c_uint64]
+    L.osscar_set_shard_reduce.argtypes = [vp, REDUCE_FN, vp]
     L.osscar_local_search.argtypes = [vp, C.POINTER(SearchParams), vp, vp, vp, vp, C.POINTER(SearchResult)]
     L.osscar_objective.argtypes = [vp, vp, vp, vp, i64, i64, C.POINTER(C.c_double)]
     L.osscar_debug_get_state.argtypes = [vp, C.c_int, vp]
@@ -253,6 +258,32 @@ class Solver:
     def set_wait_limit(self, cycles: int):
         """Budget (SM cycles) of every bounded device-side wait of this context's kernels; 0 = default."""
         _check(lib().osscar_set_wait_limit(self._h, int(cycles)), "osscar_set_wait_limit")
+
+    def set_shard_reduce(self, fn):
+        """Column shards: `fn(view, stream_ptr)` must enqueue, on the CUDA stream with that handle, an in-place sum over all
+        shards of `view`, a 1-D tensor (float32 or float64) that aliases the partial sums inside this solver's
+        workspace.  None removes the hook.  The workspace must be set before the calls that use the hook."""
+        if fn is None:
+            self._reduce_cb = None
+            _check(lib().osscar_set_shard_reduce(self._h, C.cast(None, REDUCE_FN), None), "osscar_set_shard_reduce")
+            return
+
+        def trampoline(_user, buf, count, dtype, stream):
+            try:
+                ws = self._ws
+                off = int(buf) - ws.data_ptr()
+                tdt, width = (torch.float64, 8) if dtype == FP64 else (torch.float32, 4)
+                if off < 0 or off + count * width > ws.numel():
+                    return 1
+                fn(ws[off:off + count * width].view(tdt), int(stream) if stream else 0)
+                return 0
+            except Exception:          # an exception must not unwind through the C caller
+                import traceback
+                traceback.print_exc()
+                return 1
+
+        self._reduce_cb = REDUCE_FN(trampoline)       # kept alive as long as the context may call it
+        _check(lib().osscar_set_shard_reduce(self._h, self._reduce_cb, None), "osscar_set_shard_reduce")
 
     def set_const_term(self, value: float, enabled: bool = True):
         _check(lib().osscar_set_const_term(self._h, float(value), int(enabled)), "osscar_set_const_term")

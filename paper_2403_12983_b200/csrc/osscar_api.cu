@@ -153,6 +153,15 @@ int osscar_set_wait_limit(osscar_ctx* ctx, uint64_t cycles)
     return OSSCAR_OK;
 }
 
+int osscar_set_shard_reduce(osscar_ctx* ctx, osscar_reduce_fn fn, void* user)
+{
+    if (!ctx) return OSSCAR_E_ARG;
+    ctx->reduce = fn;
+    ctx->reduce_user = fn ? user : nullptr;
+    ctx->have_state = false;
+    return OSSCAR_OK;
+}
+
 int osscar_workspace_bytes(int64_t d1, int64_t m, int32_t g, int32_t k, size_t* bytes)
 {
     if (!bytes) return OSSCAR_E_ARG;
@@ -318,6 +327,7 @@ int osscar_init_support(osscar_ctx* ctx, const float* H, const float* G, const f
     const int rc0 = make_layout(d1, m, g, k, &L);
     if (rc0 != OSSCAR_OK) return rc0;
     if (!ctx->ws || ctx->ws_bytes < L.bytes) return OSSCAR_E_WORKSPACE;
+    if (ctx->reduce && g != 1) return OSSCAR_E_ARG;             // column shards: single-row groups only
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return OSSCAR_E_CUDA;
     ctx->L = L; ctx->H = H; ctx->G = G; ctx->W = W; ctx->have_state = false;
@@ -351,6 +361,7 @@ int osscar_init_support_greedy(osscar_ctx* ctx, const float* H, const float* G, 
     const int rc0 = make_layout(d1, m, g, k, &L);
     if (rc0 != OSSCAR_OK) return rc0;
     if (t_hat < 1 || (int64_t)t_hat * g > 256) return OSSCAR_E_SHAPE;
+    if (ctx->reduce) return OSSCAR_E_ARG;                       // the nested phase is not sharded
     if (!ctx->ws || ctx->ws_bytes < L.bytes) return OSSCAR_E_WORKSPACE;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return OSSCAR_E_CUDA;
@@ -384,6 +395,8 @@ int osscar_local_search(osscar_ctx* ctx, const osscar_search_params* params,
     if (params->loop_mode < OSSCAR_LOOP_AUTO || params->loop_mode > OSSCAR_LOOP_LAUNCHES || params->wait_limit_cycles > (uint64_t)1 << 62) return OSSCAR_E_ARG;
     if (!ctx->have_state) return OSSCAR_E_STATE;
     if (params->score_mode == OSSCAR_SCORE_PAIR_EXACT && ctx->L.nJ > 0 && ctx->L.pair_capacity == 0) return OSSCAR_E_SHAPE;
+    if (ctx->reduce && (ctx->L.g != 1 || params->score_mode != OSSCAR_SCORE_INDEPENDENT || params->block_pairs > 1 ||
+                        params->loop_mode == OSSCAR_LOOP_PERSISTENT)) return OSSCAR_E_ARG;      // what column shards support
     if (params->block_pairs > 1) {      // block exchanges: independent scores, s <= min(k, pruned groups), s g rows fit the panels
         const osscar::Layout& L = ctx->L;
         const int64_t s = params->block_pairs;

@@ -53,6 +53,7 @@ struct Layout {
     size_t off_vec_begin, off_vec_end;   // the staged vectors (zeroed once when the state is built)
     size_t off_vnorm, off_rnorm, off_D, off_A, off_c, off_small, off_gramV, off_gramR;
     size_t off_perm, off_slotof, off_energy, off_panel;
+    size_t off_shard;                                                  // column shards: partial sums handed to the reduce hook
     size_t off_loop;                                                   // persistent swap loop: per-block candidates, phase timers
     size_t off_pairCinv, off_pairKK, off_pairScratch, off_pairDelta;   // PAIR_EXACT scoring
     size_t off_greedy;                                                 // scratch of the nested (greedy) phase
@@ -100,6 +101,8 @@ struct osscar_ctx {
     double user_const;
     long long wait_limit;            // context default of SearchCtl::wait_limit
     bool hd_valid;                   // the fp64 copy of the inverse matches the state
+    osscar_reduce_fn reduce;         // column shards: in-place sum over shards, enqueued by the caller's hook (or null)
+    void* reduce_user;
 };
 
 namespace osscar {
@@ -173,5 +176,7 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* p, int32_t* support_
 cudaError_t score_pass(osscar_ctx* ctx);   // full scoring pass from the current state (fills D, A)
 // fp64 copy of the inverse from the fp32 one by a Newton-Schulz step summed in fp64 (single-row groups; uses `big`)
 int build_hinv64(osscar_ctx* ctx, bool guarded);
+// column shards: sum `count` values of `buf` (inside the workspace) over all shards through the context's hook
+int shard_reduce(osscar_ctx* ctx, void* buf, int64_t count, int dtype);
 
 }  // namespace osscar

@@ -40,6 +40,7 @@ __device__ __forceinline__ float dot4f(const float4& a, const float4& b) {
 struct Ptrs {
     float *Hp, *Hinv, *V, *R, *y, *b, *u2, *bC, *u2c, *u, *d, *K, *Vq, *vnorm, *rnorm;
     double *D, *A, *c, *small, *gramV, *gramR;
+    double *shard;                                           // column shards: partial sums handed to the reduce hook
     double *Hd;                                              // fp64 copy of the inverse (single-row groups, independent scores)
     double *pairCinv, *pairKK, *pairScratch, *pairDelta;     // PAIR_EXACT scoring
     int32_t *perm, *slotof;
@@ -808,6 +809,7 @@ __global__ void k_begin(SearchCtl* ctl, double* obj_trace, int32_t* done_host)
 }
 __global__ void k_count_refresh(SearchCtl* ctl) { if (!ctl->done) ctl->n_refresh += 1; }
 __global__ void k_search_wait_limit(SearchCtl* ctl, long long cycles) { ctl->wait_limit = cycles; }
+__global__ void k_shard_scalar(SearchCtl* ctl, double* sh, int back) { if (back) ctl->acc[1] = sh[0]; else sh[0] = ctl->acc[1]; }
 __global__ void k_final_obj(SearchCtl* ctl) { ctl->acc[3] = ctl->const_term - ctl->acc[1]; }
 
 // ------------------------------------------------------------------ exhaustive pair scoring (PAIR_EXACT)
@@ -938,7 +940,7 @@ Ptrs make_ptrs(osscar_ctx* ctx)
     p.vnorm = (float*)(ws + L.off_vnorm); p.rnorm = (float*)(ws + L.off_rnorm);
     p.D = (double*)(ws + L.off_D); p.A = (double*)(ws + L.off_A); p.c = (double*)(ws + L.off_c);
     p.small = (double*)(ws + L.off_small); p.gramV = (double*)(ws + L.off_gramV); p.gramR = (double*)(ws + L.off_gramR);
-    p.Hd = (double*)(ws + L.off_Hd);
+    p.Hd = (double*)(ws + L.off_Hd); p.shard = (double*)(ws + L.off_shard);
     p.perm = (int32_t*)(ws + L.off_perm); p.slotof = (int32_t*)(ws + L.off_slotof);
     p.pairCinv = (double*)(ws + L.off_pairCinv); p.pairKK = (double*)(ws + L.off_pairKK);
     p.pairScratch = (double*)(ws + L.off_pairScratch); p.pairDelta = (double*)(ws + L.off_pairDelta);
@@ -1019,11 +1021,19 @@ int build_hinv64(osscar_ctx* ctx, bool guarded)
     return OSSCAR_OK;
 }
 
+int shard_reduce(osscar_ctx* ctx, void* buf, int64_t count, int dtype)
+{
+    if (!ctx->reduce) return OSSCAR_OK;
+    if (cudaGetLastError() != cudaSuccess) return OSSCAR_E_CUDA;
+    return ctx->reduce(ctx->reduce_user, buf, count, dtype, (void*)ctx->stream) == 0 ? OSSCAR_OK : OSSCAR_E_CUDA;
+}
+
 cudaError_t score_pass(osscar_ctx* ctx)
 {
     Ptrs p = make_ptrs(ctx);
     cudaError_t e = enqueue_scores(ctx, p, true);
     if (e != cudaSuccess) return e;
+    if (ctx->reduce && shard_reduce(ctx, p.vnorm, ctx->L.d1, OSSCAR_FP32) != OSSCAR_OK) return cudaErrorUnknown;   // row norms are sums over columns
     k_select<<<1, 1024, 0, ctx->stream>>>(p);      // also leaves the score vectors D and A readable
     count_launches(1);
     return cudaGetLastError();
@@ -1046,6 +1056,7 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
     CK(cudaGetLastError());
     CK(cudaEventRecord(ctx->ev0, st));
     const bool pair = prm->score_mode == OSSCAR_SCORE_PAIR_EXACT;
+    const bool sharded = ctx->reduce != nullptr;          // column shards: sums over shards go through the caller's hook
     const int bs = prm->block_pairs > 1 ? prm->block_pairs : 1;     // groups exchanged per iteration
     const bool block = bs > 1;
     if (block) {
@@ -1061,13 +1072,15 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
     // resident blocks per SM of one-row kernels keep more loads in flight than the loop's blocks do (measured 0.81
     // against 0.71 of copy bandwidth on the OPT-30B-shaped FC2 layer)
     const double state_bytes = 8.0 * L.nI * L.ldh + 4.0 * (L.nI + L.nJ) * L.ldm + 4.0 * L.nJ * L.ldh;
-    const bool want_persistent = prm->loop_mode == OSSCAR_LOOP_PERSISTENT || (prm->loop_mode == OSSCAR_LOOP_AUTO && state_bytes <= 96.0e6);
+    const bool want_persistent = sharded ? false : prm->loop_mode == OSSCAR_LOOP_PERSISTENT || (prm->loop_mode == OSSCAR_LOOP_AUTO && state_bytes <= 96.0e6);
     const int pgrid = (fast && want_persistent && L.nJ > 0) ? persistent_grid(L) : 0;
     if (prm->loop_mode == OSSCAR_LOOP_PERSISTENT && pgrid == 0) return OSSCAR_E_ARG;
     const bool persistent = pgrid > 0;
     if (block) max_swaps /= bs;                   // from here on: iterations
     const int64_t npairs = (int64_t)L.k * (L.ng - L.k);
+    if (sharded && !(g == 1 && !pair && !block)) return OSSCAR_E_ARG;
     if (max_swaps > 0) CK(enqueue_scores(ctx, p, true, pair));
+    if (max_swaps > 0 && sharded && shard_reduce(ctx, p.vnorm, L.d1, OSSCAR_FP32) != OSSCAR_OK) return OSSCAR_E_CUDA;
     const size_t inv_smem = ((size_t)g * g + 2 * (size_t)g) * sizeof(double);      // matrix under inversion + pivot row/column
     if (inv_smem > 48 * 1024) {
         CK(cudaFuncSetAttribute(k_small, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)inv_smem));
@@ -1175,7 +1188,9 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
             const int bi = it / batch;
             if (bi >= 2) {      // stay at most two batches ahead of the device, and stop feeding a finished loop
                 if (cudaEventSynchronize(evb[bi & 1]) != cudaSuccess) { rc = OSSCAR_E_CUDA; break; }
-                if (*ctx->done_flag_host) break;
+                // the loop's state at the end of batch bi - 2, copied in stream order: unlike the live flag, every shard
+                // of a column-sharded layer reads the same value here, so all of them stop feeding at the same step
+                if (ctx->done_flag_host[1 + (bi & 1)]) break;
             }
         }
         if (prm->refresh_every > 0 && it > 0 && it % prm->refresh_every == 0) {
@@ -1184,6 +1199,7 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
             k_count_refresh<<<1, 1, 0, st>>>(ctx->ctl);
             count_launches(1);
             if (enqueue_scores(ctx, p, true, pair) != cudaSuccess) { rc = OSSCAR_E_CUDA; break; }
+            if (sharded && shard_reduce(ctx, p.vnorm, L.d1, OSSCAR_FP32) != OSSCAR_OK) { rc = OSSCAR_E_CUDA; break; }
             if (fast && bootstrap_g1() != cudaSuccess) { rc = OSSCAR_E_CUDA; break; }
         }
         cudaEvent_t* pe = nullptr;
@@ -1193,11 +1209,25 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
         mark();
         if (block) {
             if (enqueue_block_step(ctx, p, bp, prm->accept_mode, tol, obj_trace, swap_trace, mark) != cudaSuccess) { rc = OSSCAR_E_CUDA; break; }
+        } else if (fast && sharded) {
+            // column shards: the same five launches, with the two sums over shards where a decision needs them --
+            // the cross term of the chosen pair before the accept test, the row norms before the next scores
+            const unsigned nbV = (unsigned)((L.nI + G1_RB - 1) / G1_RB), nbR = (unsigned)((L.nJ + G1_RB - 1) / G1_RB), nbH = nbR + 1;
+            k_decide_g1<<<1, 1024, 0, st>>>(p, prm->accept_mode, tol, obj_trace, swap_trace, 1);
+            if (shard_reduce(ctx, p.shard, 1, OSSCAR_FP64) != OSSCAR_OK) { rc = OSSCAR_E_CUDA; break; }
+            k_decide_g1<<<1, 1024, 0, st>>>(p, prm->accept_mode, tol, obj_trace, swap_trace, 2);   mark();
+            k_l1_g1<<<nbV + nbH, 256, 0, st>>>(p, nbV);                                          mark();
+            k_l2_g1<<<nbR + 32, 256, 0, st>>>(p, nbR);                                           mark();
+            if (shard_reduce(ctx, p.vnorm, L.d1, OSSCAR_FP32) != OSSCAR_OK) { rc = OSSCAR_E_CUDA; break; }
+            k_scores_sharded_g1<<<(unsigned)((L.d1 + 255) / 256), 256, 0, st>>>(p);
+            k_select_in_g1<<<1, 1024, 0, st>>>(p);                                               mark();
+            k_l4_g1<G1_RB4><<<(unsigned)((L.nI + G1_RB4 - 1) / G1_RB4), 256, 0, st>>>(p);        mark();
+            count_launches(7);
         } else if (fast) {
             // single-row groups: decide, {H pass || V}, {R || slot exchange}, next entering group, {Hinv + next y}
             // G1_RB rows per block; the H pass has one more block for the leaving row
             const unsigned nbV = (unsigned)((L.nI + G1_RB - 1) / G1_RB), nbR = (unsigned)((L.nJ + G1_RB - 1) / G1_RB), nbH = nbR + 1;
-            k_decide_g1<<<1, 1024, 0, st>>>(p, prm->accept_mode, tol, obj_trace, swap_trace);   mark();
+            k_decide_g1<<<1, 1024, 0, st>>>(p, prm->accept_mode, tol, obj_trace, swap_trace, 0);   mark();
             k_l1_g1<<<nbV + nbH, 256, 0, st>>>(p, nbV);                                          mark();
             k_l2_g1<<<nbR + 32, 256, 0, st>>>(p, nbR);                                           mark();
             k_select_in_g1<<<1, 1024, 0, st>>>(p);                                               mark();
@@ -1256,6 +1286,8 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
         if (pe) nmarks = slot;
         if (cudaGetLastError() != cudaSuccess) { rc = OSSCAR_E_CUDA; break; }
         if ((it + 1) % batch == 0) {
+            if (cudaMemcpyAsync((void*)(ctx->done_flag_host + 1 + ((it / batch) & 1)), &ctx->ctl->done, sizeof(int32_t),
+                                cudaMemcpyDeviceToHost, st) != cudaSuccess) { rc = OSSCAR_E_CUDA; break; }
             if (cudaEventRecord(evb[(it / batch) & 1], st) != cudaSuccess) { rc = OSSCAR_E_CUDA; break; }
         }
     }
@@ -1282,6 +1314,12 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
         // G_I in slot order, then Tr(G_I^T V)
         CK(gather_rows(st, ctx->G, L.m, L.g, p.perm, 0, L.nI, big, L.ldm));
         CK(trace_product(st, big, L.ldm, p.V, L.ldm, L.nI, L.m, ctx->partials, &ctx->ctl->acc[1]));
+        if (sharded) {      // Tr(G_I^T V) is a sum over this shard's columns
+            k_shard_scalar<<<1, 1, 0, st>>>(ctx->ctl, p.shard, 0);
+            if (shard_reduce(ctx, p.shard, 1, OSSCAR_FP64) != OSSCAR_OK) return OSSCAR_E_CUDA;
+            k_shard_scalar<<<1, 1, 0, st>>>(ctx->ctl, p.shard, 1);
+            count_launches(2);
+        }
         k_final_obj<<<1, 1, 0, st>>>(ctx->ctl);
         count_launches(3);
     }

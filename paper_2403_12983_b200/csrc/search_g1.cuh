@@ -36,6 +36,26 @@ __global__ void k_scores_g1(Ptrs p)
     }
 }
 
+// Column shards: after the row norms of V' and R' have been summed over shards, the scores of the new state.  The
+// inverse has not been updated yet (that pass needs the next entering group, which these scores decide), so its new
+// diagonal comes from the rank-two formula, as in the row update's own epilogue.
+__global__ void k_scores_sharded_g1(Ptrs p)
+{
+    if (p.ctl->done) return;
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const double Cinv = p.small[S_CINV], c1inv = p.small[S_C1INV];
+    if (i < p.nI) {
+        const double bs = p.b[i], us = p.u2[i];
+        const double hd = i == p.ctl->sel_slot ? c1inv : p.Hd[i * p.ldh + i] - bs * bs * Cinv + us * us * c1inv;
+        p.D[i] = hd > 0.0 ? (double)p.vnorm[i] / hd : INFINITY;
+    } else if (i < p.nI + p.nJ) {
+        const int64_t t = i - p.nI;
+        const double cc = p.c[t];
+        const double hd = p.Hp[(p.nI + t) * p.ldp + p.nI + t];
+        p.A[t] = cc > kAddPivotTol * hd ? (double)p.rnorm[t] / cc : -INFINITY;
+    }
+}
+
 // Block-wide arg-min of val[i] (ties -> smaller group id); result broadcast through shared memory.
 __device__ void block_argmin(const double* __restrict__ val, const int32_t* __restrict__ ids, int n, bool negate,
                              double* best_out, int* idx_out)
@@ -92,27 +112,39 @@ __global__ void __launch_bounds__(1024) k_select_in_g1(Ptrs p)
 }
 
 // One block: leaving row, exact change of obj, accept test, traces, staged vectors.
+// part 0: the whole decision; column shards run it in two parts around the sum of the cross term over shards:
+// part 1 picks the leaving row and leaves this shard's V_r . R_q in p.shard[0], part 2 continues from the summed value.
 __global__ void __launch_bounds__(1024)
-k_decide_g1(Ptrs p, int accept_mode, double accept_tol, double* __restrict__ obj_trace, int32_t* __restrict__ swap_trace)
+k_decide_g1(Ptrs p, int accept_mode, double accept_tol, double* __restrict__ obj_trace, int32_t* __restrict__ swap_trace, int part)
 {
     SearchCtl* ctl = p.ctl;
     if (ctl->done) return;
     __shared__ float redf[32];
     __shared__ int s_stop;
-    double Dbest; int slot;
-    block_argmin(p.D, p.perm, p.k, false, &Dbest, &slot);
+    double Dbest = 0.0; int slot;
+    if (part == 2) slot = ctl->sel_slot;
+    else {
+        block_argmin(p.D, p.perm, p.k, false, &Dbest, &slot);
+        if (slot < 0 || !isfinite(Dbest)) {
+            if (threadIdx.x == 0) { ctl->done = 1; ctl->stop_reason = OSSCAR_STOP_GUARD; *p.done_host = 1; }
+            return;
+        }
+    }
     const int64_t t = ctl->sel_t;
-    if (slot < 0 || !isfinite(Dbest)) {
-        if (threadIdx.x == 0) { ctl->done = 1; ctl->stop_reason = OSSCAR_STOP_GUARD; *p.done_host = 1; }
+    const int64_t r0 = slot;
+    double GX;
+    if (part == 2) GX = p.shard[0];
+    else {          // cross term V_r . R_q
+        const float4* vr = reinterpret_cast<const float4*>(p.V + r0 * p.ldm);
+        const float4* rq = reinterpret_cast<const float4*>(p.R + t * p.ldm);
+        float acc = 0.f;
+        for (int64_t c = threadIdx.x; c < p.ldm / 4; c += blockDim.x) acc += dot4(vr[c], rq[c]);
+        GX = (double)block_sum_f(acc, redf);
+    }
+    if (part == 1) {
+        if (threadIdx.x == 0) { ctl->sel_slot = slot; p.shard[0] = GX; }
         return;
     }
-    const int64_t r0 = slot;
-    // cross term V_r . R_q
-    const float4* vr = reinterpret_cast<const float4*>(p.V + r0 * p.ldm);
-    const float4* rq = reinterpret_cast<const float4*>(p.R + t * p.ldm);
-    float acc = 0.f;
-    for (int64_t c = threadIdx.x; c < p.ldm / 4; c += blockDim.x) acc += dot4(vr[c], rq[c]);
-    const double GX = (double)block_sum_f(acc, redf);
     if (threadIdx.x == 0) {
         const double C = p.Hd[r0 * p.ldh + r0], P = p.y[r0], cq = p.c[t];
         const double GV = p.vnorm[r0], GR = p.rnorm[t];

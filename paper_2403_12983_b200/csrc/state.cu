@@ -302,6 +302,12 @@ __global__ void k_add_sym(float* __restrict__ A, int64_t lda, const float* __res
     }
 }
 
+// acc[0], acc[1] -> sh[0], sh[1] (back = 0) or back again (back = 1)
+__global__ void k_pack2(SearchCtl* ctl, double* sh, int back)
+{
+    if (back) { ctl->acc[0] = sh[0]; ctl->acc[1] = sh[1]; } else { sh[0] = ctl->acc[0]; sh[1] = ctl->acc[1]; }
+}
+
 __global__ void k_set_obj(SearchCtl* ctl)   // obj = const - Tr(G_I^T V), with acc[0] = const, acc[1] = trace
 {
     ctl->const_term = ctl->acc[0];
@@ -377,8 +383,9 @@ int make_layout(int64_t d1, int64_t m, int32_t g, int32_t k, Layout* L)
     L->off_K = take(sizeof(float) * g * ldm);
     L->off_Vq = take(sizeof(float) * g * ldm);
     L->off_vec_end = off;
-    L->off_vnorm = take(sizeof(float) * nI);
-    L->off_rnorm = take(sizeof(float) * (nJ > 0 ? nJ : 1));
+    L->off_vnorm = take(sizeof(float) * (nI + nJ + 1));      // row norms of V, then of R: one buffer of d1 floats (shards sum it)
+    L->off_rnorm = L->off_vnorm + sizeof(float) * nI;
+    L->off_shard = take(sizeof(double) * 8);
     L->off_D = take(sizeof(double) * k);
     L->off_A = take(sizeof(double) * (ng - k > 0 ? ng - k : 1));
     L->off_c = take(sizeof(double) * (ng - k > 0 ? ng - k : 1) * g * g);
@@ -434,6 +441,7 @@ int select_support(osscar_ctx* ctx, int mode, int32_t* support)
         count_launches(1);
     } else {
         k_energy<<<(unsigned)L.ng, 128, 0, st>>>(ctx->H, ctx->W, L.d1, L.m, L.g, mode, e);
+        if (ctx->reduce) { const int rr = shard_reduce(ctx, e, L.ng, OSSCAR_FP64); if (rr != OSSCAR_OK) return rr; }   // energies are sums over columns
         k_rank_select<<<nb, 256, 0, st>>>(e, L.ng, L.k, kept);
     }
     k_build_perm<<<nb, 256, 0, st>>>(kept, L.ng, L.k, perm, slotof, support);
@@ -525,6 +533,15 @@ int build_state(osscar_ctx* ctx, bool guarded)
     if (ctx->have_const) CK(set_device_double(st, &ctx->ctl->acc[0], ctx->user_const));
     else CK(trace_product(st, ctx->W, L.m, ctx->G, L.m, L.d1, L.m, ctx->partials, &ctx->ctl->acc[0]));
     CK(trace_product(st, GI, L.ldm, V, L.ldm, nI, L.m, ctx->partials, &ctx->ctl->acc[1]));
+    if (ctx->reduce) {      // both traces are sums over this shard's columns (a constant given by the caller is the layer's)
+        double* sh = (double*)(ws + L.off_shard);
+        k_pack2<<<1, 1, 0, st>>>(ctx->ctl, sh, 0);
+        const int rr = shard_reduce(ctx, sh, 2, OSSCAR_FP64);
+        if (rr != OSSCAR_OK) return rr;
+        k_pack2<<<1, 1, 0, st>>>(ctx->ctl, sh, 1);
+        if (ctx->have_const) CK(set_device_double(st, &ctx->ctl->acc[0], ctx->user_const));
+        count_launches(2);
+    }
     k_set_obj<<<1, 1, 0, st>>>(ctx->ctl);
     count_launches(1);
     if (nJ > 0) {
