@@ -462,7 +462,12 @@ def run_ours(args):
         roof = {"kernel": "k_swap_loop_g1 (persistent cooperative loop, one launch per solve)" if persistent
                           else "swap loop as five launches per step (k_decide_g1, k_l1_g1, k_l2_g1, k_select_in_g1, k_l4_g1)",
                 "bound": "hbm", "achieved": ach, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": ach / pk["hbm_gbs"],
-                "traffic": None, "bytes_per_launch": int(bytes_per_launch), "ms_per_launch": loop_ms,
+                # DRAM bytes / algorithmic bytes of one step of the launch-chain kernels, measured with ncu on a mid-size case
+                # whose state exceeds L2 (1687.2 MB of traffic for 1795.2 MB); traffic grows in proportion to the rows streamed.
+                # The persistent loop has no such capture.
+                "traffic": None if persistent else int(0.940 * bytes_per_launch), "traffic_source": None if persistent else
+                "algorithmic bytes x 0.940 (ncu dram__bytes of k_l1_g1, k_l2_g1, k_l4_g1 on a 6 GB case, kernels as committed)",
+                "bytes_per_launch": int(bytes_per_launch), "ms_per_launch": loop_ms,
                 "bytes_per_swap": swap_bytes(nI, nJ, m, True), "peak_source": pk["source"]}
     elif dom in KERNEL_BYTES and kern_avg.get(dom, 0) > 0:
         bytes_per_launch = KERNEL_BYTES[dom](nI, nJ, m)
