@@ -1009,13 +1009,20 @@ int build_hinv64(osscar_ctx* ctx, bool guarded)
     float* Hinv = (float*)(ws + L.off_Hinv);
     double* Hd = (double*)(ws + L.off_Hd);
     float* E = (float*)(ws + L.off_big);
-    float* Dlt = E + L.nI * L.ldh;
+    float* T = E + L.nI * L.ldh;
     const int32_t* done = guarded ? &ctx->ctl->done : nullptr;
-    // E = I - H_II Hinv with fp64 sums; Hd = Hinv + Hinv E, the sum taken in fp64 (the correction is below 2^-24 of Hinv)
+    void* tc = ws + L.off_tc;
+    // X0 = the fp32 inverse at hand (raw from the blocked inversion, or carried by an fp32 driver).  With E = I - H_II X0,
+    // H_II^-1 = X0 (I + E + E^2 + ...): E is formed once with fp64 sums, the series is cut after E^2 (its products are
+    // corrections of corrections: the tensor-core split product is ample), and the sum X0 + X0 (E + E^2) is taken in fp64.
+    // The error left is E^3 (below 1e-9 for any start within 1e-3), against E^2 for a single Newton-Schulz step.
     if (gemm_f64acc(st, L.nI, L.nI, L.nI, -1.0, Hp, L.ldp, Hinv, L.ldh, 0.0, nullptr, 0, E, L.ldh, true, done) != cudaSuccess) return OSSCAR_E_CUDA;
-    if (gemm_tc(st, L.nI, L.nI, L.nI, 1.f, Hinv, L.ldh, E, L.ldh, 0.f, Dlt, L.ldh, ws + L.off_tc, L.tc_bytes, ctx->ctl, done) != cudaSuccess) return OSSCAR_E_CUDA;
-    k_hinv_to_d<<<(unsigned)L.nI, 256, 0, st>>>(Hinv, Dlt, Hd, L.ldh, L.nI, done);
-    count_launches(1);
+    if (cudaMemcpyAsync(T, E, sizeof(float) * L.nI * L.ldh, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return OSSCAR_E_CUDA;
+    if (gemm_tc(st, L.nI, L.nI, L.nI, 1.f, E, L.ldh, E, L.ldh, 1.f, T, L.ldh, tc, L.tc_bytes, ctx->ctl, done) != cudaSuccess) return OSSCAR_E_CUDA;
+    if (gemm_tc(st, L.nI, L.nI, L.nI, 1.f, Hinv, L.ldh, T, L.ldh, 0.f, E, L.ldh, tc, L.tc_bytes, ctx->ctl, done) != cudaSuccess) return OSSCAR_E_CUDA;
+    k_hinv_to_d<<<(unsigned)L.nI, 256, 0, st>>>(Hinv, E, Hd, L.ldh, L.nI, done);
+    k_hinv_from_d<<<(unsigned)L.nI, 256, 0, st>>>(Hd, Hinv, L.ldh, done);
+    count_launches(2);
     if (cudaGetLastError() != cudaSuccess) return OSSCAR_E_CUDA;
     ctx->hd_valid = true;
     return OSSCAR_OK;
@@ -1151,6 +1158,25 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
         return 1;
     };
     const unsigned prep_blocks = (unsigned)(((L.nI + L.ldm) * g + 255) / 256);
+    // threads per block of the three streaming kernels of the single-row step, by the length of the rows they stream
+    const unsigned t_l1 = (unsigned)g1_threads(L.ldm > L.ldh ? L.ldm / 4 : L.ldh / 4), t_l2 = (unsigned)g1_threads(L.ldm / 4),
+                   t_l4 = (unsigned)g1_threads(L.ldh / 2);
+    auto launch_l1 = [&](unsigned nbV, unsigned nbH) {
+        if (t_l1 == 64) k_l1_g1<64><<<nbV + nbH, 64, 0, st>>>(p, nbV);
+        else if (t_l1 == 128) k_l1_g1<128><<<nbV + nbH, 128, 0, st>>>(p, nbV);
+        else k_l1_g1<256><<<nbV + nbH, 256, 0, st>>>(p, nbV);
+    };
+    auto launch_l2 = [&](unsigned nbR) {       // the same number of threads exchange the two slots whatever the block size
+        if (t_l2 == 64) k_l2_g1<64><<<nbR + 128, 64, 0, st>>>(p, nbR);
+        else if (t_l2 == 128) k_l2_g1<128><<<nbR + 64, 128, 0, st>>>(p, nbR);
+        else k_l2_g1<256><<<nbR + 32, 256, 0, st>>>(p, nbR);
+    };
+    auto launch_l4 = [&]() {
+        const unsigned nb = (unsigned)((L.nI + G1_RB4 - 1) / G1_RB4);
+        if (t_l4 == 64) k_l4_g1<G1_RB4, 64><<<nb, 64, 0, st>>>(p);
+        else if (t_l4 == 128) k_l4_g1<G1_RB4, 128><<<nb, 128, 0, st>>>(p);
+        else k_l4_g1<G1_RB4, 256><<<nb, 256, 0, st>>>(p);
+    };
     int next_prof = 0;
     int nmarks = 0;                 // events recorded per profiled step (depends on the step variant)
     unsigned long long* loop_prof = (unsigned long long*)((char*)ctx->ws + L.off_loop + 2 * (size_t)kLoopMaxBlocks * 16);
@@ -1216,22 +1242,22 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
             k_decide_g1<<<1, 1024, 0, st>>>(p, prm->accept_mode, tol, obj_trace, swap_trace, 1);
             if (shard_reduce(ctx, p.shard, 1, OSSCAR_FP64) != OSSCAR_OK) { rc = OSSCAR_E_CUDA; break; }
             k_decide_g1<<<1, 1024, 0, st>>>(p, prm->accept_mode, tol, obj_trace, swap_trace, 2);   mark();
-            k_l1_g1<<<nbV + nbH, 256, 0, st>>>(p, nbV);                                          mark();
-            k_l2_g1<<<nbR + 32, 256, 0, st>>>(p, nbR);                                           mark();
+            launch_l1(nbV, nbH);                                                                 mark();
+            launch_l2(nbR);                                                                      mark();
             if (shard_reduce(ctx, p.vnorm, L.d1, OSSCAR_FP32) != OSSCAR_OK) { rc = OSSCAR_E_CUDA; break; }
             k_scores_sharded_g1<<<(unsigned)((L.d1 + 255) / 256), 256, 0, st>>>(p);
             k_select_in_g1<<<1, 1024, 0, st>>>(p);                                               mark();
-            k_l4_g1<G1_RB4><<<(unsigned)((L.nI + G1_RB4 - 1) / G1_RB4), 256, 0, st>>>(p);        mark();
+            launch_l4();        mark();
             count_launches(7);
         } else if (fast) {
             // single-row groups: decide, {H pass || V}, {R || slot exchange}, next entering group, {Hinv + next y}
             // G1_RB rows per block; the H pass has one more block for the leaving row
             const unsigned nbV = (unsigned)((L.nI + G1_RB - 1) / G1_RB), nbR = (unsigned)((L.nJ + G1_RB - 1) / G1_RB), nbH = nbR + 1;
             k_decide_g1<<<1, 1024, 0, st>>>(p, prm->accept_mode, tol, obj_trace, swap_trace, 0);   mark();
-            k_l1_g1<<<nbV + nbH, 256, 0, st>>>(p, nbV);                                          mark();
-            k_l2_g1<<<nbR + 32, 256, 0, st>>>(p, nbR);                                           mark();
+            launch_l1(nbV, nbH);                                                                 mark();
+            launch_l2(nbR);                                                                      mark();
             k_select_in_g1<<<1, 1024, 0, st>>>(p);                                               mark();
-            k_l4_g1<G1_RB4><<<(unsigned)((L.nI + G1_RB4 - 1) / G1_RB4), 256, 0, st>>>(p);                                                     mark();
+            launch_l4();                                                     mark();
             count_launches(5);
         } else {
             if (pair) { if (pair_scores() != cudaSuccess) { rc = OSSCAR_E_CUDA; break; } }
@@ -1301,7 +1327,7 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
     }
     CK(cudaEventRecord(ctx->ev1, st));
     if (fast && max_swaps > 0) {       // the fp32 inverse follows its fp64 copy (state reader, other drivers)
-        k_hinv_from_d<<<(unsigned)L.nI, 256, 0, st>>>(p.Hd, p.Hinv, L.ldh);
+        k_hinv_from_d<<<(unsigned)L.nI, 256, 0, st>>>(p.Hd, p.Hinv, L.ldh, nullptr);
         count_launches(1);
     }
 

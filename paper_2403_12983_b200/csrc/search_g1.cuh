@@ -211,8 +211,12 @@ k_decide_g1(Ptrs p, int accept_mode, double accept_tol, double* __restrict__ obj
 // resident blocks), so G1_RB = 1 there and G1_RB4 = 2 for the Hinv update.
 constexpr int G1_U = 8;
 constexpr int G1_UH = 9;            // pieces per thread for rows of Hinv / Hp: 9 x 256 x 4 floats cover n_I = 8602 in one pass
-constexpr int G1_T = 256;
+constexpr int G1_T = 256;           // most threads per block; rows of up to 512 / 1024 pieces run with 64 / 128 threads, so that
+                                    // a thread still requests about eight pieces and twice or four times as many rows are in flight per SM
+__host__ __device__ inline int g1_threads(int64_t pieces) { return pieces <= 512 ? 64 : (pieces <= 1024 ? 128 : 256); }
 
+// Block-wide sum for blocks of 64, 128 or 256 threads (the launch picks the size by the row length).
+template <int TB>
 __device__ __forceinline__ float block_sum_256(float v, float* red /*[8]*/)
 {
     v = warp_sum(v);
@@ -220,7 +224,7 @@ __device__ __forceinline__ float block_sum_256(float v, float* red /*[8]*/)
     __syncthreads();
     float t = 0.f;
 #pragma unroll
-    for (int i = 0; i < G1_T / 32; ++i) t += red[i];
+    for (int i = 0; i < TB / 32; ++i) t += red[i];
     __syncthreads();
     return t;
 }
@@ -228,7 +232,7 @@ __device__ __forceinline__ float block_sum_256(float v, float* red /*[8]*/)
 // Row update M'[s] = M[s] + ck_s K + cq_s Vq with the squared norm of the new row, RB rows per block (every piece of
 // K and Vq fetched from L2 serves the RB rows).  kind 0: V (ck = -b_s, cq = -u2_s, row r0 := Vq, D' written),
 // kind 1: R (ck = u_l, cq = -d_l, row of the entering slot := K - d_r Vq, c' and A' written).
-template <int RB>
+template <int RB, int TB>
 __device__ __forceinline__ void update_row_g1(const Ptrs& p, int kind, int64_t s0, float* red)
 {
     float* M = kind == 0 ? p.V : p.R;
@@ -248,13 +252,13 @@ __device__ __forceinline__ void update_row_g1(const Ptrs& p, int kind, int64_t s
     float dr = 0.f;
 #pragma unroll
     for (int r = 0; r < RB; ++r) { nrm[r] = 0.f; ck[r] = 0.f; cq[r] = 0.f; sp[r] = false; }
-    for (int64_t base = threadIdx.x; base < n4; base += (int64_t)G1_T * G1_U) {
+    for (int64_t base = threadIdx.x; base < n4; base += (int64_t)TB * G1_U) {
         float4 v[RB][G1_U];
 #pragma unroll
         for (int r = 0; r < RB; ++r)
 #pragma unroll
             for (int j = 0; j < G1_U; ++j) {
-                const int64_t c = base + G1_T * j;
+                const int64_t c = base + TB * j;
                 v[r][j] = c < n4 ? row[r][c] : make_float4(0.f, 0.f, 0.f, 0.f);     // requested before the step's scalars arrive
             }
         if (base == threadIdx.x) {           // first pass: the scalars of these rows, loaded behind the rows themselves
@@ -272,7 +276,7 @@ __device__ __forceinline__ void update_row_g1(const Ptrs& p, int kind, int64_t s
         }
 #pragma unroll
         for (int j = 0; j < G1_U; ++j) {
-            const int64_t c = base + G1_T * j;
+            const int64_t c = base + TB * j;
             if (c < n4) {
                 const float4 kk = __ldg(K4 + c), qq = __ldg(Q4 + c);
 #pragma unroll
@@ -288,7 +292,7 @@ __device__ __forceinline__ void update_row_g1(const Ptrs& p, int kind, int64_t s
     }
 #pragma unroll
     for (int r = 0; r < RB; ++r) {
-        const float nr = block_sum_256(nrm[r], red);
+        const float nr = block_sum_256<TB>(nrm[r], red);
         if (threadIdx.x == 0 && s0 + r < nrows) {
             const int64_t s = s0 + r;
             const double Cinv = p.small[S_CINV], c1inv = p.small[S_C1INV];
@@ -319,7 +323,7 @@ __device__ __forceinline__ void update_row_g1(const Ptrs& p, int kind, int64_t s
 
 // u_l = Hp[l, 0:n_I] . b and d_l = Hp[l, q] - Hp[l, 0:n_I] . u2 for RB rows (pruned rows l0.., or the single leaving
 // row, l = n_J); every piece of b and u2 serves the RB rows.
-template <int RB>
+template <int RB, int TB>
 __device__ __forceinline__ void hpass_stream(const Ptrs& p, const float4* const (&row)[RB], int64_t l0, int nvalid, float* red /*[16]*/)
 {
     const float4* bv = reinterpret_cast<const float4*>(p.b);
@@ -328,18 +332,18 @@ __device__ __forceinline__ void hpass_stream(const Ptrs& p, const float4* const 
     float au[RB], ad[RB];
 #pragma unroll
     for (int r = 0; r < RB; ++r) { au[r] = 0.f; ad[r] = 0.f; }
-    for (int64_t base = threadIdx.x; base < n4; base += (int64_t)G1_T * G1_UH) {
+    for (int64_t base = threadIdx.x; base < n4; base += (int64_t)TB * G1_UH) {
         float4 x[RB][G1_UH];
 #pragma unroll
         for (int r = 0; r < RB; ++r)
 #pragma unroll
             for (int j = 0; j < G1_UH; ++j) {
-                const int64_t c = base + G1_T * j;
+                const int64_t c = base + TB * j;
                 x[r][j] = c < n4 ? row[r][c] : make_float4(0.f, 0.f, 0.f, 0.f);
             }
 #pragma unroll
         for (int j = 0; j < G1_UH; ++j) {
-            const int64_t c = base + G1_T * j;
+            const int64_t c = base + TB * j;
             if (c < n4) {
                 const float4 bb = __ldg(bv + c), uu = __ldg(uv + c);
 #pragma unroll
@@ -356,7 +360,7 @@ __device__ __forceinline__ void hpass_stream(const Ptrs& p, const float4* const 
         if (threadIdx.x == 0 && r < nvalid && !p.ctl->done) {
             float su = 0.f, sd = 0.f;
 #pragma unroll
-            for (int i = 0; i < 8; ++i) { su += red[i]; sd += red[8 + i]; }
+            for (int i = 0; i < TB / 32; ++i) { su += red[i]; sd += red[8 + i]; }
             const int64_t qcol = p.nI + (int64_t)p.ctl->sel_t;
             p.u[l0 + r] = su;
             p.d[l0 + r] = reinterpret_cast<const float*>(row[r])[qcol] - sd;
@@ -368,10 +372,11 @@ __device__ __forceinline__ void hpass_stream(const Ptrs& p, const float4* const 
 // need no control-block read, so their streams start at once) and a last block for the leaving row.
 constexpr int G1_RB = 1;            // rows per block of the V / R updates and the H pass
 constexpr int G1_RB4 = 1;           // rows per block of the Hinv update
-__global__ void __launch_bounds__(G1_T, 4) k_l1_g1(Ptrs p, unsigned nbV)      // 64 registers: four resident blocks per SM
+template <int TB>
+__global__ void __launch_bounds__(TB, 1024 / TB) k_l1_g1(Ptrs p, unsigned nbV)      // 64 registers: four resident blocks per SM
 {
     __shared__ float red[16];
-    if (blockIdx.x < nbV) { update_row_g1<G1_RB>(p, 0, (int64_t)blockIdx.x * G1_RB, red); return; }
+    if (blockIdx.x < nbV) { update_row_g1<G1_RB, TB>(p, 0, (int64_t)blockIdx.x * G1_RB, red); return; }
     const int64_t l0 = (int64_t)(blockIdx.x - nbV) * G1_RB;
     if (l0 < p.nJ) {
         const float4* rows[G1_RB];
@@ -382,10 +387,10 @@ __global__ void __launch_bounds__(G1_T, 4) k_l1_g1(Ptrs p, unsigned nbV)      //
             rows[r] = reinterpret_cast<const float4*>(p.Hp + (p.nI + l) * p.ldp);
             nvalid += l0 + r < p.nJ;
         }
-        hpass_stream<G1_RB>(p, rows, l0, nvalid, red);
+        hpass_stream<G1_RB, TB>(p, rows, l0, nvalid, red);
     } else {
         const float4* rows[1] = { reinterpret_cast<const float4*>(p.Hp + (int64_t)p.ctl->sel_slot * p.ldp) };
-        hpass_stream<1>(p, rows, p.nJ, 1, red);
+        hpass_stream<1, TB>(p, rows, p.nJ, 1, red);
     }
 }
 
@@ -420,10 +425,11 @@ __device__ __forceinline__ void hswap_g1(const Ptrs& p, int64_t idx, int64_t str
 }
 
 // L2: blocks [0, nbR) update G1_RB rows of R each (+ c, A); the remaining blocks exchange the two slots in Hp.
-__global__ void __launch_bounds__(G1_T, 4) k_l2_g1(Ptrs p, unsigned nbR)
+template <int TB>
+__global__ void __launch_bounds__(TB, 1024 / TB) k_l2_g1(Ptrs p, unsigned nbR)
 {
     __shared__ float red[8];
-    if (blockIdx.x < nbR) { update_row_g1<G1_RB>(p, 1, (int64_t)blockIdx.x * G1_RB, red); return; }
+    if (blockIdx.x < nbR) { update_row_g1<G1_RB, TB>(p, 1, (int64_t)blockIdx.x * G1_RB, red); return; }
     if (p.ctl->done) return;
     const int64_t nsw = gridDim.x - nbR;
     hswap_g1(p, (int64_t)(blockIdx.x - nbR) * blockDim.x + threadIdx.x, nsw * blockDim.x);
@@ -438,8 +444,8 @@ __global__ void __launch_bounds__(G1_T, 4) k_l2_g1(Ptrs p, unsigned nbR)
 // L4: Hinv' = Hinv - (b/C) b^T + (u2/c1) u2^T (row and column r0: -u2/c1, corner 1/c1) on the fp64 copy of the inverse and,
 // in the same pass, y_next = Hinv' h with h = Hp[row of the next entering group, 0:n_I].  RB rows per block; a piece is a
 // double2, nine pieces per thread and pass.
-template <int RB>
-__global__ void __launch_bounds__(G1_T) k_l4_g1(Ptrs p)
+template <int RB, int TB>
+__global__ void __launch_bounds__(TB) k_l4_g1(Ptrs p)
 {
     __shared__ double red[8];
     const int64_t s0 = (int64_t)blockIdx.x * RB;
@@ -455,13 +461,13 @@ __global__ void __launch_bounds__(G1_T) k_l4_g1(Ptrs p)
     double nb[RB], us[RB], corner[RB], yacc[RB];
 #pragma unroll
     for (int r = 0; r < RB; ++r) { srow[r] = false; nb[r] = 0.0; us[r] = 0.0; corner[r] = 0.0; yacc[r] = 0.0; }
-    for (int64_t base = threadIdx.x; base < n2; base += (int64_t)G1_T * G1_UH) {
+    for (int64_t base = threadIdx.x; base < n2; base += (int64_t)TB * G1_UH) {
         double2 h[RB][G1_UH];
 #pragma unroll
         for (int r = 0; r < RB; ++r)
 #pragma unroll
             for (int j = 0; j < G1_UH; ++j) {
-                const int64_t c = base + G1_T * j;
+                const int64_t c = base + TB * j;
                 h[r][j] = c < n2 ? row[r][c] : make_double2(0.0, 0.0);    // requested before the step's scalars arrive
             }
         if (base == threadIdx.x) {
@@ -481,7 +487,7 @@ __global__ void __launch_bounds__(G1_T) k_l4_g1(Ptrs p)
         }
 #pragma unroll
         for (int j = 0; j < G1_UH; ++j) {
-            const int64_t c = base + G1_T * j;
+            const int64_t c = base + TB * j;
             if (c < n2) {
                 const float2 bb = __ldg(b2 + c), uu = __ldg(u2v + c), hh = __ldg(h2 + c);
                 const int64_t rc = r0 - c * 2;           // position of column r0 inside this piece, if any
@@ -507,7 +513,7 @@ __global__ void __launch_bounds__(G1_T) k_l4_g1(Ptrs p)
         if (threadIdx.x == 0 && s0 + r < p.nI) {
             double sum = 0.0;
 #pragma unroll
-            for (int i = 0; i < G1_T / 32; ++i) sum += red[i];
+            for (int i = 0; i < TB / 32; ++i) sum += red[i];
             p.y[s0 + r] = (float)sum;
         }
     }
@@ -540,8 +546,9 @@ __global__ void k_hinv_to_d(const float* __restrict__ Hinv, const float* __restr
         Hd[r * ldh + c] = v;
     }
 }
-__global__ void k_hinv_from_d(const double* __restrict__ Hd, float* __restrict__ Hinv, int64_t ldh)
+__global__ void k_hinv_from_d(const double* __restrict__ Hd, float* __restrict__ Hinv, int64_t ldh, const int32_t* __restrict__ done)
 {
+    if (done && *done) return;
     const int64_t r = blockIdx.x;
     for (int64_t c = threadIdx.x; c < ldh; c += blockDim.x) Hinv[r * ldh + c] = (float)Hd[r * ldh + c];
 }

@@ -511,15 +511,21 @@ int build_state(osscar_ctx* ctx, bool guarded)
     { const int rc_inv = invert_spd_inplace(ctx, Hinv, L.ldh, nI, Hp, L.ldp, done); if (rc_inv != OSSCAR_OK) return rc_inv; }
     // Every product below that forms a small difference of large sums is accumulated in fp64 (gemm_f64acc): the scores
     // of Eq. impact are compared at 1e-5 relative, and fp32 accumulation leaves cond(H_II) * 2^-24 in them.
-    // (1) one Newton-Schulz step on the inverse: E = I - H_II Hinv in fp64, Hinv += Hinv E (E is tiny: any product will do)
-    float* E = big;
-    float* Dlt = big + nI * L.ldh;
-    CK(gemm_f64acc(st, nI, nI, nI, -1.0, Hp, L.ldp, Hinv, L.ldh, 0.0, nullptr, 0, E, L.ldh, true, done));
-    CK(gemm_tc(st, nI, nI, nI, 1.f, Hinv, L.ldh, E, L.ldh, 0.f, Dlt, L.ldh, tc, L.tc_bytes, ctx->ctl, done));
-    k_add_sym<<<dim3((unsigned)((nI + 31) / 32), (unsigned)((nI + 31) / 32)), dim3(32, 8), 0, st>>>(Hinv, L.ldh, Dlt, L.ldh, nI, done);
-    count_launches(1);
+    // (1) the inverse.  Single-row groups: fp64 copy by a third-order correction from one fp64 residual, and the fp32
+    //     inverse rounded from it (build_hinv64).  Groups of several rows: one Newton-Schulz step, E = I - H_II Hinv in
+    //     fp64, Hinv := sym(Hinv + Hinv E) (E is tiny: any product will do)
     ctx->hd_valid = false;
-    if (L.g == 1) { const int rc_d = build_hinv64(ctx, guarded); if (rc_d != OSSCAR_OK) return rc_d; }
+    if (L.g == 1) {
+        const int rc_d = build_hinv64(ctx, guarded);
+        if (rc_d != OSSCAR_OK) return rc_d;
+    } else {
+        float* E = big;
+        float* Dlt = big + nI * L.ldh;
+        CK(gemm_f64acc(st, nI, nI, nI, -1.0, Hp, L.ldp, Hinv, L.ldh, 0.0, nullptr, 0, E, L.ldh, true, done));
+        CK(gemm_tc(st, nI, nI, nI, 1.f, Hinv, L.ldh, E, L.ldh, 0.f, Dlt, L.ldh, tc, L.tc_bytes, ctx->ctl, done));
+        k_add_sym<<<dim3((unsigned)((nI + 31) / 32), (unsigned)((nI + 31) / 32)), dim3(32, 8), 0, st>>>(Hinv, L.ldh, Dlt, L.ldh, nI, done);
+        count_launches(1);
+    }
     // (2) V = Hinv G_I on the tensor cores, then one refinement step with the residual G_I - H_II V in fp64
     float* GI = big;
     float* rV = big + nI * L.ldm;
