@@ -926,6 +926,21 @@ __global__ void __launch_bounds__(1024) k_pair_select(Ptrs p, int64_t npairs)
 
 #include "search_g1.cuh"
 
+// Launch, with `dependent` set, as a programmatic dependent of the kernel before it on the stream (see
+// pdl_wait_then_release).  Only a launch that directly follows another kernel launch of the step may be one: behind an
+// event record, a copy or a reduction by the caller's hook the launch is an ordinary, fully ordered one.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(bool dependent, void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t st, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = 0; cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = dependent ? 1 : 0;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 Ptrs make_ptrs(osscar_ctx* ctx)
 {
     const Layout& L = ctx->L;
@@ -1161,21 +1176,26 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
     // threads per block of the three streaming kernels of the single-row step, by the length of the rows they stream
     const unsigned t_l1 = (unsigned)g1_threads(L.ldm > L.ldh ? L.ldm / 4 : L.ldh / 4), t_l2 = (unsigned)g1_threads(L.ldm / 4),
                    t_l4 = (unsigned)g1_threads(L.ldh / 2);
+    bool after_kernel = false;      // the last operation put on the stream was a kernel of the step
+    auto dep = [&]() { const bool d = after_kernel; after_kernel = true; return d; };
     auto launch_l1 = [&](unsigned nbV, unsigned nbH) {
-        if (t_l1 == 64) k_l1_g1<64><<<nbV + nbH, 64, 0, st>>>(p, nbV);
-        else if (t_l1 == 128) k_l1_g1<128><<<nbV + nbH, 128, 0, st>>>(p, nbV);
-        else k_l1_g1<256><<<nbV + nbH, 256, 0, st>>>(p, nbV);
+        const bool dp = dep();
+        if (t_l1 == 64) launch_pdl(dp, k_l1_g1<64>, dim3(nbV + nbH), dim3(64), st, p, nbV);
+        else if (t_l1 == 128) launch_pdl(dp, k_l1_g1<128>, dim3(nbV + nbH), dim3(128), st, p, nbV);
+        else launch_pdl(dp, k_l1_g1<256>, dim3(nbV + nbH), dim3(256), st, p, nbV);
     };
     auto launch_l2 = [&](unsigned nbR) {       // the same number of threads exchange the two slots whatever the block size
-        if (t_l2 == 64) k_l2_g1<64><<<nbR + 128, 64, 0, st>>>(p, nbR);
-        else if (t_l2 == 128) k_l2_g1<128><<<nbR + 64, 128, 0, st>>>(p, nbR);
-        else k_l2_g1<256><<<nbR + 32, 256, 0, st>>>(p, nbR);
+        const bool dp = dep();
+        if (t_l2 == 64) launch_pdl(dp, k_l2_g1<64>, dim3(nbR + 128), dim3(64), st, p, nbR);
+        else if (t_l2 == 128) launch_pdl(dp, k_l2_g1<128>, dim3(nbR + 64), dim3(128), st, p, nbR);
+        else launch_pdl(dp, k_l2_g1<256>, dim3(nbR + 32), dim3(256), st, p, nbR);
     };
     auto launch_l4 = [&]() {
         const unsigned nb = (unsigned)((L.nI + G1_RB4 - 1) / G1_RB4);
-        if (t_l4 == 64) k_l4_g1<G1_RB4, 64><<<nb, 64, 0, st>>>(p);
-        else if (t_l4 == 128) k_l4_g1<G1_RB4, 128><<<nb, 128, 0, st>>>(p);
-        else k_l4_g1<G1_RB4, 256><<<nb, 256, 0, st>>>(p);
+        const bool dp = dep();
+        if (t_l4 == 64) launch_pdl(dp, k_l4_g1<G1_RB4, 64>, dim3(nb), dim3(64), st, p);
+        else if (t_l4 == 128) launch_pdl(dp, k_l4_g1<G1_RB4, 128>, dim3(nb), dim3(128), st, p);
+        else launch_pdl(dp, k_l4_g1<G1_RB4, 256>, dim3(nb), dim3(256), st, p);
     };
     int next_prof = 0;
     int nmarks = 0;                 // events recorded per profiled step (depends on the step variant)
@@ -1227,11 +1247,12 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
             if (enqueue_scores(ctx, p, true, pair) != cudaSuccess) { rc = OSSCAR_E_CUDA; break; }
             if (sharded && shard_reduce(ctx, p.vnorm, L.d1, OSSCAR_FP32) != OSSCAR_OK) { rc = OSSCAR_E_CUDA; break; }
             if (fast && bootstrap_g1() != cudaSuccess) { rc = OSSCAR_E_CUDA; break; }
+            after_kernel = false;
         }
         cudaEvent_t* pe = nullptr;
         if (next_prof < nprof && prof_it[next_prof] == it) pe = evp[next_prof++];
         int slot = 0;
-        auto mark = [&]() { if (pe) cudaEventRecord(pe[slot], st); ++slot; };
+        auto mark = [&]() { if (pe) { cudaEventRecord(pe[slot], st); after_kernel = false; } ++slot; };
         mark();
         if (block) {
             if (enqueue_block_step(ctx, p, bp, prm->accept_mode, tol, obj_trace, swap_trace, mark) != cudaSuccess) { rc = OSSCAR_E_CUDA; break; }
@@ -1241,22 +1262,25 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
             const unsigned nbV = (unsigned)((L.nI + G1_RB - 1) / G1_RB), nbR = (unsigned)((L.nJ + G1_RB - 1) / G1_RB), nbH = nbR + 1;
             k_decide_g1<<<1, 1024, 0, st>>>(p, prm->accept_mode, tol, obj_trace, swap_trace, 1);
             if (shard_reduce(ctx, p.shard, 1, OSSCAR_FP64) != OSSCAR_OK) { rc = OSSCAR_E_CUDA; break; }
-            k_decide_g1<<<1, 1024, 0, st>>>(p, prm->accept_mode, tol, obj_trace, swap_trace, 2);   mark();
+            k_decide_g1<<<1, 1024, 0, st>>>(p, prm->accept_mode, tol, obj_trace, swap_trace, 2);
+            after_kernel = true;                                                                 mark();
             launch_l1(nbV, nbH);                                                                 mark();
             launch_l2(nbR);                                                                      mark();
             if (shard_reduce(ctx, p.vnorm, L.d1, OSSCAR_FP32) != OSSCAR_OK) { rc = OSSCAR_E_CUDA; break; }
             k_scores_sharded_g1<<<(unsigned)((L.d1 + 255) / 256), 256, 0, st>>>(p);
-            k_select_in_g1<<<1, 1024, 0, st>>>(p);                                               mark();
+            k_select_in_g1<<<1, 1024, 0, st>>>(p);
+            after_kernel = true;                                                                 mark();
             launch_l4();        mark();
+            after_kernel = false;               // the next step opens with ordinary launches
             count_launches(7);
         } else if (fast) {
             // single-row groups: decide, {H pass || V}, {R || slot exchange}, next entering group, {Hinv + next y}
             // G1_RB rows per block; the H pass has one more block for the leaving row
             const unsigned nbV = (unsigned)((L.nI + G1_RB - 1) / G1_RB), nbR = (unsigned)((L.nJ + G1_RB - 1) / G1_RB), nbH = nbR + 1;
-            k_decide_g1<<<1, 1024, 0, st>>>(p, prm->accept_mode, tol, obj_trace, swap_trace, 0);   mark();
+            launch_pdl(dep(), k_decide_g1, dim3(1), dim3(1024), st, p, (int)prm->accept_mode, tol, obj_trace, swap_trace, 0);   mark();
             launch_l1(nbV, nbH);                                                                 mark();
             launch_l2(nbR);                                                                      mark();
-            k_select_in_g1<<<1, 1024, 0, st>>>(p);                                               mark();
+            launch_pdl(dep(), k_select_in_g1, dim3(1), dim3(1024), st, p);                              mark();
             launch_l4();                                                     mark();
             count_launches(5);
         } else {
@@ -1315,6 +1339,7 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
             if (cudaMemcpyAsync((void*)(ctx->done_flag_host + 1 + ((it / batch) & 1)), &ctx->ctl->done, sizeof(int32_t),
                                 cudaMemcpyDeviceToHost, st) != cudaSuccess) { rc = OSSCAR_E_CUDA; break; }
             if (cudaEventRecord(evb[(it / batch) & 1], st) != cudaSuccess) { rc = OSSCAR_E_CUDA; break; }
+            after_kernel = false;
         }
     }
     cudaEventDestroy(evb[0]);

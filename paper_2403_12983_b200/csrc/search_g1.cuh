@@ -13,6 +13,18 @@
 
 constexpr int G1_Q1 = 2, G1_M2 = 3, G1_HDIAG = 4;
 
+// Programmatic dependent launch: the five kernels of a step are launched so that the next one may start while the
+// current one is still running.  A kernel first requests the rows it streams (written by kernels that finished long
+// ago), then waits here for the kernel before it to complete before it reads anything that kernel wrote (staged
+// vectors, scalars, the control block), and only then lets its own successor start: a successor's early part can thus
+// overlap only the late part of its immediate predecessor.  Without the launch attribute both instructions do nothing.
+// What the predecessor wrote is read with ordinary loads only: the read-only (non-coherent) path may still hold a line
+// from the step before, since no kernel boundary separates the two any more.
+__device__ __forceinline__ void pdl_wait_then_release() {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 __device__ __forceinline__ void fma4(float4& v, float a, const float4& x) {
     v.x = fmaf(a, x.x, v.x); v.y = fmaf(a, x.y, v.y); v.z = fmaf(a, x.z, v.z); v.w = fmaf(a, x.w, v.w);
 }
@@ -41,6 +53,7 @@ __global__ void k_scores_g1(Ptrs p)
 // diagonal comes from the rank-two formula, as in the row update's own epilogue.
 __global__ void k_scores_sharded_g1(Ptrs p)
 {
+    pdl_wait_then_release();
     if (p.ctl->done) return;
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const double Cinv = p.small[S_CINV], c1inv = p.small[S_C1INV];
@@ -57,7 +70,7 @@ __global__ void k_scores_sharded_g1(Ptrs p)
 }
 
 // Block-wide arg-min of val[i] (ties -> smaller group id); result broadcast through shared memory.
-__device__ void block_argmin(const double* __restrict__ val, const int32_t* __restrict__ ids, int n, bool negate,
+__device__ void block_argmin(const double* val, const int32_t* ids, int n, bool negate,
                              double* best_out, int* idx_out)
 {
     __shared__ double sv[32]; __shared__ int sid[32]; __shared__ int sidx[32];
@@ -101,6 +114,7 @@ __device__ void block_argmin(const double* __restrict__ val, const int32_t* __re
 // q* = argmax A (the group that enters at the next step).
 __global__ void __launch_bounds__(1024) k_select_in_g1(Ptrs p)
 {
+    pdl_wait_then_release();
     SearchCtl* ctl = p.ctl;
     if (ctl->done) return;
     double best; int idx;
@@ -117,6 +131,7 @@ __global__ void __launch_bounds__(1024) k_select_in_g1(Ptrs p)
 __global__ void __launch_bounds__(1024)
 k_decide_g1(Ptrs p, int accept_mode, double accept_tol, double* __restrict__ obj_trace, int32_t* __restrict__ swap_trace, int part)
 {
+    pdl_wait_then_release();
     SearchCtl* ctl = p.ctl;
     if (ctl->done) return;
     __shared__ float redf[32];
@@ -262,6 +277,7 @@ __device__ __forceinline__ void update_row_g1(const Ptrs& p, int kind, int64_t s
                 v[r][j] = c < n4 ? row[r][c] : make_float4(0.f, 0.f, 0.f, 0.f);     // requested before the step's scalars arrive
             }
         if (base == threadIdx.x) {           // first pass: the scalars of these rows, loaded behind the rows themselves
+            pdl_wait_then_release();
             if (p.ctl->done) return;             // a stopped loop only read; nothing is written
             const int64_t special = kind == 0 ? (int64_t)p.ctl->sel_slot : (int64_t)p.ctl->sel_t;
             if (kind == 1) dr = p.d[p.nJ];
@@ -278,7 +294,7 @@ __device__ __forceinline__ void update_row_g1(const Ptrs& p, int kind, int64_t s
         for (int j = 0; j < G1_U; ++j) {
             const int64_t c = base + TB * j;
             if (c < n4) {
-                const float4 kk = __ldg(K4 + c), qq = __ldg(Q4 + c);
+                const float4 kk = K4[c], qq = Q4[c];
 #pragma unroll
                 for (int r = 0; r < RB; ++r) {
                     if (sp[r]) v[r][j] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -341,11 +357,12 @@ __device__ __forceinline__ void hpass_stream(const Ptrs& p, const float4* const 
                 const int64_t c = base + TB * j;
                 x[r][j] = c < n4 ? row[r][c] : make_float4(0.f, 0.f, 0.f, 0.f);
             }
+        if (base == threadIdx.x) pdl_wait_then_release();          // b and u2 come from the kernel before this one
 #pragma unroll
         for (int j = 0; j < G1_UH; ++j) {
             const int64_t c = base + TB * j;
             if (c < n4) {
-                const float4 bb = __ldg(bv + c), uu = __ldg(uv + c);
+                const float4 bb = bv[c], uu = uv[c];
 #pragma unroll
                 for (int r = 0; r < RB; ++r) { au[r] += dot4(x[r][j], bb); ad[r] += dot4(x[r][j], uu); }
             }
@@ -389,6 +406,7 @@ __global__ void __launch_bounds__(TB, 1024 / TB) k_l1_g1(Ptrs p, unsigned nbV)  
         }
         hpass_stream<G1_RB, TB>(p, rows, l0, nvalid, red);
     } else {
+        pdl_wait_then_release();             // the leaving row is named by the control block
         const float4* rows[1] = { reinterpret_cast<const float4*>(p.Hp + (int64_t)p.ctl->sel_slot * p.ldp) };
         hpass_stream<1, TB>(p, rows, p.nJ, 1, red);
     }
@@ -430,6 +448,7 @@ __global__ void __launch_bounds__(TB, 1024 / TB) k_l2_g1(Ptrs p, unsigned nbR)
 {
     __shared__ float red[8];
     if (blockIdx.x < nbR) { update_row_g1<G1_RB, TB>(p, 1, (int64_t)blockIdx.x * G1_RB, red); return; }
+    pdl_wait_then_release();
     if (p.ctl->done) return;
     const int64_t nsw = gridDim.x - nbR;
     hswap_g1(p, (int64_t)(blockIdx.x - nbR) * blockDim.x + threadIdx.x, nsw * blockDim.x);
@@ -471,6 +490,7 @@ __global__ void __launch_bounds__(TB) k_l4_g1(Ptrs p)
                 h[r][j] = c < n2 ? row[r][c] : make_double2(0.0, 0.0);    // requested before the step's scalars arrive
             }
         if (base == threadIdx.x) {
+            pdl_wait_then_release();
             if (p.ctl->done) return;
             r0 = p.ctl->sel_slot;
             const double Cinv = p.small[S_CINV], c1inv = p.small[S_C1INV];
@@ -489,7 +509,7 @@ __global__ void __launch_bounds__(TB) k_l4_g1(Ptrs p)
         for (int j = 0; j < G1_UH; ++j) {
             const int64_t c = base + TB * j;
             if (c < n2) {
-                const float2 bb = __ldg(b2 + c), uu = __ldg(u2v + c), hh = __ldg(h2 + c);
+                const float2 bb = b2[c], uu = u2v[c], hh = h2[c];
                 const int64_t rc = r0 - c * 2;           // position of column r0 inside this piece, if any
 #pragma unroll
                 for (int r = 0; r < RB; ++r) {
