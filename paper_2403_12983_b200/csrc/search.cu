@@ -52,6 +52,19 @@ struct Ptrs {
 // layout of the `small` region (doubles, each g*g): indices of the matrices
 enum { S_CINV = 0, S_C1INV, S_Q1, S_Q1C, S_M2, S_GV, S_GX, S_GR, S_C, S_P, S_T1, S_T2, S_T3, S_C1, S_L, S_LI };
 
+// Programmatic dependent launch: the kernels of a swap step are launched so that the next one may start while the
+// current one is still running.  A kernel of single-row groups first requests the rows it streams (written by kernels
+// that finished long ago), the kernels of wider groups begin with the wait; a kernel waits here for the kernel before
+// it to complete before it reads anything that kernel wrote (staged vectors, scalars, the control block), and only then
+// lets its own successor start: a successor's early part can thus overlap only the late part of its immediate
+// predecessor, and its blocks are already resident when the predecessor drains.  Without the launch attribute both
+// instructions do nothing.  What the predecessor wrote is read with ordinary loads only: the read-only (non-coherent)
+// path may still hold a line from the step before, since no kernel boundary separates the two any more.
+__device__ __forceinline__ void pdl_wait_then_release() {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 // ------------------------------------------------------------------ row norms / group Grams
 // norm[i] = ||M[i, 0:ld)||^2 (pads are zero); one block per row.
 __global__ void k_row_norms(const float* __restrict__ M, int64_t ld, float* __restrict__ norm, const SearchCtl* ctl)
@@ -75,6 +88,7 @@ __global__ void k_row_norms(const float* __restrict__ M, int64_t ld, float* __re
 constexpr int GG_AT = 4;
 __global__ void __launch_bounds__(256) k_group_gram(Ptrs p)
 {
+    pdl_wait_then_release();
     if (p.ctl->done) return;
     const int g = p.g;
     const bool kept = (int)blockIdx.x < p.k;
@@ -110,6 +124,7 @@ __global__ void __launch_bounds__(256) k_group_gram(Ptrs p)
 // Blocks [0, k): kept slots (M = Hinv_rr, Gram of V rows) -> D; the rest: pruned slots (M = c, Gram of R rows) -> A.
 __global__ void __launch_bounds__(1024) k_scores_general(Ptrs p)
 {
+    pdl_wait_then_release();
     if (p.ctl->done) return;
     extern __shared__ double smd[];
     const int g = p.g;
@@ -146,6 +161,7 @@ __global__ void __launch_bounds__(1024) k_scores_general(Ptrs p)
 // Cheapest drop (min D, ties -> smaller group id) and most valuable add (max A, ties -> smaller id).
 __global__ void __launch_bounds__(1024) k_select(Ptrs p)
 {
+    pdl_wait_then_release();
     SearchCtl* ctl = p.ctl;
     if (ctl->done) return;
     __shared__ double sv[32]; __shared__ int sid[32]; __shared__ int sidx[32];
@@ -198,6 +214,7 @@ __global__ void __launch_bounds__(1024) k_select(Ptrs p)
 // ------------------------------------------------------------------ y = Hinv h  (one warp per row, grid.y = e)
 __global__ void __launch_bounds__(256) k_ypass(Ptrs p)
 {
+    pdl_wait_then_release();
     if (p.ctl->done) return;
     const int e = blockIdx.y;
     const int lane = threadIdx.x & 31;
@@ -210,12 +227,12 @@ __global__ void __launch_bounds__(256) k_ypass(Ptrs p)
     int64_t c = lane;
     for (; c + 32 < n4; c += 64) {
         const float4 x0 = arow[c], x1 = arow[c + 32];
-        const float4 h0 = __ldg(hrow + c), h1 = __ldg(hrow + c + 32);
+        const float4 h0 = *(hrow + c), h1 = *(hrow + c + 32);
         a0 += x0.x * h0.x + x0.y * h0.y + x0.z * h0.z + x0.w * h0.w;
         a1 += x1.x * h1.x + x1.y * h1.y + x1.z * h1.z + x1.w * h1.w;
     }
     for (; c < n4; c += 32) {
-        const float4 x0 = arow[c]; const float4 h0 = __ldg(hrow + c);
+        const float4 x0 = arow[c]; const float4 h0 = *(hrow + c);
         a0 += x0.x * h0.x + x0.y * h0.y + x0.z * h0.z + x0.w * h0.w;
     }
     a0 = warp_sum(a0 + a1);
@@ -225,6 +242,7 @@ __global__ void __launch_bounds__(256) k_ypass(Ptrs p)
 // Grams of the chosen rows: GV = V_r V_r^T, GX = V_r R_q^T, GR = R_q R_q^T; one warp per entry.
 __global__ void __launch_bounds__(256) k_pairgram(Ptrs p)
 {
+    pdl_wait_then_release();
     if (p.ctl->done) return;
     const int g = p.g;
     const int64_t wid = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -248,6 +266,7 @@ __global__ void __launch_bounds__(256) k_pairgram(Ptrs p)
 __global__ void __launch_bounds__(1024)
 k_small(Ptrs p, int accept_mode, double accept_tol, int max_swaps, double* __restrict__ obj_trace, int32_t* __restrict__ swap_trace)
 {
+    pdl_wait_then_release();
     SearchCtl* ctl = p.ctl;
     if (ctl->done) return;
     __shared__ double red[32];
@@ -314,6 +333,7 @@ k_small(Ptrs p, int accept_mode, double accept_tol, int max_swaps, double* __res
 // Part B (threads over columns): K = C^-1 V_r, Vq = c1^-1 R_q + (c1^-1 P C^-1) V_r.
 __global__ void __launch_bounds__(256) k_prep(Ptrs p)
 {
+    pdl_wait_then_release();
     if (p.ctl->done) return;
     const int g = p.g, gg = g * g;
     const double* S = p.small;
@@ -358,6 +378,7 @@ __global__ void __launch_bounds__(256) k_prep(Ptrs p)
 template <int RPW>
 __global__ void __launch_bounds__(256) k_hpass(Ptrs p)
 {
+    pdl_wait_then_release();
     if (p.ctl->done) return;
     const int e = blockIdx.y, g = p.g;
     const int lane = threadIdx.x & 31;
@@ -379,7 +400,7 @@ __global__ void __launch_bounds__(256) k_hpass(Ptrs p)
 #pragma unroll
     for (int i = 0; i < RPW; ++i) { au[i] = 0.f; ad[i] = 0.f; }
     for (int64_t c = lane; c < p.ldh / 4; c += 32) {
-        const float4 bb = __ldg(bv + c), uu = __ldg(uv + c);
+        const float4 bb = *(bv + c), uu = *(uv + c);
 #pragma unroll
         for (int i = 0; i < RPW; ++i) {
             const float4 x = rows[i][c];
@@ -404,6 +425,7 @@ __global__ void __launch_bounds__(256) k_hpass(Ptrs p)
 constexpr int HI_RT = 8;
 __global__ void __launch_bounds__(256) k_update_hinv(Ptrs p)
 {
+    pdl_wait_then_release();
     if (p.ctl->done) return;
     const int64_t c4 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;     // float4 column index
     if (c4 * 4 >= p.ldh) return;
@@ -442,6 +464,7 @@ __global__ void __launch_bounds__(256) k_update_hinv(Ptrs p)
 constexpr int UP_ROWS = 4;
 __global__ void __launch_bounds__(256) k_update_rows(Ptrs p, int kind)
 {
+    pdl_wait_then_release();
     if (p.ctl->done) return;
     __shared__ float red[32];
     float* M = kind == 0 ? p.V : p.R;
@@ -493,6 +516,7 @@ constexpr int TP_E = 4, TP_W = 4;
 template <int TP_R>
 __global__ void __launch_bounds__(32 * TP_W) k_ypass_g(Ptrs p)
 {
+    pdl_wait_then_release();
     if (p.ctl->done) return;
     const int g = p.g, e0 = blockIdx.y * TP_E;
     const int lane = threadIdx.x & 31;
@@ -514,7 +538,7 @@ __global__ void __launch_bounds__(32 * TP_W) k_ypass_g(Ptrs p)
 #pragma unroll
         for (int i = 0; i < TP_R; ++i) x[i] = arow[i][c];
 #pragma unroll
-        for (int j = 0; j < TP_E; ++j) h[j] = __ldg(hrow[j] + c);
+        for (int j = 0; j < TP_E; ++j) h[j] = *(hrow[j] + c);
 #pragma unroll
         for (int i = 0; i < TP_R; ++i)
 #pragma unroll
@@ -533,6 +557,7 @@ __global__ void __launch_bounds__(32 * TP_W) k_ypass_g(Ptrs p)
 template <int TP_R>
 __global__ void __launch_bounds__(32 * TP_W) k_hpass_g(Ptrs p)
 {
+    pdl_wait_then_release();
     if (p.ctl->done) return;
     const int g = p.g, e0 = blockIdx.y * TP_E;
     const int lane = threadIdx.x & 31;
@@ -564,7 +589,7 @@ __global__ void __launch_bounds__(32 * TP_W) k_hpass_g(Ptrs p)
         for (int i = 0; i < TP_R; ++i) x[i] = rows[i][c];
 #pragma unroll
         for (int j = 0; j < TP_E; ++j) {
-            const float4 bb = __ldg(bv[j] + c), uu = __ldg(uv[j] + c);
+            const float4 bb = *(bv[j] + c), uu = *(uv[j] + c);
 #pragma unroll
             for (int i = 0; i < TP_R; ++i) { au[i][j] += dot4f(x[i], bb); ad[i][j] += dot4f(x[i], uu); }
         }
@@ -592,6 +617,7 @@ constexpr int TG_T = 128;
 // dynamic shared memory 2 g TG_RT floats.
 __global__ void __launch_bounds__(TG_T) k_update_hinv_g(Ptrs p)
 {
+    pdl_wait_then_release();
     if (p.ctl->done) return;
     extern __shared__ float smf[];
     const int g = p.g;
@@ -616,7 +642,7 @@ __global__ void __launch_bounds__(TG_T) k_update_hinv_g(Ptrs p)
     const float4* b4 = reinterpret_cast<const float4*>(p.b) + c4;
     const float4* u4 = reinterpret_cast<const float4*>(p.u2) + c4;
     for (int e = 0; e < g; ++e) {
-        const float4 bb = __ldg(b4 + (int64_t)e * n4), uu = __ldg(u4 + (int64_t)e * n4);
+        const float4 bb = *(b4 + (int64_t)e * n4), uu = *(u4 + (int64_t)e * n4);
 #pragma unroll
         for (int i = 0; i < TG_RT; ++i) {
             const float nb = nbs[e * TG_RT + i], us = ucs[e * TG_RT + i];
@@ -652,6 +678,7 @@ __global__ void __launch_bounds__(TG_T) k_update_hinv_g(Ptrs p)
 // The replaced rows are the same sum started from zero with their own coefficients.
 __global__ void __launch_bounds__(TG_T) k_update_rows_g(Ptrs p, int kind)
 {
+    pdl_wait_then_release();
     if (p.ctl->done) return;
     extern __shared__ float smf[];
     const int g = p.g;
@@ -688,7 +715,7 @@ __global__ void __launch_bounds__(TG_T) k_update_rows_g(Ptrs p, int kind)
     const float4* K4 = reinterpret_cast<const float4*>(p.K) + c4;
     const float4* Q4 = reinterpret_cast<const float4*>(p.Vq) + c4;
     for (int e = 0; e < g; ++e) {
-        const float4 kk = __ldg(K4 + (int64_t)e * n4), q = __ldg(Q4 + (int64_t)e * n4);
+        const float4 kk = *(K4 + (int64_t)e * n4), q = *(Q4 + (int64_t)e * n4);
 #pragma unroll
         for (int i = 0; i < TG_RT; ++i) {
             const float ck = cks[e * TG_RT + i], cq = cqs[e * TG_RT + i];
@@ -731,6 +758,7 @@ __device__ void mat_mul_nt_acc(const double* A, const double* B, double* C, int 
 // with C^-1 (c1^-1) sit in shared memory (2 g^2 doubles), the four g x g products run on the fp64 tensor-core path.
 __global__ void __launch_bounds__(1024) k_update_c(Ptrs p)
 {
+    pdl_wait_then_release();
     if (p.ctl->done) return;
     extern __shared__ double smc[];
     const int g = p.g, gg = g * g;
@@ -761,6 +789,7 @@ __global__ void __launch_bounds__(1024) k_update_c(Ptrs p)
 // phase 1 also exchanges the two groups in the slot permutation.
 __global__ void __launch_bounds__(256) k_hswap(Ptrs p, int phase)
 {
+    pdl_wait_then_release();
     if (p.ctl->done) return;
     const int g = p.g;
     const int64_t a0 = (int64_t)p.ctl->sel_slot * g, b0 = p.nI + (int64_t)p.ctl->sel_t * g;
@@ -924,22 +953,28 @@ __global__ void __launch_bounds__(1024) k_pair_select(Ptrs p, int64_t npairs)
     }
 }
 
-#include "search_g1.cuh"
-
 // Launch, with `dependent` set, as a programmatic dependent of the kernel before it on the stream (see
 // pdl_wait_then_release).  Only a launch that directly follows another kernel launch of the step may be one: behind an
 // event record, a copy or a reduction by the caller's hook the launch is an ordinary, fully ordered one.
 template <typename... KArgs, typename... Args>
-cudaError_t launch_pdl(bool dependent, void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t st, Args... args)
+cudaError_t launch_pdl_smem(bool dependent, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args)
 {
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = 0; cfg.stream = st;
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
     cudaLaunchAttribute at[1];
     at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     at[0].val.programmaticStreamSerializationAllowed = dependent ? 1 : 0;
     cfg.attrs = at; cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(bool dependent, void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t st, Args... args)
+{
+    return launch_pdl_smem(dependent, kernel, grid, block, 0, st, args...);
+}
+
+#include "search_g1.cuh"
 
 Ptrs make_ptrs(osscar_ctx* ctx)
 {
@@ -971,7 +1006,7 @@ static unsigned small_threads(int g) { return g * g >= 1024 ? 1024u : 256u; }
 #define CK(x) do { cudaError_t e_ = (x); if (e_ != cudaSuccess) return OSSCAR_E_CUDA; } while (0)
 
 // Everything the selection needs from a freshly built or freshly updated state.
-cudaError_t enqueue_scores(osscar_ctx* ctx, const Ptrs& p, bool norms, bool general = false)
+cudaError_t enqueue_scores(osscar_ctx* ctx, const Ptrs& p, bool norms, bool general = false, bool chain = false, bool dependent = false)
 {
     cudaStream_t st = ctx->stream;
     if (p.g == 1 && !general) {
@@ -984,8 +1019,9 @@ cudaError_t enqueue_scores(osscar_ctx* ctx, const Ptrs& p, bool norms, bool gene
         const size_t smem = 3 * (size_t)p.g * p.g * sizeof(double);
         cudaError_t e = cudaFuncSetAttribute(k_scores_general, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        k_group_gram<<<dim3((unsigned)p.ng, (unsigned)((p.g + GG_AT - 1) / GG_AT)), 256, 0, st>>>(p);      // kept and pruned groups together
-        k_scores_general<<<(unsigned)p.ng, small_threads(p.g), smem, st>>>(p);
+        // kept and pruned groups together; inside a swap step (chain) the two are programmatic dependents
+        launch_pdl(chain && dependent, k_group_gram, dim3((unsigned)p.ng, (unsigned)((p.g + GG_AT - 1) / GG_AT)), dim3(256), st, p);
+        launch_pdl_smem(chain, k_scores_general, dim3((unsigned)p.ng), dim3(small_threads(p.g)), smem, st, p);
         count_launches(2);
     }
     return cudaGetLastError();
@@ -1149,7 +1185,10 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
     }
     if (g > 1) CK(cudaFuncSetAttribute(k_update_c, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(2 * (size_t)g * g * sizeof(double))));
 
-    const int batch = 32;
+    // Steps per host batch.  The host stays at most two batches ahead of the device, so a loop that stops has up to
+    // three batches of launches behind it that return at once (about 2 us each): short batches for states whose step is
+    // short, where those launches would be a visible part of the solve.
+    const int batch = block ? 4 : 8;
     cudaEvent_t evb[2];
     CK(cudaEventCreateWithFlags(&evb[0], cudaEventDisableTiming));
     CK(cudaEventCreateWithFlags(&evb[1], cudaEventDisableTiming));
@@ -1284,53 +1323,53 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
             launch_l4();                                                     mark();
             count_launches(5);
         } else {
-            if (pair) { if (pair_scores() != cudaSuccess) { rc = OSSCAR_E_CUDA; break; } }
-            else k_select<<<1, 1024, 0, st>>>(p);
+            if (pair) { if (pair_scores() != cudaSuccess) { rc = OSSCAR_E_CUDA; break; } after_kernel = false; }
+            else launch_pdl(dep(), k_select, dim3(1), dim3(1024), st, p);
             mark();
-            k_pairgram<<<(unsigned)((3 * g * g + 7) / 8), 256, 0, st>>>(p);                          mark();
+            launch_pdl(dep(), k_pairgram, dim3((unsigned)((3 * g * g + 7) / 8)), dim3(256), st, p);                          mark();
             if (g > 1) {
                 const int R = tile_rows(L.nI);
-                if (R == 4) k_ypass_g<4><<<dim3(tile_blocks(L.nI, 4), gtiles), 32 * TP_W, 0, st>>>(p);
-                else if (R == 2) k_ypass_g<2><<<dim3(tile_blocks(L.nI, 2), gtiles), 32 * TP_W, 0, st>>>(p);
-                else k_ypass_g<1><<<dim3(tile_blocks(L.nI, 1), gtiles), 32 * TP_W, 0, st>>>(p);
+                if (R == 4) launch_pdl(dep(), k_ypass_g<4>, dim3(tile_blocks(L.nI, 4), gtiles), dim3(32 * TP_W), st, p);
+                else if (R == 2) launch_pdl(dep(), k_ypass_g<2>, dim3(tile_blocks(L.nI, 2), gtiles), dim3(32 * TP_W), st, p);
+                else launch_pdl(dep(), k_ypass_g<1>, dim3(tile_blocks(L.nI, 1), gtiles), dim3(32 * TP_W), st, p);
             }
-            else k_ypass<<<dim3(yblocks, 1), 256, 0, st>>>(p);
+            else launch_pdl(dep(), k_ypass, dim3(yblocks, 1), dim3(256), st, p);
             mark();
-            k_small<<<1, small_threads(g), inv_smem, st>>>(p, prm->accept_mode, tol, max_swaps, obj_trace, swap_trace);
+            launch_pdl_smem(dep(), k_small, dim3(1), dim3(small_threads(g)), inv_smem, st, p, prm->accept_mode, tol, max_swaps, obj_trace, swap_trace);
             mark();
-            k_prep<<<prep_blocks, 256, 0, st>>>(p);                                                  mark();
+            launch_pdl(dep(), k_prep, dim3(prep_blocks), dim3(256), st, p);                                                  mark();
             if (g > 1) {
                 const int R = tile_rows(L.nJ + g);
-                if (R == 4) k_hpass_g<4><<<dim3(tile_blocks(L.nJ + g, 4), gtiles), 32 * TP_W, 0, st>>>(p);
-                else if (R == 2) k_hpass_g<2><<<dim3(tile_blocks(L.nJ + g, 2), gtiles), 32 * TP_W, 0, st>>>(p);
-                else k_hpass_g<1><<<dim3(tile_blocks(L.nJ + g, 1), gtiles), 32 * TP_W, 0, st>>>(p);
+                if (R == 4) launch_pdl(dep(), k_hpass_g<4>, dim3(tile_blocks(L.nJ + g, 4), gtiles), dim3(32 * TP_W), st, p);
+                else if (R == 2) launch_pdl(dep(), k_hpass_g<2>, dim3(tile_blocks(L.nJ + g, 2), gtiles), dim3(32 * TP_W), st, p);
+                else launch_pdl(dep(), k_hpass_g<1>, dim3(tile_blocks(L.nJ + g, 1), gtiles), dim3(32 * TP_W), st, p);
             }
-            else k_hpass<RPW><<<dim3(hblocks, 1), 256, 0, st>>>(p);
+            else launch_pdl(dep(), k_hpass<RPW>, dim3(hblocks, 1), dim3(256), st, p);
             mark();
             if (g > 1) {
                 const size_t sm_t = 2 * (size_t)g * TG_RT * sizeof(float);
-                k_update_hinv_g<<<dim3((unsigned)((L.ldh / 4 + TG_T - 1) / TG_T), (unsigned)((L.nI + TG_RT - 1) / TG_RT)), TG_T, sm_t, st>>>(p);
+                launch_pdl_smem(dep(), k_update_hinv_g, dim3((unsigned)((L.ldh / 4 + TG_T - 1) / TG_T), (unsigned)((L.nI + TG_RT - 1) / TG_RT)), dim3(TG_T), sm_t, st, p);
                 mark();
                 const unsigned ctiles = (unsigned)((L.ldm / 4 + TG_T - 1) / TG_T);
-                k_update_rows_g<<<dim3(ctiles, (unsigned)((L.nI + TG_RT - 1) / TG_RT)), TG_T, sm_t, st>>>(p, 0);     mark();
-                k_update_rows_g<<<dim3(ctiles, (unsigned)((L.nJ + TG_RT - 1) / TG_RT)), TG_T, sm_t, st>>>(p, 1);     mark();
+                launch_pdl_smem(dep(), k_update_rows_g, dim3(ctiles, (unsigned)((L.nI + TG_RT - 1) / TG_RT)), dim3(TG_T), sm_t, st, p, 0);     mark();
+                launch_pdl_smem(dep(), k_update_rows_g, dim3(ctiles, (unsigned)((L.nJ + TG_RT - 1) / TG_RT)), dim3(TG_T), sm_t, st, p, 1);     mark();
             } else {
-                k_update_hinv<<<dim3((unsigned)((L.ldh / 4 + 255) / 256), (unsigned)((L.nI + HI_RT - 1) / HI_RT)), 256, 0, st>>>(p);
+                launch_pdl(dep(), k_update_hinv, dim3((unsigned)((L.ldh / 4 + 255) / 256), (unsigned)((L.nI + HI_RT - 1) / HI_RT)), dim3(256), st, p);
                 mark();
-                k_update_rows<<<(unsigned)((L.nI + UP_ROWS - 1) / UP_ROWS), 256, 0, st>>>(p, 0);          mark();
-                k_update_rows<<<(unsigned)((L.nJ + UP_ROWS - 1) / UP_ROWS), 256, 0, st>>>(p, 1);          mark();
+                launch_pdl(dep(), k_update_rows, dim3((unsigned)((L.nI + UP_ROWS - 1) / UP_ROWS)), dim3(256), st, p, 0);          mark();
+                launch_pdl(dep(), k_update_rows, dim3((unsigned)((L.nJ + UP_ROWS - 1) / UP_ROWS)), dim3(256), st, p, 1);          mark();
             }
             count_launches(9);
             if (g > 1) {
-                k_update_c<<<(unsigned)(L.ng - L.k), small_threads(g), 2 * (size_t)g * g * sizeof(double), st>>>(p);
+                launch_pdl_smem(dep(), k_update_c, dim3((unsigned)(L.ng - L.k)), dim3(small_threads(g)), 2 * (size_t)g * g * sizeof(double), st, p);
                 count_launches(1);
             }
             if (g > 1 || pair) {
-                if (enqueue_scores(ctx, p, false, pair) != cudaSuccess) { rc = OSSCAR_E_CUDA; break; }
+                if (enqueue_scores(ctx, p, false, pair, true, dep()) != cudaSuccess) { rc = OSSCAR_E_CUDA; break; }
             }
             mark();
-            k_hswap<<<(unsigned)((L.ldp * g + 255) / 256), 256, 0, st>>>(p, 0);                       mark();
-            k_hswap<<<(unsigned)((L.ldp * g + 255) / 256), 256, 0, st>>>(p, 1);                       mark();
+            launch_pdl(dep(), k_hswap, dim3((unsigned)((L.ldp * g + 255) / 256)), dim3(256), st, p, 0);                       mark();
+            launch_pdl(dep(), k_hswap, dim3((unsigned)((L.ldp * g + 255) / 256)), dim3(256), st, p, 1);                       mark();
             count_launches(2);
         }
         if (pe) nmarks = slot;

@@ -13,18 +13,6 @@
 
 constexpr int G1_Q1 = 2, G1_M2 = 3, G1_HDIAG = 4;
 
-// Programmatic dependent launch: the five kernels of a step are launched so that the next one may start while the
-// current one is still running.  A kernel first requests the rows it streams (written by kernels that finished long
-// ago), then waits here for the kernel before it to complete before it reads anything that kernel wrote (staged
-// vectors, scalars, the control block), and only then lets its own successor start: a successor's early part can thus
-// overlap only the late part of its immediate predecessor.  Without the launch attribute both instructions do nothing.
-// What the predecessor wrote is read with ordinary loads only: the read-only (non-coherent) path may still hold a line
-// from the step before, since no kernel boundary separates the two any more.
-__device__ __forceinline__ void pdl_wait_then_release() {
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-}
-
 __device__ __forceinline__ void fma4(float4& v, float a, const float4& x) {
     v.x = fmaf(a, x.x, v.x); v.y = fmaf(a, x.y, v.y); v.z = fmaf(a, x.z, v.z); v.w = fmaf(a, x.w, v.w);
 }
