@@ -615,15 +615,12 @@ constexpr int TG_T = 128;
 
 // Hinv' = Hinv - bC b^T + u2c u2^T; rows/columns of r take -u2c, the rr block c1^-1.  Grid (column tiles, row tiles),
 // dynamic shared memory 2 g TG_RT floats.
-__global__ void __launch_bounds__(TG_T) k_update_hinv_g(Ptrs p)
+__device__ __forceinline__ void update_hinv_g_tile(const Ptrs& p, float* smf, unsigned bx, unsigned by)
 {
-    pdl_wait_then_release();
-    if (p.ctl->done) return;
-    extern __shared__ float smf[];
     const int g = p.g;
     float* nbs = smf;                       // [e][i] = -bC[e][row0 + i]
     float* ucs = smf + g * TG_RT;           // [e][i] = u2c[e][row0 + i]
-    const int64_t row0 = (int64_t)blockIdx.y * TG_RT;
+    const int64_t row0 = (int64_t)by * TG_RT;
     const int64_t r0 = (int64_t)p.ctl->sel_slot * g;
     for (int idx = threadIdx.x; idx < g * TG_RT; idx += TG_T) {
         const int e = idx / TG_RT; const int64_t s = row0 + idx % TG_RT;
@@ -633,7 +630,7 @@ __global__ void __launch_bounds__(TG_T) k_update_hinv_g(Ptrs p)
     }
     __syncthreads();
     const int64_t n4 = p.ldh / 4;
-    const int64_t c4 = (int64_t)blockIdx.x * TG_T + threadIdx.x;
+    const int64_t c4 = (int64_t)bx * TG_T + threadIdx.x;
     if (c4 >= n4) return;
     float4 h[TG_RT];
 #pragma unroll
@@ -676,18 +673,15 @@ __global__ void __launch_bounds__(TG_T) k_update_hinv_g(Ptrs p)
 // V'[s] = V[s] - sum_e b[e][s] K[e] - sum_e u2[e][s] Vq[e] (rows of r: Vq) for kind 0,
 // R'[l] = R[l] + sum_e u[l][e] K[e] - sum_e d[l][e] Vq[e] (rows of q: K[e] - sum_f d[nJ+e][f] Vq[f]) for kind 1.
 // The replaced rows are the same sum started from zero with their own coefficients.
-__global__ void __launch_bounds__(TG_T) k_update_rows_g(Ptrs p, int kind)
+__device__ __forceinline__ void update_rows_g_tile(const Ptrs& p, float* smf, int kind, unsigned bx, unsigned by)
 {
-    pdl_wait_then_release();
-    if (p.ctl->done) return;
-    extern __shared__ float smf[];
     const int g = p.g;
     float* cks = smf;                       // coefficient of K[e] for row i
     float* cqs = smf + g * TG_RT;           // coefficient of Vq[e]
     float* M = kind == 0 ? p.V : p.R;
     const int64_t nrows = kind == 0 ? p.nI : p.nJ;
     const int64_t special0 = (kind == 0 ? (int64_t)p.ctl->sel_slot : (int64_t)p.ctl->sel_t) * g;
-    const int64_t row0 = (int64_t)blockIdx.y * TG_RT;
+    const int64_t row0 = (int64_t)by * TG_RT;
     for (int idx = threadIdx.x; idx < g * TG_RT; idx += TG_T) {
         const int e = idx / TG_RT; const int64_t s = row0 + idx % TG_RT;
         float ck = 0.f, cq = 0.f;
@@ -703,7 +697,7 @@ __global__ void __launch_bounds__(TG_T) k_update_rows_g(Ptrs p, int kind)
     }
     __syncthreads();
     const int64_t n4 = p.ldm / 4;
-    const int64_t c4 = (int64_t)blockIdx.x * TG_T + threadIdx.x;
+    const int64_t c4 = (int64_t)bx * TG_T + threadIdx.x;
     if (c4 >= n4) return;
     float4 v[TG_RT];
 #pragma unroll
@@ -726,6 +720,38 @@ __global__ void __launch_bounds__(TG_T) k_update_rows_g(Ptrs p, int kind)
 #pragma unroll
     for (int i = 0; i < TG_RT; ++i)
         if (row0 + i < nrows) reinterpret_cast<float4*>(M + (row0 + i) * p.ldm)[c4] = v[i];
+}
+
+__global__ void __launch_bounds__(TG_T) k_update_hinv_g(Ptrs p)
+{
+    pdl_wait_then_release();
+    if (p.ctl->done) return;
+    extern __shared__ float smf[];
+    update_hinv_g_tile(p, smf, blockIdx.x, blockIdx.y);
+}
+
+__global__ void __launch_bounds__(TG_T) k_update_rows_g(Ptrs p, int kind)
+{
+    pdl_wait_then_release();
+    if (p.ctl->done) return;
+    extern __shared__ float smf[];
+    update_rows_g_tile(p, smf, kind, blockIdx.x, blockIdx.y);
+}
+
+// The three updates of a step in one launch (they depend on the same staged vectors and on nothing of each other):
+// blocks [0, nh) are the tiles of Hinv, the next nv those of V, the rest those of R; hx and mx are the column tiles of a
+// row tile of Hinv and of V / R.
+__global__ void __launch_bounds__(TG_T) k_update_all_g(Ptrs p, unsigned nh, unsigned nv, unsigned hx, unsigned mx)
+{
+    pdl_wait_then_release();
+    if (p.ctl->done) return;
+    extern __shared__ float smf[];
+    unsigned b = blockIdx.x;
+    if (b < nh) { update_hinv_g_tile(p, smf, b % hx, b / hx); return; }
+    b -= nh;
+    if (b < nv) { update_rows_g_tile(p, smf, 0, b % mx, b / mx); return; }
+    b -= nv;
+    update_rows_g_tile(p, smf, 1, b % mx, b / mx);
 }
 
 // C += sign * A * B^T (all g x g, ld g) on the fp64 tensor-core path; each entry of C is owned by one lane.
@@ -1348,18 +1374,23 @@ int run_search(osscar_ctx* ctx, const osscar_search_params* prm, int32_t* suppor
             mark();
             if (g > 1) {
                 const size_t sm_t = 2 * (size_t)g * TG_RT * sizeof(float);
-                launch_pdl_smem(dep(), k_update_hinv_g, dim3((unsigned)((L.ldh / 4 + TG_T - 1) / TG_T), (unsigned)((L.nI + TG_RT - 1) / TG_RT)), dim3(TG_T), sm_t, st, p);
-                mark();
-                const unsigned ctiles = (unsigned)((L.ldm / 4 + TG_T - 1) / TG_T);
-                launch_pdl_smem(dep(), k_update_rows_g, dim3(ctiles, (unsigned)((L.nI + TG_RT - 1) / TG_RT)), dim3(TG_T), sm_t, st, p, 0);     mark();
-                launch_pdl_smem(dep(), k_update_rows_g, dim3(ctiles, (unsigned)((L.nJ + TG_RT - 1) / TG_RT)), dim3(TG_T), sm_t, st, p, 1);     mark();
+                const unsigned hx = (unsigned)((L.ldh / 4 + TG_T - 1) / TG_T), hy = (unsigned)((L.nI + TG_RT - 1) / TG_RT);
+                const unsigned mx = (unsigned)((L.ldm / 4 + TG_T - 1) / TG_T), ry = (unsigned)((L.nJ + TG_RT - 1) / TG_RT);
+                if (pe) {           // a profiled step times the three updates one by one
+                    launch_pdl_smem(dep(), k_update_hinv_g, dim3(hx, hy), dim3(TG_T), sm_t, st, p);          mark();
+                    launch_pdl_smem(dep(), k_update_rows_g, dim3(mx, hy), dim3(TG_T), sm_t, st, p, 0);       mark();
+                    launch_pdl_smem(dep(), k_update_rows_g, dim3(mx, ry), dim3(TG_T), sm_t, st, p, 1);       mark();
+                } else {
+                    launch_pdl_smem(dep(), k_update_all_g, dim3(hx * hy + mx * hy + mx * ry), dim3(TG_T), sm_t, st, p, hx * hy, mx * hy, hx, mx);
+                    mark(); mark(); mark();
+                }
             } else {
                 launch_pdl(dep(), k_update_hinv, dim3((unsigned)((L.ldh / 4 + 255) / 256), (unsigned)((L.nI + HI_RT - 1) / HI_RT)), dim3(256), st, p);
                 mark();
                 launch_pdl(dep(), k_update_rows, dim3((unsigned)((L.nI + UP_ROWS - 1) / UP_ROWS)), dim3(256), st, p, 0);          mark();
                 launch_pdl(dep(), k_update_rows, dim3((unsigned)((L.nJ + UP_ROWS - 1) / UP_ROWS)), dim3(256), st, p, 1);          mark();
             }
-            count_launches(9);
+            count_launches(g > 1 && !pe ? 7 : 9);
             if (g > 1) {
                 launch_pdl_smem(dep(), k_update_c, dim3((unsigned)(L.ng - L.k)), dim3(small_threads(g)), 2 * (size_t)g * g * sizeof(double), st, p);
                 count_launches(1);
