@@ -315,25 +315,58 @@ k_mma_pipe(const __grid_constant__ Maps maps, int64_t M, int64_t N, int64_t K, f
     if (threadIdx.x == 0 && *abort_flag) ctl->status = OSSCAR_E_TIMEOUT;
 }
 
-// x = x1 + x2 + x3 with bf16 terms (round to nearest each time); dst rows are ldd wide, the tail is zero.
+// x = x1 + x2 + x3 with bf16 terms (round to nearest each time); dst rows are ldd wide (a multiple of 8), the tail is
+// zero.  A thread converts eight consecutive elements of a row: two 16-byte loads where the source allows it (vec),
+// one 16-byte store per term.
+__device__ __forceinline__ void split3_one(float x, __nv_bfloat16& a, __nv_bfloat16& b, __nv_bfloat16& c)
+{
+    a = __float2bfloat16_rn(x);
+    x -= __bfloat162float(a);
+    b = __float2bfloat16_rn(x);
+    x -= __bfloat162float(b);
+    c = __float2bfloat16_rn(x);
+}
+
 __global__ void k_split3(const float* __restrict__ src, int64_t lds, int64_t rows, int64_t cols,
                          __nv_bfloat16* __restrict__ d1, __nv_bfloat16* __restrict__ d2, __nv_bfloat16* __restrict__ d3,
-                         int64_t ldd, const int32_t* __restrict__ done)
+                         int64_t ldd, int vec, const int32_t* __restrict__ done)
 {
     if (done && *done) return;
-    const int64_t total = rows * ldd;
+    const int64_t per_row = ldd / 8, total = rows * per_row;
     const bool small = total < (int64_t)0x7fffffff;          // 32-bit index arithmetic where it fits (64-bit division is slow)
     for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
-        int64_t r, c;
-        if (small) { const uint32_t i32 = (uint32_t)idx, l32 = (uint32_t)ldd; r = i32 / l32; c = i32 % l32; }
-        else { r = idx / ldd; c = idx % ldd; }
-        float x = c < cols ? src[r * lds + c] : 0.f;
-        const __nv_bfloat16 a = __float2bfloat16_rn(x);
-        x -= __bfloat162float(a);
-        const __nv_bfloat16 b = __float2bfloat16_rn(x);
-        x -= __bfloat162float(b);
-        d1[idx] = a; d2[idx] = b; d3[idx] = __float2bfloat16_rn(x);
+        int64_t r, j;
+        if (small) { const uint32_t i32 = (uint32_t)idx, l32 = (uint32_t)per_row; r = i32 / l32; j = i32 % l32; }
+        else { r = idx / per_row; j = idx % per_row; }
+        const int64_t c0 = j * 8;
+        const float* s = src + r * lds + c0;
+        float x[8];
+        if (vec && c0 + 8 <= cols) {
+            const float4 lo = *reinterpret_cast<const float4*>(s), hi = *reinterpret_cast<const float4*>(s + 4);
+            x[0] = lo.x; x[1] = lo.y; x[2] = lo.z; x[3] = lo.w; x[4] = hi.x; x[5] = hi.y; x[6] = hi.z; x[7] = hi.w;
+        } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) x[i] = c0 + i < cols ? s[i] : 0.f;
+        }
+        __align__(16) __nv_bfloat16 a[8], b[8], c[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) split3_one(x[i], a[i], b[i], c[i]);
+        const int64_t o = r * ldd + c0;
+        *reinterpret_cast<uint4*>(d1 + o) = *reinterpret_cast<const uint4*>(a);
+        *reinterpret_cast<uint4*>(d2 + o) = *reinterpret_cast<const uint4*>(b);
+        *reinterpret_cast<uint4*>(d3 + o) = *reinterpret_cast<const uint4*>(c);
     }
+}
+
+// Launch of k_split3: 16-byte loads when the source rows start on 16-byte boundaries.
+static void launch_split3(cudaStream_t st, const float* src, int64_t lds, int64_t rows, int64_t cols,
+                          __nv_bfloat16* d1, __nv_bfloat16* d2, __nv_bfloat16* d3, int64_t ldd, const int32_t* done)
+{
+    const int vec = (((uintptr_t)src & 15) == 0 && (lds % 4) == 0) ? 1 : 0;
+    const int64_t work = rows * (ldd / 8);
+    unsigned blocks = (unsigned)((work + 255) / 256 < 1184 ? (work + 255) / 256 : 1184);
+    if (blocks < 1) blocks = 1;
+    k_split3<<<blocks, 256, 0, st>>>(src, lds, rows, cols, d1, d2, d3, ldd, vec, done);
 }
 
 // ---------------------------------------------------------------------------------------------------------------
@@ -608,8 +641,8 @@ cudaError_t gemm_tc(cudaStream_t st, int64_t M, int64_t N, int64_t K, float alph
     for (int64_t k0 = 0; k0 < K; k0 += kc) {
         const int64_t kw = K - k0 < kc ? K - k0 : kc;
         const int64_t kw8 = round_up(kw, 8);                    // row stride of the A terms
-        k_split3<<<1184, 256, 0, st>>>(A + k0, lda, M, kw, ap[0], ap[1], ap[2], kw8, done);
-        k_split3<<<1184, 256, 0, st>>>(B + k0 * ldb, ldb, kw, N, bp[0], bp[1], bp[2], ldn, done);
+        launch_split3(st, A + k0, lda, M, kw, ap[0], ap[1], ap[2], kw8, done);
+        launch_split3(st, B + k0 * ldb, ldb, kw, N, bp[0], bp[1], bp[2], ldn, done);
         Maps maps;
         for (int i = 0; i < 3; ++i) {
             // A terms: inner dimension k (kw valid, rows kw8 apart), box 64 x 128; B terms: inner n, box 64 x 64
@@ -672,8 +705,8 @@ cudaError_t rank_update_tc(cudaStream_t st, int64_t M, int64_t N, int64_t K, flo
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(k_rank_update, cudaFuncAttributeMaxDynamicSharedMemorySize, RU_SMEM);
     if (e != cudaSuccess) return e;
-    k_split3<<<1184, 256, 0, st>>>(U, ldu, M, K, up[0], up[1], up[2], k8, done);
-    k_split3<<<1184, 256, 0, st>>>(W, ldw, K, N, wp[0], wp[1], wp[2], ldn, done);
+    launch_split3(st, U, ldu, M, K, up[0], up[1], up[2], k8, done);
+    launch_split3(st, W, ldw, K, N, wp[0], wp[1], wp[2], ldn, done);
     Maps maps;
     for (int i = 0; i < 3; ++i) {
         if (!encode_2d(enc, &maps.a[i], up[i], (uint64_t)K, (uint64_t)M, (uint64_t)k8, BLOCK_K, TILE_M)) return cudaErrorInvalidValue;
@@ -749,7 +782,7 @@ cudaError_t gram_tc2(cudaStream_t st, const void* X, int64_t n_rows, int64_t d1,
     if (!scratch || scratch_bytes < 3 * piece || ((uintptr_t)scratch & 255)) return cudaErrorInvalidValue;
     __nv_bfloat16* yp[3];
     for (int i = 0; i < 3; ++i) yp[i] = (__nv_bfloat16*)((char*)scratch + i * piece);
-    k_split3<<<1184, 256, 0, st>>>((const float*)Y, m, n_rows, m, yp[0], yp[1], yp[2], ldn, nullptr);
+    launch_split3(st, (const float*)Y, m, n_rows, m, yp[0], yp[1], yp[2], ldn, nullptr);
     for (int i = 0; i < 3; ++i)
         if (!encode_2d(enc, &maps.b[i], yp[i], (uint64_t)m, (uint64_t)n_rows, (uint64_t)ldn, 64, BLOCK_K)) return cudaErrorInvalidValue;
     e = cudaFuncSetAttribute(k_mma_pipe<MODE_CROSS3>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
@@ -792,7 +825,7 @@ cudaError_t gram_tc3(cudaStream_t st, const float* X, int64_t n_rows, int64_t d1
     const int vec_ok = (((uintptr_t)C & 15) == 0 && (d1 % 4) == 0) ? 1 : 0;
     for (int64_t r0 = 0; r0 < n_rows; r0 += panel) {
         const int64_t rows = n_rows - r0 < panel ? n_rows - r0 : panel;
-        k_split3<<<1184, 256, 0, st>>>(X + r0 * d1, d1, rows, d1, xp[0], xp[1], xp[2], ldn, nullptr);
+        launch_split3(st, X + r0 * d1, d1, rows, d1, xp[0], xp[1], xp[2], ldn, nullptr);
         Maps maps;
         for (int i = 0; i < 3; ++i) {
             if (!encode_2d(enc, &maps.a[i], xp[i], (uint64_t)d1, (uint64_t)rows, (uint64_t)ldn, 64, BLOCK_K)) return cudaErrorInvalidValue;

@@ -23,6 +23,7 @@ struct BlockPtrs {
     int s, G;
 };
 constexpr int kBlockSmall = 18;
+constexpr int kBlockMaxPairs = OSSCAR_MAX_GROUP;      // s g <= OSSCAR_MAX_GROUP rows per side, hence at most that many groups
 enum { B_CQ = 16, B_HY = 17 };     // joint Schur complement of the entering rows, h^T y
 
 size_t block_bytes_for(const Layout& L, int G) { return osscar::block_region_bytes(L.ldh, L.ldm, L.nJ, G); }
@@ -57,73 +58,165 @@ BlockPtrs make_block_ptrs(osscar_ctx* ctx, int s)
 __device__ __forceinline__ int64_t blk_rrow(const Ptrs& p, const BlockPtrs& bp, int e) { return (int64_t)bp.rslot[e / p.g] * p.g + e % p.g; }
 __device__ __forceinline__ int64_t blk_qrow(const Ptrs& p, const BlockPtrs& bp, int e) { return (int64_t)bp.tslot[e / p.g] * p.g + e % p.g; }
 
+// Monotone map of a double onto an unsigned integer (smaller value, smaller key); -0 counts as +0.
+__device__ __forceinline__ unsigned long long blk_ordered_key(double v)
+{
+    const unsigned long long u = (unsigned long long)__double_as_longlong(v + 0.0);
+    return (u >> 63) ? ~u : (u | 0x8000000000000000ull);
+}
+
+// One digit of a radix selection over the block: among the n items that `in_class` admits, the digit (0..255) whose
+// bin holds the item of rank `want` (1-based, ascending), how many admitted items lie in the bins below it and how many
+// in that bin.  hist is [32 warps][256] in shared memory; every thread of the block calls this with the same n and want.
+template <class Digit>
+__device__ __forceinline__ void blk_radix_digit(int n, int want, Digit&& digit_of, unsigned* hist, unsigned* bcast, int& digit, int& below,
+                                                int& in_bin)
+{
+    const int t = threadIdx.x, lane = t & 31, w = t >> 5, nt = blockDim.x, nw = nt >> 5;
+    for (int i = t; i < nw * 256; i += nt) hist[i] = 0;
+    __syncthreads();
+    constexpr int RB = 8;                                 // items per thread whose loads are in flight together
+    for (int i0 = 0; i0 < n; i0 += nt * RB) {             // whole warps stay together for the lane vote
+        int d[RB];
+#pragma unroll
+        for (int b = 0; b < RB; ++b) {
+            const int i = i0 + b * nt + t;
+            d[b] = i < n ? digit_of(i) : -1;              // -1: not in the class
+        }
+#pragma unroll
+        for (int b = 0; b < RB; ++b) {
+            const unsigned peers = __match_any_sync(0xffffffffu, d[b]);
+            if (d[b] >= 0 && lane == __ffs(peers) - 1) hist[w * 256 + d[b]] += __popc(peers);    // one lane per distinct digit
+            __syncwarp();
+        }
+    }
+    __syncthreads();
+    if (t < 256) { unsigned c = 0; for (int ww = 0; ww < nw; ++ww) c += hist[ww * 256 + t]; hist[t] = c; }
+    __syncthreads();
+    if (w == 0) {                                         // lane owns bins 8 lane .. 8 lane + 7
+        unsigned c[8], sum = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { c[j] = hist[lane * 8 + j]; sum += c[j]; }
+        unsigned incl = sum;
+        for (int o = 1; o < 32; o <<= 1) { const unsigned v = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += v; }
+        unsigned run = incl - sum;                        // items in the bins of the lanes before this one
+        const bool mine = run < (unsigned)want && (unsigned)want <= incl;
+        if (mine) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                if (run < (unsigned)want && (unsigned)want <= run + c[j]) { bcast[0] = lane * 8 + j; bcast[1] = run; bcast[2] = c[j]; }
+                run += c[j];
+            }
+        }
+    }
+    __syncthreads();
+    digit = (int)bcast[0]; below = (int)bcast[1]; in_bin = (int)bcast[2];
+    __syncthreads();
+}
+
 // The s cheapest kept slots (block 0) and the s most valuable pruned slots (block 1), from the scores at the current
-// support; ties go to the smaller group id.  Every thread keeps the best of its own strided share of the scores;
-// a round reduces those over the block, and only the winner's owner rescans its share.  Chosen entries of D and A
-// are overwritten with +-inf while the lists are drawn.
+// support; ties go to the smaller group id; the lists come out in the order in which a repeated arg-min would draw
+// them.  Radix selection: 8-bit digits of the ordered key, most significant first, narrow down the value of the s-th
+// item until the bin of the current digit holds only items that belong; if several items share that value exactly,
+// digits of their group ids fix the last id that still belongs; the members are then gathered and ranked among
+// themselves.
 __global__ void __launch_bounds__(1024) k_blk_select(Ptrs p, BlockPtrs bp)
 {
     SearchCtl* ctl = p.ctl;
     if (ctl->done) return;
-    __shared__ double sv[32]; __shared__ int sid[32]; __shared__ int sidx[32];
+    __shared__ unsigned hist[32 * 256];
+    __shared__ unsigned bcast[3];
+    __shared__ int guard;
+    __shared__ unsigned long long selk[kBlockMaxPairs];
+    __shared__ int selid[kBlockMaxPairs], selix[kBlockMaxPairs];
+    __shared__ int nsel;
     const int side = blockIdx.x;
     const int n = side == 0 ? p.k : (int)(p.ng - p.k);
     double* val = side == 0 ? p.D : p.A;
     const int32_t* ids = side == 0 ? p.perm : p.perm + p.k;
     int32_t* out = side == 0 ? bp.rslot : bp.tslot;
-    const int t = threadIdx.x, lane = t & 31, w = t >> 5, nt = blockDim.x;
+    const int t = threadIdx.x, nt = blockDim.x, s = bp.s;
     if (p.g == 1) {                       // single-row groups: scores from the row norms
-        for (int i = t; i < n; i += nt) {
-            if (side == 0) {
-                const double hd = p.Hinv[(int64_t)i * p.ldh + i];
-                val[i] = hd > 0.0 ? (double)p.vnorm[i] / hd : INFINITY;
-            } else {
-                const double cc = p.c[i];
-                const double hd = p.Hp[(p.nI + i) * p.ldp + p.nI + i];
-                val[i] = cc > kAddPivotTol * hd ? (double)p.rnorm[i] / cc : -INFINITY;
+        constexpr int SB = 8;             // diagonal entries (one DRAM sector each) requested together
+        for (int i0 = 0; i0 < n; i0 += nt * SB) {
+            float hd[SB];
+#pragma unroll
+            for (int b = 0; b < SB; ++b) {
+                const int64_t i = i0 + b * nt + t;
+                hd[b] = i < n ? (side == 0 ? p.Hinv[i * p.ldh + i] : p.Hp[(p.nI + i) * p.ldp + p.nI + i]) : 0.f;
+            }
+#pragma unroll
+            for (int b = 0; b < SB; ++b) {
+                const int i = i0 + b * nt + t;
+                if (i >= n) continue;
+                if (side == 0) val[i] = hd[b] > 0.f ? (double)p.vnorm[i] / (double)hd[b] : INFINITY;
+                else {
+                    const double cc = p.c[i];
+                    val[i] = cc > kAddPivotTol * (double)hd[b] ? (double)p.rnorm[i] / cc : -INFINITY;
+                }
             }
         }
+        __syncthreads();
     }
     const double sign = side == 0 ? 1.0 : -1.0;
-    double best; int bid, bidx;
-    auto rescan = [&]() {                 // a thread only ever reads entries it wrote or that no thread writes
-        best = INFINITY; bid = INT_MAX; bidx = -1;
-        for (int i = t; i < n; i += nt) {
-            const double v = sign * val[i];
-            const int id = ids[i];
-            if (v < best || (v == best && id < bid)) { best = v; bid = id; bidx = i; }
+    auto key_of = [&](int i) { return blk_ordered_key(sign * val[i]); };
+    // Leading digits of the s-th smallest key.  As soon as the bin of the current digit holds no more items than are
+    // still wanted, every item of it belongs and the remaining digits need not be resolved (usually after 3-4 of 8).
+    unsigned long long T = 0;
+    int want = s, kshift = 0;
+    bool open = true;                     // the bin of the last digit still holds items that do not belong
+    for (int pass = 0; pass < 8 && open; ++pass) {
+        const int shift = 56 - 8 * pass;
+        int digit, below, in_bin;
+        blk_radix_digit(n, want, [&](int i) {
+            const unsigned long long k = key_of(i);
+            return (pass == 0 || (k >> (shift + 8)) == (T >> (shift + 8))) ? (int)((k >> shift) & 255) : -1;
+        }, hist, bcast, digit, below, in_bin);
+        T |= (unsigned long long)digit << shift;
+        want -= below;
+        kshift = shift;
+        open = in_bin > want;
+    }
+    // still open after the last digit: several items have exactly the value T and `want` of them belong, those with
+    // the smallest ids
+    unsigned idT = 0;
+    int ishift = 32;                      // 32: no id digit was needed
+    for (int pass = 0; pass < 4 && open; ++pass) {
+        const int shift = 24 - 8 * pass;
+        int digit, below, in_bin;
+        blk_radix_digit(n, want, [&](int i) {
+            if (key_of(i) != T) return -1;
+            const unsigned id = (unsigned)ids[i];
+            return (pass == 0 || (id >> (shift + 8)) == (idT >> (shift + 8))) ? (int)((id >> shift) & 255) : -1;
+        }, hist, bcast, digit, below, in_bin);
+        idT |= (unsigned)digit << shift;
+        want -= below;
+        ishift = shift;
+        open = in_bin > want;
+    }
+    if (t == 0) { nsel = 0; guard = 0; }
+    __syncthreads();
+    const unsigned long long kInf = blk_ordered_key(INFINITY);
+    for (int i = t; i < n; i += nt) {
+        const unsigned long long k = key_of(i);
+        const int id = ids[i];
+        const bool member = ishift == 32 ? (k >> kshift) <= (T >> kshift)
+                                         : (k < T || (k == T && ((unsigned)id >> ishift) <= (idT >> ishift)));
+        if (member) {
+            const int at = atomicAdd(&nsel, 1);
+            if (at < kBlockMaxPairs) { selk[at] = k; selid[at] = id; selix[at] = i; }
+            if (k >= kInf) guard = 1;     // fewer than s candidates with a finite score
         }
-    };
-    rescan();
-    for (int round = 0; round < bp.s; ++round) {
-        double rv = best; int rid = bid, rix = bidx;
-        for (int o = 16; o > 0; o >>= 1) {
-            const double ov = __shfl_xor_sync(0xffffffffu, rv, o);
-            const int oid = __shfl_xor_sync(0xffffffffu, rid, o);
-            const int oix = __shfl_xor_sync(0xffffffffu, rix, o);
-            if (ov < rv || (ov == rv && oid < rid)) { rv = ov; rid = oid; rix = oix; }
-        }
-        if (lane == 0) { sv[w] = rv; sid[w] = rid; sidx[w] = rix; }
-        __syncthreads();
-        if (w == 0) {
-            rv = lane < (nt >> 5) ? sv[lane] : INFINITY; rid = lane < (nt >> 5) ? sid[lane] : INT_MAX; rix = lane < (nt >> 5) ? sidx[lane] : -1;
-            for (int o = 16; o > 0; o >>= 1) {
-                const double ov = __shfl_xor_sync(0xffffffffu, rv, o);
-                const int oid = __shfl_xor_sync(0xffffffffu, rid, o);
-                const int oix = __shfl_xor_sync(0xffffffffu, rix, o);
-                if (ov < rv || (ov == rv && oid < rid)) { rv = ov; rid = oid; rix = oix; }
-            }
-            if (lane == 0) { sv[0] = rv; sidx[0] = rix; }
-        }
-        __syncthreads();
-        const double wv = sv[0]; const int wix = sidx[0];
-        __syncthreads();
-        if (wix < 0 || !isfinite(wv)) {
-            if (t == 0) { ctl->done = 1; ctl->stop_reason = OSSCAR_STOP_GUARD; *p.done_host = 1; }
-            return;
-        }
-        if (t == 0) out[round] = wix;
-        if (wix % nt == t) { val[wix] = sign * INFINITY; rescan(); }
+    }
+    __syncthreads();
+    if (guard) {
+        if (t == 0) { ctl->done = 1; ctl->stop_reason = OSSCAR_STOP_GUARD; *p.done_host = 1; }
+        return;
+    }
+    if (t < s) {                          // exactly s members; rank each among them by (value, id)
+        int rank = 0;
+        for (int j = 0; j < s; ++j) rank += (selk[j] < selk[t] || (selk[j] == selk[t] && selid[j] < selid[t])) ? 1 : 0;
+        out[rank] = selix[t];
     }
 }
 
@@ -493,23 +586,35 @@ __global__ void __launch_bounds__(256) k_blk_update_c_g1(Ptrs p, BlockPtrs bp)
 }
 
 // Exchange the rows (phase 0) or columns (phase 1) of Hp of every leaving / entering pair; phase 1 also exchanges
-// the groups in the slot permutation.
+// the groups in the slot permutation.  Phase 0: grid (pieces of a row, G), a block moves 256 consecutive floats of the
+// two rows of one pair.  Phase 1: a warp owns one row of Hp and its lanes take the pairs, so that the 2 G scattered
+// floats a warp touches lie in one row of the matrix (one DRAM page neighbourhood) instead of in 32 rows.
 __global__ void __launch_bounds__(256) k_blk_hswap(Ptrs p, BlockPtrs bp, int phase)
 {
     if (p.ctl->done) return;
     const int G = bp.G;
-    const int64_t n = p.ldp * G;
-    for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < n; idx += (int64_t)gridDim.x * blockDim.x) {
-        const int e = (int)(idx / p.ldp); const int64_t x = idx % p.ldp;
-        const int64_t a = blk_rrow(p, bp, e), b = p.nI + blk_qrow(p, bp, e);
-        float *pa, *pb;
-        if (phase == 0) { pa = p.Hp + a * p.ldp + x; pb = p.Hp + b * p.ldp + x; }
-        else {
-            if (x >= p.nI + p.nJ) continue;
-            pa = p.Hp + x * p.ldp + a; pb = p.Hp + x * p.ldp + b;
+    if (phase == 0) {
+        const int e = blockIdx.y;
+        const int64_t x = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+        if (x < p.ldp) {
+            float* pa = p.Hp + blk_rrow(p, bp, e) * p.ldp + x;
+            float* pb = p.Hp + (p.nI + blk_qrow(p, bp, e)) * p.ldp + x;
+            const float va = *pa, vb = *pb;
+            *pa = vb; *pb = va;
         }
-        const float va = *pa, vb = *pb;
-        *pa = vb; *pb = va;
+    } else {
+        __shared__ int32_t sa[OSSCAR_MAX_GROUP], sb[OSSCAR_MAX_GROUP];
+        for (int e = threadIdx.x; e < G; e += blockDim.x) { sa[e] = (int32_t)blk_rrow(p, bp, e); sb[e] = (int32_t)(p.nI + blk_qrow(p, bp, e)); }
+        __syncthreads();
+        const int lane = threadIdx.x & 31;
+        const int64_t x = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+        if (x < p.nI + p.nJ) {
+            float* row = p.Hp + x * p.ldp;
+            for (int e = lane; e < G; e += 32) {
+                const float va = row[sa[e]], vb = row[sb[e]];
+                row[sa[e]] = vb; row[sb[e]] = va;
+            }
+        }
     }
     if (phase == 1 && blockIdx.x == 0 && threadIdx.x == 0) {
         for (int t = 0; t < bp.s; ++t) {
@@ -560,8 +665,8 @@ cudaError_t enqueue_block_step(osscar_ctx* ctx, const Ptrs& p, const BlockPtrs& 
     if (L.g == 1) k_blk_update_c_g1<<<296, 256, 2 * (size_t)G * G * sizeof(float), st>>>(p, bp);
     else k_blk_update_c<<<(unsigned)(L.ng - L.k), 128, 2 * (size_t)L.g * G * sizeof(double), st>>>(p, bp);
     k_blk_fix<<<(unsigned)G, 256, 0, st>>>(p, bp);                                              mark();
-    k_blk_hswap<<<(unsigned)((L.ldp * G + 255) / 256), 256, 0, st>>>(p, bp, 0);
-    k_blk_hswap<<<(unsigned)((L.ldp * G + 255) / 256), 256, 0, st>>>(p, bp, 1);                 mark();
+    k_blk_hswap<<<dim3((unsigned)((L.ldp + 255) / 256), (unsigned)G), 256, 0, st>>>(p, bp, 0);
+    k_blk_hswap<<<(unsigned)((L.d1 + 7) / 8), 256, 0, st>>>(p, bp, 1);                           mark();
     count_launches(12);
     BK(enqueue_scores(ctx, p, !fused_norms, false));                                           mark();
 #undef BK
