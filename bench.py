@@ -391,12 +391,13 @@ def run_ours(args):
             if s_pairs * wl.g > 96 or s_pairs > min(wl.k, wl.ngroups - wl.k):
                 continue
             f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            torch.cuda.synchronize()
-            f0.record()
-            rb = pkg.solve_layer(solver, x_dev, W, wl.g, wl.k, max_swaps, damp=wl.damp, accept_mode=accept, accept_rel_tol=wl.eps_acc,
-                                 H=H, G=G, block_pairs=s_pairs)
-            f1.record()
-            torch.cuda.synchronize()
+            for rep in range(2):          # the first solve warms this code path up (attributes, first-touch of the panels)
+                torch.cuda.synchronize()
+                f0.record()
+                rb = pkg.solve_layer(solver, x_dev, W, wl.g, wl.k, max_swaps, damp=wl.damp, accept_mode=accept,
+                                     accept_rel_tol=wl.eps_acc, H=H, G=G, block_pairs=s_pairs)
+                f1.record()
+                torch.cuda.synchronize()
             block_extra.append({"pairs_per_iteration": s_pairs, "swaps": rb.n_swaps, "iterations": rb.n_swaps // s_pairs,
                                 "layer_solve_s": f0.elapsed_time(f1) / 1e3, "search_ms": rb.ms["search"],
                                 "swaps_per_s": rb.n_swaps / max(rb.ms["search"] * 1e-3, 1e-9),
