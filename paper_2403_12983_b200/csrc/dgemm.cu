@@ -38,11 +38,14 @@ __device__ __forceinline__ float4 load4_guard(const float* __restrict__ row, int
 }
 
 // mode 0: C = beta * C0 + alpha * A B (C0 may alias C);  mode 1: C = I + alpha * A B (C0 unused).  OutT float or double.
+// tri (B square and symmetric, K = N): B is replaced by its block upper triangle U with the 64 x 64 diagonal blocks
+// halved, B = U + U^T, so that x^T B x = 2 x^T U x needs only the k-range [0, n0 + 64) of every column tile: half the
+// flops when only such quadratic forms of the rows of A are wanted (the Schur complements of single-row groups).
 template <typename OutT>
 __global__ void __launch_bounds__(DG_T, 2)
 k_gemm_f64acc(int64_t M, int64_t N, int64_t K, double alpha, const float* __restrict__ A, int64_t lda,
               const float* __restrict__ B, int64_t ldb, double beta, const float* C0, int64_t ldc0,
-              OutT* C, int64_t ldc, int mode, int vecA, int vecB, const int32_t* __restrict__ done)
+              OutT* C, int64_t ldc, int mode, int vecA, int vecB, int tri, const int32_t* __restrict__ done)
 {
     if (done && *done) return;
     extern __shared__ double dg_smem[];
@@ -65,14 +68,17 @@ k_gemm_f64acc(int64_t M, int64_t N, int64_t K, double alpha, const float* __rest
 #pragma unroll
         for (int j = 0; j < 4; ++j) { acc[i][j][0] = 0.0; acc[i][j][1] = 0.0; }
 
-    const int nk = (int)((K + DG_BK - 1) / DG_BK);
+    const int64_t kend = tri && n0 + DG_BN < K ? n0 + DG_BN : K;
+    const int nk = (int)((kend + DG_BK - 1) / DG_BK);
     float4 ra0, ra1, rb;
+    double rbs = 1.0;                                          // 0.5 on the rows of the diagonal block (tri)
     auto fetch = [&](int kt) {
         const int64_t k0 = (int64_t)kt * DG_BK;
         ra0 = a0ok ? load4_guard(Ar0, k0 + ac, K, vecA) : make_float4(0.f, 0.f, 0.f, 0.f);
         ra1 = a1ok ? load4_guard(Ar1, k0 + ac, K, vecA) : make_float4(0.f, 0.f, 0.f, 0.f);
         const int64_t kr = k0 + br;
         rb = kr < K ? load4_guard(B + kr * ldb, n0 + bc, N, vecB) : make_float4(0.f, 0.f, 0.f, 0.f);
+        rbs = tri && kr >= n0 ? 0.5 : 1.0;
     };
     auto stash = [&](int buf) {
         double* a = As[buf]; double* b = Bs[buf];
@@ -80,8 +86,8 @@ k_gemm_f64acc(int64_t M, int64_t N, int64_t K, double alpha, const float* __rest
         a[ar * DG_AS + ac + 2] = (double)ra0.z; a[ar * DG_AS + ac + 3] = (double)ra0.w;
         a[(ar + 64) * DG_AS + ac + 0] = (double)ra1.x; a[(ar + 64) * DG_AS + ac + 1] = (double)ra1.y;
         a[(ar + 64) * DG_AS + ac + 2] = (double)ra1.z; a[(ar + 64) * DG_AS + ac + 3] = (double)ra1.w;
-        b[br * DG_BS + bc + 0] = (double)rb.x; b[br * DG_BS + bc + 1] = (double)rb.y;
-        b[br * DG_BS + bc + 2] = (double)rb.z; b[br * DG_BS + bc + 3] = (double)rb.w;
+        b[br * DG_BS + bc + 0] = rbs * (double)rb.x; b[br * DG_BS + bc + 1] = rbs * (double)rb.y;
+        b[br * DG_BS + bc + 2] = rbs * (double)rb.z; b[br * DG_BS + bc + 3] = rbs * (double)rb.w;
     };
     fetch(0);
     stash(0);
@@ -140,23 +146,25 @@ cudaError_t gemm_f64acc(cudaStream_t st, int64_t M, int64_t N, int64_t K, double
     constexpr int smem = (2 * DG_BM * DG_AS + 2 * DG_BK * DG_BS) * (int)sizeof(double);
     cudaError_t e = cudaFuncSetAttribute(k_gemm_f64acc<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
-    k_gemm_f64acc<float><<<grid, DG_T, smem, st>>>(M, N, K, alpha, A, lda, B, ldb, beta, C0, ldc0, C, ldc, identity_plus ? 1 : 0, vecA, vecB, done);
+    k_gemm_f64acc<float><<<grid, DG_T, smem, st>>>(M, N, K, alpha, A, lda, B, ldb, beta, C0, ldc0, C, ldc, identity_plus ? 1 : 0, vecA, vecB, 0, done);
     count_launches(1);
     return cudaGetLastError();
 }
 
-// The plain product with the result kept in fp64: C (M x N doubles, row stride ldc) = A * B.
+// The plain product with the result kept in fp64: C (M x N doubles, row stride ldc) = A * B; with `tri` (B symmetric,
+// K == N) C = A * U for the halved block upper triangle U of B (see the kernel).
 cudaError_t gemm_f64out(cudaStream_t st, int64_t M, int64_t N, int64_t K, const float* A, int64_t lda,
-                        const float* B, int64_t ldb, double* C, int64_t ldc, const int32_t* done)
+                        const float* B, int64_t ldb, double* C, int64_t ldc, const int32_t* done, bool tri)
 {
     if (M <= 0 || N <= 0) return cudaSuccess;
+    if (tri && K != N) return cudaErrorInvalidValue;
     const int vecA = (((uintptr_t)A & 15) == 0 && (lda % 4) == 0) ? 1 : 0;
     const int vecB = (((uintptr_t)B & 15) == 0 && (ldb % 4) == 0) ? 1 : 0;
     dim3 grid((unsigned)((N + DG_BN - 1) / DG_BN), (unsigned)((M + DG_BM - 1) / DG_BM));
     constexpr int smem = (2 * DG_BM * DG_AS + 2 * DG_BK * DG_BS) * (int)sizeof(double);
     cudaError_t e = cudaFuncSetAttribute(k_gemm_f64acc<double>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
-    k_gemm_f64acc<double><<<grid, DG_T, smem, st>>>(M, N, K, 1.0, A, lda, B, ldb, 0.0, nullptr, 0, C, ldc, 0, vecA, vecB, done);
+    k_gemm_f64acc<double><<<grid, DG_T, smem, st>>>(M, N, K, 1.0, A, lda, B, ldb, 0.0, nullptr, 0, C, ldc, 0, vecA, vecB, tri ? 1 : 0, done);
     count_launches(1);
     return cudaGetLastError();
 }

@@ -120,7 +120,7 @@ cudaError_t gemm_f64acc(cudaStream_t st, int64_t M, int64_t N, int64_t K, double
                         const float* B, int64_t ldb, double beta, const float* C0, int64_t ldc0, float* C, int64_t ldc,
                         bool identity_plus, const int32_t* done = nullptr);
 cudaError_t gemm_f64out(cudaStream_t st, int64_t M, int64_t N, int64_t K, const float* A, int64_t lda,
-                        const float* B, int64_t ldb, double* C, int64_t ldc, const int32_t* done = nullptr);
+                        const float* B, int64_t ldb, double* C, int64_t ldc, const int32_t* done = nullptr, bool tri = false);
 
 // ---- panel_tc.cu: Y[i*so_row + e*so_col] = sum_k A[i][k] * P[e][k] on the tensor cores; A (M x K, streamed once) is split
 // into bf16 terms on the way (fp32-accurate); P is an N x K panel

@@ -247,10 +247,11 @@ __global__ void k_gj_writeback(float* __restrict__ A, int64_t lda, int64_t n, in
     }
 }
 
-// c_t[a][b] = Hp[J_ta][J_tb] - sum_s Pm[ta][s] * Hp[J_tb][s]  for pruned slot t; one block per t.
-// Pm holds the rows of the pruned slots [t0, t0 + gridDim.x) in fp64 (row stride ldpm).
+// c_t[a][b] = Hp[J_ta][J_tb] - twice * sum_s Pm[ta][s] * Hp[J_tb][s]  for pruned slot t; one block per t.
+// Pm holds the rows of the pruned slots [t0, t0 + gridDim.x) in fp64 (row stride ldpm): H_JI Hinv (twice = 1), or, for
+// single-row groups, H_JI U with U the halved block upper triangle of Hinv (twice = 2: h^T Hinv h = 2 h^T U h).
 __global__ void k_schur(const float* __restrict__ Hp, int64_t ldp, const double* __restrict__ Pm, int64_t ldpm,
-                        int64_t nI, int g, double* __restrict__ c, int64_t t0, const int32_t* __restrict__ done)
+                        int64_t nI, int g, double* __restrict__ c, int64_t t0, double twice, const int32_t* __restrict__ done)
 {
     if (done && *done) return;
     const int64_t t = t0 + blockIdx.x;
@@ -262,7 +263,7 @@ __global__ void k_schur(const float* __restrict__ Hp, int64_t ldp, const double*
         double s = 0.0;
         for (int64_t x = lane; x < nI; x += 32) s = fma(pr[x], (double)hr[x], s);
         s = warp_sum(s);
-        if (lane == 0) c[(t * g + a) * g + b] = (double)Hp[(nI + t * g + a) * ldp + nI + t * g + b] - s;
+        if (lane == 0) c[(t * g + a) * g + b] = (double)Hp[(nI + t * g + a) * ldp + nI + t * g + b] - twice * s;
     }
 }
 
@@ -563,8 +564,9 @@ int build_state(osscar_ctx* ctx, bool guarded)
         if (gpp < 1) return OSSCAR_E_WORKSPACE;
         for (int64_t t0 = 0; t0 < L.ng - L.k; t0 += gpp) {
             const int64_t ngr = L.ng - L.k - t0 < gpp ? L.ng - L.k - t0 : gpp;
-            CK(gemm_f64out(st, ngr * L.g, nI, nI, Hp + (nI + t0 * L.g) * L.ldp, L.ldp, Hinv, L.ldh, Pm, L.ldh, done));
-            k_schur<<<(unsigned)ngr, 256, 0, st>>>(Hp, L.ldp, Pm, L.ldh, nI, L.g, c, t0, done);
+            const bool tri = L.g == 1;         // one quadratic form per pruned row: half of the symmetric inverse is enough
+            CK(gemm_f64out(st, ngr * L.g, nI, nI, Hp + (nI + t0 * L.g) * L.ldp, L.ldp, Hinv, L.ldh, Pm, L.ldh, done, tri));
+            k_schur<<<(unsigned)ngr, 256, 0, st>>>(Hp, L.ldp, Pm, L.ldh, nI, L.g, c, t0, tri ? 2.0 : 1.0, done);
             count_launches(1);
         }
     }

@@ -413,6 +413,48 @@ def test_block_exchange_matches_oracle(solver, name, over, seed, s, max_swaps, a
     assert np.allclose(c, cref, rtol=2e-3, atol=2e-3 * np.abs(cref).max())
 
 
+def test_block_exchange_breaks_exact_ties_at_the_cut_by_group_id(solver, osscar):
+    """Sixteen kept features that are uncorrelated with everything else and carry no weight have V_i = 0, hence drop
+    scores that are exactly zero on both sides: more ties than the s = 5 places.  The rule (ties to the smaller id) then
+    fixes which five leave in each iteration, and in which order they are listed."""
+    b = osscar.binding
+    rng = np.random.default_rng(5)
+    nA, nZ, m, s = 72, 24, 24, 5
+    d1 = nA + nZ
+    X = rng.standard_normal((400, nA))
+    H64 = np.zeros((d1, d1))
+    H64[:nA, :nA] = X.T @ X
+    H64[nA:, nA:] = np.diag(rng.uniform(50.0, 150.0, nZ))
+    W = np.zeros((d1, m))
+    W[:nA] = rng.standard_normal((nA, m))
+    H64 = H64.astype(np.float32).astype(np.float64)
+    W = W.astype(np.float32).astype(np.float64)
+    G64 = H64 @ W
+    assert not G64[nA:].any()
+    keptZ = np.array([95, 73, 80, 76, 90, 74, 88, 79, 93, 72, 85, 91, 77, 83, 94, 81])
+    keptA = rng.permutation(nA)[:32]
+    S0 = rng.permutation(np.concatenate([keptA, keptZ])).astype(np.int32)      # the slot order must not matter
+    H, G, Wd = dev(H64), dev(G64), dev(W)
+    Hr, Gr = H.cpu().numpy().astype(np.float64), G.cpu().numpy().astype(np.float64)
+    const_r = float(np.sum(W * Gr))
+    support, obj0 = solver.init_support(H, G, Wd, 1, len(S0), mode=b.INIT_USER, support=torch.as_tensor(S0))
+    out = solver.local_search(3 * s, accept_mode=b.ACCEPT_ALWAYS, block_pairs=s)
+    assert out.n_swaps == 3 * s
+    swaps = [tuple(int(v) for v in r) for r in out.swap_trace.cpu().numpy()]
+    order = sorted(int(z) for z in keptZ)
+    for it in range(3):
+        assert [o for o, _ in swaps[it * s:(it + 1) * s]] == order[it * s:(it + 1) * s], f"iteration {it}"
+    # the oracle, which breaks ties the same way, takes the same groups out
+    srch = orc.BlockSearch(Hr, Gr, const_r, 1, np.sort(S0), s, accept="always")
+    for it in range(3):
+        info = srch.propose()
+        assert sorted(int(o) for o in info.out) == order[it * s:(it + 1) * s]
+        slots = [int(np.nonzero(srch.st.S == o)[0][0]) for o, _ in swaps[it * s:(it + 1) * s]]
+        srch.apply(slots, [i for _, i in swaps[it * s:(it + 1) * s]])
+    follow_block(Hr, Gr, const_r, 1, np.sort(S0), s, swaps, out.obj_trace.cpu().numpy(), accept="always", gpu_stop=out.stop_reason,
+                 max_iters=3)
+
+
 @pytest.mark.parametrize("name,over,s,greedy", [
     ("c2", dict(n=4096, d1=520, m=150, k=207, chunk_rows=4096), 8, 0),
     ("c4", dict(n=49 * 40, d1=9 * 100, m=130, k=50, chunk_rows=49 * 40), 3, 0),
