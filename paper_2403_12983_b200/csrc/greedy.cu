@@ -370,7 +370,8 @@ int greedy_support(osscar_ctx* ctx, int t_hat, int32_t* support, int32_t* drop_t
     k_identity_perm<<<nbg, 256, 0, st>>>(p.perm, slotof, ng);
     k_copy_pad2<<<(unsigned)d1, 256, 0, st>>>(ctx->H, d1, d1, p.A, p.lda);
     count_launches(2);
-    int rc = invert_spd_inplace(ctx, p.A, p.lda, d1, ctx->H, d1, nullptr);
+    // fp32 pipes for the rank-64 updates: no correction of the inverse follows here
+    int rc = invert_spd_inplace(ctx, p.A, p.lda, d1, ctx->H, d1, nullptr, false);
     if (rc != OSSCAR_OK) return rc;
     // W* = H^-1 G (Algorithm 1, line 1)
     if (L.ldm != L.m) CK(cudaMemsetAsync(p.V, 0, sizeof(float) * d1 * L.ldm, st));

@@ -160,7 +160,8 @@ cudaError_t gram_mirror(cudaStream_t st, float* H, int64_t d1);   // copy upper 
 // ---- state.cu: support selection and state construction --------------------------------------
 int select_support(osscar_ctx* ctx, int mode, int32_t* support);
 int build_state(osscar_ctx* ctx, bool guarded);
-int invert_spd_inplace(osscar_ctx* ctx, float* A, int64_t lda, int64_t n, const float* ref, int64_t ldref, const int32_t* done);
+int invert_spd_inplace(osscar_ctx* ctx, float* A, int64_t lda, int64_t n, const float* ref, int64_t ldref, const int32_t* done,
+                       bool tensor_updates);
 cudaError_t gather_rows(cudaStream_t st, const float* src, int64_t m, int g, const int32_t* perm,
                         int64_t slot_row0, int64_t nrows, float* dst, int64_t ld);
 cudaError_t trace_product(cudaStream_t st, const float* A, int64_t lda, const float* B, int64_t ldb,

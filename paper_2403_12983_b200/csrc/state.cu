@@ -454,7 +454,11 @@ int select_support(osscar_ctx* ctx, int mode, int32_t* support)
 // In-place inverse of the n x n SPD matrix A (row stride lda) by the blocked exchange (Gauss-Jordan) scheme:
 // per 64-wide pivot block an fp64 Gauss-Jordan inverse in shared memory, then one rank-64 update of the whole matrix in a GEMM.
 // `ref` (row stride ldref) supplies the original diagonal, the scale of the positive-definiteness test.
-int invert_spd_inplace(osscar_ctx* ctx, float* A, int64_t lda, int64_t n, const float* ref, int64_t ldref, const int32_t* done)
+// With `tensor_updates` the rank-64 updates of large matrices run on the tensor cores (three bf16 terms per operand,
+// k_rank_update): their accumulation chains are 64 products long, so the truncating accumulator costs nothing that
+// the correction of the inverse from an fp64 residual, which the caller then applies, does not remove.
+int invert_spd_inplace(osscar_ctx* ctx, float* A, int64_t lda, int64_t n, const float* ref, int64_t ldref, const int32_t* done,
+                       bool tensor_updates)
 {
     const Layout& L = ctx->L;
     cudaStream_t st = ctx->stream;
@@ -462,6 +466,8 @@ int invert_spd_inplace(osscar_ctx* ctx, float* A, int64_t lda, int64_t n, const 
     float* U = T + L.d1 * NB;
     float* Un = U + NB * L.ldp;
     float* Dinv = Un + NB * L.ldp;
+    const bool tc_updates = tensor_updates && n >= 4096 && (lda % 4) == 0 && (((uintptr_t)A & 15) == 0);
+    if (tc_updates) CK(cudaMemsetAsync(U, 0, sizeof(float) * NB * lda, st));       // the pad columns of the row panel stay zero
     for (int64_t p0 = 0; p0 < n; p0 += NB) {
         const int nb = (int)(n - p0 < NB ? n - p0 : NB);
         k_pivot_inverse<<<1, 1024, 0, st>>>(A, lda, p0, nb, Dinv, ref, ldref, ctx->ctl);
@@ -473,9 +479,11 @@ int invert_spd_inplace(osscar_ctx* ctx, float* A, int64_t lda, int64_t n, const 
             k_copy_rows<<<grid, 256, 0, st>>>(A, lda, p0, nb, n, U, lda);
         }
         CK(sgemm(st, false, false, nb, n, nb, -1.f, Dinv, NB, U, lda, 0.f, Un, lda, done));
-        // the rank-64 updates stay on the fp32 pipes: the inversion amplifies rounding by cond(A), and the tensor
-        // core's truncating accumulation is biased where fp32 FMA chains are not
-        CK(sgemm(st, false, false, n, n, nb, -1.f, T, NB, U, lda, 1.f, A, lda, done));
+        // the rank-64 update of the whole matrix
+        if (tc_updates)
+            CK(rank_update_tc(st, n, lda, nb, -1.f, T, NB, U, lda, A, lda, (char*)ctx->ws + L.off_tc, L.tc_bytes, ctx->ctl, done));
+        else
+            CK(sgemm(st, false, false, n, n, nb, -1.f, T, NB, U, lda, 1.f, A, lda, done));
         k_gj_writeback<<<(unsigned)((n * nb + 255) / 256), 256, 0, st>>>(A, lda, n, p0, nb, T, NB, Un, lda, Dinv);
         count_launches(4);     // pivot inverse, zero rows, copy rows, write-back (the GEMMs count themselves)
     }
@@ -509,7 +517,7 @@ int build_state(osscar_ctx* ctx, bool guarded)
     k_copy_pad<<<(unsigned)nI, 256, 0, st>>>(Hp, L.ldp, nI, nI, Hinv, L.ldh);
     count_launches(2);
     CK(cudaGetLastError());
-    { const int rc_inv = invert_spd_inplace(ctx, Hinv, L.ldh, nI, Hp, L.ldp, done); if (rc_inv != OSSCAR_OK) return rc_inv; }
+    { const int rc_inv = invert_spd_inplace(ctx, Hinv, L.ldh, nI, Hp, L.ldp, done, true); if (rc_inv != OSSCAR_OK) return rc_inv; }
     // Every product below that forms a small difference of large sums is accumulated in fp64 (gemm_f64acc): the scores
     // of Eq. impact are compared at 1e-5 relative, and fp32 accumulation leaves cond(H_II) * 2^-24 in them.
     // (1) the inverse.  Single-row groups: fp64 copy by a third-order correction from one fp64 residual, and the fp32
