@@ -71,14 +71,13 @@ k_gemm_f64acc(int64_t M, int64_t N, int64_t K, double alpha, const float* __rest
     const int64_t kend = tri && n0 + DG_BN < K ? n0 + DG_BN : K;
     const int nk = (int)((kend + DG_BK - 1) / DG_BK);
     float4 ra0, ra1, rb;
-    double rbs = 1.0;                                          // 0.5 on the rows of the diagonal block (tri)
     auto fetch = [&](int kt) {
         const int64_t k0 = (int64_t)kt * DG_BK;
         ra0 = a0ok ? load4_guard(Ar0, k0 + ac, K, vecA) : make_float4(0.f, 0.f, 0.f, 0.f);
         ra1 = a1ok ? load4_guard(Ar1, k0 + ac, K, vecA) : make_float4(0.f, 0.f, 0.f, 0.f);
         const int64_t kr = k0 + br;
         rb = kr < K ? load4_guard(B + kr * ldb, n0 + bc, N, vecB) : make_float4(0.f, 0.f, 0.f, 0.f);
-        rbs = tri && kr >= n0 ? 0.5 : 1.0;
+        if (tri && kr >= n0) { rb.x *= 0.5f; rb.y *= 0.5f; rb.z *= 0.5f; rb.w *= 0.5f; }      // rows of the diagonal block, exact in fp32
     };
     auto stash = [&](int buf) {
         double* a = As[buf]; double* b = Bs[buf];
@@ -86,8 +85,8 @@ k_gemm_f64acc(int64_t M, int64_t N, int64_t K, double alpha, const float* __rest
         a[ar * DG_AS + ac + 2] = (double)ra0.z; a[ar * DG_AS + ac + 3] = (double)ra0.w;
         a[(ar + 64) * DG_AS + ac + 0] = (double)ra1.x; a[(ar + 64) * DG_AS + ac + 1] = (double)ra1.y;
         a[(ar + 64) * DG_AS + ac + 2] = (double)ra1.z; a[(ar + 64) * DG_AS + ac + 3] = (double)ra1.w;
-        b[br * DG_BS + bc + 0] = rbs * (double)rb.x; b[br * DG_BS + bc + 1] = rbs * (double)rb.y;
-        b[br * DG_BS + bc + 2] = rbs * (double)rb.z; b[br * DG_BS + bc + 3] = rbs * (double)rb.w;
+        b[br * DG_BS + bc + 0] = (double)rb.x; b[br * DG_BS + bc + 1] = (double)rb.y;
+        b[br * DG_BS + bc + 2] = (double)rb.z; b[br * DG_BS + bc + 3] = (double)rb.w;
     };
     fetch(0);
     stash(0);
